@@ -1,0 +1,161 @@
+/*
+ * amx.h - C ABI of the AMXFP4 quantize + GEMM library for NVIDIA B200 (sm_100a).
+ *
+ * AMXFP4 (arXiv 2411.09909, Sections 4.2-4.3, Eq. 1): FP4 E2M1 elements in groups
+ * of 32 along the reduction axis; each group carries two shared FP8 E5M2 scales,
+ * one applied to the elements whose sign bit is 0 and one to those whose sign
+ * bit is 1.  Decoded value = (-1)^s * E2M1 * scale_s.
+ *
+ * Conventions for every entry point
+ *   - Pointers are DEVICE pointers owned by the caller unless the name of the
+ *     argument ends in _host.  The library allocates no device memory and keeps
+ *     no state between calls; scratch comes from the caller as `workspace`.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Work is enqueued on it; calls return without synchronising
+ *     unless stated otherwise.
+ *   - Return value: AMX_OK (0) or a negative amx_status; on error nothing was
+ *     launched.  amx_status_string() names the code.
+ *   - Quantized tensor layout ("canonical"), for a logical [rows, K] operand:
+ *       codes   uint8 [rows, K/2]      byte j of a row holds element 2j in its low
+ *                                      nibble and element 2j+1 in its high nibble;
+ *                                      a nibble is sign<<3 | E2M1 magnitude code
+ *       scales  uint8 [rows, K/gs, 2]  E5M2 bytes: [..][0] positive-side scale,
+ *                                      [..][1] negative-side scale
+ *     That is 4.5 bits per element at gs = 32.
+ *   - group_size (gs) must be 16, 32, 64 or 128 and divide K.
+ *   - NaN / Inf inputs are outside the format's definition; results for them are
+ *     unspecified (no fault).
+ */
+#ifndef AMX_H_
+#define AMX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum amx_status {
+    AMX_OK = 0,
+    AMX_ERR_NULL = -1,       /* a required pointer is NULL */
+    AMX_ERR_SHAPE = -2,      /* bad sizes: non-positive, K % gs != 0, unsupported gs, ld too small */
+    AMX_ERR_ALIGN = -3,      /* pointer or leading dimension not aligned as documented */
+    AMX_ERR_WORKSPACE = -4,  /* workspace missing or smaller than amx_workspace_bytes() */
+    AMX_ERR_FLAGS = -5,      /* unknown or contradictory flags */
+    AMX_ERR_CUDA = -6,       /* a CUDA runtime call failed (launch or copy) */
+    AMX_ERR_DEVICE = -7,     /* the device is not compute capability 10.x */
+    AMX_ERR_TIMEOUT = -8     /* a bounded device-side wait expired (reported by amx_gemm_status) */
+} amx_status;
+
+/* flags for amx_dequantize: output element type (default bf16) */
+#define AMX_OUT_BF16 0x0u
+#define AMX_OUT_F32 0x1u
+/* flags for amx_gemm / amx_quant_gemm: kernel choice (default: tensor-core path when the
+ * shape allows it, else the SIMT path) */
+#define AMX_GEMM_AUTO 0x0u
+#define AMX_GEMM_SIMT 0x10u  /* plain CUDA-core kernel: any shape, any supported gs */
+#define AMX_GEMM_TC 0x20u    /* tcgen05 kernel only: AMX_ERR_SHAPE if the shape does not fit */
+
+/*
+ * amx_quantize - direct cast of a bf16 matrix to AMXFP4 (Sections 4.2-4.3; procedure per
+ * Algorithm 1 applied to each sign with the FP8 scale of Section 4.2, as in the worked example
+ * of Appendix B.3).
+ * Per group of gs consecutive elements of a row:
+ *   pmax = largest element with sign bit 0, nmax = largest magnitude with sign bit 1;
+ *   scale_side = E5M2 nearest (ties to even, saturating at 57344) to max_side / 6;
+ *   magnitude  = E2M1 nearest (ties to even) to |x| / scale_side, clamped at 6 (0 if the scale is 0);
+ *   the sign bit of a code is the sign bit of x.
+ *   x       bf16 [rows, ld_x] row-major, ld_x >= K in elements; 16-byte aligned, ld_x % 8 == 0
+ *   codes   out, [rows, K/2], 4-byte aligned
+ *   scales  out, [rows, K/gs, 2], 2-byte aligned
+ * K % 8 == 0 is required.  rows == 0 is a no-op.
+ */
+int amx_quantize(const void* x, int64_t rows, int64_t K, int64_t ld_x, int group_size,
+                 uint8_t* codes, uint8_t* scales, void* stream);
+
+/*
+ * amx_quantize_t - the same cast with the groups running DOWN the rows of x (the strided axis):
+ * x is bf16 [R, C] row-major (ld_x >= C), groups are gs consecutive rows of one column, and the
+ * result is laid out as the canonical quantization of x transposed:
+ *   codes [C, R/2], scales [C, R/gs, 2].
+ * This is how V enters the P*V product with groups along the sequence (Appendix C: Value and the
+ * self-attention map are quantized too).  R % gs == 0, R % 2 == 0; x 2-byte aligned.
+ */
+int amx_quantize_t(const void* x, int64_t R, int64_t C, int64_t ld_x, int group_size,
+                   uint8_t* codes, uint8_t* scales, void* stream);
+
+/*
+ * amx_dequantize - Eq. 1 evaluated: out[r,k] = (-1)^s * E2M1 * (s ? scale_neg : scale_pos).
+ * Every result has at most 5 significant bits and is exact in bf16 and in fp32.
+ *   out  bf16 or fp32 (flags) [rows, ld_out], ld_out >= K; 16-byte aligned, ld_out % 8 == 0
+ */
+int amx_dequantize(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K,
+                   int group_size, uint32_t flags, void* out, int64_t ld_out, void* stream);
+
+/*
+ * amx_gemm - C[m,n] = sum_k Ahat[m,k] * What[n,k] with Ahat, What the decoded operands
+ * (Section 4.3: each factor uses the shared scale its own sign selects), fp32 accumulation.
+ *   a_codes/a_scales  canonical [M, K];  w_codes/w_scales canonical [N, K] (both K-major)
+ *   C   out fp32 [M, ld_c], ld_c >= N; 16-byte aligned, ld_c % 4 == 0
+ *   workspace  device scratch of at least amx_workspace_bytes(M, N, K, gs, flags) bytes,
+ *              256-byte aligned (may be NULL when that size is 0)
+ * M == 0 or N == 0 is a no-op.
+ */
+int amx_gemm(const uint8_t* a_codes, const uint8_t* a_scales,
+             const uint8_t* w_codes, const uint8_t* w_scales,
+             int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags,
+             float* C, int64_t ld_c, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * amx_quant_gemm - the fully quantized linear layer of Section 5 ("quantize input operands for
+ * all decoder-layer matrix multiplications"): quantizes the bf16 activation A[M, ld_a] and
+ * multiplies it with an already quantized weight.  Same result as amx_quantize followed by
+ * amx_gemm.  The workspace additionally holds the quantized activation.
+ */
+int amx_quant_gemm(const void* A, int64_t ld_a,
+                   const uint8_t* w_codes, const uint8_t* w_scales,
+                   int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags,
+                   float* C, int64_t ld_c, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * amx_softmax_bf16 - the step between the two attention products: P = softmax(alpha * S) per
+ * row in fp32, rounded to bf16 (the quantizer's input type) so that the normalised
+ * self-attention map can be quantized along the key axis (Appendix C).
+ *   S  fp32 [rows, ld_s];  P  out bf16 [rows, ld_p];  cols <= ld_s, ld_p
+ */
+int amx_softmax_bf16(const float* S, int64_t rows, int64_t cols, int64_t ld_s, float alpha,
+                     void* P, int64_t ld_p, void* stream);
+
+/*
+ * amx_linear_host - one whole layer from HOST memory: copies the bf16 activation A_host[M,K] and
+ * weight W_host[N,K] to the device, quantizes both, multiplies, and copies C back to
+ * C_host[M,N] (fp32).  All copies and kernels are enqueued on `stream`; the call returns after
+ * synchronising it.  Host buffers should be page-locked for the copies to be asynchronous.
+ *   workspace  device scratch, at least amx_linear_host_workspace_bytes(M, N, K, gs) bytes
+ */
+int amx_linear_host(const void* A_host, const void* W_host, int64_t M, int64_t N, int64_t K,
+                    int group_size, uint32_t flags, float* C_host,
+                    void* workspace, size_t workspace_bytes, void* stream);
+
+/* Scratch sizes (bytes; 0 is possible).  Return 0 for invalid shapes. */
+size_t amx_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags);
+size_t amx_quant_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags);
+size_t amx_linear_host_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size);
+
+/* Which kernel amx_gemm would run for this shape and flags: AMX_GEMM_SIMT or AMX_GEMM_TC. */
+uint32_t amx_gemm_kernel_for(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags);
+
+/*
+ * Status word of the most recent tensor-core GEMM that used `workspace`: AMX_OK, or
+ * AMX_ERR_TIMEOUT when a bounded wait inside the kernel expired (the kernel then stopped
+ * issuing work, released its resources and returned; C is not valid).  Synchronises `stream`.
+ */
+int amx_gemm_status(const void* workspace, void* stream);
+
+const char* amx_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AMX_H_ */

@@ -1,0 +1,194 @@
+"""Thin Python binding of the C-ABI CUDA library (``include/amx.h``).
+
+Argument marshalling only: every function checks tensor types, allocates outputs with
+torch (device memory and streams are all torch is used for) and forwards pointers to the
+entry point of the same name.  There is no fallback of any kind: if ``libamx_b200.so``
+has not been built (``python -m paper_2411_09909_b200.build``) the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libamx_b200.so")
+_lib = None
+
+OUT_BF16, OUT_F32 = 0x0, 0x1
+GEMM_AUTO, GEMM_SIMT, GEMM_TC = 0x0, 0x10, 0x20
+
+# every symbol include/amx.h declares
+SYMBOLS = (
+    "amx_quantize", "amx_quantize_t", "amx_dequantize", "amx_gemm", "amx_quant_gemm",
+    "amx_softmax_bf16", "amx_linear_host", "amx_workspace_bytes",
+    "amx_quant_gemm_workspace_bytes", "amx_linear_host_workspace_bytes",
+    "amx_gemm_kernel_for", "amx_gemm_status", "amx_status_string",
+)
+
+
+class AmxError(RuntimeError):
+    pass
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise AmxError(f"{_LIB_PATH} is missing: build it with `python -m paper_2411_09909_b200.build`")
+        L = ctypes.CDLL(_LIB_PATH)
+        i64, p, i, u32, sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_uint32, ctypes.c_size_t
+        L.amx_quantize.argtypes = [p, i64, i64, i64, i, p, p, p]
+        L.amx_quantize_t.argtypes = [p, i64, i64, i64, i, p, p, p]
+        L.amx_dequantize.argtypes = [p, p, i64, i64, i, u32, p, i64, p]
+        L.amx_gemm.argtypes = [p, p, p, p, i64, i64, i64, i, u32, p, i64, p, sz, p]
+        L.amx_quant_gemm.argtypes = [p, i64, p, p, i64, i64, i64, i, u32, p, i64, p, sz, p]
+        L.amx_softmax_bf16.argtypes = [p, i64, i64, i64, ctypes.c_float, p, i64, p]
+        L.amx_linear_host.argtypes = [p, p, i64, i64, i64, i, u32, p, p, sz, p]
+        for name in ("amx_workspace_bytes", "amx_quant_gemm_workspace_bytes"):
+            getattr(L, name).argtypes = [i64, i64, i64, i, u32]
+            getattr(L, name).restype = sz
+        L.amx_linear_host_workspace_bytes.argtypes = [i64, i64, i64, i]
+        L.amx_linear_host_workspace_bytes.restype = sz
+        L.amx_gemm_kernel_for.argtypes = [i64, i64, i64, i, u32]
+        L.amx_gemm_kernel_for.restype = u32
+        L.amx_gemm_status.argtypes = [p, p]
+        L.amx_status_string.argtypes = [i]
+        L.amx_status_string.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def status_string(rc: int) -> str:
+    return lib().amx_status_string(int(rc)).decode()
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise AmxError(f"{what}: {status_string(rc)} ({rc})")
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dev(t: torch.Tensor, dtype, name: str):
+    if not t.is_cuda or t.dtype != dtype:
+        raise AmxError(f"{name} must be a CUDA tensor of {dtype}")
+    return t
+
+
+def _ws(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def quantize(x: torch.Tensor, group_size: int = 32):
+    """bf16 [rows, K] (row stride allowed) -> (codes u8 [rows, K/2], scales u8 [rows, K/gs, 2])."""
+    _dev(x, torch.bfloat16, "x")
+    assert x.dim() == 2 and x.stride(1) == 1
+    rows, K = x.shape
+    codes = torch.empty((rows, K // 2), dtype=torch.uint8, device=x.device)
+    scales = torch.empty((rows, max(K // group_size, 0), 2), dtype=torch.uint8, device=x.device)
+    _check(lib().amx_quantize(x.data_ptr(), rows, K, x.stride(0) if rows > 1 else max(K, x.stride(0)),
+                              group_size, codes.data_ptr(), scales.data_ptr(), _stream()), "amx_quantize")
+    return codes, scales
+
+
+def quantize_t(x: torch.Tensor, group_size: int = 32):
+    """bf16 [R, C], groups down the rows -> canonical quantization of x^T: codes [C, R/2], scales [C, R/gs, 2]."""
+    _dev(x, torch.bfloat16, "x")
+    assert x.dim() == 2 and x.stride(1) == 1
+    R, C = x.shape
+    codes = torch.empty((C, R // 2), dtype=torch.uint8, device=x.device)
+    scales = torch.empty((C, R // group_size, 2), dtype=torch.uint8, device=x.device)
+    _check(lib().amx_quantize_t(x.data_ptr(), R, C, x.stride(0), group_size, codes.data_ptr(),
+                                scales.data_ptr(), _stream()), "amx_quantize_t")
+    return codes, scales
+
+
+def dequantize(codes: torch.Tensor, scales: torch.Tensor, group_size: int = 32, dtype=torch.bfloat16):
+    _dev(codes, torch.uint8, "codes"), _dev(scales, torch.uint8, "scales")
+    rows, K = codes.shape[0], codes.shape[1] * 2
+    out = torch.empty((rows, K), dtype=dtype, device=codes.device)
+    flag = {torch.bfloat16: OUT_BF16, torch.float32: OUT_F32}[dtype]
+    _check(lib().amx_dequantize(codes.data_ptr(), scales.data_ptr(), rows, K, group_size, flag,
+                                out.data_ptr(), K, _stream()), "amx_dequantize")
+    return out
+
+
+def gemm(a_codes, a_scales, w_codes, w_scales, group_size: int = 32, flags: int = GEMM_AUTO,
+         out: torch.Tensor | None = None, workspace: torch.Tensor | None = None):
+    """fp32 [M, N] = decoded A [M, K] times decoded W [N, K] transposed."""
+    for t, n in ((a_codes, "a_codes"), (a_scales, "a_scales"), (w_codes, "w_codes"), (w_scales, "w_scales")):
+        _dev(t, torch.uint8, n)
+        assert t.is_contiguous()
+    M, K = a_codes.shape[0], a_codes.shape[1] * 2
+    N = w_codes.shape[0]
+    assert w_codes.shape[1] * 2 == K
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float32, device=a_codes.device)
+    need = lib().amx_workspace_bytes(M, N, K, group_size, flags)
+    if workspace is None:
+        workspace = _ws(need, a_codes.device)
+    _check(lib().amx_gemm(a_codes.data_ptr(), a_scales.data_ptr(), w_codes.data_ptr(), w_scales.data_ptr(),
+                          M, N, K, group_size, flags, out.data_ptr(), out.stride(0), workspace.data_ptr(),
+                          workspace.numel(), _stream()), "amx_gemm")
+    return out
+
+
+def gemm_status(workspace: torch.Tensor) -> int:
+    return int(lib().amx_gemm_status(workspace.data_ptr(), _stream()))
+
+
+def quant_gemm(a: torch.Tensor, w_codes, w_scales, group_size: int = 32, flags: int = GEMM_AUTO,
+               out: torch.Tensor | None = None, workspace: torch.Tensor | None = None):
+    """fp32 [M, N] = AMXFP4(a) x quantized W; a is bf16 [M, K]."""
+    _dev(a, torch.bfloat16, "a")
+    M, K = a.shape
+    N = w_codes.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float32, device=a.device)
+    need = lib().amx_quant_gemm_workspace_bytes(M, N, K, group_size, flags)
+    if workspace is None:
+        workspace = _ws(need, a.device)
+    _check(lib().amx_quant_gemm(a.data_ptr(), a.stride(0), w_codes.data_ptr(), w_scales.data_ptr(), M, N, K,
+                                group_size, flags, out.data_ptr(), out.stride(0), workspace.data_ptr(),
+                                workspace.numel(), _stream()), "amx_quant_gemm")
+    return out
+
+
+def softmax_bf16(S: torch.Tensor, alpha: float, out: torch.Tensor | None = None):
+    _dev(S, torch.float32, "S")
+    rows, cols = S.shape
+    if out is None:
+        out = torch.empty((rows, cols), dtype=torch.bfloat16, device=S.device)
+    _check(lib().amx_softmax_bf16(S.data_ptr(), rows, cols, S.stride(0), float(alpha), out.data_ptr(),
+                                  out.stride(0), _stream()), "amx_softmax_bf16")
+    return out
+
+
+def linear_host(a_host: torch.Tensor, w_host: torch.Tensor, c_host: torch.Tensor, workspace: torch.Tensor,
+                group_size: int = 32, flags: int = GEMM_AUTO):
+    """Whole layer from (pinned) host bf16 tensors a[M,K], w[N,K] into host fp32 c[M,N]; synchronises."""
+    assert not a_host.is_cuda and not w_host.is_cuda and not c_host.is_cuda and workspace.is_cuda
+    assert a_host.dtype == w_host.dtype == torch.bfloat16 and c_host.dtype == torch.float32
+    M, K = a_host.shape
+    N = w_host.shape[0]
+    _check(lib().amx_linear_host(a_host.data_ptr(), w_host.data_ptr(), M, N, K, group_size, flags,
+                                 c_host.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream()),
+           "amx_linear_host")
+    return c_host
+
+
+def attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, group_size: int = 32, flags: int = GEMM_AUTO):
+    """Fully quantized attention for one head (Appendix C: Q, K, the self-attention map and V are all
+    quantized): S = AMX(q) AMX(k)^T (groups along head_dim), P = softmax(S / sqrt(d)) rounded to bf16,
+    O = AMX(P) AMX(v) with groups along the key axis.  q, k, v: bf16 [L, d].  Returns (O fp32 [L, d], P bf16)."""
+    L, d = q.shape
+    qc, qs = quantize(q, group_size)
+    kc, ks = quantize(k, group_size)
+    S = gemm(qc, qs, kc, ks, group_size, flags)
+    P = softmax_bf16(S, d ** -0.5)
+    pc, ps = quantize(P, group_size)
+    vc, vs = quantize_t(v, group_size)
+    return gemm(pc, ps, vc, vs, group_size, flags), P

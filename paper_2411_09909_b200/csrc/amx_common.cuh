@@ -1,0 +1,37 @@
+// Shared host/device helpers of the AMXFP4 CUDA library (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "amx.h"
+
+namespace amx {
+
+inline bool valid_group_size(int gs) { return gs == 16 || gs == 32 || gs == 64 || gs == 128; }
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// Returns AMX_OK when the last launch was accepted, AMX_ERR_CUDA otherwise.
+inline int launch_status() { return cudaGetLastError() == cudaSuccess ? AMX_OK : AMX_ERR_CUDA; }
+
+// ---- device-side number formats -------------------------------------------------------------
+
+// fp32 value of an E5M2 byte: E5M2 is the upper byte of an IEEE half.
+__device__ __forceinline__ float e5m2_to_float(uint32_t byte) {
+    float f;
+    unsigned short h = (unsigned short)(byte << 8);
+    asm("cvt.f32.f16 %0, %1;" : "=f"(f) : "h"(h));
+    return f;
+}
+
+// fp32 magnitude of a 3-bit E2M1 code EEM: 0, .5, 1, 1.5, 2, 3, 4, 6.
+// For EE > 0 the bits placed at fp32 exponent/mantissa positions give 2^(EE-1) * (1 + M/2);
+// EE == 0 is the subnormal M * 0.5.
+__device__ __forceinline__ float e2m1_mag_to_float(uint32_t c3) {
+    uint32_t bits = (c3 << 22) + (126u << 23);   // exponent field EE + 126, mantissa msb = M
+    float v = __uint_as_float(bits);
+    return (c3 & 6u) ? v : 0.5f * (float)(c3 & 1u);
+}
+
+}  // namespace amx

@@ -1,0 +1,154 @@
+// C-ABI entry points that combine kernels: GEMM dispatch, quantize+GEMM, the host-buffer
+// layer call, workspace sizing and status strings.
+#include "gemm.cuh"
+
+namespace amx {
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t round_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+bool gemm_shape_ok(int64_t M, int64_t N, int64_t K, int gs) {
+    return valid_group_size(gs) && M >= 0 && N >= 0 && K > 0 && K % gs == 0 && K % 8 == 0;
+}
+
+// AMX_GEMM_SIMT / AMX_GEMM_TC, or 0 when the flags cannot be honoured for this shape.
+uint32_t pick_kernel(int64_t M, int64_t N, int64_t K, int gs, uint32_t flags) {
+    const uint32_t want = flags & (AMX_GEMM_SIMT | AMX_GEMM_TC);
+    if (want == (AMX_GEMM_SIMT | AMX_GEMM_TC)) return 0;
+    const bool tc = gemm_tc_supported(M, N, K, gs);
+    if (want == AMX_GEMM_TC) return tc ? AMX_GEMM_TC : 0;
+    if (want == AMX_GEMM_SIMT) return AMX_GEMM_SIMT;
+    return tc ? AMX_GEMM_TC : AMX_GEMM_SIMT;
+}
+
+struct QuantSizes {
+    size_t codes, scales;
+};
+QuantSizes quant_sizes(int64_t rows, int64_t K, int gs) {
+    return {round_up((size_t)rows * (size_t)(K / 2)), round_up((size_t)rows * (size_t)(K / gs) * 2)};
+}
+
+}  // namespace
+}  // namespace amx
+
+using namespace amx;
+
+extern "C" uint32_t amx_gemm_kernel_for(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags) {
+    if (!gemm_shape_ok(M, N, K, group_size)) return 0;
+    return pick_kernel(M, N, K, group_size, flags);
+}
+
+extern "C" size_t amx_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags) {
+    if (!gemm_shape_ok(M, N, K, group_size)) return 0;
+    return pick_kernel(M, N, K, group_size, flags) == AMX_GEMM_TC ? round_up(gemm_tc_workspace_bytes(M, N, K)) : 0;
+}
+
+extern "C" size_t amx_quant_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags) {
+    if (!gemm_shape_ok(M, N, K, group_size)) return 0;
+    const QuantSizes a = quant_sizes(M, K, group_size);
+    return amx_workspace_bytes(M, N, K, group_size, flags) + a.codes + a.scales;
+}
+
+extern "C" size_t amx_linear_host_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size) {
+    if (!gemm_shape_ok(M, N, K, group_size)) return 0;
+    const QuantSizes a = quant_sizes(M, K, group_size), w = quant_sizes(N, K, group_size);
+    return amx_workspace_bytes(M, N, K, group_size, AMX_GEMM_AUTO) + a.codes + a.scales + w.codes + w.scales +
+           round_up((size_t)M * K * 2) + round_up((size_t)N * K * 2) + round_up((size_t)M * N * 4);
+}
+
+extern "C" int amx_gemm(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes,
+                        const uint8_t* w_scales, int64_t M, int64_t N, int64_t K, int group_size,
+                        uint32_t flags, float* C, int64_t ld_c, void* workspace, size_t workspace_bytes,
+                        void* stream) {
+    if (flags & ~(AMX_GEMM_SIMT | AMX_GEMM_TC)) return AMX_ERR_FLAGS;
+    if (!gemm_shape_ok(M, N, K, group_size) || ld_c < N) return AMX_ERR_SHAPE;
+    const uint32_t kernel = pick_kernel(M, N, K, group_size, flags);
+    if (!kernel) return (flags & AMX_GEMM_SIMT) ? AMX_ERR_FLAGS : AMX_ERR_SHAPE;
+    if (M == 0 || N == 0) return AMX_OK;
+    if (!a_codes || !a_scales || !w_codes || !w_scales || !C) return AMX_ERR_NULL;
+    if (!aligned(a_codes, 16) || !aligned(w_codes, 16) || !aligned(a_scales, 2) || !aligned(w_scales, 2) ||
+        !aligned(C, 16) || ld_c % 4)
+        return AMX_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (kernel == AMX_GEMM_SIMT)
+        return gemm_simt(a_codes, a_scales, w_codes, w_scales, M, N, K, group_size, C, ld_c, st);
+    const size_t need = round_up(gemm_tc_workspace_bytes(M, N, K));
+    if (need && (!workspace || workspace_bytes < need)) return AMX_ERR_WORKSPACE;
+    if (need && !aligned(workspace, kAlign)) return AMX_ERR_ALIGN;
+    return gemm_tc(a_codes, a_scales, w_codes, w_scales, M, N, K, C, ld_c, workspace, st);
+}
+
+extern "C" int amx_quant_gemm(const void* A, int64_t ld_a, const uint8_t* w_codes, const uint8_t* w_scales,
+                              int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags, float* C,
+                              int64_t ld_c, void* workspace, size_t workspace_bytes, void* stream) {
+    if (flags & ~(AMX_GEMM_SIMT | AMX_GEMM_TC)) return AMX_ERR_FLAGS;
+    if (!gemm_shape_ok(M, N, K, group_size) || ld_a < K || ld_c < N) return AMX_ERR_SHAPE;
+    if (M == 0 || N == 0) return AMX_OK;
+    const size_t need = amx_quant_gemm_workspace_bytes(M, N, K, group_size, flags);
+    if (!workspace || workspace_bytes < need) return AMX_ERR_WORKSPACE;
+    if (!aligned(workspace, kAlign)) return AMX_ERR_ALIGN;
+    const size_t gemm_ws = amx_workspace_bytes(M, N, K, group_size, flags);
+    const QuantSizes a = quant_sizes(M, K, group_size);
+    uint8_t* base = static_cast<uint8_t*>(workspace);
+    uint8_t* a_codes = base + gemm_ws;
+    uint8_t* a_scales = a_codes + a.codes;
+    int rc = amx_quantize(A, M, K, ld_a, group_size, a_codes, a_scales, stream);
+    if (rc != AMX_OK) return rc;
+    return amx_gemm(a_codes, a_scales, w_codes, w_scales, M, N, K, group_size, flags, C, ld_c, base, gemm_ws, stream);
+}
+
+extern "C" int amx_linear_host(const void* A_host, const void* W_host, int64_t M, int64_t N, int64_t K,
+                               int group_size, uint32_t flags, float* C_host, void* workspace,
+                               size_t workspace_bytes, void* stream) {
+    if (flags & ~(AMX_GEMM_SIMT | AMX_GEMM_TC)) return AMX_ERR_FLAGS;
+    if (!gemm_shape_ok(M, N, K, group_size)) return AMX_ERR_SHAPE;
+    if (M == 0 || N == 0) return AMX_OK;
+    if (!A_host || !W_host || !C_host) return AMX_ERR_NULL;
+    const size_t need = amx_linear_host_workspace_bytes(M, N, K, group_size);
+    if (!workspace || workspace_bytes < need) return AMX_ERR_WORKSPACE;
+    if (!aligned(workspace, kAlign)) return AMX_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t gemm_ws = amx_workspace_bytes(M, N, K, group_size, AMX_GEMM_AUTO);
+    const QuantSizes a = quant_sizes(M, K, group_size), w = quant_sizes(N, K, group_size);
+    uint8_t* p = static_cast<uint8_t*>(workspace);
+    uint8_t* gemm_base = p;            p += gemm_ws;
+    uint8_t* a_codes = p;              p += a.codes;
+    uint8_t* a_scales = p;             p += a.scales;
+    uint8_t* w_codes = p;              p += w.codes;
+    uint8_t* w_scales = p;             p += w.scales;
+    uint8_t* a_dev = p;                p += round_up((size_t)M * K * 2);
+    uint8_t* w_dev = p;                p += round_up((size_t)N * K * 2);
+    float* c_dev = reinterpret_cast<float*>(p);
+    if (cudaMemcpyAsync(a_dev, A_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(w_dev, W_host, (size_t)N * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return AMX_ERR_CUDA;
+    int rc = amx_quantize(a_dev, M, K, K, group_size, a_codes, a_scales, stream);
+    if (rc == AMX_OK) rc = amx_quantize(w_dev, N, K, K, group_size, w_codes, w_scales, stream);
+    if (rc == AMX_OK)
+        rc = amx_gemm(a_codes, a_scales, w_codes, w_scales, M, N, K, group_size, flags, c_dev, N, gemm_base,
+                      gemm_ws, stream);
+    if (rc != AMX_OK) return rc;
+    if (cudaMemcpyAsync(C_host, c_dev, (size_t)M * N * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return AMX_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? AMX_OK : AMX_ERR_CUDA;
+}
+
+extern "C" int amx_gemm_status(const void* workspace, void* stream) {
+    return gemm_tc_status(workspace, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" const char* amx_status_string(int status) {
+    switch (status) {
+        case AMX_OK: return "ok";
+        case AMX_ERR_NULL: return "null pointer";
+        case AMX_ERR_SHAPE: return "unsupported shape or group size";
+        case AMX_ERR_ALIGN: return "misaligned pointer or leading dimension";
+        case AMX_ERR_WORKSPACE: return "workspace missing or too small";
+        case AMX_ERR_FLAGS: return "bad flags";
+        case AMX_ERR_CUDA: return "CUDA runtime error";
+        case AMX_ERR_DEVICE: return "device is not sm_100";
+        case AMX_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}

@@ -1,0 +1,20 @@
+// Internal launchers of the two GEMM kernels.
+#pragma once
+
+#include "amx_common.cuh"
+
+namespace amx {
+
+int gemm_simt(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes,
+              const uint8_t* w_scales, int64_t M, int64_t N, int64_t K, int gs, float* C,
+              int64_t ld_c, cudaStream_t st);
+
+// Tensor-core (tcgen05) kernel: shapes it accepts, scratch it needs, launcher.
+bool gemm_tc_supported(int64_t M, int64_t N, int64_t K, int gs);
+size_t gemm_tc_workspace_bytes(int64_t M, int64_t N, int64_t K);
+int gemm_tc(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes,
+            const uint8_t* w_scales, int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c,
+            void* workspace, cudaStream_t st);
+int gemm_tc_status(const void* workspace, cudaStream_t st);
+
+}  // namespace amx

@@ -1,0 +1,225 @@
+// bf16 -> AMXFP4 direct cast (arXiv 2411.09909, Sections 4.2-4.3; Algorithm 1 applied per sign
+// with the FP8 E5M2 shared scale).  HBM-bound: 2 B read + 0.5625 B written per element.
+//
+// Exactness of the arithmetic (all decisions are bit-identical to exact rational arithmetic):
+//   * Side maxima are taken on the bf16 bit patterns as signed 16-bit integers.  Non-negative
+//     floats order like their bit patterns, negative ones become non-negative after flipping
+//     the sign bit, and the other side is removed by the max with 0.
+//   * scale = RNE_E5M2(max / 6) and magnitude = RNE_E2M1(|x| / scale) are evaluated as
+//     "multiply by a reciprocal that is slightly too large, then truncate to 12 significant
+//     bits".  max and x have 8 significant bits and every rounding midpoint times its divisor
+//     has at most 6, so a quotient is either exactly a midpoint (the tie: the product then
+//     overshoots by < 2^-18 relative and truncation returns the midpoint itself, which the
+//     converter resolves to even) or at least 2^-8 relative away from every midpoint
+//     (overshoot + truncation move it by < 2^-11: it stays on its side).
+//   * The final roundings are the hardware converts cvt.rn.satfinite.{e5m2x2,e2m1x2}.f32.
+#include <cuda_bf16.h>
+
+#include "amx_common.cuh"
+
+namespace amx {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kUnroll = 4;  // independent 16-byte loads in flight per thread
+
+// 1/6 rounded up a few ulps (0x3E2AAAAB is the nearest float, already above 1/6).
+__device__ __forceinline__ float sixth_up() { return __uint_as_float(0x3E2AAAAFu); }
+
+__device__ __forceinline__ float trunc12(float v) {
+    return __uint_as_float(__float_as_uint(v) & 0xFFFFF000u);
+}
+
+// {hi, lo} -> two E5M2 bytes, hi in bits 15..8.
+__device__ __forceinline__ uint32_t cvt_e5m2x2(float hi, float lo) {
+    unsigned short d;
+    asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+// Four pairs of quotients -> eight E2M1 nibbles; element i lands in nibble i.
+__device__ __forceinline__ uint32_t cvt_e2m1x8(const float (&r)[8]) {
+    uint32_t d;
+    asm("{\n"
+        ".reg .b8 b0, b1, b2, b3;\n"
+        "cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n"
+        "cvt.rn.satfinite.e2m1x2.f32 b1, %4, %3;\n"
+        "cvt.rn.satfinite.e2m1x2.f32 b2, %6, %5;\n"
+        "cvt.rn.satfinite.e2m1x2.f32 b3, %8, %7;\n"
+        "mov.b32 %0, {b0, b1, b2, b3};\n"
+        "}"
+        : "=r"(d)
+        : "f"(r[0]), "f"(r[1]), "f"(r[2]), "f"(r[3]), "f"(r[4]), "f"(r[5]), "f"(r[6]), "f"(r[7]));
+    return d;
+}
+
+// Reciprocal of an E5M2 value, biased upward by < 2^-18 relative; 0 for a zero scale.
+__device__ __forceinline__ float inv_scale_up(float s) {
+    float r;
+    asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(s));
+    r = __uint_as_float(__float_as_uint(r) + 16u);
+    return s > 0.0f ? r : 0.0f;
+}
+
+// Quantizes 8 consecutive elements held as 4 bf16x2 words.  `width` threads (8*width = group
+// size) hold one group and sit in consecutive lanes.  Returns the 8 nibbles; `sc` receives the
+// two scale bytes (positive side in bits 7..0, negative side in bits 15..8).
+template <int TPG>
+__device__ __forceinline__ uint32_t quantize8(const uint4 q, uint32_t& sc) {
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+    // per-halfword maxima: positive side on the raw bits, negative side on sign-flipped bits
+    uint32_t pm = __vimax3_s16x2_relu(w[0], w[1], __vmaxs2(w[2], w[3]));
+    uint32_t nm = __vimax3_s16x2_relu(w[0] ^ 0x80008000u, w[1] ^ 0x80008000u,
+                                      __vmaxs2(w[2] ^ 0x80008000u, w[3] ^ 0x80008000u));
+    // fold the two halfwords: result = {nmax bits : pmax bits}
+    uint32_t c = __vmaxs2(__byte_perm(pm, nm, 0x5410), __byte_perm(pm, nm, 0x7632));
+#pragma unroll
+    for (int d = 1; d < TPG; d <<= 1) c = __vmaxs2(c, __shfl_xor_sync(0xFFFFFFFFu, c, d));
+
+    const float pmax = __uint_as_float(c << 16);
+    const float nmax = __uint_as_float(c & 0xFFFF0000u);
+    sc = cvt_e5m2x2(trunc12(nmax * sixth_up()), trunc12(pmax * sixth_up()));
+    const float inv_p = inv_scale_up(e5m2_to_float(sc & 0xFFu));
+    const float inv_n = inv_scale_up(e5m2_to_float(sc >> 8));
+
+    float r[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float lo = __uint_as_float(w[i] << 16);
+        const float hi = __uint_as_float(w[i] & 0xFFFF0000u);
+        r[2 * i] = trunc12(lo * ((int)__float_as_uint(lo) < 0 ? inv_n : inv_p));
+        r[2 * i + 1] = trunc12(hi * ((int)w[i] < 0 ? inv_n : inv_p));
+    }
+    return cvt_e2m1x8(r);
+}
+
+// Groups along the contiguous axis.  One thread per 8 elements; n_vec = rows * K / 8.
+template <int TPG, bool CONTIG>
+__global__ void __launch_bounds__(kThreads)
+quantize_rows_kernel(const uint4* __restrict__ x, int64_t n_vec, int64_t vec_per_row,
+                     int64_t ld_vec, uint32_t* __restrict__ codes, uint16_t* __restrict__ scales) {
+    const int64_t base = (int64_t)blockIdx.x * (kThreads * kUnroll) + threadIdx.x;
+    uint4 q[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+        const int64_t v = base + (int64_t)u * kThreads;
+        q[u] = make_uint4(0, 0, 0, 0);
+        if (v < n_vec) {
+            int64_t off = v;
+            if (!CONTIG) off = (v / vec_per_row) * ld_vec + (v % vec_per_row);
+            q[u] = __ldcs(x + off);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+        const int64_t v = base + (int64_t)u * kThreads;
+        uint32_t sc;
+        const uint32_t nib = quantize8<TPG>(q[u], sc);
+        if (v < n_vec) {
+            codes[v] = nib;
+            if ((threadIdx.x & (TPG - 1)) == 0) scales[v / TPG] = (uint16_t)sc;
+        }
+    }
+}
+
+// Groups DOWN the rows (strided axis): x is [R, C]; output is the canonical layout of x^T.
+// A block stages a [64 rows x 64 columns] tile in shared memory and re-reads it column-wise.
+constexpr int kTR = 64, kTC = 64;
+
+template <int TPG>
+__global__ void __launch_bounds__(kThreads)
+quantize_cols_kernel(const __nv_bfloat16* __restrict__ x, int64_t R, int64_t C, int64_t ld,
+                     uint32_t* __restrict__ codes, uint16_t* __restrict__ scales, int gs) {
+    __shared__ uint16_t tile[kTC][kTR + 2];  // [column][row], padded
+    const int64_t r0 = (int64_t)blockIdx.y * kTR, c0 = (int64_t)blockIdx.x * kTC;
+    const uint16_t* xs = reinterpret_cast<const uint16_t*>(x);
+    for (int i = threadIdx.x; i < kTR * kTC; i += kThreads) {
+        const int rr = i / kTC, cc = i % kTC;
+        uint16_t v = 0;
+        if (r0 + rr < R && c0 + cc < C) v = xs[(r0 + rr) * ld + c0 + cc];
+        tile[cc][rr] = v;
+    }
+    __syncthreads();
+    // kTR/8 = 8 threads cover one column's 64 rows; 256 threads -> 32 columns per pass
+    for (int pass = 0; pass < kTC / (kThreads / (kTR / 8)); ++pass) {
+        const int cc = pass * (kThreads / (kTR / 8)) + threadIdx.x / (kTR / 8);
+        const int seg = threadIdx.x % (kTR / 8);
+        const uint16_t* t = &tile[cc][seg * 8];
+        uint4 q;
+        q.x = t[0] | ((uint32_t)t[1] << 16);
+        q.y = t[2] | ((uint32_t)t[3] << 16);
+        q.z = t[4] | ((uint32_t)t[5] << 16);
+        q.w = t[6] | ((uint32_t)t[7] << 16);
+        uint32_t sc;
+        const uint32_t nib = quantize8<TPG>(q, sc);
+        const int64_t col = c0 + cc, row = r0 + seg * 8;
+        if (col < C && row < R) {  // R % 8 == 0, so the 8 rows are all valid or all invalid
+            codes[(col * R + row) / 8] = nib;
+            if ((seg & (TPG - 1)) == 0) scales[(col * R + row) / gs] = (uint16_t)sc;
+        }
+    }
+}
+
+template <int TPG>
+int launch_rows(const void* x, int64_t rows, int64_t K, int64_t ld, uint8_t* codes,
+                uint8_t* scales, cudaStream_t st) {
+    const int64_t n_vec = rows * (K / 8);
+    const int64_t per_block = (int64_t)kThreads * kUnroll;
+    const int64_t blocks = (n_vec + per_block - 1) / per_block;
+    if (blocks > 0x7FFFFFFF) return AMX_ERR_SHAPE;
+    auto* xv = reinterpret_cast<const uint4*>(x);
+    auto* cv = reinterpret_cast<uint32_t*>(codes);
+    auto* sv = reinterpret_cast<uint16_t*>(scales);
+    if (ld == K)
+        quantize_rows_kernel<TPG, true><<<(unsigned)blocks, kThreads, 0, st>>>(xv, n_vec, K / 8, ld / 8, cv, sv);
+    else
+        quantize_rows_kernel<TPG, false><<<(unsigned)blocks, kThreads, 0, st>>>(xv, n_vec, K / 8, ld / 8, cv, sv);
+    return launch_status();
+}
+
+template <int TPG>
+int launch_cols(const void* x, int64_t R, int64_t C, int64_t ld, int gs, uint8_t* codes,
+                uint8_t* scales, cudaStream_t st) {
+    dim3 grid((unsigned)((C + kTC - 1) / kTC), (unsigned)((R + kTR - 1) / kTR));
+    if (grid.y > 65535) return AMX_ERR_SHAPE;
+    quantize_cols_kernel<TPG><<<grid, kThreads, 0, st>>>(
+        reinterpret_cast<const __nv_bfloat16*>(x), R, C, ld, reinterpret_cast<uint32_t*>(codes),
+        reinterpret_cast<uint16_t*>(scales), gs);
+    return launch_status();
+}
+
+}  // namespace
+}  // namespace amx
+
+extern "C" int amx_quantize(const void* x, int64_t rows, int64_t K, int64_t ld_x, int group_size,
+                            uint8_t* codes, uint8_t* scales, void* stream) {
+    using namespace amx;
+    if (!valid_group_size(group_size) || rows < 0 || K <= 0 || K % group_size || K % 8 || ld_x < K)
+        return AMX_ERR_SHAPE;
+    if (rows == 0) return AMX_OK;
+    if (!x || !codes || !scales) return AMX_ERR_NULL;
+    if (!aligned(x, 16) || ld_x % 8 || !aligned(codes, 4) || !aligned(scales, 2)) return AMX_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    switch (group_size) {
+        case 16: return launch_rows<2>(x, rows, K, ld_x, codes, scales, st);
+        case 32: return launch_rows<4>(x, rows, K, ld_x, codes, scales, st);
+        case 64: return launch_rows<8>(x, rows, K, ld_x, codes, scales, st);
+        default: return launch_rows<16>(x, rows, K, ld_x, codes, scales, st);
+    }
+}
+
+extern "C" int amx_quantize_t(const void* x, int64_t R, int64_t C, int64_t ld_x, int group_size,
+                              uint8_t* codes, uint8_t* scales, void* stream) {
+    using namespace amx;
+    if (!valid_group_size(group_size) || R < 0 || C < 0 || R % group_size || ld_x < C) return AMX_ERR_SHAPE;
+    if (R == 0 || C == 0) return AMX_OK;
+    if (!x || !codes || !scales) return AMX_ERR_NULL;
+    if (!aligned(x, 2) || !aligned(codes, 4) || !aligned(scales, 2)) return AMX_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    switch (group_size) {  // a 64-row tile holds whole groups only for gs <= 64
+        case 16: return launch_cols<2>(x, R, C, ld_x, group_size, codes, scales, st);
+        case 32: return launch_cols<4>(x, R, C, ld_x, group_size, codes, scales, st);
+        case 64: return launch_cols<8>(x, R, C, ld_x, group_size, codes, scales, st);
+        default: return AMX_ERR_SHAPE;
+    }
+}

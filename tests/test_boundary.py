@@ -1,0 +1,81 @@
+"""CPU-side checks of the C-ABI boundary: the library loads without a GPU, exports every symbol the
+header declares, and rejects bad arguments on the host before anything is launched."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    from paper_2411_09909_b200 import build, amx
+    build.build()
+    return amx.lib()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "amx.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(amx_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(L):
+    from paper_2411_09909_b200 import amx
+    declared = _declared_symbols()
+    assert len(declared) >= 13
+    for name in declared:
+        assert hasattr(L, name), name
+    assert sorted(amx.SYMBOLS) == declared
+
+
+def test_status_strings(L):
+    assert L.amx_status_string(0) == b"ok"
+    seen = {L.amx_status_string(c) for c in range(-8, 1)}
+    assert len(seen) == 9 and b"unknown status" not in seen
+    assert L.amx_status_string(-99) == b"unknown status"
+
+
+def test_host_detected_argument_errors(L):
+    fake = ctypes.c_void_p(0x1000)          # never dereferenced: every call below fails validation first
+    odd = ctypes.c_void_p(0x1001)
+    q = L.amx_quantize
+    assert q(None, 0, 64, 64, 32, None, None, None) == 0                # rows == 0: no-op
+    assert q(None, 4, 64, 64, 32, None, None, None) == -1               # NULL
+    assert q(fake, 4, 64, 64, 24, fake, fake, None) == -2               # group size
+    assert q(fake, 4, 80, 80, 32, fake, fake, None) == -2               # K % gs
+    assert q(fake, 4, 64, 32, 32, fake, fake, None) == -2               # ld < K
+    assert q(odd, 4, 64, 64, 32, fake, fake, None) == -3                # alignment
+    assert q(fake, 4, 64, 68, 32, fake, fake, None) == -3               # ld % 8
+    assert L.amx_quantize_t(fake, 48, 8, 8, 32, fake, fake, None) == -2  # R % gs
+    assert L.amx_dequantize(fake, fake, 4, 64, 32, 0x2, fake, 64, None) == -5
+    assert L.amx_dequantize(fake, fake, 4, 64, 32, 0, None, 64, None) == -1
+    g = L.amx_gemm
+    assert g(fake, fake, fake, fake, 4, 4, 64, 32, 0x30, fake, 4, None, 0, None) == -5  # both kernels asked
+    assert g(fake, fake, fake, fake, 4, 4, 64, 32, 0x100, fake, 4, None, 0, None) == -5
+    assert g(fake, fake, fake, fake, 4, 8, 64, 32, 0, fake, 4, None, 0, None) == -2     # ld_c < N
+    assert g(None, fake, fake, fake, 4, 4, 64, 32, 0x10, fake, 4, None, 0, None) == -1
+    assert g(fake, fake, fake, fake, 0, 4, 64, 32, 0x10, fake, 4, None, 0, None) == 0   # empty
+    assert L.amx_quant_gemm(fake, 64, fake, fake, 4, 4, 64, 32, 0x10, fake, 4, None, 0, None) == -4
+    assert L.amx_softmax_bf16(fake, 4, 0, 0, 1.0, fake, 0, None) == -2
+
+
+def test_workspace_sizes(L):
+    assert L.amx_workspace_bytes(128, 128, 100, 32, 0) == 0            # invalid shape
+    simt = L.amx_workspace_bytes(100, 100, 64, 32, 0x10)
+    assert simt == 0
+    qg = L.amx_quant_gemm_workspace_bytes(100, 100, 64, 32, 0x10)
+    assert qg >= 100 * 32 + 100 * 2 * 2 and qg % 256 == 0
+    lh = L.amx_linear_host_workspace_bytes(128, 256, 512, 32)
+    assert lh >= 128 * 512 * 2 + 256 * 512 * 2 + 128 * 256 * 4
+    assert L.amx_gemm_kernel_for(100, 100, 64, 32, 0x10) == 0x10
+
+
+def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
+    from paper_2411_09909_b200 import amx
+    monkeypatch.setattr(amx, "_lib", None)
+    monkeypatch.setattr(amx, "_LIB_PATH", str(tmp_path / "missing.so"))
+    with pytest.raises(amx.AmxError):
+        amx.lib()

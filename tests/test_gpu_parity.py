@@ -1,0 +1,229 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs.  Codes and scales must match bit for bit; GEMM outputs within 1e-3 relative Frobenius
+error of the oracle's fp64 product of the decoded operands."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2411_09909_b200 import amx, inputs
+
+pytestmark = pytest.mark.gpu
+GEMM_TOL = 1e-3
+
+
+def dev_bf16(bits: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def rel_fro(got: np.ndarray, ref: np.ndarray) -> float:
+    den = np.linalg.norm(ref.astype(np.float64))
+    num = np.linalg.norm(got.astype(np.float64) - ref.astype(np.float64))
+    return num / den if den > 0 else num
+
+
+def check_quantize(bits, gs=32):
+    c, s = amx.quantize(dev_bf16(bits), gs)
+    oc, os_ = oracle.quantize(bits, gs)
+    assert np.array_equal(c.cpu().numpy(), oc)
+    assert np.array_equal(s.cpu().numpy(), os_)
+    return c, s
+
+
+# ------------------------------------------------------------------ quantize --
+
+@pytest.mark.parametrize("gs", [16, 32, 64, 128])
+@pytest.mark.parametrize("kind", ["normal", "wide", "mixed"])
+def test_quantize_bit_exact_random_groups(gs, kind):
+    check_quantize(inputs.random_groups(31, 257, 1280, kind), gs)      # ragged: 257 rows, 10 tiles + tail
+
+
+def test_quantize_exhaustive_bf16_times_scale_codes():
+    """Every finite bf16 value against every normal/subnormal E5M2 scale code, on both sides."""
+    finite = np.concatenate([np.arange(0, 0x7F80), np.arange(0x8000, 0xFF80)]).astype(np.uint16)
+    per = 30
+    n_groups = -(-finite.size // per)
+    payload = np.zeros(n_groups * per, np.uint16)
+    payload[: finite.size] = finite
+    payload = payload.reshape(n_groups, per)
+    rows = []
+    for sc in range(1, 0x7C):
+        m_pos = inputs.f32_to_bf16_bits(np.array([6.0 * oracle.e5m2_value(sc)], np.float32))[0]
+        sc_n = (sc * 7) % 0x7B + 1
+        m_neg = inputs.f32_to_bf16_bits(np.array([-6.0 * oracle.e5m2_value(sc_n)], np.float32))[0]
+        g = np.empty((n_groups, 32), np.uint16)
+        g[:, 0], g[:, 1], g[:, 2:] = m_pos, m_neg, payload
+        rows.append(g.reshape(-1))
+    check_quantize(np.stack(rows), 32)
+
+
+def test_quantize_scale_rounding_all_maxima():
+    """Every finite positive bf16 value as the group maximum (scale = nearest E5M2 of max/6)."""
+    vals = np.arange(0, 0x7F80, dtype=np.uint16)
+    bits = np.zeros((vals.size, 32), np.uint16)
+    bits[:, 5] = vals
+    bits[:, 9] = vals[::-1] | 0x8000
+    check_quantize(bits.reshape(-1, 32 * 64), 32)
+
+
+def test_quantize_strided_rows_and_tiny_shapes():
+    bits = inputs.random_groups(32, 5, 96, "mixed")
+    x = torch.zeros((5, 160), dtype=torch.bfloat16, device="cuda")
+    x[:, :96] = dev_bf16(bits)
+    c, s = amx.quantize(x[:, :96], 32)
+    oc, os_ = oracle.quantize(bits, 32)
+    assert np.array_equal(c.cpu().numpy(), oc) and np.array_equal(s.cpu().numpy(), os_)
+    check_quantize(inputs.random_groups(33, 1, 32, "normal"), 32)        # a single group
+    c0, s0 = amx.quantize(torch.empty((0, 64), dtype=torch.bfloat16, device="cuda"), 32)
+    assert c0.shape == (0, 32) and s0.shape == (0, 2, 2)
+
+
+@pytest.mark.parametrize("gs", [16, 32, 64])
+def test_quantize_t_matches_oracle_on_transpose(gs):
+    bits = inputs.random_groups(34, 192, 128, "mixed")[:, :100]           # R=192, C=100 (ragged tiles)
+    bits = np.ascontiguousarray(bits)
+    c, s = amx.quantize_t(dev_bf16(bits), gs)
+    oc, os_ = oracle.quantize(np.ascontiguousarray(bits.T), gs)
+    assert np.array_equal(c.cpu().numpy(), oc) and np.array_equal(s.cpu().numpy(), os_)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_dequantize_exact(dtype):
+    bits = inputs.random_groups(35, 100, 640, "wide")
+    oc, os_ = oracle.quantize(bits, 32)
+    out = amx.dequantize(torch.from_numpy(oc).cuda(), torch.from_numpy(os_).cuda(), 32, dtype)
+    assert np.array_equal(out.double().cpu().numpy(), oracle.dequantize(oc, os_, 32))
+
+
+def test_dequantize_all_codes_all_scales():
+    codes = np.tile(np.arange(16, dtype=np.uint8), 2)                     # one group: every code twice
+    packed = oracle.pack_codes(np.tile(codes, (0x7C, 1)))
+    scales = np.zeros((0x7C, 1, 2), np.uint8)
+    scales[:, 0, 0] = np.arange(0x7C)
+    scales[:, 0, 1] = np.arange(0x7C)[::-1]
+    out = amx.dequantize(torch.from_numpy(packed).cuda(), torch.from_numpy(scales).cuda(), 32, torch.float32)
+    assert np.array_equal(out.double().cpu().numpy(), oracle.dequantize(packed, scales, 32))
+
+
+# ---------------------------------------------------------------------- GEMM --
+
+def _gemm_case(seed, M, N, K, gs, flags, kind="mixed"):
+    a = inputs.random_groups(seed, M, K, kind)
+    w = inputs.random_groups(seed + 1, N, K, "normal")
+    (ac, as_), (wc, ws) = oracle.quantize(a, gs), oracle.quantize(w, gs)
+    got = amx.gemm(*(torch.from_numpy(t).cuda() for t in (ac, as_, wc, ws)), gs, flags).cpu().numpy()
+    ref = oracle.gemm(ac, as_, wc, ws, gs)
+    return got, ref
+
+
+@pytest.mark.parametrize("shape", [(1, 1, 32), (70, 130, 96), (128, 256, 512), (200, 72, 1024)])
+@pytest.mark.parametrize("gs", [16, 32, 128])
+def test_gemm_simt_against_oracle(shape, gs):
+    M, N, K = shape
+    if K % gs:
+        pytest.skip("K not a multiple of the group size")
+    got, ref = _gemm_case(41, M, N, K, gs, amx.GEMM_SIMT, "normal")
+    assert rel_fro(got, ref) <= GEMM_TOL
+    assert rel_fro(got, ref) <= 1e-5          # fp32 accumulation of <= 10-bit products is far tighter
+
+
+def test_gemm_wide_dynamic_range_rows():
+    got, ref = _gemm_case(42, 96, 64, 256, 32, amx.GEMM_SIMT, "mixed")
+    for m in range(96):                        # row-wise: rows differ by many orders of magnitude
+        if np.all(np.isfinite(ref[m])) and np.linalg.norm(ref[m]) > 0:
+            assert rel_fro(got[m], ref[m]) <= GEMM_TOL
+
+
+def test_gemm_exact_on_small_integers():
+    rng = np.random.default_rng(7)
+    grid = np.array([0, 1, 2, 3, 4, 6], np.float32)
+    def ints(r, k):
+        t = grid[rng.integers(0, 6, size=(r, k))] * rng.choice([-1.0, 1.0], size=(r, k)).astype(np.float32)
+        t[:, ::32], t[:, 1::32] = 6.0, -6.0
+        return t
+    a, w = ints(130, 256), ints(70, 256)
+    qa, qw = oracle.quantize(inputs.f32_to_bf16_bits(a), 32), oracle.quantize(inputs.f32_to_bf16_bits(w), 32)
+    got = amx.gemm(*(torch.from_numpy(t).cuda() for t in (*qa, *qw)), 32, amx.GEMM_SIMT).cpu().numpy()
+    assert np.array_equal(got, (a.astype(np.int64) @ w.astype(np.int64).T).astype(np.float32))
+
+
+def test_quant_gemm_equals_quantize_then_gemm():
+    a = dev_bf16(inputs.activation(1, 0))
+    wc, ws = amx.quantize(dev_bf16(inputs.weight(1, 0)), 32)
+    ac, as_ = amx.quantize(a, 32)
+    assert torch.equal(amx.quant_gemm(a, wc, ws, 32), amx.gemm(ac, as_, wc, ws, 32))
+
+
+def test_config1_full_layer():
+    a_bits, w_bits = inputs.activation(1, 0), inputs.weight(1, 0)
+    ac, as_ = check_quantize(a_bits)
+    wc, ws = check_quantize(w_bits)
+    got = amx.gemm(ac, as_, wc, ws, 32).cpu().numpy()
+    ref = oracle.gemm(ac.cpu().numpy(), as_.cpu().numpy(), wc.cpu().numpy(), ws.cpu().numpy(), 32)
+    assert rel_fro(got, ref) <= GEMM_TOL
+
+
+def test_linear_host_entry_point():
+    a_bits, w_bits = inputs.activation(1, 0), inputs.weight(1, 0, N=256)
+    a = torch.from_numpy(a_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+    w = torch.from_numpy(w_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+    c = torch.empty((128, 256), dtype=torch.float32).pin_memory()
+    ws = torch.empty(amx.lib().amx_linear_host_workspace_bytes(128, 256, 1024, 32), dtype=torch.uint8, device="cuda")
+    amx.linear_host(a, w, c, ws)
+    ref = oracle.gemm(*oracle.quantize(a_bits, 32), *oracle.quantize(w_bits, 32), 32)
+    assert rel_fro(c.numpy(), ref) <= GEMM_TOL
+
+
+# ----------------------------------------------------------- attention glue --
+
+def test_softmax_bf16_against_oracle():
+    rng = np.random.default_rng(8)
+    S = (rng.standard_normal((40, 1000)) * 30).astype(np.float32)
+    got = amx.softmax_bf16(torch.from_numpy(S).cuda(), 128 ** -0.5).view(torch.int16).cpu().numpy().view(np.uint16)
+    want = oracle.softmax_bf16(S, 128 ** -0.5)
+    # fp32 exp on the device vs fp64 exp on the host: allow one bf16 ulp on a small fraction
+    diff = np.abs(got.astype(np.int32) - want.astype(np.int32))
+    assert diff.max() <= 1 and np.mean(diff != 0) < 0.02
+
+
+def test_attention_small_head_against_oracle_pipeline():
+    """Config-5 pipeline at reduced size: Q/K/V codes bit-exact; the device quantizer applied to the
+    device's own bf16 P equals the oracle quantizer on the same bits; O within tolerance of the all-CPU
+    pipeline."""
+    qb, kb, vb = (t[0] for t in inputs.attention_qkv(heads=1, seq=256))
+    O, P = amx.attention(dev_bf16(qb), dev_bf16(kb), dev_bf16(vb))
+    check_quantize(qb), check_quantize(kb)
+    vc, vs = amx.quantize_t(dev_bf16(vb), 32)
+    ovc, ovs = oracle.quantize(np.ascontiguousarray(vb.T), 32)
+    assert np.array_equal(vc.cpu().numpy(), ovc) and np.array_equal(vs.cpu().numpy(), ovs)
+    p_bits = P.view(torch.int16).cpu().numpy().view(np.uint16)
+    check_quantize(p_bits)
+    # all-CPU pipeline
+    S = oracle.gemm(*oracle.quantize(qb, 32), *oracle.quantize(kb, 32), 32)
+    Pcpu = oracle.softmax_bf16(S, 128 ** -0.5)
+    Ocpu = oracle.gemm(*oracle.quantize(Pcpu, 32), ovc, ovs, 32)
+    assert rel_fro(O.cpu().numpy(), Ocpu) <= GEMM_TOL
+
+
+# ------------------------------------------------ full-size configurations --
+
+@pytest.mark.parametrize("config,layer", [(2, 0), (2, 3), (3, 1), (4, 2)])
+def test_full_size_layer_sampled(config, layer):
+    """Whole-tensor launches at the benchmark's sizes; codes and scales compared on the whole activation
+    for config 2 and on sampled rows otherwise; GEMM compared on 64 sampled rows x all N."""
+    spec = inputs.LINEAR_CONFIGS[config]
+    M = spec["M"]
+    a_bits, w_bits = inputs.activation(config, layer), inputs.weight(config, layer)
+    ac, as_ = amx.quantize(dev_bf16(a_bits), 32)
+    wc, ws = amx.quantize(dev_bf16(w_bits), 32)
+    rng = np.random.default_rng(100 * config + layer)
+    rows = np.sort(rng.choice(M, size=64, replace=False))
+    arow = np.arange(M) if config == 2 else np.union1d(rows, rng.choice(M, size=256, replace=False))
+    oac, oas = oracle.quantize(a_bits[arow], 32)
+    assert np.array_equal(ac.cpu().numpy()[arow], oac) and np.array_equal(as_.cpu().numpy()[arow], oas)
+    wrow = np.sort(rng.choice(w_bits.shape[0], size=512, replace=False))
+    owc, ows = oracle.quantize(w_bits[wrow], 32)
+    assert np.array_equal(wc.cpu().numpy()[wrow], owc) and np.array_equal(ws.cpu().numpy()[wrow], ows)
+    got = amx.gemm(ac, as_, wc, ws, 32).cpu().numpy()[rows]
+    ref = oracle.gemm(ac.cpu().numpy(), as_.cpu().numpy(), wc.cpu().numpy(), ws.cpu().numpy(), 32, rows=rows)
+    assert rel_fro(got, ref) <= GEMM_TOL
