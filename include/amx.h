@@ -80,7 +80,7 @@ int amx_quantize(const void* x, int64_t rows, int64_t K, int64_t ld_x, int group
  * result is laid out as the canonical quantization of x transposed:
  *   codes [C, R/2], scales [C, R/gs, 2].
  * This is how V enters the P*V product with groups along the sequence (Appendix C: Value and the
- * self-attention map are quantized too).  R % gs == 0, R % 2 == 0; x 2-byte aligned.
+ * self-attention map are quantized too).  R % gs == 0; gs is 16, 32 or 64 here; x 2-byte aligned.
  */
 int amx_quantize_t(const void* x, int64_t R, int64_t C, int64_t ld_x, int group_size,
                    uint8_t* codes, uint8_t* scales, void* stream);
@@ -97,7 +97,9 @@ int amx_dequantize(const uint8_t* codes, const uint8_t* scales, int64_t rows, in
  * amx_gemm - C[m,n] = sum_k Ahat[m,k] * What[n,k] with Ahat, What the decoded operands
  * (Section 4.3: each factor uses the shared scale its own sign selects), fp32 accumulation.
  *   a_codes/a_scales  canonical [M, K];  w_codes/w_scales canonical [N, K] (both K-major)
- *   C   out fp32 [M, ld_c], ld_c >= N; 16-byte aligned, ld_c % 4 == 0
+ *   C   out fp32 [M, ld_c], ld_c >= N
+ *   alignment: codes 4 bytes, scales 2 bytes, C 4 bytes for the SIMT kernel; the tensor-core
+ *   kernel needs codes and C 16-byte aligned and ld_c % 4 == 0
  *   workspace  device scratch of at least amx_workspace_bytes(M, N, K, gs, flags) bytes,
  *              256-byte aligned (may be NULL when that size is 0)
  * M == 0 or N == 0 is a no-op.
