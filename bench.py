@@ -74,6 +74,11 @@ class ClockSampler:
         except OSError:
             pass
 
+    def mark(self):
+        """Samples written before this call (warm-up, idle) are ignored by stop()."""
+        self.file.flush()
+        self.skip = sum(1 for l in open(self.file.name) if l.strip())
+
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
         if self.proc is None:
@@ -84,7 +89,7 @@ class ClockSampler:
         except subprocess.TimeoutExpired:
             self.proc.kill()
         self.file.flush()
-        rows = [l.strip().split(", ") for l in open(self.file.name) if l.strip()]
+        rows = [l.strip().split(", ") for l in open(self.file.name) if l.strip()][getattr(self, "skip", 0):]
         os.unlink(self.file.name)
         sm, reasons = [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
@@ -222,10 +227,13 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local) if rank == 0 else None   # started early: nvidia-smi needs ~0.2 s to begin
     for _ in range(max(args.warmup, 3)):
         step(False)
     barrier()
-    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        time.sleep(0.3)
+        sampler.mark()
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_start.record()
     for _ in range(args.steps):
@@ -323,7 +331,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()

@@ -98,8 +98,8 @@ int amx_dequantize(const uint8_t* codes, const uint8_t* scales, int64_t rows, in
  * (Section 4.3: each factor uses the shared scale its own sign selects), fp32 accumulation.
  *   a_codes/a_scales  canonical [M, K];  w_codes/w_scales canonical [N, K] (both K-major)
  *   C   out fp32 [M, ld_c], ld_c >= N
- *   alignment: codes 4 bytes, scales 2 bytes, C 4 bytes for the SIMT kernel; the tensor-core
- *   kernel needs codes and C 16-byte aligned and ld_c % 4 == 0
+ *   alignment: codes 4 bytes (16 bytes for the tensor-core kernel), scales 2 bytes, C 4 bytes
+ *   (the tensor-core kernel stores vectors when C is 16-byte aligned and ld_c % 4 == 0)
  *   workspace  device scratch of at least amx_workspace_bytes(M, N, K, gs, flags) bytes,
  *              256-byte aligned (may be NULL when that size is 0)
  * M == 0 or N == 0 is a no-op.

@@ -63,7 +63,7 @@ extern "C" int amx_gemm(const uint8_t* a_codes, const uint8_t* a_scales, const u
                         void* stream) {
     if (flags & ~(AMX_GEMM_SIMT | AMX_GEMM_TC)) return AMX_ERR_FLAGS;
     if (!gemm_shape_ok(M, N, K, group_size) || ld_c < N) return AMX_ERR_SHAPE;
-    const uint32_t kernel = pick_kernel(M, N, K, group_size, flags);
+    uint32_t kernel = pick_kernel(M, N, K, group_size, flags);
     if (!kernel) return (flags & AMX_GEMM_SIMT) ? AMX_ERR_FLAGS : AMX_ERR_SHAPE;
     if (M == 0 || N == 0) return AMX_OK;
     if (!a_codes || !a_scales || !w_codes || !w_scales || !C) return AMX_ERR_NULL;
@@ -73,7 +73,7 @@ extern "C" int amx_gemm(const uint8_t* a_codes, const uint8_t* a_scales, const u
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (kernel == AMX_GEMM_SIMT)
         return gemm_simt(a_codes, a_scales, w_codes, w_scales, M, N, K, group_size, C, ld_c, st);
-    if (!aligned(a_codes, 16) || !aligned(w_codes, 16) || !aligned(C, 16) || ld_c % 4) return AMX_ERR_ALIGN;
+    if (!aligned(a_codes, 16) || !aligned(w_codes, 16)) return AMX_ERR_ALIGN;
     const size_t need = round_up(gemm_tc_workspace_bytes(M, N, K));
     if (need && (!workspace || workspace_bytes < need)) return AMX_ERR_WORKSPACE;
     if (need && !aligned(workspace, kAlign)) return AMX_ERR_ALIGN;

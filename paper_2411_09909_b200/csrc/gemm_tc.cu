@@ -1,13 +1,335 @@
-// Placeholder until the tcgen05 kernel lands: reports that no shape is supported, so that
-// AMX_GEMM_AUTO picks the SIMT kernel and AMX_GEMM_TC returns AMX_ERR_SHAPE.
+// AMXFP4 x AMXFP4 -> fp32 on the 5th-generation tensor cores (tcgen05, sm_100a), exact-decode
+// variant: C[m,n] = sum_k Ahat[m,k] * What[n,k] (arXiv 2411.09909, Section 4.3).
+//
+// The format gives every element one of TWO group scales, picked by the element's own sign, so
+// an operand tile is not a single block-scaled FP4 matrix.  Here each tile is decoded exactly to
+// bf16 in shared memory (a decoded value has at most 5 significant bits) and multiplied with
+// tcgen05.mma kind::f16, fp32 accumulators in tensor memory.
+//
+// One CTA computes one 128 x 256 tile of C.  Roles:
+//   warps 0..7  producers: read 4-bit codes + E5M2 scales from global memory, decode one 64-wide
+//               K block to bf16 in the 128-byte-swizzled K-major layout the MMA reads; afterwards
+//               they are the epilogue (TMEM -> registers -> global)
+//   warp 8      allocates tensor memory; one elected lane issues the MMAs and commits them to
+//               mbarriers
+// Two shared-memory stages (48 KB each) cycle through full/empty mbarriers; two CTAs share an SM
+// so that one CTA's epilogue overlaps the other's main loop.
+//
+// Decode: per 32-element group the 2 x 8 possible values (magnitude x side scale) are computed
+// once with packed bf16 multiplies and held as byte-plane lookup tables in registers; elements
+// are then looked up four at a time with byte permutes and the side is chosen with a mask built
+// from the sign bits.
+//
+// Every wait is bounded: when a limit expires the CTA records AMX_ERR_TIMEOUT in the status word,
+// all roles leave their loops, tensor memory is released and the kernel returns.
+#include <cuda_bf16.h>
+
 #include "gemm.cuh"
 
 namespace amx {
+namespace {
 
-bool gemm_tc_supported(int64_t, int64_t, int64_t, int) { return false; }
-size_t gemm_tc_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
-int gemm_tc(const uint8_t*, const uint8_t*, const uint8_t*, const uint8_t*, int64_t, int64_t,
-            int64_t, float*, int64_t, void*, cudaStream_t) { return AMX_ERR_SHAPE; }
-int gemm_tc_status(const void*, cudaStream_t) { return AMX_OK; }
+constexpr int BM = 128, BN = 256, BK = 64;       // tile; BK bf16 = one 128-byte swizzle row
+constexpr int kStages = 2;
+constexpr int kProducerWarps = 8;
+constexpr int kThreads = (kProducerWarps + 1) * 32;
+constexpr int kTileA = BM * BK * 2, kTileB = BN * BK * 2, kStageBytes = kTileA + kTileB;
+constexpr int kTmemCols = 256;
+constexpr uint32_t kSpinLimit = 1u << 24;         // mbarrier polls before giving up
+
+struct __align__(8) Control {
+    uint64_t full[kStages], empty[kStages], accum;
+    uint32_t tmem_base;
+    volatile int abort;
+};
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + sizeof(Control);
+
+// ---------------------------------------------------------------------------- PTX wrappers --
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* b, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(b)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* b) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* b, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the limit expired or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, Control* ctl, int* status) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try_wait(b, parity)) return true;
+        if (ctl->abort) return false;
+    }
+    ctl->abort = 1;
+    if (status) atomicExch(status, (int)AMX_ERR_TIMEOUT);
+    return false;
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst)), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate; issued by one thread.
+__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// mbarrier arrive once all MMAs issued so far by this thread have completed.
+__device__ __forceinline__ void mma_commit(uint64_t* b) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(b)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows 128 B apart, groups of
+// 8 rows 1024 B apart (stride byte offset); the leading byte offset is unused for this layout.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M x N.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+// ---------------------------------------------------------------------------------- decode --
+// prmt.b32: result byte i = byte (selector nibble i & 7) of {b, a}; when bit 3 of the nibble is set the
+// byte's sign bit is replicated over the whole result byte instead.
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+struct GroupTables {   // byte planes of the 8 values per side: [side][plane lo/hi][2 regs]
+    uint32_t lo_p0, lo_p1, hi_p0, hi_p1, lo_n0, lo_n1, hi_n0, hi_n1;
+};
+
+// bf16x2 {s, s} of an E5M2 byte (exact: E5M2 is the top byte of a half; a half widens exactly).
+__device__ __forceinline__ uint32_t scale_pair(uint32_t byte) {
+    const uint32_t f = __float_as_uint(e5m2_to_float(byte));
+    return prmt(f, f, 0x3232);
+}
+__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
+    __nv_bfloat162 r = __hmul2(*reinterpret_cast<__nv_bfloat162*>(&a), *reinterpret_cast<__nv_bfloat162*>(&b));
+    return *reinterpret_cast<uint32_t*>(&r);
+}
+__device__ __forceinline__ GroupTables make_tables(uint32_t sc) {
+    // E2M1 magnitudes as bf16 pairs: {0, .5} {1, 1.5} {2, 3} {4, 6}
+    const uint32_t c01 = 0x3F000000u, c23 = 0x3FC03F80u, c45 = 0x40404000u, c67 = 0x40C04080u;
+    const uint32_t sp = scale_pair(sc & 0xFFu), sn = scale_pair(sc >> 8) ^ 0x80008000u;
+    GroupTables t;
+    uint32_t a = mul_bf16x2(c01, sp), b = mul_bf16x2(c23, sp), c = mul_bf16x2(c45, sp), d = mul_bf16x2(c67, sp);
+    t.lo_p0 = prmt(a, b, 0x6420); t.hi_p0 = prmt(a, b, 0x7531);
+    t.lo_p1 = prmt(c, d, 0x6420); t.hi_p1 = prmt(c, d, 0x7531);
+    a = mul_bf16x2(c01, sn); b = mul_bf16x2(c23, sn); c = mul_bf16x2(c45, sn); d = mul_bf16x2(c67, sn);
+    t.lo_n0 = prmt(a, b, 0x6420); t.hi_n0 = prmt(a, b, 0x7531);
+    t.lo_n1 = prmt(c, d, 0x6420); t.hi_n1 = prmt(c, d, 0x7531);
+    return t;
+}
+// 8 codes (one 32-bit word) -> 8 bf16 values (16 bytes).
+__device__ __forceinline__ uint4 decode_word(uint32_t w, const GroupTables& t) {
+    const uint32_t sel = w & 0x77777777u, selh = sel >> 16, ws = w << 4;
+    const uint32_t m0 = prmt(ws, w, 0xD9C8), m1 = prmt(ws, w, 0xFBEA);  // 0xFF where negative
+    uint32_t lo, hi;
+    uint4 o;
+    lo = (prmt(t.lo_p0, t.lo_p1, sel) & ~m0) | (prmt(t.lo_n0, t.lo_n1, sel) & m0);
+    hi = (prmt(t.hi_p0, t.hi_p1, sel) & ~m0) | (prmt(t.hi_n0, t.hi_n1, sel) & m0);
+    o.x = prmt(lo, hi, 0x5140); o.y = prmt(lo, hi, 0x7362);
+    lo = (prmt(t.lo_p0, t.lo_p1, selh) & ~m1) | (prmt(t.lo_n0, t.lo_n1, selh) & m1);
+    hi = (prmt(t.hi_p0, t.hi_p1, selh) & ~m1) | (prmt(t.hi_n0, t.hi_n1, selh) & m1);
+    o.z = prmt(lo, hi, 0x5140); o.w = prmt(lo, hi, 0x7362);
+    return o;
+}
+
+struct Task {      // one 32-element group of one tile row
+    uint4 codes;
+    uint32_t scales;
+};
+constexpr int kTasksPerThread = (BM + BN) * 2 / (kProducerWarps * 32);   // 3
+
+__device__ __forceinline__ Task load_task(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales,
+                                          int64_t row, int64_t rows, int64_t K, int64_t k) {
+    Task t;
+    t.codes = make_uint4(0, 0, 0, 0);
+    t.scales = 0;
+    if (row < rows && k < K) {
+        t.codes = __ldg(reinterpret_cast<const uint4*>(codes + row * (K / 2) + k / 2));
+        t.scales = __ldg(reinterpret_cast<const unsigned short*>(scales + (row * (K / 32) + k / 32) * 2));
+    }
+    return t;
+}
+
+__global__ void __launch_bounds__(kThreads, 2)
+gemm_tc_kernel(const uint8_t* __restrict__ a_codes, const uint8_t* __restrict__ a_scales,
+               const uint8_t* __restrict__ w_codes, const uint8_t* __restrict__ w_scales,
+               int64_t M, int64_t N, int64_t K, float* __restrict__ C, int64_t ld_c, int vec_store,
+               int* __restrict__ status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    Control* ctl = reinterpret_cast<Control*>(tiles + kStages * kStageBytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t m0 = (int64_t)blockIdx.y * BM, n0 = (int64_t)blockIdx.x * BN;
+    const int num_kb = (int)((K + BK - 1) / BK);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&ctl->full[s], kProducerWarps);
+            mbar_init(&ctl->empty[s], 1);
+        }
+        mbar_init(&ctl->accum, 1);
+        ctl->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kProducerWarps) tmem_alloc(&ctl->tmem_base, kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = ctl->tmem_base;
+
+    if (warp < kProducerWarps) {
+        // ------------------------------------------------------------------ producers
+        // task i of this thread: tile row (tid >> 1) + 128 * i, group (tid & 1) of the K block
+        const int tid = threadIdx.x, half = tid & 1, r = tid >> 1;
+        Task cur[kTasksPerThread], nxt[kTasksPerThread];
+        auto load_all = [&](Task (&t)[kTasksPerThread], int kb) {
+            const int64_t k = (int64_t)kb * BK + half * 32;
+            t[0] = load_task(a_codes, a_scales, m0 + r, M, K, k);
+#pragma unroll
+            for (int i = 1; i < kTasksPerThread; ++i)
+                t[i] = load_task(w_codes, w_scales, n0 + r + 128 * (i - 1), N, K, k);
+        };
+        load_all(cur, 0);
+        bool ok = true;
+        for (int kb = 0; kb < num_kb && ok; ++kb) {
+            const int s = kb % kStages;
+            if (kb + 1 < num_kb) load_all(nxt, kb + 1);
+            if (kb >= kStages) ok = mbar_wait(&ctl->empty[s], ((kb / kStages) - 1) & 1, ctl, status);
+            if (!ok) break;
+            uint8_t* stage = tiles + s * kStageBytes;
+#pragma unroll
+            for (int i = 0; i < kTasksPerThread; ++i) {
+                const GroupTables t = make_tables(cur[i].scales);
+                const int row = r + 128 * i;                       // row inside [A tile | B tile]
+                uint8_t* dst = stage + row * 128;                  // A tile is 128 rows: B rows follow it
+                const uint32_t w[4] = {cur[i].codes.x, cur[i].codes.y, cur[i].codes.z, cur[i].codes.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int chunk = half * 4 + j;                // 16-byte chunk inside the 128-byte row
+                    *reinterpret_cast<uint4*>(dst + ((chunk ^ (row & 7)) << 4)) = decode_word(w[j], t);
+                }
+            }
+            fence_proxy_async();          // make the generic-proxy stores visible to the tensor core
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->full[s]);
+#pragma unroll
+            for (int i = 0; i < kTasksPerThread; ++i) cur[i] = nxt[i];
+        }
+        // ------------------------------------------------------------------ epilogue
+        if (ok) ok = mbar_wait(&ctl->accum, 0, ctl, status);
+        tc_fence_after();
+        if (ok) {
+            const int q = warp & 3, h = warp >> 2;                 // lane quarter, column half
+            const int64_t m = m0 + q * 32 + lane;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN / 2; c0 += 32) {
+                uint32_t v[32];
+                const int col = h * (BN / 2) + c0;
+                tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)col, v);
+                tmem_ld_wait();
+                if (m < M) {
+                    float* out = C + m * ld_c + n0 + col;
+                    if (vec_store && n0 + col + 32 <= N) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<float4*>(out + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                                              __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (n0 + col + j < N) out[j] = __uint_as_float(v[j]);
+                    }
+                }
+            }
+        }
+    } else if (lane == 0) {
+        // ------------------------------------------------------------------ MMA issuer
+        bool ok = true;
+        for (int kb = 0; kb < num_kb && ok; ++kb) {
+            const int s = kb % kStages;
+            ok = mbar_wait(&ctl->full[s], (kb / kStages) & 1, ctl, status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t a_addr = smem_u32(tiles + s * kStageBytes), b_addr = a_addr + kTileA;
+#pragma unroll
+            for (int k = 0; k < BK / 16; ++k)     // 16 bf16 = 32 bytes further along the swizzled row
+                mma_bf16(tmem, smem_desc_sw128(a_addr + k * 32), smem_desc_sw128(b_addr + k * 32), kIdesc,
+                         (kb | k) ? 1u : 0u);
+            mma_commit(&ctl->empty[s]);           // frees the stage once these MMAs have read it
+        }
+        if (ok) mma_commit(&ctl->accum);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kProducerWarps) {
+        tc_fence_after();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+}  // namespace
+
+bool gemm_tc_supported(int64_t M, int64_t N, int64_t K, int gs) {
+    return gs == 32 && M > 0 && N > 0 && K > 0 && K % 32 == 0 && (M + BM - 1) / BM <= 65535;
+}
+
+size_t gemm_tc_workspace_bytes(int64_t, int64_t, int64_t) { return 256; }   // the status word
+
+int gemm_tc(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes, const uint8_t* w_scales,
+            int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {
+    static bool configured = false;   // per process; the attribute is per function, not per device state we keep
+    if (!configured) {
+        if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+            return AMX_ERR_CUDA;
+        configured = true;
+    }
+    int* status = static_cast<int*>(workspace);
+    if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return AMX_ERR_CUDA;
+    dim3 grid((unsigned)((N + BN - 1) / BN), (unsigned)((M + BM - 1) / BM));
+    const int vec_store = aligned(C, 16) && ld_c % 4 == 0;   // else the epilogue stores scalars
+    gemm_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(a_codes, a_scales, w_codes, w_scales, M, N, K, C, ld_c, vec_store, status);
+    return launch_status();
+}
+
+int gemm_tc_status(const void* workspace, cudaStream_t st) {
+    if (!workspace) return AMX_OK;
+    int v = 0;
+    if (cudaMemcpyAsync(&v, workspace, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return AMX_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return AMX_ERR_CUDA;
+    return v;
+}
 
 }  // namespace amx

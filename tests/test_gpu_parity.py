@@ -127,6 +127,47 @@ def test_gemm_simt_against_oracle(shape, gs):
     assert rel_fro(got, ref) <= 1e-5          # fp32 accumulation of <= 10-bit products is far tighter
 
 
+@pytest.mark.parametrize("shape", [(128, 256, 64), (128, 256, 256), (1, 1, 32), (130, 260, 96), (300, 520, 1056),
+                                   (256, 512, 4096)])
+def test_gemm_tensor_core_against_oracle(shape):
+    """tcgen05 path: one tile, several K blocks, a single group, ragged M/N/K tails, several tiles."""
+    M, N, K = shape
+    assert amx.lib().amx_gemm_kernel_for(M, N, K, 32, amx.GEMM_TC) == amx.GEMM_TC
+    a = inputs.random_groups(51, M, K, "mixed")
+    w = inputs.random_groups(52, N, K, "normal")
+    (ac, as_), (wc, ws) = oracle.quantize(a, 32), oracle.quantize(w, 32)
+    work = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    got = amx.gemm(*(torch.from_numpy(t).cuda() for t in (ac, as_, wc, ws)), 32, amx.GEMM_TC, workspace=work)
+    assert amx.gemm_status(work) == 0
+    got = got.cpu().numpy()
+    ref = oracle.gemm(ac, as_, wc, ws, 32)
+    for m in range(M):                         # row-wise: "mixed" rows differ by many orders of magnitude
+        if np.all(np.isfinite(ref[m])) and np.linalg.norm(ref[m]) > 0:
+            assert rel_fro(got[m], ref[m]) <= 1e-5, m
+
+
+def test_gemm_tensor_core_exact_on_small_integers():
+    rng = np.random.default_rng(9)
+    grid = np.array([0, 1, 2, 3, 4, 6], np.float32)
+    def ints(r, k):
+        t = grid[rng.integers(0, 6, size=(r, k))] * rng.choice([-1.0, 1.0], size=(r, k)).astype(np.float32)
+        t[:, ::32], t[:, 1::32] = 6.0, -6.0
+        return t
+    a, w = ints(200, 320), ints(300, 320)
+    qa, qw = oracle.quantize(inputs.f32_to_bf16_bits(a), 32), oracle.quantize(inputs.f32_to_bf16_bits(w), 32)
+    got = amx.gemm(*(torch.from_numpy(t).cuda() for t in (*qa, *qw)), 32, amx.GEMM_TC).cpu().numpy()
+    assert np.array_equal(got, (a.astype(np.int64) @ w.astype(np.int64).T).astype(np.float32))
+
+
+def test_gemm_tensor_core_matches_simt_at_scale():
+    a = dev_bf16(inputs.activation(2, 1))                 # 2048 x 4096
+    w = dev_bf16(inputs.weight(2, 1))                     # 4096 x 4096
+    (ac, as_), (wc, ws) = amx.quantize(a, 32), amx.quantize(w, 32)
+    tc = amx.gemm(ac, as_, wc, ws, 32, amx.GEMM_TC)
+    simt = amx.gemm(ac, as_, wc, ws, 32, amx.GEMM_SIMT)
+    assert rel_fro(tc.cpu().numpy(), simt.cpu().numpy()) <= 1e-5
+
+
 def test_gemm_wide_dynamic_range_rows():
     got, ref = _gemm_case(42, 96, 64, 256, 32, amx.GEMM_SIMT, "mixed")
     for m in range(96):                        # row-wise: rows differ by many orders of magnitude
