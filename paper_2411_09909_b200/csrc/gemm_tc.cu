@@ -310,11 +310,13 @@ size_t gemm_tc_workspace_bytes(int64_t, int64_t, int64_t) { return 256; }   // t
 
 int gemm_tc(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes, const uint8_t* w_scales,
             int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {
-    static bool configured = false;   // per process; the attribute is per function, not per device state we keep
-    if (!configured) {
+    static bool configured[64] = {};   // the opt-in to > 48 KB of dynamic shared memory is per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AMX_ERR_CUDA;
+    if (!configured[dev]) {
         if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
             return AMX_ERR_CUDA;
-        configured = true;
+        configured[dev] = true;
     }
     int* status = static_cast<int*>(workspace);
     if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return AMX_ERR_CUDA;
