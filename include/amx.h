@@ -45,7 +45,8 @@ typedef enum amx_status {
     AMX_ERR_FLAGS = -5,      /* unknown or contradictory flags */
     AMX_ERR_CUDA = -6,       /* a CUDA runtime call failed (launch or copy) */
     AMX_ERR_DEVICE = -7,     /* the device is not compute capability 10.x */
-    AMX_ERR_TIMEOUT = -8     /* a bounded device-side wait expired (reported by amx_gemm_status) */
+    AMX_ERR_TIMEOUT = -8,    /* a bounded device-side wait expired (reported by amx_gemm_status) */
+    AMX_ERR_TOO_LARGE = -9   /* the problem needs more scratch than a fixed-capacity entry point holds */
 } amx_status;
 
 /* flags for amx_dequantize: output element type (default bf16) */
@@ -139,6 +140,29 @@ int amx_softmax_bf16(const float* S, int64_t rows, int64_t cols, int64_t ld_s, f
 int amx_linear_host(const void* A_host, const void* W_host, int64_t M, int64_t N, int64_t K,
                     int group_size, uint32_t flags, float* C_host,
                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * amx_quant_gemm_static - amx_quant_gemm without a workspace argument, for callers that cannot
+ * allocate device memory: processes that gave the whole GPU to their own memory pool at start-up,
+ * plug-ins that must not touch the allocator, and latency-critical loops that cannot afford an
+ * allocation's implicit synchronisation.  (The paper has no counterpart; this is a deployment
+ * convenience of this library.)  Same arguments and result as amx_quant_gemm otherwise.
+ *   - The scratch (quantized activation + status word) is a fixed 16 MiB array that is part of the
+ *     library image: every GPU that loads the library holds it until the process exits.
+ *     amx_quant_gemm_static_capacity() returns its size; a problem for which
+ *     amx_quant_gemm_workspace_bytes() exceeds it is rejected with AMX_ERR_TOO_LARGE and nothing runs.
+ *   - The entry point calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - The first call on each device looks up the array's device address; make that first call
+ *     outside any stream capture.
+ *   - All calls share the one array, which keeps whatever the previous call left in it.  The
+ *     call itself re-initialises what it needs; but two calls whose work overlaps on the GPU
+ *     (different streams or host threads) race on the array - serialise them.
+ */
+int amx_quant_gemm_static(const void* A, int64_t ld_a,
+                          const uint8_t* w_codes, const uint8_t* w_scales,
+                          int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags,
+                          float* C, int64_t ld_c, void* stream);
+size_t amx_quant_gemm_static_capacity(void);
 
 /* Scratch sizes (bytes; 0 is possible).  Return 0 for invalid shapes. */
 size_t amx_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags);

@@ -24,6 +24,7 @@ SYMBOLS = (
     "amx_softmax_bf16", "amx_linear_host", "amx_workspace_bytes",
     "amx_quant_gemm_workspace_bytes", "amx_linear_host_workspace_bytes",
     "amx_gemm_kernel_for", "amx_gemm_status", "amx_status_string",
+    "amx_quant_gemm_static", "amx_quant_gemm_static_capacity",
 )
 
 
@@ -43,6 +44,9 @@ def lib() -> ctypes.CDLL:
         L.amx_dequantize.argtypes = [p, p, i64, i64, i, u32, p, i64, p]
         L.amx_gemm.argtypes = [p, p, p, p, i64, i64, i64, i, u32, p, i64, p, sz, p]
         L.amx_quant_gemm.argtypes = [p, i64, p, p, i64, i64, i64, i, u32, p, i64, p, sz, p]
+        L.amx_quant_gemm_static.argtypes = [p, i64, p, p, i64, i64, i64, i, u32, p, i64, p]
+        L.amx_quant_gemm_static_capacity.argtypes = []
+        L.amx_quant_gemm_static_capacity.restype = sz
         L.amx_softmax_bf16.argtypes = [p, i64, i64, i64, ctypes.c_float, p, i64, p]
         L.amx_linear_host.argtypes = [p, p, i64, i64, i64, i, u32, p, p, sz, p]
         for name in ("amx_workspace_bytes", "amx_quant_gemm_workspace_bytes"):

@@ -150,6 +150,7 @@ extern "C" const char* amx_status_string(int status) {
         case AMX_ERR_CUDA: return "CUDA runtime error";
         case AMX_ERR_DEVICE: return "device is not sm_100";
         case AMX_ERR_TIMEOUT: return "device-side wait timed out";
+        case AMX_ERR_TOO_LARGE: return "problem exceeds the fixed scratch capacity";
         default: return "unknown status";
     }
 }

@@ -33,8 +33,8 @@ def test_every_declared_symbol_is_exported(L):
 
 def test_status_strings(L):
     assert L.amx_status_string(0) == b"ok"
-    seen = {L.amx_status_string(c) for c in range(-8, 1)}
-    assert len(seen) == 9 and b"unknown status" not in seen
+    seen = {L.amx_status_string(c) for c in range(-9, 1)}
+    assert len(seen) == 10 and b"unknown status" not in seen
     assert L.amx_status_string(-99) == b"unknown status"
 
 
