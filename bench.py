@@ -174,6 +174,11 @@ def run_ours(args):
     L = amx.lib()
     peaks = measured_peaks()
     M, layers = layer_shapes()
+    keep = [int(t) for t in args.layers.split(",") if t != ""] or list(range(len(layers)))
+    layer_ids = keep
+    layers = [layers[i] for i in keep]
+    flops_step = sum(2.0 * M * N * K for K, N in layers)
+    elems_step = sum(M * K + N * K for K, N in layers)
 
     def to_dev(bits):
         return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
@@ -182,7 +187,7 @@ def run_ours(args):
     A, W, bufs = [], [], []
     host = []
     for li, (K, N) in enumerate(layers):
-        a_bits, w_bits = inputs.activation(CONFIG, li), inputs.weight(CONFIG, li)
+        a_bits, w_bits = inputs.activation(CONFIG, layer_ids[li]), inputs.weight(CONFIG, layer_ids[li])
         host.append((a_bits, w_bits))
         A.append(to_dev(a_bits))
         W.append(to_dev(w_bits))
@@ -252,7 +257,7 @@ def run_ours(args):
 
     # ---- end to end through the host-buffer entry point (pinned host tensors, copies inside the timing)
     e2e = None
-    if rank == 0 or world > 1:
+    if (rank == 0 or world > 1) and not args.skip_extras:
         pinned = []
         for li, (K, N) in enumerate(layers):
             a_bits, w_bits = host[li]
@@ -280,8 +285,8 @@ def run_ours(args):
             t = torch.tensor([e2e_s], device="cuda")
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             e2e_s = float(t.item())
-        e2e = {"value": world * total_flops() / e2e_s / 1e12, "unit": "TFLOP/s",
-               "h2d_bytes_per_step": int(quantized_elements() * 2),
+        e2e = {"value": world * flops_step / e2e_s / 1e12, "unit": "TFLOP/s",
+               "h2d_bytes_per_step": int(elems_step * 2),
                "d2h_bytes_per_step": int(sum(M * N * 4 for _, N in layers)),
                "ms_per_step": e2e_s * 1e3}
 
@@ -292,9 +297,9 @@ def run_ours(args):
         return
 
     ms_per_step = elapsed_ms / args.steps
-    value = world * total_flops() / (ms_per_step * 1e-3) / 1e12
-    gemm_tflops = args.steps * total_flops() / (g_ms * 1e-3) / 1e12
-    quant_gbs = args.steps * quantized_elements() * BYTES_PER_ELEM / (q_ms * 1e-3) / 1e9
+    value = world * flops_step / (ms_per_step * 1e-3) / 1e12
+    gemm_tflops = args.steps * flops_step / (g_ms * 1e-3) / 1e12
+    quant_gbs = args.steps * elems_step * BYTES_PER_ELEM / (q_ms * 1e-3) / 1e9
     fp4_peak = 4.0 * peaks["bf16_tflops_sustained"]
     line = {
         "metric": "AMXFP4 quant+GEMM TFLOPS", "value": value, "unit": "TFLOP/s", "n_gpus": world,
@@ -320,7 +325,9 @@ def run_ours(args):
         "e2e": e2e,
         "gpu_launches": 3 * len(layers) * args.steps,
     }
-    if world == 1:
+    if len(layer_ids) != 4:
+        line["config"]["layers"] = layer_ids
+    if world == 1 and not args.skip_extras:
         line["cpu_baseline"] = cpu_baseline()
     print(json.dumps(line))
     if world > 1:
@@ -334,6 +341,8 @@ def main():
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", default="", help="comma-separated layer indices to run (profiling aid; default all)")
+    ap.add_argument("--skip-extras", action="store_true", help="skip the e2e and cpu_baseline legs (profiling aid)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
