@@ -68,7 +68,7 @@ typedef enum amx_status {
  *   magnitude  = E2M1 nearest (ties to even) to |x| / scale_side, clamped at 6 (0 if the scale is 0);
  *   the sign bit of a code is the sign bit of x.
  *   x       bf16 [rows, ld_x] row-major, ld_x >= K in elements; 16-byte aligned, ld_x % 8 == 0
- *   codes   out, [rows, K/2], 4-byte aligned
+ *   codes   out, [rows, K/2], 16-byte aligned (8-byte for gs = 16)
  *   scales  out, [rows, K/gs, 2], 2-byte aligned
  * K % 8 == 0 is required.  rows == 0 is a no-op.
  */

@@ -21,7 +21,6 @@ namespace amx {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kUnroll = 4;  // independent 16-byte loads in flight per thread
 
 // 1/6 rounded up a few ulps (0x3E2AAAAB is the nearest float, already above 1/6).
 __device__ __forceinline__ float sixth_up() { return __uint_as_float(0x3E2AAAAFu); }
@@ -61,27 +60,40 @@ __device__ __forceinline__ float inv_scale_up(float s) {
     return s > 0.0f ? r : 0.0f;
 }
 
-// Quantizes 8 consecutive elements held as 4 bf16x2 words.  `width` threads (8*width = group
-// size) hold one group and sit in consecutive lanes.  Returns the 8 nibbles; `sc` receives the
-// two scale bytes (positive side in bits 7..0, negative side in bits 15..8).
-template <int TPG>
-__device__ __forceinline__ uint32_t quantize8(const uint4 q, uint32_t& sc) {
-    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-    // per-halfword maxima: positive side on the raw bits, negative side on sign-flipped bits
-    uint32_t pm = __vimax3_s16x2_relu(w[0], w[1], __vmaxs2(w[2], w[3]));
-    uint32_t nm = __vimax3_s16x2_relu(w[0] ^ 0x80008000u, w[1] ^ 0x80008000u,
-                                      __vmaxs2(w[2] ^ 0x80008000u, w[3] ^ 0x80008000u));
-    // fold the two halfwords: result = {nmax bits : pmax bits}
-    uint32_t c = __vmaxs2(__byte_perm(pm, nm, 0x5410), __byte_perm(pm, nm, 0x7632));
+// Side maxima of NW bf16x2 words as one word {nmax bits : pmax bits}.  Signed 16-bit max over the
+// raw patterns, clamped at 0, is the largest non-negative value; unsigned 16-bit max is the negative
+// value of largest magnitude whenever a negative one exists (its sign bit is then flipped away).
+template <int NW>
+__device__ __forceinline__ uint32_t side_maxima(const uint32_t (&w)[NW]) {
+    uint32_t pm = w[0], nm = w[0];
 #pragma unroll
-    for (int d = 1; d < TPG; d <<= 1) c = __vmaxs2(c, __shfl_xor_sync(0xFFFFFFFFu, c, d));
+    for (int i = 1; i + 1 < NW; i += 2) {
+        pm = __vimax3_s16x2(pm, w[i], w[i + 1]);
+        nm = __vimax3_u16x2(nm, w[i], w[i + 1]);
+    }
+    if (NW % 2 == 0) {
+        pm = __vmaxs2(pm, w[NW - 1]);
+        nm = __vmaxu2(nm, w[NW - 1]);
+    }
+    nm ^= 0x80008000u;
+    pm = __vimax_s16x2_relu(pm, pm);
+    nm = __vimax_s16x2_relu(nm, nm);
+    return __vmaxs2(__byte_perm(pm, nm, 0x5410), __byte_perm(pm, nm, 0x7632));
+}
 
+// The two E5M2 scale bytes of a group from its side maxima {nmax : pmax} (positive side in bits
+// 7..0, negative side in bits 15..8), and the two biased reciprocals the elements are multiplied by.
+__device__ __forceinline__ uint32_t group_scales(uint32_t c, float& inv_p, float& inv_n) {
     const float pmax = __uint_as_float(c << 16);
     const float nmax = __uint_as_float(c & 0xFFFF0000u);
-    sc = cvt_e5m2x2(trunc12(nmax * sixth_up()), trunc12(pmax * sixth_up()));
-    const float inv_p = inv_scale_up(e5m2_to_float(sc & 0xFFu));
-    const float inv_n = inv_scale_up(e5m2_to_float(sc >> 8));
+    const uint32_t sc = cvt_e5m2x2(trunc12(nmax * sixth_up()), trunc12(pmax * sixth_up()));
+    inv_p = inv_scale_up(e5m2_to_float(sc & 0xFFu));
+    inv_n = inv_scale_up(e5m2_to_float(sc >> 8));
+    return sc;
+}
 
+// 8 consecutive elements (4 bf16x2 words) -> 8 nibbles.
+__device__ __forceinline__ uint32_t encode8(const uint32_t* w, float inv_p, float inv_n) {
     float r[8];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -93,32 +105,52 @@ __device__ __forceinline__ uint32_t quantize8(const uint4 q, uint32_t& sc) {
     return cvt_e2m1x8(r);
 }
 
-// Groups along the contiguous axis.  One thread per 8 elements; n_vec = rows * K / 8.
-template <int TPG, bool CONTIG>
+// Quantizes 8 consecutive elements held as 4 bf16x2 words.  TPG threads (8*TPG = group size) hold
+// one group and sit in consecutive lanes.  Returns the 8 nibbles; `sc` receives the scale bytes.
+template <int TPG>
+__device__ __forceinline__ uint32_t quantize8(const uint4 q, uint32_t& sc) {
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+    uint32_t c = side_maxima<4>(w);
+#pragma unroll
+    for (int d = 1; d < TPG; d <<= 1) c = __vmaxs2(c, __shfl_xor_sync(0xFFFFFFFFu, c, d));
+    float inv_p, inv_n;
+    sc = group_scales(c, inv_p, inv_n);
+    return encode8(w, inv_p, inv_n);
+}
+
+// Groups along the contiguous axis.  Each thread owns EPT = min(gs, 32) consecutive elements
+// (EPT/8 16-byte loads, one EPT/2-byte store); a group is TPG = gs / EPT consecutive lanes, so a
+// 16- or 32-group needs no shuffle and its scales are computed once.  n_items = rows * K / EPT.
+template <int EPT, int TPG, bool CONTIG>
 __global__ void __launch_bounds__(kThreads)
-quantize_rows_kernel(const uint4* __restrict__ x, int64_t n_vec, int64_t vec_per_row,
-                     int64_t ld_vec, uint32_t* __restrict__ codes, uint16_t* __restrict__ scales) {
-    const int64_t base = (int64_t)blockIdx.x * (kThreads * kUnroll) + threadIdx.x;
-    uint4 q[kUnroll];
+quantize_rows_kernel(const uint4* __restrict__ x, int64_t n_items, int64_t items_per_row,
+                     int64_t ld_vec, uint4* __restrict__ codes, uint16_t* __restrict__ scales) {
+    constexpr int NV = EPT / 8;
+    const int64_t v = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    uint32_t w[NV * 4];
+    const bool live = v < n_items;
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-        const int64_t v = base + (int64_t)u * kThreads;
-        q[u] = make_uint4(0, 0, 0, 0);
-        if (v < n_vec) {
-            int64_t off = v;
-            if (!CONTIG) off = (v / vec_per_row) * ld_vec + (v % vec_per_row);
-            q[u] = __ldcs(x + off);
+    for (int j = 0; j < NV; ++j) {
+        uint4 q = make_uint4(0, 0, 0, 0);
+        if (live) {
+            int64_t off = v * NV + j;
+            if (!CONTIG) off = (v / items_per_row) * ld_vec + (v % items_per_row) * NV + j;
+            q = __ldg(x + off);
         }
+        w[4 * j] = q.x; w[4 * j + 1] = q.y; w[4 * j + 2] = q.z; w[4 * j + 3] = q.w;
     }
+    uint32_t c = side_maxima<NV * 4>(w);
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-        const int64_t v = base + (int64_t)u * kThreads;
-        uint32_t sc;
-        const uint32_t nib = quantize8<TPG>(q[u], sc);
-        if (v < n_vec) {
-            codes[v] = nib;
-            if ((threadIdx.x & (TPG - 1)) == 0) scales[v / TPG] = (uint16_t)sc;
-        }
+    for (int d = 1; d < TPG; d <<= 1) c = __vmaxs2(c, __shfl_xor_sync(0xFFFFFFFFu, c, d));
+    float inv_p, inv_n;
+    const uint32_t sc = group_scales(c, inv_p, inv_n);
+    uint32_t nib[NV];
+#pragma unroll
+    for (int j = 0; j < NV; ++j) nib[j] = encode8(w + 4 * j, inv_p, inv_n);
+    if (live) {
+        if (NV == 4) codes[v] = make_uint4(nib[0], nib[1], nib[2], nib[NV - 1]);
+        else *reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(codes) + v * 8) = make_uint2(nib[0], nib[NV - 1]);
+        if ((threadIdx.x & (TPG - 1)) == 0) scales[v / TPG] = (uint16_t)sc;
     }
 }
 
@@ -160,20 +192,19 @@ quantize_cols_kernel(const __nv_bfloat16* __restrict__ x, int64_t R, int64_t C, 
     }
 }
 
-template <int TPG>
+template <int EPT, int TPG>
 int launch_rows(const void* x, int64_t rows, int64_t K, int64_t ld, uint8_t* codes,
                 uint8_t* scales, cudaStream_t st) {
-    const int64_t n_vec = rows * (K / 8);
-    const int64_t per_block = (int64_t)kThreads * kUnroll;
-    const int64_t blocks = (n_vec + per_block - 1) / per_block;
+    const int64_t n_items = rows * (K / EPT);
+    const int64_t blocks = (n_items + kThreads - 1) / kThreads;
     if (blocks > 0x7FFFFFFF) return AMX_ERR_SHAPE;
     auto* xv = reinterpret_cast<const uint4*>(x);
-    auto* cv = reinterpret_cast<uint32_t*>(codes);
+    auto* cv = reinterpret_cast<uint4*>(codes);
     auto* sv = reinterpret_cast<uint16_t*>(scales);
     if (ld == K)
-        quantize_rows_kernel<TPG, true><<<(unsigned)blocks, kThreads, 0, st>>>(xv, n_vec, K / 8, ld / 8, cv, sv);
+        quantize_rows_kernel<EPT, TPG, true><<<(unsigned)blocks, kThreads, 0, st>>>(xv, n_items, K / EPT, ld / 8, cv, sv);
     else
-        quantize_rows_kernel<TPG, false><<<(unsigned)blocks, kThreads, 0, st>>>(xv, n_vec, K / 8, ld / 8, cv, sv);
+        quantize_rows_kernel<EPT, TPG, false><<<(unsigned)blocks, kThreads, 0, st>>>(xv, n_items, K / EPT, ld / 8, cv, sv);
     return launch_status();
 }
 
@@ -198,13 +229,13 @@ extern "C" int amx_quantize(const void* x, int64_t rows, int64_t K, int64_t ld_x
         return AMX_ERR_SHAPE;
     if (rows == 0) return AMX_OK;
     if (!x || !codes || !scales) return AMX_ERR_NULL;
-    if (!aligned(x, 16) || ld_x % 8 || !aligned(codes, 4) || !aligned(scales, 2)) return AMX_ERR_ALIGN;
+    if (!aligned(x, 16) || ld_x % 8 || !aligned(codes, group_size == 16 ? 8 : 16) || !aligned(scales, 2)) return AMX_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     switch (group_size) {
-        case 16: return launch_rows<2>(x, rows, K, ld_x, codes, scales, st);
-        case 32: return launch_rows<4>(x, rows, K, ld_x, codes, scales, st);
-        case 64: return launch_rows<8>(x, rows, K, ld_x, codes, scales, st);
-        default: return launch_rows<16>(x, rows, K, ld_x, codes, scales, st);
+        case 16: return launch_rows<16, 1>(x, rows, K, ld_x, codes, scales, st);
+        case 32: return launch_rows<32, 1>(x, rows, K, ld_x, codes, scales, st);
+        case 64: return launch_rows<32, 2>(x, rows, K, ld_x, codes, scales, st);
+        default: return launch_rows<32, 4>(x, rows, K, ld_x, codes, scales, st);
     }
 }
 
