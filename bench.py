@@ -255,6 +255,30 @@ def run_ours(args):
     q_ms = sum(a.elapsed_time(b) for a, b in ev_q)
     g_ms = sum(a.elapsed_time(b) for a, b in ev_g)
 
+    # ---- the cast alone on a tensor larger than L2 (config-4 activation shape, 16384 x 8192 = 268 MB of bf16)
+    quant_large = None
+    if not args.layers:
+        qr, qk = 16384, 8192
+        xq = to_dev(inputs.activation(4, 0, M=256)).repeat(qr // 256, 1).contiguous()
+        qc = torch.empty((qr, qk // 2), dtype=torch.uint8, device="cuda")
+        qs = torch.empty((qr, qk // GS, 2), dtype=torch.uint8, device="cuda")
+        for _ in range(3):
+            check(L.amx_quantize(xq.data_ptr(), qr, qk, qk, GS, qc.data_ptr(), qs.data_ptr(), stream))
+        q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        q_iters = 20
+        torch.cuda.synchronize()
+        q0.record()
+        for _ in range(q_iters):
+            check(L.amx_quantize(xq.data_ptr(), qr, qk, qk, GS, qc.data_ptr(), qs.data_ptr(), stream))
+        q1.record()
+        torch.cuda.synchronize()
+        q_us = q0.elapsed_time(q1) * 1e3 / q_iters
+        gbs = qr * qk * BYTES_PER_ELEM / (q_us * 1e-6) / 1e9
+        quant_large = {"shape": [qr, qk], "us": q_us, "gb_per_s": gbs,
+                       "pct_of_nominal_hbm_8TBs": 100.0 * gbs / NOMINAL_HBM_GBS,
+                       "frac_of_measured_copy": gbs / peaks["hbm_gbs"]}
+        del xq, qc, qs
+
     # ---- end to end through the host-buffer entry point (pinned host tensors, copies inside the timing)
     e2e = None
     if (rank == 0 or world > 1) and not args.skip_extras:
@@ -314,7 +338,7 @@ def run_ours(args):
         "nominal_fp4_peak_tflops": NOMINAL_FP4_TFLOPS,
         "quantize": {"gb_per_s": quant_gbs, "pct_of_nominal_hbm_8TBs": 100.0 * quant_gbs / NOMINAL_HBM_GBS,
                      "frac_of_measured_copy": quant_gbs / peaks["hbm_gbs"], "bytes_per_element": BYTES_PER_ELEM,
-                     "ms_per_step": q_ms / args.steps},
+                     "ms_per_step": q_ms / args.steps, "large_tensor": quant_large},
         "gemm": {"useful_tflops": gemm_tflops, "ms_per_step": g_ms / args.steps,
                  "pct_of_nominal_fp4_peak": 100.0 * gemm_tflops / NOMINAL_FP4_TFLOPS},
         "roofline": {"bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",

@@ -92,15 +92,23 @@ __device__ __forceinline__ uint32_t group_scales(uint32_t c, float& inv_p, float
     return sc;
 }
 
+// x * (sign(x) ? inv_n : inv_p).  The choice is an integer multiply-add on the reciprocals' bit
+// patterns (inv_p + sign * (inv_n - inv_p)): it runs on the FMA pipe, which this kernel leaves
+// mostly idle, instead of adding a compare and a select to the saturated integer/logic pipe.
+__device__ __forceinline__ float scale_by_side(uint32_t x_bits, uint32_t inv_p, uint32_t inv_diff) {
+    uint32_t sel;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(sel) : "r"(x_bits >> 31), "r"(inv_diff), "r"(inv_p));
+    return __uint_as_float(x_bits) * __uint_as_float(sel);
+}
+
 // 8 consecutive elements (4 bf16x2 words) -> 8 nibbles.
 __device__ __forceinline__ uint32_t encode8(const uint32_t* w, float inv_p, float inv_n) {
+    const uint32_t ip = __float_as_uint(inv_p), idiff = __float_as_uint(inv_n) - ip;
     float r[8];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        const float lo = __uint_as_float(w[i] << 16);
-        const float hi = __uint_as_float(w[i] & 0xFFFF0000u);
-        r[2 * i] = trunc12(lo * ((int)__float_as_uint(lo) < 0 ? inv_n : inv_p));
-        r[2 * i + 1] = trunc12(hi * ((int)w[i] < 0 ? inv_n : inv_p));
+        r[2 * i] = trunc12(scale_by_side(w[i] << 16, ip, idiff));
+        r[2 * i + 1] = trunc12(scale_by_side(w[i] & 0xFFFF0000u, ip, idiff));
     }
     return cvt_e2m1x8(r);
 }
