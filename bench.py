@@ -174,6 +174,7 @@ def run_ours(args):
     L = amx.lib()
     peaks = measured_peaks()
     M, layers = layer_shapes()
+    gemm_flag = {"auto": 0, "simt": 0x10, "tc": 0x20, "fp4": 0x40}[args.gemm]
     keep = [int(t) for t in args.layers.split(",") if t != ""] or list(range(len(layers)))
     layer_ids = keep
     layers = [layers[i] for i in keep]
@@ -191,7 +192,7 @@ def run_ours(args):
         host.append((a_bits, w_bits))
         A.append(to_dev(a_bits))
         W.append(to_dev(w_bits))
-        ws_bytes = max(L.amx_workspace_bytes(M, N, K, GS, 0), 256)
+        ws_bytes = max(L.amx_workspace_bytes(M, N, K, GS, gemm_flag), 256)
         bufs.append({
             "ac": torch.empty((M, K // 2), dtype=torch.uint8, device="cuda"),
             "as": torch.empty((M, K // GS, 2), dtype=torch.uint8, device="cuda"),
@@ -201,7 +202,8 @@ def run_ours(args):
             "work": torch.empty(ws_bytes, dtype=torch.uint8, device="cuda"),
         })
     stream = torch.cuda.current_stream().cuda_stream
-    gemm_kernel = {0x10: "simt", 0x20: "tcgen05"}[L.amx_gemm_kernel_for(M, layers[0][1], layers[0][0], GS, 0)]
+    gemm_kernel = {0x10: "simt", 0x20: "tcgen05 kind::f16 (bf16 decode)", 0x40: "tcgen05 kind::mxf4nvf4 (sign split)"}[
+        L.amx_gemm_kernel_for(M, layers[0][1], layers[0][0], GS, gemm_flag)]
 
     def check(rc):
         if rc != 0:
@@ -220,7 +222,8 @@ def run_ours(args):
             if record:
                 e1.record()
             check(L.amx_gemm(b["ac"].data_ptr(), b["as"].data_ptr(), b["wc"].data_ptr(), b["ws"].data_ptr(),
-                             M, N, K, GS, 0, b["c"].data_ptr(), N, b["work"].data_ptr(), b["work"].numel(), stream))
+                             M, N, K, GS, gemm_flag, b["c"].data_ptr(), N, b["work"].data_ptr(), b["work"].numel(),
+                             stream))
             if record:
                 e2.record()
                 ev_q.append((e0, e1))
@@ -365,6 +368,7 @@ def main():
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--gemm", default="auto", choices=["auto", "simt", "tc", "fp4"], help="GEMM kernel to time")
     ap.add_argument("--layers", default="", help="comma-separated layer indices to run (profiling aid; default all)")
     ap.add_argument("--skip-extras", action="store_true", help="skip the e2e and cpu_baseline legs (profiling aid)")
     args = ap.parse_args()

@@ -56,7 +56,11 @@ typedef enum amx_status {
  * shape allows it, else the SIMT path) */
 #define AMX_GEMM_AUTO 0x0u
 #define AMX_GEMM_SIMT 0x10u  /* plain CUDA-core kernel: any shape, any supported gs */
-#define AMX_GEMM_TC 0x20u    /* tcgen05 kernel only: AMX_ERR_SHAPE if the shape does not fit */
+#define AMX_GEMM_TC 0x20u    /* tcgen05 kernel, exact bf16 decode: AMX_ERR_SHAPE if the shape does not fit */
+#define AMX_GEMM_FP4 0x40u   /* tcgen05 block-scaled FP4 kernel (four sign-pair MMAs per tile).  Scales more
+                              * than 14 binades below the largest scale of their operand row are flushed to
+                              * zero (relative effect < 2^-14 per row); otherwise same result up to fp32
+                              * summation order.  Needs the larger workspace amx_workspace_bytes() reports. */
 
 /*
  * amx_quantize - direct cast of a bf16 matrix to AMXFP4 (Sections 4.2-4.3; procedure per

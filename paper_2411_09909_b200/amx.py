@@ -16,7 +16,7 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libamx_b20
 _lib = None
 
 OUT_BF16, OUT_F32 = 0x0, 0x1
-GEMM_AUTO, GEMM_SIMT, GEMM_TC = 0x0, 0x10, 0x20
+GEMM_AUTO, GEMM_SIMT, GEMM_TC, GEMM_FP4 = 0x0, 0x10, 0x20, 0x40
 
 # every symbol include/amx.h declares
 SYMBOLS = (

@@ -12,14 +12,23 @@ bool gemm_shape_ok(int64_t M, int64_t N, int64_t K, int gs) {
     return valid_group_size(gs) && M >= 0 && N >= 0 && K > 0 && K % gs == 0 && K % 8 == 0;
 }
 
-// AMX_GEMM_SIMT / AMX_GEMM_TC, or 0 when the flags cannot be honoured for this shape.
+constexpr uint32_t kKernelMask = AMX_GEMM_SIMT | AMX_GEMM_TC | AMX_GEMM_FP4;
+
+// The kernel to run (one AMX_GEMM_* bit), or 0 when the flags cannot be honoured for this shape.
 uint32_t pick_kernel(int64_t M, int64_t N, int64_t K, int gs, uint32_t flags) {
-    const uint32_t want = flags & (AMX_GEMM_SIMT | AMX_GEMM_TC);
-    if (want == (AMX_GEMM_SIMT | AMX_GEMM_TC)) return 0;
+    const uint32_t want = flags & kKernelMask;
+    if (want & (want - 1)) return 0;                                   // more than one kernel asked for
+    if (want == AMX_GEMM_FP4) return gemm_fp4_supported(M, N, K, gs) ? AMX_GEMM_FP4 : 0;
     const bool tc = gemm_tc_supported(M, N, K, gs);
     if (want == AMX_GEMM_TC) return tc ? AMX_GEMM_TC : 0;
     if (want == AMX_GEMM_SIMT) return AMX_GEMM_SIMT;
     return tc ? AMX_GEMM_TC : AMX_GEMM_SIMT;
+}
+
+size_t kernel_workspace(uint32_t kernel, int64_t M, int64_t N, int64_t K) {
+    if (kernel == AMX_GEMM_TC) return round_up(gemm_tc_workspace_bytes(M, N, K));
+    if (kernel == AMX_GEMM_FP4) return round_up(gemm_fp4_workspace_bytes(M, N, K));
+    return 0;
 }
 
 struct QuantSizes {
@@ -41,7 +50,7 @@ extern "C" uint32_t amx_gemm_kernel_for(int64_t M, int64_t N, int64_t K, int gro
 
 extern "C" size_t amx_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags) {
     if (!gemm_shape_ok(M, N, K, group_size)) return 0;
-    return pick_kernel(M, N, K, group_size, flags) == AMX_GEMM_TC ? round_up(gemm_tc_workspace_bytes(M, N, K)) : 0;
+    return kernel_workspace(pick_kernel(M, N, K, group_size, flags), M, N, K);
 }
 
 extern "C" size_t amx_quant_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags) {
@@ -61,10 +70,10 @@ extern "C" int amx_gemm(const uint8_t* a_codes, const uint8_t* a_scales, const u
                         const uint8_t* w_scales, int64_t M, int64_t N, int64_t K, int group_size,
                         uint32_t flags, float* C, int64_t ld_c, void* workspace, size_t workspace_bytes,
                         void* stream) {
-    if (flags & ~(AMX_GEMM_SIMT | AMX_GEMM_TC)) return AMX_ERR_FLAGS;
+    if (flags & ~kKernelMask) return AMX_ERR_FLAGS;
     if (!gemm_shape_ok(M, N, K, group_size) || ld_c < N) return AMX_ERR_SHAPE;
     uint32_t kernel = pick_kernel(M, N, K, group_size, flags);
-    if (!kernel) return (flags & AMX_GEMM_SIMT) ? AMX_ERR_FLAGS : AMX_ERR_SHAPE;
+    if (!kernel) return ((flags & kKernelMask) & ((flags & kKernelMask) - 1)) ? AMX_ERR_FLAGS : AMX_ERR_SHAPE;
     if (M == 0 || N == 0) return AMX_OK;
     if (!a_codes || !a_scales || !w_codes || !w_scales || !C) return AMX_ERR_NULL;
     if (!aligned(a_codes, 4) || !aligned(w_codes, 4) || !aligned(a_scales, 2) || !aligned(w_scales, 2) ||
@@ -74,16 +83,18 @@ extern "C" int amx_gemm(const uint8_t* a_codes, const uint8_t* a_scales, const u
     if (kernel == AMX_GEMM_SIMT)
         return gemm_simt(a_codes, a_scales, w_codes, w_scales, M, N, K, group_size, C, ld_c, st);
     if (!aligned(a_codes, 16) || !aligned(w_codes, 16)) return AMX_ERR_ALIGN;
-    const size_t need = round_up(gemm_tc_workspace_bytes(M, N, K));
+    const size_t need = kernel_workspace(kernel, M, N, K);
     if (need && (!workspace || workspace_bytes < need)) return AMX_ERR_WORKSPACE;
     if (need && !aligned(workspace, kAlign)) return AMX_ERR_ALIGN;
+    if (kernel == AMX_GEMM_FP4)
+        return gemm_fp4(a_codes, a_scales, w_codes, w_scales, M, N, K, C, ld_c, workspace, st);
     return gemm_tc(a_codes, a_scales, w_codes, w_scales, M, N, K, C, ld_c, workspace, st);
 }
 
 extern "C" int amx_quant_gemm(const void* A, int64_t ld_a, const uint8_t* w_codes, const uint8_t* w_scales,
                               int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags, float* C,
                               int64_t ld_c, void* workspace, size_t workspace_bytes, void* stream) {
-    if (flags & ~(AMX_GEMM_SIMT | AMX_GEMM_TC)) return AMX_ERR_FLAGS;
+    if (flags & ~kKernelMask) return AMX_ERR_FLAGS;
     if (!gemm_shape_ok(M, N, K, group_size) || ld_a < K || ld_c < N) return AMX_ERR_SHAPE;
     if (M == 0 || N == 0) return AMX_OK;
     const size_t need = amx_quant_gemm_workspace_bytes(M, N, K, group_size, flags);
@@ -102,7 +113,7 @@ extern "C" int amx_quant_gemm(const void* A, int64_t ld_a, const uint8_t* w_code
 extern "C" int amx_linear_host(const void* A_host, const void* W_host, int64_t M, int64_t N, int64_t K,
                                int group_size, uint32_t flags, float* C_host, void* workspace,
                                size_t workspace_bytes, void* stream) {
-    if (flags & ~(AMX_GEMM_SIMT | AMX_GEMM_TC)) return AMX_ERR_FLAGS;
+    if (flags & ~kKernelMask) return AMX_ERR_FLAGS;
     if (!gemm_shape_ok(M, N, K, group_size)) return AMX_ERR_SHAPE;
     if (M == 0 || N == 0) return AMX_OK;
     if (!A_host || !W_host || !C_host) return AMX_ERR_NULL;

@@ -17,4 +17,12 @@ int gemm_tc(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_co
             void* workspace, cudaStream_t st);
 int gemm_tc_status(const void* workspace, cudaStream_t st);
 
+// FP4-pipe kernel (four block-scaled MMAs per tile pair): same contract; the workspace also holds
+// the prepared operands (sign planes, UE4M3 scale-factor blocks, row offsets).
+bool gemm_fp4_supported(int64_t M, int64_t N, int64_t K, int gs);
+size_t gemm_fp4_workspace_bytes(int64_t M, int64_t N, int64_t K);
+int gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes,
+             const uint8_t* w_scales, int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c,
+             void* workspace, cudaStream_t st);
+
 }  // namespace amx

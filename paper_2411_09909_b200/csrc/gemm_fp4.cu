@@ -1,0 +1,403 @@
+// AMXFP4 x AMXFP4 -> fp32 on the FP4 tensor-core pipe (tcgen05 block-scaled MMA, sm_100a).
+//
+// The format picks one of two group scales per ELEMENT (by the element's sign; arXiv 2411.09909,
+// Section 4.3), while a block-scaled MMA operand has one scale per (row, K block).  So each decoded
+// operand is written as the sum of two single-scale operands,
+//     Ahat = S_p o A+  +  S_n o A-      (A+ / A- = the codes with the other sign's nibbles zeroed),
+// and the product becomes four block-scaled FP4 MMAs accumulating into one TMEM tile:
+//     Ahat What^T = A+ W+^T + A+ W-^T + A- W+^T + A- W-^T.
+//
+// Scales: the MMA takes UE4M3 scales, one per 16 elements.  An E5M2 scale has the same four
+// significands but a wider exponent range, so every operand row gets a power-of-two offset that
+// maps its largest scale to the top UE4M3 binade; scale * 2^-offset is written as UE4M3 (each
+// 32-group's scale twice) and the fp32 accumulator is multiplied by 2^(offset_A[m] + offset_W[n])
+// in the epilogue (exact).  Scales more than 14 binades below their row's largest scale do not fit
+// and are flushed to zero: their groups contribute less than 2^-14 of the row's largest group.
+//
+// Pipeline per CTA (128 x 256 tile of C, 256-element K blocks, two stages of 108 KB):
+//   warp 0   TMA producer: four 128-byte-swizzled code tiles (A+, A-, W+, W-) and the scale-factor
+//            blocks (plain bulk copies) per stage, completion on the stage's `full` mbarrier
+//   warp 1   allocates TMEM; one lane copies the stage's scale factors shared -> tensor memory
+//            (tcgen05.cp) and issues 16 MMAs (4 sign pairs x 4 K steps of 64), then commits to the
+//            stage's `empty` mbarrier
+//   warps 2-5  epilogue: TMEM -> registers, power-of-two rescale, fp32 stores
+// A preparation pass (two small kernels per operand) derives the planes, the UE4M3 scale-factor
+// blocks in the 128 x 4 interleaved layout the MMA reads, and the row offsets from the canonical
+// codes and scales.  Every device-side wait is bounded.
+#include <cuda.h>
+
+#include <mutex>
+
+#include "gemm.cuh"
+#include "tcgen05.cuh"
+
+namespace amx {
+namespace {
+
+using namespace tc;
+
+constexpr int BM = 128, BN = 256;
+constexpr int BK = 256;                 // elements per K block = 128 bytes of codes per row
+constexpr int kRowBytes = BK / 2;
+constexpr int kStages = 2;
+constexpr int kThreads = 192;
+constexpr int kTileA = BM * kRowBytes, kTileB = BN * kRowBytes;       // one plane
+constexpr int kSfChunk = 512;           // scale factors of 128 rows x 64 elements (4 per row)
+constexpr int kSfA = 4 * kSfChunk;      // one plane, one K block, 128 rows
+constexpr int kSfB = 2 * kSfA;          // 256 rows
+constexpr int kOffAp = 0, kOffAn = kTileA, kOffWp = 2 * kTileA, kOffWn = 2 * kTileA + kTileB;
+constexpr int kOffSfA = 2 * kTileA + 2 * kTileB, kOffSfB = kOffSfA + 2 * kSfA;
+constexpr int kStageBytes = kOffSfB + 2 * kSfB;                       // 110592
+constexpr int kTmemCols = 512;
+constexpr uint32_t kTmemSfA = 256, kTmemSfB = 256 + 32;               // after the 256 accumulator columns
+
+struct __align__(8) Control {
+    uint64_t full[kStages], empty[kStages], accum;
+    uint32_t tmem_base;
+    volatile int abort;
+    int w_exp[BN];
+};
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 + sizeof(Control);
+
+// Instruction descriptor, kind::mxf4nvf4 block-scaled: A and B E2M1 (format code 1), K-major,
+// UE4M3 scale factors (bit 23 = 0), N >> 3 at bit 17, M >> 4 at bit 24, K = 64 (bit 31 = 0).
+constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+// ------------------------------------------------------------------------- preparation --
+// Sign planes: nibble kept where its sign bit matches the plane, zero elsewhere.
+__global__ void __launch_bounds__(256)
+split_planes_kernel(const uint4* __restrict__ codes, int64_t n_vec, uint4* __restrict__ pos, uint4* __restrict__ neg) {
+    const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (i >= n_vec) return;
+    const uint4 w = __ldg(codes + i);
+    const uint32_t v[4] = {w.x, w.y, w.z, w.w};
+    uint32_t p[4], n[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint32_t m = ((v[j] >> 3) & 0x11111111u) * 15u;   // 0xF on negative nibbles
+        n[j] = v[j] & m;
+        p[j] = v[j] & ~m;
+    }
+    pos[i] = make_uint4(p[0], p[1], p[2], p[3]);
+    neg[i] = make_uint4(n[0], n[1], n[2], n[3]);
+}
+
+// Exponent key of an E5M2 scale byte: unbiased exponent + 17 (1 for 2^-16), 0 for a zero scale.
+__device__ __forceinline__ int scale_key(uint32_t b) {
+    const int e = (b >> 2) & 31, m = b & 3;
+    return e ? e + 2 : (m == 0 ? 0 : (m == 1 ? 1 : 2));
+}
+// UE4M3 byte of the E5M2 byte b for a row whose largest key is kmax (0 when it does not fit).
+__device__ __forceinline__ uint32_t to_ue4m3(uint32_t b, int kmax) {
+    const int e = (b >> 2) & 31, m = b & 3;
+    const int f = scale_key(b) - kmax + 15;                      // UE4M3 exponent field
+    const int mant = e ? m : (m == 3 ? 2 : 0);                   // subnormals: 1, 2, 3 x 2^-16
+    return (f >= 1 && scale_key(b) > 0) ? (uint32_t)((f << 3) | (mant << 1)) : 0u;
+}
+
+// One block per 128 operand rows: row offsets, then the scale-factor blocks of both planes.
+// sf layout: [plane][row block][K/64 block][512 B], byte (r%32)*16 + (r/32)*4 + (k16 % 4).
+__global__ void __launch_bounds__(256)
+scale_factors_kernel(const uint8_t* __restrict__ scales, int64_t R, int64_t G /*groups per row*/, int nk64,
+                     uint8_t* __restrict__ sf_pos, uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp) {
+    __shared__ int kmax_s[128];
+    const int64_t rb = blockIdx.x, row0 = rb * 128;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int r = warp; r < 128; r += 8) {
+        const int64_t row = row0 + r;
+        int kmax = 0;
+        if (row < R) {
+            const unsigned short* s2 = reinterpret_cast<const unsigned short*>(scales + row * G * 2);
+            for (int64_t g = lane; g < G; g += 32) {
+                const uint32_t v = __ldg(s2 + g);
+                kmax = max(kmax, max(scale_key(v & 0xFF), scale_key(v >> 8)));
+            }
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, d));
+        if (lane == 0) {
+            kmax_s[r] = kmax;
+            if (row < R) row_exp[row] = kmax ? kmax - 25 : 0;   // true scale = UE4M3 value * 2^(kmax - 25)
+        }
+    }
+    __syncthreads();
+    for (int item = threadIdx.x; item < nk64 * 128; item += 256) {
+        const int c = item >> 7, u = item & 127;                 // K/64 block, 4-byte word inside its chunk
+        const int r = (u & 3) * 32 + (u >> 2);
+        const int64_t row = row0 + r;
+        uint32_t wp = 0, wn = 0;
+        if (row < R) {
+            const int kmax = kmax_s[r];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {                        // the two 32-groups of this 64-element block
+                const int64_t g = (int64_t)c * 2 + h;
+                if (g < G) {
+                    const uint32_t v = __ldg(reinterpret_cast<const unsigned short*>(scales + (row * G + g) * 2));
+                    const uint32_t up = to_ue4m3(v & 0xFF, kmax), un = to_ue4m3(v >> 8, kmax);
+                    wp |= (up | (up << 8)) << (16 * h);          // one scale per 16 elements: each twice
+                    wn |= (un | (un << 8)) << (16 * h);
+                }
+            }
+        }
+        const int64_t off = (rb * nk64 + c) * (int64_t)kSfChunk + u * 4;
+        *reinterpret_cast<uint32_t*>(sf_pos + off) = wp;
+        *reinterpret_cast<uint32_t*>(sf_neg + off) = wn;
+    }
+}
+
+// -------------------------------------------------------------------------------- GEMM --
+struct Params {
+    const uint8_t *sfa_pos, *sfa_neg, *sfb_pos, *sfb_neg;
+    const int *a_exp, *w_exp;
+    int64_t M, N, K, ld_c;
+    float* C;
+    int nk64, vec_store;
+    int* status;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant__ CUtensorMap tm_an,
+                const __grid_constant__ CUtensorMap tm_wp, const __grid_constant__ CUtensorMap tm_wn, const Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    Control* ctl = reinterpret_cast<Control*>(tiles + kStages * kStageBytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t m0 = (int64_t)blockIdx.y * BM, n0 = (int64_t)blockIdx.x * BN;
+    const int num_kb = (int)((p.K + BK - 1) / BK);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&ctl->full[s], 1);
+            mbar_init(&ctl->empty[s], 1);
+        }
+        mbar_init(&ctl->accum, 1);
+        ctl->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(&ctl->tmem_base, kTmemCols);
+    if (warp >= 2)
+        for (int i = threadIdx.x - 64; i < BN; i += 128) ctl->w_exp[i] = (n0 + i < p.N) ? p.w_exp[n0 + i] : 0;
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = ctl->tmem_base;
+
+    if (warp == 0) {
+        // -------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            int issued = 0;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % kStages;
+                if (kb >= kStages && !mbar_wait(&ctl->empty[s], ((kb / kStages) - 1) & 1, &ctl->abort, p.status)) break;
+                uint8_t* st = tiles + s * kStageBytes;
+                mbar_expect_tx(&ctl->full[s], kStageBytes);
+                const int x = kb * kRowBytes;
+                tma_load_2d(st + kOffAp, &tm_ap, x, (int)m0, &ctl->full[s]);
+                tma_load_2d(st + kOffAn, &tm_an, x, (int)m0, &ctl->full[s]);
+                tma_load_2d(st + kOffWp, &tm_wp, x, (int)n0, &ctl->full[s]);
+                tma_load_2d(st + kOffWn, &tm_wn, x, (int)n0, &ctl->full[s]);
+                const int64_t a_off = ((int64_t)blockIdx.y * p.nk64 + kb * 4) * kSfChunk;
+                bulk_load(st + kOffSfA, p.sfa_pos + a_off, kSfA, &ctl->full[s]);
+                bulk_load(st + kOffSfA + kSfA, p.sfa_neg + a_off, kSfA, &ctl->full[s]);
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {                    // the tile's two 128-row blocks of W
+                    const int64_t w_off = (((int64_t)blockIdx.x * 2 + j) * p.nk64 + kb * 4) * kSfChunk;
+                    bulk_load(st + kOffSfB + j * kSfA, p.sfb_pos + w_off, kSfA, &ctl->full[s]);
+                    bulk_load(st + kOffSfB + kSfB + j * kSfA, p.sfb_neg + w_off, kSfA, &ctl->full[s]);
+                }
+                issued = kb + 1;
+            }
+            // after an abort: let the copies already in flight land before shared memory is released
+            if (ctl->abort)
+                for (int kb = max(0, issued - kStages); kb < issued; ++kb)
+                    for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(&ctl->full[kb % kStages], (kb / kStages) & 1); ++i) {}
+        }
+    } else if (warp == 1) {
+        // -------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            bool ok = true;
+            for (int kb = 0; kb < num_kb && ok; ++kb) {
+                const int s = kb % kStages;
+                ok = mbar_wait(&ctl->full[s], (kb / kStages) & 1, &ctl->abort, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t st = smem_u32(tiles + s * kStageBytes);
+#pragma unroll
+                for (int pl = 0; pl < 2; ++pl)
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        tmem_cp_32x128b_warpx4(tmem + kTmemSfA + (pl * 4 + kk) * 4,
+                                               smem_desc_rows16(st + kOffSfA + pl * kSfA + kk * kSfChunk));
+#pragma unroll
+                        for (int j = 0; j < 2; ++j)
+                            tmem_cp_32x128b_warpx4(tmem + kTmemSfB + (pl * 4 + kk) * 8 + j * 4,
+                                                   smem_desc_rows16(st + kOffSfB + pl * kSfB + j * kSfA + kk * kSfChunk));
+                    }
+#pragma unroll
+                for (int pa = 0; pa < 2; ++pa)
+#pragma unroll
+                    for (int pw = 0; pw < 2; ++pw)
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)           // 64 elements = 32 bytes along the swizzled row
+                            mma_fp4_block16(tmem, smem_desc_sw128(st + (pa ? kOffAn : kOffAp) + kk * 32),
+                                            smem_desc_sw128(st + (pw ? kOffWn : kOffWp) + kk * 32), kIdesc,
+                                            tmem + kTmemSfA + (pa * 4 + kk) * 4, tmem + kTmemSfB + (pw * 4 + kk) * 8,
+                                            (kb | pa | pw | kk) ? 1u : 0u);
+                mma_commit(&ctl->empty[s]);
+            }
+            if (ok) mma_commit(&ctl->accum);
+        }
+    } else {
+        // -------------------------------------------------------------- epilogue
+        const bool ok = mbar_wait(&ctl->accum, 0, &ctl->abort, p.status);
+        tc_fence_after();
+        if (ok) {
+            const int q = warp & 3;                              // warps 2..5 cover the four lane quarters
+            const int64_t m = m0 + q * 32 + lane;
+            const int a_exp = (m < p.M) ? p.a_exp[m] : 0;
+#pragma unroll 1
+            for (int col = 0; col < BN; col += 32) {
+                uint32_t v[32];
+                tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)col, v);
+                tmem_ld_wait();
+                if (m < p.M) {
+                    float* out = p.C + m * p.ld_c + n0 + col;
+                    float f[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int e = min(127, max(-126, a_exp + ctl->w_exp[col + j]));
+                        f[j] = __uint_as_float(v[j]) * __uint_as_float((uint32_t)(e + 127) << 23);
+                    }
+                    if (p.vec_store && n0 + col + 32 <= p.N) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<float4*>(out + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (n0 + col + j < p.N) out[j] = f[j];
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+// ---------------------------------------------------------------------------------- host --
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(f);
+    });
+    return fn;
+}
+
+// [rows, K/2] bytes, row-major; box = 128 bytes x box_rows, 128-byte swizzle, zero fill outside.
+bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t K, int box_rows) {
+    EncodeTiledFn fn = encode_tiled();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)(K / 2), (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)(K / 2)};
+    const cuuint32_t box[2] = {(cuuint32_t)kRowBytes, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline size_t up256(size_t v) { return (v + 255) / 256 * 256; }
+
+struct OperandLayout {      // offsets inside the workspace of one prepared operand
+    size_t plane, sf, exps, total;
+    int64_t row_blocks;
+    int nk64;
+};
+OperandLayout operand_layout(int64_t rows, int64_t K, int rows_per_tile) {
+    OperandLayout o;
+    o.row_blocks = (rows + rows_per_tile - 1) / rows_per_tile * (rows_per_tile / 128);
+    o.nk64 = (int)((K + BK - 1) / BK) * 4;
+    o.plane = up256((size_t)rows * (K / 2));
+    o.sf = up256((size_t)o.row_blocks * o.nk64 * kSfChunk);
+    o.exps = up256((size_t)rows * 4);
+    o.total = 2 * o.plane + 2 * o.sf + o.exps;
+    return o;
+}
+
+int prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, const OperandLayout& o,
+            uint8_t* base, cudaStream_t st) {
+    const int64_t n_vec = rows * (K / 32);
+    split_planes_kernel<<<(unsigned)((n_vec + 255) / 256), 256, 0, st>>>(
+        reinterpret_cast<const uint4*>(codes), n_vec, reinterpret_cast<uint4*>(base), reinterpret_cast<uint4*>(base + o.plane));
+    scale_factors_kernel<<<(unsigned)o.row_blocks, 256, 0, st>>>(scales, rows, K / 32, o.nk64, base + 2 * o.plane,
+                                                              base + 2 * o.plane + o.sf,
+                                                              reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf));
+    return launch_status();
+}
+
+}  // namespace
+
+bool gemm_fp4_supported(int64_t M, int64_t N, int64_t K, int gs) {
+    return gs == 32 && M > 0 && N > 0 && K > 0 && K % 32 == 0 && (M + BM - 1) / BM <= 65535 &&
+           M < (1ll << 31) && N < (1ll << 31) && K < (1ll << 31);
+}
+
+size_t gemm_fp4_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+    return 256 + operand_layout(M, K, BM).total + operand_layout(N, K, BN).total;
+}
+
+int gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes, const uint8_t* w_scales,
+             int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {
+    static bool configured[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AMX_ERR_CUDA;
+    if (!configured[dev]) {
+        if (cudaFuncSetAttribute(gemm_fp4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+            return AMX_ERR_CUDA;
+        configured[dev] = true;
+    }
+    const OperandLayout oa = operand_layout(M, K, BM), ow = operand_layout(N, K, BN);
+    uint8_t* base = static_cast<uint8_t*>(workspace);
+    int* status = reinterpret_cast<int*>(base);
+    uint8_t* pa = base + 256;
+    uint8_t* pw = pa + oa.total;
+    if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return AMX_ERR_CUDA;
+    int rc = prepare(a_codes, a_scales, M, K, oa, pa, st);
+    if (rc == AMX_OK) rc = prepare(w_codes, w_scales, N, K, ow, pw, st);
+    if (rc != AMX_OK) return rc;
+
+    CUtensorMap tm_ap, tm_an, tm_wp, tm_wn;
+    if (!make_map(&tm_ap, pa, M, K, BM) || !make_map(&tm_an, pa + oa.plane, M, K, BM) ||
+        !make_map(&tm_wp, pw, N, K, BN) || !make_map(&tm_wn, pw + ow.plane, N, K, BN))
+        return AMX_ERR_CUDA;
+    Params p;
+    p.sfa_pos = pa + 2 * oa.plane;
+    p.sfa_neg = p.sfa_pos + oa.sf;
+    p.a_exp = reinterpret_cast<const int*>(pa + 2 * oa.plane + 2 * oa.sf);
+    p.sfb_pos = pw + 2 * ow.plane;
+    p.sfb_neg = p.sfb_pos + ow.sf;
+    p.w_exp = reinterpret_cast<const int*>(pw + 2 * ow.plane + 2 * ow.sf);
+    p.M = M; p.N = N; p.K = K; p.ld_c = ld_c; p.C = C;
+    p.nk64 = oa.nk64;
+    p.vec_store = aligned(C, 16) && ld_c % 4 == 0;
+    p.status = status;
+    dim3 grid((unsigned)((N + BN - 1) / BN), (unsigned)((M + BM - 1) / BM));
+    gemm_fp4_kernel<<<grid, kThreads, kSmemBytes, st>>>(tm_ap, tm_an, tm_wp, tm_wn, p);
+    return launch_status();
+}
+
+}  // namespace amx

@@ -25,9 +25,12 @@
 #include <cuda_bf16.h>
 
 #include "gemm.cuh"
+#include "tcgen05.cuh"
 
 namespace amx {
 namespace {
+
+using namespace tc;
 
 constexpr int BM = 128, BN = 256, BK = 64;       // tile; BK bf16 = one 128-byte swizzle row
 constexpr int kStages = 2;
@@ -35,7 +38,6 @@ constexpr int kProducerWarps = 8;
 constexpr int kThreads = (kProducerWarps + 1) * 32;
 constexpr int kTileA = BM * BK * 2, kTileB = BN * BK * 2, kStageBytes = kTileA + kTileB;
 constexpr int kTmemCols = 256;
-constexpr uint32_t kSpinLimit = 1u << 24;         // mbarrier polls before giving up
 
 struct __align__(8) Control {
     uint64_t full[kStages], empty[kStages], accum;
@@ -44,75 +46,6 @@ struct __align__(8) Control {
 };
 constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + sizeof(Control);
 
-// ---------------------------------------------------------------------------- PTX wrappers --
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* b, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(b)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* b) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* b, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false when the limit expired or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, Control* ctl, int* status) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        if (mbar_try_wait(b, parity)) return true;
-        if (ctl->abort) return false;
-    }
-    ctl->abort = 1;
-    if (status) atomicExch(status, (int)AMX_ERR_TIMEOUT);
-    return false;
-}
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc(uint32_t* dst, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst)), "r"(cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
-}
-// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate; issued by one thread.
-__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// mbarrier arrive once all MMAs issued so far by this thread have completed.
-__device__ __forceinline__ void mma_commit(uint64_t* b) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(b)) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows 128 B apart, groups of
-// 8 rows 1024 B apart (stride byte offset); the leading byte offset is unused for this layout.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
-    return (uint64_t)((addr >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
-}
 // Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M x N.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
@@ -227,7 +160,7 @@ gemm_tc_kernel(const uint8_t* __restrict__ a_codes, const uint8_t* __restrict__ 
         for (int kb = 0; kb < num_kb && ok; ++kb) {
             const int s = kb % kStages;
             if (kb + 1 < num_kb) load_all(nxt, kb + 1);
-            if (kb >= kStages) ok = mbar_wait(&ctl->empty[s], ((kb / kStages) - 1) & 1, ctl, status);
+            if (kb >= kStages) ok = mbar_wait(&ctl->empty[s], ((kb / kStages) - 1) & 1, &ctl->abort, status);
             if (!ok) break;
             uint8_t* stage = tiles + s * kStageBytes;
 #pragma unroll
@@ -249,7 +182,7 @@ gemm_tc_kernel(const uint8_t* __restrict__ a_codes, const uint8_t* __restrict__ 
             for (int i = 0; i < kTasksPerThread; ++i) cur[i] = nxt[i];
         }
         // ------------------------------------------------------------------ epilogue
-        if (ok) ok = mbar_wait(&ctl->accum, 0, ctl, status);
+        if (ok) ok = mbar_wait(&ctl->accum, 0, &ctl->abort, status);
         tc_fence_after();
         if (ok) {
             const int q = warp & 3, h = warp >> 2;                 // lane quarter, column half
@@ -280,7 +213,7 @@ gemm_tc_kernel(const uint8_t* __restrict__ a_codes, const uint8_t* __restrict__ 
         bool ok = true;
         for (int kb = 0; kb < num_kb && ok; ++kb) {
             const int s = kb % kStages;
-            ok = mbar_wait(&ctl->full[s], (kb / kStages) & 1, ctl, status);
+            ok = mbar_wait(&ctl->full[s], (kb / kStages) & 1, &ctl->abort, status);
             if (!ok) break;
             tc_fence_after();
             const uint32_t a_addr = smem_u32(tiles + s * kStageBytes), b_addr = a_addr + kTileA;

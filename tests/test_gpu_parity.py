@@ -127,26 +127,34 @@ def test_gemm_simt_against_oracle(shape, gs):
     assert rel_fro(got, ref) <= 1e-5          # fp32 accumulation of <= 10-bit products is far tighter
 
 
+TC_KERNELS = [("tc", 0x20, 1e-5), ("fp4", 0x40, 1e-4)]
+
+
 @pytest.mark.parametrize("shape", [(128, 256, 64), (128, 256, 256), (1, 1, 32), (130, 260, 96), (300, 520, 1056),
                                    (256, 512, 4096)])
-def test_gemm_tensor_core_against_oracle(shape):
-    """tcgen05 path: one tile, several K blocks, a single group, ragged M/N/K tails, several tiles."""
+@pytest.mark.parametrize("kernel", TC_KERNELS, ids=lambda k: k[0])
+def test_gemm_tensor_core_against_oracle(shape, kernel):
+    """tcgen05 paths: one tile, several K blocks, a single group, ragged M/N/K tails, several tiles.
+    The bf16-decode kernel is exact up to summation order; the FP4 kernel additionally flushes scales
+    more than 14 binades below their row's largest scale."""
     M, N, K = shape
-    assert amx.lib().amx_gemm_kernel_for(M, N, K, 32, amx.GEMM_TC) == amx.GEMM_TC
+    _, flag, tol = kernel
+    assert amx.lib().amx_gemm_kernel_for(M, N, K, 32, flag) == flag
     a = inputs.random_groups(51, M, K, "mixed")
     w = inputs.random_groups(52, N, K, "normal")
     (ac, as_), (wc, ws) = oracle.quantize(a, 32), oracle.quantize(w, 32)
-    work = torch.zeros(256, dtype=torch.uint8, device="cuda")
-    got = amx.gemm(*(torch.from_numpy(t).cuda() for t in (ac, as_, wc, ws)), 32, amx.GEMM_TC, workspace=work)
+    work = torch.zeros(max(256, amx.lib().amx_workspace_bytes(M, N, K, 32, flag)), dtype=torch.uint8, device="cuda")
+    got = amx.gemm(*(torch.from_numpy(t).cuda() for t in (ac, as_, wc, ws)), 32, flag, workspace=work)
     assert amx.gemm_status(work) == 0
     got = got.cpu().numpy()
     ref = oracle.gemm(ac, as_, wc, ws, 32)
     for m in range(M):                         # row-wise: "mixed" rows differ by many orders of magnitude
         if np.all(np.isfinite(ref[m])) and np.linalg.norm(ref[m]) > 0:
-            assert rel_fro(got[m], ref[m]) <= 1e-5, m
+            assert rel_fro(got[m], ref[m]) <= tol, m
 
 
-def test_gemm_tensor_core_exact_on_small_integers():
+@pytest.mark.parametrize("kernel", TC_KERNELS, ids=lambda k: k[0])
+def test_gemm_tensor_core_exact_on_small_integers(kernel):
     rng = np.random.default_rng(9)
     grid = np.array([0, 1, 2, 3, 4, 6], np.float32)
     def ints(r, k):
@@ -155,15 +163,35 @@ def test_gemm_tensor_core_exact_on_small_integers():
         return t
     a, w = ints(200, 320), ints(300, 320)
     qa, qw = oracle.quantize(inputs.f32_to_bf16_bits(a), 32), oracle.quantize(inputs.f32_to_bf16_bits(w), 32)
-    got = amx.gemm(*(torch.from_numpy(t).cuda() for t in (*qa, *qw)), 32, amx.GEMM_TC).cpu().numpy()
+    got = amx.gemm(*(torch.from_numpy(t).cuda() for t in (*qa, *qw)), 32, kernel[1]).cpu().numpy()
     assert np.array_equal(got, (a.astype(np.int64) @ w.astype(np.int64).T).astype(np.float32))
 
 
-def test_gemm_tensor_core_matches_simt_at_scale():
+def test_gemm_fp4_scale_range_handling():
+    """Rows whose scales span more than the UE4M3 range: the small groups are flushed, the result stays
+    within 2^-13 of the row's norm; rows of zeros and one-sided rows give exact zeros / exact values."""
+    rng = np.random.default_rng(10)
+    a = rng.standard_normal((64, 256)).astype(np.float32)
+    a[:, 32:64] *= 2.0 ** 20                    # one dominant group per row, 20 binades above the rest
+    a[5] = 0.0                                  # all-zero row
+    a[6] = np.abs(a[6])                         # no negative side
+    w = rng.standard_normal((96, 256)).astype(np.float32)
+    w[:, :32] *= 2.0 ** -18
+    qa, qw = oracle.quantize(inputs.f32_to_bf16_bits(a), 32), oracle.quantize(inputs.f32_to_bf16_bits(w), 32)
+    got = amx.gemm(*(torch.from_numpy(t).cuda() for t in (*qa, *qw)), 32, amx.GEMM_FP4).cpu().numpy()
+    ref = oracle.gemm(*qa, *qw, 32)
+    assert np.all(got[5] == 0.0)
+    for m in range(64):
+        if m != 5:
+            assert rel_fro(got[m], ref[m]) <= 2.0 ** -13
+
+
+@pytest.mark.parametrize("flag", [0x20, 0x40], ids=["tc", "fp4"])
+def test_gemm_tensor_core_matches_simt_at_scale(flag):
     a = dev_bf16(inputs.activation(2, 1))                 # 2048 x 4096
     w = dev_bf16(inputs.weight(2, 1))                     # 4096 x 4096
     (ac, as_), (wc, ws) = amx.quantize(a, 32), amx.quantize(w, 32)
-    tc = amx.gemm(ac, as_, wc, ws, 32, amx.GEMM_TC)
+    tc = amx.gemm(ac, as_, wc, ws, 32, flag)
     simt = amx.gemm(ac, as_, wc, ws, 32, amx.GEMM_SIMT)
     assert rel_fro(tc.cpu().numpy(), simt.cpu().numpy()) <= 1e-5
 
