@@ -95,51 +95,61 @@ __device__ __forceinline__ uint32_t to_ue4m3(uint32_t b, int kmax) {
     return (f >= 1 && scale_key(b) > 0) ? (uint32_t)((f << 3) | (mant << 1)) : 0u;
 }
 
-// One block per 128 operand rows: row offsets, then the scale-factor blocks of both planes.
-// sf layout: [plane][row block][K/64 block][512 B], byte (r%32)*16 + (r/32)*4 + (k16 % 4).
+// Row offsets: one warp per operand row finds the largest exponent key among the row's scales.
+// kmax[row] = that key; row_exp[row] = kmax - 25, the power of two by which the UE4M3 scales of the
+// row understate the true ones (0 for an all-zero row).
 __global__ void __launch_bounds__(256)
-scale_factors_kernel(const uint8_t* __restrict__ scales, int64_t R, int64_t G /*groups per row*/, int nk64,
-                     uint8_t* __restrict__ sf_pos, uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp) {
-    __shared__ int kmax_s[128];
-    const int64_t rb = blockIdx.x, row0 = rb * 128;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int r = warp; r < 128; r += 8) {
-        const int64_t row = row0 + r;
-        int kmax = 0;
-        if (row < R) {
-            const unsigned short* s2 = reinterpret_cast<const unsigned short*>(scales + row * G * 2);
-            for (int64_t g = lane; g < G; g += 32) {
-                const uint32_t v = __ldg(s2 + g);
-                kmax = max(kmax, max(scale_key(v & 0xFF), scale_key(v >> 8)));
-            }
-        }
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, d));
-        if (lane == 0) {
-            kmax_s[r] = kmax;
-            if (row < R) row_exp[row] = kmax ? kmax - 25 : 0;   // true scale = UE4M3 value * 2^(kmax - 25)
-        }
+row_offsets_kernel(const uint8_t* __restrict__ scales, int64_t R, int64_t G /*groups per row*/,
+                   int* __restrict__ kmax_out, int* __restrict__ row_exp) {
+    const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= R) return;
+    const unsigned short* s2 = reinterpret_cast<const unsigned short*>(scales + row * G * 2);
+    int kmax = 0;
+    for (int64_t g = lane; g < G; g += 32) {
+        const uint32_t v = __ldg(s2 + g);
+        kmax = max(kmax, max(scale_key(v & 0xFF), scale_key(v >> 8)));
     }
-    __syncthreads();
-    for (int item = threadIdx.x; item < nk64 * 128; item += 256) {
-        const int c = item >> 7, u = item & 127;                 // K/64 block, 4-byte word inside its chunk
-        const int r = (u & 3) * 32 + (u >> 2);
-        const int64_t row = row0 + r;
-        uint32_t wp = 0, wn = 0;
-        if (row < R) {
-            const int kmax = kmax_s[r];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {                        // the two 32-groups of this 64-element block
-                const int64_t g = (int64_t)c * 2 + h;
-                if (g < G) {
-                    const uint32_t v = __ldg(reinterpret_cast<const unsigned short*>(scales + (row * G + g) * 2));
-                    const uint32_t up = to_ue4m3(v & 0xFF, kmax), un = to_ue4m3(v >> 8, kmax);
-                    wp |= (up | (up << 8)) << (16 * h);          // one scale per 16 elements: each twice
-                    wn |= (un | (un << 8)) << (16 * h);
-                }
-            }
+    for (int d = 16; d > 0; d >>= 1) kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, d));
+    if (lane == 0) {
+        kmax_out[row] = kmax;
+        row_exp[row] = kmax ? kmax - 25 : 0;
+    }
+}
+
+// Scale-factor blocks of both planes.  One block = 128 operand rows x 8 K/64 blocks (16 groups):
+// the E5M2 pairs are staged in shared memory (one 32-byte run per row), then written out in the
+// layout the MMA reads: [plane][row block][K/64 block][512 B], byte (r%32)*16 + (r/32)*4 + (k16 % 4).
+constexpr int kSfBlocksPerCta = 8;
+__global__ void __launch_bounds__(256)
+scale_factors_kernel(const uint8_t* __restrict__ scales, const int* __restrict__ kmax_in, int64_t R, int64_t G,
+                     int nk64, uint8_t* __restrict__ sf_pos, uint8_t* __restrict__ sf_neg) {
+    __shared__ unsigned short sc[128][2 * kSfBlocksPerCta + 1];
+    __shared__ int kmax_s[128];
+    const int64_t rb = blockIdx.y, row0 = rb * 128;
+    const int c0 = blockIdx.x * kSfBlocksPerCta;
+    for (int i = threadIdx.x; i < 128 * 2 * kSfBlocksPerCta; i += 256) {
+        const int r = i / (2 * kSfBlocksPerCta), gl = i % (2 * kSfBlocksPerCta);
+        const int64_t row = row0 + r, g = (int64_t)c0 * 2 + gl;
+        sc[r][gl] = (row < R && g < G) ? __ldg(reinterpret_cast<const unsigned short*>(scales + (row * G + g) * 2)) : 0;
+    }
+    if (threadIdx.x < 128) kmax_s[threadIdx.x] = (row0 + threadIdx.x < R) ? kmax_in[row0 + threadIdx.x] : 0;
+    __syncthreads();
+    for (int item = threadIdx.x; item < kSfBlocksPerCta * 128; item += 256) {
+        const int cc = item >> 7, u = item & 127;                // K/64 block, 4-byte word inside its chunk
+        if (c0 + cc >= nk64) break;
+        const int r = (u & 3) * 32 + (u >> 2);
+        const int kmax = kmax_s[r];
+        uint32_t wp = 0, wn = 0;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {                            // the two 32-groups of this 64-element block
+            const uint32_t v = sc[r][2 * cc + h];
+            const uint32_t up = to_ue4m3(v & 0xFF, kmax), un = to_ue4m3(v >> 8, kmax);
+            wp |= (up | (up << 8)) << (16 * h);                  // one scale per 16 elements: each twice
+            wn |= (un | (un << 8)) << (16 * h);
         }
-        const int64_t off = (rb * nk64 + c) * (int64_t)kSfChunk + u * 4;
+        const int64_t off = (rb * nk64 + c0 + cc) * (int64_t)kSfChunk + u * 4;
         *reinterpret_cast<uint32_t*>(sf_pos + off) = wp;
         *reinterpret_cast<uint32_t*>(sf_neg + off) = wn;
     }
@@ -333,7 +343,7 @@ OperandLayout operand_layout(int64_t rows, int64_t K, int rows_per_tile) {
     o.nk64 = (int)((K + BK - 1) / BK) * 4;
     o.plane = up256((size_t)rows * (K / 2));
     o.sf = up256((size_t)o.row_blocks * o.nk64 * kSfChunk);
-    o.exps = up256((size_t)rows * 4);
+    o.exps = up256((size_t)rows * 8);      // row offsets, then the rows' largest exponent keys
     o.total = 2 * o.plane + 2 * o.sf + o.exps;
     return o;
 }
@@ -343,9 +353,12 @@ int prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K
     const int64_t n_vec = rows * (K / 32);
     split_planes_kernel<<<(unsigned)((n_vec + 255) / 256), 256, 0, st>>>(
         reinterpret_cast<const uint4*>(codes), n_vec, reinterpret_cast<uint4*>(base), reinterpret_cast<uint4*>(base + o.plane));
-    scale_factors_kernel<<<(unsigned)o.row_blocks, 256, 0, st>>>(scales, rows, K / 32, o.nk64, base + 2 * o.plane,
-                                                              base + 2 * o.plane + o.sf,
-                                                              reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf));
+    int* exps = reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf);
+    int* kmax = exps + rows;
+    row_offsets_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(scales, rows, K / 32, kmax, exps);
+    dim3 grid((unsigned)((o.nk64 + kSfBlocksPerCta - 1) / kSfBlocksPerCta), (unsigned)o.row_blocks);
+    scale_factors_kernel<<<grid, 256, 0, st>>>(scales, kmax, rows, K / 32, o.nk64, base + 2 * o.plane,
+                                               base + 2 * o.plane + o.sf);
     return launch_status();
 }
 
