@@ -17,15 +17,17 @@
 // Pipeline per CTA (128 x 256 tile of C, 256-element K blocks, two stages of 108 KB):
 //   warp 0   TMA producer: four 128-byte-swizzled code tiles (A+, A-, W+, W-) and the scale-factor
 //            blocks (plain bulk copies) per stage, completion on the stage's `full` mbarrier
-//   warp 1   allocates TMEM; one lane copies the stage's scale factors shared -> tensor memory
-//            (tcgen05.cp) and issues 16 MMAs (4 sign pairs x 4 K steps of 64), then commits to the
-//            stage's `empty` mbarrier
-//   warps 2-5  epilogue: TMEM -> registers, power-of-two rescale, fp32 stores
+//   warp 1   allocates TMEM; one lane issues the stage's MMAs (4 sign pairs x K steps of 64), then
+//            commits to the stage's `empty` mbarrier
+//   warps 2-5  move each stage's scale factors shared -> registers -> tensor memory (tcgen05.st; this
+//            keeps the copies off the in-order MMA queue), signal `sf_full`; afterwards they are the
+//            epilogue: TMEM -> registers, power-of-two rescale, fp32 stores
 // A preparation pass (two small kernels per operand) derives the planes, the UE4M3 scale-factor
 // blocks in the 128 x 4 interleaved layout the MMA reads, and the row offsets from the canonical
 // codes and scales.  Every device-side wait is bounded.
 #include <cuda.h>
 
+#include <cstdlib>
 #include <mutex>
 
 #include "gemm.cuh"
@@ -37,27 +39,49 @@ namespace {
 using namespace tc;
 
 constexpr int BM = 128, BN = 256;
-constexpr int BK = 256;                 // elements per K block = 128 bytes of codes per row
-constexpr int kRowBytes = BK / 2;
-constexpr int kStages = 2;
 constexpr int kThreads = 192;
-constexpr int kTileA = BM * kRowBytes, kTileB = BN * kRowBytes;       // one plane
 constexpr int kSfChunk = 512;           // scale factors of 128 rows x 64 elements (4 per row)
-constexpr int kSfA = 4 * kSfChunk;      // one plane, one K block, 128 rows
-constexpr int kSfB = 2 * kSfA;          // 256 rows
-constexpr int kOffAp = 0, kOffAn = kTileA, kOffWp = 2 * kTileA, kOffWn = 2 * kTileA + kTileB;
-constexpr int kOffSfA = 2 * kTileA + 2 * kTileB, kOffSfB = kOffSfA + 2 * kSfA;
-constexpr int kStageBytes = kOffSfB + 2 * kSfB;                       // 110592
 constexpr int kTmemCols = 512;
-constexpr uint32_t kTmemSfA = 256, kTmemSfB = 256 + 32;               // after the 256 accumulator columns
+constexpr uint32_t kTmemSf = 256;      // scale-factor columns follow the 256 accumulator columns
+
+// Shared-memory stage geometry for a K block of BK elements (BK/2 bytes of codes per row and plane).
+// BK = 256: 128-byte rows, 128-byte swizzle, 2 stages of 108 KB.
+// BK = 128:  64-byte rows,  64-byte swizzle, 4 stages of  54 KB (finer-grained prefetch).
+template <int BK_>
+struct Cfg {
+    static constexpr int BK = BK_;
+    static constexpr int kRowBytes = BK / 2;
+    static constexpr int kSteps = BK / 64;                            // MMAs (K = 64) per K block and sign pair
+    static constexpr int kStages = BK == 256 ? 2 : 4;
+    static constexpr int kTileA = BM * kRowBytes, kTileB = BN * kRowBytes;   // one plane
+    static constexpr int kSfA = kSteps * kSfChunk;                    // one plane, one K block, 128 rows
+    static constexpr int kSfB = 2 * kSfA;                             // 256 rows
+    static constexpr int kOffAp = 0, kOffAn = kTileA, kOffWp = 2 * kTileA, kOffWn = 2 * kTileA + kTileB;
+    static constexpr int kOffSfA = 2 * kTileA + 2 * kTileB, kOffSfB = kOffSfA + 2 * kSfA;
+    static constexpr int kStageBytes = kOffSfB + 2 * kSfB;
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 2048;   // + alignment slack + Control
+    // TMEM columns of one stage's scale factors: A planes (4 columns per K step), then W planes (8)
+    static constexpr int kSfColsA = 2 * kSteps * 4, kSfCols = kSfColsA + 2 * kSteps * 8;
+    static_assert(256 + kStages * kSfCols <= kTmemCols, "scale factors do not fit tensor memory");
+};
+constexpr int kMaxStages = 4;
 
 struct __align__(8) Control {
-    uint64_t full[kStages], empty[kStages], accum;
+    uint64_t full[kMaxStages], sf_full[kMaxStages], empty[kMaxStages], accum;
     uint32_t tmem_base;
     volatile int abort;
     int w_exp[BN];
 };
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 + sizeof(Control);
+static_assert(sizeof(Control) <= 2048, "Control must fit its reserved space");
+
+// K-major operand rows of 64 bytes with the 64-byte swizzle: groups of 8 rows are 512 B apart.
+__device__ __forceinline__ uint64_t smem_desc_sw64(uint32_t addr) {
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)(512 >> 4) << 32) | (1ull << 46) | (4ull << 61);
+}
+template <int BK_>
+__device__ __forceinline__ uint64_t operand_desc(uint32_t addr) {
+    return BK_ == 256 ? smem_desc_sw128(addr) : smem_desc_sw64(addr);
+}
 
 // Instruction descriptor, kind::mxf4nvf4 block-scaled: A and B E2M1 (format code 1), K-major,
 // UE4M3 scale factors (bit 23 = 0), N >> 3 at bit 17, M >> 4 at bit 24, K = 64 (bit 31 = 0).
@@ -165,9 +189,13 @@ struct Params {
     int* status;
 };
 
+template <int BK_>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant__ CUtensorMap tm_an,
                 const __grid_constant__ CUtensorMap tm_wp, const __grid_constant__ CUtensorMap tm_wn, const Params p) {
+    using C_ = Cfg<BK_>;
+    constexpr int BK = C_::BK, kRowBytes = C_::kRowBytes, kSteps = C_::kSteps, kStages = C_::kStages;
+    constexpr int kStageBytes = C_::kStageBytes, kSfA = C_::kSfA, kSfB = C_::kSfB;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     Control* ctl = reinterpret_cast<Control*>(tiles + kStages * kStageBytes);
@@ -178,6 +206,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&ctl->full[s], 1);
+            mbar_init(&ctl->sf_full[s], 4);
             mbar_init(&ctl->empty[s], 1);
         }
         mbar_init(&ctl->accum, 1);
@@ -202,18 +231,18 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant
                 uint8_t* st = tiles + s * kStageBytes;
                 mbar_expect_tx(&ctl->full[s], kStageBytes);
                 const int x = kb * kRowBytes;
-                tma_load_2d(st + kOffAp, &tm_ap, x, (int)m0, &ctl->full[s]);
-                tma_load_2d(st + kOffAn, &tm_an, x, (int)m0, &ctl->full[s]);
-                tma_load_2d(st + kOffWp, &tm_wp, x, (int)n0, &ctl->full[s]);
-                tma_load_2d(st + kOffWn, &tm_wn, x, (int)n0, &ctl->full[s]);
-                const int64_t a_off = ((int64_t)blockIdx.y * p.nk64 + kb * 4) * kSfChunk;
-                bulk_load(st + kOffSfA, p.sfa_pos + a_off, kSfA, &ctl->full[s]);
-                bulk_load(st + kOffSfA + kSfA, p.sfa_neg + a_off, kSfA, &ctl->full[s]);
+                tma_load_2d(st + C_::kOffAp, &tm_ap, x, (int)m0, &ctl->full[s]);
+                tma_load_2d(st + C_::kOffAn, &tm_an, x, (int)m0, &ctl->full[s]);
+                tma_load_2d(st + C_::kOffWp, &tm_wp, x, (int)n0, &ctl->full[s]);
+                tma_load_2d(st + C_::kOffWn, &tm_wn, x, (int)n0, &ctl->full[s]);
+                const int64_t a_off = ((int64_t)blockIdx.y * p.nk64 + kb * kSteps) * kSfChunk;
+                bulk_load(st + C_::kOffSfA, p.sfa_pos + a_off, kSfA, &ctl->full[s]);
+                bulk_load(st + C_::kOffSfA + kSfA, p.sfa_neg + a_off, kSfA, &ctl->full[s]);
 #pragma unroll
                 for (int j = 0; j < 2; ++j) {                    // the tile's two 128-row blocks of W
-                    const int64_t w_off = (((int64_t)blockIdx.x * 2 + j) * p.nk64 + kb * 4) * kSfChunk;
-                    bulk_load(st + kOffSfB + j * kSfA, p.sfb_pos + w_off, kSfA, &ctl->full[s]);
-                    bulk_load(st + kOffSfB + kSfB + j * kSfA, p.sfb_neg + w_off, kSfA, &ctl->full[s]);
+                    const int64_t w_off = (((int64_t)blockIdx.x * 2 + j) * p.nk64 + kb * kSteps) * kSfChunk;
+                    bulk_load(st + C_::kOffSfB + j * kSfA, p.sfb_pos + w_off, kSfA, &ctl->full[s]);
+                    bulk_load(st + C_::kOffSfB + kSfB + j * kSfA, p.sfb_neg + w_off, kSfA, &ctl->full[s]);
                 }
                 issued = kb + 1;
             }
@@ -228,41 +257,60 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant
             bool ok = true;
             for (int kb = 0; kb < num_kb && ok; ++kb) {
                 const int s = kb % kStages;
-                ok = mbar_wait(&ctl->full[s], (kb / kStages) & 1, &ctl->abort, p.status);
+                ok = mbar_wait(&ctl->full[s], (kb / kStages) & 1, &ctl->abort, p.status) &&
+                     mbar_wait(&ctl->sf_full[s], (kb / kStages) & 1, &ctl->abort, p.status);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t st = smem_u32(tiles + s * kStageBytes);
-#pragma unroll
-                for (int pl = 0; pl < 2; ++pl)
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        tmem_cp_32x128b_warpx4(tmem + kTmemSfA + (pl * 4 + kk) * 4,
-                                               smem_desc_rows16(st + kOffSfA + pl * kSfA + kk * kSfChunk));
-#pragma unroll
-                        for (int j = 0; j < 2; ++j)
-                            tmem_cp_32x128b_warpx4(tmem + kTmemSfB + (pl * 4 + kk) * 8 + j * 4,
-                                                   smem_desc_rows16(st + kOffSfB + pl * kSfB + j * kSfA + kk * kSfChunk));
-                    }
+                const uint32_t sfa = tmem + kTmemSf + s * C_::kSfCols, sfb = sfa + C_::kSfColsA;
 #pragma unroll
                 for (int pa = 0; pa < 2; ++pa)
 #pragma unroll
                     for (int pw = 0; pw < 2; ++pw)
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)           // 64 elements = 32 bytes along the swizzled row
-                            mma_fp4_block16(tmem, smem_desc_sw128(st + (pa ? kOffAn : kOffAp) + kk * 32),
-                                            smem_desc_sw128(st + (pw ? kOffWn : kOffWp) + kk * 32), kIdesc,
-                                            tmem + kTmemSfA + (pa * 4 + kk) * 4, tmem + kTmemSfB + (pw * 4 + kk) * 8,
+                        for (int kk = 0; kk < kSteps; ++kk)      // 64 elements = 32 bytes along the swizzled row
+                            mma_fp4_block16(tmem, operand_desc<BK_>(st + (pa ? C_::kOffAn : C_::kOffAp) + kk * 32),
+                                            operand_desc<BK_>(st + (pw ? C_::kOffWn : C_::kOffWp) + kk * 32), kIdesc,
+                                            sfa + (pa * kSteps + kk) * 4, sfb + (pw * kSteps + kk) * 8,
                                             (kb | pa | pw | kk) ? 1u : 0u);
                 mma_commit(&ctl->empty[s]);
             }
             if (ok) mma_commit(&ctl->accum);
         }
     } else {
-        // -------------------------------------------------------------- epilogue
-        const bool ok = mbar_wait(&ctl->accum, 0, &ctl->abort, p.status);
+        // ------------------------------------------------ scale factors, then epilogue
+        // Each of the four warps owns one 32-lane quarter of tensor memory.  Per stage it reads the
+        // stage's scale-factor blocks from shared memory (16 bytes per lane and block: the 4-byte
+        // scale words of rows lane, lane+32, lane+64, lane+96) and stores them into its quarter's
+        // copy of the scale-factor columns, which every quarter has to hold.
+        const int q = warp & 3;                                  // warps 2..5 cover the four lane quarters
+        bool ok = true;
+        for (int kb = 0; kb < num_kb && ok; ++kb) {
+            const int s = kb % kStages;
+            ok = mbar_wait(&ctl->full[s], (kb / kStages) & 1, &ctl->abort, p.status);
+            if (!ok) break;
+            const uint8_t* st = tiles + s * kStageBytes;
+            const uint32_t sfa = tmem + ((uint32_t)(q * 32) << 16) + kTmemSf + s * C_::kSfCols, sfb = sfa + C_::kSfColsA;
+#pragma unroll
+            for (int pl = 0; pl < 2; ++pl)
+#pragma unroll
+                for (int kk = 0; kk < kSteps; ++kk) {
+                    const uint4 a = *reinterpret_cast<const uint4*>(st + C_::kOffSfA + pl * kSfA + kk * kSfChunk + lane * 16);
+                    tmem_st4(sfa + (pl * kSteps + kk) * 4, a.x, a.y, a.z, a.w);
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        const uint4 b = *reinterpret_cast<const uint4*>(st + C_::kOffSfB + pl * kSfB + j * kSfA + kk * kSfChunk + lane * 16);
+                        tmem_st4(sfb + (pl * kSteps + kk) * 8 + j * 4, b.x, b.y, b.z, b.w);
+                    }
+                }
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->sf_full[s]);
+        }
+        if (ok) ok = mbar_wait(&ctl->accum, 0, &ctl->abort, p.status);
         tc_fence_after();
         if (ok) {
-            const int q = warp & 3;                              // warps 2..5 cover the four lane quarters
             const int64_t m = m0 + q * 32 + lane;
             const int a_exp = (m < p.M) ? p.a_exp[m] : 0;
 #pragma unroll 1
@@ -318,15 +366,16 @@ EncodeTiledFn encode_tiled() {
 }
 
 // [rows, K/2] bytes, row-major; box = 128 bytes x box_rows, 128-byte swizzle, zero fill outside.
-bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t K, int box_rows) {
+bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t K, int box_rows, int row_bytes) {
     EncodeTiledFn fn = encode_tiled();
     if (!fn) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)(K / 2), (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)(K / 2)};
-    const cuuint32_t box[2] = {(cuuint32_t)kRowBytes, (cuuint32_t)box_rows};
+    const cuuint32_t box[2] = {(cuuint32_t)row_bytes, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -340,7 +389,7 @@ struct OperandLayout {      // offsets inside the workspace of one prepared oper
 OperandLayout operand_layout(int64_t rows, int64_t K, int rows_per_tile) {
     OperandLayout o;
     o.row_blocks = (rows + rows_per_tile - 1) / rows_per_tile * (rows_per_tile / 128);
-    o.nk64 = (int)((K + BK - 1) / BK) * 4;
+    o.nk64 = (int)((K + 255) / 256) * 4;    // padded to whole 256-element blocks
     o.plane = up256((size_t)rows * (K / 2));
     o.sf = up256((size_t)o.row_blocks * o.nk64 * kSfChunk);
     o.exps = up256((size_t)rows * 8);      // row offsets, then the rows' largest exponent keys
@@ -373,16 +422,42 @@ size_t gemm_fp4_workspace_bytes(int64_t M, int64_t N, int64_t K) {
     return 256 + operand_layout(M, K, BM).total + operand_layout(N, K, BN).total;
 }
 
-int gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes, const uint8_t* w_scales,
-             int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {
+namespace {
+
+template <int BK_>
+int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, const OperandLayout& ow, Params p,
+               int dev, cudaStream_t st) {
+    using C_ = Cfg<BK_>;
     static bool configured[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AMX_ERR_CUDA;
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(gemm_fp4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(gemm_fp4_kernel<BK_>, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::kSmemBytes) != cudaSuccess)
             return AMX_ERR_CUDA;
         configured[dev] = true;
     }
+    CUtensorMap tm_ap, tm_an, tm_wp, tm_wn;
+    if (!make_map(&tm_ap, pa, p.M, p.K, BM, C_::kRowBytes) || !make_map(&tm_an, pa + oa.plane, p.M, p.K, BM, C_::kRowBytes) ||
+        !make_map(&tm_wp, pw, p.N, p.K, BN, C_::kRowBytes) || !make_map(&tm_wn, pw + ow.plane, p.N, p.K, BN, C_::kRowBytes))
+        return AMX_ERR_CUDA;
+    dim3 grid((unsigned)((p.N + BN - 1) / BN), (unsigned)((p.M + BM - 1) / BM));
+    gemm_fp4_kernel<BK_><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_ap, tm_an, tm_wp, tm_wn, p);
+    return launch_status();
+}
+
+// K-block size of the main loop: 128 (four 54 KB stages) unless AMX_FP4_BK=256 asks for two 108 KB stages.
+int fp4_block_k() {
+    static const int bk = [] {
+        const char* e = getenv("AMX_FP4_BK");
+        return (e && atoi(e) == 256) ? 256 : 128;
+    }();
+    return bk;
+}
+
+}  // namespace
+
+int gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes, const uint8_t* w_scales,
+             int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AMX_ERR_CUDA;
     const OperandLayout oa = operand_layout(M, K, BM), ow = operand_layout(N, K, BN);
     uint8_t* base = static_cast<uint8_t*>(workspace);
     int* status = reinterpret_cast<int*>(base);
@@ -392,11 +467,6 @@ int gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_c
     int rc = prepare(a_codes, a_scales, M, K, oa, pa, st);
     if (rc == AMX_OK) rc = prepare(w_codes, w_scales, N, K, ow, pw, st);
     if (rc != AMX_OK) return rc;
-
-    CUtensorMap tm_ap, tm_an, tm_wp, tm_wn;
-    if (!make_map(&tm_ap, pa, M, K, BM) || !make_map(&tm_an, pa + oa.plane, M, K, BM) ||
-        !make_map(&tm_wp, pw, N, K, BN) || !make_map(&tm_wn, pw + ow.plane, N, K, BN))
-        return AMX_ERR_CUDA;
     Params p;
     p.sfa_pos = pa + 2 * oa.plane;
     p.sfa_neg = p.sfa_pos + oa.sf;
@@ -408,9 +478,7 @@ int gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_c
     p.nk64 = oa.nk64;
     p.vec_store = aligned(C, 16) && ld_c % 4 == 0;
     p.status = status;
-    dim3 grid((unsigned)((N + BN - 1) / BN), (unsigned)((M + BM - 1) / BM));
-    gemm_fp4_kernel<<<grid, kThreads, kSmemBytes, st>>>(tm_ap, tm_an, tm_wp, tm_wn, p);
-    return launch_status();
+    return fp4_block_k() == 256 ? launch_fp4<256>(pa, pw, oa, ow, p, dev, st) : launch_fp4<128>(pa, pw, oa, ow, p, dev, st);
 }
 
 }  // namespace amx
