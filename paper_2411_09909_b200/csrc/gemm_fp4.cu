@@ -14,7 +14,8 @@
 // in the epilogue (exact).  Scales more than 14 binades below their row's largest scale do not fit
 // and are flushed to zero: their groups contribute less than 2^-14 of the row's largest group.
 //
-// Pipeline per CTA (128 x 256 tile of C, 256-element K blocks, two stages of 108 KB):
+// Persistent CTAs (one per SM) walk over 128 x 256 tiles of C; K blocks of 128 elements cycle through
+// four 54 KB shared-memory stages (two 108 KB stages with 256-element blocks):
 //   warp 0   TMA producer: four 128-byte-swizzled code tiles (A+, A-, W+, W-) and the scale-factor
 //            blocks (plain bulk copies) per stage, completion on the stage's `full` mbarrier
 //   warp 1   allocates TMEM; one lane issues the stage's MMAs (4 sign pairs x K steps of 64), then
@@ -22,6 +23,8 @@
 //   warps 2-5  move each stage's scale factors shared -> registers -> tensor memory (tcgen05.st; this
 //            keeps the copies off the in-order MMA queue), signal `sf_full`; afterwards they are the
 //            epilogue: TMEM -> registers, power-of-two rescale, fp32 stores
+//   warps 6-9  epilogue only (the other half of the columns).  While a tile's accumulator is read out the
+//            producer already prefetches the next tile's stages; the MMA issuer waits for `accum_empty`.
 // A preparation pass (two small kernels per operand) derives the planes, the UE4M3 scale-factor
 // blocks in the 128 x 4 interleaved layout the MMA reads, and the row offsets from the canonical
 // codes and scales.  Every device-side wait is bounded.
@@ -39,7 +42,8 @@ namespace {
 using namespace tc;
 
 constexpr int BM = 128, BN = 256;
-constexpr int kThreads = 192;
+constexpr int kEpilogueWarps = 8;
+constexpr int kThreads = (2 + kEpilogueWarps) * 32;
 constexpr int kSfChunk = 512;           // scale factors of 128 rows x 64 elements (4 per row)
 constexpr int kTmemCols = 512;
 constexpr uint32_t kTmemSf = 256;      // scale-factor columns follow the 256 accumulator columns
@@ -59,7 +63,7 @@ struct Cfg {
     static constexpr int kOffAp = 0, kOffAn = kTileA, kOffWp = 2 * kTileA, kOffWn = 2 * kTileA + kTileB;
     static constexpr int kOffSfA = 2 * kTileA + 2 * kTileB, kOffSfB = kOffSfA + 2 * kSfA;
     static constexpr int kStageBytes = kOffSfB + 2 * kSfB;
-    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 2048;   // + alignment slack + Control
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 2048 + 256;   // + alignment slack + Control
     // TMEM columns of one stage's scale factors: A planes (4 columns per K step), then W planes (8)
     static constexpr int kSfColsA = 2 * kSteps * 4, kSfCols = kSfColsA + 2 * kSteps * 8;
     static_assert(256 + kStages * kSfCols <= kTmemCols, "scale factors do not fit tensor memory");
@@ -67,12 +71,12 @@ struct Cfg {
 constexpr int kMaxStages = 4;
 
 struct __align__(8) Control {
-    uint64_t full[kMaxStages], sf_full[kMaxStages], empty[kMaxStages], accum;
+    uint64_t full[kMaxStages], sf_full[kMaxStages], empty[kMaxStages], accum_full, accum_empty;
     uint32_t tmem_base;
     volatile int abort;
-    int w_exp[BN];
+    int w_exp[2][BN];
 };
-static_assert(sizeof(Control) <= 2048, "Control must fit its reserved space");
+static_assert(sizeof(Control) <= 2048 + 256, "Control must fit its reserved space");
 
 // K-major operand rows of 64 bytes with the 64-byte swizzle: groups of 8 rows are 512 B apart.
 __device__ __forceinline__ uint64_t smem_desc_sw64(uint32_t addr) {
@@ -200,8 +204,9 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     Control* ctl = reinterpret_cast<Control*>(tiles + kStages * kStageBytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t m0 = (int64_t)blockIdx.y * BM, n0 = (int64_t)blockIdx.x * BN;
     const int num_kb = (int)((p.K + BK - 1) / BK);
+    // Persistent CTA: tiles blockIdx.x, blockIdx.x + gridDim.x, ...; neighbouring tiles share their A rows.
+    const int64_t n_tiles = (p.N + BN - 1) / BN, total_tiles = ((p.M + BM - 1) / BM) * n_tiles;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -209,13 +214,12 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant
             mbar_init(&ctl->sf_full[s], 4);
             mbar_init(&ctl->empty[s], 1);
         }
-        mbar_init(&ctl->accum, 1);
+        mbar_init(&ctl->accum_full, 1);
+        mbar_init(&ctl->accum_empty, kEpilogueWarps);
         ctl->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(&ctl->tmem_base, kTmemCols);
-    if (warp >= 2)
-        for (int i = threadIdx.x - 64; i < BN; i += 128) ctl->w_exp[i] = (n0 + i < p.N) ? p.w_exp[n0 + i] : 0;
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -224,118 +228,149 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant
     if (warp == 0) {
         // -------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            int issued = 0;
-            for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % kStages;
-                if (kb >= kStages && !mbar_wait(&ctl->empty[s], ((kb / kStages) - 1) & 1, &ctl->abort, p.status)) break;
-                uint8_t* st = tiles + s * kStageBytes;
-                mbar_expect_tx(&ctl->full[s], kStageBytes);
-                const int x = kb * kRowBytes;
-                tma_load_2d(st + C_::kOffAp, &tm_ap, x, (int)m0, &ctl->full[s]);
-                tma_load_2d(st + C_::kOffAn, &tm_an, x, (int)m0, &ctl->full[s]);
-                tma_load_2d(st + C_::kOffWp, &tm_wp, x, (int)n0, &ctl->full[s]);
-                tma_load_2d(st + C_::kOffWn, &tm_wn, x, (int)n0, &ctl->full[s]);
-                const int64_t a_off = ((int64_t)blockIdx.y * p.nk64 + kb * kSteps) * kSfChunk;
-                bulk_load(st + C_::kOffSfA, p.sfa_pos + a_off, kSfA, &ctl->full[s]);
-                bulk_load(st + C_::kOffSfA + kSfA, p.sfa_neg + a_off, kSfA, &ctl->full[s]);
+            int it = 0;                                          // K blocks issued so far, over all tiles
+            bool ok = true;
+            for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int64_t m_blk = tile / n_tiles, n_blk = tile % n_tiles;
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = it % kStages;
+                    if (it >= kStages && !mbar_wait(&ctl->empty[s], ((it / kStages) - 1) & 1, &ctl->abort, p.status)) {
+                        ok = false;
+                        break;
+                    }
+                    uint8_t* st = tiles + s * kStageBytes;
+                    mbar_expect_tx(&ctl->full[s], kStageBytes);
+                    const int x = kb * kRowBytes;
+                    tma_load_2d(st + C_::kOffAp, &tm_ap, x, (int)(m_blk * BM), &ctl->full[s]);
+                    tma_load_2d(st + C_::kOffAn, &tm_an, x, (int)(m_blk * BM), &ctl->full[s]);
+                    tma_load_2d(st + C_::kOffWp, &tm_wp, x, (int)(n_blk * BN), &ctl->full[s]);
+                    tma_load_2d(st + C_::kOffWn, &tm_wn, x, (int)(n_blk * BN), &ctl->full[s]);
+                    const int64_t a_off = (m_blk * p.nk64 + kb * kSteps) * kSfChunk;
+                    bulk_load(st + C_::kOffSfA, p.sfa_pos + a_off, kSfA, &ctl->full[s]);
+                    bulk_load(st + C_::kOffSfA + kSfA, p.sfa_neg + a_off, kSfA, &ctl->full[s]);
 #pragma unroll
-                for (int j = 0; j < 2; ++j) {                    // the tile's two 128-row blocks of W
-                    const int64_t w_off = (((int64_t)blockIdx.x * 2 + j) * p.nk64 + kb * kSteps) * kSfChunk;
-                    bulk_load(st + C_::kOffSfB + j * kSfA, p.sfb_pos + w_off, kSfA, &ctl->full[s]);
-                    bulk_load(st + C_::kOffSfB + kSfB + j * kSfA, p.sfb_neg + w_off, kSfA, &ctl->full[s]);
+                    for (int j = 0; j < 2; ++j) {                // the tile's two 128-row blocks of W
+                        const int64_t w_off = ((n_blk * 2 + j) * p.nk64 + kb * kSteps) * kSfChunk;
+                        bulk_load(st + C_::kOffSfB + j * kSfA, p.sfb_pos + w_off, kSfA, &ctl->full[s]);
+                        bulk_load(st + C_::kOffSfB + kSfB + j * kSfA, p.sfb_neg + w_off, kSfA, &ctl->full[s]);
+                    }
                 }
-                issued = kb + 1;
             }
             // after an abort: let the copies already in flight land before shared memory is released
             if (ctl->abort)
-                for (int kb = max(0, issued - kStages); kb < issued; ++kb)
-                    for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(&ctl->full[kb % kStages], (kb / kStages) & 1); ++i) {}
+                for (int i = max(0, it - kStages); i < it; ++i)
+                    for (uint32_t n = 0; n < kSpinLimit && !mbar_try_wait(&ctl->full[i % kStages], (i / kStages) & 1); ++n) {}
         }
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer
         if (lane == 0) {
+            int it = 0, t = 0;
             bool ok = true;
-            for (int kb = 0; kb < num_kb && ok; ++kb) {
-                const int s = kb % kStages;
-                ok = mbar_wait(&ctl->full[s], (kb / kStages) & 1, &ctl->abort, p.status) &&
-                     mbar_wait(&ctl->sf_full[s], (kb / kStages) & 1, &ctl->abort, p.status);
-                if (!ok) break;
+            for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t) {
+                // the previous tile's accumulator must have been read out before it is overwritten
+                if (t > 0) ok = mbar_wait(&ctl->accum_empty, (t - 1) & 1, &ctl->abort, p.status);
                 tc_fence_after();
-                const uint32_t st = smem_u32(tiles + s * kStageBytes);
-                const uint32_t sfa = tmem + kTmemSf + s * C_::kSfCols, sfb = sfa + C_::kSfColsA;
+                for (int kb = 0; kb < num_kb && ok; ++kb, ++it) {
+                    const int s = it % kStages;
+                    ok = mbar_wait(&ctl->full[s], (it / kStages) & 1, &ctl->abort, p.status) &&
+                         mbar_wait(&ctl->sf_full[s], (it / kStages) & 1, &ctl->abort, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t st = smem_u32(tiles + s * kStageBytes);
+                    const uint32_t sfa = tmem + kTmemSf + s * C_::kSfCols, sfb = sfa + C_::kSfColsA;
 #pragma unroll
-                for (int pa = 0; pa < 2; ++pa)
+                    for (int pa = 0; pa < 2; ++pa)
 #pragma unroll
-                    for (int pw = 0; pw < 2; ++pw)
+                        for (int pw = 0; pw < 2; ++pw)
 #pragma unroll
-                        for (int kk = 0; kk < kSteps; ++kk)      // 64 elements = 32 bytes along the swizzled row
-                            mma_fp4_block16(tmem, operand_desc<BK_>(st + (pa ? C_::kOffAn : C_::kOffAp) + kk * 32),
-                                            operand_desc<BK_>(st + (pw ? C_::kOffWn : C_::kOffWp) + kk * 32), kIdesc,
-                                            sfa + (pa * kSteps + kk) * 4, sfb + (pw * kSteps + kk) * 8,
-                                            (kb | pa | pw | kk) ? 1u : 0u);
-                mma_commit(&ctl->empty[s]);
+                            for (int kk = 0; kk < kSteps; ++kk)  // 64 elements = 32 bytes along the swizzled row
+                                mma_fp4_block16(tmem, operand_desc<BK_>(st + (pa ? C_::kOffAn : C_::kOffAp) + kk * 32),
+                                                operand_desc<BK_>(st + (pw ? C_::kOffWn : C_::kOffWp) + kk * 32), kIdesc,
+                                                sfa + (pa * kSteps + kk) * 4, sfb + (pw * kSteps + kk) * 8,
+                                                (kb | pa | pw | kk) ? 1u : 0u);
+                    mma_commit(&ctl->empty[s]);
+                }
+                if (ok) mma_commit(&ctl->accum_full);
             }
-            if (ok) mma_commit(&ctl->accum);
         }
     } else {
-        // ------------------------------------------------ scale factors, then epilogue
-        // Each of the four warps owns one 32-lane quarter of tensor memory.  Per stage it reads the
-        // stage's scale-factor blocks from shared memory (16 bytes per lane and block: the 4-byte
-        // scale words of rows lane, lane+32, lane+64, lane+96) and stores them into its quarter's
-        // copy of the scale-factor columns, which every quarter has to hold.
-        const int q = warp & 3;                                  // warps 2..5 cover the four lane quarters
+        // ------------------------------------------------ scale factors and epilogue
+        // Warps 2..5 own one 32-lane quarter of tensor memory each.  Per stage they read the stage's
+        // scale-factor blocks from shared memory (16 bytes per lane and block: the 4-byte scale words of
+        // rows lane, lane+32, lane+64, lane+96) and store them into their quarter's copy of the
+        // scale-factor columns (every quarter has to hold one).  Warps 6..9 only help with the epilogue:
+        // quarter q = warp % 4 again, the other half of the columns.
+        const int q = warp & 3;
+        const bool sf_warp = warp < 2 + 4;
+        const int col_base = sf_warp ? 0 : BN / 2;
+        int it = 0, t = 0;
         bool ok = true;
-        for (int kb = 0; kb < num_kb && ok; ++kb) {
-            const int s = kb % kStages;
-            ok = mbar_wait(&ctl->full[s], (kb / kStages) & 1, &ctl->abort, p.status);
-            if (!ok) break;
-            const uint8_t* st = tiles + s * kStageBytes;
-            const uint32_t sfa = tmem + ((uint32_t)(q * 32) << 16) + kTmemSf + s * C_::kSfCols, sfb = sfa + C_::kSfColsA;
+        for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t) {
+            const int64_t m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
+            int* w_exp = ctl->w_exp[t & 1];
+            for (int i = threadIdx.x - 64; i < BN; i += kEpilogueWarps * 32) w_exp[i] = (n0 + i < p.N) ? p.w_exp[n0 + i] : 0;
+            if (sf_warp) {
+                for (int kb = 0; kb < num_kb && ok; ++kb, ++it) {
+                    const int s = it % kStages;
+                    ok = mbar_wait(&ctl->full[s], (it / kStages) & 1, &ctl->abort, p.status);
+                    if (!ok) break;
+                    const uint8_t* st = tiles + s * kStageBytes;
+                    const uint32_t sfa = tmem + ((uint32_t)(q * 32) << 16) + kTmemSf + s * C_::kSfCols, sfb = sfa + C_::kSfColsA;
 #pragma unroll
-            for (int pl = 0; pl < 2; ++pl)
+                    for (int pl = 0; pl < 2; ++pl)
 #pragma unroll
-                for (int kk = 0; kk < kSteps; ++kk) {
-                    const uint4 a = *reinterpret_cast<const uint4*>(st + C_::kOffSfA + pl * kSfA + kk * kSfChunk + lane * 16);
-                    tmem_st4(sfa + (pl * kSteps + kk) * 4, a.x, a.y, a.z, a.w);
+                        for (int kk = 0; kk < kSteps; ++kk) {
+                            const uint4 a = *reinterpret_cast<const uint4*>(st + C_::kOffSfA + pl * kSfA + kk * kSfChunk + lane * 16);
+                            tmem_st4(sfa + (pl * kSteps + kk) * 4, a.x, a.y, a.z, a.w);
 #pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        const uint4 b = *reinterpret_cast<const uint4*>(st + C_::kOffSfB + pl * kSfB + j * kSfA + kk * kSfChunk + lane * 16);
-                        tmem_st4(sfb + (pl * kSteps + kk) * 8 + j * 4, b.x, b.y, b.z, b.w);
-                    }
+                            for (int j = 0; j < 2; ++j) {
+                                const uint4 b = *reinterpret_cast<const uint4*>(st + C_::kOffSfB + pl * kSfB + j * kSfA + kk * kSfChunk + lane * 16);
+                                tmem_st4(sfb + (pl * kSteps + kk) * 8 + j * 4, b.x, b.y, b.z, b.w);
+                            }
+                        }
+                    tmem_st_wait();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&ctl->sf_full[s]);
                 }
-            tmem_st_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&ctl->sf_full[s]);
-        }
-        if (ok) ok = mbar_wait(&ctl->accum, 0, &ctl->abort, p.status);
-        tc_fence_after();
-        if (ok) {
-            const int64_t m = m0 + q * 32 + lane;
-            const int a_exp = (m < p.M) ? p.a_exp[m] : 0;
+            }
+            if (ok) ok = mbar_wait(&ctl->accum_full, t & 1, &ctl->abort, p.status);
+            tc_fence_after();
+            // all epilogue warps have written their part of w_exp (a named barrier: the producer and
+            // MMA warps do not take part)
+            asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueWarps * 32) : "memory");
+            if (ok) {
+                const int64_t m = m0 + q * 32 + lane;
+                const int a_exp = (m < p.M) ? p.a_exp[m] : 0;
 #pragma unroll 1
-            for (int col = 0; col < BN; col += 32) {
-                uint32_t v[32];
-                tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)col, v);
-                tmem_ld_wait();
-                if (m < p.M) {
-                    float* out = p.C + m * p.ld_c + n0 + col;
-                    float f[32];
+                for (int c = 0; c < BN / 2; c += 32) {
+                    const int col = col_base + c;
+                    uint32_t v[32];
+                    tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)col, v);
+                    tmem_ld_wait();
+                    if (m < p.M) {
+                        float* out = p.C + m * p.ld_c + n0 + col;
+                        float f[32];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int e = min(127, max(-126, a_exp + ctl->w_exp[col + j]));
-                        f[j] = __uint_as_float(v[j]) * __uint_as_float((uint32_t)(e + 127) << 23);
-                    }
-                    if (p.vec_store && n0 + col + 32 <= p.N) {
+                        for (int j = 0; j < 32; ++j) {
+                            const int e = min(127, max(-126, a_exp + w_exp[col + j]));
+                            f[j] = __uint_as_float(v[j]) * __uint_as_float((uint32_t)(e + 127) << 23);
+                        }
+                        if (p.vec_store && n0 + col + 32 <= p.N) {
 #pragma unroll
-                        for (int j = 0; j < 32; j += 4)
-                            *reinterpret_cast<float4*>(out + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
-                    } else {
+                            for (int j = 0; j < 32; j += 4)
+                                *reinterpret_cast<float4*>(out + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
+                        } else {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (n0 + col + j < p.N) out[j] = f[j];
+                            for (int j = 0; j < 32; ++j)
+                                if (n0 + col + j < p.N) out[j] = f[j];
+                        }
                     }
                 }
+                // this warp's part of the accumulator has been read: the next tile may overwrite it
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->accum_empty);
             }
         }
     }
@@ -438,7 +473,11 @@ int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, co
     if (!make_map(&tm_ap, pa, p.M, p.K, BM, C_::kRowBytes) || !make_map(&tm_an, pa + oa.plane, p.M, p.K, BM, C_::kRowBytes) ||
         !make_map(&tm_wp, pw, p.N, p.K, BN, C_::kRowBytes) || !make_map(&tm_wn, pw + ow.plane, p.N, p.K, BN, C_::kRowBytes))
         return AMX_ERR_CUDA;
-    dim3 grid((unsigned)((p.N + BN - 1) / BN), (unsigned)((p.M + BM - 1) / BM));
+    static int sm_count[64] = {};
+    if (!sm_count[dev] && cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return AMX_ERR_CUDA;
+    const int64_t tiles = ((p.N + BN - 1) / BN) * ((p.M + BM - 1) / BM);
+    const unsigned grid = (unsigned)(tiles < sm_count[dev] ? tiles : sm_count[dev]);   // one persistent CTA per SM
     gemm_fp4_kernel<BK_><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_ap, tm_an, tm_wp, tm_wn, p);
     return launch_status();
 }
