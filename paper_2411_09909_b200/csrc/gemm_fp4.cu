@@ -211,7 +211,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&ctl->full[s], 1);
-            mbar_init(&ctl->sf_full[s], 4);
+            mbar_init(&ctl->sf_full[s], kEpilogueWarps);
             mbar_init(&ctl->empty[s], 1);
         }
         mbar_init(&ctl->accum_full, 1);
@@ -295,11 +295,11 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant
         }
     } else {
         // ------------------------------------------------ scale factors and epilogue
-        // Warps 2..5 own one 32-lane quarter of tensor memory each.  Per stage they read the stage's
-        // scale-factor blocks from shared memory (16 bytes per lane and block: the 4-byte scale words of
-        // rows lane, lane+32, lane+64, lane+96) and store them into their quarter's copy of the
-        // scale-factor columns (every quarter has to hold one).  Warps 6..9 only help with the epilogue:
-        // quarter q = warp % 4 again, the other half of the columns.
+        // Warp w works on the 32-lane quarter w % 4 of tensor memory.  Per stage it reads scale-factor
+        // blocks from shared memory (16 bytes per lane and block: the 4-byte scale words of rows lane,
+        // lane+32, lane+64, lane+96) and stores them into its quarter's copy of the scale-factor columns
+        // (every quarter has to hold one): warps 2..5 the positive planes', warps 6..9 the negative
+        // planes'.  In the epilogue the two warps of a quarter take one half of the columns each.
         const int q = warp & 3;
         const bool sf_warp = warp < 2 + 4;
         const int col_base = sf_warp ? 0 : BN / 2;
@@ -309,15 +309,14 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant
             const int64_t m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
             int* w_exp = ctl->w_exp[t & 1];
             for (int i = threadIdx.x - 64; i < BN; i += kEpilogueWarps * 32) w_exp[i] = (n0 + i < p.N) ? p.w_exp[n0 + i] : 0;
-            if (sf_warp) {
+            {
+                const int pl = sf_warp ? 0 : 1;                  // warps 2..5: positive planes, warps 6..9: negative
                 for (int kb = 0; kb < num_kb && ok; ++kb, ++it) {
                     const int s = it % kStages;
                     ok = mbar_wait(&ctl->full[s], (it / kStages) & 1, &ctl->abort, p.status);
                     if (!ok) break;
                     const uint8_t* st = tiles + s * kStageBytes;
                     const uint32_t sfa = tmem + ((uint32_t)(q * 32) << 16) + kTmemSf + s * C_::kSfCols, sfb = sfa + C_::kSfColsA;
-#pragma unroll
-                    for (int pl = 0; pl < 2; ++pl)
 #pragma unroll
                         for (int kk = 0; kk < kSteps; ++kk) {
                             const uint4 a = *reinterpret_cast<const uint4*>(st + C_::kOffSfA + pl * kSfA + kk * kSfChunk + lane * 16);
