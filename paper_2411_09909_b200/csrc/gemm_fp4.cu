@@ -21,10 +21,11 @@
 //   warp 1   allocates TMEM; one lane issues the stage's MMAs (4 sign pairs x K steps of 64), then
 //            commits to the stage's `empty` mbarrier
 //   warps 2-5  move each stage's scale factors shared -> registers -> tensor memory (tcgen05.st; this
-//            keeps the copies off the in-order MMA queue), signal `sf_full`; afterwards they are the
-//            epilogue: TMEM -> registers, power-of-two rescale, fp32 stores
-//   warps 6-9  epilogue only (the other half of the columns).  While a tile's accumulator is read out the
-//            producer already prefetches the next tile's stages; the MMA issuer waits for `accum_empty`.
+//            keeps the copies off the in-order MMA queue) and signal `sf_full`; they follow only the
+//            `full` barriers and so run ahead into the next tile
+//   warps 6-13 epilogue: TMEM -> registers (double-buffered loads), power-of-two rescale, 32-byte fp32
+//            stores.  While a tile's accumulator is read out the producer already prefetches the next
+//            tile's stages; the MMA issuer waits for `accum_empty`.
 // A preparation pass (two small kernels per operand) derives the planes, the UE4M3 scale-factor
 // blocks in the 128 x 4 interleaved layout the MMA reads, and the row offsets from the canonical
 // codes and scales.  Every device-side wait is bounded.
@@ -42,8 +43,8 @@ namespace {
 using namespace tc;
 
 constexpr int BM = 128, BN = 256;
-constexpr int kEpilogueWarps = 8;
-constexpr int kThreads = (2 + kEpilogueWarps) * 32;
+constexpr int kSfWarps = 4, kEpilogueWarps = 8;
+constexpr int kThreads = (2 + kSfWarps + kEpilogueWarps) * 32;
 constexpr int kSfChunk = 512;           // scale factors of 128 rows x 64 elements (4 per row)
 constexpr int kTmemCols = 512;
 constexpr uint32_t kTmemSf = 256;      // scale-factor columns follow the 256 accumulator columns
@@ -74,7 +75,7 @@ struct __align__(8) Control {
     uint64_t full[kMaxStages], sf_full[kMaxStages], empty[kMaxStages], accum_full, accum_empty;
     uint32_t tmem_base;
     volatile int abort;
-    int w_exp[2][BN];
+    alignas(16) int w_exp[2][BN];   // read as int4 in the epilogue
 };
 static_assert(sizeof(Control) <= 2048 + 256, "Control must fit its reserved space");
 
@@ -193,6 +194,20 @@ struct Params {
     int* status;
 };
 
+// 32 consecutive fp32 results of one row -> global memory, as four 32-byte stores when allowed.
+__device__ __forceinline__ void store_row32(float* out, const float (&f)[32], bool vec, int64_t n_left) {
+    if (vec && n_left >= 32) {
+#pragma unroll
+        for (int j = 0; j < 32; j += 8)
+            asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(out + j), "f"(f[j]), "f"(f[j + 1]),
+                         "f"(f[j + 2]), "f"(f[j + 3]), "f"(f[j + 4]), "f"(f[j + 5]), "f"(f[j + 6]), "f"(f[j + 7]) : "memory");
+    } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+            if (j < n_left) out[j] = f[j];
+    }
+}
+
 template <int BK_>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant__ CUtensorMap tm_an,
@@ -211,7 +226,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&ctl->full[s], 1);
-            mbar_init(&ctl->sf_full[s], kEpilogueWarps);
+            mbar_init(&ctl->sf_full[s], kSfWarps);
             mbar_init(&ctl->empty[s], 1);
         }
         mbar_init(&ctl->accum_full, 1);
@@ -264,107 +279,115 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer
         if (lane == 0) {
+            // All operand descriptors differ from the first stage's only in their 14-bit address field
+            // (bytes >> 4); the per-stage, per-plane, per-K-step offsets below are compile-time constants.
+            const uint64_t desc0 = operand_desc<BK_>(smem_u32(tiles));
             int it = 0, t = 0;
             bool ok = true;
             for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t) {
                 // the previous tile's accumulator must have been read out before it is overwritten
                 if (t > 0) ok = mbar_wait(&ctl->accum_empty, (t - 1) & 1, &ctl->abort, p.status);
                 tc_fence_after();
+                uint32_t accumulate = 0;
                 for (int kb = 0; kb < num_kb && ok; ++kb, ++it) {
                     const int s = it % kStages;
                     ok = mbar_wait(&ctl->full[s], (it / kStages) & 1, &ctl->abort, p.status) &&
                          mbar_wait(&ctl->sf_full[s], (it / kStages) & 1, &ctl->abort, p.status);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t st = smem_u32(tiles + s * kStageBytes);
+                    const uint64_t dstage = desc0 + (uint64_t)((s * kStageBytes) >> 4);
                     const uint32_t sfa = tmem + kTmemSf + s * C_::kSfCols, sfb = sfa + C_::kSfColsA;
 #pragma unroll
                     for (int pa = 0; pa < 2; ++pa)
 #pragma unroll
                         for (int pw = 0; pw < 2; ++pw)
 #pragma unroll
-                            for (int kk = 0; kk < kSteps; ++kk)  // 64 elements = 32 bytes along the swizzled row
-                                mma_fp4_block16(tmem, operand_desc<BK_>(st + (pa ? C_::kOffAn : C_::kOffAp) + kk * 32),
-                                                operand_desc<BK_>(st + (pw ? C_::kOffWn : C_::kOffWp) + kk * 32), kIdesc,
-                                                sfa + (pa * kSteps + kk) * 4, sfb + (pw * kSteps + kk) * 8,
-                                                (kb | pa | pw | kk) ? 1u : 0u);
+                            for (int kk = 0; kk < kSteps; ++kk) {   // 64 elements = 32 bytes along the swizzled row
+                                mma_fp4_block16(tmem, dstage + (((pa ? C_::kOffAn : C_::kOffAp) + kk * 32) >> 4),
+                                                dstage + (((pw ? C_::kOffWn : C_::kOffWp) + kk * 32) >> 4), kIdesc,
+                                                sfa + (pa * kSteps + kk) * 4, sfb + (pw * kSteps + kk) * 8, accumulate);
+                                accumulate = 1;
+                            }
                     mma_commit(&ctl->empty[s]);
                 }
                 if (ok) mma_commit(&ctl->accum_full);
             }
         }
-    } else {
-        // ------------------------------------------------ scale factors and epilogue
-        // Warp w works on the 32-lane quarter w % 4 of tensor memory.  Per stage it reads scale-factor
-        // blocks from shared memory (16 bytes per lane and block: the 4-byte scale words of rows lane,
-        // lane+32, lane+64, lane+96) and stores them into its quarter's copy of the scale-factor columns
-        // (every quarter has to hold one): warps 2..5 the positive planes', warps 6..9 the negative
-        // planes'.  In the epilogue the two warps of a quarter take one half of the columns each.
+    } else if (warp < 2 + kSfWarps) {
+        // -------------------------------------------------------------- scale factors
+        // Warp w serves the 32-lane quarter w % 4 of tensor memory.  Per stage it reads the stage's
+        // scale-factor blocks from shared memory (16 bytes per lane and block: the 4-byte scale words of
+        // rows lane, lane+32, lane+64, lane+96) and stores them into its quarter's copy of the
+        // scale-factor columns (every quarter has to hold one).  These warps only follow the `full`
+        // barriers, so they run ahead into the next tile while the epilogue drains the accumulator.
         const int q = warp & 3;
-        const bool sf_warp = warp < 2 + 4;
-        const int col_base = sf_warp ? 0 : BN / 2;
-        int it = 0, t = 0;
+        int it = 0;
+        bool ok = true;
+        for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            for (int kb = 0; kb < num_kb && ok; ++kb, ++it) {
+                const int s = it % kStages;
+                ok = mbar_wait(&ctl->full[s], (it / kStages) & 1, &ctl->abort, p.status);
+                if (!ok) break;
+                const uint8_t* st = tiles + s * kStageBytes;
+                const uint32_t sfa = tmem + ((uint32_t)(q * 32) << 16) + kTmemSf + s * C_::kSfCols, sfb = sfa + C_::kSfColsA;
+#pragma unroll
+                for (int pl = 0; pl < 2; ++pl)
+#pragma unroll
+                    for (int kk = 0; kk < kSteps; ++kk) {
+                        const uint4 a = *reinterpret_cast<const uint4*>(st + C_::kOffSfA + pl * kSfA + kk * kSfChunk + lane * 16);
+                        tmem_st4(sfa + (pl * kSteps + kk) * 4, a.x, a.y, a.z, a.w);
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {
+                            const uint4 b = *reinterpret_cast<const uint4*>(st + C_::kOffSfB + pl * kSfB + j * kSfA + kk * kSfChunk + lane * 16);
+                            tmem_st4(sfb + (pl * kSteps + kk) * 8 + j * 4, b.x, b.y, b.z, b.w);
+                        }
+                    }
+                tmem_st_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->sf_full[s]);
+            }
+        }
+    } else {
+        // -------------------------------------------------------------- epilogue
+        // Eight warps: quarter q = warp % 4 of the lanes (= rows), one half of the columns each.
+        const int e = warp - (2 + kSfWarps);                     // 0..7
+        const int q = warp & 3, col_base = (e >> 2) * (BN / 2);
+        const int tid_e = threadIdx.x - (2 + kSfWarps) * 32;
+        int t = 0;
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t) {
             const int64_t m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
             int* w_exp = ctl->w_exp[t & 1];
-            for (int i = threadIdx.x - 64; i < BN; i += kEpilogueWarps * 32) w_exp[i] = (n0 + i < p.N) ? p.w_exp[n0 + i] : 0;
-            {
-                const int pl = sf_warp ? 0 : 1;                  // warps 2..5: positive planes, warps 6..9: negative
-                for (int kb = 0; kb < num_kb && ok; ++kb, ++it) {
-                    const int s = it % kStages;
-                    ok = mbar_wait(&ctl->full[s], (it / kStages) & 1, &ctl->abort, p.status);
-                    if (!ok) break;
-                    const uint8_t* st = tiles + s * kStageBytes;
-                    const uint32_t sfa = tmem + ((uint32_t)(q * 32) << 16) + kTmemSf + s * C_::kSfCols, sfb = sfa + C_::kSfColsA;
-#pragma unroll
-                        for (int kk = 0; kk < kSteps; ++kk) {
-                            const uint4 a = *reinterpret_cast<const uint4*>(st + C_::kOffSfA + pl * kSfA + kk * kSfChunk + lane * 16);
-                            tmem_st4(sfa + (pl * kSteps + kk) * 4, a.x, a.y, a.z, a.w);
-#pragma unroll
-                            for (int j = 0; j < 2; ++j) {
-                                const uint4 b = *reinterpret_cast<const uint4*>(st + C_::kOffSfB + pl * kSfB + j * kSfA + kk * kSfChunk + lane * 16);
-                                tmem_st4(sfb + (pl * kSteps + kk) * 8 + j * 4, b.x, b.y, b.z, b.w);
-                            }
-                        }
-                    tmem_st_wait();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&ctl->sf_full[s]);
-                }
-            }
-            if (ok) ok = mbar_wait(&ctl->accum_full, t & 1, &ctl->abort, p.status);
+            for (int i = tid_e; i < BN; i += kEpilogueWarps * 32) w_exp[i] = (n0 + i < p.N) ? p.w_exp[n0 + i] : 0;
+            const int64_t m = m0 + q * 32 + lane;
+            const int a_exp = (m < p.M) ? p.a_exp[m] : 0;
+            ok = mbar_wait(&ctl->accum_full, t & 1, &ctl->abort, p.status);
             tc_fence_after();
-            // all epilogue warps have written their part of w_exp (a named barrier: the producer and
-            // MMA warps do not take part)
+            // every epilogue warp has written its part of w_exp (named barrier: the other roles do not join)
             asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueWarps * 32) : "memory");
             if (ok) {
-                const int64_t m = m0 + q * 32 + lane;
-                const int a_exp = (m < p.M) ? p.a_exp[m] : 0;
-#pragma unroll 1
+                const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)col_base;
+                uint32_t v[2][32];
+                tmem_ld32(taddr, v[0]);
+#pragma unroll
                 for (int c = 0; c < BN / 2; c += 32) {
-                    const int col = col_base + c;
-                    uint32_t v[32];
-                    tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)col, v);
+                    const int buf = (c / 32) & 1;
                     tmem_ld_wait();
-                    if (m < p.M) {
-                        float* out = p.C + m * p.ld_c + n0 + col;
-                        float f[32];
+                    if (c + 32 < BN / 2) tmem_ld32(taddr + c + 32, v[buf ^ 1]);   // next chunk loads while this one is stored
+                    const int col = col_base + c;
+                    float f[32];
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            const int e = min(127, max(-126, a_exp + w_exp[col + j]));
-                            f[j] = __uint_as_float(v[j]) * __uint_as_float((uint32_t)(e + 127) << 23);
-                        }
-                        if (p.vec_store && n0 + col + 32 <= p.N) {
+                    for (int j = 0; j < 32; j += 4) {
+                        const int4 we = *reinterpret_cast<const int4*>(&w_exp[col + j]);
+                        const int ex[4] = {we.x, we.y, we.z, we.w};
 #pragma unroll
-                            for (int j = 0; j < 32; j += 4)
-                                *reinterpret_cast<float4*>(out + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (n0 + col + j < p.N) out[j] = f[j];
+                        for (int i = 0; i < 4; ++i) {
+                            const int sh = min(127, max(-126, a_exp + ex[i]));
+                            f[j + i] = __uint_as_float(v[buf][j + i]) * __uint_as_float((uint32_t)(sh + 127) << 23);
                         }
                     }
+                    if (m < p.M) store_row32(p.C + m * p.ld_c + n0 + col, f, p.vec_store != 0, p.N - (n0 + col));
                 }
                 // this warp's part of the accumulator has been read: the next tile may overwrite it
                 tc_fence_before();
@@ -514,7 +537,7 @@ int gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_c
     p.w_exp = reinterpret_cast<const int*>(pw + 2 * ow.plane + 2 * ow.sf);
     p.M = M; p.N = N; p.K = K; p.ld_c = ld_c; p.C = C;
     p.nk64 = oa.nk64;
-    p.vec_store = aligned(C, 16) && ld_c % 4 == 0;
+    p.vec_store = aligned(C, 32) && ld_c % 8 == 0;     // 32-byte stores in the epilogue
     p.status = status;
     return fp4_block_k() == 256 ? launch_fp4<256>(pa, pw, oa, ow, p, dev, st) : launch_fp4<128>(pa, pw, oa, ow, p, dev, st);
 }
