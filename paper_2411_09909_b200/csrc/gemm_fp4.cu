@@ -20,10 +20,10 @@
 //            blocks (plain bulk copies) per stage, completion on the stage's `full` mbarrier
 //   warp 1   allocates TMEM; one lane issues the stage's MMAs (4 sign pairs x K steps of 64), then
 //            commits to the stage's `empty` mbarrier
-//   warps 2-5  move each stage's scale factors shared -> registers -> tensor memory (tcgen05.st; this
+//   warps 2-9  (two groups of four, alternating K blocks) move each stage's scale factors shared -> registers -> tensor memory (tcgen05.st; this
 //            keeps the copies off the in-order MMA queue) and signal `sf_full`; they follow only the
 //            `full` barriers and so run ahead into the next tile
-//   warps 6-13 epilogue: TMEM -> registers (double-buffered loads), power-of-two rescale, 32-byte fp32
+//   warps 10-17 epilogue: TMEM -> registers (double-buffered loads), power-of-two rescale, 32-byte fp32
 //            stores.  While a tile's accumulator is read out the producer already prefetches the next
 //            tile's stages; the MMA issuer waits for `accum_empty`.
 // A preparation pass (two small kernels per operand) derives the planes, the UE4M3 scale-factor
@@ -43,7 +43,7 @@ namespace {
 using namespace tc;
 
 constexpr int BM = 128, BN = 256;
-constexpr int kSfWarps = 4, kEpilogueWarps = 8;
+constexpr int kSfGroups = 2, kSfWarps = 4 * kSfGroups, kEpilogueWarps = 8;
 constexpr int kThreads = (2 + kSfWarps + kEpilogueWarps) * 32;
 constexpr int kSfChunk = 512;           // scale factors of 128 rows x 64 elements (4 per row)
 constexpr int kTmemCols = 512;
@@ -71,7 +71,7 @@ struct Cfg {
 };
 constexpr int kMaxStages = 4;
 
-struct __align__(8) Control {
+struct __align__(16) Control {
     uint64_t full[kMaxStages], sf_full[kMaxStages], empty[kMaxStages], accum_full, accum_empty;
     uint32_t tmem_base;
     volatile int abort;
@@ -194,16 +194,16 @@ struct Params {
     int* status;
 };
 
-// 32 consecutive fp32 results of one row -> global memory, as four 32-byte stores when allowed.
-__device__ __forceinline__ void store_row32(float* out, const float (&f)[32], bool vec, int64_t n_left) {
-    if (vec && n_left >= 32) {
+// 16 consecutive fp32 results of one row -> global memory, as two 32-byte stores when allowed.
+__device__ __forceinline__ void store_row16(float* out, const float (&f)[16], bool vec, int64_t n_left) {
+    if (vec && n_left >= 16) {
 #pragma unroll
-        for (int j = 0; j < 32; j += 8)
+        for (int j = 0; j < 16; j += 8)
             asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(out + j), "f"(f[j]), "f"(f[j + 1]),
                          "f"(f[j + 2]), "f"(f[j + 3]), "f"(f[j + 4]), "f"(f[j + 5]), "f"(f[j + 6]), "f"(f[j + 7]) : "memory");
     } else {
 #pragma unroll
-        for (int j = 0; j < 32; ++j)
+        for (int j = 0; j < 16; ++j)
             if (j < n_left) out[j] = f[j];
     }
 }
@@ -226,7 +226,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&ctl->full[s], 1);
-            mbar_init(&ctl->sf_full[s], kSfWarps);
+            mbar_init(&ctl->sf_full[s], 4);
             mbar_init(&ctl->empty[s], 1);
         }
         mbar_init(&ctl->accum_full, 1);
@@ -320,11 +320,14 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant
         // rows lane, lane+32, lane+64, lane+96) and stores them into its quarter's copy of the
         // scale-factor columns (every quarter has to hold one).  These warps only follow the `full`
         // barriers, so they run ahead into the next tile while the epilogue drains the accumulator.
-        const int q = warp & 3;
+        // Two groups of four warps take alternate K blocks: the register round trip of one block
+        // (loads, tcgen05.st, wait) then overlaps the other group's.
+        const int q = warp & 3, group = (warp - 2) >> 2;
         int it = 0;
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
             for (int kb = 0; kb < num_kb && ok; ++kb, ++it) {
+                if ((it % kSfGroups) != group) continue;
                 const int s = it % kStages;
                 ok = mbar_wait(&ctl->full[s], (it / kStages) & 1, &ctl->abort, p.status);
                 if (!ok) break;
@@ -368,17 +371,17 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant
             asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueWarps * 32) : "memory");
             if (ok) {
                 const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)col_base;
-                uint32_t v[2][32];
-                tmem_ld32(taddr, v[0]);
+                uint32_t v[2][16];
+                tmem_ld16(taddr, v[0]);
 #pragma unroll
-                for (int c = 0; c < BN / 2; c += 32) {
-                    const int buf = (c / 32) & 1;
+                for (int c = 0; c < BN / 2; c += 16) {
+                    const int buf = (c / 16) & 1;
                     tmem_ld_wait();
-                    if (c + 32 < BN / 2) tmem_ld32(taddr + c + 32, v[buf ^ 1]);   // next chunk loads while this one is stored
+                    if (c + 16 < BN / 2) tmem_ld16(taddr + c + 16, v[buf ^ 1]);   // next chunk loads while this one is stored
                     const int col = col_base + c;
-                    float f[32];
+                    float f[16];
 #pragma unroll
-                    for (int j = 0; j < 32; j += 4) {
+                    for (int j = 0; j < 16; j += 4) {
                         const int4 we = *reinterpret_cast<const int4*>(&w_exp[col + j]);
                         const int ex[4] = {we.x, we.y, we.z, we.w};
 #pragma unroll
@@ -387,7 +390,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant
                             f[j + i] = __uint_as_float(v[buf][j + i]) * __uint_as_float((uint32_t)(sh + 127) << 23);
                         }
                     }
-                    if (m < p.M) store_row32(p.C + m * p.ld_c + n0 + col, f, p.vec_store != 0, p.N - (n0 + col));
+                    if (m < p.M) store_row16(p.C + m * p.ld_c + n0 + col, f, p.vec_store != 0, p.N - (n0 + col));
                 }
                 // this warp's part of the accumulator has been read: the next tile may overwrite it
                 tc_fence_before();
