@@ -16,12 +16,12 @@
 //
 // Persistent CTAs (one per SM) walk over 128 x 256 tiles of C; K blocks of 128 elements cycle through
 // four 54 KB shared-memory stages (two 108 KB stages with 256-element blocks):
-//   warp 0   TMA producer: four 128-byte-swizzled code tiles (A+, A-, W+, W-) and the scale-factor
-//            blocks (plain bulk copies) per stage, completion on the stage's `full` mbarrier
+//   warp 0   TMA producer: per stage one 3-D tile {A+, A-} and one {W+, W-} (64- or 128-byte swizzle),
+//            completion on the stage's `full` mbarrier
 //   warp 1   allocates TMEM; one lane issues the stage's MMAs (4 sign pairs x K steps of 64), then
 //            commits to the stage's `empty` mbarrier
 //   warps 2-9  (two groups of four, alternating K blocks) move each stage's scale factors shared -> registers -> tensor memory (tcgen05.st; this
-//            keeps the copies off the in-order MMA queue) and signal `sf_full`; they follow only the
+//            keeps the copies off the in-order MMA queue) and arrive on the stage's `full` barrier; they follow only the
 //            `full` barriers and so run ahead into the next tile
 //   warps 10-17 epilogue: TMEM -> registers (double-buffered loads), power-of-two rescale, 32-byte fp32
 //            stores.  While a tile's accumulator is read out the producer already prefetches the next
@@ -50,8 +50,8 @@ constexpr int kTmemCols = 512;
 constexpr uint32_t kTmemSf = 256;      // scale-factor columns follow the 256 accumulator columns
 
 // Shared-memory stage geometry for a K block of BK elements (BK/2 bytes of codes per row and plane).
-// BK = 256: 128-byte rows, 128-byte swizzle, 2 stages of 108 KB.
-// BK = 128:  64-byte rows,  64-byte swizzle, 4 stages of  54 KB (finer-grained prefetch).
+// BK = 256: 128-byte rows, 128-byte swizzle, 2 stages of 96 KB.
+// BK = 128:  64-byte rows,  64-byte swizzle, 4 stages of 48 KB (finer-grained prefetch).
 template <int BK_>
 struct Cfg {
     static constexpr int BK = BK_;
@@ -59,11 +59,8 @@ struct Cfg {
     static constexpr int kSteps = BK / 64;                            // MMAs (K = 64) per K block and sign pair
     static constexpr int kStages = BK == 256 ? 2 : 4;
     static constexpr int kTileA = BM * kRowBytes, kTileB = BN * kRowBytes;   // one plane
-    static constexpr int kSfA = kSteps * kSfChunk;                    // one plane, one K block, 128 rows
-    static constexpr int kSfB = 2 * kSfA;                             // 256 rows
     static constexpr int kOffAp = 0, kOffAn = kTileA, kOffWp = 2 * kTileA, kOffWn = 2 * kTileA + kTileB;
-    static constexpr int kOffSfA = 2 * kTileA + 2 * kTileB, kOffSfB = kOffSfA + 2 * kSfA;
-    static constexpr int kStageBytes = kOffSfB + 2 * kSfB;
+    static constexpr int kStageBytes = 2 * kTileA + 2 * kTileB;       // {A+, A-} and {W+, W-}: one TMA each
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 2048 + 256;   // + alignment slack + Control
     // TMEM columns of one stage's scale factors: A planes (4 columns per K step), then W planes (8)
     static constexpr int kSfColsA = 2 * kSteps * 4, kSfCols = kSfColsA + 2 * kSteps * 8;
@@ -72,7 +69,7 @@ struct Cfg {
 constexpr int kMaxStages = 4;
 
 struct __align__(16) Control {
-    uint64_t full[kMaxStages], sf_full[kMaxStages], empty[kMaxStages], accum_full, accum_empty;
+    uint64_t full[kMaxStages], empty[kMaxStages], accum_full, accum_empty;
     uint32_t tmem_base;
     volatile int abort;
     alignas(16) int w_exp[2][BN];   // read as int4 in the epilogue
@@ -210,11 +207,10 @@ __device__ __forceinline__ void store_row16(float* out, const float (&f)[16], bo
 
 template <int BK_>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant__ CUtensorMap tm_an,
-                const __grid_constant__ CUtensorMap tm_wp, const __grid_constant__ CUtensorMap tm_wn, const Params p) {
+gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w, const Params p) {
     using C_ = Cfg<BK_>;
     constexpr int BK = C_::BK, kRowBytes = C_::kRowBytes, kSteps = C_::kSteps, kStages = C_::kStages;
-    constexpr int kStageBytes = C_::kStageBytes, kSfA = C_::kSfA, kSfB = C_::kSfB;
+    constexpr int kStageBytes = C_::kStageBytes;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     Control* ctl = reinterpret_cast<Control*>(tiles + kStages * kStageBytes);
@@ -225,8 +221,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(&ctl->full[s], 1);
-            mbar_init(&ctl->sf_full[s], 4);
+            mbar_init(&ctl->full[s], 1 + 4);               // producer (with the TMA byte count) + four scale-factor warps
             mbar_init(&ctl->empty[s], 1);
         }
         mbar_init(&ctl->accum_full, 1);
@@ -255,20 +250,9 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant
                     }
                     uint8_t* st = tiles + s * kStageBytes;
                     mbar_expect_tx(&ctl->full[s], kStageBytes);
-                    const int x = kb * kRowBytes;
-                    tma_load_2d(st + C_::kOffAp, &tm_ap, x, (int)(m_blk * BM), &ctl->full[s]);
-                    tma_load_2d(st + C_::kOffAn, &tm_an, x, (int)(m_blk * BM), &ctl->full[s]);
-                    tma_load_2d(st + C_::kOffWp, &tm_wp, x, (int)(n_blk * BN), &ctl->full[s]);
-                    tma_load_2d(st + C_::kOffWn, &tm_wn, x, (int)(n_blk * BN), &ctl->full[s]);
-                    const int64_t a_off = (m_blk * p.nk64 + kb * kSteps) * kSfChunk;
-                    bulk_load(st + C_::kOffSfA, p.sfa_pos + a_off, kSfA, &ctl->full[s]);
-                    bulk_load(st + C_::kOffSfA + kSfA, p.sfa_neg + a_off, kSfA, &ctl->full[s]);
-#pragma unroll
-                    for (int j = 0; j < 2; ++j) {                // the tile's two 128-row blocks of W
-                        const int64_t w_off = ((n_blk * 2 + j) * p.nk64 + kb * kSteps) * kSfChunk;
-                        bulk_load(st + C_::kOffSfB + j * kSfA, p.sfb_pos + w_off, kSfA, &ctl->full[s]);
-                        bulk_load(st + C_::kOffSfB + kSfB + j * kSfA, p.sfb_neg + w_off, kSfA, &ctl->full[s]);
-                    }
+                    // one 3-D tile per operand: {row bytes, rows, both sign planes}
+                    tma_load_3d(st + C_::kOffAp, &tm_a, kb * kRowBytes, (int)(m_blk * BM), 0, &ctl->full[s]);
+                    tma_load_3d(st + C_::kOffWp, &tm_w, kb * kRowBytes, (int)(n_blk * BN), 0, &ctl->full[s]);
                 }
             }
             // after an abort: let the copies already in flight land before shared memory is released
@@ -278,78 +262,99 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_ap, const __grid_constant
         }
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
-            // All operand descriptors differ from the first stage's only in their 14-bit address field
-            // (bytes >> 4); the per-stage, per-plane, per-K-step offsets below are compile-time constants.
-            const uint64_t desc0 = operand_desc<BK_>(smem_u32(tiles));
-            int it = 0, t = 0;
-            bool ok = true;
-            for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t) {
-                // the previous tile's accumulator must have been read out before it is overwritten
-                if (t > 0) ok = mbar_wait(&ctl->accum_empty, (t - 1) & 1, &ctl->abort, p.status);
+        // The whole warp runs the loop (so that addresses and descriptors stay warp-uniform); one elected
+        // lane issues.  All operand descriptors differ from the first stage's only in their 14-bit address
+        // field (bytes >> 4); the per-plane and per-K-step offsets are compile-time constants.
+        const uint64_t desc0 = operand_desc<BK_>(smem_u32(tiles));
+        int it = 0, t = 0;
+        bool ok = true;
+        for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t) {
+            // the previous tile's accumulator must have been read out before it is overwritten
+            if (t > 0) ok = mbar_wait(&ctl->accum_empty, (t - 1) & 1, &ctl->abort, p.status);
+            tc_fence_after();
+            uint32_t accumulate = 0;
+            for (int kb = 0; kb < num_kb && ok; ++kb, ++it) {
+                const int s = it % kStages;
+                // tiles landed (TMA byte count) and scale factors stored (four warp arrivals)
+                ok = mbar_wait(&ctl->full[s], (it / kStages) & 1, &ctl->abort, p.status);
+                if (!ok) break;
                 tc_fence_after();
-                uint32_t accumulate = 0;
-                for (int kb = 0; kb < num_kb && ok; ++kb, ++it) {
-                    const int s = it % kStages;
-                    ok = mbar_wait(&ctl->full[s], (it / kStages) & 1, &ctl->abort, p.status) &&
-                         mbar_wait(&ctl->sf_full[s], (it / kStages) & 1, &ctl->abort, p.status);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint64_t dstage = desc0 + (uint64_t)((s * kStageBytes) >> 4);
-                    const uint32_t sfa = tmem + kTmemSf + s * C_::kSfCols, sfb = sfa + C_::kSfColsA;
+                const uint64_t dstage = desc0 + (uint64_t)((s * kStageBytes) >> 4);
+                const uint32_t sfa = tmem + kTmemSf + s * C_::kSfCols, sfb = sfa + C_::kSfColsA;
+                if (elect_one()) {
 #pragma unroll
                     for (int pa = 0; pa < 2; ++pa)
 #pragma unroll
                         for (int pw = 0; pw < 2; ++pw)
 #pragma unroll
-                            for (int kk = 0; kk < kSteps; ++kk) {   // 64 elements = 32 bytes along the swizzled row
+                            for (int kk = 0; kk < kSteps; ++kk)   // 64 elements = 32 bytes along the swizzled row
                                 mma_fp4_block16(tmem, dstage + (((pa ? C_::kOffAn : C_::kOffAp) + kk * 32) >> 4),
                                                 dstage + (((pw ? C_::kOffWn : C_::kOffWp) + kk * 32) >> 4), kIdesc,
-                                                sfa + (pa * kSteps + kk) * 4, sfb + (pw * kSteps + kk) * 8, accumulate);
-                                accumulate = 1;
-                            }
+                                                sfa + (pa * kSteps + kk) * 4, sfb + (pw * kSteps + kk) * 8,
+                                                (pa | pw | kk) ? 1u : accumulate);
                     mma_commit(&ctl->empty[s]);
                 }
-                if (ok) mma_commit(&ctl->accum_full);
+                __syncwarp();
+                accumulate = 1;
             }
+            if (ok && elect_one()) mma_commit(&ctl->accum_full);
+            __syncwarp();
         }
     } else if (warp < 2 + kSfWarps) {
         // -------------------------------------------------------------- scale factors
-        // Warp w serves the 32-lane quarter w % 4 of tensor memory.  Per stage it reads the stage's
-        // scale-factor blocks from shared memory (16 bytes per lane and block: the 4-byte scale words of
-        // rows lane, lane+32, lane+64, lane+96) and stores them into its quarter's copy of the
-        // scale-factor columns (every quarter has to hold one).  These warps only follow the `full`
-        // barriers, so they run ahead into the next tile while the epilogue drains the accumulator.
-        // Two groups of four warps take alternate K blocks: the register round trip of one block
-        // (loads, tcgen05.st, wait) then overlaps the other group's.
+        // Warp w serves the 32-lane quarter w % 4 of tensor memory: every quarter has to hold a copy of
+        // the scale-factor columns.  Per K block a lane reads 16 bytes of each 512-byte scale-factor block
+        // straight from global memory (the 4-byte scale words of rows lane, lane+32, lane+64, lane+96) and
+        // stores them to its quarter with tcgen05.st.  The values for the group's next K block are fetched
+        // before the wait for the TMEM buffer, so the global latency stays off the critical path, and the
+        // scale factors are normally in place before the TMA tiles of the same stage land.
+        // Two groups of four warps take alternate K blocks.
         const int q = warp & 3, group = (warp - 2) >> 2;
-        int it = 0;
+        constexpr int kBlocks = 2 * kSteps * 3;                  // per K block: A (1) + W (2 row blocks), x planes x steps
+        uint4 sfv[kBlocks];
+        auto fetch = [&](int64_t tile, int kb) {
+            const int64_t m_blk = tile / n_tiles, n_blk = tile % n_tiles;
+#pragma unroll
+            for (int pl = 0; pl < 2; ++pl)
+#pragma unroll
+                for (int kk = 0; kk < kSteps; ++kk) {
+                    const int64_t c = (int64_t)kb * kSteps + kk;
+                    const uint8_t* a = (pl ? p.sfa_neg : p.sfa_pos) + (m_blk * p.nk64 + c) * kSfChunk + lane * 16;
+                    const uint8_t* w = (pl ? p.sfb_neg : p.sfb_pos) + ((n_blk * 2) * p.nk64 + c) * kSfChunk + lane * 16;
+                    sfv[(pl * kSteps + kk) * 3 + 0] = __ldg(reinterpret_cast<const uint4*>(a));
+                    sfv[(pl * kSteps + kk) * 3 + 1] = __ldg(reinterpret_cast<const uint4*>(w));
+                    sfv[(pl * kSteps + kk) * 3 + 2] = __ldg(reinterpret_cast<const uint4*>(w + (int64_t)p.nk64 * kSfChunk));
+                }
+        };
+        // this group's K blocks, in order, over all tiles: (tile, kb) with global index it = group, group + 2, ...
+        int64_t tile = blockIdx.x;
+        int kb = group;
+        while (tile < total_tiles && kb >= num_kb) { kb -= num_kb; tile += gridDim.x; }
+        int it = group;
         bool ok = true;
-        for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-            for (int kb = 0; kb < num_kb && ok; ++kb, ++it) {
-                if ((it % kSfGroups) != group) continue;
-                const int s = it % kStages;
-                ok = mbar_wait(&ctl->full[s], (it / kStages) & 1, &ctl->abort, p.status);
-                if (!ok) break;
-                const uint8_t* st = tiles + s * kStageBytes;
-                const uint32_t sfa = tmem + ((uint32_t)(q * 32) << 16) + kTmemSf + s * C_::kSfCols, sfb = sfa + C_::kSfColsA;
+        if (tile < total_tiles) fetch(tile, kb);
+        while (tile < total_tiles && ok) {
+            const int s = it % kStages;
+            // the stage's TMEM scale-factor buffer is free once the MMAs of K block it - kStages are done
+            if (it >= kStages) ok = mbar_wait(&ctl->empty[s], ((it / kStages) - 1) & 1, &ctl->abort, p.status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t sfa = tmem + ((uint32_t)(q * 32) << 16) + kTmemSf + s * C_::kSfCols, sfb = sfa + C_::kSfColsA;
 #pragma unroll
-                for (int pl = 0; pl < 2; ++pl)
-#pragma unroll
-                    for (int kk = 0; kk < kSteps; ++kk) {
-                        const uint4 a = *reinterpret_cast<const uint4*>(st + C_::kOffSfA + pl * kSfA + kk * kSfChunk + lane * 16);
-                        tmem_st4(sfa + (pl * kSteps + kk) * 4, a.x, a.y, a.z, a.w);
-#pragma unroll
-                        for (int j = 0; j < 2; ++j) {
-                            const uint4 b = *reinterpret_cast<const uint4*>(st + C_::kOffSfB + pl * kSfB + j * kSfA + kk * kSfChunk + lane * 16);
-                            tmem_st4(sfb + (pl * kSteps + kk) * 8 + j * 4, b.x, b.y, b.z, b.w);
-                        }
-                    }
-                tmem_st_wait();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&ctl->sf_full[s]);
+            for (int i = 0; i < 2 * kSteps; ++i) {
+                tmem_st4(sfa + i * 4, sfv[i * 3].x, sfv[i * 3].y, sfv[i * 3].z, sfv[i * 3].w);
+                tmem_st4(sfb + i * 8, sfv[i * 3 + 1].x, sfv[i * 3 + 1].y, sfv[i * 3 + 1].z, sfv[i * 3 + 1].w);
+                tmem_st4(sfb + i * 8 + 4, sfv[i * 3 + 2].x, sfv[i * 3 + 2].y, sfv[i * 3 + 2].z, sfv[i * 3 + 2].w);
             }
+            // next K block of this group
+            it += kSfGroups;
+            kb += kSfGroups;
+            while (tile < total_tiles && kb >= num_kb) { kb -= num_kb; tile += gridDim.x; }
+            if (tile < total_tiles) fetch(tile, kb);             // in flight during the wait below
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->full[s]);
         }
     } else {
         // -------------------------------------------------------------- epilogue
@@ -425,15 +430,17 @@ EncodeTiledFn encode_tiled() {
     return fn;
 }
 
-// [rows, K/2] bytes, row-major; box = 128 bytes x box_rows, 128-byte swizzle, zero fill outside.
-bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t K, int box_rows, int row_bytes) {
+// Both sign planes of an operand as one 3-D tensor [2][rows][K/2] of bytes (plane_stride bytes apart);
+// box = {row_bytes, box_rows, 2}, 128- or 64-byte swizzle, zero fill outside.
+bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t K, size_t plane_stride, int box_rows,
+              int row_bytes) {
     EncodeTiledFn fn = encode_tiled();
     if (!fn) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)(K / 2), (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)(K / 2)};
-    const cuuint32_t box[2] = {(cuuint32_t)row_bytes, (cuuint32_t)box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+    const cuuint64_t dims[3] = {(cuuint64_t)(K / 2), (cuuint64_t)rows, 2};
+    const cuuint64_t strides[2] = {(cuuint64_t)(K / 2), (cuuint64_t)plane_stride};
+    const cuuint32_t box[3] = {(cuuint32_t)row_bytes, (cuuint32_t)box_rows, 2};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
               CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -494,16 +501,15 @@ int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, co
             return AMX_ERR_CUDA;
         configured[dev] = true;
     }
-    CUtensorMap tm_ap, tm_an, tm_wp, tm_wn;
-    if (!make_map(&tm_ap, pa, p.M, p.K, BM, C_::kRowBytes) || !make_map(&tm_an, pa + oa.plane, p.M, p.K, BM, C_::kRowBytes) ||
-        !make_map(&tm_wp, pw, p.N, p.K, BN, C_::kRowBytes) || !make_map(&tm_wn, pw + ow.plane, p.N, p.K, BN, C_::kRowBytes))
+    CUtensorMap tm_a, tm_w;
+    if (!make_map(&tm_a, pa, p.M, p.K, oa.plane, BM, C_::kRowBytes) || !make_map(&tm_w, pw, p.N, p.K, ow.plane, BN, C_::kRowBytes))
         return AMX_ERR_CUDA;
     static int sm_count[64] = {};
     if (!sm_count[dev] && cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return AMX_ERR_CUDA;
     const int64_t tiles = ((p.N + BN - 1) / BN) * ((p.M + BM - 1) / BM);
     const unsigned grid = (unsigned)(tiles < sm_count[dev] ? tiles : sm_count[dev]);   // one persistent CTA per SM
-    gemm_fp4_kernel<BK_><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_ap, tm_an, tm_wp, tm_wn, p);
+    gemm_fp4_kernel<BK_><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_a, tm_w, p);
     return launch_status();
 }
 
