@@ -32,6 +32,9 @@ GS = 32
 NOMINAL_FP4_TFLOPS = 9000.0      # NVIDIA's dense FP4 figure for one B200 (HGX B200 data sheet)
 NOMINAL_HBM_GBS = 8000.0
 BYTES_PER_ELEM = 2.0 + 0.5 + 2.0 / 32.0   # bf16 read + 4-bit code + two scale bytes per 32
+# DRAM bytes (read + write) per GEMM launch, mean over the four layer shapes, from the ncu capture summarised
+# in profiles/; None until a capture of the current kernel exists.
+GEMM_DRAM_TRAFFIC_PER_LAUNCH = {}
 
 
 def measured_peaks():
@@ -112,7 +115,7 @@ class ClockSampler:
         return out
 
 
-def cpu_baseline(sample_rows: int = 1024, layer: int = 1):
+def cpu_baseline(sample_rows: int = 2048, layer: int = 0):
     """The oracle, as it stands, on the host cores: quantize a row sample of the activation and the whole
     weight of one layer, then the fp64 product of that sample."""
     import oracle
@@ -345,12 +348,14 @@ def run_ours(args):
         "gemm": {"useful_tflops": gemm_tflops, "ms_per_step": g_ms / args.steps,
                  "pct_of_nominal_fp4_peak": 100.0 * gemm_tflops / NOMINAL_FP4_TFLOPS},
         "roofline": {"bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
-                     "frac": gemm_tflops / fp4_peak, "traffic": None,
+                     "frac": gemm_tflops / fp4_peak, "traffic": GEMM_DRAM_TRAFFIC_PER_LAUNCH.get(args.gemm),
+                     "exact_mapping_ceiling_frac": 0.25,
                      "kernel": f"amx_gemm ({gemm_kernel})",
                      "peak_source": f"4 x sustained bf16 cuBLAS rate ({peaks['source']}), nominal FP4:bf16 ratio"},
         "clocks": clocks,
         "e2e": e2e,
-        "gpu_launches": 3 * len(layers) * args.steps,
+        # per layer: 2 casts + the GEMM; the FP4 kernel adds 3 preparation kernels per operand
+        "gpu_launches": (9 if "mxf4" in gemm_kernel else 3) * len(layers) * args.steps,
     }
     if len(layer_ids) != 4:
         line["config"]["layers"] = layer_ids

@@ -52,8 +52,9 @@ typedef enum amx_status {
 /* flags for amx_dequantize: output element type (default bf16) */
 #define AMX_OUT_BF16 0x0u
 #define AMX_OUT_F32 0x1u
-/* flags for amx_gemm / amx_quant_gemm: kernel choice (default: tensor-core path when the
- * shape allows it, else the SIMT path) */
+/* flags for amx_gemm / amx_quant_gemm: kernel choice.  Default (AMX_GEMM_AUTO): group size 32 runs on
+ * the tensor cores - the FP4 kernel when M*N*K >= 2^27, the exact bf16-decode kernel below that - and
+ * other group sizes on the SIMT kernel. */
 #define AMX_GEMM_AUTO 0x0u
 #define AMX_GEMM_SIMT 0x10u  /* plain CUDA-core kernel: any shape, any supported gs */
 #define AMX_GEMM_TC 0x20u    /* tcgen05 kernel, exact bf16 decode: AMX_ERR_SHAPE if the shape does not fit */

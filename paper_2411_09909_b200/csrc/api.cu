@@ -22,6 +22,10 @@ uint32_t pick_kernel(int64_t M, int64_t N, int64_t K, int gs, uint32_t flags) {
     const bool tc = gemm_tc_supported(M, N, K, gs);
     if (want == AMX_GEMM_TC) return tc ? AMX_GEMM_TC : 0;
     if (want == AMX_GEMM_SIMT) return AMX_GEMM_SIMT;
+    // AMX_GEMM_AUTO: the FP4-pipe kernel for anything that fills the machine (it is about twice as fast as
+    // the bf16-decode kernel); the exact bf16-decode kernel for small products, where launch count matters
+    // more than throughput; the SIMT kernel for group sizes the tensor-core kernels do not take.
+    if (gemm_fp4_supported(M, N, K, gs) && (double)M * (double)N * (double)K >= 128.0 * 1024.0 * 1024.0) return AMX_GEMM_FP4;
     return tc ? AMX_GEMM_TC : AMX_GEMM_SIMT;
 }
 
