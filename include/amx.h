@@ -136,6 +136,22 @@ int amx_softmax_bf16(const float* S, int64_t rows, int64_t cols, int64_t ld_s, f
                      void* P, int64_t ld_p, void* stream);
 
 /*
+ * amx_attention - fully quantized attention, one call for all heads (Appendix C: Query, Key, the
+ * self-attention map and Value are all quantized; Section 1: these are the products rotation methods
+ * leave in 16 bits).  Per head h:
+ *   S = AMX(Q_h) AMX(K_h)^T          groups along head_dim
+ *   P = softmax(S / sqrt(d)) per row, fp32, rounded to bf16; no mask
+ *   O_h = AMX(P) AMX(V_h)            groups along the key axis (V is quantized down its rows)
+ *   q, k, v  bf16 [heads, L, d] contiguous;  o  out fp32 [heads, L, d]
+ *   d % 32 == 0, L % 32 == 0 (group size 32 on both axes)
+ *   workspace  at least amx_attention_workspace_bytes(L, d) bytes (reused head after head), 256-aligned
+ * The heads are processed one after another on `stream`.
+ */
+int amx_attention(const void* q, const void* k, const void* v, int64_t heads, int64_t L, int64_t d,
+                  uint32_t flags, float* o, void* workspace, size_t workspace_bytes, void* stream);
+size_t amx_attention_workspace_bytes(int64_t L, int64_t d);
+
+/*
  * amx_linear_host - one whole layer from HOST memory: copies the bf16 activation A_host[M,K] and
  * weight W_host[N,K] to the device, quantizes both, multiplies, and copies C back to
  * C_host[M,N] (fp32).  All copies and kernels are enqueued on `stream`; the call returns after

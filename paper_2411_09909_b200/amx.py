@@ -25,6 +25,7 @@ SYMBOLS = (
     "amx_quant_gemm_workspace_bytes", "amx_linear_host_workspace_bytes",
     "amx_gemm_kernel_for", "amx_gemm_status", "amx_status_string",
     "amx_quant_gemm_static", "amx_quant_gemm_static_capacity",
+    "amx_attention", "amx_attention_workspace_bytes",
 )
 
 
@@ -47,6 +48,9 @@ def lib() -> ctypes.CDLL:
         L.amx_quant_gemm_static.argtypes = [p, i64, p, p, i64, i64, i64, i, u32, p, i64, p]
         L.amx_quant_gemm_static_capacity.argtypes = []
         L.amx_quant_gemm_static_capacity.restype = sz
+        L.amx_attention.argtypes = [p, p, p, i64, i64, i64, u32, p, p, sz, p]
+        L.amx_attention_workspace_bytes.argtypes = [i64, i64]
+        L.amx_attention_workspace_bytes.restype = sz
         L.amx_softmax_bf16.argtypes = [p, i64, i64, i64, ctypes.c_float, p, i64, p]
         L.amx_linear_host.argtypes = [p, p, i64, i64, i64, i, u32, p, p, sz, p]
         for name in ("amx_workspace_bytes", "amx_quant_gemm_workspace_bytes"):
@@ -182,6 +186,23 @@ def linear_host(a_host: torch.Tensor, w_host: torch.Tensor, c_host: torch.Tensor
                                  c_host.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream()),
            "amx_linear_host")
     return c_host
+
+
+def attention_heads(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, flags: int = GEMM_AUTO,
+                    workspace: torch.Tensor | None = None):
+    """Fully quantized attention for all heads through the single C entry point.  q, k, v: bf16 [H, L, d]
+    contiguous.  Returns O fp32 [H, L, d]."""
+    for t in (q, k, v):
+        _dev(t, torch.bfloat16, "q/k/v")
+        assert t.is_contiguous() and t.shape == q.shape
+    H, Lq, d = q.shape
+    need = lib().amx_attention_workspace_bytes(Lq, d)
+    if workspace is None:
+        workspace = _ws(need, q.device)
+    out = torch.empty((H, Lq, d), dtype=torch.float32, device=q.device)
+    _check(lib().amx_attention(q.data_ptr(), k.data_ptr(), v.data_ptr(), H, Lq, d, flags, out.data_ptr(),
+                               workspace.data_ptr(), workspace.numel(), _stream()), "amx_attention")
+    return out
 
 
 def attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, group_size: int = 32, flags: int = GEMM_AUTO):

@@ -1,5 +1,7 @@
 // C-ABI entry points that combine kernels: GEMM dispatch, quantize+GEMM, the host-buffer
 // layer call, workspace sizing and status strings.
+#include <cmath>
+
 #include "gemm.cuh"
 
 namespace amx {
@@ -148,6 +150,67 @@ extern "C" int amx_linear_host(const void* A_host, const void* W_host, int64_t M
     if (cudaMemcpyAsync(C_host, c_dev, (size_t)M * N * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return AMX_ERR_CUDA;
     return cudaStreamSynchronize(st) == cudaSuccess ? AMX_OK : AMX_ERR_CUDA;
+}
+
+namespace {
+struct AttnLayout {
+    size_t qc, qs, kc, ks, vc, vs, pc, ps, S, P, gemm, total;
+};
+AttnLayout attn_layout(int64_t L, int64_t d) {
+    AttnLayout a;
+    const QuantSizes qd = quant_sizes(L, d, 32), ql = quant_sizes(L, L, 32), qv = quant_sizes(d, L, 32);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off += round_up(bytes); return o; };
+    a.qc = take(qd.codes); a.qs = take(qd.scales); a.kc = take(qd.codes); a.ks = take(qd.scales);
+    a.vc = take(qv.codes); a.vs = take(qv.scales); a.pc = take(ql.codes); a.ps = take(ql.scales);
+    a.S = take((size_t)L * L * 4);
+    a.P = take((size_t)L * L * 2);
+    a.gemm = off;
+    const size_t g1 = amx_workspace_bytes(L, L, d, 32, AMX_GEMM_AUTO), g2 = amx_workspace_bytes(L, d, L, 32, AMX_GEMM_AUTO);
+    const size_t g3 = amx_workspace_bytes(L, L, d, 32, AMX_GEMM_FP4), g4 = amx_workspace_bytes(L, d, L, 32, AMX_GEMM_FP4);
+    size_t g = g1 > g2 ? g1 : g2;
+    g = g > g3 ? g : g3;
+    g = g > g4 ? g : g4;
+    a.total = off + g;
+    return a;
+}
+}  // namespace
+
+extern "C" size_t amx_attention_workspace_bytes(int64_t L, int64_t d) {
+    if (L <= 0 || d <= 0 || L % 32 || d % 32) return 0;
+    return attn_layout(L, d).total;
+}
+
+extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_t heads, int64_t L, int64_t d,
+                             uint32_t flags, float* o, void* workspace, size_t workspace_bytes, void* stream) {
+    if (flags & ~kKernelMask) return AMX_ERR_FLAGS;
+    if (heads < 0 || L <= 0 || d <= 0 || L % 32 || d % 32) return AMX_ERR_SHAPE;
+    if (heads == 0) return AMX_OK;
+    if (!q || !k || !v || !o) return AMX_ERR_NULL;
+    const AttnLayout a = attn_layout(L, d);
+    if (!workspace || workspace_bytes < a.total) return AMX_ERR_WORKSPACE;
+    if (!aligned(workspace, kAlign) || !aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16)) return AMX_ERR_ALIGN;
+    uint8_t* w = static_cast<uint8_t*>(workspace);
+    const size_t gemm_bytes = a.total - a.gemm;
+    const float alpha = 1.0f / sqrtf((float)d);
+    for (int64_t h = 0; h < heads; ++h) {
+        const uint8_t* qh = static_cast<const uint8_t*>(q) + (size_t)h * L * d * 2;
+        const uint8_t* kh = static_cast<const uint8_t*>(k) + (size_t)h * L * d * 2;
+        const uint8_t* vh = static_cast<const uint8_t*>(v) + (size_t)h * L * d * 2;
+        int rc = amx_quantize(qh, L, d, d, 32, w + a.qc, w + a.qs, stream);
+        if (rc == AMX_OK) rc = amx_quantize(kh, L, d, d, 32, w + a.kc, w + a.ks, stream);
+        if (rc == AMX_OK) rc = amx_quantize_t(vh, L, d, d, 32, w + a.vc, w + a.vs, stream);
+        if (rc == AMX_OK)
+            rc = amx_gemm(w + a.qc, w + a.qs, w + a.kc, w + a.ks, L, L, d, 32, flags, reinterpret_cast<float*>(w + a.S), L,
+                          w + a.gemm, gemm_bytes, stream);
+        if (rc == AMX_OK) rc = amx_softmax_bf16(reinterpret_cast<const float*>(w + a.S), L, L, L, alpha, w + a.P, L, stream);
+        if (rc == AMX_OK) rc = amx_quantize(w + a.P, L, L, L, 32, w + a.pc, w + a.ps, stream);
+        if (rc == AMX_OK)
+            rc = amx_gemm(w + a.pc, w + a.ps, w + a.vc, w + a.vs, L, d, L, 32, flags, o + (size_t)h * L * d, d, w + a.gemm,
+                          gemm_bytes, stream);
+        if (rc != AMX_OK) return rc;
+    }
+    return AMX_OK;
 }
 
 extern "C" int amx_gemm_status(const void* workspace, void* stream) {

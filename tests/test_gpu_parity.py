@@ -274,9 +274,44 @@ def test_attention_small_head_against_oracle_pipeline():
     assert rel_fro(O.cpu().numpy(), Ocpu) <= GEMM_TOL
 
 
+def test_attention_all_heads_entry_point_matches_per_head_pipeline():
+    q, k, v = (dev_bf16(t) for t in inputs.attention_qkv(heads=3, seq=320))
+    O = amx.attention_heads(q, k, v)
+    for h in range(3):
+        Oh, _ = amx.attention(q[h], k[h], v[h])
+        assert torch.equal(O[h], Oh)
+
+
+def test_config5_full_size_attention_sampled():
+    """32 heads x 8192 tokens x 128: every head through amx_attention; heads 0 and 31 checked against the
+    all-CPU pipeline on sampled query rows, and the device quantizer against the oracle on the device's own
+    bf16 attention map."""
+    qb, kb, vb = inputs.attention_qkv()
+    q, k, v = dev_bf16(qb), dev_bf16(kb), dev_bf16(vb)
+    O = amx.attention_heads(q, k, v).cpu().numpy()
+    assert np.all(np.isfinite(O))
+    rng = np.random.default_rng(55)
+    for h in (0, 31):
+        rows = np.sort(rng.choice(8192, size=48, replace=False))
+        qc, qs = oracle.quantize(qb[h][rows], 32)
+        kc, ks = oracle.quantize(kb[h], 32)
+        vc, vs = oracle.quantize(np.ascontiguousarray(vb[h].T), 32)
+        S = oracle.gemm(qc, qs, kc, ks, 32)
+        P = oracle.softmax_bf16(S, 128 ** -0.5)
+        ref = oracle.gemm(*oracle.quantize(P, 32), vc, vs, 32)
+        assert rel_fro(O[h][rows], ref) <= GEMM_TOL, h
+    # the device quantizer on the device's own attention map (head 0), sampled rows
+    _, Pdev = amx.attention(q[0], k[0], v[0])
+    pc, ps = amx.quantize(Pdev, 32)
+    rows = np.sort(rng.choice(8192, size=256, replace=False))
+    p_bits = Pdev[torch.from_numpy(rows).cuda()].view(torch.int16).cpu().numpy().view(np.uint16)
+    opc, ops = oracle.quantize(p_bits, 32)
+    assert np.array_equal(pc.cpu().numpy()[rows], opc) and np.array_equal(ps.cpu().numpy()[rows], ops)
+
+
 # ------------------------------------------------ full-size configurations --
 
-@pytest.mark.parametrize("config,layer", [(2, 0), (2, 3), (3, 1), (4, 2)])
+@pytest.mark.parametrize("config,layer", [(2, 0), (2, 3), (3, 0), (3, 1), (3, 3), (4, 0), (4, 2)])
 def test_full_size_layer_sampled(config, layer):
     """Whole-tensor launches at the benchmark's sizes; codes and scales compared on the whole activation
     for config 2 and on sampled rows otherwise; GEMM compared on 64 sampled rows x all N."""
