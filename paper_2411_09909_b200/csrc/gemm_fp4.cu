@@ -26,7 +26,7 @@
 //   warps 10-17 epilogue: TMEM -> registers (double-buffered loads), power-of-two rescale, 32-byte fp32
 //            stores.  While a tile's accumulator is read out the producer already prefetches the next
 //            tile's stages; the MMA issuer waits for `accum_empty`.
-// A preparation pass (two small kernels per operand) derives the planes, the UE4M3 scale-factor
+// A preparation kernel per operand derives the planes, the UE4M3 scale-factor
 // blocks in the 128 x 4 interleaved layout the MMA reads, and the row offsets from the canonical
 // codes and scales.  Every device-side wait is bounded.
 #include <cuda.h>
@@ -90,24 +90,6 @@ __device__ __forceinline__ uint64_t operand_desc(uint32_t addr) {
 constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
 // ------------------------------------------------------------------------- preparation --
-// Sign planes: nibble kept where its sign bit matches the plane, zero elsewhere.
-__global__ void __launch_bounds__(256)
-split_planes_kernel(const uint4* __restrict__ codes, int64_t n_vec, uint4* __restrict__ pos, uint4* __restrict__ neg) {
-    const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
-    if (i >= n_vec) return;
-    const uint4 w = __ldg(codes + i);
-    const uint32_t v[4] = {w.x, w.y, w.z, w.w};
-    uint32_t p[4], n[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const uint32_t m = ((v[j] >> 3) & 0x11111111u) * 15u;   // 0xF on negative nibbles
-        n[j] = v[j] & m;
-        p[j] = v[j] & ~m;
-    }
-    pos[i] = make_uint4(p[0], p[1], p[2], p[3]);
-    neg[i] = make_uint4(n[0], n[1], n[2], n[3]);
-}
-
 // Exponent key of an E5M2 scale byte: unbiased exponent + 17 (1 for 2^-16), 0 for a zero scale.
 __device__ __forceinline__ int scale_key(uint32_t b) {
     const int e = (b >> 2) & 31, m = b & 3;
@@ -121,61 +103,81 @@ __device__ __forceinline__ uint32_t to_ue4m3(uint32_t b, int kmax) {
     return (f >= 1 && scale_key(b) > 0) ? (uint32_t)((f << 3) | (mant << 1)) : 0u;
 }
 
-// Row offsets: one warp per operand row finds the largest exponent key among the row's scales.
-// kmax[row] = that key; row_exp[row] = kmax - 25, the power of two by which the UE4M3 scales of the
-// row understate the true ones (0 for an all-zero row).
+// One launch per operand; one block per 32 operand rows (rows beyond R, up to the padded row count,
+// get zero scale factors so that padded tile rows multiply zero codes by a finite scale).
+//   1. row offsets: a warp per row finds the largest exponent key kmax among the row's scales;
+//      row_exp = kmax - 25 is the power of two by which the row's UE4M3 scales understate the true ones
+//   2. sign planes: every nibble goes to the plane of its sign bit, zero in the other plane
+//   3. scale factors of both planes in the layout the MMA reads:
+//      [plane][row block of 128][K/64 block][512 B], byte (r%32)*16 + (r/32)*4 + (k16 % 4);
+//      one scale per 16 elements, so each 32-group's scale is written twice
+constexpr int kPrepRows = 8;
 __global__ void __launch_bounds__(256)
-row_offsets_kernel(const uint8_t* __restrict__ scales, int64_t R, int64_t G /*groups per row*/,
-                   int* __restrict__ kmax_out, int* __restrict__ row_exp) {
-    const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (row >= R) return;
-    const unsigned short* s2 = reinterpret_cast<const unsigned short*>(scales + row * G * 2);
-    int kmax = 0;
-    for (int64_t g = lane; g < G; g += 32) {
-        const uint32_t v = __ldg(s2 + g);
-        kmax = max(kmax, max(scale_key(v & 0xFF), scale_key(v >> 8)));
-    }
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, d));
-    if (lane == 0) {
-        kmax_out[row] = kmax;
-        row_exp[row] = kmax ? kmax - 25 : 0;
-    }
-}
-
-// Scale-factor blocks of both planes.  One block = 128 operand rows x 8 K/64 blocks (16 groups):
-// the E5M2 pairs are staged in shared memory (one 32-byte run per row), then written out in the
-// layout the MMA reads: [plane][row block][K/64 block][512 B], byte (r%32)*16 + (r/32)*4 + (k16 % 4).
-constexpr int kSfBlocksPerCta = 8;
-__global__ void __launch_bounds__(256)
-scale_factors_kernel(const uint8_t* __restrict__ scales, const int* __restrict__ kmax_in, int64_t R, int64_t G,
-                     int nk64, uint8_t* __restrict__ sf_pos, uint8_t* __restrict__ sf_neg) {
-    __shared__ unsigned short sc[128][2 * kSfBlocksPerCta + 1];
-    __shared__ int kmax_s[128];
-    const int64_t rb = blockIdx.y, row0 = rb * 128;
-    const int c0 = blockIdx.x * kSfBlocksPerCta;
-    for (int i = threadIdx.x; i < 128 * 2 * kSfBlocksPerCta; i += 256) {
-        const int r = i / (2 * kSfBlocksPerCta), gl = i % (2 * kSfBlocksPerCta);
-        const int64_t row = row0 + r, g = (int64_t)c0 * 2 + gl;
-        sc[r][gl] = (row < R && g < G) ? __ldg(reinterpret_cast<const unsigned short*>(scales + (row * G + g) * 2)) : 0;
-    }
-    if (threadIdx.x < 128) kmax_s[threadIdx.x] = (row0 + threadIdx.x < R) ? kmax_in[row0 + threadIdx.x] : 0;
-    __syncthreads();
-    for (int item = threadIdx.x; item < kSfBlocksPerCta * 128; item += 256) {
-        const int cc = item >> 7, u = item & 127;                // K/64 block, 4-byte word inside its chunk
-        if (c0 + cc >= nk64) break;
-        const int r = (u & 3) * 32 + (u >> 2);
-        const int kmax = kmax_s[r];
-        uint32_t wp = 0, wn = 0;
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {                            // the two 32-groups of this 64-element block
-            const uint32_t v = sc[r][2 * cc + h];
-            const uint32_t up = to_ue4m3(v & 0xFF, kmax), un = to_ue4m3(v >> 8, kmax);
-            wp |= (up | (up << 8)) << (16 * h);                  // one scale per 16 elements: each twice
-            wn |= (un | (un << 8)) << (16 * h);
+prepare_operand_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales, int64_t R, int64_t K,
+                       int nk64, uint4* __restrict__ pos, uint4* __restrict__ neg, uint8_t* __restrict__ sf_pos,
+                       uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp) {
+    __shared__ int kmax_s[kPrepRows];
+    const int64_t row0 = (int64_t)blockIdx.x * kPrepRows, G = K / 32;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int r = warp; r < kPrepRows; r += 8) {
+        const int64_t row = row0 + r;
+        int kmax = 0;
+        if (row < R) {
+            const unsigned short* s2 = reinterpret_cast<const unsigned short*>(scales + row * G * 2);
+            for (int64_t g = lane; g < G; g += 32) {
+                const uint32_t v = __ldg(s2 + g);
+                kmax = max(kmax, max(scale_key(v & 0xFF), scale_key(v >> 8)));
+            }
         }
-        const int64_t off = (rb * nk64 + c0 + cc) * (int64_t)kSfChunk + u * 4;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, d));
+        if (lane == 0) {
+            kmax_s[r] = kmax;
+            if (row < R) row_exp[row] = kmax ? kmax - 25 : 0;
+        }
+    }
+    // sign planes of this block's rows (contiguous in memory: rows are K/2 bytes apart)
+    const int64_t rows_here = min((int64_t)kPrepRows, R - row0);
+    if (rows_here > 0) {
+        const int64_t v0 = row0 * (K / 32), n_vec = rows_here * (K / 32);
+        const uint4* src = reinterpret_cast<const uint4*>(codes) + v0;
+        for (int64_t i = threadIdx.x; i < n_vec; i += 256) {
+            const uint4 w = __ldg(src + i);
+            const uint32_t v[4] = {w.x, w.y, w.z, w.w};
+            uint32_t p[4], n[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t m = ((v[j] >> 3) & 0x11111111u) * 15u;   // 0xF on negative nibbles
+                n[j] = v[j] & m;
+                p[j] = v[j] & ~m;
+            }
+            pos[v0 + i] = make_uint4(p[0], p[1], p[2], p[3]);
+            neg[v0 + i] = make_uint4(n[0], n[1], n[2], n[3]);
+        }
+    }
+    __syncthreads();
+    // scale factors: item = (K/64 block c, row r); consecutive threads take consecutive rows
+    const int64_t rb = row0 / 128;
+    const int r_in_blk0 = (int)(row0 % 128);
+    for (int item = threadIdx.x; item < nk64 * kPrepRows; item += 256) {
+        const int c = item / kPrepRows, r = item % kPrepRows;
+        const int64_t row = row0 + r;
+        uint32_t wp = 0, wn = 0;
+        if (row < R) {
+            const int kmax = kmax_s[r];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {                        // the two 32-groups of this 64-element block
+                const int64_t g = (int64_t)c * 2 + h;
+                if (g < G) {
+                    const uint32_t v = __ldg(reinterpret_cast<const unsigned short*>(scales + (row * G + g) * 2));
+                    const uint32_t up = to_ue4m3(v & 0xFF, kmax), un = to_ue4m3(v >> 8, kmax);
+                    wp |= (up | (up << 8)) << (16 * h);
+                    wn |= (un | (un << 8)) << (16 * h);
+                }
+            }
+        }
+        const int rr = r_in_blk0 + r;                            // row inside its block of 128
+        const int64_t off = (rb * nk64 + c) * (int64_t)kSfChunk + (rr % 32) * 16 + (rr / 32) * 4;
         *reinterpret_cast<uint32_t*>(sf_pos + off) = wp;
         *reinterpret_cast<uint32_t*>(sf_neg + off) = wn;
     }
@@ -459,22 +461,17 @@ OperandLayout operand_layout(int64_t rows, int64_t K, int rows_per_tile) {
     o.nk64 = (int)((K + 255) / 256) * 4;    // padded to whole 256-element blocks
     o.plane = up256((size_t)rows * (K / 2));
     o.sf = up256((size_t)o.row_blocks * o.nk64 * kSfChunk);
-    o.exps = up256((size_t)rows * 8);      // row offsets, then the rows' largest exponent keys
+    o.exps = up256((size_t)rows * 4);      // row offsets
     o.total = 2 * o.plane + 2 * o.sf + o.exps;
     return o;
 }
 
 int prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, const OperandLayout& o,
             uint8_t* base, cudaStream_t st) {
-    const int64_t n_vec = rows * (K / 32);
-    split_planes_kernel<<<(unsigned)((n_vec + 255) / 256), 256, 0, st>>>(
-        reinterpret_cast<const uint4*>(codes), n_vec, reinterpret_cast<uint4*>(base), reinterpret_cast<uint4*>(base + o.plane));
-    int* exps = reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf);
-    int* kmax = exps + rows;
-    row_offsets_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(scales, rows, K / 32, kmax, exps);
-    dim3 grid((unsigned)((o.nk64 + kSfBlocksPerCta - 1) / kSfBlocksPerCta), (unsigned)o.row_blocks);
-    scale_factors_kernel<<<grid, 256, 0, st>>>(scales, kmax, rows, K / 32, o.nk64, base + 2 * o.plane,
-                                               base + 2 * o.plane + o.sf);
+    const int64_t padded_rows = o.row_blocks * 128;
+    prepare_operand_kernel<<<(unsigned)(padded_rows / kPrepRows), 256, 0, st>>>(
+        codes, scales, rows, K, o.nk64, reinterpret_cast<uint4*>(base), reinterpret_cast<uint4*>(base + o.plane),
+        base + 2 * o.plane, base + 2 * o.plane + o.sf, reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf));
     return launch_status();
 }
 
