@@ -354,8 +354,8 @@ def run_ours(args):
                      "peak_source": f"4 x sustained bf16 cuBLAS rate ({peaks['source']}), nominal FP4:bf16 ratio"},
         "clocks": clocks,
         "e2e": e2e,
-        # per layer: 2 casts + the GEMM; the FP4 kernel adds 3 preparation kernels per operand
-        "gpu_launches": (9 if "mxf4" in gemm_kernel else 3) * len(layers) * args.steps,
+        # per layer: 2 casts + the GEMM; the FP4 kernel adds one preparation kernel per operand
+        "gpu_launches": (5 if "mxf4" in gemm_kernel else 3) * len(layers) * args.steps,
     }
     if len(layer_ids) != 4:
         line["config"]["layers"] = layer_ids

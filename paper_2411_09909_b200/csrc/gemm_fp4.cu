@@ -269,7 +269,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         // field (bytes >> 4); the per-plane and per-K-step offsets are compile-time constants.
         const uint64_t desc0 = operand_desc<BK_>(smem_u32(tiles));
         int it = 0, t = 0;
-        bool ok = true;
+        bool ok = true, ready = false;                           // ready: the next K block's barrier was seen complete
         for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t) {
             // the previous tile's accumulator must have been read out before it is overwritten
             if (t > 0) ok = mbar_wait(&ctl->accum_empty, (t - 1) & 1, &ctl->abort, p.status);
@@ -277,26 +277,34 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             uint32_t accumulate = 0;
             for (int kb = 0; kb < num_kb && ok; ++kb, ++it) {
                 const int s = it % kStages;
-                // tiles landed (TMA byte count) and scale factors stored (four warp arrivals)
-                ok = mbar_wait(&ctl->full[s], (it / kStages) & 1, &ctl->abort, p.status);
+                // tiles landed (TMA byte count) and scale factors stored (four warp arrivals); usually already
+                // seen by the poll that was slipped between the previous block's MMAs
+                if (!ready) ok = mbar_wait(&ctl->full[s], (it / kStages) & 1, &ctl->abort, p.status);
                 if (!ok) break;
                 tc_fence_after();
                 const uint64_t dstage = desc0 + (uint64_t)((s * kStageBytes) >> 4);
                 const uint32_t sfa = tmem + kTmemSf + s * C_::kSfCols, sfb = sfa + C_::kSfColsA;
+                const int s_next = (it + 1) % kStages;
+                const uint32_t parity_next = ((it + 1) / kStages) & 1;
+                uint32_t seen = 0;
                 if (elect_one()) {
 #pragma unroll
                     for (int pa = 0; pa < 2; ++pa)
 #pragma unroll
                         for (int pw = 0; pw < 2; ++pw)
 #pragma unroll
-                            for (int kk = 0; kk < kSteps; ++kk)   // 64 elements = 32 bytes along the swizzled row
+                            for (int kk = 0; kk < kSteps; ++kk) {   // 64 elements = 32 bytes along the swizzled row
                                 mma_fp4_block16(tmem, dstage + (((pa ? C_::kOffAn : C_::kOffAp) + kk * 32) >> 4),
                                                 dstage + (((pw ? C_::kOffWn : C_::kOffWp) + kk * 32) >> 4), kIdesc,
                                                 sfa + (pa * kSteps + kk) * 4, sfb + (pw * kSteps + kk) * 8,
                                                 (pa | pw | kk) ? 1u : accumulate);
+                                // with two MMAs still to go (they keep the pipe busy meanwhile), look whether the
+                                // next K block is complete, so that its MMAs can follow without a wait
+                                if (pa == 1 && pw == 0 && kk == kSteps - 1) seen = mbar_try_wait(&ctl->full[s_next], parity_next);
+                            }
                     mma_commit(&ctl->empty[s]);
                 }
-                __syncwarp();
+                ready = __any_sync(0xFFFFFFFFu, seen) != 0;
                 accumulate = 1;
             }
             if (ok && elect_one()) mma_commit(&ctl->accum_full);
