@@ -164,7 +164,7 @@ def run_reference(args):
 
 def run_ours(args):
     import torch
-    from paper_2411_09909_b200 import amx, inputs, build
+    from paper_2411_09909_b200 import amx, inputs, build, sharding
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -253,11 +253,7 @@ def run_ours(args):
     barrier()
     elapsed_ms = t_start.elapsed_time(t_end)
     clocks = sampler.stop() if sampler else None
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([elapsed_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = sharding.max_over_ranks(elapsed_ms, "cuda")      # the slowest rank's time
     q_ms = sum(a.elapsed_time(b) for a, b in ev_q)
     g_ms = sum(a.elapsed_time(b) for a, b in ev_g)
 
@@ -310,11 +306,7 @@ def run_ours(args):
             e2e_step()
         torch.cuda.synchronize()
         e2e_s = (time.perf_counter() - t0) / e2e_steps
-        if world > 1:
-            import torch.distributed as dist
-            t = torch.tensor([e2e_s], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = float(t.item())
+        e2e_s = sharding.max_over_ranks(e2e_s, "cuda")
         e2e = {"value": world * flops_step / e2e_s / 1e12, "unit": "TFLOP/s",
                "h2d_bytes_per_step": int(elems_step * 2),
                "d2h_bytes_per_step": int(sum(M * N * 4 for _, N in layers)),
@@ -327,7 +319,7 @@ def run_ours(args):
         return
 
     ms_per_step = elapsed_ms / args.steps
-    value = world * flops_step / (ms_per_step * 1e-3) / 1e12
+    value = sharding.aggregate_rate(flops_step, world, ms_per_step) / 1e12
     gemm_tflops = args.steps * flops_step / (g_ms * 1e-3) / 1e12
     quant_gbs = args.steps * elems_step * BYTES_PER_ELEM / (q_ms * 1e-3) / 1e9
     fp4_peak = 4.0 * peaks["bf16_tflops_sustained"]
