@@ -214,7 +214,7 @@ def run_ours(args):
 
     ev_q, ev_g = [], []
 
-    def step(record: bool):
+    def step(record: bool, stream=stream):
         for li, (K, N) in enumerate(layers):
             b = bufs[li]
             if record:
@@ -245,17 +245,37 @@ def run_ours(args):
     if sampler:
         time.sleep(0.3)
         sampler.mark()
+    # The step is launch-bound in places (20 kernels, some of a few microseconds), so the timed region
+    # replays a CUDA graph of one step; --no-graph times plain launches instead.
+    graph = None
+    if not args.no_graph:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            step(False, torch.cuda.current_stream().cuda_stream)
+        for _ in range(3):
+            graph.replay()
+        barrier()
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_start.record()
     for _ in range(args.steps):
-        step(True)
+        if graph is not None:
+            graph.replay()
+        else:
+            step(False)
     t_end.record()
     barrier()
     elapsed_ms = t_start.elapsed_time(t_end)
     clocks = sampler.stop() if sampler else None
     elapsed_ms = sharding.max_over_ranks(elapsed_ms, "cuda")      # the slowest rank's time
-    q_ms = sum(a.elapsed_time(b) for a, b in ev_q)
-    g_ms = sum(a.elapsed_time(b) for a, b in ev_g)
+    # per-kernel-type times: a separate pass of plain launches with CUDA events around the casts and the GEMM
+    event_steps = min(args.steps, 50)
+    for _ in range(event_steps):
+        step(True)
+    torch.cuda.synchronize()
+    q_ms = sum(a.elapsed_time(b) for a, b in ev_q) * args.steps / event_steps
+    g_ms = sum(a.elapsed_time(b) for a, b in ev_g) * args.steps / event_steps
 
     # ---- the cast alone on a tensor larger than L2 (config-4 activation shape, 16384 x 8192 = 268 MB of bf16)
     quant_large = None
@@ -331,7 +351,8 @@ def run_ours(args):
         "config": {"workload": "config 2: LLaMA-7B-shaped prefill linears, M=2048, 4 layers; activations and "
                                "weights both cast to AMXFP4 every step, then GEMM",
                    "group_size": GS, "gemm_kernel": gemm_kernel,
-                   "l2": "per-step inputs (~410 MB of bf16) exceed the 126 MB L2"},
+                   "l2": "per-step inputs (~410 MB of bf16) exceed the 126 MB L2",
+                   "launch": "plain launches" if args.no_graph else "CUDA graph of one step, replayed"},
         "pct_of_nominal_fp4_peak": 100.0 * value / world / NOMINAL_FP4_TFLOPS,
         "nominal_fp4_peak_tflops": NOMINAL_FP4_TFLOPS,
         "quantize": {"gb_per_s": quant_gbs, "pct_of_nominal_hbm_8TBs": 100.0 * quant_gbs / NOMINAL_HBM_GBS,
@@ -366,6 +387,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--gemm", default="auto", choices=["auto", "simt", "tc", "fp4"], help="GEMM kernel to time")
+    ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of a CUDA graph of the step")
     ap.add_argument("--layers", default="", help="comma-separated layer indices to run (profiling aid; default all)")
     ap.add_argument("--skip-extras", action="store_true", help="skip the e2e and cpu_baseline legs (profiling aid)")
     args = ap.parse_args()
