@@ -116,6 +116,24 @@ int amx_gemm(const uint8_t* a_codes, const uint8_t* a_scales,
              float* C, int64_t ld_c, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Two-phase form of the AMX_GEMM_FP4 kernel, for operands that are reused (the quantized weight of a
+ * layer, across calls).  amx_gemm with AMX_GEMM_FP4 prepares both operands on every call; here
+ *   amx_prepare        turns one canonical operand [rows, K] (gs = 32) into its "prepared" form - the two
+ *                      sign planes, the UE4M3 scale factors in the tensor cores' layout and a power-of-two
+ *                      offset per row - in a caller-owned buffer of amx_prepared_bytes() bytes
+ *                      (256-byte aligned).  is_weight selects the padding of the W (right-hand) operand.
+ *   amx_gemm_prepared  multiplies a prepared A [M, K] with a prepared W [N, K]; same result as amx_gemm
+ *                      with AMX_GEMM_FP4.  workspace: 256 bytes (status word, see amx_gemm_status).
+ * This is how Section 4.3's product runs when the weights were cast once ahead of time.
+ */
+size_t amx_prepared_bytes(int64_t rows, int64_t K, int group_size, int is_weight);
+int amx_prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, int group_size,
+                int is_weight, void* prepared, size_t prepared_bytes, void* stream);
+int amx_gemm_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
+                      int group_size, float* C, int64_t ld_c, void* workspace, size_t workspace_bytes,
+                      void* stream);
+
+/*
  * amx_quant_gemm - the fully quantized linear layer of Section 5 ("quantize input operands for
  * all decoder-layer matrix multiplications"): quantizes the bf16 activation A[M, ld_a] and
  * multiplies it with an already quantized weight.  Same result as amx_quantize followed by

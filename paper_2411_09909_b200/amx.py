@@ -26,6 +26,7 @@ SYMBOLS = (
     "amx_gemm_kernel_for", "amx_gemm_status", "amx_status_string",
     "amx_quant_gemm_static", "amx_quant_gemm_static_capacity",
     "amx_attention", "amx_attention_workspace_bytes",
+    "amx_prepared_bytes", "amx_prepare", "amx_gemm_prepared",
 )
 
 
@@ -51,6 +52,10 @@ def lib() -> ctypes.CDLL:
         L.amx_attention.argtypes = [p, p, p, i64, i64, i64, u32, p, p, sz, p]
         L.amx_attention_workspace_bytes.argtypes = [i64, i64]
         L.amx_attention_workspace_bytes.restype = sz
+        L.amx_prepared_bytes.argtypes = [i64, i64, i, i]
+        L.amx_prepared_bytes.restype = sz
+        L.amx_prepare.argtypes = [p, p, i64, i64, i, i, p, sz, p]
+        L.amx_gemm_prepared.argtypes = [p, p, i64, i64, i64, i, p, i64, p, sz, p]
         L.amx_softmax_bf16.argtypes = [p, i64, i64, i64, ctypes.c_float, p, i64, p]
         L.amx_linear_host.argtypes = [p, p, i64, i64, i64, i, u32, p, p, sz, p]
         for name in ("amx_workspace_bytes", "amx_quant_gemm_workspace_bytes"):
@@ -141,6 +146,27 @@ def gemm(a_codes, a_scales, w_codes, w_scales, group_size: int = 32, flags: int 
     _check(lib().amx_gemm(a_codes.data_ptr(), a_scales.data_ptr(), w_codes.data_ptr(), w_scales.data_ptr(),
                           M, N, K, group_size, flags, out.data_ptr(), out.stride(0), workspace.data_ptr(),
                           workspace.numel(), _stream()), "amx_gemm")
+    return out
+
+
+def prepare(codes: torch.Tensor, scales: torch.Tensor, is_weight: bool, group_size: int = 32) -> torch.Tensor:
+    """Canonical operand -> prepared operand of the FP4 kernel (reusable across amx_gemm_prepared calls)."""
+    _dev(codes, torch.uint8, "codes"), _dev(scales, torch.uint8, "scales")
+    rows, K = codes.shape[0], codes.shape[1] * 2
+    buf = _ws(lib().amx_prepared_bytes(rows, K, group_size, int(is_weight)), codes.device)
+    _check(lib().amx_prepare(codes.data_ptr(), scales.data_ptr(), rows, K, group_size, int(is_weight), buf.data_ptr(),
+                             buf.numel(), _stream()), "amx_prepare")
+    return buf
+
+
+def gemm_prepared(a_prepared: torch.Tensor, w_prepared: torch.Tensor, M: int, N: int, K: int, group_size: int = 32,
+                  out: torch.Tensor | None = None, workspace: torch.Tensor | None = None):
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float32, device=a_prepared.device)
+    if workspace is None:
+        workspace = _ws(256, a_prepared.device)
+    _check(lib().amx_gemm_prepared(a_prepared.data_ptr(), w_prepared.data_ptr(), M, N, K, group_size, out.data_ptr(),
+                                   out.stride(0), workspace.data_ptr(), workspace.numel(), _stream()), "amx_gemm_prepared")
     return out
 
 

@@ -97,6 +97,31 @@ extern "C" int amx_gemm(const uint8_t* a_codes, const uint8_t* a_scales, const u
     return gemm_tc(a_codes, a_scales, w_codes, w_scales, M, N, K, C, ld_c, workspace, st);
 }
 
+extern "C" size_t amx_prepared_bytes(int64_t rows, int64_t K, int group_size, int is_weight) {
+    if (rows <= 0 || !gemm_fp4_supported(rows, rows, K, group_size)) return 0;
+    return round_up(gemm_fp4_prepared_bytes(rows, K, is_weight != 0));
+}
+
+extern "C" int amx_prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, int group_size,
+                           int is_weight, void* prepared, size_t prepared_bytes, void* stream) {
+    if (rows <= 0 || !gemm_fp4_supported(rows, rows, K, group_size)) return AMX_ERR_SHAPE;
+    if (!codes || !scales || !prepared) return AMX_ERR_NULL;
+    if (prepared_bytes < amx_prepared_bytes(rows, K, group_size, is_weight)) return AMX_ERR_WORKSPACE;
+    if (!aligned(codes, 16) || !aligned(scales, 2) || !aligned(prepared, kAlign)) return AMX_ERR_ALIGN;
+    return gemm_fp4_prepare(codes, scales, rows, K, is_weight != 0, prepared, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int amx_gemm_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
+                                 int group_size, float* C, int64_t ld_c, void* workspace, size_t workspace_bytes,
+                                 void* stream) {
+    if (M <= 0 || N <= 0 || !gemm_fp4_supported(M, N, K, group_size) || ld_c < N) return AMX_ERR_SHAPE;
+    if (!a_prepared || !w_prepared || !C) return AMX_ERR_NULL;
+    if (!workspace || workspace_bytes < 256) return AMX_ERR_WORKSPACE;
+    if (!aligned(a_prepared, kAlign) || !aligned(w_prepared, kAlign) || !aligned(workspace, kAlign) || !aligned(C, 4))
+        return AMX_ERR_ALIGN;
+    return gemm_fp4_prepared(a_prepared, w_prepared, M, N, K, C, ld_c, workspace, static_cast<cudaStream_t>(stream));
+}
+
 extern "C" int amx_quant_gemm(const void* A, int64_t ld_a, const uint8_t* w_codes, const uint8_t* w_scales,
                               int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags, float* C,
                               int64_t ld_c, void* workspace, size_t workspace_bytes, void* stream) {

@@ -24,5 +24,11 @@ size_t gemm_fp4_workspace_bytes(int64_t M, int64_t N, int64_t K);
 int gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes,
              const uint8_t* w_scales, int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c,
              void* workspace, cudaStream_t st);
+// The same in two phases, so that an operand (typically the weight) is prepared once and reused.
+size_t gemm_fp4_prepared_bytes(int64_t rows, int64_t K, bool is_weight);
+int gemm_fp4_prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, bool is_weight,
+                     void* prepared, cudaStream_t st);
+int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
+                      float* C, int64_t ld_c, void* workspace /* 256 B: status word */, cudaStream_t st);
 
 }  // namespace amx

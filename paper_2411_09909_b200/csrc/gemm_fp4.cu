@@ -529,19 +529,16 @@ int fp4_block_k() {
 
 }  // namespace
 
-int gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes, const uint8_t* w_scales,
-             int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {
+// The GEMM proper on two prepared operands (each laid out by operand_layout()).
+int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K, float* C,
+                      int64_t ld_c, void* workspace, cudaStream_t st) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AMX_ERR_CUDA;
     const OperandLayout oa = operand_layout(M, K, BM), ow = operand_layout(N, K, BN);
-    uint8_t* base = static_cast<uint8_t*>(workspace);
-    int* status = reinterpret_cast<int*>(base);
-    uint8_t* pa = base + 256;
-    uint8_t* pw = pa + oa.total;
+    const uint8_t* pa = static_cast<const uint8_t*>(a_prepared);
+    const uint8_t* pw = static_cast<const uint8_t*>(w_prepared);
+    int* status = static_cast<int*>(workspace);
     if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return AMX_ERR_CUDA;
-    int rc = prepare(a_codes, a_scales, M, K, oa, pa, st);
-    if (rc == AMX_OK) rc = prepare(w_codes, w_scales, N, K, ow, pw, st);
-    if (rc != AMX_OK) return rc;
     Params p;
     p.sfa_pos = pa + 2 * oa.plane;
     p.sfa_neg = p.sfa_pos + oa.sf;
@@ -554,6 +551,28 @@ int gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_c
     p.vec_store = aligned(C, 32) && ld_c % 8 == 0;     // 32-byte stores in the epilogue
     p.status = status;
     return fp4_block_k() == 256 ? launch_fp4<256>(pa, pw, oa, ow, p, dev, st) : launch_fp4<128>(pa, pw, oa, ow, p, dev, st);
+}
+
+// Size of a prepared operand: as the A operand (rows padded to 128) or the W operand (rows padded to 256).
+size_t gemm_fp4_prepared_bytes(int64_t rows, int64_t K, bool is_weight) {
+    return operand_layout(rows, K, is_weight ? BN : BM).total;
+}
+
+int gemm_fp4_prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, bool is_weight,
+                     void* prepared, cudaStream_t st) {
+    return prepare(codes, scales, rows, K, operand_layout(rows, K, is_weight ? BN : BM), static_cast<uint8_t*>(prepared), st);
+}
+
+int gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes, const uint8_t* w_scales,
+             int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {
+    const OperandLayout oa = operand_layout(M, K, BM), ow = operand_layout(N, K, BN);
+    uint8_t* base = static_cast<uint8_t*>(workspace);
+    uint8_t* pa = base + 256;
+    uint8_t* pw = pa + oa.total;
+    int rc = prepare(a_codes, a_scales, M, K, oa, pa, st);
+    if (rc == AMX_OK) rc = prepare(w_codes, w_scales, N, K, ow, pw, st);
+    if (rc != AMX_OK) return rc;
+    return gemm_fp4_prepared(pa, pw, M, N, K, C, ld_c, base, st);
 }
 
 }  // namespace amx

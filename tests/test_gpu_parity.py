@@ -196,6 +196,17 @@ def test_gemm_tensor_core_matches_simt_at_scale(flag):
     assert rel_fro(tc.cpu().numpy(), simt.cpu().numpy()) <= 1e-5
 
 
+def test_gemm_prepared_two_phase_equals_one_call():
+    a = inputs.random_groups(61, 300, 1056, "mixed")
+    w = inputs.random_groups(62, 520, 1056, "normal")
+    (ac, as_), (wc, ws) = oracle.quantize(a, 32), oracle.quantize(w, 32)
+    ac, as_, wc, ws = (torch.from_numpy(t).cuda() for t in (ac, as_, wc, ws))
+    pa, pw = amx.prepare(ac, as_, False), amx.prepare(wc, ws, True)
+    one = amx.gemm(ac, as_, wc, ws, 32, amx.GEMM_FP4)
+    for _ in range(2):                                       # the prepared weight is reused
+        assert torch.equal(amx.gemm_prepared(pa, pw, 300, 520, 1056), one)
+
+
 def test_gemm_wide_dynamic_range_rows():
     got, ref = _gemm_case(42, 96, 64, 256, 32, amx.GEMM_SIMT, "mixed")
     for m in range(96):                        # row-wise: rows differ by many orders of magnitude
