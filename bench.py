@@ -205,6 +205,11 @@ def run_ours(args):
             "work": torch.empty(ws_bytes, dtype=torch.uint8, device="cuda"),
         })
     stream = torch.cuda.current_stream().cuda_stream
+    fused_prepare = L.amx_gemm_kernel_for(M, layers[0][1], layers[0][0], GS, gemm_flag) == 0x40 and not args.unfused
+    if fused_prepare:
+        for li, (K, N) in enumerate(layers):
+            bufs[li]["pa"] = torch.empty(L.amx_prepared_bytes(M, K, GS, 0), dtype=torch.uint8, device="cuda")
+            bufs[li]["pw"] = torch.empty(L.amx_prepared_bytes(N, K, GS, 1), dtype=torch.uint8, device="cuda")
     gemm_kernel = {0x10: "simt", 0x20: "tcgen05 kind::f16 (bf16 decode)", 0x40: "tcgen05 kind::mxf4nvf4 (sign split)"}[
         L.amx_gemm_kernel_for(M, layers[0][1], layers[0][0], GS, gemm_flag)]
 
@@ -220,13 +225,24 @@ def run_ours(args):
             if record:
                 e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
                 e0.record()
-            check(L.amx_quantize(A[li].data_ptr(), M, K, K, GS, b["ac"].data_ptr(), b["as"].data_ptr(), stream))
-            check(L.amx_quantize(W[li].data_ptr(), N, K, K, GS, b["wc"].data_ptr(), b["ws"].data_ptr(), stream))
-            if record:
-                e1.record()
-            check(L.amx_gemm(b["ac"].data_ptr(), b["as"].data_ptr(), b["wc"].data_ptr(), b["ws"].data_ptr(),
-                             M, N, K, GS, gemm_flag, b["c"].data_ptr(), N, b["work"].data_ptr(), b["work"].numel(),
-                             stream))
+            if fused_prepare:
+                # FP4 kernel: the cast writes the GEMM-ready operand (sign planes, scale factors) directly
+                check(L.amx_quantize_prepared(A[li].data_ptr(), M, K, GS, 0, b["ac"].data_ptr(), b["as"].data_ptr(),
+                                              b["pa"].data_ptr(), b["pa"].numel(), stream))
+                check(L.amx_quantize_prepared(W[li].data_ptr(), N, K, GS, 1, b["wc"].data_ptr(), b["ws"].data_ptr(),
+                                              b["pw"].data_ptr(), b["pw"].numel(), stream))
+                if record:
+                    e1.record()
+                check(L.amx_gemm_prepared(b["pa"].data_ptr(), b["pw"].data_ptr(), M, N, K, GS, b["c"].data_ptr(), N,
+                                          b["work"].data_ptr(), b["work"].numel(), stream))
+            else:
+                check(L.amx_quantize(A[li].data_ptr(), M, K, K, GS, b["ac"].data_ptr(), b["as"].data_ptr(), stream))
+                check(L.amx_quantize(W[li].data_ptr(), N, K, K, GS, b["wc"].data_ptr(), b["ws"].data_ptr(), stream))
+                if record:
+                    e1.record()
+                check(L.amx_gemm(b["ac"].data_ptr(), b["as"].data_ptr(), b["wc"].data_ptr(), b["ws"].data_ptr(),
+                                 M, N, K, GS, gemm_flag, b["c"].data_ptr(), N, b["work"].data_ptr(), b["work"].numel(),
+                                 stream))
             if record:
                 e2.record()
                 ev_q.append((e0, e1))
@@ -292,8 +308,8 @@ def run_ours(args):
         def cached_step(stream):
             for li, (K, N) in enumerate(layers):
                 b, (pa, pw) = bufs[li], prep[li]
-                check(L.amx_quantize(A[li].data_ptr(), M, K, K, GS, b["ac"].data_ptr(), b["as"].data_ptr(), stream))
-                check(L.amx_prepare(b["ac"].data_ptr(), b["as"].data_ptr(), M, K, GS, 0, pa.data_ptr(), pa.numel(), stream))
+                check(L.amx_quantize_prepared(A[li].data_ptr(), M, K, GS, 0, b["ac"].data_ptr(), b["as"].data_ptr(),
+                                              pa.data_ptr(), pa.numel(), stream))
                 check(L.amx_gemm_prepared(pa.data_ptr(), pw.data_ptr(), M, N, K, GS, b["c"].data_ptr(), N,
                                           b["work"].data_ptr(), b["work"].numel(), stream))
 
@@ -393,13 +409,17 @@ def run_ours(args):
         "config": {"workload": "config 2: LLaMA-7B-shaped prefill linears, M=2048, 4 layers; activations and "
                                "weights both cast to AMXFP4 every step, then GEMM",
                    "group_size": GS, "gemm_kernel": gemm_kernel,
+                   "entry_points": "amx_quantize_prepared + amx_gemm_prepared" if fused_prepare else "amx_quantize + amx_gemm",
                    "l2": "per-step inputs (~410 MB of bf16) exceed the 126 MB L2",
                    "launch": "plain launches" if args.no_graph else "CUDA graph of one step, replayed"},
         "pct_of_nominal_fp4_peak": 100.0 * value / world / NOMINAL_FP4_TFLOPS,
         "nominal_fp4_peak_tflops": NOMINAL_FP4_TFLOPS,
         "quantize": {"gb_per_s": quant_gbs, "pct_of_nominal_hbm_8TBs": 100.0 * quant_gbs / NOMINAL_HBM_GBS,
                      "frac_of_measured_copy": quant_gbs / peaks["hbm_gbs"], "bytes_per_element": BYTES_PER_ELEM,
-                     "ms_per_step": q_ms / args.steps, "large_tensor": quant_large},
+                     "ms_per_step": q_ms / args.steps, "large_tensor": quant_large,
+                     "note": ("GB/s counts the canonical bytes only; the step's casts also write the GEMM-ready sign "
+                              "planes and scale factors (+1.125 B/element) and run the scale-factor kernel; "
+                              "large_tensor is the plain amx_quantize") if fused_prepare else "plain amx_quantize"},
         "gemm": {"useful_tflops": gemm_tflops, "ms_per_step": g_ms / args.steps,
                  "pct_of_nominal_fp4_peak": 100.0 * gemm_tflops / NOMINAL_FP4_TFLOPS},
         "roofline": {"bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
@@ -411,6 +431,7 @@ def run_ours(args):
         "clocks": clocks,
         "e2e": e2e,
         # per layer: 2 casts + the GEMM; the FP4 kernel adds one preparation kernel per operand
+        # (with the fused entry points: 2 casts + 2 scale-factor kernels + the GEMM)
         "gpu_launches": (5 if "mxf4" in gemm_kernel else 3) * len(layers) * args.steps,
     }
     if len(layer_ids) != 4:
@@ -430,6 +451,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--gemm", default="auto", choices=["auto", "simt", "tc", "fp4"], help="GEMM kernel to time")
+    ap.add_argument("--unfused", action="store_true", help="amx_quantize + amx_gemm instead of the fused-preparation entry points")
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of a CUDA graph of the step")
     ap.add_argument("--layers", default="", help="comma-separated layer indices to run (profiling aid; default all)")
     ap.add_argument("--skip-extras", action="store_true", help="skip the e2e and cpu_baseline legs (profiling aid)")

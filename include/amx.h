@@ -124,8 +124,13 @@ int amx_gemm(const uint8_t* a_codes, const uint8_t* a_scales,
  *                      (256-byte aligned).  is_weight selects the padding of the W (right-hand) operand.
  *   amx_gemm_prepared  multiplies a prepared A [M, K] with a prepared W [N, K]; same result as amx_gemm
  *                      with AMX_GEMM_FP4.  workspace: 256 bytes (status word, see amx_gemm_status).
+ *   amx_quantize_prepared  amx_quantize (x bf16 [rows, K], contiguous rows, gs = 32) and amx_prepare in one
+ *                      go: the cast kernel itself writes the sign planes, so the codes are not read again.
+ *                      Writes the canonical codes and scales too.
  * This is how Section 4.3's product runs when the weights were cast once ahead of time.
  */
+int amx_quantize_prepared(const void* x, int64_t rows, int64_t K, int group_size, int is_weight,
+                          uint8_t* codes, uint8_t* scales, void* prepared, size_t prepared_bytes, void* stream);
 size_t amx_prepared_bytes(int64_t rows, int64_t K, int group_size, int is_weight);
 int amx_prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, int group_size,
                 int is_weight, void* prepared, size_t prepared_bytes, void* stream);

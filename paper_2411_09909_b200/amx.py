@@ -26,7 +26,7 @@ SYMBOLS = (
     "amx_gemm_kernel_for", "amx_gemm_status", "amx_status_string",
     "amx_quant_gemm_static", "amx_quant_gemm_static_capacity",
     "amx_attention", "amx_attention_workspace_bytes",
-    "amx_prepared_bytes", "amx_prepare", "amx_gemm_prepared",
+    "amx_prepared_bytes", "amx_prepare", "amx_gemm_prepared", "amx_quantize_prepared",
 )
 
 
@@ -55,6 +55,7 @@ def lib() -> ctypes.CDLL:
         L.amx_prepared_bytes.argtypes = [i64, i64, i, i]
         L.amx_prepared_bytes.restype = sz
         L.amx_prepare.argtypes = [p, p, i64, i64, i, i, p, sz, p]
+        L.amx_quantize_prepared.argtypes = [p, i64, i64, i, i, p, p, p, sz, p]
         L.amx_gemm_prepared.argtypes = [p, p, i64, i64, i64, i, p, i64, p, sz, p]
         L.amx_softmax_bf16.argtypes = [p, i64, i64, i64, ctypes.c_float, p, i64, p]
         L.amx_linear_host.argtypes = [p, p, i64, i64, i64, i, u32, p, p, sz, p]
@@ -157,6 +158,19 @@ def prepare(codes: torch.Tensor, scales: torch.Tensor, is_weight: bool, group_si
     _check(lib().amx_prepare(codes.data_ptr(), scales.data_ptr(), rows, K, group_size, int(is_weight), buf.data_ptr(),
                              buf.numel(), _stream()), "amx_prepare")
     return buf
+
+
+def quantize_prepared(x: torch.Tensor, is_weight: bool, group_size: int = 32):
+    """Cast and prepare in one go: returns (codes, scales, prepared)."""
+    _dev(x, torch.bfloat16, "x")
+    assert x.is_contiguous()
+    rows, K = x.shape
+    codes = torch.empty((rows, K // 2), dtype=torch.uint8, device=x.device)
+    scales = torch.empty((rows, K // group_size, 2), dtype=torch.uint8, device=x.device)
+    buf = _ws(lib().amx_prepared_bytes(rows, K, group_size, int(is_weight)), x.device)
+    _check(lib().amx_quantize_prepared(x.data_ptr(), rows, K, group_size, int(is_weight), codes.data_ptr(),
+                                       scales.data_ptr(), buf.data_ptr(), buf.numel(), _stream()), "amx_quantize_prepared")
+    return codes, scales, buf
 
 
 def gemm_prepared(a_prepared: torch.Tensor, w_prepared: torch.Tensor, M: int, N: int, K: int, group_size: int = 32,

@@ -34,4 +34,18 @@ __device__ __forceinline__ float e2m1_mag_to_float(uint32_t c3) {
     return (c3 & 6u) ? v : 0.5f * (float)(c3 & 1u);
 }
 
+// Exponent key of an E5M2 scale byte: unbiased exponent + 17 (1 for 2^-16), 0 for a zero scale.
+__device__ __forceinline__ int scale_key(uint32_t b) {
+    const int e = (b >> 2) & 31, m = b & 3;
+    return e ? e + 2 : (m == 0 ? 0 : (m == 1 ? 1 : 2));
+}
+// UE4M3 byte of the E5M2 byte b for a row whose largest key is kmax (0 when it does not fit).
+__device__ __forceinline__ uint32_t to_ue4m3(uint32_t b, int kmax) {
+    const int e = (b >> 2) & 31, m = b & 3;
+    const int f = scale_key(b) - kmax + 15;                      // UE4M3 exponent field
+    const int mant = e ? m : (m == 3 ? 2 : 0);                   // subnormals: 1, 2, 3 x 2^-16
+    return (f >= 1 && scale_key(b) > 0) ? (uint32_t)((f << 3) | (mant << 1)) : 0u;
+}
+
+
 }  // namespace amx

@@ -111,6 +111,16 @@ extern "C" int amx_prepare(const uint8_t* codes, const uint8_t* scales, int64_t 
     return gemm_fp4_prepare(codes, scales, rows, K, is_weight != 0, prepared, static_cast<cudaStream_t>(stream));
 }
 
+extern "C" int amx_quantize_prepared(const void* x, int64_t rows, int64_t K, int group_size, int is_weight,
+                                     uint8_t* codes, uint8_t* scales, void* prepared, size_t prepared_bytes,
+                                     void* stream) {
+    if (rows <= 0 || !gemm_fp4_supported(rows, rows, K, group_size)) return AMX_ERR_SHAPE;
+    if (!x || !codes || !scales || !prepared) return AMX_ERR_NULL;
+    if (prepared_bytes < amx_prepared_bytes(rows, K, group_size, is_weight)) return AMX_ERR_WORKSPACE;
+    if (!aligned(x, 16) || !aligned(codes, 16) || !aligned(scales, 2) || !aligned(prepared, kAlign)) return AMX_ERR_ALIGN;
+    return gemm_fp4_quantize_prepared(x, rows, K, is_weight != 0, codes, scales, prepared, static_cast<cudaStream_t>(stream));
+}
+
 extern "C" int amx_gemm_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
                                  int group_size, float* C, int64_t ld_c, void* workspace, size_t workspace_bytes,
                                  void* stream) {

@@ -90,19 +90,6 @@ __device__ __forceinline__ uint64_t operand_desc(uint32_t addr) {
 constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
 // ------------------------------------------------------------------------- preparation --
-// Exponent key of an E5M2 scale byte: unbiased exponent + 17 (1 for 2^-16), 0 for a zero scale.
-__device__ __forceinline__ int scale_key(uint32_t b) {
-    const int e = (b >> 2) & 31, m = b & 3;
-    return e ? e + 2 : (m == 0 ? 0 : (m == 1 ? 1 : 2));
-}
-// UE4M3 byte of the E5M2 byte b for a row whose largest key is kmax (0 when it does not fit).
-__device__ __forceinline__ uint32_t to_ue4m3(uint32_t b, int kmax) {
-    const int e = (b >> 2) & 31, m = b & 3;
-    const int f = scale_key(b) - kmax + 15;                      // UE4M3 exponent field
-    const int mant = e ? m : (m == 3 ? 2 : 0);                   // subnormals: 1, 2, 3 x 2^-16
-    return (f >= 1 && scale_key(b) > 0) ? (uint32_t)((f << 3) | (mant << 1)) : 0u;
-}
-
 // One launch per operand; one block per 32 operand rows (rows beyond R, up to the padded row count,
 // get zero scale factors so that padded tile rows multiply zero codes by a finite scale).
 //   1. row offsets: a warp per row finds the largest exponent key kmax among the row's scales;
@@ -115,14 +102,17 @@ constexpr int kPrepRows = 8;
 __global__ void __launch_bounds__(256)
 prepare_operand_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales, int64_t R, int64_t K,
                        int nk64, uint4* __restrict__ pos, uint4* __restrict__ neg, uint8_t* __restrict__ sf_pos,
-                       uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp) {
+                       uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp, const int* __restrict__ kmax_in) {
+    // kmax_in != nullptr: steps 1 and 2 were already done by the cast kernel (fused preparation)
     __shared__ int kmax_s[kPrepRows];
     const int64_t row0 = (int64_t)blockIdx.x * kPrepRows, G = K / 32;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int r = warp; r < kPrepRows; r += 8) {
         const int64_t row = row0 + r;
         int kmax = 0;
-        if (row < R) {
+        if (row < R && kmax_in) {
+            kmax = kmax_in[row];
+        } else if (row < R) {
             const unsigned short* s2 = reinterpret_cast<const unsigned short*>(scales + row * G * 2);
             for (int64_t g = lane; g < G; g += 32) {
                 const uint32_t v = __ldg(s2 + g);
@@ -138,7 +128,7 @@ prepare_operand_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restr
     }
     // sign planes of this block's rows (contiguous in memory: rows are K/2 bytes apart)
     const int64_t rows_here = min((int64_t)kPrepRows, R - row0);
-    if (rows_here > 0) {
+    if (rows_here > 0 && !kmax_in) {
         const int64_t v0 = row0 * (K / 32), n_vec = rows_here * (K / 32);
         const uint4* src = reinterpret_cast<const uint4*>(codes) + v0;
         for (int64_t i = threadIdx.x; i < n_vec; i += 256) {
@@ -469,7 +459,7 @@ OperandLayout operand_layout(int64_t rows, int64_t K, int rows_per_tile) {
     o.nk64 = (int)((K + 255) / 256) * 4;    // padded to whole 256-element blocks
     o.plane = up256((size_t)rows * (K / 2));
     o.sf = up256((size_t)o.row_blocks * o.nk64 * kSfChunk);
-    o.exps = up256((size_t)rows * 4);      // row offsets
+    o.exps = up256((size_t)rows * 4) * 2;  // row offsets, then scratch for the rows' largest exponent keys
     o.total = 2 * o.plane + 2 * o.sf + o.exps;
     return o;
 }
@@ -479,7 +469,7 @@ int prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K
     const int64_t padded_rows = o.row_blocks * 128;
     prepare_operand_kernel<<<(unsigned)(padded_rows / kPrepRows), 256, 0, st>>>(
         codes, scales, rows, K, o.nk64, reinterpret_cast<uint4*>(base), reinterpret_cast<uint4*>(base + o.plane),
-        base + 2 * o.plane, base + 2 * o.plane + o.sf, reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf));
+        base + 2 * o.plane, base + 2 * o.plane + o.sf, reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf), nullptr);
     return launch_status();
 }
 
@@ -556,6 +546,23 @@ int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M,
 // Size of a prepared operand: as the A operand (rows padded to 128) or the W operand (rows padded to 256).
 size_t gemm_fp4_prepared_bytes(int64_t rows, int64_t K, bool is_weight) {
     return operand_layout(rows, K, is_weight ? BN : BM).total;
+}
+
+// Fused form: the cast kernel writes the planes and the rows' exponent-key maxima, a small second kernel the
+// scale factors and row offsets.
+int gemm_fp4_quantize_prepared(const void* x, int64_t rows, int64_t K, bool is_weight, uint8_t* codes, uint8_t* scales,
+                               void* prepared, cudaStream_t st) {
+    const OperandLayout o = operand_layout(rows, K, is_weight ? BN : BM);
+    uint8_t* base = static_cast<uint8_t*>(prepared);
+    int* exps = reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf);
+    int* kmax = reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf + o.exps / 2);
+    if (cudaMemsetAsync(kmax, 0, (size_t)rows * 4, st) != cudaSuccess) return AMX_ERR_CUDA;
+    int rc = quantize_rows_prepared(x, rows, K, codes, scales, base, base + o.plane, kmax, st);
+    if (rc != AMX_OK) return rc;
+    const int64_t padded_rows = o.row_blocks * 128;
+    prepare_operand_kernel<<<(unsigned)(padded_rows / kPrepRows), 256, 0, st>>>(
+        codes, scales, rows, K, o.nk64, nullptr, nullptr, base + 2 * o.plane, base + 2 * o.plane + o.sf, exps, kmax);
+    return launch_status();
 }
 
 int gemm_fp4_prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, bool is_weight,

@@ -129,10 +129,15 @@ __device__ __forceinline__ uint32_t quantize8(const uint4 q, uint32_t& sc) {
 // Groups along the contiguous axis.  Each thread owns EPT = min(gs, 32) consecutive elements
 // (EPT/8 16-byte loads, one EPT/2-byte store); a group is TPG = gs / EPT consecutive lanes, so a
 // 16- or 32-group needs no shuffle and its scales are computed once.  n_items = rows * K / EPT.
-template <int EPT, int TPG, bool CONTIG>
+// With PREP (32-groups, contiguous rows) the kernel also writes what the FP4 GEMM's operand preparation
+// would otherwise derive in a second pass over the codes: the two sign planes (every nibble in the plane of
+// its sign bit, zero in the other) and, per row, the largest exponent key of the row's scales (atomic max).
+template <int EPT, int TPG, bool CONTIG, bool PREP = false>
 __global__ void __launch_bounds__(kThreads)
 quantize_rows_kernel(const uint4* __restrict__ x, int64_t n_items, int64_t items_per_row,
-                     int64_t ld_vec, uint4* __restrict__ codes, uint16_t* __restrict__ scales) {
+                     int64_t ld_vec, uint4* __restrict__ codes, uint16_t* __restrict__ scales,
+                     uint4* __restrict__ pos = nullptr, uint4* __restrict__ neg = nullptr,
+                     int* __restrict__ row_kmax = nullptr) {
     constexpr int NV = EPT / 8;
     const int64_t v = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     uint32_t w[NV * 4];
@@ -159,6 +164,32 @@ quantize_rows_kernel(const uint4* __restrict__ x, int64_t n_items, int64_t items
         if (NV == 4) codes[v] = make_uint4(nib[0], nib[1], nib[2], nib[NV - 1]);
         else *reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(codes) + v * 8) = make_uint2(nib[0], nib[NV - 1]);
         if ((threadIdx.x & (TPG - 1)) == 0) scales[v / TPG] = (uint16_t)sc;
+    }
+    if (PREP) {
+        static_assert(!PREP || (NV == 4 && TPG == 1 && CONTIG), "prepared output: 32-groups of contiguous rows");
+        if (live) {
+            uint32_t pp[4], nn[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t m = ((nib[j] >> 3) & 0x11111111u) * 15u;   // 0xF on negative nibbles
+                nn[j] = nib[j] & m;
+                pp[j] = nib[j] & ~m;
+            }
+            pos[v] = make_uint4(pp[0], pp[1], pp[2], pp[3]);
+            neg[v] = make_uint4(nn[0], nn[1], nn[2], nn[3]);
+        }
+        // row maximum of the scale exponent keys: one atomic per warp when the warp sits inside one row
+        const int key = live ? max(scale_key(sc & 0xFFu), scale_key(sc >> 8)) : 0;
+        const int64_t row = v / items_per_row;
+        const int64_t v_first = v - (threadIdx.x & 31), v_last = min(v_first + 31, n_items - 1);
+        if (v_first < n_items) {
+            if (v_first / items_per_row == v_last / items_per_row) {
+                const int wmax = __reduce_max_sync(0xFFFFFFFFu, key);
+                if ((threadIdx.x & 31) == 0 && wmax > 0) atomicMax(row_kmax + row, wmax);
+            } else if (live && key > 0) {
+                atomicMax(row_kmax + row, key);
+            }
+        }
     }
 }
 
@@ -215,6 +246,23 @@ int launch_rows(const void* x, int64_t rows, int64_t K, int64_t ld, uint8_t* cod
         quantize_rows_kernel<EPT, TPG, false><<<(unsigned)blocks, kThreads, 0, st>>>(xv, n_items, K / EPT, ld / 8, cv, sv);
     return launch_status();
 }
+
+}  // namespace
+
+// Cast with fused FP4-operand preparation (gs = 32, contiguous rows): canonical codes and scales plus the
+// sign planes and the per-row maximum exponent keys (row_kmax must be zero on entry).
+int quantize_rows_prepared(const void* x, int64_t rows, int64_t K, uint8_t* codes, uint8_t* scales, void* pos,
+                           void* neg, int* row_kmax, cudaStream_t st) {
+    const int64_t n_items = rows * (K / 32);
+    const int64_t blocks = (n_items + kThreads - 1) / kThreads;
+    if (blocks > 0x7FFFFFFF) return AMX_ERR_SHAPE;
+    quantize_rows_kernel<32, 1, true, true><<<(unsigned)blocks, kThreads, 0, st>>>(
+        reinterpret_cast<const uint4*>(x), n_items, K / 32, K / 8, reinterpret_cast<uint4*>(codes),
+        reinterpret_cast<uint16_t*>(scales), reinterpret_cast<uint4*>(pos), reinterpret_cast<uint4*>(neg), row_kmax);
+    return launch_status();
+}
+
+namespace {
 
 template <int TPG>
 int launch_cols(const void* x, int64_t R, int64_t C, int64_t ld, int gs, uint8_t* codes,

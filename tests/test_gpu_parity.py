@@ -207,6 +207,29 @@ def test_gemm_prepared_two_phase_equals_one_call():
         assert torch.equal(amx.gemm_prepared(pa, pw, 300, 520, 1056), one)
 
 
+def test_quantize_prepared_equals_quantize_then_prepare():
+    for rows, K, is_w, kind in ((300, 1056, False, "mixed"), (520, 1056, True, "wide"), (130, 96, True, "mixed")):
+        bits = inputs.random_groups(63, rows, K, kind)
+        x = dev_bf16(bits)
+        c, s_, prep = amx.quantize_prepared(x, is_w)
+        c2, s2 = amx.quantize(x, 32)
+        assert torch.equal(c, c2) and torch.equal(s_, s2)
+        oc, os_ = oracle.quantize(bits, 32)
+        assert np.array_equal(c.cpu().numpy(), oc) and np.array_equal(s_.cpu().numpy(), os_)
+        # the prepared operands drive the GEMM to the same result
+        w_bits = inputs.random_groups(64, 200, K, "normal")
+        wc, ws = amx.quantize(dev_bf16(w_bits), 32)
+        if is_w:
+            other = amx.prepare(wc, ws, False)
+            got = amx.gemm_prepared(other, prep, 200, rows, K)
+            want = amx.gemm_prepared(other, amx.prepare(c2, s2, True), 200, rows, K)
+        else:
+            other = amx.prepare(wc, ws, True)
+            got = amx.gemm_prepared(prep, other, rows, 200, K)
+            want = amx.gemm_prepared(amx.prepare(c2, s2, False), other, rows, 200, K)
+        assert torch.equal(got, want)
+
+
 def test_gemm_wide_dynamic_range_rows():
     got, ref = _gemm_case(42, 96, 64, 256, 32, amx.GEMM_SIMT, "mixed")
     for m in range(96):                        # row-wise: rows differ by many orders of magnitude
