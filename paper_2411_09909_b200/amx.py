@@ -160,14 +160,14 @@ def prepare(codes: torch.Tensor, scales: torch.Tensor, is_weight: bool, group_si
     return buf
 
 
-def quantize_prepared(x: torch.Tensor, is_weight: bool, group_size: int = 32):
+def quantize_prepared(x: torch.Tensor, is_weight: bool, group_size: int = 32, prepared: torch.Tensor | None = None):
     """Cast and prepare in one go: returns (codes, scales, prepared)."""
     _dev(x, torch.bfloat16, "x")
     assert x.is_contiguous()
     rows, K = x.shape
     codes = torch.empty((rows, K // 2), dtype=torch.uint8, device=x.device)
     scales = torch.empty((rows, K // group_size, 2), dtype=torch.uint8, device=x.device)
-    buf = _ws(lib().amx_prepared_bytes(rows, K, group_size, int(is_weight)), x.device)
+    buf = prepared if prepared is not None else _ws(lib().amx_prepared_bytes(rows, K, group_size, int(is_weight)), x.device)
     _check(lib().amx_quantize_prepared(x.data_ptr(), rows, K, group_size, int(is_weight), codes.data_ptr(),
                                        scales.data_ptr(), buf.data_ptr(), buf.numel(), _stream()), "amx_quantize_prepared")
     return codes, scales, buf

@@ -31,7 +31,8 @@ int gemm_fp4_prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, 
 int gemm_fp4_quantize_prepared(const void* x, int64_t rows, int64_t K, bool is_weight, uint8_t* codes,
                                uint8_t* scales, void* prepared, cudaStream_t st);
 int quantize_rows_prepared(const void* x, int64_t rows, int64_t K, uint8_t* codes, uint8_t* scales, void* pos,
-                           void* neg, int* row_kmax, cudaStream_t st);
+                           void* neg, uint8_t* sf_pos, uint8_t* sf_neg, int* row_exp, int nk64, int64_t padded_rows,
+                           cudaStream_t st);
 int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
                       float* C, int64_t ld_c, void* workspace /* 256 B: status word */, cudaStream_t st);
 

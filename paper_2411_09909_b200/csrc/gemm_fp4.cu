@@ -102,17 +102,14 @@ constexpr int kPrepRows = 8;
 __global__ void __launch_bounds__(256)
 prepare_operand_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales, int64_t R, int64_t K,
                        int nk64, uint4* __restrict__ pos, uint4* __restrict__ neg, uint8_t* __restrict__ sf_pos,
-                       uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp, const int* __restrict__ kmax_in) {
-    // kmax_in != nullptr: steps 1 and 2 were already done by the cast kernel (fused preparation)
+                       uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp) {
     __shared__ int kmax_s[kPrepRows];
     const int64_t row0 = (int64_t)blockIdx.x * kPrepRows, G = K / 32;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int r = warp; r < kPrepRows; r += 8) {
         const int64_t row = row0 + r;
         int kmax = 0;
-        if (row < R && kmax_in) {
-            kmax = kmax_in[row];
-        } else if (row < R) {
+        if (row < R) {
             const unsigned short* s2 = reinterpret_cast<const unsigned short*>(scales + row * G * 2);
             for (int64_t g = lane; g < G; g += 32) {
                 const uint32_t v = __ldg(s2 + g);
@@ -128,7 +125,7 @@ prepare_operand_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restr
     }
     // sign planes of this block's rows (contiguous in memory: rows are K/2 bytes apart)
     const int64_t rows_here = min((int64_t)kPrepRows, R - row0);
-    if (rows_here > 0 && !kmax_in) {
+    if (rows_here > 0) {
         const int64_t v0 = row0 * (K / 32), n_vec = rows_here * (K / 32);
         const uint4* src = reinterpret_cast<const uint4*>(codes) + v0;
         for (int64_t i = threadIdx.x; i < n_vec; i += 256) {
@@ -459,7 +456,7 @@ OperandLayout operand_layout(int64_t rows, int64_t K, int rows_per_tile) {
     o.nk64 = (int)((K + 255) / 256) * 4;    // padded to whole 256-element blocks
     o.plane = up256((size_t)rows * (K / 2));
     o.sf = up256((size_t)o.row_blocks * o.nk64 * kSfChunk);
-    o.exps = up256((size_t)rows * 4) * 2;  // row offsets, then scratch for the rows' largest exponent keys
+    o.exps = up256((size_t)rows * 4);      // row offsets
     o.total = 2 * o.plane + 2 * o.sf + o.exps;
     return o;
 }
@@ -469,7 +466,7 @@ int prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K
     const int64_t padded_rows = o.row_blocks * 128;
     prepare_operand_kernel<<<(unsigned)(padded_rows / kPrepRows), 256, 0, st>>>(
         codes, scales, rows, K, o.nk64, reinterpret_cast<uint4*>(base), reinterpret_cast<uint4*>(base + o.plane),
-        base + 2 * o.plane, base + 2 * o.plane + o.sf, reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf), nullptr);
+        base + 2 * o.plane, base + 2 * o.plane + o.sf, reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf));
     return launch_status();
 }
 
@@ -548,21 +545,14 @@ size_t gemm_fp4_prepared_bytes(int64_t rows, int64_t K, bool is_weight) {
     return operand_layout(rows, K, is_weight ? BN : BM).total;
 }
 
-// Fused form: the cast kernel writes the planes and the rows' exponent-key maxima, a small second kernel the
-// scale factors and row offsets.
+// Fused form: one launch of the cast kernel writes the canonical operand and the prepared one.
 int gemm_fp4_quantize_prepared(const void* x, int64_t rows, int64_t K, bool is_weight, uint8_t* codes, uint8_t* scales,
                                void* prepared, cudaStream_t st) {
     const OperandLayout o = operand_layout(rows, K, is_weight ? BN : BM);
     uint8_t* base = static_cast<uint8_t*>(prepared);
-    int* exps = reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf);
-    int* kmax = reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf + o.exps / 2);
-    if (cudaMemsetAsync(kmax, 0, (size_t)rows * 4, st) != cudaSuccess) return AMX_ERR_CUDA;
-    int rc = quantize_rows_prepared(x, rows, K, codes, scales, base, base + o.plane, kmax, st);
-    if (rc != AMX_OK) return rc;
-    const int64_t padded_rows = o.row_blocks * 128;
-    prepare_operand_kernel<<<(unsigned)(padded_rows / kPrepRows), 256, 0, st>>>(
-        codes, scales, rows, K, o.nk64, nullptr, nullptr, base + 2 * o.plane, base + 2 * o.plane + o.sf, exps, kmax);
-    return launch_status();
+    return quantize_rows_prepared(x, rows, K, codes, scales, base, base + o.plane, base + 2 * o.plane,
+                                  base + 2 * o.plane + o.sf, reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf), o.nk64,
+                                  o.row_blocks * 128, st);
 }
 
 int gemm_fp4_prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, bool is_weight,

@@ -1,117 +1,16 @@
 // bf16 -> AMXFP4 direct cast (arXiv 2411.09909, Sections 4.2-4.3; Algorithm 1 applied per sign
-// with the FP8 E5M2 shared scale).  HBM-bound: 2 B read + 0.5625 B written per element.
-//
-// Exactness of the arithmetic (all decisions are bit-identical to exact rational arithmetic):
-//   * Side maxima are taken on the bf16 bit patterns as signed 16-bit integers.  Non-negative
-//     floats order like their bit patterns, negative ones become non-negative after flipping
-//     the sign bit, and the other side is removed by the max with 0.
-//   * scale = RNE_E5M2(max / 6) and magnitude = RNE_E2M1(|x| / scale) are evaluated as
-//     "multiply by a reciprocal that is slightly too large, then truncate to 12 significant
-//     bits".  max and x have 8 significant bits and every rounding midpoint times its divisor
-//     has at most 6, so a quotient is either exactly a midpoint (the tie: the product then
-//     overshoots by < 2^-18 relative and truncation returns the midpoint itself, which the
-//     converter resolves to even) or at least 2^-8 relative away from every midpoint
-//     (overshoot + truncation move it by < 2^-11: it stays on its side).
-//   * The final roundings are the hardware converts cvt.rn.satfinite.{e5m2x2,e2m1x2}.f32.
+// with the FP8 E5M2 shared scale).  HBM-bound: 2 B read + 0.5625 B written per element.  The per-group
+// arithmetic, with the argument for its exactness, is in cast_math.cuh.
 #include <cuda_bf16.h>
 
-#include "amx_common.cuh"
+#include "cast_math.cuh"
 
 namespace amx {
 namespace {
 
+using namespace cast;
+
 constexpr int kThreads = 256;
-
-// 1/6 rounded up a few ulps (0x3E2AAAAB is the nearest float, already above 1/6).
-__device__ __forceinline__ float sixth_up() { return __uint_as_float(0x3E2AAAAFu); }
-
-__device__ __forceinline__ float trunc12(float v) {
-    return __uint_as_float(__float_as_uint(v) & 0xFFFFF000u);
-}
-
-// {hi, lo} -> two E5M2 bytes, hi in bits 15..8.
-__device__ __forceinline__ uint32_t cvt_e5m2x2(float hi, float lo) {
-    unsigned short d;
-    asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));
-    return d;
-}
-
-// Four pairs of quotients -> eight E2M1 nibbles; element i lands in nibble i.
-__device__ __forceinline__ uint32_t cvt_e2m1x8(const float (&r)[8]) {
-    uint32_t d;
-    asm("{\n"
-        ".reg .b8 b0, b1, b2, b3;\n"
-        "cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n"
-        "cvt.rn.satfinite.e2m1x2.f32 b1, %4, %3;\n"
-        "cvt.rn.satfinite.e2m1x2.f32 b2, %6, %5;\n"
-        "cvt.rn.satfinite.e2m1x2.f32 b3, %8, %7;\n"
-        "mov.b32 %0, {b0, b1, b2, b3};\n"
-        "}"
-        : "=r"(d)
-        : "f"(r[0]), "f"(r[1]), "f"(r[2]), "f"(r[3]), "f"(r[4]), "f"(r[5]), "f"(r[6]), "f"(r[7]));
-    return d;
-}
-
-// Reciprocal of an E5M2 value, biased upward by < 2^-18 relative; 0 for a zero scale.
-__device__ __forceinline__ float inv_scale_up(float s) {
-    float r;
-    asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(s));
-    r = __uint_as_float(__float_as_uint(r) + 16u);
-    return s > 0.0f ? r : 0.0f;
-}
-
-// Side maxima of NW bf16x2 words as one word {nmax bits : pmax bits}.  Signed 16-bit max over the
-// raw patterns, clamped at 0, is the largest non-negative value; unsigned 16-bit max is the negative
-// value of largest magnitude whenever a negative one exists (its sign bit is then flipped away).
-template <int NW>
-__device__ __forceinline__ uint32_t side_maxima(const uint32_t (&w)[NW]) {
-    uint32_t pm = w[0], nm = w[0];
-#pragma unroll
-    for (int i = 1; i + 1 < NW; i += 2) {
-        pm = __vimax3_s16x2(pm, w[i], w[i + 1]);
-        nm = __vimax3_u16x2(nm, w[i], w[i + 1]);
-    }
-    if (NW % 2 == 0) {
-        pm = __vmaxs2(pm, w[NW - 1]);
-        nm = __vmaxu2(nm, w[NW - 1]);
-    }
-    nm ^= 0x80008000u;
-    pm = __vimax_s16x2_relu(pm, pm);
-    nm = __vimax_s16x2_relu(nm, nm);
-    return __vmaxs2(__byte_perm(pm, nm, 0x5410), __byte_perm(pm, nm, 0x7632));
-}
-
-// The two E5M2 scale bytes of a group from its side maxima {nmax : pmax} (positive side in bits
-// 7..0, negative side in bits 15..8), and the two biased reciprocals the elements are multiplied by.
-__device__ __forceinline__ uint32_t group_scales(uint32_t c, float& inv_p, float& inv_n) {
-    const float pmax = __uint_as_float(c << 16);
-    const float nmax = __uint_as_float(c & 0xFFFF0000u);
-    const uint32_t sc = cvt_e5m2x2(trunc12(nmax * sixth_up()), trunc12(pmax * sixth_up()));
-    inv_p = inv_scale_up(e5m2_to_float(sc & 0xFFu));
-    inv_n = inv_scale_up(e5m2_to_float(sc >> 8));
-    return sc;
-}
-
-// x * (sign(x) ? inv_n : inv_p).  The choice is an integer multiply-add on the reciprocals' bit
-// patterns (inv_p + sign * (inv_n - inv_p)): it runs on the FMA pipe, which this kernel leaves
-// mostly idle, instead of adding a compare and a select to the saturated integer/logic pipe.
-__device__ __forceinline__ float scale_by_side(uint32_t x_bits, uint32_t inv_p, uint32_t inv_diff) {
-    uint32_t sel;
-    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(sel) : "r"(x_bits >> 31), "r"(inv_diff), "r"(inv_p));
-    return __uint_as_float(x_bits) * __uint_as_float(sel);
-}
-
-// 8 consecutive elements (4 bf16x2 words) -> 8 nibbles.
-__device__ __forceinline__ uint32_t encode8(const uint32_t* w, float inv_p, float inv_n) {
-    const uint32_t ip = __float_as_uint(inv_p), idiff = __float_as_uint(inv_n) - ip;
-    float r[8];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        r[2 * i] = trunc12(scale_by_side(w[i] << 16, ip, idiff));
-        r[2 * i + 1] = trunc12(scale_by_side(w[i] & 0xFFFF0000u, ip, idiff));
-    }
-    return cvt_e2m1x8(r);
-}
 
 // Quantizes 8 consecutive elements held as 4 bf16x2 words.  TPG threads (8*TPG = group size) hold
 // one group and sit in consecutive lanes.  Returns the 8 nibbles; `sc` receives the scale bytes.
@@ -129,15 +28,10 @@ __device__ __forceinline__ uint32_t quantize8(const uint4 q, uint32_t& sc) {
 // Groups along the contiguous axis.  Each thread owns EPT = min(gs, 32) consecutive elements
 // (EPT/8 16-byte loads, one EPT/2-byte store); a group is TPG = gs / EPT consecutive lanes, so a
 // 16- or 32-group needs no shuffle and its scales are computed once.  n_items = rows * K / EPT.
-// With PREP (32-groups, contiguous rows) the kernel also writes what the FP4 GEMM's operand preparation
-// would otherwise derive in a second pass over the codes: the two sign planes (every nibble in the plane of
-// its sign bit, zero in the other) and, per row, the largest exponent key of the row's scales (atomic max).
-template <int EPT, int TPG, bool CONTIG, bool PREP = false>
+template <int EPT, int TPG, bool CONTIG>
 __global__ void __launch_bounds__(kThreads)
 quantize_rows_kernel(const uint4* __restrict__ x, int64_t n_items, int64_t items_per_row,
-                     int64_t ld_vec, uint4* __restrict__ codes, uint16_t* __restrict__ scales,
-                     uint4* __restrict__ pos = nullptr, uint4* __restrict__ neg = nullptr,
-                     int* __restrict__ row_kmax = nullptr) {
+                     int64_t ld_vec, uint4* __restrict__ codes, uint16_t* __restrict__ scales) {
     constexpr int NV = EPT / 8;
     const int64_t v = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     uint32_t w[NV * 4];
@@ -164,32 +58,6 @@ quantize_rows_kernel(const uint4* __restrict__ x, int64_t n_items, int64_t items
         if (NV == 4) codes[v] = make_uint4(nib[0], nib[1], nib[2], nib[NV - 1]);
         else *reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(codes) + v * 8) = make_uint2(nib[0], nib[NV - 1]);
         if ((threadIdx.x & (TPG - 1)) == 0) scales[v / TPG] = (uint16_t)sc;
-    }
-    if (PREP) {
-        static_assert(!PREP || (NV == 4 && TPG == 1 && CONTIG), "prepared output: 32-groups of contiguous rows");
-        if (live) {
-            uint32_t pp[4], nn[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint32_t m = ((nib[j] >> 3) & 0x11111111u) * 15u;   // 0xF on negative nibbles
-                nn[j] = nib[j] & m;
-                pp[j] = nib[j] & ~m;
-            }
-            pos[v] = make_uint4(pp[0], pp[1], pp[2], pp[3]);
-            neg[v] = make_uint4(nn[0], nn[1], nn[2], nn[3]);
-        }
-        // row maximum of the scale exponent keys: one atomic per warp when the warp sits inside one row
-        const int key = live ? max(scale_key(sc & 0xFFu), scale_key(sc >> 8)) : 0;
-        const int64_t row = v / items_per_row;
-        const int64_t v_first = v - (threadIdx.x & 31), v_last = min(v_first + 31, n_items - 1);
-        if (v_first < n_items) {
-            if (v_first / items_per_row == v_last / items_per_row) {
-                const int wmax = __reduce_max_sync(0xFFFFFFFFu, key);
-                if ((threadIdx.x & 31) == 0 && wmax > 0) atomicMax(row_kmax + row, wmax);
-            } else if (live && key > 0) {
-                atomicMax(row_kmax + row, key);
-            }
-        }
     }
 }
 
@@ -231,6 +99,85 @@ quantize_cols_kernel(const __nv_bfloat16* __restrict__ x, int64_t R, int64_t C, 
     }
 }
 
+// The cast for an operand of the FP4 GEMM (32-groups, contiguous rows).  Besides the canonical codes and scales
+// it writes, in the same pass, everything the GEMM reads: the two sign planes (every nibble in the plane of its
+// sign bit, zero in the other), the UE4M3 scale factors of both planes - byte (r%32)*16 + (r/32)*4 + k16%4 of
+// the 512-byte chunk of [128 rows x 64 elements]; one scale per 16 elements, so a 32-group's scale is stored
+// twice - and per row the power of two by which those scale factors understate the true scales
+// (row_exp = largest exponent key of the row - 25).  The scale factors depend on the row's largest scale, so a
+// block owns whole rows, one thread per group (threads stride over the groups when a row is longer than the
+// block).  Blocks past the last row, and groups past the last group, zero the padding of the scale-factor
+// array, so that padded tile rows and columns multiply zero codes by a finite scale.
+// Block shape (GX, RB): thread (x, y) owns groups x, x + GX, ... of row blockIdx.x * RB + y.  GX is a multiple
+// of 32, so a warp never spans two rows.
+constexpr int kPrepMaxRows = 8;
+constexpr int kSfChunkBytes = 512;
+
+// 40 registers (three blocks of 512 per SM): at 32 the kernel spills and is 12 % slower.
+__global__ void __launch_bounds__(512, 3)
+cast_prepared_kernel(const uint4* __restrict__ x, int64_t R, int G, uint4* __restrict__ codes,
+                     uint16_t* __restrict__ scales, uint4* __restrict__ pos, uint4* __restrict__ neg,
+                     uint8_t* __restrict__ sf_pos, uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp, int nk64) {
+    __shared__ int kmax_s[kPrepMaxRows];
+    const int gx = threadIdx.x, rl = threadIdx.y, GX = blockDim.x;
+    const int64_t row = (int64_t)blockIdx.x * blockDim.y + rl;
+    const bool row_live = row < R;
+    if (gx == 0) kmax_s[rl] = 0;
+    __syncthreads();
+    const int64_t v_row = row * G;
+    uint32_t sc_first = 0;                      // scale bytes of this thread's first group (its only one when
+                                                // the block is as wide as its rows)
+    uint32_t top = 0;                           // largest scale byte seen by this thread
+    for (int g = gx; g < G; g += GX) {
+        if (!row_live) break;                   // uniform over the warp: a warp sits inside one row
+        const int64_t v = v_row + g;
+        uint32_t w[16];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint4 q = __ldg(x + v * 4 + j);
+            w[4 * j] = q.x; w[4 * j + 1] = q.y; w[4 * j + 2] = q.z; w[4 * j + 3] = q.w;
+        }
+        float inv_p, inv_n;
+        const uint32_t sc = group_scales(side_maxima<16>(w), inv_p, inv_n);
+        uint32_t nib[4], pp[4], nn[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            nib[j] = encode8(w + 4 * j, inv_p, inv_n);
+            const uint32_t m = ((nib[j] >> 3) & 0x11111111u) * 15u;   // 0xF on negative nibbles
+            nn[j] = nib[j] & m;
+            pp[j] = nib[j] & ~m;
+        }
+        codes[v] = make_uint4(nib[0], nib[1], nib[2], nib[3]);
+        pos[v] = make_uint4(pp[0], pp[1], pp[2], pp[3]);
+        neg[v] = make_uint4(nn[0], nn[1], nn[2], nn[3]);
+        scales[v] = (uint16_t)sc;
+        if (g == gx) sc_first = sc;
+        top = max(top, max(sc & 0xFFu, sc >> 8));
+    }
+    // Row maximum of the exponent keys, one shared-memory atomic per warp.  The key of an E5M2 byte grows
+    // with the byte (scales carry no sign bit), so the largest byte has the largest key.
+    top = __reduce_max_sync(0xFFFFFFFFu, top);
+    if ((gx & 31) == 0 && top > 0) atomicMax(&kmax_s[rl], scale_key(top));
+    __syncthreads();
+    const int kmax = kmax_s[rl];
+    // offset of this row's bytes inside a chunk; the chunks of one block of 128 rows are consecutive along K
+    const int rr = (int)(row & 127);
+    const int64_t sf_row = (row >> 7) * nk64 * (int64_t)kSfChunkBytes + (rr & 31) * 16 + (rr >> 5) * 4;
+    for (int g = gx; g < nk64 * 2; g += GX) {      // groups past G: padding to whole 256-element blocks
+        uint32_t up = 0, un = 0;
+        if (row_live && g < G) {
+            // a later group of a striding thread: re-read the scale bytes this thread stored above
+            const uint32_t sc = (g == gx) ? sc_first : scales[v_row + g];
+            up = to_ue4m3(sc & 0xFFu, kmax);
+            un = to_ue4m3(sc >> 8, kmax);
+        }
+        const int64_t off = sf_row + (g >> 1) * kSfChunkBytes + (g & 1) * 2;
+        *reinterpret_cast<uint16_t*>(sf_pos + off) = (uint16_t)(up | (up << 8));
+        *reinterpret_cast<uint16_t*>(sf_neg + off) = (uint16_t)(un | (un << 8));
+    }
+    if (gx == 0 && row_live) row_exp[row] = kmax ? kmax - 25 : 0;
+}
+
 template <int EPT, int TPG>
 int launch_rows(const void* x, int64_t rows, int64_t K, int64_t ld, uint8_t* codes,
                 uint8_t* scales, cudaStream_t st) {
@@ -249,16 +196,23 @@ int launch_rows(const void* x, int64_t rows, int64_t K, int64_t ld, uint8_t* cod
 
 }  // namespace
 
-// Cast with fused FP4-operand preparation (gs = 32, contiguous rows): canonical codes and scales plus the
-// sign planes and the per-row maximum exponent keys (row_kmax must be zero on entry).
+// Cast with the FP4 GEMM's operand preparation in the same launch (gs = 32, contiguous rows): canonical codes
+// and scales, the two sign planes, the UE4M3 scale factors of both planes in the tensor cores' layout (nk64
+// chunks of 512 B per block of 128 rows, rows padded to padded_rows) and the rows' power-of-two offsets.
 int quantize_rows_prepared(const void* x, int64_t rows, int64_t K, uint8_t* codes, uint8_t* scales, void* pos,
-                           void* neg, int* row_kmax, cudaStream_t st) {
-    const int64_t n_items = rows * (K / 32);
-    const int64_t blocks = (n_items + kThreads - 1) / kThreads;
+                           void* neg, uint8_t* sf_pos, uint8_t* sf_neg, int* row_exp, int nk64, int64_t padded_rows,
+                           cudaStream_t st) {
+    const int64_t G = K / 32;
+    // one thread per group when a row fits a block of 512, several rows per block when rows are short
+    const int gx = (int)((G < 512 ? G : 512) + 31) / 32 * 32;
+    int rb = 1;
+    while (rb < kPrepMaxRows && rb * 2 * gx <= 256) rb *= 2;
+    const int64_t blocks = (padded_rows + rb - 1) / rb;
     if (blocks > 0x7FFFFFFF) return AMX_ERR_SHAPE;
-    quantize_rows_kernel<32, 1, true, true><<<(unsigned)blocks, kThreads, 0, st>>>(
-        reinterpret_cast<const uint4*>(x), n_items, K / 32, K / 8, reinterpret_cast<uint4*>(codes),
-        reinterpret_cast<uint16_t*>(scales), reinterpret_cast<uint4*>(pos), reinterpret_cast<uint4*>(neg), row_kmax);
+    cast_prepared_kernel<<<(unsigned)blocks, dim3(gx, rb), 0, st>>>(
+        reinterpret_cast<const uint4*>(x), rows, (int)G, reinterpret_cast<uint4*>(codes),
+        reinterpret_cast<uint16_t*>(scales), reinterpret_cast<uint4*>(pos), reinterpret_cast<uint4*>(neg), sf_pos, sf_neg,
+        row_exp, nk64);
     return launch_status();
 }
 

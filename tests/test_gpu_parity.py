@@ -208,10 +208,16 @@ def test_gemm_prepared_two_phase_equals_one_call():
 
 
 def test_quantize_prepared_equals_quantize_then_prepare():
-    for rows, K, is_w, kind in ((300, 1056, False, "mixed"), (520, 1056, True, "wide"), (130, 96, True, "mixed")):
+    # row lengths below, at and above one block of the cast kernel (several rows, one row and a fraction of a
+    # row per block; threads striding over a long row), ragged row counts, both paddings
+    cases = ((300, 1056, False, "mixed"), (520, 1056, True, "wide"), (130, 96, True, "mixed"), (8, 32, False, "normal"),
+             (77, 11008, False, "mixed"), (20, 16448, True, "mixed"), (129, 4096, True, "wide"))
+    for rows, K, is_w, kind in cases:
         bits = inputs.random_groups(63, rows, K, kind)
         x = dev_bf16(bits)
-        c, s_, prep = amx.quantize_prepared(x, is_w)
+        # a buffer full of 0xFF: every byte the GEMM reads must have been written by the call
+        dirty = torch.full((amx.lib().amx_prepared_bytes(rows, K, 32, int(is_w)),), 0xFF, dtype=torch.uint8, device="cuda")
+        c, s_, prep = amx.quantize_prepared(x, is_w, prepared=dirty)
         c2, s2 = amx.quantize(x, 32)
         assert torch.equal(c, c2) and torch.equal(s_, s2)
         oc, os_ = oracle.quantize(bits, 32)
