@@ -62,6 +62,12 @@ typedef enum amx_status {
                               * than 14 binades below the largest scale of their operand row are flushed to
                               * zero (relative effect < 2^-14 per row); otherwise same result up to fp32
                               * summation order.  Needs the larger workspace amx_workspace_bytes() reports. */
+/* extra flag for amx_quant_gemm, only together with AMX_GEMM_TC: one launch, the GEMM's operand-staging
+ * warps cast each activation tile to AMXFP4 in registers instead of reading codes a separate cast launch
+ * wrote.  Bit-identical result.  The tile is cast once per column of output tiles, and the staging warps
+ * are what bounds that kernel, so this is slower than the default two launches (measured 1.05x at
+ * 128 x 1024 x 1024, 1.25x at 2048 x 12288 x 4096); it is for callers that must not hold the codes. */
+#define AMX_GEMM_CAST_IN_KERNEL 0x80u
 
 /*
  * amx_quantize - direct cast of a bf16 matrix to AMXFP4 (Sections 4.2-4.3; procedure per
@@ -142,7 +148,9 @@ int amx_gemm_prepared(const void* a_prepared, const void* w_prepared, int64_t M,
  * amx_quant_gemm - the fully quantized linear layer of Section 5 ("quantize input operands for
  * all decoder-layer matrix multiplications"): quantizes the bf16 activation A[M, ld_a] and
  * multiplies it with an already quantized weight.  Same result as amx_quantize followed by
- * amx_gemm.  The workspace additionally holds the quantized activation.
+ * amx_gemm, which is also how it runs (two launches; the workspace additionally holds the quantized
+ * activation) unless AMX_GEMM_TC | AMX_GEMM_CAST_IN_KERNEL asks for the single-launch kernel.
+ * AMX_GEMM_CAST_IN_KERNEL with any other kernel choice: AMX_ERR_FLAGS.  A 16-byte aligned, ld_a % 8 == 0.
  */
 int amx_quant_gemm(const void* A, int64_t ld_a,
                    const uint8_t* w_codes, const uint8_t* w_scales,

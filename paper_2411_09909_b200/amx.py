@@ -17,6 +17,7 @@ _lib = None
 
 OUT_BF16, OUT_F32 = 0x0, 0x1
 GEMM_AUTO, GEMM_SIMT, GEMM_TC, GEMM_FP4 = 0x0, 0x10, 0x20, 0x40
+GEMM_CAST_IN_KERNEL = 0x80      # amx_quant_gemm only, together with GEMM_TC
 
 # every symbol include/amx.h declares
 SYMBOLS = (
@@ -196,7 +197,7 @@ def quant_gemm(a: torch.Tensor, w_codes, w_scales, group_size: int = 32, flags: 
     N = w_codes.shape[0]
     if out is None:
         out = torch.empty((M, N), dtype=torch.float32, device=a.device)
-    need = lib().amx_quant_gemm_workspace_bytes(M, N, K, group_size, flags)
+    need = lib().amx_quant_gemm_workspace_bytes(M, N, K, group_size, flags & ~GEMM_CAST_IN_KERNEL)
     if workspace is None:
         workspace = _ws(need, a.device)
     _check(lib().amx_quant_gemm(a.data_ptr(), a.stride(0), w_codes.data_ptr(), w_scales.data_ptr(), M, N, K,

@@ -135,6 +135,9 @@ extern "C" int amx_gemm_prepared(const void* a_prepared, const void* w_prepared,
 extern "C" int amx_quant_gemm(const void* A, int64_t ld_a, const uint8_t* w_codes, const uint8_t* w_scales,
                               int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags, float* C,
                               int64_t ld_c, void* workspace, size_t workspace_bytes, void* stream) {
+    const bool cast_in_kernel = flags & AMX_GEMM_CAST_IN_KERNEL;
+    if (cast_in_kernel && (flags & kKernelMask) != AMX_GEMM_TC) return AMX_ERR_FLAGS;
+    flags &= ~AMX_GEMM_CAST_IN_KERNEL;
     if (flags & ~kKernelMask) return AMX_ERR_FLAGS;
     if (!gemm_shape_ok(M, N, K, group_size) || ld_a < K || ld_c < N) return AMX_ERR_SHAPE;
     if (M == 0 || N == 0) return AMX_OK;
@@ -144,6 +147,15 @@ extern "C" int amx_quant_gemm(const void* A, int64_t ld_a, const uint8_t* w_code
     const size_t gemm_ws = amx_workspace_bytes(M, N, K, group_size, flags);
     const QuantSizes a = quant_sizes(M, K, group_size);
     uint8_t* base = static_cast<uint8_t*>(workspace);
+    if (cast_in_kernel) {
+        // one launch: the kernel's producers cast the activation tile in registers (same arithmetic as
+        // amx_quantize, so the result is bit-identical to the two-call sequence)
+        if (!gemm_tc_supported(M, N, K, group_size)) return AMX_ERR_SHAPE;
+        if (!A || !w_codes || !w_scales || !C) return AMX_ERR_NULL;
+        if (!aligned(A, 16) || ld_a % 8 || !aligned(w_codes, 16) || !aligned(w_scales, 2) || !aligned(C, 4))
+            return AMX_ERR_ALIGN;
+        return gemm_tc_cast(A, ld_a, w_codes, w_scales, M, N, K, C, ld_c, base, static_cast<cudaStream_t>(stream));
+    }
     uint8_t* a_codes = base + gemm_ws;
     uint8_t* a_scales = a_codes + a.codes;
     int rc = amx_quantize(A, M, K, ld_a, group_size, a_codes, a_scales, stream);

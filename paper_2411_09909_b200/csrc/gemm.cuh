@@ -15,6 +15,9 @@ size_t gemm_tc_workspace_bytes(int64_t M, int64_t N, int64_t K);
 int gemm_tc(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes,
             const uint8_t* w_scales, int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c,
             void* workspace, cudaStream_t st);
+// The same product with the cast of the bf16 activation X [M, ld_a] done inside the kernel.
+int gemm_tc_cast(const void* x, int64_t ld_a, const uint8_t* w_codes, const uint8_t* w_scales, int64_t M,
+                 int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st);
 int gemm_tc_status(const void* workspace, cudaStream_t st);
 
 // FP4-pipe kernel (four block-scaled MMAs per tile pair): same contract; the workspace also holds

@@ -24,6 +24,7 @@
 // all roles leave their loops, tensor memory is released and the kernel returns.
 #include <cuda_bf16.h>
 
+#include "cast_math.cuh"
 #include "gemm.cuh"
 #include "tcgen05.cuh"
 
@@ -116,8 +117,46 @@ __device__ __forceinline__ Task load_task(const uint8_t* __restrict__ codes, con
     return t;
 }
 
+// One 32-element group of a bf16 activation row, as loaded (CAST_A).
+struct RawGroup {
+    uint4 q[4];
+};
+__device__ __forceinline__ RawGroup load_raw(const uint16_t* __restrict__ x, int64_t ld, int64_t row, int64_t rows,
+                                             int64_t K, int64_t k) {
+    RawGroup g;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) g.q[j] = make_uint4(0, 0, 0, 0);
+    if (row < rows && k < K) {
+        const uint4* p = reinterpret_cast<const uint4*>(x + row * ld + k);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) g.q[j] = __ldg(p + j);
+    }
+    return g;
+}
+// The direct cast of one group (Section 4.2), same arithmetic as the cast kernel: codes and scale bytes.
+__device__ __forceinline__ Task cast_task(const RawGroup& g) {
+    uint32_t w[16];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        w[4 * j] = g.q[j].x; w[4 * j + 1] = g.q[j].y; w[4 * j + 2] = g.q[j].z; w[4 * j + 3] = g.q[j].w;
+    }
+    float inv_p, inv_n;
+    Task t;
+    t.scales = cast::group_scales(cast::side_maxima<16>(w), inv_p, inv_n);
+    t.codes.x = cast::encode8(w, inv_p, inv_n);
+    t.codes.y = cast::encode8(w + 4, inv_p, inv_n);
+    t.codes.z = cast::encode8(w + 8, inv_p, inv_n);
+    t.codes.w = cast::encode8(w + 12, inv_p, inv_n);
+    return t;
+}
+
+// CAST_A: the A operand is the bf16 activation itself (a_x, leading dimension ld_a); the producer
+// that owns a group casts it to AMXFP4 in registers and decodes the result, so the activation is read once
+// from global memory and its codes never exist there (a_codes / a_scales are unused).
+template <bool CAST_A>
 __global__ void __launch_bounds__(kThreads, 2)
 gemm_tc_kernel(const uint8_t* __restrict__ a_codes, const uint8_t* __restrict__ a_scales,
+               const uint16_t* __restrict__ a_x, int64_t ld_a,
                const uint8_t* __restrict__ w_codes, const uint8_t* __restrict__ w_scales,
                int64_t M, int64_t N, int64_t K, float* __restrict__ C, int64_t ld_c, int vec_store,
                int* __restrict__ status) {
@@ -148,14 +187,17 @@ gemm_tc_kernel(const uint8_t* __restrict__ a_codes, const uint8_t* __restrict__ 
         // task i of this thread: tile row (tid >> 1) + 128 * i, group (tid & 1) of the K block
         const int tid = threadIdx.x, half = tid & 1, r = tid >> 1;
         Task cur[kTasksPerThread], nxt[kTasksPerThread];
+        RawGroup raw;
         auto load_all = [&](Task (&t)[kTasksPerThread], int kb) {
             const int64_t k = (int64_t)kb * BK + half * 32;
-            t[0] = load_task(a_codes, a_scales, m0 + r, M, K, k);
+            if (CAST_A) raw = load_raw(a_x, ld_a, m0 + r, M, K, k);
+            else t[0] = load_task(a_codes, a_scales, m0 + r, M, K, k);
 #pragma unroll
             for (int i = 1; i < kTasksPerThread; ++i)
                 t[i] = load_task(w_codes, w_scales, n0 + r + 128 * (i - 1), N, K, k);
         };
         load_all(cur, 0);
+        if (CAST_A) cur[0] = cast_task(raw);
         bool ok = true;
         for (int kb = 0; kb < num_kb && ok; ++kb) {
             const int s = kb % kStages;
@@ -180,6 +222,7 @@ gemm_tc_kernel(const uint8_t* __restrict__ a_codes, const uint8_t* __restrict__ 
             if (lane == 0) mbar_arrive(&ctl->full[s]);
 #pragma unroll
             for (int i = 0; i < kTasksPerThread; ++i) cur[i] = nxt[i];
+            if (CAST_A && kb + 1 < num_kb) cur[0] = cast_task(raw);
         }
         // ------------------------------------------------------------------ epilogue
         if (ok) ok = mbar_wait(&ctl->accum, 0, &ctl->abort, status);
@@ -241,13 +284,17 @@ bool gemm_tc_supported(int64_t M, int64_t N, int64_t K, int gs) {
 
 size_t gemm_tc_workspace_bytes(int64_t, int64_t, int64_t) { return 256; }   // the status word
 
-int gemm_tc(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes, const uint8_t* w_scales,
-            int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {
+namespace {
+
+int launch_tc(const uint8_t* a_codes, const uint8_t* a_scales, const uint16_t* a_x, int64_t ld_a,
+              const uint8_t* w_codes, const uint8_t* w_scales, int64_t M, int64_t N, int64_t K, float* C,
+              int64_t ld_c, void* workspace, cudaStream_t st) {
     static bool configured[64] = {};   // the opt-in to > 48 KB of dynamic shared memory is per device
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AMX_ERR_CUDA;
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
             return AMX_ERR_CUDA;
         configured[dev] = true;
     }
@@ -255,8 +302,28 @@ int gemm_tc(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_co
     if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return AMX_ERR_CUDA;
     dim3 grid((unsigned)((N + BN - 1) / BN), (unsigned)((M + BM - 1) / BM));
     const int vec_store = aligned(C, 16) && ld_c % 4 == 0;   // else the epilogue stores scalars
-    gemm_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(a_codes, a_scales, w_codes, w_scales, M, N, K, C, ld_c, vec_store, status);
+    if (a_x)
+        gemm_tc_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(nullptr, nullptr, a_x, ld_a, w_codes, w_scales, M, N, K, C,
+                                                                 ld_c, vec_store, status);
+    else
+        gemm_tc_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(a_codes, a_scales, nullptr, 0, w_codes, w_scales, M, N, K,
+                                                                  C, ld_c, vec_store, status);
     return launch_status();
+}
+
+}  // namespace
+
+int gemm_tc(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes, const uint8_t* w_scales,
+            int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {
+    return launch_tc(a_codes, a_scales, nullptr, 0, w_codes, w_scales, M, N, K, C, ld_c, workspace, st);
+}
+
+// C = cast(X) What^T with the cast of X done by the kernel's producers.  X: bf16 [M, ld_a], 16-byte aligned,
+// ld_a % 8 == 0.
+int gemm_tc_cast(const void* x, int64_t ld_a, const uint8_t* w_codes, const uint8_t* w_scales, int64_t M, int64_t N,
+                 int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {
+    return launch_tc(nullptr, nullptr, static_cast<const uint16_t*>(x), ld_a, w_codes, w_scales, M, N, K, C, ld_c,
+                     workspace, st);
 }
 
 int gemm_tc_status(const void* workspace, cudaStream_t st) {

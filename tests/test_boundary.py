@@ -59,6 +59,9 @@ def test_host_detected_argument_errors(L):
     assert g(None, fake, fake, fake, 4, 4, 64, 32, 0x10, fake, 4, None, 0, None) == -1
     assert g(fake, fake, fake, fake, 0, 4, 64, 32, 0x10, fake, 4, None, 0, None) == 0   # empty
     assert L.amx_quant_gemm(fake, 64, fake, fake, 4, 4, 64, 32, 0x10, fake, 4, None, 0, None) == -4
+    assert L.amx_quant_gemm(fake, 64, fake, fake, 4, 4, 64, 32, 0x80, fake, 4, fake, 4096, None) == -5   # cast-in-kernel
+    assert L.amx_quant_gemm(fake, 64, fake, fake, 4, 4, 64, 32, 0xC0, fake, 4, fake, 4096, None) == -5   # needs the TC kernel
+    assert L.amx_gemm(fake, fake, fake, fake, 4, 4, 64, 32, 0xA0, fake, 4, None, 0, None) == -5          # not an amx_gemm flag
     assert L.amx_softmax_bf16(fake, 4, 0, 0, 1.0, fake, 0, None) == -2
 
 

@@ -263,6 +263,27 @@ def test_quant_gemm_equals_quantize_then_gemm():
     assert torch.equal(amx.quant_gemm(a, wc, ws, 32), amx.gemm(ac, as_, wc, ws, 32))
 
 
+@pytest.mark.parametrize("M,N,K,kind", [(128, 512, 1024, "mixed"), (130, 300, 96, "wide"), (1, 8, 32, "normal"),
+                                        (257, 260, 4096, "mixed")])
+def test_quant_gemm_cast_in_kernel(M, N, K, kind):
+    """The tensor-core kernel whose producers cast the activation tile themselves: bit-identical to
+    amx_quantize followed by amx_gemm on the same kernel, and within tolerance of the oracle."""
+    a_bits = inputs.random_groups(301 + M, M, K, kind)
+    w_bits = inputs.random_groups(302 + N, N, K, "normal")
+    a = dev_bf16(a_bits)
+    wc, ws = amx.quantize(dev_bf16(w_bits), 32)
+    ac, as_ = amx.quantize(a, 32)
+    fused = amx.GEMM_TC | amx.GEMM_CAST_IN_KERNEL
+    got = amx.quant_gemm(a, wc, ws, 32, flags=fused)
+    assert torch.equal(got, amx.gemm(ac, as_, wc, ws, 32, flags=amx.GEMM_TC))
+    ref = oracle.gemm(*oracle.quantize(a_bits, 32), wc.cpu().numpy(), ws.cpu().numpy(), 32)
+    assert rel_fro(got.cpu().numpy(), ref) <= GEMM_TOL
+    # a row-strided activation (a view into a wider buffer) gives the same result
+    wide = torch.zeros((M, K + 64), dtype=torch.bfloat16, device="cuda")
+    wide[:, 8:8 + K] = a
+    assert torch.equal(amx.quant_gemm(wide[:, 8:8 + K], wc, ws, 32, flags=fused), got)
+
+
 def test_config1_full_layer():
     a_bits, w_bits = inputs.activation(1, 0), inputs.weight(1, 0)
     ac, as_ = check_quantize(a_bits)
