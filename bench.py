@@ -390,6 +390,60 @@ def run_ours(args):
                        "frac_of_measured_copy": gbs / peaks["hbm_gbs"]}
         del xq, qc, qs
 
+    # ---- config 5: fully quantized attention for all heads (32 x 8192 x 128), one call of amx_attention
+    attention = None
+    if not args.layers and not args.skip_extras and world == 1:
+        H5, L5, D5 = 32, 8192, 128
+        q5, k5, v5 = (to_dev(t.reshape(H5 * L5, D5)).view(H5, L5, D5) for t in inputs.attention_qkv(H5, L5))
+        ws5 = torch.empty(L.amx_attention_workspace_bytes(L5, D5), dtype=torch.uint8, device="cuda")
+        o5 = torch.empty((H5, L5, D5), dtype=torch.float32, device="cuda")
+
+        def attn():
+            check(L.amx_attention(q5.data_ptr(), k5.data_ptr(), v5.data_ptr(), H5, L5, D5, 0, o5.data_ptr(),
+                                  ws5.data_ptr(), ws5.numel(), stream))
+
+        attn()
+        torch.cuda.synchronize()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a_iters = 3
+        a0.record()
+        for _ in range(a_iters):
+            attn()
+        a1.record()
+        torch.cuda.synchronize()
+        a_ms = a0.elapsed_time(a1) / a_iters
+        attention = {"workload": "config 5: 32 heads x 8192 x 128, non-causal; Q, K, V and the attention map all cast to AMXFP4",
+                     "ms": a_ms, "useful_tflops": 4.0 * H5 * L5 * L5 * D5 / (a_ms * 1e-3) / 1e12,
+                     "ms_per_head": a_ms / H5}
+        del q5, k5, v5, ws5, o5
+
+    # ---- config 1: one small layer (128 x 1024 -> 1024), latency-bound: microseconds per call of amx_quant_gemm
+    small_case = None
+    if not args.layers and not args.skip_extras and world == 1:
+        a1b, w1b = to_dev(inputs.activation(1, 0)), to_dev(inputs.weight(1, 0))
+        w1c, w1s = amx.quantize(w1b, GS)
+        M1, K1 = a1b.shape
+        N1 = w1c.shape[0]
+        c1 = torch.empty((M1, N1), dtype=torch.float32, device="cuda")
+        ws1 = torch.empty(max(L.amx_quant_gemm_workspace_bytes(M1, N1, K1, GS, 0), 256), dtype=torch.uint8, device="cuda")
+
+        def small():
+            check(L.amx_quant_gemm(a1b.data_ptr(), K1, w1c.data_ptr(), w1s.data_ptr(), M1, N1, K1, GS, 0, c1.data_ptr(), N1,
+                                   ws1.data_ptr(), ws1.numel(), stream))
+
+        for _ in range(5):
+            small()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        s0.record()
+        for _ in range(200):
+            small()
+        s1.record()
+        torch.cuda.synchronize()
+        small_case = {"workload": f"config 1: A {M1}x{K1} cast per call, W {N1}x{K1} cast once; amx_quant_gemm",
+                      "us_per_call": s0.elapsed_time(s1) * 1e3 / 200,
+                      "note": "launch-latency-bound (32 output tiles at most): microseconds, not a roofline fraction"}
+
     # ---- end to end through the host-buffer entry point (pinned host tensors, copies inside the timing)
     e2e = None
     if (rank == 0 or world > 1) and not args.skip_extras:
@@ -461,6 +515,8 @@ def run_ours(args):
                      "kernel": f"amx_gemm ({gemm_kernel})",
                      "peak_source": f"4 x sustained bf16 cuBLAS rate ({peaks['source']}), nominal FP4:bf16 ratio"},
         "weights_cached": weights_cached,
+        "attention": attention,
+        "small_case": small_case,
         "clocks": clocks,
         "e2e": e2e,
         # kernels per layer: 2 casts + the GEMM; without the fused entry points the FP4 kernel's operands need
