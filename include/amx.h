@@ -167,11 +167,25 @@ int amx_softmax_bf16(const float* S, int64_t rows, int64_t cols, int64_t ld_s, f
                      void* P, int64_t ld_p, void* stream);
 
 /*
+ * amx_softmax_quantize - the same step and the cast that follows it in one kernel (Appendix C: the
+ * self-attention map is quantized): per row P = softmax(alpha * S) in fp32, rounded to bf16, then cast to
+ * AMXFP4 with groups of 32 along the row, exactly as amx_softmax_bf16 followed by amx_quantize would (same
+ * bits), but the map never reaches memory as fp32 or bf16.
+ *   S  fp32 [rows, ld_s], cols % 32 == 0;  codes u8 [rows, cols/2], scales u8 [rows, cols/32, 2]
+ *   prepared  NULL, or a buffer of amx_prepared_bytes(rows, cols, 32, is_weight) bytes (256-aligned) that also
+ *             receives the operand in the form amx_gemm_prepared reads (as amx_quantize_prepared writes it)
+ */
+int amx_softmax_quantize(const float* S, int64_t rows, int64_t cols, int64_t ld_s, float alpha,
+                         uint8_t* codes, uint8_t* scales, int is_weight, void* prepared, size_t prepared_bytes,
+                         void* stream);
+
+/*
  * amx_attention - fully quantized attention, one call for all heads (Appendix C: Query, Key, the
  * self-attention map and Value are all quantized; Section 1: these are the products rotation methods
  * leave in 16 bits).  Per head h:
  *   S = AMX(Q_h) AMX(K_h)^T          groups along head_dim
- *   P = softmax(S / sqrt(d)) per row, fp32, rounded to bf16; no mask
+ *   P = softmax(S / sqrt(d)) per row, fp32, rounded to bf16; no mask (cast in the same kernel: P itself is
+ *       never stored, only its codes and scales)
  *   O_h = AMX(P) AMX(V_h)            groups along the key axis (V is quantized down its rows)
  *   q, k, v  bf16 [heads, L, d] contiguous;  o  out fp32 [heads, L, d]
  *   d % 32 == 0, L % 32 == 0 (group size 32 on both axes)

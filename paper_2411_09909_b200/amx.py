@@ -27,7 +27,7 @@ SYMBOLS = (
     "amx_gemm_kernel_for", "amx_gemm_status", "amx_status_string",
     "amx_quant_gemm_static", "amx_quant_gemm_static_capacity",
     "amx_attention", "amx_attention_workspace_bytes",
-    "amx_prepared_bytes", "amx_prepare", "amx_gemm_prepared", "amx_quantize_prepared",
+    "amx_prepared_bytes", "amx_prepare", "amx_gemm_prepared", "amx_quantize_prepared", "amx_softmax_quantize",
 )
 
 
@@ -59,6 +59,7 @@ def lib() -> ctypes.CDLL:
         L.amx_quantize_prepared.argtypes = [p, i64, i64, i, i, p, p, p, sz, p]
         L.amx_gemm_prepared.argtypes = [p, p, i64, i64, i64, i, p, i64, p, sz, p]
         L.amx_softmax_bf16.argtypes = [p, i64, i64, i64, ctypes.c_float, p, i64, p]
+        L.amx_softmax_quantize.argtypes = [p, i64, i64, i64, ctypes.c_float, p, p, i, p, sz, p]
         L.amx_linear_host.argtypes = [p, p, i64, i64, i64, i, u32, p, p, sz, p]
         for name in ("amx_workspace_bytes", "amx_quant_gemm_workspace_bytes"):
             getattr(L, name).argtypes = [i64, i64, i64, i, u32]
@@ -214,6 +215,23 @@ def softmax_bf16(S: torch.Tensor, alpha: float, out: torch.Tensor | None = None)
     _check(lib().amx_softmax_bf16(S.data_ptr(), rows, cols, S.stride(0), float(alpha), out.data_ptr(),
                                   out.stride(0), _stream()), "amx_softmax_bf16")
     return out
+
+
+def softmax_quantize(S: torch.Tensor, alpha: float, prepared_as: str | None = None):
+    """Row softmax, rounding to bf16 and the AMXFP4 cast in one kernel.  Returns (codes, scales) or, with
+    prepared_as = "a" / "w", (codes, scales, prepared) for amx_gemm_prepared."""
+    _dev(S, torch.float32, "S")
+    rows, cols = S.shape
+    codes = torch.empty((rows, cols // 2), dtype=torch.uint8, device=S.device)
+    scales = torch.empty((rows, cols // 32, 2), dtype=torch.uint8, device=S.device)
+    buf, nbytes, is_w = None, 0, int(prepared_as == "w")
+    if prepared_as is not None:
+        nbytes = lib().amx_prepared_bytes(rows, cols, 32, is_w)
+        buf = torch.full((max(nbytes, 256),), 0xFF, dtype=torch.uint8, device=S.device)
+    _check(lib().amx_softmax_quantize(S.data_ptr(), rows, cols, S.stride(0), float(alpha), codes.data_ptr(),
+                                      scales.data_ptr(), is_w, buf.data_ptr() if buf is not None else None, nbytes,
+                                      _stream()), "amx_softmax_quantize")
+    return (codes, scales) if buf is None else (codes, scales, buf)
 
 
 def linear_host(a_host: torch.Tensor, w_host: torch.Tensor, c_host: torch.Tensor, workspace: torch.Tensor,

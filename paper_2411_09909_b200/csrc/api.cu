@@ -199,9 +199,28 @@ extern "C" int amx_linear_host(const void* A_host, const void* W_host, int64_t M
     return cudaStreamSynchronize(st) == cudaSuccess ? AMX_OK : AMX_ERR_CUDA;
 }
 
+extern "C" int amx_softmax_quantize(const float* S, int64_t rows, int64_t cols, int64_t ld_s, float alpha,
+                                    uint8_t* codes, uint8_t* scales, int is_weight, void* prepared,
+                                    size_t prepared_bytes, void* stream) {
+    if (rows < 0 || cols <= 0 || cols % 32 || ld_s < cols) return AMX_ERR_SHAPE;
+    if (rows == 0) return AMX_OK;
+    if (!S || !codes || !scales) return AMX_ERR_NULL;
+    if (!aligned(S, 4) || !aligned(codes, 16) || !aligned(scales, 2)) return AMX_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!prepared) return softmax_cast_rows(S, rows, cols, ld_s, alpha, codes, scales, nullptr, nullptr, nullptr, nullptr,
+                                            nullptr, 0, rows, st);
+    if (!gemm_fp4_supported(rows, rows, cols, 32)) return AMX_ERR_SHAPE;
+    if (prepared_bytes < amx_prepared_bytes(rows, cols, 32, is_weight)) return AMX_ERR_WORKSPACE;
+    if (!aligned(prepared, kAlign)) return AMX_ERR_ALIGN;
+    return gemm_fp4_softmax_prepared(S, rows, cols, ld_s, alpha, is_weight != 0, codes, scales, prepared, st);
+}
+
 namespace {
+// Workspace of amx_attention: canonical codes and scales of Q, K, V^T and P, the logits S, then either the
+// prepared operands of the FP4 kernel (Q and P as left-hand, K and V^T as right-hand operands) or the other
+// kernels' own scratch, and the status word.
 struct AttnLayout {
-    size_t qc, qs, kc, ks, vc, vs, pc, ps, S, P, gemm, total;
+    size_t qc, qs, kc, ks, vc, vs, pc, ps, S, pq, pk, pv, pp, gemm, total;
 };
 AttnLayout attn_layout(int64_t L, int64_t d) {
     AttnLayout a;
@@ -211,14 +230,13 @@ AttnLayout attn_layout(int64_t L, int64_t d) {
     a.qc = take(qd.codes); a.qs = take(qd.scales); a.kc = take(qd.codes); a.ks = take(qd.scales);
     a.vc = take(qv.codes); a.vs = take(qv.scales); a.pc = take(ql.codes); a.ps = take(ql.scales);
     a.S = take((size_t)L * L * 4);
-    a.P = take((size_t)L * L * 2);
+    a.pq = take(gemm_fp4_prepared_bytes(L, d, false));
+    a.pk = take(gemm_fp4_prepared_bytes(L, d, true));
+    a.pv = take(gemm_fp4_prepared_bytes(d, L, true));
+    a.pp = take(gemm_fp4_prepared_bytes(L, L, false));
     a.gemm = off;
-    const size_t g1 = amx_workspace_bytes(L, L, d, 32, AMX_GEMM_AUTO), g2 = amx_workspace_bytes(L, d, L, 32, AMX_GEMM_AUTO);
-    const size_t g3 = amx_workspace_bytes(L, L, d, 32, AMX_GEMM_FP4), g4 = amx_workspace_bytes(L, d, L, 32, AMX_GEMM_FP4);
-    size_t g = g1 > g2 ? g1 : g2;
-    g = g > g3 ? g : g3;
-    g = g > g4 ? g : g4;
-    a.total = off + g;
+    const size_t g1 = amx_workspace_bytes(L, L, d, 32, AMX_GEMM_TC), g2 = amx_workspace_bytes(L, d, L, 32, AMX_GEMM_TC);
+    a.total = off + (g1 > g2 ? g1 : g2) + 256;
     return a;
 }
 }  // namespace
@@ -232,29 +250,48 @@ extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_
                              uint32_t flags, float* o, void* workspace, size_t workspace_bytes, void* stream) {
     if (flags & ~kKernelMask) return AMX_ERR_FLAGS;
     if (heads < 0 || L <= 0 || d <= 0 || L % 32 || d % 32) return AMX_ERR_SHAPE;
+    const uint32_t k_qk = pick_kernel(L, L, d, 32, flags), k_pv = pick_kernel(L, d, L, 32, flags);
+    if (!k_qk || !k_pv) return ((flags & kKernelMask) & ((flags & kKernelMask) - 1)) ? AMX_ERR_FLAGS : AMX_ERR_SHAPE;
     if (heads == 0) return AMX_OK;
     if (!q || !k || !v || !o) return AMX_ERR_NULL;
     const AttnLayout a = attn_layout(L, d);
     if (!workspace || workspace_bytes < a.total) return AMX_ERR_WORKSPACE;
-    if (!aligned(workspace, kAlign) || !aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16)) return AMX_ERR_ALIGN;
+    if (!aligned(workspace, kAlign) || !aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 4))
+        return AMX_ERR_ALIGN;
     uint8_t* w = static_cast<uint8_t*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t gemm_bytes = a.total - a.gemm;
     const float alpha = 1.0f / sqrtf((float)d);
+    float* S = reinterpret_cast<float*>(w + a.S);
     for (int64_t h = 0; h < heads; ++h) {
         const uint8_t* qh = static_cast<const uint8_t*>(q) + (size_t)h * L * d * 2;
         const uint8_t* kh = static_cast<const uint8_t*>(k) + (size_t)h * L * d * 2;
         const uint8_t* vh = static_cast<const uint8_t*>(v) + (size_t)h * L * d * 2;
-        int rc = amx_quantize(qh, L, d, d, 32, w + a.qc, w + a.qs, stream);
-        if (rc == AMX_OK) rc = amx_quantize(kh, L, d, d, 32, w + a.kc, w + a.ks, stream);
+        float* oh = o + (size_t)h * L * d;
+        int rc;
+        // S = AMX(Q) AMX(K)^T: with the FP4 kernel the casts write the prepared operands themselves
+        if (k_qk == AMX_GEMM_FP4) {
+            rc = gemm_fp4_quantize_prepared(qh, L, d, false, w + a.qc, w + a.qs, w + a.pq, st);
+            if (rc == AMX_OK) rc = gemm_fp4_quantize_prepared(kh, L, d, true, w + a.kc, w + a.ks, w + a.pk, st);
+            if (rc == AMX_OK) rc = gemm_fp4_prepared(w + a.pq, w + a.pk, L, L, d, S, L, w + a.gemm, st);
+        } else {
+            rc = amx_quantize(qh, L, d, d, 32, w + a.qc, w + a.qs, stream);
+            if (rc == AMX_OK) rc = amx_quantize(kh, L, d, d, 32, w + a.kc, w + a.ks, stream);
+            if (rc == AMX_OK)
+                rc = amx_gemm(w + a.qc, w + a.qs, w + a.kc, w + a.ks, L, L, d, 32, k_qk, S, L, w + a.gemm, gemm_bytes, stream);
+        }
+        // V along the sequence; softmax, rounding to bf16 and the cast of P in one kernel; O = AMX(P) AMX(V)
         if (rc == AMX_OK) rc = amx_quantize_t(vh, L, d, d, 32, w + a.vc, w + a.vs, stream);
-        if (rc == AMX_OK)
-            rc = amx_gemm(w + a.qc, w + a.qs, w + a.kc, w + a.ks, L, L, d, 32, flags, reinterpret_cast<float*>(w + a.S), L,
-                          w + a.gemm, gemm_bytes, stream);
-        if (rc == AMX_OK) rc = amx_softmax_bf16(reinterpret_cast<const float*>(w + a.S), L, L, L, alpha, w + a.P, L, stream);
-        if (rc == AMX_OK) rc = amx_quantize(w + a.P, L, L, L, 32, w + a.pc, w + a.ps, stream);
-        if (rc == AMX_OK)
-            rc = amx_gemm(w + a.pc, w + a.ps, w + a.vc, w + a.vs, L, d, L, 32, flags, o + (size_t)h * L * d, d, w + a.gemm,
-                          gemm_bytes, stream);
+        if (rc != AMX_OK) return rc;
+        if (k_pv == AMX_GEMM_FP4) {
+            rc = gemm_fp4_prepare(w + a.vc, w + a.vs, d, L, true, w + a.pv, st);
+            if (rc == AMX_OK) rc = gemm_fp4_softmax_prepared(S, L, L, L, alpha, false, w + a.pc, w + a.ps, w + a.pp, st);
+            if (rc == AMX_OK) rc = gemm_fp4_prepared(w + a.pp, w + a.pv, L, d, L, oh, d, w + a.gemm, st);
+        } else {
+            rc = softmax_cast_rows(S, L, L, L, alpha, w + a.pc, w + a.ps, nullptr, nullptr, nullptr, nullptr, nullptr, 0, L, st);
+            if (rc == AMX_OK)
+                rc = amx_gemm(w + a.pc, w + a.ps, w + a.vc, w + a.vs, L, d, L, 32, k_pv, oh, d, w + a.gemm, gemm_bytes, stream);
+        }
         if (rc != AMX_OK) return rc;
     }
     return AMX_OK;

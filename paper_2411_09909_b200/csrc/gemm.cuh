@@ -36,6 +36,13 @@ int gemm_fp4_quantize_prepared(const void* x, int64_t rows, int64_t K, bool is_w
 int quantize_rows_prepared(const void* x, int64_t rows, int64_t K, uint8_t* codes, uint8_t* scales, void* pos,
                            void* neg, uint8_t* sf_pos, uint8_t* sf_neg, int* row_exp, int nk64, int64_t padded_rows,
                            cudaStream_t st);
+// Softmax of the rows of S, rounded to bf16 and cast in one launch (cols % 32 == 0); pos == nullptr: canonical
+// output only.  gemm_fp4_softmax_prepared lays the prepared operand out like gemm_fp4_quantize_prepared.
+int softmax_cast_rows(const float* S, int64_t rows, int64_t cols, int64_t ld_s, float alpha, uint8_t* codes,
+                      uint8_t* scales, void* pos, void* neg, uint8_t* sf_pos, uint8_t* sf_neg, int* row_exp, int nk64,
+                      int64_t padded_rows, cudaStream_t st);
+int gemm_fp4_softmax_prepared(const float* S, int64_t rows, int64_t cols, int64_t ld_s, float alpha, bool is_weight,
+                              uint8_t* codes, uint8_t* scales, void* prepared, cudaStream_t st);
 int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
                       float* C, int64_t ld_c, void* workspace /* 256 B: status word */, cudaStream_t st);
 

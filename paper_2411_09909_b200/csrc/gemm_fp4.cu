@@ -555,6 +555,15 @@ int gemm_fp4_quantize_prepared(const void* x, int64_t rows, int64_t K, bool is_w
                                   o.row_blocks * 128, st);
 }
 
+int gemm_fp4_softmax_prepared(const float* S, int64_t rows, int64_t cols, int64_t ld_s, float alpha, bool is_weight,
+                              uint8_t* codes, uint8_t* scales, void* prepared, cudaStream_t st) {
+    const OperandLayout o = operand_layout(rows, cols, is_weight ? BN : BM);
+    uint8_t* base = static_cast<uint8_t*>(prepared);
+    return softmax_cast_rows(S, rows, cols, ld_s, alpha, codes, scales, base, base + o.plane, base + 2 * o.plane,
+                             base + 2 * o.plane + o.sf, reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf), o.nk64,
+                             o.row_blocks * 128, st);
+}
+
 int gemm_fp4_prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, bool is_weight,
                      void* prepared, cudaStream_t st) {
     return prepare(codes, scales, rows, K, operand_layout(rows, K, is_weight ? BN : BM), static_cast<uint8_t*>(prepared), st);

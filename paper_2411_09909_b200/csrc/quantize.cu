@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 
 #include "cast_math.cuh"
+#include "softmax_math.cuh"
 
 namespace amx {
 namespace {
@@ -113,6 +114,62 @@ quantize_cols_kernel(const __nv_bfloat16* __restrict__ x, int64_t R, int64_t C, 
 constexpr int kPrepMaxRows = 8;
 constexpr int kSfChunkBytes = 512;
 
+// One group of an FP4-GEMM operand from its 16 bf16x2 words: canonical codes and scale bytes at group index v,
+// and (pos != nullptr) the two sign planes.  Returns the scale bytes.
+__device__ __forceinline__ uint32_t emit_group(const uint32_t (&w)[16], int64_t v, uint4* __restrict__ codes,
+                                               uint16_t* __restrict__ scales, uint4* __restrict__ pos,
+                                               uint4* __restrict__ neg) {
+    float inv_p, inv_n;
+    const uint32_t sc = group_scales(side_maxima<16>(w), inv_p, inv_n);
+    uint32_t nib[4], pp[4], nn[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        nib[j] = encode8(w + 4 * j, inv_p, inv_n);
+        const uint32_t m = ((nib[j] >> 3) & 0x11111111u) * 15u;   // 0xF on negative nibbles
+        nn[j] = nib[j] & m;
+        pp[j] = nib[j] & ~m;
+    }
+    codes[v] = make_uint4(nib[0], nib[1], nib[2], nib[3]);
+    if (pos) {
+        pos[v] = make_uint4(pp[0], pp[1], pp[2], pp[3]);
+        neg[v] = make_uint4(nn[0], nn[1], nn[2], nn[3]);
+    }
+    scales[v] = (uint16_t)sc;
+    return sc;
+}
+
+// Second half of a prepared cast, for the GX threads (a multiple of 32) that own row `row` (`top`: largest scale
+// byte the thread has seen; kmax_s: the row's shared-memory slot, zero on entry): row maximum of the exponent
+// keys, the row's scale factors in the tensor cores' layout, padding included, and the row offset.
+__device__ __forceinline__ void finish_prepared_row(int64_t row, bool row_live, int G, int gx, int GX, uint32_t top,
+                                                    uint32_t sc_first, const uint16_t* __restrict__ scales,
+                                                    int* kmax_s, uint8_t* __restrict__ sf_pos,
+                                                    uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp, int nk64) {
+    // One shared-memory atomic per warp.  The key of an E5M2 byte grows with the byte (scales carry no sign
+    // bit), so the largest byte has the largest key.
+    top = __reduce_max_sync(0xFFFFFFFFu, top);
+    if ((gx & 31) == 0 && top > 0) atomicMax(kmax_s, scale_key(top));
+    __syncthreads();
+    const int kmax = *kmax_s;
+    // offset of this row's bytes inside a chunk; the chunks of one block of 128 rows are consecutive along K
+    const int rr = (int)(row & 127);
+    const int64_t sf_row = (row >> 7) * nk64 * (int64_t)kSfChunkBytes + (rr & 31) * 16 + (rr >> 5) * 4;
+    const int64_t v_row = row * G;
+    for (int g = gx; g < nk64 * 2; g += GX) {      // groups past G: padding to whole 256-element blocks
+        uint32_t up = 0, un = 0;
+        if (row_live && g < G) {
+            // a later group of a striding thread: re-read the scale bytes this thread stored before
+            const uint32_t sc = (g == gx) ? sc_first : scales[v_row + g];
+            up = to_ue4m3(sc & 0xFFu, kmax);
+            un = to_ue4m3(sc >> 8, kmax);
+        }
+        const int64_t off = sf_row + (g >> 1) * kSfChunkBytes + (g & 1) * 2;
+        *reinterpret_cast<uint16_t*>(sf_pos + off) = (uint16_t)(up | (up << 8));
+        *reinterpret_cast<uint16_t*>(sf_neg + off) = (uint16_t)(un | (un << 8));
+    }
+    if (gx == 0 && row_live) row_exp[row] = kmax ? kmax - 25 : 0;
+}
+
 // 40 registers (three blocks of 512 per SM): at 32 the kernel spills and is 12 % slower.
 __global__ void __launch_bounds__(512, 3)
 cast_prepared_kernel(const uint4* __restrict__ x, int64_t R, int G, uint4* __restrict__ codes,
@@ -137,45 +194,77 @@ cast_prepared_kernel(const uint4* __restrict__ x, int64_t R, int G, uint4* __res
             const uint4 q = __ldg(x + v * 4 + j);
             w[4 * j] = q.x; w[4 * j + 1] = q.y; w[4 * j + 2] = q.z; w[4 * j + 3] = q.w;
         }
-        float inv_p, inv_n;
-        const uint32_t sc = group_scales(side_maxima<16>(w), inv_p, inv_n);
-        uint32_t nib[4], pp[4], nn[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            nib[j] = encode8(w + 4 * j, inv_p, inv_n);
-            const uint32_t m = ((nib[j] >> 3) & 0x11111111u) * 15u;   // 0xF on negative nibbles
-            nn[j] = nib[j] & m;
-            pp[j] = nib[j] & ~m;
-        }
-        codes[v] = make_uint4(nib[0], nib[1], nib[2], nib[3]);
-        pos[v] = make_uint4(pp[0], pp[1], pp[2], pp[3]);
-        neg[v] = make_uint4(nn[0], nn[1], nn[2], nn[3]);
-        scales[v] = (uint16_t)sc;
+        const uint32_t sc = emit_group(w, v, codes, scales, pos, neg);
         if (g == gx) sc_first = sc;
         top = max(top, max(sc & 0xFFu, sc >> 8));
     }
-    // Row maximum of the exponent keys, one shared-memory atomic per warp.  The key of an E5M2 byte grows
-    // with the byte (scales carry no sign bit), so the largest byte has the largest key.
-    top = __reduce_max_sync(0xFFFFFFFFu, top);
-    if ((gx & 31) == 0 && top > 0) atomicMax(&kmax_s[rl], scale_key(top));
-    __syncthreads();
-    const int kmax = kmax_s[rl];
-    // offset of this row's bytes inside a chunk; the chunks of one block of 128 rows are consecutive along K
-    const int rr = (int)(row & 127);
-    const int64_t sf_row = (row >> 7) * nk64 * (int64_t)kSfChunkBytes + (rr & 31) * 16 + (rr >> 5) * 4;
-    for (int g = gx; g < nk64 * 2; g += GX) {      // groups past G: padding to whole 256-element blocks
-        uint32_t up = 0, un = 0;
-        if (row_live && g < G) {
-            // a later group of a striding thread: re-read the scale bytes this thread stored above
-            const uint32_t sc = (g == gx) ? sc_first : scales[v_row + g];
-            up = to_ue4m3(sc & 0xFFu, kmax);
-            un = to_ue4m3(sc >> 8, kmax);
+    finish_prepared_row(row, row_live, G, gx, GX, top, sc_first, scales, &kmax_s[rl], sf_pos, sf_neg, row_exp, nk64);
+}
+
+// Attention glue in one pass (Appendix C): row softmax of the fp32 logits (times alpha), rounding of the
+// normalised map to bf16 - the cast's input type - and the cast of that row to AMXFP4, without the map ever
+// reaching global memory as fp32 or bf16.  One block of softmax::kT threads per row (grid = padded rows when the
+// prepared form is written, blocks past the last row only zero scale-factor padding).  Same bits as the
+// stand-alone softmax kernel followed by the cast: both use softmax_math.cuh and cast_math.cuh.
+// CACHED: the row has at most kT groups, so each thread keeps its one group in registers between the passes.
+template <bool CACHED>
+__global__ void __launch_bounds__(softmax::kT)
+softmax_cast_kernel(const float* __restrict__ S, int64_t R, int G, int64_t ld_s, float alpha, int vec,
+                    uint4* __restrict__ codes, uint16_t* __restrict__ scales, uint4* __restrict__ pos,
+                    uint4* __restrict__ neg, uint8_t* __restrict__ sf_pos, uint8_t* __restrict__ sf_neg,
+                    int* __restrict__ row_exp, int nk64) {
+    __shared__ float sh[softmax::kT / 32];
+    __shared__ int kmax_s;
+    const int gx = threadIdx.x;
+    const int64_t row = blockIdx.x;
+    const bool row_live = row < R;                  // uniform over the block
+    if (gx == 0) kmax_s = 0;
+    uint32_t sc_first = 0, top = 0;
+    if (row_live) {
+        const float* s = S + row * ld_s;
+        const int64_t cols = (int64_t)G * 32, v_row = row * G;
+        if (CACHED) {
+            float t[32];
+            const bool own = gx < G;
+            if (own) {
+                softmax::load_group(s, gx, cols, vec != 0, alpha, t);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) t[i] = -INFINITY;
+            }
+            float mx = -INFINITY, sum = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, t[i]);
+            mx = softmax::block_reduce(mx, true, sh);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                t[i] = expf(t[i] - mx);
+                sum += t[i];
+            }
+            sum = softmax::block_reduce(sum, false, sh);
+            if (own) {
+                uint32_t w[16];
+                softmax::normalised_group_e(t, sum, w);
+                sc_first = emit_group(w, v_row + gx, codes, scales, pos, neg);
+                top = max(sc_first & 0xFFu, sc_first >> 8);
+            }
+        } else {
+            float mx, sum;
+            softmax::row_stats(s, cols, vec != 0, alpha, sh, mx, sum);
+            for (int g = gx; g < G; g += softmax::kT) {
+                float t[32];
+                uint32_t w[16];
+                softmax::load_group(s, g, cols, vec != 0, alpha, t);
+                softmax::normalised_group(t, mx, sum, w);
+                const uint32_t sc = emit_group(w, v_row + g, codes, scales, pos, neg);
+                if (g == gx) sc_first = sc;
+                top = max(top, max(sc & 0xFFu, sc >> 8));
+            }
         }
-        const int64_t off = sf_row + (g >> 1) * kSfChunkBytes + (g & 1) * 2;
-        *reinterpret_cast<uint16_t*>(sf_pos + off) = (uint16_t)(up | (up << 8));
-        *reinterpret_cast<uint16_t*>(sf_neg + off) = (uint16_t)(un | (un << 8));
     }
-    if (gx == 0 && row_live) row_exp[row] = kmax ? kmax - 25 : 0;
+    if (!pos) return;                               // canonical output only
+    __syncthreads();                                // kmax_s is zero before the first atomic
+    finish_prepared_row(row, row_live, G, gx, softmax::kT, top, sc_first, scales, &kmax_s, sf_pos, sf_neg, row_exp, nk64);
 }
 
 template <int EPT, int TPG>
@@ -213,6 +302,21 @@ int quantize_rows_prepared(const void* x, int64_t rows, int64_t K, uint8_t* code
         reinterpret_cast<const uint4*>(x), rows, (int)G, reinterpret_cast<uint4*>(codes),
         reinterpret_cast<uint16_t*>(scales), reinterpret_cast<uint4*>(pos), reinterpret_cast<uint4*>(neg), sf_pos, sf_neg,
         row_exp, nk64);
+    return launch_status();
+}
+
+// Softmax of the rows of S (fp32 [rows, ld_s], cols % 32 == 0), rounded to bf16 and cast, in one launch.  With
+// pos == nullptr only the canonical codes and scales are written.
+int softmax_cast_rows(const float* S, int64_t rows, int64_t cols, int64_t ld_s, float alpha, uint8_t* codes,
+                      uint8_t* scales, void* pos, void* neg, uint8_t* sf_pos, uint8_t* sf_neg, int* row_exp, int nk64,
+                      int64_t padded_rows, cudaStream_t st) {
+    const int64_t G = cols / 32, blocks = pos ? padded_rows : rows;
+    if (blocks > 0x7FFFFFFF || G > 0x7FFFFFFF / 32) return AMX_ERR_SHAPE;
+    const int vec = aligned(S, 16) && ld_s % 4 == 0;
+    auto* kernel = G <= softmax::kT ? softmax_cast_kernel<true> : softmax_cast_kernel<false>;
+    kernel<<<(unsigned)blocks, softmax::kT, 0, st>>>(S, rows, (int)G, ld_s, alpha, vec, reinterpret_cast<uint4*>(codes),
+                                                     reinterpret_cast<uint16_t*>(scales), reinterpret_cast<uint4*>(pos),
+                                                     reinterpret_cast<uint4*>(neg), sf_pos, sf_neg, row_exp, nk64);
     return launch_status();
 }
 

@@ -1,44 +1,40 @@
 // Row softmax in fp32 with bf16 output: the step between the two attention products.  The
 // normalised self-attention map is what gets quantized (arXiv 2411.09909, Appendix C), and the
-// quantizer reads bf16, so P is rounded to bf16 (nearest even) here.
-#include <cuda_bf16.h>
-
-#include "amx_common.cuh"
+// quantizer reads bf16, so P is rounded to bf16 (nearest even) here.  The arithmetic is in
+// softmax_math.cuh; the kernel that also casts the map is in quantize.cu.
+#include "softmax_math.cuh"
 
 namespace amx {
 namespace {
 
-constexpr int kT = 256;
-
-__device__ __forceinline__ float block_reduce(float v, bool is_max, float* sh) {
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) {
-        const float o = __shfl_xor_sync(0xFFFFFFFFu, v, d);
-        v = is_max ? fmaxf(v, o) : v + o;
-    }
-    __syncthreads();  // sh may still be read from a previous reduction
-    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
-    __syncthreads();
-    v = sh[0];
-#pragma unroll
-    for (int i = 1; i < kT / 32; ++i) v = is_max ? fmaxf(v, sh[i]) : v + sh[i];
-    return v;
-}
+using namespace softmax;
 
 __global__ void __launch_bounds__(kT)
 softmax_bf16_kernel(const float* __restrict__ S, int64_t cols, int64_t ld_s, float alpha,
-                    __nv_bfloat16* __restrict__ P, int64_t ld_p) {
+                    uint16_t* __restrict__ P, int64_t ld_p, int vec_in, int vec_out) {
     __shared__ float sh[kT / 32];
     const float* s = S + (int64_t)blockIdx.x * ld_s;
-    __nv_bfloat16* p = P + (int64_t)blockIdx.x * ld_p;
-    float mx = -INFINITY;
-    for (int64_t c = threadIdx.x; c < cols; c += kT) mx = fmaxf(mx, alpha * s[c]);
-    mx = block_reduce(mx, true, sh);
-    float sum = 0.f;
-    for (int64_t c = threadIdx.x; c < cols; c += kT) sum += expf(alpha * s[c] - mx);
-    sum = block_reduce(sum, false, sh);
-    for (int64_t c = threadIdx.x; c < cols; c += kT)
-        p[c] = __float2bfloat16_rn(expf(alpha * s[c] - mx) / sum);
+    uint16_t* p = P + (int64_t)blockIdx.x * ld_p;
+    float mx, sum;
+    row_stats(s, cols, vec_in != 0, alpha, sh, mx, sum);
+    const int64_t G = (cols + 31) / 32;
+    for (int64_t g = threadIdx.x; g < G; g += kT) {
+        float t[32];
+        uint32_t w[16];
+        load_group(s, g, cols, vec_in != 0, alpha, t);
+        normalised_group(t, mx, sum, w);
+        if (vec_out) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                reinterpret_cast<uint4*>(p + g * 32)[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const int64_t c = g * 32 + i;
+                if (c < cols) p[c] = (uint16_t)(w[i >> 1] >> ((i & 1) * 16));
+            }
+        }
+    }
 }
 
 }  // namespace
@@ -51,7 +47,10 @@ extern "C" int amx_softmax_bf16(const float* S, int64_t rows, int64_t cols, int6
     if (rows == 0) return AMX_OK;
     if (!S || !P) return AMX_ERR_NULL;
     if (!aligned(S, 4) || !aligned(P, 2)) return AMX_ERR_ALIGN;
-    softmax_bf16_kernel<<<(unsigned)rows, kT, 0, static_cast<cudaStream_t>(stream)>>>(
-        S, cols, ld_s, alpha, reinterpret_cast<__nv_bfloat16*>(P), ld_p);
+    const int whole = cols % 32 == 0;
+    const int vec_in = whole && aligned(S, 16) && ld_s % 4 == 0;
+    const int vec_out = whole && aligned(P, 16) && ld_p % 8 == 0;
+    softmax_bf16_kernel<<<(unsigned)rows, softmax::kT, 0, static_cast<cudaStream_t>(stream)>>>(
+        S, cols, ld_s, alpha, reinterpret_cast<uint16_t*>(P), ld_p, vec_in, vec_out);
     return launch_status();
 }

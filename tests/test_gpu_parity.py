@@ -316,6 +316,41 @@ def test_softmax_bf16_against_oracle():
     assert diff.max() <= 1 and np.mean(diff != 0) < 0.02
 
 
+@pytest.mark.parametrize("rows,cols,scale", [(40, 1024, 30.0), (130, 96, 3.0), (9, 8192, 50.0), (5, 8224, 8.0),
+                                             (3, 32, 1.0)])
+def test_softmax_quantize_fused_equals_two_kernels(rows, cols, scale):
+    """amx_softmax_quantize: same bits as amx_softmax_bf16 followed by amx_quantize; the oracle quantizer on the
+    device's own bf16 map gives the same codes and scales; the prepared form drives the GEMM to the same result.
+    Rows of at most 8192 columns take the register-cached path, longer ones the re-reading one."""
+    rng = np.random.default_rng(80 + rows)
+    S_np = (rng.standard_normal((rows, cols)) * scale).astype(np.float32)
+    S_np[0, : cols // 2] = -1e4                              # half a row underflows to exactly zero
+    S = torch.from_numpy(S_np).cuda()
+    alpha = 128 ** -0.5
+    P = amx.softmax_bf16(S, alpha)
+    c2, s2 = amx.quantize(P, 32)
+    c, s_ = amx.softmax_quantize(S, alpha)
+    assert torch.equal(c, c2) and torch.equal(s_, s2)
+    oc, os_ = oracle.quantize(P.view(torch.int16).cpu().numpy().view(np.uint16), 32)
+    assert np.array_equal(c.cpu().numpy(), oc) and np.array_equal(s_.cpu().numpy(), os_)
+    # strided logits (a view into a wider buffer)
+    wide = torch.zeros((rows, cols + 40), dtype=torch.float32, device="cuda")
+    wide[:, 4:4 + cols] = S
+    cw, sw = amx.softmax_quantize(wide[:, 4:4 + cols], alpha)
+    assert torch.equal(cw, c) and torch.equal(sw, s_)
+    wide[:, 1:1 + cols] = S                                   # rows not 16-byte aligned: scalar loads
+    cw, sw = amx.softmax_quantize(wide[:, 1:1 + cols], alpha)
+    assert torch.equal(cw, c) and torch.equal(sw, s_)
+    # prepared form, as the left-hand operand of P V
+    cp, sp, prep = amx.softmax_quantize(S, alpha, prepared_as="a")
+    assert torch.equal(cp, c) and torch.equal(sp, s_)
+    v_bits = inputs.random_groups(81, 64, cols, "normal")
+    vc, vs = amx.quantize(dev_bf16(v_bits), 32)
+    pv = amx.prepare(vc, vs, True)
+    assert torch.equal(amx.gemm_prepared(prep, pv, rows, 64, cols),
+                       amx.gemm_prepared(amx.prepare(c2, s2, False), pv, rows, 64, cols))
+
+
 def test_attention_small_head_against_oracle_pipeline():
     """Config-5 pipeline at reduced size: Q/K/V codes bit-exact; the device quantizer applied to the
     device's own bf16 P equals the oracle quantizer on the same bits; O within tolerance of the all-CPU
