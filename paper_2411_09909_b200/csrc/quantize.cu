@@ -224,27 +224,11 @@ softmax_cast_kernel(const float* __restrict__ S, int64_t R, int G, int64_t ld_s,
         const float* s = S + row * ld_s;
         const int64_t cols = (int64_t)G * 32, v_row = row * G;
         if (CACHED) {
-            float t[32];
-            const bool own = gx < G;
-            if (own) {
-                softmax::load_group(s, gx, cols, vec != 0, alpha, t);
-            } else {
-#pragma unroll
-                for (int i = 0; i < 32; ++i) t[i] = -INFINITY;
-            }
-            float mx = -INFINITY, sum = 0.f;
-#pragma unroll
-            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, t[i]);
-            mx = softmax::block_reduce(mx, true, sh);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                t[i] = expf(t[i] - mx);
-                sum += t[i];
-            }
-            sum = softmax::block_reduce(sum, false, sh);
-            if (own) {
+            float e[32];
+            const float sum = softmax::cached_row_exp(s, G, vec != 0, alpha, sh, e);
+            if (gx < G) {
                 uint32_t w[16];
-                softmax::normalised_group_e(t, sum, w);
+                softmax::normalised_group_e(e, sum, w);
                 sc_first = emit_group(w, v_row + gx, codes, scales, pos, neg);
                 top = max(sc_first & 0xFFu, sc_first >> 8);
             }

@@ -28,6 +28,19 @@ __device__ __forceinline__ float block_reduce(float v, bool is_max, float* sh) {
     return v;
 }
 
+// exp(t - mx) as 2^(t * log2(e) - mx * log2(e)): one fused multiply-add (the product is not rounded) and the
+// hardware's base-2 exponential (relative error 2^-22; results below the smallest normal float flush to zero).
+// neg_mx_l2e = -(mx * log2(e)), rounded once per row: the rounding error is a common factor of the whole row and
+// cancels in the normalisation.  What remains is the rounding of the exponent itself, |t - mx| * 2^-24 relative,
+// which any fp32 evaluation of exp(t - mx) has as well.
+__device__ __forceinline__ float neg_max_log2e(float mx) { return -(mx * 1.4426950408889634f); }
+__device__ __forceinline__ float exp_rel(float t, float neg_mx_l2e) {
+    const float y = fmaf(t, 1.4426950408889634f, neg_mx_l2e);
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(y));
+    return r;
+}
+
 // alpha * s for the 32 columns of group g of a row; -inf past the last column (contributes exp() = 0).
 // vec: the row is 16-byte aligned and holds whole groups, so the group is read with eight 16-byte loads.
 __device__ __forceinline__ void load_group(const float* __restrict__ s, int64_t g, int64_t cols, bool vec, float alpha,
@@ -48,6 +61,29 @@ __device__ __forceinline__ void load_group(const float* __restrict__ s, int64_t 
     }
 }
 
+// Softmax of a row of at most kT groups with the thread's group kept in registers: on return e holds
+// exp(alpha * s - max) of the thread's own group (zeros for a thread without one); returns the row sum.
+__device__ __forceinline__ float cached_row_exp(const float* __restrict__ s, int G, bool vec, float alpha, float* sh,
+                                                float (&e)[32]) {
+    if ((int)threadIdx.x < G) {
+        load_group(s, threadIdx.x, (int64_t)G * 32, vec, alpha, e);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) e[i] = -INFINITY;
+    }
+    float mx = -INFINITY, sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, e[i]);
+    mx = block_reduce(mx, true, sh);
+    const float nm = neg_max_log2e(mx);
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        e[i] = exp_rel(e[i], nm);
+        sum += e[i];
+    }
+    return block_reduce(sum, false, sh);
+}
+
 // Row maximum and the sum of exp(alpha * s - max) for the row this block owns.
 __device__ __forceinline__ void row_stats(const float* __restrict__ s, int64_t cols, bool vec, float alpha, float* sh,
                                           float& mx, float& sum) {
@@ -61,28 +97,32 @@ __device__ __forceinline__ void row_stats(const float* __restrict__ s, int64_t c
     }
     mx = block_reduce(mx, true, sh);
     sum = 0.f;
+    const float nm = neg_max_log2e(mx);
     for (int64_t g = threadIdx.x; g < G; g += kT) {
         load_group(s, g, cols, vec, alpha, t);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) sum += expf(t[i] - mx);
+        for (int i = 0; i < 32; ++i) sum += exp_rel(t[i], nm);
     }
     sum = block_reduce(sum, false, sh);
 }
 
 // e / sum for the 32 values e = exp(alpha * s - max) of one group, rounded to bf16 (nearest even), as 16 bf16x2
 // words.
+// The division is one reciprocal per row and a multiply per element (within 1.5 fp32 ulp of the quotient, far
+// inside the bf16 rounding that follows).
 __device__ __forceinline__ void normalised_group_e(const float (&e)[32], float sum, uint32_t (&w)[16]) {
+    const float inv = 1.0f / sum;
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
-        const __nv_bfloat16 lo = __float2bfloat16_rn(e[2 * i] / sum);
-        const __nv_bfloat16 hi = __float2bfloat16_rn(e[2 * i + 1] / sum);
-        w[i] = (uint32_t)__bfloat16_as_ushort(lo) | ((uint32_t)__bfloat16_as_ushort(hi) << 16);
+        const __nv_bfloat162 pr = __floats2bfloat162_rn(e[2 * i] * inv, e[2 * i + 1] * inv);   // .x = low half
+        w[i] = *reinterpret_cast<const uint32_t*>(&pr);
     }
 }
 // The same from t = alpha * s.
 __device__ __forceinline__ void normalised_group(float (&t)[32], float mx, float sum, uint32_t (&w)[16]) {
+    const float nm = neg_max_log2e(mx);
 #pragma unroll
-    for (int i = 0; i < 32; ++i) t[i] = expf(t[i] - mx);
+    for (int i = 0; i < 32; ++i) t[i] = exp_rel(t[i], nm);
     normalised_group_e(t, sum, w);
 }
 
