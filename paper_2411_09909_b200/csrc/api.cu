@@ -216,23 +216,30 @@ extern "C" int amx_softmax_quantize(const float* S, int64_t rows, int64_t cols, 
 }
 
 namespace {
-// Workspace of amx_attention: canonical codes and scales of Q, K, V^T and P, the logits S, then either the
-// prepared operands of the FP4 kernel (Q and P as left-hand, K and V^T as right-hand operands) or the other
-// kernels' own scratch, and the status word.
+// Workspace of amx_attention.  Heads are taken in chunks: the casts of Q, K and V (small per head) run once per
+// chunk on the stacked heads, the two products and the softmax once per head.  Holds the canonical codes and
+// scales of the chunk's Q, K and V^T and of one head's P, the logits S of one head, then either the prepared
+// operands of the FP4 kernel (Q and P as left-hand, K and V^T as right-hand operands) or the other kernels' own
+// scratch, and the status word.
+constexpr int64_t kAttnChunk = 8;
+int64_t attn_chunk(int64_t L, int64_t d) { return (L % 128 == 0 && d % 128 == 0) ? kAttnChunk : 1; }
+
 struct AttnLayout {
     size_t qc, qs, kc, ks, vc, vs, pc, ps, S, pq, pk, pv, pp, gemm, total;
 };
 AttnLayout attn_layout(int64_t L, int64_t d) {
     AttnLayout a;
-    const QuantSizes qd = quant_sizes(L, d, 32), ql = quant_sizes(L, L, 32), qv = quant_sizes(d, L, 32);
+    const int64_t hc = attn_chunk(L, d);
+    const QuantSizes qd = quant_sizes(hc * L, d, 32), ql = quant_sizes(L, L, 32), qv = quant_sizes(hc * d, L, 32);
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off += round_up(bytes); return o; };
     a.qc = take(qd.codes); a.qs = take(qd.scales); a.kc = take(qd.codes); a.ks = take(qd.scales);
     a.vc = take(qv.codes); a.vs = take(qv.scales); a.pc = take(ql.codes); a.ps = take(ql.scales);
     a.S = take((size_t)L * L * 4);
-    a.pq = take(gemm_fp4_prepared_bytes(L, d, false));
-    a.pk = take(gemm_fp4_prepared_bytes(L, d, true));
-    a.pv = take(gemm_fp4_prepared_bytes(d, L, true));
+    // right-hand operands are laid out for 128 rows more: the last head's 256-row tiles may reach past the stack
+    a.pq = take(gemm_fp4_prepared_bytes(hc * L, d, false));
+    a.pk = take(gemm_fp4_prepared_bytes(hc * L + 128, d, true));
+    a.pv = take(gemm_fp4_prepared_bytes(hc * d + 128, L, true));
     a.pp = take(gemm_fp4_prepared_bytes(L, L, false));
     a.gemm = off;
     const size_t g1 = amx_workspace_bytes(L, L, d, 32, AMX_GEMM_TC), g2 = amx_workspace_bytes(L, d, L, 32, AMX_GEMM_TC);
@@ -263,36 +270,54 @@ extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_
     const size_t gemm_bytes = a.total - a.gemm;
     const float alpha = 1.0f / sqrtf((float)d);
     float* S = reinterpret_cast<float*>(w + a.S);
-    for (int64_t h = 0; h < heads; ++h) {
-        const uint8_t* qh = static_cast<const uint8_t*>(q) + (size_t)h * L * d * 2;
-        const uint8_t* kh = static_cast<const uint8_t*>(k) + (size_t)h * L * d * 2;
-        const uint8_t* vh = static_cast<const uint8_t*>(v) + (size_t)h * L * d * 2;
-        float* oh = o + (size_t)h * L * d;
+    const int64_t chunk = attn_chunk(L, d);
+    const size_t head_in = (size_t)L * d * 2;                       // bytes of one head of q, k or v
+    const size_t qk_codes = (size_t)L * d / 2, qk_scales = (size_t)L * (d / 32) * 2;   // one head of Q or K, canonical
+    const size_t v_codes = (size_t)d * L / 2, v_scales = (size_t)d * (L / 32) * 2;     // one head of V^T
+    for (int64_t h0 = 0; h0 < heads; h0 += chunk) {
+        const int64_t hc = heads - h0 < chunk ? heads - h0 : chunk;
+        const uint8_t* qh = static_cast<const uint8_t*>(q) + h0 * head_in;
+        const uint8_t* kh = static_cast<const uint8_t*>(k) + h0 * head_in;
+        const uint8_t* vh = static_cast<const uint8_t*>(v) + h0 * head_in;
+        // casts of the chunk's heads, stacked row-wise: Q and K along head_dim, V along the sequence (V^T)
         int rc;
-        // S = AMX(Q) AMX(K)^T: with the FP4 kernel the casts write the prepared operands themselves
         if (k_qk == AMX_GEMM_FP4) {
-            rc = gemm_fp4_quantize_prepared(qh, L, d, false, w + a.qc, w + a.qs, w + a.pq, st);
-            if (rc == AMX_OK) rc = gemm_fp4_quantize_prepared(kh, L, d, true, w + a.kc, w + a.ks, w + a.pk, st);
-            if (rc == AMX_OK) rc = gemm_fp4_prepared(w + a.pq, w + a.pk, L, L, d, S, L, w + a.gemm, st);
-        } else {
-            rc = amx_quantize(qh, L, d, d, 32, w + a.qc, w + a.qs, stream);
-            if (rc == AMX_OK) rc = amx_quantize(kh, L, d, d, 32, w + a.kc, w + a.ks, stream);
+            rc = gemm_fp4_quantize_prepared(qh, hc * L, d, false, w + a.qc, w + a.qs, w + a.pq, st, chunk * L);
             if (rc == AMX_OK)
-                rc = amx_gemm(w + a.qc, w + a.qs, w + a.kc, w + a.ks, L, L, d, 32, k_qk, S, L, w + a.gemm, gemm_bytes, stream);
-        }
-        // V along the sequence; softmax, rounding to bf16 and the cast of P in one kernel; O = AMX(P) AMX(V)
-        if (rc == AMX_OK) rc = amx_quantize_t(vh, L, d, d, 32, w + a.vc, w + a.vs, stream);
-        if (rc != AMX_OK) return rc;
-        if (k_pv == AMX_GEMM_FP4) {
-            rc = gemm_fp4_prepare(w + a.vc, w + a.vs, d, L, true, w + a.pv, st);
-            if (rc == AMX_OK) rc = gemm_fp4_softmax_prepared(S, L, L, L, alpha, false, w + a.pc, w + a.ps, w + a.pp, st);
-            if (rc == AMX_OK) rc = gemm_fp4_prepared(w + a.pp, w + a.pv, L, d, L, oh, d, w + a.gemm, st);
+                rc = gemm_fp4_quantize_prepared(kh, hc * L, d, true, w + a.kc, w + a.ks, w + a.pk, st, chunk * L + 128);
         } else {
-            rc = softmax_cast_rows(S, L, L, L, alpha, w + a.pc, w + a.ps, nullptr, nullptr, nullptr, nullptr, nullptr, 0, L, st);
-            if (rc == AMX_OK)
-                rc = amx_gemm(w + a.pc, w + a.ps, w + a.vc, w + a.vs, L, d, L, 32, k_pv, oh, d, w + a.gemm, gemm_bytes, stream);
+            rc = amx_quantize(qh, hc * L, d, d, 32, w + a.qc, w + a.qs, stream);
+            if (rc == AMX_OK) rc = amx_quantize(kh, hc * L, d, d, 32, w + a.kc, w + a.ks, stream);
         }
+        if (rc == AMX_OK) rc = quantize_cols_batched(vh, hc, L, d, w + a.vc, w + a.vs, st);
+        if (rc == AMX_OK && k_pv == AMX_GEMM_FP4)
+            rc = gemm_fp4_prepare(w + a.vc, w + a.vs, hc * d, L, true, w + a.pv, st, chunk * d + 128);
         if (rc != AMX_OK) return rc;
+        for (int64_t i = 0; i < hc; ++i) {
+            float* oh = o + (size_t)(h0 + i) * L * d;
+            // S = AMX(Q) AMX(K)^T
+            if (k_qk == AMX_GEMM_FP4)
+                rc = gemm_fp4_prepared_at({w + a.pq, hc * L, chunk * L, i * L}, {w + a.pk, hc * L, chunk * L + 128, i * L}, L,
+                                          L, d, S, L, w + a.gemm, st);
+            else
+                rc = amx_gemm(w + a.qc + i * qk_codes, w + a.qs + i * qk_scales, w + a.kc + i * qk_codes,
+                              w + a.ks + i * qk_scales, L, L, d, 32, k_qk, S, L, w + a.gemm, gemm_bytes, stream);
+            if (rc != AMX_OK) return rc;
+            // softmax, rounding to bf16 and the cast of P in one kernel; O = AMX(P) AMX(V)
+            if (k_pv == AMX_GEMM_FP4) {
+                rc = gemm_fp4_softmax_prepared(S, L, L, L, alpha, false, w + a.pc, w + a.ps, w + a.pp, st);
+                if (rc == AMX_OK)
+                    rc = gemm_fp4_prepared_at({w + a.pp, L, L, 0}, {w + a.pv, hc * d, chunk * d + 128, i * d}, L, d, L, oh, d,
+                                              w + a.gemm, st);
+            } else {
+                rc = softmax_cast_rows(S, L, L, L, alpha, w + a.pc, w + a.ps, nullptr, nullptr, nullptr, nullptr, nullptr, 0, L,
+                                       st);
+                if (rc == AMX_OK)
+                    rc = amx_gemm(w + a.pc, w + a.ps, w + a.vc + i * v_codes, w + a.vs + i * v_scales, L, d, L, 32, k_pv, oh,
+                                  d, w + a.gemm, gemm_bytes, stream);
+            }
+            if (rc != AMX_OK) return rc;
+        }
     }
     return AMX_OK;
 }

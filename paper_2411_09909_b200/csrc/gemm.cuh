@@ -30,9 +30,9 @@ int gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_c
 // The same in two phases, so that an operand (typically the weight) is prepared once and reused.
 size_t gemm_fp4_prepared_bytes(int64_t rows, int64_t K, bool is_weight);
 int gemm_fp4_prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, bool is_weight,
-                     void* prepared, cudaStream_t st);
+                     void* prepared, cudaStream_t st, int64_t layout_rows = 0 /* 0: rows */);
 int gemm_fp4_quantize_prepared(const void* x, int64_t rows, int64_t K, bool is_weight, uint8_t* codes,
-                               uint8_t* scales, void* prepared, cudaStream_t st);
+                               uint8_t* scales, void* prepared, cudaStream_t st, int64_t layout_rows = 0);
 int quantize_rows_prepared(const void* x, int64_t rows, int64_t K, uint8_t* codes, uint8_t* scales, void* pos,
                            void* neg, uint8_t* sf_pos, uint8_t* sf_neg, int* row_exp, int nk64, int64_t padded_rows,
                            cudaStream_t st);
@@ -43,6 +43,17 @@ int softmax_cast_rows(const float* S, int64_t rows, int64_t cols, int64_t ld_s, 
                       int64_t padded_rows, cudaStream_t st);
 int gemm_fp4_softmax_prepared(const float* S, int64_t rows, int64_t cols, int64_t ld_s, float alpha, bool is_weight,
                               uint8_t* codes, uint8_t* scales, void* prepared, cudaStream_t st);
+// A prepared operand that stacks several matrices row-wise (rows_total rows, laid out for layout_rows >=
+// rows_total rows) and the first row of the one to multiply; row0 % 128 == 0.  A right-hand operand whose 256-row
+// tiles can reach past rows_total needs layout_rows >= rows_total + 128.
+struct Fp4Operand {
+    const void* prepared;
+    int64_t rows_total, layout_rows, row0;
+};
+int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
+                         int64_t ld_c, void* workspace, cudaStream_t st);
+int quantize_cols_batched(const void* x, int64_t batch, int64_t R, int64_t C, uint8_t* codes, uint8_t* scales,
+                          cudaStream_t st);
 int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
                       float* C, int64_t ld_c, void* workspace /* 256 B: status word */, cudaStream_t st);
 

@@ -175,6 +175,7 @@ struct Params {
     const uint8_t *sfa_pos, *sfa_neg, *sfb_pos, *sfb_neg;
     const int *a_exp, *w_exp;
     int64_t M, N, K, ld_c;
+    int64_t a_row0, w_row0;      // first rows of this product's operands inside the (stacked) prepared operands
     float* C;
     int nk64, vec_store;
     int* status;
@@ -240,8 +241,8 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                     uint8_t* st = tiles + s * kStageBytes;
                     mbar_expect_tx(&ctl->full[s], kStageBytes);
                     // one 3-D tile per operand: {row bytes, rows, both sign planes}
-                    tma_load_3d(st + C_::kOffAp, &tm_a, kb * kRowBytes, (int)(m_blk * BM), 0, &ctl->full[s]);
-                    tma_load_3d(st + C_::kOffWp, &tm_w, kb * kRowBytes, (int)(n_blk * BN), 0, &ctl->full[s]);
+                    tma_load_3d(st + C_::kOffAp, &tm_a, kb * kRowBytes, (int)(p.a_row0 + m_blk * BM), 0, &ctl->full[s]);
+                    tma_load_3d(st + C_::kOffWp, &tm_w, kb * kRowBytes, (int)(p.w_row0 + n_blk * BN), 0, &ctl->full[s]);
                 }
             }
             // after an abort: let the copies already in flight land before shared memory is released
@@ -484,8 +485,8 @@ size_t gemm_fp4_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 namespace {
 
 template <int BK_>
-int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, const OperandLayout& ow, Params p,
-               int dev, cudaStream_t st) {
+int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, const OperandLayout& ow, int64_t a_rows,
+               int64_t w_rows, Params p, int dev, cudaStream_t st) {
     using C_ = Cfg<BK_>;
     static bool configured[64] = {};
     if (!configured[dev]) {
@@ -494,7 +495,7 @@ int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, co
         configured[dev] = true;
     }
     CUtensorMap tm_a, tm_w;
-    if (!make_map(&tm_a, pa, p.M, p.K, oa.plane, BM, C_::kRowBytes) || !make_map(&tm_w, pw, p.N, p.K, ow.plane, BN, C_::kRowBytes))
+    if (!make_map(&tm_a, pa, a_rows, p.K, oa.plane, BM, C_::kRowBytes) || !make_map(&tm_w, pw, w_rows, p.K, ow.plane, BN, C_::kRowBytes))
         return AMX_ERR_CUDA;
     static int sm_count[64] = {};
     if (!sm_count[dev] && cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
@@ -516,28 +517,38 @@ int fp4_block_k() {
 
 }  // namespace
 
-// The GEMM proper on two prepared operands (each laid out by operand_layout()).
-int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K, float* C,
-                      int64_t ld_c, void* workspace, cudaStream_t st) {
+// The GEMM proper on two prepared operands (each laid out by operand_layout()), or on row ranges of them.
+int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
+                         int64_t ld_c, void* workspace, cudaStream_t st) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AMX_ERR_CUDA;
-    const OperandLayout oa = operand_layout(M, K, BM), ow = operand_layout(N, K, BN);
-    const uint8_t* pa = static_cast<const uint8_t*>(a_prepared);
-    const uint8_t* pw = static_cast<const uint8_t*>(w_prepared);
+    if (a.row0 % 128 || w.row0 % 128) return AMX_ERR_SHAPE;
+    const OperandLayout oa = operand_layout(a.layout_rows, K, BM), ow = operand_layout(w.layout_rows, K, BN);
+    const uint8_t* pa = static_cast<const uint8_t*>(a.prepared);
+    const uint8_t* pw = static_cast<const uint8_t*>(w.prepared);
     int* status = static_cast<int*>(workspace);
     if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return AMX_ERR_CUDA;
     Params p;
-    p.sfa_pos = pa + 2 * oa.plane;
+    // scale factors come in chunks per 128 rows, row offsets per row: the range starts at a pointer offset
+    const size_t a_sf0 = (size_t)(a.row0 / 128) * oa.nk64 * kSfChunk, w_sf0 = (size_t)(w.row0 / 128) * ow.nk64 * kSfChunk;
+    p.sfa_pos = pa + 2 * oa.plane + a_sf0;
     p.sfa_neg = p.sfa_pos + oa.sf;
-    p.a_exp = reinterpret_cast<const int*>(pa + 2 * oa.plane + 2 * oa.sf);
-    p.sfb_pos = pw + 2 * ow.plane;
+    p.a_exp = reinterpret_cast<const int*>(pa + 2 * oa.plane + 2 * oa.sf) + a.row0;
+    p.sfb_pos = pw + 2 * ow.plane + w_sf0;
     p.sfb_neg = p.sfb_pos + ow.sf;
-    p.w_exp = reinterpret_cast<const int*>(pw + 2 * ow.plane + 2 * ow.sf);
+    p.w_exp = reinterpret_cast<const int*>(pw + 2 * ow.plane + 2 * ow.sf) + w.row0;
     p.M = M; p.N = N; p.K = K; p.ld_c = ld_c; p.C = C;
+    p.a_row0 = a.row0; p.w_row0 = w.row0;
     p.nk64 = oa.nk64;
     p.vec_store = aligned(C, 32) && ld_c % 8 == 0;     // 32-byte stores in the epilogue
     p.status = status;
-    return fp4_block_k() == 256 ? launch_fp4<256>(pa, pw, oa, ow, p, dev, st) : launch_fp4<128>(pa, pw, oa, ow, p, dev, st);
+    return fp4_block_k() == 256 ? launch_fp4<256>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st)
+                                : launch_fp4<128>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
+}
+
+int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K, float* C,
+                      int64_t ld_c, void* workspace, cudaStream_t st) {
+    return gemm_fp4_prepared_at({a_prepared, M, M, 0}, {w_prepared, N, N, 0}, M, N, K, C, ld_c, workspace, st);
 }
 
 // Size of a prepared operand: as the A operand (rows padded to 128) or the W operand (rows padded to 256).
@@ -547,8 +558,8 @@ size_t gemm_fp4_prepared_bytes(int64_t rows, int64_t K, bool is_weight) {
 
 // Fused form: one launch of the cast kernel writes the canonical operand and the prepared one.
 int gemm_fp4_quantize_prepared(const void* x, int64_t rows, int64_t K, bool is_weight, uint8_t* codes, uint8_t* scales,
-                               void* prepared, cudaStream_t st) {
-    const OperandLayout o = operand_layout(rows, K, is_weight ? BN : BM);
+                               void* prepared, cudaStream_t st, int64_t layout_rows) {
+    const OperandLayout o = operand_layout(layout_rows ? layout_rows : rows, K, is_weight ? BN : BM);
     uint8_t* base = static_cast<uint8_t*>(prepared);
     return quantize_rows_prepared(x, rows, K, codes, scales, base, base + o.plane, base + 2 * o.plane,
                                   base + 2 * o.plane + o.sf, reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf), o.nk64,
@@ -565,8 +576,9 @@ int gemm_fp4_softmax_prepared(const float* S, int64_t rows, int64_t cols, int64_
 }
 
 int gemm_fp4_prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, bool is_weight,
-                     void* prepared, cudaStream_t st) {
-    return prepare(codes, scales, rows, K, operand_layout(rows, K, is_weight ? BN : BM), static_cast<uint8_t*>(prepared), st);
+                     void* prepared, cudaStream_t st, int64_t layout_rows) {
+    return prepare(codes, scales, rows, K, operand_layout(layout_rows ? layout_rows : rows, K, is_weight ? BN : BM),
+                   static_cast<uint8_t*>(prepared), st);
 }
 
 int gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes, const uint8_t* w_scales,

@@ -70,9 +70,13 @@ template <int TPG>
 __global__ void __launch_bounds__(kThreads)
 quantize_cols_kernel(const __nv_bfloat16* __restrict__ x, int64_t R, int64_t C, int64_t ld,
                      uint32_t* __restrict__ codes, uint16_t* __restrict__ scales, int gs) {
+    // blockIdx.z: one of several [R, C] matrices stored one after another (R * ld elements apart); their
+    // transposed outputs follow one another as well
     __shared__ uint16_t tile[kTC][kTR + 2];  // [column][row], padded
     const int64_t r0 = (int64_t)blockIdx.y * kTR, c0 = (int64_t)blockIdx.x * kTC;
-    const uint16_t* xs = reinterpret_cast<const uint16_t*>(x);
+    const uint16_t* xs = reinterpret_cast<const uint16_t*>(x) + (int64_t)blockIdx.z * R * ld;
+    codes += (int64_t)blockIdx.z * (C * R / 8);
+    scales += (int64_t)blockIdx.z * (C * R / gs);
     for (int i = threadIdx.x; i < kTR * kTC; i += kThreads) {
         const int rr = i / kTC, cc = i % kTC;
         uint16_t v = 0;
@@ -308,9 +312,9 @@ namespace {
 
 template <int TPG>
 int launch_cols(const void* x, int64_t R, int64_t C, int64_t ld, int gs, uint8_t* codes,
-                uint8_t* scales, cudaStream_t st) {
-    dim3 grid((unsigned)((C + kTC - 1) / kTC), (unsigned)((R + kTR - 1) / kTR));
-    if (grid.y > 65535) return AMX_ERR_SHAPE;
+                uint8_t* scales, cudaStream_t st, int64_t batch = 1) {
+    dim3 grid((unsigned)((C + kTC - 1) / kTC), (unsigned)((R + kTR - 1) / kTR), (unsigned)batch);
+    if (grid.y > 65535 || batch > 65535) return AMX_ERR_SHAPE;
     quantize_cols_kernel<TPG><<<grid, kThreads, 0, st>>>(
         reinterpret_cast<const __nv_bfloat16*>(x), R, C, ld, reinterpret_cast<uint32_t*>(codes),
         reinterpret_cast<uint16_t*>(scales), gs);
@@ -318,6 +322,14 @@ int launch_cols(const void* x, int64_t R, int64_t C, int64_t ld, int gs, uint8_t
 }
 
 }  // namespace
+
+// amx_quantize_t with group size 32 on `batch` matrices [R, C] stored one after another (contiguous rows); the
+// canonical outputs of their transposes follow one another too.
+int quantize_cols_batched(const void* x, int64_t batch, int64_t R, int64_t C, uint8_t* codes, uint8_t* scales,
+                          cudaStream_t st) {
+    return launch_cols<4>(x, R, C, C, 32, codes, scales, st, batch);
+}
+
 }  // namespace amx
 
 extern "C" int amx_quantize(const void* x, int64_t rows, int64_t K, int64_t ld_x, int group_size,

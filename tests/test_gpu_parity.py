@@ -370,12 +370,16 @@ def test_attention_small_head_against_oracle_pipeline():
     assert rel_fro(O.cpu().numpy(), Ocpu) <= GEMM_TOL
 
 
-def test_attention_all_heads_entry_point_matches_per_head_pipeline():
-    q, k, v = (dev_bf16(t) for t in inputs.attention_qkv(heads=3, seq=320))
-    O = amx.attention_heads(q, k, v)
-    for h in range(3):
-        Oh, _ = amx.attention(q[h], k[h], v[h])
-        assert torch.equal(O[h], Oh)
+@pytest.mark.parametrize("heads,seq,flags", [(3, 320, amx.GEMM_AUTO),      # head by head (seq % 128 != 0)
+                                             (10, 128, amx.GEMM_AUTO),     # chunks of 8 + 2 heads, small-product kernel
+                                             (9, 256, amx.GEMM_FP4),       # chunks of 8 + 1, FP4 kernel on stacked operands
+                                             (2, 1024, amx.GEMM_AUTO)])    # AUTO picks the FP4 kernel
+def test_attention_all_heads_entry_point_matches_per_head_pipeline(heads, seq, flags):
+    q, k, v = (dev_bf16(t) for t in inputs.attention_qkv(heads=heads, seq=seq))
+    O = amx.attention_heads(q, k, v, flags=flags)
+    for h in range(heads):
+        Oh, _ = amx.attention(q[h], k[h], v[h], flags=flags)
+        assert torch.equal(O[h], Oh), h
 
 
 def test_config5_full_size_attention_sampled():
