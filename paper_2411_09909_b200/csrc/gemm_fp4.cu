@@ -176,6 +176,7 @@ struct Params {
     const int *a_exp, *w_exp;
     int64_t M, N, K, ld_c;
     int64_t a_row0, w_row0;      // first rows of this product's operands inside the (stacked) prepared operands
+    int a_planes;                // 1: the left-hand operand has no negative elements, its negative plane is skipped
     float* C;
     int nk64, vec_store;
     int* status;
@@ -276,19 +277,23 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 const uint32_t parity_next = ((it + 1) / kStages) & 1;
                 uint32_t seen = 0;
                 if (elect_one()) {
+                    const int n_mma = p.a_planes * 2 * kSteps;
 #pragma unroll
                     for (int pa = 0; pa < 2; ++pa)
 #pragma unroll
                         for (int pw = 0; pw < 2; ++pw)
 #pragma unroll
                             for (int kk = 0; kk < kSteps; ++kk) {   // 64 elements = 32 bytes along the swizzled row
-                                mma_fp4_block16(tmem, dstage + (((pa ? C_::kOffAn : C_::kOffAp) + kk * 32) >> 4),
-                                                dstage + (((pw ? C_::kOffWn : C_::kOffWp) + kk * 32) >> 4), kIdesc,
-                                                sfa + (pa * kSteps + kk) * 4, sfb + (pw * kSteps + kk) * 8,
-                                                (pa | pw | kk) ? 1u : accumulate);
-                                // with two MMAs still to go (they keep the pipe busy meanwhile), look whether the
-                                // next K block is complete, so that its MMAs can follow without a wait
-                                if (pa == 1 && pw == 0 && kk == kSteps - 1) seen = mbar_try_wait(&ctl->full[s_next], parity_next);
+                                const int n = (pa * 2 + pw) * kSteps + kk;
+                                if (n < n_mma) {
+                                    mma_fp4_block16(tmem, dstage + (((pa ? C_::kOffAn : C_::kOffAp) + kk * 32) >> 4),
+                                                    dstage + (((pw ? C_::kOffWn : C_::kOffWp) + kk * 32) >> 4), kIdesc,
+                                                    sfa + (pa * kSteps + kk) * 4, sfb + (pw * kSteps + kk) * 8,
+                                                    (pa | pw | kk) ? 1u : accumulate);
+                                    // with two MMAs still to go (they keep the pipe busy meanwhile), look whether the
+                                    // next K block is complete, so that its MMAs can follow without a wait
+                                    if (n == n_mma - 3) seen = mbar_try_wait(&ctl->full[s_next], parity_next);
+                                }
                             }
                     mma_commit(&ctl->empty[s]);
                 }
@@ -539,6 +544,7 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
     p.w_exp = reinterpret_cast<const int*>(pw + 2 * ow.plane + 2 * ow.sf) + w.row0;
     p.M = M; p.N = N; p.K = K; p.ld_c = ld_c; p.C = C;
     p.a_row0 = a.row0; p.w_row0 = w.row0;
+    p.a_planes = a.nonneg ? 1 : 2;
     p.nk64 = oa.nk64;
     p.vec_store = aligned(C, 32) && ld_c % 8 == 0;     // 32-byte stores in the epilogue
     p.status = status;
