@@ -34,7 +34,7 @@ NOMINAL_HBM_GBS = 8000.0
 BYTES_PER_ELEM = 2.0 + 0.5 + 2.0 / 32.0   # bf16 read + 4-bit code + two scale bytes per 32
 # DRAM bytes (read + write) per GEMM launch, mean over the four layer shapes, from the ncu capture summarised
 # in profiles/; None until a capture of the current kernel exists.
-GEMM_DRAM_TRAFFIC_PER_LAUNCH = {"auto": 169.2e6, "fp4": 169.2e6}
+GEMM_DRAM_TRAFFIC_PER_LAUNCH = {"auto": 178.9e6, "fp4": 178.9e6}
 
 
 def measured_peaks():
@@ -160,6 +160,36 @@ def run_reference(args):
         "gpu_launches": 0,
     }
     print(json.dumps(line))
+
+
+def time_attention(heads: int, iters: int = 3):
+    """Config 5 (heads x 8192 x 128, non-causal) through amx_attention: milliseconds per call."""
+    import torch
+    from paper_2411_09909_b200 import amx, inputs
+    L = amx.lib()
+    L5, D5 = 8192, 128
+    q5, k5, v5 = (torch.from_numpy(t.view(np.int16)).cuda().view(torch.bfloat16) for t in inputs.attention_qkv(heads, L5))
+    ws5 = torch.empty(L.amx_attention_workspace_bytes(L5, D5), dtype=torch.uint8, device="cuda")
+    o5 = torch.empty((heads, L5, D5), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def attn():
+        rc = L.amx_attention(q5.data_ptr(), k5.data_ptr(), v5.data_ptr(), heads, L5, D5, 0, o5.data_ptr(),
+                             ws5.data_ptr(), ws5.numel(), stream)
+        if rc != 0:
+            raise RuntimeError(amx.status_string(rc))
+
+    attn()
+    torch.cuda.synchronize()
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a0.record()
+    for _ in range(iters):
+        attn()
+    a1.record()
+    torch.cuda.synchronize()
+    a_ms = a0.elapsed_time(a1) / iters
+    return {"workload": f"config 5: {heads} heads x {L5} x {D5}, non-causal; Q, K, V and the attention map all cast to AMXFP4",
+            "ms": a_ms, "useful_tflops": 4.0 * heads * L5 * L5 * D5 / (a_ms * 1e-3) / 1e12, "ms_per_head": a_ms / heads}
 
 
 def run_ours(args):
@@ -393,29 +423,7 @@ def run_ours(args):
     # ---- config 5: fully quantized attention for all heads (32 x 8192 x 128), one call of amx_attention
     attention = None
     if not args.layers and not args.skip_extras and world == 1:
-        H5, L5, D5 = 32, 8192, 128
-        q5, k5, v5 = (to_dev(t.reshape(H5 * L5, D5)).view(H5, L5, D5) for t in inputs.attention_qkv(H5, L5))
-        ws5 = torch.empty(L.amx_attention_workspace_bytes(L5, D5), dtype=torch.uint8, device="cuda")
-        o5 = torch.empty((H5, L5, D5), dtype=torch.float32, device="cuda")
-
-        def attn():
-            check(L.amx_attention(q5.data_ptr(), k5.data_ptr(), v5.data_ptr(), H5, L5, D5, 0, o5.data_ptr(),
-                                  ws5.data_ptr(), ws5.numel(), stream))
-
-        attn()
-        torch.cuda.synchronize()
-        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a_iters = 3
-        a0.record()
-        for _ in range(a_iters):
-            attn()
-        a1.record()
-        torch.cuda.synchronize()
-        a_ms = a0.elapsed_time(a1) / a_iters
-        attention = {"workload": "config 5: 32 heads x 8192 x 128, non-causal; Q, K, V and the attention map all cast to AMXFP4",
-                     "ms": a_ms, "useful_tflops": 4.0 * H5 * L5 * L5 * D5 / (a_ms * 1e-3) / 1e12,
-                     "ms_per_head": a_ms / H5}
-        del q5, k5, v5, ws5, o5
+        attention = time_attention(32)
 
     # ---- config 1: one small layer (128 x 1024 -> 1024), latency-bound: microseconds per call of amx_quant_gemm
     small_case = None
@@ -546,8 +554,16 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of a CUDA graph of the step")
     ap.add_argument("--layers", default="", help="comma-separated layer indices to run (profiling aid; default all)")
     ap.add_argument("--skip-extras", action="store_true", help="skip the e2e and cpu_baseline legs (profiling aid)")
+    ap.add_argument("--attention-only", action="store_true", help="time only the config-5 attention call (profiling aid)")
+    ap.add_argument("--heads", type=int, default=32, help="heads for --attention-only")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.attention_only:
+        import torch
+        from paper_2411_09909_b200 import build
+        torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+        build.build()
+        print(json.dumps({"attention": time_attention(args.heads, iters=1)}))
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

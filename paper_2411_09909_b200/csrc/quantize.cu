@@ -152,6 +152,7 @@ __device__ __forceinline__ void finish_prepared_row(int64_t row, bool row_live, 
     // One shared-memory atomic per warp.  The key of an E5M2 byte grows with the byte (scales carry no sign
     // bit), so the largest byte has the largest key.
     top = __reduce_max_sync(0xFFFFFFFFu, top);
+    __syncthreads();                               // the slot was zeroed at the top of the kernel
     if ((gx & 31) == 0 && top > 0) atomicMax(kmax_s, scale_key(top));
     __syncthreads();
     const int kmax = *kmax_s;
@@ -183,8 +184,7 @@ cast_prepared_kernel(const uint4* __restrict__ x, int64_t R, int G, uint4* __res
     const int gx = threadIdx.x, rl = threadIdx.y, GX = blockDim.x;
     const int64_t row = (int64_t)blockIdx.x * blockDim.y + rl;
     const bool row_live = row < R;
-    if (gx == 0) kmax_s[rl] = 0;
-    __syncthreads();
+    if (gx == 0) kmax_s[rl] = 0;                    // visible to all after the barrier in finish_prepared_row
     const int64_t v_row = row * G;
     uint32_t sc_first = 0;                      // scale bytes of this thread's first group (its only one when
                                                 // the block is as wide as its rows)
@@ -251,7 +251,6 @@ softmax_cast_kernel(const float* __restrict__ S, int64_t R, int G, int64_t ld_s,
         }
     }
     if (!pos) return;                               // canonical output only
-    __syncthreads();                                // kmax_s is zero before the first atomic
     finish_prepared_row(row, row_live, G, gx, softmax::kT, top, sc_first, scales, &kmax_s, sf_pos, sf_neg, row_exp, nk64);
 }
 
