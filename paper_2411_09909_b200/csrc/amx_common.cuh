@@ -39,6 +39,20 @@ __device__ __forceinline__ int scale_key(uint32_t b) {
     const int e = (b >> 2) & 31, m = b & 3;
     return e ? e + 2 : (m == 0 ? 0 : (m == 1 ? 1 : 2));
 }
+// Per-row word of a prepared FP4-GEMM operand: bits 15..0 the row's power-of-two offset (largest exponent key
+// - 25; 0 for an all-zero row) as a signed 16-bit number, bit 16 set when some group of the row has a nonzero
+// positive-side scale, bit 17 the same for the negative side.  A tile whose rows all lack a side has an
+// all-zero plane for it, and the GEMM does not issue that plane's products.
+constexpr int kRowHasPos = 1 << 16, kRowHasNeg = 1 << 17;
+__host__ __device__ __forceinline__ int row_word(int kmax, int side_bits) {
+    return ((kmax ? kmax - 25 : 0) & 0xFFFF) | side_bits;
+}
+__host__ __device__ __forceinline__ int row_word_exp(int w) { return (int)(short)(w & 0xFFFF); }
+// side bits of a group's scale bytes {neg : pos}
+__device__ __forceinline__ int side_bits_of(uint32_t sc) {
+    return ((sc & 0xFFu) ? kRowHasPos : 0) | ((sc >> 8) ? kRowHasNeg : 0);
+}
+
 // UE4M3 byte of the E5M2 byte b for a row whose largest key is kmax (0 when it does not fit).
 __device__ __forceinline__ uint32_t to_ue4m3(uint32_t b, int kmax) {
     const int e = (b >> 2) & 31, m = b & 3;

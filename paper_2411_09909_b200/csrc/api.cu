@@ -307,7 +307,7 @@ extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_
             if (k_pv == AMX_GEMM_FP4) {
                 rc = gemm_fp4_softmax_prepared(S, L, L, L, alpha, false, w + a.pc, w + a.ps, w + a.pp, st);
                 if (rc == AMX_OK)
-                    rc = gemm_fp4_prepared_at({w + a.pp, L, L, 0, /*nonneg=*/true}, {w + a.pv, hc * d, chunk * d + 128, i * d}, L, d, L, oh, d,
+                    rc = gemm_fp4_prepared_at({w + a.pp, L, L, 0}, {w + a.pv, hc * d, chunk * d + 128, i * d}, L, d, L, oh, d,
                                               w + a.gemm, st);
             } else {
                 rc = softmax_cast_rows(S, L, L, L, alpha, w + a.pc, w + a.ps, nullptr, nullptr, nullptr, nullptr, nullptr, 0, L,

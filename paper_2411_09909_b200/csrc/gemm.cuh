@@ -49,8 +49,6 @@ int gemm_fp4_softmax_prepared(const float* S, int64_t rows, int64_t cols, int64_
 struct Fp4Operand {
     const void* prepared;
     int64_t rows_total, layout_rows, row0;
-    bool nonneg = false;   // left-hand operand only: no element is negative (a softmax output), so the products
-                           // with its all-zero negative plane are not issued
 };
 int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
                          int64_t ld_c, void* workspace, cudaStream_t st);

@@ -92,8 +92,8 @@ constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17)
 // ------------------------------------------------------------------------- preparation --
 // One launch per operand; one block per 32 operand rows (rows beyond R, up to the padded row count,
 // get zero scale factors so that padded tile rows multiply zero codes by a finite scale).
-//   1. row offsets: a warp per row finds the largest exponent key kmax among the row's scales;
-//      row_exp = kmax - 25 is the power of two by which the row's UE4M3 scales understate the true ones
+//   1. row words: a warp per row finds the largest exponent key kmax among the row's scales (kmax - 25 is the
+//      power of two by which the row's UE4M3 scales understate the true ones) and which sides occur at all
 //   2. sign planes: every nibble goes to the plane of its sign bit, zero in the other plane
 //   3. scale factors of both planes in the layout the MMA reads:
 //      [plane][row block of 128][K/64 block][512 B], byte (r%32)*16 + (r/32)*4 + (k16 % 4);
@@ -108,19 +108,20 @@ prepare_operand_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restr
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int r = warp; r < kPrepRows; r += 8) {
         const int64_t row = row0 + r;
-        int kmax = 0;
+        int kmax = 0, sides = 0;
         if (row < R) {
             const unsigned short* s2 = reinterpret_cast<const unsigned short*>(scales + row * G * 2);
             for (int64_t g = lane; g < G; g += 32) {
                 const uint32_t v = __ldg(s2 + g);
                 kmax = max(kmax, max(scale_key(v & 0xFF), scale_key(v >> 8)));
+                sides |= side_bits_of(v);
             }
         }
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, d));
+        kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+        sides = __reduce_or_sync(0xFFFFFFFFu, sides);
         if (lane == 0) {
             kmax_s[r] = kmax;
-            if (row < R) row_exp[row] = kmax ? kmax - 25 : 0;
+            if (row < R) row_exp[row] = row_word(kmax, sides);
         }
     }
     // sign planes of this block's rows (contiguous in memory: rows are K/2 bytes apart)
@@ -176,7 +177,7 @@ struct Params {
     const int *a_exp, *w_exp;
     int64_t M, N, K, ld_c;
     int64_t a_row0, w_row0;      // first rows of this product's operands inside the (stacked) prepared operands
-    int a_planes;                // 1: the left-hand operand has no negative elements, its negative plane is skipped
+
     float* C;
     int nk64, vec_store;
     int* status;
@@ -259,7 +260,29 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         const uint64_t desc0 = operand_desc<BK_>(smem_u32(tiles));
         int it = 0, t = 0;
         bool ok = true, ready = false;                           // ready: the next K block's barrier was seen complete
+        // Which sign planes a tile's rows use at all (bits of the row words, OR-ed over the tile's 128 + 256
+        // rows): the products with a plane that is zero for the whole tile are not issued.  The words of the
+        // next tile are fetched while the current one runs.
+        auto tile_sides = [&](int64_t tile) {
+            int bits = 0;
+            if (tile < total_tiles) {
+                const int64_t m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
+#pragma unroll
+                for (int i = 0; i < BM / 32; ++i)
+                    if (m0 + i * 32 + lane < p.M) bits |= (__ldg(p.a_exp + m0 + i * 32 + lane) >> 16) & 3;
+#pragma unroll
+                for (int i = 0; i < BN / 32; ++i)
+                    if (n0 + i * 32 + lane < p.N) bits |= ((__ldg(p.w_exp + n0 + i * 32 + lane) >> 16) & 3) << 2;
+            }
+            return bits;
+        };
+        int sides_next = tile_sides(blockIdx.x);
         for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t) {
+            int sides = __reduce_or_sync(0xFFFFFFFFu, sides_next);   // bit 0/1: A has +/-, bit 2/3: W has +/-
+            sides_next = tile_sides(tile + gridDim.x);
+            if (!(sides & 3)) sides |= 1;                        // an all-zero operand: one product, which zeroes the tile
+            if (!(sides & 12)) sides |= 4;
+            const int n_mma = ((sides & 1) + ((sides >> 1) & 1)) * (((sides >> 2) & 1) + ((sides >> 3) & 1)) * kSteps;
             // the previous tile's accumulator must have been read out before it is overwritten
             if (t > 0) ok = mbar_wait(&ctl->accum_empty, (t - 1) & 1, &ctl->abort, p.status);
             tc_fence_after();
@@ -277,22 +300,22 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 const uint32_t parity_next = ((it + 1) / kStages) & 1;
                 uint32_t seen = 0;
                 if (elect_one()) {
-                    const int n_mma = p.a_planes * 2 * kSteps;
+                    int idx = 0;                                 // MMAs issued so far in this K block
 #pragma unroll
                     for (int pa = 0; pa < 2; ++pa)
 #pragma unroll
                         for (int pw = 0; pw < 2; ++pw)
 #pragma unroll
                             for (int kk = 0; kk < kSteps; ++kk) {   // 64 elements = 32 bytes along the swizzled row
-                                const int n = (pa * 2 + pw) * kSteps + kk;
-                                if (n < n_mma) {
+                                if (((sides >> pa) & 1) && ((sides >> (2 + pw)) & 1)) {
                                     mma_fp4_block16(tmem, dstage + (((pa ? C_::kOffAn : C_::kOffAp) + kk * 32) >> 4),
                                                     dstage + (((pw ? C_::kOffWn : C_::kOffWp) + kk * 32) >> 4), kIdesc,
                                                     sfa + (pa * kSteps + kk) * 4, sfb + (pw * kSteps + kk) * 8,
-                                                    (pa | pw | kk) ? 1u : accumulate);
+                                                    idx ? 1u : accumulate);
                                     // with two MMAs still to go (they keep the pipe busy meanwhile), look whether the
                                     // next K block is complete, so that its MMAs can follow without a wait
-                                    if (n == n_mma - 3) seen = mbar_try_wait(&ctl->full[s_next], parity_next);
+                                    if (idx == max(n_mma - 3, 0)) seen = mbar_try_wait(&ctl->full[s_next], parity_next);
+                                    ++idx;
                                 }
                             }
                     mma_commit(&ctl->empty[s]);
@@ -370,9 +393,9 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t) {
             const int64_t m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
             int* w_exp = ctl->w_exp[t & 1];
-            for (int i = tid_e; i < BN; i += kEpilogueWarps * 32) w_exp[i] = (n0 + i < p.N) ? p.w_exp[n0 + i] : 0;
+            for (int i = tid_e; i < BN; i += kEpilogueWarps * 32) w_exp[i] = (n0 + i < p.N) ? row_word_exp(p.w_exp[n0 + i]) : 0;
             const int64_t m = m0 + q * 32 + lane;
-            const int a_exp = (m < p.M) ? p.a_exp[m] : 0;
+            const int a_exp = (m < p.M) ? row_word_exp(p.a_exp[m]) : 0;
             ok = mbar_wait(&ctl->accum_full, t & 1, &ctl->abort, p.status);
             tc_fence_after();
             // every epilogue warp has written its part of w_exp (named barrier: the other roles do not join)
@@ -544,7 +567,7 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
     p.w_exp = reinterpret_cast<const int*>(pw + 2 * ow.plane + 2 * ow.sf) + w.row0;
     p.M = M; p.N = N; p.K = K; p.ld_c = ld_c; p.C = C;
     p.a_row0 = a.row0; p.w_row0 = w.row0;
-    p.a_planes = a.nonneg ? 1 : 2;
+
     p.nk64 = oa.nk64;
     p.vec_store = aligned(C, 32) && ld_c % 8 == 0;     // 32-byte stores in the epilogue
     p.status = status;

@@ -142,20 +142,24 @@ __device__ __forceinline__ uint32_t emit_group(const uint32_t (&w)[16], int64_t 
     return sc;
 }
 
-// Second half of a prepared cast, for the GX threads (a multiple of 32) that own row `row` (`top`: largest scale
-// byte the thread has seen; kmax_s: the row's shared-memory slot, zero on entry): row maximum of the exponent
-// keys, the row's scale factors in the tensor cores' layout, padding included, and the row offset.
+// Second half of a prepared cast, for the GX threads (a multiple of 32) that own row `row` (`top`: the largest
+// positive-side scale byte the thread has seen in bits 7..0, the largest negative-side one in bits 15..8;
+// slot: the row's two shared-memory words, zero on entry): row maximum of the exponent keys and which sides
+// occur, the row's scale factors in the tensor cores' layout, padding included, and the row word.
 __device__ __forceinline__ void finish_prepared_row(int64_t row, bool row_live, int G, int gx, int GX, uint32_t top,
                                                     uint32_t sc_first, const uint16_t* __restrict__ scales,
-                                                    int* kmax_s, uint8_t* __restrict__ sf_pos,
+                                                    int* slot, uint8_t* __restrict__ sf_pos,
                                                     uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp, int nk64) {
-    // One shared-memory atomic per warp.  The key of an E5M2 byte grows with the byte (scales carry no sign
+    // Two shared-memory atomics per warp.  The key of an E5M2 byte grows with the byte (scales carry no sign
     // bit), so the largest byte has the largest key.
-    top = __reduce_max_sync(0xFFFFFFFFu, top);
+    const uint32_t top_p = __reduce_max_sync(0xFFFFFFFFu, top & 0xFFu), top_n = __reduce_max_sync(0xFFFFFFFFu, top >> 8);
     __syncthreads();                               // the slot was zeroed at the top of the kernel
-    if ((gx & 31) == 0 && top > 0) atomicMax(kmax_s, scale_key(top));
+    if ((gx & 31) == 0 && (top_p | top_n)) {
+        atomicMax(&slot[0], scale_key(max(top_p, top_n)));
+        atomicOr(&slot[1], side_bits_of(top_p | (top_n << 8)));
+    }
     __syncthreads();
-    const int kmax = *kmax_s;
+    const int kmax = slot[0];
     // offset of this row's bytes inside a chunk; the chunks of one block of 128 rows are consecutive along K
     const int rr = (int)(row & 127);
     const int64_t sf_row = (row >> 7) * nk64 * (int64_t)kSfChunkBytes + (rr & 31) * 16 + (rr >> 5) * 4;
@@ -172,7 +176,7 @@ __device__ __forceinline__ void finish_prepared_row(int64_t row, bool row_live, 
         *reinterpret_cast<uint16_t*>(sf_pos + off) = (uint16_t)(up | (up << 8));
         *reinterpret_cast<uint16_t*>(sf_neg + off) = (uint16_t)(un | (un << 8));
     }
-    if (gx == 0 && row_live) row_exp[row] = kmax ? kmax - 25 : 0;
+    if (gx == 0 && row_live) row_exp[row] = row_word(kmax, slot[1]);
 }
 
 // 40 registers (three blocks of 512 per SM): at 32 the kernel spills and is 12 % slower.
@@ -180,15 +184,15 @@ __global__ void __launch_bounds__(512, 3)
 cast_prepared_kernel(const uint4* __restrict__ x, int64_t R, int G, uint4* __restrict__ codes,
                      uint16_t* __restrict__ scales, uint4* __restrict__ pos, uint4* __restrict__ neg,
                      uint8_t* __restrict__ sf_pos, uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp, int nk64) {
-    __shared__ int kmax_s[kPrepMaxRows];
+    __shared__ int slot_s[kPrepMaxRows][2];
     const int gx = threadIdx.x, rl = threadIdx.y, GX = blockDim.x;
     const int64_t row = (int64_t)blockIdx.x * blockDim.y + rl;
     const bool row_live = row < R;
-    if (gx == 0) kmax_s[rl] = 0;                    // visible to all after the barrier in finish_prepared_row
+    if (gx < 2) slot_s[rl][gx] = 0;                 // visible to all after the barrier in finish_prepared_row
     const int64_t v_row = row * G;
     uint32_t sc_first = 0;                      // scale bytes of this thread's first group (its only one when
                                                 // the block is as wide as its rows)
-    uint32_t top = 0;                           // largest scale byte seen by this thread
+    uint32_t top = 0;                           // largest scale bytes seen by this thread, {neg : pos}
     for (int g = gx; g < G; g += GX) {
         if (!row_live) break;                   // uniform over the warp: a warp sits inside one row
         const int64_t v = v_row + g;
@@ -200,9 +204,9 @@ cast_prepared_kernel(const uint4* __restrict__ x, int64_t R, int G, uint4* __res
         }
         const uint32_t sc = emit_group(w, v, codes, scales, pos, neg);
         if (g == gx) sc_first = sc;
-        top = max(top, max(sc & 0xFFu, sc >> 8));
+        top = __vmaxu4(top, sc);                // byte-wise maximum
     }
-    finish_prepared_row(row, row_live, G, gx, GX, top, sc_first, scales, &kmax_s[rl], sf_pos, sf_neg, row_exp, nk64);
+    finish_prepared_row(row, row_live, G, gx, GX, top, sc_first, scales, slot_s[rl], sf_pos, sf_neg, row_exp, nk64);
 }
 
 // Attention glue in one pass (Appendix C): row softmax of the fp32 logits (times alpha), rounding of the
@@ -218,11 +222,11 @@ softmax_cast_kernel(const float* __restrict__ S, int64_t R, int G, int64_t ld_s,
                     uint4* __restrict__ neg, uint8_t* __restrict__ sf_pos, uint8_t* __restrict__ sf_neg,
                     int* __restrict__ row_exp, int nk64) {
     __shared__ float sh[softmax::kT / 32];
-    __shared__ int kmax_s;
+    __shared__ int slot_s[2];
     const int gx = threadIdx.x;
     const int64_t row = blockIdx.x;
     const bool row_live = row < R;                  // uniform over the block
-    if (gx == 0) kmax_s = 0;
+    if (gx < 2) slot_s[gx] = 0;
     uint32_t sc_first = 0, top = 0;
     if (row_live) {
         const float* s = S + row * ld_s;
@@ -234,7 +238,7 @@ softmax_cast_kernel(const float* __restrict__ S, int64_t R, int G, int64_t ld_s,
                 uint32_t w[16];
                 softmax::normalised_group_e(e, sum, w);
                 sc_first = emit_group(w, v_row + gx, codes, scales, pos, neg);
-                top = max(sc_first & 0xFFu, sc_first >> 8);
+                top = sc_first;
             }
         } else {
             float mx, sum;
@@ -246,12 +250,12 @@ softmax_cast_kernel(const float* __restrict__ S, int64_t R, int G, int64_t ld_s,
                 softmax::normalised_group(t, mx, sum, w);
                 const uint32_t sc = emit_group(w, v_row + g, codes, scales, pos, neg);
                 if (g == gx) sc_first = sc;
-                top = max(top, max(sc & 0xFFu, sc >> 8));
+                top = __vmaxu4(top, sc);
             }
         }
     }
     if (!pos) return;                               // canonical output only
-    finish_prepared_row(row, row_live, G, gx, softmax::kT, top, sc_first, scales, &kmax_s, sf_pos, sf_neg, row_exp, nk64);
+    finish_prepared_row(row, row_live, G, gx, softmax::kT, top, sc_first, scales, slot_s, sf_pos, sf_neg, row_exp, nk64);
 }
 
 template <int EPT, int TPG>

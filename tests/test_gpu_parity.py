@@ -207,6 +207,32 @@ def test_gemm_prepared_two_phase_equals_one_call():
         assert torch.equal(amx.gemm_prepared(pa, pw, 300, 520, 1056), one)
 
 
+@pytest.mark.parametrize("a_side,w_side", [(1, 0), (0, -1), (1, 1), (-1, 1), (2, 0)])
+def test_gemm_fp4_one_sided_operands(a_side, w_side):
+    """Operands without negative (or without positive) elements have an all-zero sign plane; the FP4 kernel then
+    does not issue that plane's products.  side: 0 = mixed signs, +1 / -1 = all elements of that sign,
+    2 = the first 128 rows non-negative and the rest mixed (tiles differ)."""
+    def one_sided(bits, side):
+        x = bits.copy()
+        if side == 1:
+            x &= 0x7FFF
+        elif side == -1:
+            x |= 0x8000
+        elif side == 2:
+            x[:128] &= 0x7FFF
+        return x
+    a = one_sided(inputs.random_groups(71, 300, 1056, "normal"), a_side)
+    w = one_sided(inputs.random_groups(72, 520, 1056, "normal"), w_side)
+    qa, qw = oracle.quantize(a, 32), oracle.quantize(w, 32)
+    ref = oracle.gemm(*qa, *qw, 32)
+    dev = [torch.from_numpy(t).cuda() for t in (*qa, *qw)]
+    assert rel_fro(amx.gemm(*dev, 32, amx.GEMM_FP4).cpu().numpy(), ref) <= GEMM_TOL
+    # through the fused cast as well
+    _, _, pa = amx.quantize_prepared(dev_bf16(a), False)
+    _, _, pw = amx.quantize_prepared(dev_bf16(w), True)
+    assert rel_fro(amx.gemm_prepared(pa, pw, 300, 520, 1056).cpu().numpy(), ref) <= GEMM_TOL
+
+
 def test_quantize_prepared_equals_quantize_then_prepare():
     # row lengths below, at and above one block of the cast kernel (several rows, one row and a fraction of a
     # row per block; threads striding over a long row), ragged row counts, both paddings
