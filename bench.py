@@ -396,6 +396,53 @@ def run_ours(args):
                           "what": "weights cast and prepared once; per step: cast + prepare activations, GEMM"}
         del prep
 
+    # ---- the same GEMM kernel on operands without negative elements (|A|, |W|): their negative planes are all
+    # zero, so the kernel issues one product per tile pair instead of four.  This is what a symmetric FP4 format
+    # with one scale per group would cost on this kernel: the FP4-pipe ceiling of the design.
+    one_sided = None
+    if "mxf4" in gemm_kernel and not args.layers and not args.skip_extras:
+        prep1 = []
+        for li, (K, N) in enumerate(layers):
+            b = bufs[li]
+            a_abs = (A[li].view(torch.int16) & 0x7FFF).view(torch.bfloat16)
+            w_abs = (W[li].view(torch.int16) & 0x7FFF).view(torch.bfloat16)
+            pa = torch.empty(L.amx_prepared_bytes(M, K, GS, 0), dtype=torch.uint8, device="cuda")
+            pw = torch.empty(L.amx_prepared_bytes(N, K, GS, 1), dtype=torch.uint8, device="cuda")
+            check(L.amx_quantize_prepared(a_abs.data_ptr(), M, K, GS, 0, b["ac"].data_ptr(), b["as"].data_ptr(),
+                                          pa.data_ptr(), pa.numel(), stream))
+            check(L.amx_quantize_prepared(w_abs.data_ptr(), N, K, GS, 1, b["wc"].data_ptr(), b["ws"].data_ptr(),
+                                          pw.data_ptr(), pw.numel(), stream))
+            prep1.append((pa, pw))
+            del a_abs, w_abs
+
+        def gemms_only(stream):
+            for li, (K, N) in enumerate(layers):
+                b, (pa, pw) = bufs[li], prep1[li]
+                check(L.amx_gemm_prepared(pa.data_ptr(), pw.data_ptr(), M, N, K, GS, b["c"].data_ptr(), N,
+                                          b["work"].data_ptr(), b["work"].numel(), stream))
+
+        gemms_only(stream)
+        torch.cuda.synchronize()
+        side3 = torch.cuda.Stream()
+        side3.wait_stream(torch.cuda.current_stream())
+        g3 = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g3, stream=side3):
+            gemms_only(torch.cuda.current_stream().cuda_stream)
+        for _ in range(3):
+            g3.replay()
+        o0, o1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        o0.record()
+        for _ in range(args.steps):
+            g3.replay()
+        o1.record()
+        torch.cuda.synchronize()
+        o_ms = o0.elapsed_time(o1) / args.steps
+        one_sided = {"tflops": flops_step / (o_ms * 1e-3) / 1e12, "ms_per_step": o_ms,
+                     "what": "the four GEMMs alone on |A| and |W| (no negative elements: one FP4 product per tile "
+                             "pair instead of four), i.e. the rate a one-scale-per-group FP4 format gets from this kernel"}
+        del prep1
+
     # ---- the cast alone on a tensor larger than L2 (config-4 activation shape, 16384 x 8192 = 268 MB of bf16)
     quant_large = None
     if not args.layers:
@@ -523,6 +570,7 @@ def run_ours(args):
                      "kernel": f"amx_gemm ({gemm_kernel})",
                      "peak_source": f"4 x sustained bf16 cuBLAS rate ({peaks['source']}), nominal FP4:bf16 ratio"},
         "weights_cached": weights_cached,
+        "gemm_one_sided_operands": one_sided,
         "attention": attention,
         "small_case": small_case,
         "clocks": clocks,
