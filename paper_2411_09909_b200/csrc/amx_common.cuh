@@ -53,6 +53,16 @@ __device__ __forceinline__ int side_bits_of(uint32_t sc) {
     return ((sc & 0xFFu) ? kRowHasPos : 0) | ((sc >> 8) ? kRowHasNeg : 0);
 }
 
+// Scale factors of a prepared operand: chunks of 512 bytes per [128 rows x 64 elements], the chunks of one block
+// of 128 rows consecutive along K; inside a chunk byte (r % 32) * 16 + (r / 32) * 4 + (k16 % 4), one scale per 16
+// elements.  Offset of row `row`'s bytes of its first chunk, and of 32-group g's two bytes relative to that.
+constexpr int kSfChunkBytes = 512;
+__host__ __device__ __forceinline__ int64_t sf_row_offset(int64_t row, int nk64) {
+    const int rr = (int)(row & 127);
+    return (row >> 7) * nk64 * (int64_t)kSfChunkBytes + (rr & 31) * 16 + (rr >> 5) * 4;
+}
+__host__ __device__ __forceinline__ int64_t sf_group_offset(int g) { return (int64_t)(g >> 1) * kSfChunkBytes + (g & 1) * 2; }
+
 // UE4M3 byte of the E5M2 byte b for a row whose largest key is kmax (0 when it does not fit).
 __device__ __forceinline__ uint32_t to_ue4m3(uint32_t b, int kmax) {
     const int e = (b >> 2) & 31, m = b & 3;

@@ -271,6 +271,10 @@ extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_
     const float alpha = 1.0f / sqrtf((float)d);
     float* S = reinterpret_cast<float*>(w + a.S);
     const int64_t chunk = attn_chunk(L, d);
+    // both products on the FP4 kernel and whole 256-column tiles: softmax and cast run in the first product's
+    // epilogue (the S region of the workspace then only holds the per-tile row statistics)
+    const bool two_pass = k_qk == AMX_GEMM_FP4 && k_pv == AMX_GEMM_FP4 && L % 256 == 0 &&
+                          gemm_fp4_attn_scratch_bytes(L) <= (size_t)L * L * 4;
     const size_t head_in = (size_t)L * d * 2;                       // bytes of one head of q, k or v
     const size_t qk_codes = (size_t)L * d / 2, qk_scales = (size_t)L * (d / 32) * 2;   // one head of Q or K, canonical
     const size_t v_codes = (size_t)d * L / 2, v_scales = (size_t)d * (L / 32) * 2;     // one head of V^T
@@ -295,6 +299,16 @@ extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_
         if (rc != AMX_OK) return rc;
         for (int64_t i = 0; i < hc; ++i) {
             float* oh = o + (size_t)(h0 + i) * L * d;
+            if (two_pass) {
+                // the logits never reach memory: Q K^T runs twice, its epilogues do the softmax and the cast of P
+                rc = gemm_fp4_attn_scores({w + a.pq, hc * L, chunk * L, i * L}, {w + a.pk, hc * L, chunk * L + 128, i * L}, L, d,
+                                          alpha, S, w + a.pc, w + a.ps, w + a.pp, w + a.gemm, st);
+                if (rc == AMX_OK)
+                    rc = gemm_fp4_prepared_at({w + a.pp, L, L, 0}, {w + a.pv, hc * d, chunk * d + 128, i * d}, L, d, L, oh, d,
+                                              w + a.gemm, st);
+                if (rc != AMX_OK) return rc;
+                continue;
+            }
             // S = AMX(Q) AMX(K)^T
             if (k_qk == AMX_GEMM_FP4)
                 rc = gemm_fp4_prepared_at({w + a.pq, hc * L, chunk * L, i * L}, {w + a.pk, hc * L, chunk * L + 128, i * L}, L,

@@ -111,5 +111,27 @@ __device__ __forceinline__ uint32_t encode8(const uint32_t* w, float inv_p, floa
     return cvt_e2m1x8(r);
 }
 
+// One group of an FP4-GEMM operand from its 16 bf16x2 words: canonical codes and scale bytes at group index v,
+// and the sign planes that are asked for (pos / neg may be nullptr).  Returns the scale bytes {neg : pos}.
+__device__ __forceinline__ uint32_t emit_group(const uint32_t (&w)[16], int64_t v, uint4* __restrict__ codes,
+                                               uint16_t* __restrict__ scales, uint4* __restrict__ pos,
+                                               uint4* __restrict__ neg) {
+    float inv_p, inv_n;
+    const uint32_t sc = group_scales(side_maxima<16>(w), inv_p, inv_n);
+    uint32_t nib[4], pp[4], nn[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        nib[j] = encode8(w + 4 * j, inv_p, inv_n);
+        const uint32_t m = ((nib[j] >> 3) & 0x11111111u) * 15u;   // 0xF on negative nibbles
+        nn[j] = nib[j] & m;
+        pp[j] = nib[j] & ~m;
+    }
+    codes[v] = make_uint4(nib[0], nib[1], nib[2], nib[3]);
+    if (pos) pos[v] = make_uint4(pp[0], pp[1], pp[2], pp[3]);
+    if (neg) neg[v] = make_uint4(nn[0], nn[1], nn[2], nn[3]);
+    scales[v] = (uint16_t)sc;
+    return sc;
+}
+
 }  // namespace cast
 }  // namespace amx

@@ -52,6 +52,11 @@ struct Fp4Operand {
 };
 int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
                          int64_t ld_c, void* workspace, cudaStream_t st);
+// P = softmax(alpha * Q K^T) cast to AMXFP4 (canonical + prepared left-hand operand) without the logits in
+// memory; L % 256 == 0; scratch of gemm_fp4_attn_scratch_bytes(L) bytes.
+size_t gemm_fp4_attn_scratch_bytes(int64_t L);
+int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, int64_t d, float alpha, void* scratch,
+                         uint8_t* p_codes, uint8_t* p_scales, void* p_prepared, void* workspace, cudaStream_t st);
 int quantize_cols_batched(const void* x, int64_t batch, int64_t R, int64_t C, uint8_t* codes, uint8_t* scales,
                           cudaStream_t st);
 int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,

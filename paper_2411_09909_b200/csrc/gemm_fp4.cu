@@ -34,7 +34,9 @@
 #include <cstdlib>
 #include <mutex>
 
+#include "cast_math.cuh"
 #include "gemm.cuh"
+#include "softmax_math.cuh"
 #include "tcgen05.cuh"
 
 namespace amx {
@@ -181,7 +183,19 @@ struct Params {
     float* C;
     int nk64, vec_store;
     int* status;
+    // attention epilogues (kEpiStats, kEpiCast): the tile holds logits S = Q K^T; `alpha` scales them
+    float alpha;
+    float2* part;            // kEpiStats out: per row and half tile {max, sum of exp} of alpha * S, [M][2 * n_tiles]
+    const float2* rowstat;   // kEpiCast in: per row {-max * log2(e), 1 / sum}
+    const int* p_kmax;       // kEpiCast in: per row the largest exponent key of the row's scales
+    uint4 *p_codes, *p_pos;  // kEpiCast out: canonical codes of P = softmax(alpha * S) and its positive plane
+    uint16_t* p_scales;
+    uint8_t* p_sf;           // scale factors of the positive plane (P has no negative element)
+    int p_nk64;
 };
+// What the epilogue does with a finished tile: store it as fp32; or, when the tile is a block of attention
+// logits, reduce it to per-row softmax statistics; or turn it into the AMXFP4 cast of the normalised map.
+constexpr int kEpiStore = 0, kEpiStats = 1, kEpiCast = 2;
 
 // 16 consecutive fp32 results of one row -> global memory, as two 32-byte stores when allowed.
 __device__ __forceinline__ void store_row16(float* out, const float (&f)[16], bool vec, int64_t n_left) {
@@ -197,7 +211,7 @@ __device__ __forceinline__ void store_row16(float* out, const float (&f)[16], bo
     }
 }
 
-template <int BK_>
+template <int BK_, int EPI = kEpiStore>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w, const Params p) {
     using C_ = Cfg<BK_>;
@@ -402,26 +416,91 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueWarps * 32) : "memory");
             if (ok) {
                 const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)col_base;
-                uint32_t v[2][16];
-                tmem_ld16(taddr, v[0]);
+                if constexpr (EPI == kEpiStore) {
+                    uint32_t v[2][16];
+                    tmem_ld16(taddr, v[0]);
 #pragma unroll
-                for (int c = 0; c < BN / 2; c += 16) {
-                    const int buf = (c / 16) & 1;
-                    tmem_ld_wait();
-                    if (c + 16 < BN / 2) tmem_ld16(taddr + c + 16, v[buf ^ 1]);   // next chunk loads while this one is stored
-                    const int col = col_base + c;
-                    float f[16];
+                    for (int c = 0; c < BN / 2; c += 16) {
+                        const int buf = (c / 16) & 1;
+                        tmem_ld_wait();
+                        if (c + 16 < BN / 2) tmem_ld16(taddr + c + 16, v[buf ^ 1]);   // next chunk loads while this one is stored
+                        const int col = col_base + c;
+                        float f[16];
 #pragma unroll
-                    for (int j = 0; j < 16; j += 4) {
-                        const int4 we = *reinterpret_cast<const int4*>(&w_exp[col + j]);
-                        const int ex[4] = {we.x, we.y, we.z, we.w};
+                        for (int j = 0; j < 16; j += 4) {
+                            const int4 we = *reinterpret_cast<const int4*>(&w_exp[col + j]);
+                            const int ex[4] = {we.x, we.y, we.z, we.w};
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int sh = min(127, max(-126, a_exp + ex[i]));
-                            f[j + i] = __uint_as_float(v[buf][j + i]) * __uint_as_float((uint32_t)(sh + 127) << 23);
+                            for (int i = 0; i < 4; ++i) {
+                                const int sh = min(127, max(-126, a_exp + ex[i]));
+                                f[j + i] = __uint_as_float(v[buf][j + i]) * __uint_as_float((uint32_t)(sh + 127) << 23);
+                            }
+                        }
+                        if (m < p.M) store_row16(p.C + m * p.ld_c + n0 + col, f, p.vec_store != 0, p.N - (n0 + col));
+                    }
+                } else {
+                    // The thread's 128 columns come from tensor memory 16 at a time, the next chunk in flight while
+                    // the current one is worked on.  logits: the chunk rescaled and multiplied by alpha.
+                    uint32_t v[2][16];
+                    tmem_ld16(taddr, v[0]);
+                    auto logits16 = [&](int c, float (&f)[16]) {
+                        const int buf = (c / 16) & 1;
+                        tmem_ld_wait();
+                        if (c + 16 < BN / 2) tmem_ld16(taddr + c + 16, v[buf ^ 1]);
+#pragma unroll
+                        for (int j = 0; j < 16; j += 4) {
+                            const int4 we = *reinterpret_cast<const int4*>(&w_exp[col_base + c + j]);
+                            const int ex[4] = {we.x, we.y, we.z, we.w};
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                f[j + i] = __uint_as_float(v[buf][j + i]) * __uint_as_float((uint32_t)(a_exp + ex[i] + 127) << 23) * p.alpha;
+                        }
+                    };
+                    if constexpr (EPI == kEpiStats) {
+                        // One sweep: running maximum, and the sum of exp rescaled whenever the maximum grows.
+                        float mx = -INFINITY, sum = 0.f;
+#pragma unroll
+                        for (int c = 0; c < BN / 2; c += 16) {
+                            float f[16];
+                            logits16(c, f);
+                            float cm = f[0];
+#pragma unroll
+                            for (int j = 1; j < 16; ++j) cm = fmaxf(cm, f[j]);
+                            const float nmx = fmaxf(mx, cm), nm = softmax::neg_max_log2e(nmx);
+                            sum *= softmax::exp_rel(mx, nm);             // exp(-inf) = 0 on the first chunk
+                            mx = nmx;
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) sum += softmax::exp_rel(f[j], nm);
+                        }
+                        if (m < p.M) p.part[m * (2 * n_tiles) + (tile % n_tiles) * 2 + (e >> 2)] = make_float2(mx, sum);
+                    } else {
+                        // Four 32-column groups per thread: normalise with the row's statistics, round to bf16, cast.
+                        const float2 rs = (m < p.M) ? p.rowstat[m] : make_float2(0.f, 0.f);
+                        const int kmax = (m < p.M) ? p.p_kmax[m] : 0;
+                        const int64_t G = p.N / 32, g0 = (n0 + col_base) / 32;
+                        const int64_t sf_row = sf_row_offset(m, p.p_nk64);
+#pragma unroll
+                        for (int gi = 0; gi < BN / 2 / 32; ++gi) {
+                            uint32_t w[16];
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                float f[16];
+                                logits16(gi * 32 + h * 16, f);
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) {
+                                    const __nv_bfloat162 pr = __floats2bfloat162_rn(softmax::exp_rel(f[2 * i], rs.x) * rs.y,
+                                                                                    softmax::exp_rel(f[2 * i + 1], rs.x) * rs.y);
+                                    w[h * 8 + i] = *reinterpret_cast<const uint32_t*>(&pr);
+                                }
+                            }
+                            if (m < p.M) {
+                                const int64_t g = g0 + gi;
+                                const uint32_t sc = cast::emit_group(w, m * G + g, p.p_codes, p.p_scales, p.p_pos, nullptr);
+                                const uint32_t up = to_ue4m3(sc & 0xFFu, kmax);
+                                *reinterpret_cast<uint16_t*>(p.p_sf + sf_row + sf_group_offset((int)g)) = (uint16_t)(up | (up << 8));
+                            }
                         }
                     }
-                    if (m < p.M) store_row16(p.C + m * p.ld_c + n0 + col, f, p.vec_store != 0, p.N - (n0 + col));
                 }
                 // this warp's part of the accumulator has been read: the next tile may overwrite it
                 tc_fence_before();
@@ -512,13 +591,13 @@ size_t gemm_fp4_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 
 namespace {
 
-template <int BK_>
+template <int BK_, int EPI = kEpiStore>
 int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, const OperandLayout& ow, int64_t a_rows,
                int64_t w_rows, Params p, int dev, cudaStream_t st) {
     using C_ = Cfg<BK_>;
     static bool configured[64] = {};
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(gemm_fp4_kernel<BK_>, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(gemm_fp4_kernel<BK_, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::kSmemBytes) != cudaSuccess)
             return AMX_ERR_CUDA;
         configured[dev] = true;
     }
@@ -530,7 +609,7 @@ int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, co
         return AMX_ERR_CUDA;
     const int64_t tiles = ((p.N + BN - 1) / BN) * ((p.M + BM - 1) / BM);
     const unsigned grid = (unsigned)(tiles < sm_count[dev] ? tiles : sm_count[dev]);   // one persistent CTA per SM
-    gemm_fp4_kernel<BK_><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_a, tm_w, p);
+    gemm_fp4_kernel<BK_, EPI><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_a, tm_w, p);
     return launch_status();
 }
 
@@ -545,19 +624,20 @@ int fp4_block_k() {
 
 }  // namespace
 
-// The GEMM proper on two prepared operands (each laid out by operand_layout()), or on row ranges of them.
-int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
-                         int64_t ld_c, void* workspace, cudaStream_t st) {
-    int dev = 0;
+namespace {
+// Kernel parameters for the product of row ranges of two prepared operands.
+int fill_params(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c,
+                void* workspace, cudaStream_t st, Params& p, OperandLayout& oa, OperandLayout& ow, int& dev) {
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AMX_ERR_CUDA;
     if (a.row0 % 128 || w.row0 % 128) return AMX_ERR_SHAPE;
-    const OperandLayout oa = operand_layout(a.layout_rows, K, BM), ow = operand_layout(w.layout_rows, K, BN);
+    oa = operand_layout(a.layout_rows, K, BM);
+    ow = operand_layout(w.layout_rows, K, BN);
     const uint8_t* pa = static_cast<const uint8_t*>(a.prepared);
     const uint8_t* pw = static_cast<const uint8_t*>(w.prepared);
     int* status = static_cast<int*>(workspace);
     if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return AMX_ERR_CUDA;
-    Params p;
-    // scale factors come in chunks per 128 rows, row offsets per row: the range starts at a pointer offset
+    p = Params{};
+    // scale factors come in chunks per 128 rows, row words per row: the range starts at a pointer offset
     const size_t a_sf0 = (size_t)(a.row0 / 128) * oa.nk64 * kSfChunk, w_sf0 = (size_t)(w.row0 / 128) * ow.nk64 * kSfChunk;
     p.sfa_pos = pa + 2 * oa.plane + a_sf0;
     p.sfa_neg = p.sfa_pos + oa.sf;
@@ -567,12 +647,96 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
     p.w_exp = reinterpret_cast<const int*>(pw + 2 * ow.plane + 2 * ow.sf) + w.row0;
     p.M = M; p.N = N; p.K = K; p.ld_c = ld_c; p.C = C;
     p.a_row0 = a.row0; p.w_row0 = w.row0;
-
     p.nk64 = oa.nk64;
-    p.vec_store = aligned(C, 32) && ld_c % 8 == 0;     // 32-byte stores in the epilogue
+    p.vec_store = C && aligned(C, 32) && ld_c % 8 == 0;     // 32-byte stores in the epilogue
     p.status = status;
+    return AMX_OK;
+}
+
+// One warp per query row: the row's softmax statistics from the per-tile partial ones, and the row word of
+// the cast attention map (its largest element is exp(0) / sum, whose group has the row's largest scale).
+__global__ void __launch_bounds__(256)
+attn_row_reduce_kernel(const float2* __restrict__ part, int n_parts, int64_t L, float2* __restrict__ rowstat,
+                       int* __restrict__ p_kmax, int* __restrict__ p_row_word) {
+    const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= L) return;
+    const float2* pr = part + row * n_parts;
+    float mx = -INFINITY;
+    for (int j = lane; j < n_parts; j += 32) mx = fmaxf(mx, pr[j].x);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, d));
+    const float nm = softmax::neg_max_log2e(mx);
+    float sum = 0.f;
+    for (int j = lane; j < n_parts; j += 32) sum += pr[j].y * softmax::exp_rel(pr[j].x, nm);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, d);
+    if (lane) return;
+    const float inv = 1.0f / sum;
+    rowstat[row] = make_float2(nm, inv);
+    const __nv_bfloat16 pmax = __float2bfloat16_rn(softmax::exp_rel(mx, nm) * inv);
+    float inv_p, inv_n;
+    const uint32_t sc = cast::group_scales((uint32_t)__bfloat16_as_ushort(pmax), inv_p, inv_n);   // {nmax = 0 : pmax}
+    const int kmax = scale_key(sc & 0xFFu);
+    p_kmax[row] = kmax;
+    p_row_word[row] = row_word(kmax, side_bits_of(sc));
+}
+}  // namespace
+
+// The GEMM proper on two prepared operands (each laid out by operand_layout()), or on row ranges of them.
+int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
+                         int64_t ld_c, void* workspace, cudaStream_t st) {
+    Params p;
+    OperandLayout oa, ow;
+    int dev;
+    const int rc = fill_params(a, w, M, N, K, C, ld_c, workspace, st, p, oa, ow, dev);
+    if (rc != AMX_OK) return rc;
+    const uint8_t* pa = static_cast<const uint8_t*>(a.prepared);
+    const uint8_t* pw = static_cast<const uint8_t*>(w.prepared);
     return fp4_block_k() == 256 ? launch_fp4<256>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st)
                                 : launch_fp4<128>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
+}
+
+// Attention scores without the logits in memory: P = softmax(alpha * Q K^T) cast to AMXFP4 as the prepared
+// left-hand operand of P V (and its canonical codes and scales).  The product runs twice: the first pass keeps
+// only per-row softmax statistics of each tile, a small kernel merges them, the second pass normalises, rounds
+// to bf16 and casts each tile in the epilogue.  L % 256 == 0.  scratch: fused_attention_scratch_bytes(L).
+size_t gemm_fp4_attn_scratch_bytes(int64_t L) {
+    return up256((size_t)L * (2 * (L / BN)) * sizeof(float2)) + up256((size_t)L * sizeof(float2)) + up256((size_t)L * 4);
+}
+int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, int64_t d, float alpha, void* scratch,
+                         uint8_t* p_codes, uint8_t* p_scales, void* p_prepared, void* workspace, cudaStream_t st) {
+    if (L % BN) return AMX_ERR_SHAPE;
+    Params p;
+    OperandLayout oq, ok_;
+    int dev;
+    int rc = fill_params(q, k, L, L, d, nullptr, L, workspace, st, p, oq, ok_, dev);
+    if (rc != AMX_OK) return rc;
+    const uint8_t* pq = static_cast<const uint8_t*>(q.prepared);
+    const uint8_t* pk = static_cast<const uint8_t*>(k.prepared);
+    const int n_parts = (int)(2 * (L / BN));
+    uint8_t* sc = static_cast<uint8_t*>(scratch);
+    float2* part = reinterpret_cast<float2*>(sc);
+    float2* rowstat = reinterpret_cast<float2*>(sc + up256((size_t)L * n_parts * sizeof(float2)));
+    int* p_kmax = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(rowstat) + up256((size_t)L * sizeof(float2)));
+    const OperandLayout op = operand_layout(L, L, BM);
+    uint8_t* pp = static_cast<uint8_t*>(p_prepared);
+    p.alpha = alpha;
+    p.part = part;
+    p.rowstat = rowstat;
+    p.p_kmax = p_kmax;
+    p.p_codes = reinterpret_cast<uint4*>(p_codes);
+    p.p_scales = reinterpret_cast<uint16_t*>(p_scales);
+    p.p_pos = reinterpret_cast<uint4*>(pp);
+    p.p_sf = pp + 2 * op.plane;
+    p.p_nk64 = op.nk64;
+    rc = launch_fp4<128, kEpiStats>(pq, pk, oq, ok_, q.rows_total, k.rows_total, p, dev, st);
+    if (rc != AMX_OK) return rc;
+    attn_row_reduce_kernel<<<(unsigned)((L + 7) / 8), 256, 0, st>>>(part, n_parts, L, rowstat, p_kmax,
+                                                                        reinterpret_cast<int*>(pp + 2 * op.plane + 2 * op.sf));
+    rc = launch_status();
+    if (rc != AMX_OK) return rc;
+    return launch_fp4<128, kEpiCast>(pq, pk, oq, ok_, q.rows_total, k.rows_total, p, dev, st);
 }
 
 int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K, float* C,

@@ -116,31 +116,6 @@ quantize_cols_kernel(const __nv_bfloat16* __restrict__ x, int64_t R, int64_t C, 
 // Block shape (GX, RB): thread (x, y) owns groups x, x + GX, ... of row blockIdx.x * RB + y.  GX is a multiple
 // of 32, so a warp never spans two rows.
 constexpr int kPrepMaxRows = 8;
-constexpr int kSfChunkBytes = 512;
-
-// One group of an FP4-GEMM operand from its 16 bf16x2 words: canonical codes and scale bytes at group index v,
-// and (pos != nullptr) the two sign planes.  Returns the scale bytes.
-__device__ __forceinline__ uint32_t emit_group(const uint32_t (&w)[16], int64_t v, uint4* __restrict__ codes,
-                                               uint16_t* __restrict__ scales, uint4* __restrict__ pos,
-                                               uint4* __restrict__ neg) {
-    float inv_p, inv_n;
-    const uint32_t sc = group_scales(side_maxima<16>(w), inv_p, inv_n);
-    uint32_t nib[4], pp[4], nn[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        nib[j] = encode8(w + 4 * j, inv_p, inv_n);
-        const uint32_t m = ((nib[j] >> 3) & 0x11111111u) * 15u;   // 0xF on negative nibbles
-        nn[j] = nib[j] & m;
-        pp[j] = nib[j] & ~m;
-    }
-    codes[v] = make_uint4(nib[0], nib[1], nib[2], nib[3]);
-    if (pos) {
-        pos[v] = make_uint4(pp[0], pp[1], pp[2], pp[3]);
-        neg[v] = make_uint4(nn[0], nn[1], nn[2], nn[3]);
-    }
-    scales[v] = (uint16_t)sc;
-    return sc;
-}
 
 // Second half of a prepared cast, for the GX threads (a multiple of 32) that own row `row` (`top`: the largest
 // positive-side scale byte the thread has seen in bits 7..0, the largest negative-side one in bits 15..8;
@@ -161,8 +136,7 @@ __device__ __forceinline__ void finish_prepared_row(int64_t row, bool row_live, 
     __syncthreads();
     const int kmax = slot[0];
     // offset of this row's bytes inside a chunk; the chunks of one block of 128 rows are consecutive along K
-    const int rr = (int)(row & 127);
-    const int64_t sf_row = (row >> 7) * nk64 * (int64_t)kSfChunkBytes + (rr & 31) * 16 + (rr >> 5) * 4;
+    const int64_t sf_row = sf_row_offset(row, nk64);
     const int64_t v_row = row * G;
     for (int g = gx; g < nk64 * 2; g += GX) {      // groups past G: padding to whole 256-element blocks
         uint32_t up = 0, un = 0;
@@ -172,7 +146,7 @@ __device__ __forceinline__ void finish_prepared_row(int64_t row, bool row_live, 
             up = to_ue4m3(sc & 0xFFu, kmax);
             un = to_ue4m3(sc >> 8, kmax);
         }
-        const int64_t off = sf_row + (g >> 1) * kSfChunkBytes + (g & 1) * 2;
+        const int64_t off = sf_row + sf_group_offset(g);
         *reinterpret_cast<uint16_t*>(sf_pos + off) = (uint16_t)(up | (up << 8));
         *reinterpret_cast<uint16_t*>(sf_neg + off) = (uint16_t)(un | (un << 8));
     }
