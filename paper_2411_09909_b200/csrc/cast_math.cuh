@@ -133,5 +133,31 @@ __device__ __forceinline__ uint32_t emit_group(const uint32_t (&w)[16], int64_t 
     return sc;
 }
 
+// The same for a group without negative elements (a softmax output) when only the FP4 GEMM's operand is wanted:
+// its positive sign plane is its code word, the negative plane and scale are zero.  Same arithmetic as above,
+// minus everything the negative side needs.  Stores the plane at group index v, returns the positive scale byte.
+__device__ __forceinline__ uint32_t emit_nonneg_plane(const uint32_t (&w)[16], int64_t v, uint4* __restrict__ plane) {
+    uint32_t pm = w[0];
+#pragma unroll
+    for (int i = 1; i + 1 < 16; i += 2) pm = __vimax3_s16x2(pm, w[i], w[i + 1]);
+    pm = __vmaxs2(pm, w[15]);
+    pm = __vmaxs2(pm, pm >> 16) & 0xFFFFu;                       // the group maximum's bf16 bits
+    const uint32_t sc = cvt_e5m2x2(0.0f, trunc12(__uint_as_float(pm << 16) * sixth_up())) & 0xFFu;
+    const float inv = inv_scale_up(e5m2_to_float(sc));
+    uint32_t nib[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        float r[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            r[2 * i] = trunc12(__uint_as_float(w[4 * j + i] << 16) * inv);
+            r[2 * i + 1] = trunc12(__uint_as_float(w[4 * j + i] & 0xFFFF0000u) * inv);
+        }
+        nib[j] = cvt_e2m1x8(r);
+    }
+    plane[v] = make_uint4(nib[0], nib[1], nib[2], nib[3]);
+    return sc;
+}
+
 }  // namespace cast
 }  // namespace amx

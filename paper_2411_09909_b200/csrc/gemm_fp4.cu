@@ -74,7 +74,7 @@ struct __align__(16) Control {
     uint64_t full[kMaxStages], empty[kMaxStages], accum_full, accum_empty;
     uint32_t tmem_base;
     volatile int abort;
-    alignas(16) int w_exp[2][BN];   // read as int4 in the epilogue
+    alignas(16) int w_exp[2][BN];   // read as int4 in the epilogue (as float4 column factors in the attention modes)
 };
 static_assert(sizeof(Control) <= 2048 + 256, "Control must fit its reserved space");
 
@@ -407,7 +407,11 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t) {
             const int64_t m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
             int* w_exp = ctl->w_exp[t & 1];
-            for (int i = tid_e; i < BN; i += kEpilogueWarps * 32) w_exp[i] = (n0 + i < p.N) ? row_word_exp(p.w_exp[n0 + i]) : 0;
+            for (int i = tid_e; i < BN; i += kEpilogueWarps * 32) {
+                const int ex = (n0 + i < p.N) ? row_word_exp(p.w_exp[n0 + i]) : 0;
+                if constexpr (EPI == kEpiStore) w_exp[i] = ex;
+                else w_exp[i] = __float_as_int(p.alpha * 1.4426950408889634f * __uint_as_float((uint32_t)(ex + 127) << 23));
+            }
             const int64_t m = m0 + q * 32 + lane;
             const int a_exp = (m < p.M) ? row_word_exp(p.a_exp[m]) : 0;
             ok = mbar_wait(&ctl->accum_full, t & 1, &ctl->abort, p.status);
@@ -440,41 +444,51 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                     }
                 } else {
                     // The thread's 128 columns come from tensor memory 16 at a time, the next chunk in flight while
-                    // the current one is worked on.  logits: the chunk rescaled and multiplied by alpha.
+                    // the current one is worked on.  u = accumulator x (alpha log2(e) 2^w_exp[col]) is the logit in
+                    // base-2 units up to the row's power of two ra, by which multiplying is exact: t = u ra.
+                    const float* w_fac = reinterpret_cast<const float*>(w_exp);
+                    const float ra = __uint_as_float((uint32_t)(a_exp + 127) << 23);
                     uint32_t v[2][16];
                     tmem_ld16(taddr, v[0]);
-                    auto logits16 = [&](int c, float (&f)[16]) {
+                    auto chunk16 = [&](int c, float (&u)[16]) {
                         const int buf = (c / 16) & 1;
                         tmem_ld_wait();
                         if (c + 16 < BN / 2) tmem_ld16(taddr + c + 16, v[buf ^ 1]);
 #pragma unroll
                         for (int j = 0; j < 16; j += 4) {
-                            const int4 we = *reinterpret_cast<const int4*>(&w_exp[col_base + c + j]);
-                            const int ex[4] = {we.x, we.y, we.z, we.w};
-#pragma unroll
-                            for (int i = 0; i < 4; ++i)
-                                f[j + i] = __uint_as_float(v[buf][j + i]) * __uint_as_float((uint32_t)(a_exp + ex[i] + 127) << 23) * p.alpha;
+                            const float4 k = *reinterpret_cast<const float4*>(&w_fac[col_base + c + j]);
+                            u[j] = __uint_as_float(v[buf][j]) * k.x;
+                            u[j + 1] = __uint_as_float(v[buf][j + 1]) * k.y;
+                            u[j + 2] = __uint_as_float(v[buf][j + 2]) * k.z;
+                            u[j + 3] = __uint_as_float(v[buf][j + 3]) * k.w;
                         }
                     };
+                    auto exp2_approx = [](float y) {
+                        float r;
+                        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(y));
+                        return r;
+                    };
                     if constexpr (EPI == kEpiStats) {
-                        // One sweep: running maximum, and the sum of exp rescaled whenever the maximum grows.
+                        // One sweep: running maximum (base-2 units), and the sum of 2^(t - max) rescaled whenever the
+                        // maximum grows.
                         float mx = -INFINITY, sum = 0.f;
 #pragma unroll
                         for (int c = 0; c < BN / 2; c += 16) {
-                            float f[16];
-                            logits16(c, f);
-                            float cm = f[0];
+                            float u[16];
+                            chunk16(c, u);
+                            float cm = u[0];
 #pragma unroll
-                            for (int j = 1; j < 16; ++j) cm = fmaxf(cm, f[j]);
-                            const float nmx = fmaxf(mx, cm), nm = softmax::neg_max_log2e(nmx);
-                            sum *= softmax::exp_rel(mx, nm);             // exp(-inf) = 0 on the first chunk
+                            for (int j = 1; j < 16; ++j) cm = fmaxf(cm, u[j]);
+                            const float nmx = fmaxf(mx, cm * ra);
+                            sum *= exp2_approx(mx - nmx);                // 2^(-inf) = 0 on the first chunk
                             mx = nmx;
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) sum += softmax::exp_rel(f[j], nm);
+                            for (int j = 0; j < 16; ++j) sum += exp2_approx(fmaf(u[j], ra, -nmx));
                         }
                         if (m < p.M) p.part[m * (2 * n_tiles) + (tile % n_tiles) * 2 + (e >> 2)] = make_float2(mx, sum);
                     } else {
-                        // Four 32-column groups per thread: normalise with the row's statistics, round to bf16, cast.
+                        // Four 32-column groups per thread: normalise with the row's statistics {-max, 1 / sum}, round
+                        // to bf16, cast.  P has no negative element: only its positive plane and scale factors exist.
                         const float2 rs = (m < p.M) ? p.rowstat[m] : make_float2(0.f, 0.f);
                         const int kmax = (m < p.M) ? p.p_kmax[m] : 0;
                         const int64_t G = p.N / 32, g0 = (n0 + col_base) / 32;
@@ -484,19 +498,18 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                             uint32_t w[16];
 #pragma unroll
                             for (int h = 0; h < 2; ++h) {
-                                float f[16];
-                                logits16(gi * 32 + h * 16, f);
+                                float u[16];
+                                chunk16(gi * 32 + h * 16, u);
 #pragma unroll
                                 for (int i = 0; i < 8; ++i) {
-                                    const __nv_bfloat162 pr = __floats2bfloat162_rn(softmax::exp_rel(f[2 * i], rs.x) * rs.y,
-                                                                                    softmax::exp_rel(f[2 * i + 1], rs.x) * rs.y);
+                                    const __nv_bfloat162 pr = __floats2bfloat162_rn(exp2_approx(fmaf(u[2 * i], ra, rs.x)) * rs.y,
+                                                                                    exp2_approx(fmaf(u[2 * i + 1], ra, rs.x)) * rs.y);
                                     w[h * 8 + i] = *reinterpret_cast<const uint32_t*>(&pr);
                                 }
                             }
                             if (m < p.M) {
                                 const int64_t g = g0 + gi;
-                                const uint32_t sc = cast::emit_group(w, m * G + g, p.p_codes, p.p_scales, p.p_pos, nullptr);
-                                const uint32_t up = to_ue4m3(sc & 0xFFu, kmax);
+                                const uint32_t up = to_ue4m3(cast::emit_nonneg_plane(w, m * G + g, p.p_pos), kmax);
                                 *reinterpret_cast<uint16_t*>(p.p_sf + sf_row + sf_group_offset((int)g)) = (uint16_t)(up | (up << 8));
                             }
                         }
@@ -661,20 +674,20 @@ attn_row_reduce_kernel(const float2* __restrict__ part, int n_parts, int64_t L, 
     const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= L) return;
-    const float2* pr = part + row * n_parts;
+    const float2* pr = part + row * n_parts;          // {max, sum of 2^(t - max)} per half tile, base-2 units
     float mx = -INFINITY;
     for (int j = lane; j < n_parts; j += 32) mx = fmaxf(mx, pr[j].x);
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, d));
-    const float nm = softmax::neg_max_log2e(mx);
     float sum = 0.f;
-    for (int j = lane; j < n_parts; j += 32) sum += pr[j].y * softmax::exp_rel(pr[j].x, nm);
+    for (int j = lane; j < n_parts; j += 32) sum += pr[j].y * exp2f(pr[j].x - mx);
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, d);
     if (lane) return;
     const float inv = 1.0f / sum;
-    rowstat[row] = make_float2(nm, inv);
-    const __nv_bfloat16 pmax = __float2bfloat16_rn(softmax::exp_rel(mx, nm) * inv);
+    rowstat[row] = make_float2(-mx, inv);
+    // the row's largest element is 2^0 / sum
+    const __nv_bfloat16 pmax = __float2bfloat16_rn(inv);
     float inv_p, inv_n;
     const uint32_t sc = cast::group_scales((uint32_t)__bfloat16_as_ushort(pmax), inv_p, inv_n);   // {nmax = 0 : pmax}
     const int kmax = scale_key(sc & 0xFFu);
@@ -725,7 +738,7 @@ int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, in
     p.part = part;
     p.rowstat = rowstat;
     p.p_kmax = p_kmax;
-    p.p_codes = reinterpret_cast<uint4*>(p_codes);
+    p.p_codes = reinterpret_cast<uint4*>(p_codes);      // not written: the prepared operand is all P V needs
     p.p_scales = reinterpret_cast<uint16_t*>(p_scales);
     p.p_pos = reinterpret_cast<uint4*>(pp);
     p.p_sf = pp + 2 * op.plane;
