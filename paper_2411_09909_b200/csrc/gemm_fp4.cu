@@ -476,14 +476,18 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                         for (int c = 0; c < BN / 2; c += 16) {
                             float u[16];
                             chunk16(c, u);
-                            float cm = u[0];
+                            // four chains instead of one: the two epilogue warps of a scheduler are latency-bound
+                            float c4[4] = {u[0], u[1], u[2], u[3]};
 #pragma unroll
-                            for (int j = 1; j < 16; ++j) cm = fmaxf(cm, u[j]);
+                            for (int j = 4; j < 16; ++j) c4[j & 3] = fmaxf(c4[j & 3], u[j]);
+                            const float cm = fmaxf(fmaxf(c4[0], c4[1]), fmaxf(c4[2], c4[3]));
                             const float nmx = fmaxf(mx, cm * ra);
                             sum *= exp2_approx(mx - nmx);                // 2^(-inf) = 0 on the first chunk
                             mx = nmx;
+                            float s4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) sum += exp2_approx(fmaf(u[j], ra, -nmx));
+                            for (int j = 0; j < 16; ++j) s4[j & 3] += exp2_approx(fmaf(u[j], ra, -nmx));
+                            sum += (s4[0] + s4[1]) + (s4[2] + s4[3]);
                         }
                         if (m < p.M) p.part[m * (2 * n_tiles) + (tile % n_tiles) * 2 + (e >> 2)] = make_float2(mx, sum);
                     } else {
