@@ -184,8 +184,11 @@ int amx_softmax_quantize(const float* S, int64_t rows, int64_t cols, int64_t ld_
  * self-attention map and Value are all quantized; Section 1: these are the products rotation methods
  * leave in 16 bits).  Per head h:
  *   S = AMX(Q_h) AMX(K_h)^T          groups along head_dim
- *   P = softmax(S / sqrt(d)) per row, fp32, rounded to bf16; no mask (cast in the same kernel: P itself is
- *       never stored, only its codes and scales)
+ *   P = softmax(S / sqrt(d)) per row, fp32, rounded to bf16; no mask.  P itself is never stored.  When both
+ *       products run on the FP4 kernel and L % 256 == 0, S is not stored either: Q K^T runs twice, the first
+ *       pass keeps per-row softmax statistics, the second normalises and casts each tile in its epilogue
+ *       (row sums are then taken tile by tile, so single elements of P may round to the neighbouring bf16
+ *       value compared with amx_softmax_quantize on a stored S; O agrees to ~1e-5 relative)
  *   O_h = AMX(P) AMX(V_h)            groups along the key axis (V is quantized down its rows)
  *   q, k, v  bf16 [heads, L, d] contiguous;  o  out fp32 [heads, L, d]
  *   d % 32 == 0, L % 32 == 0 (group size 32 on both axes)
