@@ -46,6 +46,7 @@ def lib() -> ctypes.CDLL:
         L.amx_oracle_e5m2_encode.restype = ctypes.c_uint8
         L.amx_oracle_e5m2_encode.argtypes = [dbl]
         L.amx_oracle_quantize.argtypes = [p, i64, i64, i64, ctypes.c_int, p, p]
+        L.amx_oracle_quantize_variant.argtypes = [p, i64, i64, i64, ctypes.c_int, ctypes.c_int, p, p]
         L.amx_oracle_quantize_f64.argtypes = [p, i64, i64, ctypes.c_int, p, p]
         L.amx_oracle_dequantize.argtypes = [p, p, i64, i64, ctypes.c_int, p]
         L.amx_oracle_gemm.argtypes = [p, p, p, p, i64, i64, i64, ctypes.c_int, p, i64, p]
@@ -93,6 +94,22 @@ def quantize(x_bf16_bits: np.ndarray, group_size: int = 32):
     rc = lib().amx_oracle_quantize(_ptr(x), rows, K, K, group_size, _ptr(codes), _ptr(scales))
     if rc:
         raise ValueError(f"amx_oracle_quantize: bad shape (rc={rc})")
+    return codes, scales
+
+
+SYMMETRIC_FP8, MXFP4 = 1, 2
+
+
+def quantize_variant(x_bf16_bits: np.ndarray, group_size: int, mode: int):
+    """The symmetric comparison formats in AMXFP4's storage layout (both scale bytes equal): mode SYMMETRIC_FP8 =
+    one E5M2 scale per group from max|x| / 6; mode MXFP4 = Algorithm 1's power-of-two floor scale."""
+    x = _c(x_bf16_bits, np.uint16)
+    rows, K = x.shape
+    codes = np.zeros((rows, K // 2), np.uint8)
+    scales = np.zeros((rows, K // group_size, 2), np.uint8)
+    rc = lib().amx_oracle_quantize_variant(_ptr(x), rows, K, K, group_size, mode, _ptr(codes), _ptr(scales))
+    if rc != 0:
+        raise ValueError("bad shape, group size or mode")
     return codes, scales
 
 

@@ -201,6 +201,64 @@ int amx_oracle_quantize(const uint16_t *x, int64_t rows, int64_t K, int64_t ld, 
     return 0;
 }
 
+/*
+ * The two symmetric formats the paper compares AMXFP4 with, in the same storage
+ * layout (both scale bytes of a group hold the one shared scale, so the decoder
+ * and the matrix product need no change):
+ *   mode 1  one FP8 E5M2 scale per group, nearest to max|x| / 6 - Section 4.2's
+ *           FP8 shared scale without Section 4.3's split by sign;
+ *   mode 2  MXFP4 - Algorithm 1: shared_exp = floor(log2(max|x|)) - 2 (2 = the
+ *           largest E2M1 exponent), X = 2^shared_exp, elements nearest E2M1 of
+ *           x / X with clamping.  X is stored as the E5M2 byte of the same power
+ *           of two; a shared_exp above 15 is stored as 2^15 and one below -16 as
+ *           a zero scale (Algorithm 1's 8-bit exponent reaches further: a range
+ *           difference only, outside [2^-14, 2^18) group maxima).
+ * Element rounding, sign bit and zero-scale rules are those of the quantizer
+ * above.
+ */
+int amx_oracle_quantize_variant(const uint16_t *x, int64_t rows, int64_t K, int64_t ld, int gs,
+                                int mode, uint8_t *codes, uint8_t *scales)
+{
+    if (gs <= 0 || K % gs != 0 || (K & 1) || (mode != 1 && mode != 2))
+        return -1;
+    int64_t G = K / gs;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t g = 0; g < G; ++g) {
+            const uint16_t *xg = x + r * ld + g * gs;
+            double amax = 0.0;
+            for (int i = 0; i < gs; ++i) {
+                double a = fabs(bf16_to_double(xg[i]));
+                if (a > amax) amax = a;
+            }
+            uint8_t sb;
+            if (mode == 1) {
+                sb = amx_oracle_e5m2_encode(amax / 6.0);
+            } else if (amax > 0.0) {
+                int e;
+                frexp(amax, &e);                       /* amax = f * 2^e, 0.5 <= f < 1 */
+                int shared_exp = (e - 1) - 2;          /* floor(log2(amax)) - emax_elem */
+                if (shared_exp > 15) shared_exp = 15;
+                sb = shared_exp < -16 ? 0 : amx_oracle_e5m2_encode(ldexp(1.0, shared_exp));
+            } else {
+                sb = 0;
+            }
+            double sv = amx_oracle_e5m2_value(sb);
+            for (int i = 0; i < gs; ++i) {
+                int sign = xg[i] >> 15;
+                int mag = sv > 0.0 ? amx_oracle_e2m1_encode(fabs(bf16_to_double(xg[i])) / sv) : 0;
+                uint8_t c = (uint8_t)((sign << 3) | mag);
+                int64_t k = g * gs + i;
+                uint8_t *byte = codes + r * (K / 2) + k / 2;
+                if (k & 1) *byte = (uint8_t)((*byte & 0x0F) | (c << 4));
+                else       *byte = (uint8_t)((*byte & 0xF0) | c);
+            }
+            scales[(r * G + g) * 2 + 0] = sb;
+            scales[(r * G + g) * 2 + 1] = sb;
+        }
+    return 0;
+}
+
 /* Same quantizer on fp64 inputs, one code per byte (used by the pins). */
 int amx_oracle_quantize_f64(const double *x, int64_t rows, int64_t K, int gs,
                             uint8_t *code4, uint8_t *scales)
