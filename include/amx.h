@@ -49,6 +49,14 @@ typedef enum amx_status {
     AMX_ERR_TOO_LARGE = -9   /* the problem needs more scratch than a fixed-capacity entry point holds */
 } amx_status;
 
+/* formats for amx_quantize_fmt / amx_quantize_prepared_fmt.  The two symmetric ones are the formats the
+ * paper compares AMXFP4 with; they are stored in AMXFP4's layout with the one shared scale of a group in both
+ * scale bytes, so every other entry point (dequantize, GEMMs, attention) takes them unchanged. */
+#define AMX_FMT_AMXFP4 0    /* two E5M2 scales per group, selected by the element's sign (Section 4.3) */
+#define AMX_FMT_SYM_FP8 1   /* one E5M2 scale per group, nearest to max|x| / 6 (Section 4.2 without the split) */
+#define AMX_FMT_MXFP4 2     /* Algorithm 1: scale 2^(floor(log2 max|x|) - 2), stored as the E5M2 byte of that power
+                             * of two; exponents above 15 are stored as 2^15, below -16 as a zero scale */
+
 /* flags for amx_dequantize: output element type (default bf16) */
 #define AMX_OUT_BF16 0x0u
 #define AMX_OUT_F32 0x1u
@@ -85,6 +93,10 @@ typedef enum amx_status {
  */
 int amx_quantize(const void* x, int64_t rows, int64_t K, int64_t ld_x, int group_size,
                  uint8_t* codes, uint8_t* scales, void* stream);
+/* amx_quantize for one of the AMX_FMT_* formats (AMX_ERR_FLAGS for an unknown one); AMX_FMT_AMXFP4 is
+ * amx_quantize itself.  Element rounding, sign bit and zero-scale rules are the same for all formats. */
+int amx_quantize_fmt(const void* x, int64_t rows, int64_t K, int64_t ld_x, int group_size, int format,
+                     uint8_t* codes, uint8_t* scales, void* stream);
 
 /*
  * amx_quantize_t - the same cast with the groups running DOWN the rows of x (the strided axis):
@@ -137,6 +149,12 @@ int amx_gemm(const uint8_t* a_codes, const uint8_t* a_scales,
  */
 int amx_quantize_prepared(const void* x, int64_t rows, int64_t K, int group_size, int is_weight,
                           uint8_t* codes, uint8_t* scales, void* prepared, size_t prepared_bytes, void* stream);
+/* The same for one of the AMX_FMT_* formats.  A symmetric format needs no split by sign: its prepared form
+ * holds the signed codes as one plane, and amx_gemm_prepared issues one product per tile pair instead of four
+ * (amx_prepare and amx_gemm detect operand rows whose two scales agree in every group and do the same). */
+int amx_quantize_prepared_fmt(const void* x, int64_t rows, int64_t K, int group_size, int is_weight, int format,
+                              uint8_t* codes, uint8_t* scales, void* prepared, size_t prepared_bytes,
+                              void* stream);
 size_t amx_prepared_bytes(int64_t rows, int64_t K, int group_size, int is_weight);
 int amx_prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, int group_size,
                 int is_weight, void* prepared, size_t prepared_bytes, void* stream);

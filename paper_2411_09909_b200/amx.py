@@ -18,6 +18,7 @@ _lib = None
 OUT_BF16, OUT_F32 = 0x0, 0x1
 GEMM_AUTO, GEMM_SIMT, GEMM_TC, GEMM_FP4 = 0x0, 0x10, 0x20, 0x40
 GEMM_CAST_IN_KERNEL = 0x80      # amx_quant_gemm only, together with GEMM_TC
+FMT_AMXFP4, FMT_SYM_FP8, FMT_MXFP4 = 0, 1, 2
 
 # every symbol include/amx.h declares
 SYMBOLS = (
@@ -28,6 +29,7 @@ SYMBOLS = (
     "amx_quant_gemm_static", "amx_quant_gemm_static_capacity",
     "amx_attention", "amx_attention_workspace_bytes",
     "amx_prepared_bytes", "amx_prepare", "amx_gemm_prepared", "amx_quantize_prepared", "amx_softmax_quantize",
+    "amx_quantize_fmt", "amx_quantize_prepared_fmt",
 )
 
 
@@ -44,6 +46,8 @@ def lib() -> ctypes.CDLL:
         i64, p, i, u32, sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_uint32, ctypes.c_size_t
         L.amx_quantize.argtypes = [p, i64, i64, i64, i, p, p, p]
         L.amx_quantize_t.argtypes = [p, i64, i64, i64, i, p, p, p]
+        L.amx_quantize_fmt.argtypes = [p, i64, i64, i64, i, i, p, p, p]
+        L.amx_quantize_prepared_fmt.argtypes = [p, i64, i64, i, i, i, p, p, p, sz, p]
         L.amx_dequantize.argtypes = [p, p, i64, i64, i, u32, p, i64, p]
         L.amx_gemm.argtypes = [p, p, p, p, i64, i64, i64, i, u32, p, i64, p, sz, p]
         L.amx_quant_gemm.argtypes = [p, i64, p, p, i64, i64, i64, i, u32, p, i64, p, sz, p]
@@ -98,15 +102,20 @@ def _ws(nbytes: int, device) -> torch.Tensor:
     return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
 
 
-def quantize(x: torch.Tensor, group_size: int = 32):
+def quantize(x: torch.Tensor, group_size: int = 32, fmt: int = FMT_AMXFP4):
     """bf16 [rows, K] (row stride allowed) -> (codes u8 [rows, K/2], scales u8 [rows, K/gs, 2])."""
     _dev(x, torch.bfloat16, "x")
     assert x.dim() == 2 and x.stride(1) == 1
     rows, K = x.shape
     codes = torch.empty((rows, K // 2), dtype=torch.uint8, device=x.device)
     scales = torch.empty((rows, max(K // group_size, 0), 2), dtype=torch.uint8, device=x.device)
-    _check(lib().amx_quantize(x.data_ptr(), rows, K, x.stride(0) if rows > 1 else max(K, x.stride(0)),
-                              group_size, codes.data_ptr(), scales.data_ptr(), _stream()), "amx_quantize")
+    ld = x.stride(0) if rows > 1 else max(K, x.stride(0))
+    if fmt == FMT_AMXFP4:
+        _check(lib().amx_quantize(x.data_ptr(), rows, K, ld, group_size, codes.data_ptr(), scales.data_ptr(), _stream()),
+               "amx_quantize")
+    else:
+        _check(lib().amx_quantize_fmt(x.data_ptr(), rows, K, ld, group_size, fmt, codes.data_ptr(), scales.data_ptr(),
+                                      _stream()), "amx_quantize_fmt")
     return codes, scales
 
 
@@ -162,7 +171,8 @@ def prepare(codes: torch.Tensor, scales: torch.Tensor, is_weight: bool, group_si
     return buf
 
 
-def quantize_prepared(x: torch.Tensor, is_weight: bool, group_size: int = 32, prepared: torch.Tensor | None = None):
+def quantize_prepared(x: torch.Tensor, is_weight: bool, group_size: int = 32, prepared: torch.Tensor | None = None,
+                      fmt: int = FMT_AMXFP4):
     """Cast and prepare in one go: returns (codes, scales, prepared)."""
     _dev(x, torch.bfloat16, "x")
     assert x.is_contiguous()
@@ -170,8 +180,13 @@ def quantize_prepared(x: torch.Tensor, is_weight: bool, group_size: int = 32, pr
     codes = torch.empty((rows, K // 2), dtype=torch.uint8, device=x.device)
     scales = torch.empty((rows, K // group_size, 2), dtype=torch.uint8, device=x.device)
     buf = prepared if prepared is not None else _ws(lib().amx_prepared_bytes(rows, K, group_size, int(is_weight)), x.device)
-    _check(lib().amx_quantize_prepared(x.data_ptr(), rows, K, group_size, int(is_weight), codes.data_ptr(),
-                                       scales.data_ptr(), buf.data_ptr(), buf.numel(), _stream()), "amx_quantize_prepared")
+    if fmt == FMT_AMXFP4:
+        _check(lib().amx_quantize_prepared(x.data_ptr(), rows, K, group_size, int(is_weight), codes.data_ptr(),
+                                           scales.data_ptr(), buf.data_ptr(), buf.numel(), _stream()), "amx_quantize_prepared")
+    else:
+        _check(lib().amx_quantize_prepared_fmt(x.data_ptr(), rows, K, group_size, int(is_weight), fmt, codes.data_ptr(),
+                                               scales.data_ptr(), buf.data_ptr(), buf.numel(), _stream()),
+               "amx_quantize_prepared_fmt")
     return codes, scales, buf
 
 

@@ -114,11 +114,20 @@ extern "C" int amx_prepare(const uint8_t* codes, const uint8_t* scales, int64_t 
 extern "C" int amx_quantize_prepared(const void* x, int64_t rows, int64_t K, int group_size, int is_weight,
                                      uint8_t* codes, uint8_t* scales, void* prepared, size_t prepared_bytes,
                                      void* stream) {
+    return amx_quantize_prepared_fmt(x, rows, K, group_size, is_weight, AMX_FMT_AMXFP4, codes, scales, prepared,
+                                     prepared_bytes, stream);
+}
+
+extern "C" int amx_quantize_prepared_fmt(const void* x, int64_t rows, int64_t K, int group_size, int is_weight,
+                                         int format, uint8_t* codes, uint8_t* scales, void* prepared,
+                                         size_t prepared_bytes, void* stream) {
+    if (format != AMX_FMT_AMXFP4 && format != AMX_FMT_SYM_FP8 && format != AMX_FMT_MXFP4) return AMX_ERR_FLAGS;
     if (rows <= 0 || !gemm_fp4_supported(rows, rows, K, group_size)) return AMX_ERR_SHAPE;
     if (!x || !codes || !scales || !prepared) return AMX_ERR_NULL;
     if (prepared_bytes < amx_prepared_bytes(rows, K, group_size, is_weight)) return AMX_ERR_WORKSPACE;
     if (!aligned(x, 16) || !aligned(codes, 16) || !aligned(scales, 2) || !aligned(prepared, kAlign)) return AMX_ERR_ALIGN;
-    return gemm_fp4_quantize_prepared(x, rows, K, is_weight != 0, codes, scales, prepared, static_cast<cudaStream_t>(stream));
+    return gemm_fp4_quantize_prepared(x, rows, K, is_weight != 0, codes, scales, prepared, static_cast<cudaStream_t>(stream),
+                                      0, format);
 }
 
 extern "C" int amx_gemm_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,

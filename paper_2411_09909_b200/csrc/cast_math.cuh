@@ -90,6 +90,28 @@ __device__ __forceinline__ uint32_t group_scales(uint32_t c, float& inv_p, float
     return sc;
 }
 
+// The same for the symmetric comparison formats, which store their one shared scale in both bytes
+// (FMT: AMX_FMT_AMXFP4 = 0, AMX_FMT_SYM_FP8 = 1, AMX_FMT_MXFP4 = 2):
+//   SYM_FP8  the scale of the larger side maximum, used by both sides;
+//   MXFP4    Algorithm 1: X = 2^(floor(log2 max|x|) - 2), from the exponent field E of the maximum's bf16
+//            pattern: X's E5M2 exponent field is E - 127 - 2 + 15 = E - 114; fields 0 and -1 are the
+//            subnormals 2^-15 (byte 2) and 2^-16 (byte 1), smaller ones store a zero scale, larger than 30
+//            store 2^15.
+template <int FMT>
+__device__ __forceinline__ uint32_t group_scales_fmt(uint32_t c, float& inv_p, float& inv_n) {
+    if (FMT == 0) return group_scales(c, inv_p, inv_n);
+    const uint32_t amax = max(c & 0xFFFFu, c >> 16);              // both halves are non-negative bf16 patterns
+    uint32_t b;
+    if (FMT == 1) {
+        b = cvt_e5m2x2(0.0f, trunc12(__uint_as_float(amax << 16) * sixth_up())) & 0xFFu;
+    } else {
+        const int e5 = (int)(amax >> 7) - 114;
+        b = e5 > 30 ? 0x78u : e5 >= 1 ? (uint32_t)e5 << 2 : e5 == 0 ? 2u : e5 == -1 ? 1u : 0u;
+    }
+    inv_p = inv_n = inv_scale_up(e5m2_to_float(b));
+    return b | (b << 8);
+}
+
 // x * (sign(x) ? inv_n : inv_p).  The choice is an integer multiply-add on the reciprocals' bit
 // patterns (inv_p + sign * (inv_n - inv_p)): it runs on the FMA pipe, which this kernel leaves
 // mostly idle, instead of adding a compare and a select to the saturated integer/logic pipe.
@@ -113,16 +135,19 @@ __device__ __forceinline__ uint32_t encode8(const uint32_t* w, float inv_p, floa
 
 // One group of an FP4-GEMM operand from its 16 bf16x2 words: canonical codes and scale bytes at group index v,
 // and the sign planes that are asked for (pos / neg may be nullptr).  Returns the scale bytes {neg : pos}.
+// With a symmetric format (FMT != 0) the operand needs no split: the signed codes go to the "positive" plane
+// as they are, the other plane is zero, and the returned bytes name the one scale as the positive side's only.
+template <int FMT = 0>
 __device__ __forceinline__ uint32_t emit_group(const uint32_t (&w)[16], int64_t v, uint4* __restrict__ codes,
                                                uint16_t* __restrict__ scales, uint4* __restrict__ pos,
                                                uint4* __restrict__ neg) {
     float inv_p, inv_n;
-    const uint32_t sc = group_scales(side_maxima<16>(w), inv_p, inv_n);
+    const uint32_t sc = group_scales_fmt<FMT>(side_maxima<16>(w), inv_p, inv_n);
     uint32_t nib[4], pp[4], nn[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         nib[j] = encode8(w + 4 * j, inv_p, inv_n);
-        const uint32_t m = ((nib[j] >> 3) & 0x11111111u) * 15u;   // 0xF on negative nibbles
+        const uint32_t m = FMT ? 0u : ((nib[j] >> 3) & 0x11111111u) * 15u;   // 0xF on negative nibbles
         nn[j] = nib[j] & m;
         pp[j] = nib[j] & ~m;
     }
@@ -130,7 +155,7 @@ __device__ __forceinline__ uint32_t emit_group(const uint32_t (&w)[16], int64_t 
     if (pos) pos[v] = make_uint4(pp[0], pp[1], pp[2], pp[3]);
     if (neg) neg[v] = make_uint4(nn[0], nn[1], nn[2], nn[3]);
     scales[v] = (uint16_t)sc;
-    return sc;
+    return FMT ? (sc & 0xFFu) : sc;
 }
 
 // The same for a group without negative elements (a softmax output) when only the FP4 GEMM's operand is wanted:

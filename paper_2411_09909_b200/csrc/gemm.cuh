@@ -32,10 +32,11 @@ size_t gemm_fp4_prepared_bytes(int64_t rows, int64_t K, bool is_weight);
 int gemm_fp4_prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, bool is_weight,
                      void* prepared, cudaStream_t st, int64_t layout_rows = 0 /* 0: rows */);
 int gemm_fp4_quantize_prepared(const void* x, int64_t rows, int64_t K, bool is_weight, uint8_t* codes,
-                               uint8_t* scales, void* prepared, cudaStream_t st, int64_t layout_rows = 0);
+                               uint8_t* scales, void* prepared, cudaStream_t st, int64_t layout_rows = 0,
+                               int format = AMX_FMT_AMXFP4);
 int quantize_rows_prepared(const void* x, int64_t rows, int64_t K, uint8_t* codes, uint8_t* scales, void* pos,
                            void* neg, uint8_t* sf_pos, uint8_t* sf_neg, int* row_exp, int nk64, int64_t padded_rows,
-                           cudaStream_t st);
+                           cudaStream_t st, int format = AMX_FMT_AMXFP4);
 // Softmax of the rows of S, rounded to bf16 and cast in one launch (cols % 32 == 0); pos == nullptr: canonical
 // output only.  gemm_fp4_softmax_prepared lays the prepared operand out like gemm_fp4_quantize_prepared.
 int softmax_cast_rows(const float* S, int64_t rows, int64_t cols, int64_t ld_s, float alpha, uint8_t* codes,

@@ -106,27 +106,37 @@ prepare_operand_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restr
                        int nk64, uint4* __restrict__ pos, uint4* __restrict__ neg, uint8_t* __restrict__ sf_pos,
                        uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp) {
     __shared__ int kmax_s[kPrepRows];
+    __shared__ int unsplit_s[kPrepRows];
     const int64_t row0 = (int64_t)blockIdx.x * kPrepRows, G = K / 32;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int r = warp; r < kPrepRows; r += 8) {
         const int64_t row = row0 + r;
         int kmax = 0, sides = 0;
+        uint32_t differ = 0;
         if (row < R) {
             const unsigned short* s2 = reinterpret_cast<const unsigned short*>(scales + row * G * 2);
             for (int64_t g = lane; g < G; g += 32) {
                 const uint32_t v = __ldg(s2 + g);
                 kmax = max(kmax, max(scale_key(v & 0xFF), scale_key(v >> 8)));
                 sides |= side_bits_of(v);
+                differ |= (v & 0xFF) ^ (v >> 8);
             }
         }
         kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
         sides = __reduce_or_sync(0xFFFFFFFFu, sides);
+        differ = __reduce_or_sync(0xFFFFFFFFu, differ);
+        // A row whose two scales agree in every group (a symmetric format) needs no split: sum over both signs of
+        // code x scale_side = code x scale.  Its signed codes go to the positive plane as they are.
+        const bool unsplit = !differ;
+        if (unsplit) sides &= kRowHasPos;
         if (lane == 0) {
             kmax_s[r] = kmax;
+            unsplit_s[r] = unsplit;
             if (row < R) row_exp[row] = row_word(kmax, sides);
         }
     }
     // sign planes of this block's rows (contiguous in memory: rows are K/2 bytes apart)
+    __syncthreads();                                             // unsplit_s is complete
     const int64_t rows_here = min((int64_t)kPrepRows, R - row0);
     if (rows_here > 0) {
         const int64_t v0 = row0 * (K / 32), n_vec = rows_here * (K / 32);
@@ -134,10 +144,11 @@ prepare_operand_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restr
         for (int64_t i = threadIdx.x; i < n_vec; i += 256) {
             const uint4 w = __ldg(src + i);
             const uint32_t v[4] = {w.x, w.y, w.z, w.w};
+            const uint32_t keep = unsplit_s[i / G] ? 0u : 0xFFFFFFFFu;
             uint32_t p[4], n[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const uint32_t m = ((v[j] >> 3) & 0x11111111u) * 15u;   // 0xF on negative nibbles
+                const uint32_t m = ((v[j] >> 3) & 0x11111111u) * 15u & keep;   // 0xF on negative nibbles
                 n[j] = v[j] & m;
                 p[j] = v[j] & ~m;
             }
@@ -160,7 +171,7 @@ prepare_operand_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restr
                 const int64_t g = (int64_t)c * 2 + h;
                 if (g < G) {
                     const uint32_t v = __ldg(reinterpret_cast<const unsigned short*>(scales + (row * G + g) * 2));
-                    const uint32_t up = to_ue4m3(v & 0xFF, kmax), un = to_ue4m3(v >> 8, kmax);
+                    const uint32_t up = to_ue4m3(v & 0xFF, kmax), un = unsplit_s[r] ? 0u : to_ue4m3(v >> 8, kmax);
                     wp |= (up | (up << 8)) << (16 * h);
                     wn |= (un | (un << 8)) << (16 * h);
                 }
@@ -768,12 +779,12 @@ size_t gemm_fp4_prepared_bytes(int64_t rows, int64_t K, bool is_weight) {
 
 // Fused form: one launch of the cast kernel writes the canonical operand and the prepared one.
 int gemm_fp4_quantize_prepared(const void* x, int64_t rows, int64_t K, bool is_weight, uint8_t* codes, uint8_t* scales,
-                               void* prepared, cudaStream_t st, int64_t layout_rows) {
+                               void* prepared, cudaStream_t st, int64_t layout_rows, int format) {
     const OperandLayout o = operand_layout(layout_rows ? layout_rows : rows, K, is_weight ? BN : BM);
     uint8_t* base = static_cast<uint8_t*>(prepared);
     return quantize_rows_prepared(x, rows, K, codes, scales, base, base + o.plane, base + 2 * o.plane,
                                   base + 2 * o.plane + o.sf, reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf), o.nk64,
-                                  o.row_blocks * 128, st);
+                                  o.row_blocks * 128, st, format);
 }
 
 int gemm_fp4_softmax_prepared(const float* S, int64_t rows, int64_t cols, int64_t ld_s, float alpha, bool is_weight,

@@ -29,7 +29,7 @@ __device__ __forceinline__ uint32_t quantize8(const uint4 q, uint32_t& sc) {
 // Groups along the contiguous axis.  Each thread owns EPT = min(gs, 32) consecutive elements
 // (EPT/8 16-byte loads, one EPT/2-byte store); a group is TPG = gs / EPT consecutive lanes, so a
 // 16- or 32-group needs no shuffle and its scales are computed once.  n_items = rows * K / EPT.
-template <int EPT, int TPG, bool CONTIG>
+template <int EPT, int TPG, bool CONTIG, int FMT = 0>
 __global__ void __launch_bounds__(kThreads)
 quantize_rows_kernel(const uint4* __restrict__ x, int64_t n_items, int64_t items_per_row,
                      int64_t ld_vec, uint4* __restrict__ codes, uint16_t* __restrict__ scales) {
@@ -51,7 +51,7 @@ quantize_rows_kernel(const uint4* __restrict__ x, int64_t n_items, int64_t items
 #pragma unroll
     for (int d = 1; d < TPG; d <<= 1) c = __vmaxs2(c, __shfl_xor_sync(0xFFFFFFFFu, c, d));
     float inv_p, inv_n;
-    const uint32_t sc = group_scales(c, inv_p, inv_n);
+    const uint32_t sc = group_scales_fmt<FMT>(c, inv_p, inv_n);
     uint32_t nib[NV];
 #pragma unroll
     for (int j = 0; j < NV; ++j) nib[j] = encode8(w + 4 * j, inv_p, inv_n);
@@ -154,6 +154,7 @@ __device__ __forceinline__ void finish_prepared_row(int64_t row, bool row_live, 
 }
 
 // 40 registers (three blocks of 512 per SM): at 32 the kernel spills and is 12 % slower.
+template <int FMT>
 __global__ void __launch_bounds__(512, 3)
 cast_prepared_kernel(const uint4* __restrict__ x, int64_t R, int G, uint4* __restrict__ codes,
                      uint16_t* __restrict__ scales, uint4* __restrict__ pos, uint4* __restrict__ neg,
@@ -176,7 +177,7 @@ cast_prepared_kernel(const uint4* __restrict__ x, int64_t R, int G, uint4* __res
             const uint4 q = __ldg(x + v * 4 + j);
             w[4 * j] = q.x; w[4 * j + 1] = q.y; w[4 * j + 2] = q.z; w[4 * j + 3] = q.w;
         }
-        const uint32_t sc = emit_group(w, v, codes, scales, pos, neg);
+        const uint32_t sc = emit_group<FMT>(w, v, codes, scales, pos, neg);
         if (g == gx) sc_first = sc;
         top = __vmaxu4(top, sc);                // byte-wise maximum
     }
@@ -232,7 +233,7 @@ softmax_cast_kernel(const float* __restrict__ S, int64_t R, int G, int64_t ld_s,
     finish_prepared_row(row, row_live, G, gx, softmax::kT, top, sc_first, scales, slot_s, sf_pos, sf_neg, row_exp, nk64);
 }
 
-template <int EPT, int TPG>
+template <int EPT, int TPG, int FMT = 0>
 int launch_rows(const void* x, int64_t rows, int64_t K, int64_t ld, uint8_t* codes,
                 uint8_t* scales, cudaStream_t st) {
     const int64_t n_items = rows * (K / EPT);
@@ -242,9 +243,9 @@ int launch_rows(const void* x, int64_t rows, int64_t K, int64_t ld, uint8_t* cod
     auto* cv = reinterpret_cast<uint4*>(codes);
     auto* sv = reinterpret_cast<uint16_t*>(scales);
     if (ld == K)
-        quantize_rows_kernel<EPT, TPG, true><<<(unsigned)blocks, kThreads, 0, st>>>(xv, n_items, K / EPT, ld / 8, cv, sv);
+        quantize_rows_kernel<EPT, TPG, true, FMT><<<(unsigned)blocks, kThreads, 0, st>>>(xv, n_items, K / EPT, ld / 8, cv, sv);
     else
-        quantize_rows_kernel<EPT, TPG, false><<<(unsigned)blocks, kThreads, 0, st>>>(xv, n_items, K / EPT, ld / 8, cv, sv);
+        quantize_rows_kernel<EPT, TPG, false, FMT><<<(unsigned)blocks, kThreads, 0, st>>>(xv, n_items, K / EPT, ld / 8, cv, sv);
     return launch_status();
 }
 
@@ -255,7 +256,7 @@ int launch_rows(const void* x, int64_t rows, int64_t K, int64_t ld, uint8_t* cod
 // chunks of 512 B per block of 128 rows, rows padded to padded_rows) and the rows' power-of-two offsets.
 int quantize_rows_prepared(const void* x, int64_t rows, int64_t K, uint8_t* codes, uint8_t* scales, void* pos,
                            void* neg, uint8_t* sf_pos, uint8_t* sf_neg, int* row_exp, int nk64, int64_t padded_rows,
-                           cudaStream_t st) {
+                           cudaStream_t st, int format) {
     const int64_t G = K / 32;
     // one thread per group when a row fits a block of 512, several rows per block when rows are short
     const int gx = (int)((G < 512 ? G : 512) + 31) / 32 * 32;
@@ -263,7 +264,9 @@ int quantize_rows_prepared(const void* x, int64_t rows, int64_t K, uint8_t* code
     while (rb < kPrepMaxRows && rb * 2 * gx <= 256) rb *= 2;
     const int64_t blocks = (padded_rows + rb - 1) / rb;
     if (blocks > 0x7FFFFFFF) return AMX_ERR_SHAPE;
-    cast_prepared_kernel<<<(unsigned)blocks, dim3(gx, rb), 0, st>>>(
+    auto* kernel = format == AMX_FMT_SYM_FP8 ? cast_prepared_kernel<1> : format == AMX_FMT_MXFP4 ? cast_prepared_kernel<2>
+                                                                                                  : cast_prepared_kernel<0>;
+    kernel<<<(unsigned)blocks, dim3(gx, rb), 0, st>>>(
         reinterpret_cast<const uint4*>(x), rows, (int)G, reinterpret_cast<uint4*>(codes),
         reinterpret_cast<uint16_t*>(scales), reinterpret_cast<uint4*>(pos), reinterpret_cast<uint4*>(neg), sf_pos, sf_neg,
         row_exp, nk64);
@@ -309,21 +312,39 @@ int quantize_cols_batched(const void* x, int64_t batch, int64_t R, int64_t C, ui
 
 }  // namespace amx
 
+namespace amx {
+namespace {
+template <int FMT>
+int launch_rows_gs(const void* x, int64_t rows, int64_t K, int64_t ld_x, int group_size, uint8_t* codes, uint8_t* scales,
+                   cudaStream_t st) {
+    switch (group_size) {
+        case 16: return launch_rows<16, 1, FMT>(x, rows, K, ld_x, codes, scales, st);
+        case 32: return launch_rows<32, 1, FMT>(x, rows, K, ld_x, codes, scales, st);
+        case 64: return launch_rows<32, 2, FMT>(x, rows, K, ld_x, codes, scales, st);
+        default: return launch_rows<32, 4, FMT>(x, rows, K, ld_x, codes, scales, st);
+    }
+}
+}  // namespace
+}  // namespace amx
+
 extern "C" int amx_quantize(const void* x, int64_t rows, int64_t K, int64_t ld_x, int group_size,
                             uint8_t* codes, uint8_t* scales, void* stream) {
+    return amx_quantize_fmt(x, rows, K, ld_x, group_size, AMX_FMT_AMXFP4, codes, scales, stream);
+}
+
+extern "C" int amx_quantize_fmt(const void* x, int64_t rows, int64_t K, int64_t ld_x, int group_size, int format,
+                                uint8_t* codes, uint8_t* scales, void* stream) {
     using namespace amx;
+    if (format != AMX_FMT_AMXFP4 && format != AMX_FMT_SYM_FP8 && format != AMX_FMT_MXFP4) return AMX_ERR_FLAGS;
     if (!valid_group_size(group_size) || rows < 0 || K <= 0 || K % group_size || K % 8 || ld_x < K)
         return AMX_ERR_SHAPE;
     if (rows == 0) return AMX_OK;
     if (!x || !codes || !scales) return AMX_ERR_NULL;
     if (!aligned(x, 16) || ld_x % 8 || !aligned(codes, group_size == 16 ? 8 : 16) || !aligned(scales, 2)) return AMX_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    switch (group_size) {
-        case 16: return launch_rows<16, 1>(x, rows, K, ld_x, codes, scales, st);
-        case 32: return launch_rows<32, 1>(x, rows, K, ld_x, codes, scales, st);
-        case 64: return launch_rows<32, 2>(x, rows, K, ld_x, codes, scales, st);
-        default: return launch_rows<32, 4>(x, rows, K, ld_x, codes, scales, st);
-    }
+    if (format == AMX_FMT_SYM_FP8) return launch_rows_gs<1>(x, rows, K, ld_x, group_size, codes, scales, st);
+    if (format == AMX_FMT_MXFP4) return launch_rows_gs<2>(x, rows, K, ld_x, group_size, codes, scales, st);
+    return launch_rows_gs<0>(x, rows, K, ld_x, group_size, codes, scales, st);
 }
 
 extern "C" int amx_quantize_t(const void* x, int64_t R, int64_t C, int64_t ld_x, int group_size,

@@ -233,6 +233,53 @@ def test_gemm_fp4_one_sided_operands(a_side, w_side):
     assert rel_fro(amx.gemm_prepared(pa, pw, 300, 520, 1056).cpu().numpy(), ref) <= GEMM_TOL
 
 
+@pytest.mark.parametrize("fmt,mode", [(amx.FMT_SYM_FP8, oracle.SYMMETRIC_FP8), (amx.FMT_MXFP4, oracle.MXFP4)])
+def test_symmetric_formats(fmt, mode):
+    """The paper's symmetric comparison formats: codes and scales bit-exact against the oracle for every group
+    size, on fuzz rows (ties, tiny, huge, one-sided and all-zero groups); the GEMMs take them unchanged; the FP4
+    kernel needs one product per tile pair for them, from the fused cast and from amx_prepare alike."""
+    for gs in (16, 32, 64, 128):
+        for kind in ("mixed", "wide"):
+            bits = inputs.random_groups(300 + gs, 96, 512, kind)
+            c, s_ = amx.quantize(dev_bf16(bits), gs, fmt=fmt)
+            oc, os_ = oracle.quantize_variant(bits, gs, mode)
+            assert np.array_equal(c.cpu().numpy(), oc) and np.array_equal(s_.cpu().numpy(), os_), (gs, kind)
+    # every bf16 value as a group maximum, and every bf16 value against a fixed maximum
+    allv = np.arange(0x7F80, dtype=np.uint16)
+    bits = np.zeros((allv.size, 32), np.uint16)
+    bits[:, 0] = allv
+    bits[:, 1] = allv | 0x8000
+    bits[:, 2] = 0x3F80
+    c, s_ = amx.quantize(dev_bf16(bits), 32, fmt=fmt)
+    oc, os_ = oracle.quantize_variant(bits, 32, mode)
+    assert np.array_equal(c.cpu().numpy(), oc) and np.array_equal(s_.cpu().numpy(), os_)
+    bits = np.full((allv.size, 32), 0x0000, np.uint16)
+    bits[:, 0] = 0x4416                                     # 600.0: the scale is fixed, every value is an element
+    bits[:, 1] = allv
+    bits[:, 2] = allv | 0x8000
+    c, s_ = amx.quantize(dev_bf16(bits), 32, fmt=fmt)
+    oc, os_ = oracle.quantize_variant(bits, 32, mode)
+    assert np.array_equal(c.cpu().numpy(), oc) and np.array_equal(s_.cpu().numpy(), os_)
+    # products
+    a_bits = inputs.random_groups(311, 300, 1056, "normal")
+    w_bits = inputs.random_groups(312, 520, 1056, "normal")
+    qa, qw = oracle.quantize_variant(a_bits, 32, mode), oracle.quantize_variant(w_bits, 32, mode)
+    ref = oracle.gemm(*qa, *qw, 32)
+    ac, as_ = amx.quantize(dev_bf16(a_bits), 32, fmt=fmt)
+    wc, ws = amx.quantize(dev_bf16(w_bits), 32, fmt=fmt)
+    for flags in (amx.GEMM_SIMT, amx.GEMM_TC, amx.GEMM_FP4):
+        assert rel_fro(amx.gemm(ac, as_, wc, ws, 32, flags).cpu().numpy(), ref) <= GEMM_TOL, flags
+    c2, s2, pa = amx.quantize_prepared(dev_bf16(a_bits), False, fmt=fmt)
+    _, _, pw = amx.quantize_prepared(dev_bf16(w_bits), True, fmt=fmt)
+    assert torch.equal(c2, ac) and torch.equal(s2, as_)
+    got = amx.gemm_prepared(pa, pw, 300, 520, 1056)
+    assert rel_fro(got.cpu().numpy(), ref) <= GEMM_TOL
+    # a symmetric operand against an asymmetric one
+    wq = oracle.quantize(w_bits, 32)
+    pw_amx = amx.prepare(*(torch.from_numpy(t).cuda() for t in wq), True)
+    assert rel_fro(amx.gemm_prepared(pa, pw_amx, 300, 520, 1056).cpu().numpy(), oracle.gemm(*qa, *wq, 32)) <= GEMM_TOL
+
+
 def test_quantize_prepared_equals_quantize_then_prepare():
     # row lengths below, at and above one block of the cast kernel (several rows, one row and a fraction of a
     # row per block; threads striding over a long row), ragged row counts, both paddings
