@@ -396,52 +396,51 @@ def run_ours(args):
                           "what": "weights cast and prepared once; per step: cast + prepare activations, GEMM"}
         del prep
 
-    # ---- the same GEMM kernel on operands without negative elements (|A|, |W|): their negative planes are all
-    # zero, so the kernel issues one product per tile pair instead of four.  This is what a symmetric FP4 format
-    # with one scale per group would cost on this kernel: the FP4-pipe ceiling of the design.
-    one_sided = None
+    # ---- the paper's symmetric comparison formats on the same kernels (one shared scale per group: no split by
+    # sign, one FP4 product per tile pair instead of four).  Shows what AMXFP4's asymmetry costs on this GPU, and
+    # the rate of the FP4 pipe on this kernel design when nothing is split.
+    format_variants = None
     if "mxf4" in gemm_kernel and not args.layers and not args.skip_extras:
-        prep1 = []
-        for li, (K, N) in enumerate(layers):
-            b = bufs[li]
-            a_abs = (A[li].view(torch.int16) & 0x7FFF).view(torch.bfloat16)
-            w_abs = (W[li].view(torch.int16) & 0x7FFF).view(torch.bfloat16)
-            pa = torch.empty(L.amx_prepared_bytes(M, K, GS, 0), dtype=torch.uint8, device="cuda")
-            pw = torch.empty(L.amx_prepared_bytes(N, K, GS, 1), dtype=torch.uint8, device="cuda")
-            check(L.amx_quantize_prepared(a_abs.data_ptr(), M, K, GS, 0, b["ac"].data_ptr(), b["as"].data_ptr(),
-                                          pa.data_ptr(), pa.numel(), stream))
-            check(L.amx_quantize_prepared(w_abs.data_ptr(), N, K, GS, 1, b["wc"].data_ptr(), b["ws"].data_ptr(),
-                                          pw.data_ptr(), pw.numel(), stream))
-            prep1.append((pa, pw))
-            del a_abs, w_abs
+        format_variants = {}
+        for name, fmt in (("sym_fp8", 1), ("mxfp4", 2)):
+            def fmt_step(stream, with_casts, fmt=fmt):
+                for li, (K, N) in enumerate(layers):
+                    b = bufs[li]
+                    if with_casts:
+                        check(L.amx_quantize_prepared_fmt(A[li].data_ptr(), M, K, GS, 0, fmt, b["ac"].data_ptr(),
+                                                          b["as"].data_ptr(), b["pa"].data_ptr(), b["pa"].numel(), stream))
+                        check(L.amx_quantize_prepared_fmt(W[li].data_ptr(), N, K, GS, 1, fmt, b["wc"].data_ptr(),
+                                                          b["ws"].data_ptr(), b["pw"].data_ptr(), b["pw"].numel(), stream))
+                    check(L.amx_gemm_prepared(b["pa"].data_ptr(), b["pw"].data_ptr(), M, N, K, GS, b["c"].data_ptr(), N,
+                                              b["work"].data_ptr(), b["work"].numel(), stream))
 
-        def gemms_only(stream):
-            for li, (K, N) in enumerate(layers):
-                b, (pa, pw) = bufs[li], prep1[li]
-                check(L.amx_gemm_prepared(pa.data_ptr(), pw.data_ptr(), M, N, K, GS, b["c"].data_ptr(), N,
-                                          b["work"].data_ptr(), b["work"].numel(), stream))
-
-        gemms_only(stream)
+            res = {}
+            for key, with_casts in (("step", True), ("gemm", False)):
+                fmt_step(stream, True)
+                torch.cuda.synchronize()
+                sv = torch.cuda.Stream()
+                sv.wait_stream(torch.cuda.current_stream())
+                gv = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gv, stream=sv):
+                    fmt_step(torch.cuda.current_stream().cuda_stream, with_casts)
+                for _ in range(3):
+                    gv.replay()
+                v0, v1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                v0.record()
+                for _ in range(args.steps):
+                    gv.replay()
+                v1.record()
+                torch.cuda.synchronize()
+                v_ms = v0.elapsed_time(v1) / args.steps
+                res[key + "_tflops"] = flops_step / (v_ms * 1e-3) / 1e12
+                res[key + "_ms"] = v_ms
+            format_variants[name] = res
+        format_variants["what"] = ("same workload and kernels with the symmetric formats (amx_quantize_prepared_fmt): "
+                                   "step = casts of both operands + GEMMs, gemm = the four GEMMs alone")
+        # leave the buffers as the headline step writes them
+        step(False, stream)
         torch.cuda.synchronize()
-        side3 = torch.cuda.Stream()
-        side3.wait_stream(torch.cuda.current_stream())
-        g3 = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g3, stream=side3):
-            gemms_only(torch.cuda.current_stream().cuda_stream)
-        for _ in range(3):
-            g3.replay()
-        o0, o1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        o0.record()
-        for _ in range(args.steps):
-            g3.replay()
-        o1.record()
-        torch.cuda.synchronize()
-        o_ms = o0.elapsed_time(o1) / args.steps
-        one_sided = {"tflops": flops_step / (o_ms * 1e-3) / 1e12, "ms_per_step": o_ms,
-                     "what": "the four GEMMs alone on |A| and |W| (no negative elements: one FP4 product per tile "
-                             "pair instead of four), i.e. the rate a one-scale-per-group FP4 format gets from this kernel"}
-        del prep1
 
     # ---- the cast alone on a tensor larger than L2 (config-4 activation shape, 16384 x 8192 = 268 MB of bf16)
     quant_large = None
@@ -570,7 +569,7 @@ def run_ours(args):
                      "kernel": f"amx_gemm ({gemm_kernel})",
                      "peak_source": f"4 x sustained bf16 cuBLAS rate ({peaks['source']}), nominal FP4:bf16 ratio"},
         "weights_cached": weights_cached,
-        "gemm_one_sided_operands": one_sided,
+        "format_variants": format_variants,
         "attention": attention,
         "small_case": small_case,
         "clocks": clocks,
