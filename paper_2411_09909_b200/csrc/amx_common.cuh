@@ -34,11 +34,14 @@ __device__ __forceinline__ float e2m1_mag_to_float(uint32_t c3) {
     return (c3 & 6u) ? v : 0.5f * (float)(c3 & 1u);
 }
 
-// Exponent key of an E5M2 scale byte: unbiased exponent + 17 (1 for 2^-16), 0 for a zero scale.
-__device__ __forceinline__ int scale_key(uint32_t b) {
-    const int e = (b >> 2) & 31, m = b & 3;
-    return e ? e + 2 : (m == 0 ? 0 : (m == 1 ? 1 : 2));
+// An E5M2 scale byte as (key << 2) | mantissa of its normalised form: key = unbiased exponent + 17 (so that
+// 2^-16 has key 1) and two mantissa bits.  Normal bytes (b >= 4) are b + 8; the subnormals 1, 2, 3 x 2^-16 are
+// 1.0 x 2^-16, 1.0 x 2^-15 and 1.5 x 2^-15: 4, 8 and 10 (read from a packed table); 0 for a zero scale.
+__device__ __forceinline__ uint32_t scale_norm(uint32_t b) {
+    return b >= 4 ? b + 8 : (0x0A080400u >> (b * 8)) & 0xFFu;
 }
+// Exponent key of an E5M2 scale byte, 0 for a zero scale.
+__device__ __forceinline__ int scale_key(uint32_t b) { return (int)(scale_norm(b) >> 2); }
 // Per-row word of a prepared FP4-GEMM operand: bits 15..0 the row's power-of-two offset (largest exponent key
 // - 25; 0 for an all-zero row) as a signed 16-bit number, bit 16 set when some group of the row has a nonzero
 // positive-side scale, bit 17 the same for the negative side.  A tile whose rows all lack a side has an
@@ -63,13 +66,11 @@ __host__ __device__ __forceinline__ int64_t sf_row_offset(int64_t row, int nk64)
 }
 __host__ __device__ __forceinline__ int64_t sf_group_offset(int g) { return (int64_t)(g >> 1) * kSfChunkBytes + (g & 1) * 2; }
 
-// UE4M3 byte of the E5M2 byte b for a row whose largest key is kmax (0 when it does not fit).
+// UE4M3 byte of the E5M2 byte b for a row whose largest key is kmax (0 when it does not fit): exponent field
+// key - kmax + 15 (at least 1), the two mantissa bits in bits 2..1.
 __device__ __forceinline__ uint32_t to_ue4m3(uint32_t b, int kmax) {
-    const int e = (b >> 2) & 31, m = b & 3;
-    const int f = scale_key(b) - kmax + 15;                      // UE4M3 exponent field
-    const int mant = e ? m : (m == 3 ? 2 : 0);                   // subnormals: 1, 2, 3 x 2^-16
-    return (f >= 1 && scale_key(b) > 0) ? (uint32_t)((f << 3) | (mant << 1)) : 0u;
+    const int t = (int)scale_norm(b) + ((15 - kmax) << 2);       // (exponent field << 2) | mantissa
+    return (b != 0 && t >= 4) ? (uint32_t)t << 1 : 0u;
 }
-
 
 }  // namespace amx
