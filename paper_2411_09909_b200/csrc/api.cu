@@ -167,6 +167,19 @@ extern "C" int amx_quant_gemm(const void* A, int64_t ld_a, const uint8_t* w_code
     }
     uint8_t* a_codes = base + gemm_ws;
     uint8_t* a_scales = a_codes + a.codes;
+    if (pick_kernel(M, N, K, group_size, flags) == AMX_GEMM_FP4 && ld_a == K) {
+        // the activation's cast writes the kernel's operand itself (one launch less, the codes are not re-read);
+        // same workspace layout as amx_gemm's: status word, prepared A, prepared W
+        if (!A || !w_codes || !w_scales || !C) return AMX_ERR_NULL;
+        if (!aligned(A, 16) || !aligned(w_codes, 16) || !aligned(w_scales, 2) || !aligned(C, 4)) return AMX_ERR_ALIGN;
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        uint8_t* pa = base + 256;
+        uint8_t* pw = pa + gemm_fp4_prepared_bytes(M, K, false);
+        int rc = gemm_fp4_quantize_prepared(A, M, K, false, a_codes, a_scales, pa, st);
+        if (rc == AMX_OK) rc = gemm_fp4_prepare(w_codes, w_scales, N, K, true, pw, st);
+        if (rc != AMX_OK) return rc;
+        return gemm_fp4_prepared(pa, pw, M, N, K, C, ld_c, base, st);
+    }
     int rc = amx_quantize(A, M, K, ld_a, group_size, a_codes, a_scales, stream);
     if (rc != AMX_OK) return rc;
     return amx_gemm(a_codes, a_scales, w_codes, w_scales, M, N, K, group_size, flags, C, ld_c, base, gemm_ws, stream);
