@@ -280,6 +280,31 @@ def test_symmetric_formats(fmt, mode):
     assert rel_fro(amx.gemm_prepared(pa, pw_amx, 300, 520, 1056).cpu().numpy(), oracle.gemm(*qa, *wq, 32)) <= GEMM_TOL
 
 
+def test_fp4_path_shape_sweep():
+    """Seeded sweep of ragged shapes through the fused cast and the FP4 kernel (prepared buffers pre-filled with
+    0xFF, padded output), against the oracle on the oracle's own codes."""
+    rng = np.random.default_rng(2411)
+    for case in range(10):
+        M, N = int(rng.integers(1, 400)), int(rng.integers(1, 600))
+        K = 32 * int(rng.integers(1, 72))
+        fmt, mode = [(amx.FMT_AMXFP4, 0), (amx.FMT_SYM_FP8, oracle.SYMMETRIC_FP8), (amx.FMT_MXFP4, oracle.MXFP4)][case % 3]
+        a_bits = inputs.random_groups(500 + case, M, K, "mixed" if case % 2 else "normal")
+        w_bits = inputs.random_groups(600 + case, N, K, "normal")
+        quant = (lambda b: oracle.quantize(b, 32)) if mode == 0 else (lambda b: oracle.quantize_variant(b, 32, mode))
+        qa, qw = quant(a_bits), quant(w_bits)
+        dirty = lambda rows, w: torch.full((amx.lib().amx_prepared_bytes(rows, K, 32, w),), 0xFF, dtype=torch.uint8, device="cuda")
+        ac, as_, pa = amx.quantize_prepared(dev_bf16(a_bits), False, prepared=dirty(M, 0), fmt=fmt)
+        wc, ws, pw = amx.quantize_prepared(dev_bf16(w_bits), True, prepared=dirty(N, 1), fmt=fmt)
+        assert np.array_equal(ac.cpu().numpy(), qa[0]) and np.array_equal(as_.cpu().numpy(), qa[1]), (case, M, K)
+        assert np.array_equal(wc.cpu().numpy(), qw[0]) and np.array_equal(ws.cpu().numpy(), qw[1]), (case, N, K)
+        wide = torch.full((M, N + 5), -3.0, dtype=torch.float32, device="cuda")
+        got = amx.gemm_prepared(pa, pw, M, N, K, out=wide[:, :N])
+        ref = oracle.gemm(*qa, *qw, 32)
+        if np.linalg.norm(ref) > 0:
+            assert rel_fro(got.cpu().numpy(), ref) <= 2e-4, (case, M, N, K, fmt)
+        assert torch.all(wide[:, N:] == -3.0)
+
+
 def test_quantize_prepared_equals_quantize_then_prepare():
     # row lengths below, at and above one block of the cast kernel (several rows, one row and a fraction of a
     # row per block; threads striding over a long row), ragged row counts, both paddings
