@@ -501,6 +501,49 @@ def run_ours(args):
                       "us_per_call": s0.elapsed_time(s1) * 1e3 / 200,
                       "note": "launch-latency-bound (32 output tiles at most): microseconds, not a roofline fraction"}
 
+    # ---- decode-like shape: 16 token rows against the config-2 weights (cast once), amx_quant_gemm per layer,
+    # replayed as a CUDA graph.  Bound by streaming the 4.5-bit weights: report the rate at which they are read.
+    decode = None
+    if not args.layers and not args.skip_extras and world == 1 and CONFIG == 2:
+        Md = 16
+        dd = []
+        for li, (K, N) in enumerate(layers):
+            wc_, ws_ = amx.quantize(W[li], GS)
+            ad = A[li][:Md].contiguous()
+            need = max(L.amx_quant_gemm_workspace_bytes(Md, N, K, GS, 0), 256)
+            dd.append((ad, wc_, ws_, torch.empty((Md, N), dtype=torch.float32, device="cuda"),
+                       torch.empty(need, dtype=torch.uint8, device="cuda")))
+
+        def decode_step(stream):
+            for li, (K, N) in enumerate(layers):
+                ad, wc_, ws_, cd, wsd = dd[li]
+                check(L.amx_quant_gemm(ad.data_ptr(), K, wc_.data_ptr(), ws_.data_ptr(), Md, N, K, GS, 0, cd.data_ptr(), N,
+                                       wsd.data_ptr(), wsd.numel(), stream))
+
+        decode_step(stream)
+        torch.cuda.synchronize()
+        sd = torch.cuda.Stream()
+        sd.wait_stream(torch.cuda.current_stream())
+        gd = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gd, stream=sd):
+            decode_step(torch.cuda.current_stream().cuda_stream)
+        for _ in range(3):
+            gd.replay()
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        d0.record()
+        for _ in range(args.steps):
+            gd.replay()
+        d1.record()
+        torch.cuda.synchronize()
+        d_us = d0.elapsed_time(d1) / args.steps * 1e3
+        w_bytes = sum(N * K for K, N in layers) * (0.5 + 2.0 / 32.0)
+        decode = {"workload": f"{Md} token rows x the four config-2 weights (cast once); amx_quant_gemm per layer, graph replay",
+                  "us_per_step": d_us, "weight_gb_per_s": w_bytes / (d_us * 1e-6) / 1e9,
+                  "frac_of_measured_copy": w_bytes / (d_us * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                  "kernel": "tcgen05 kind::f16 (bf16 decode), K cut into slices over CTAs"}
+        del dd
+
     # ---- end to end through the host-buffer entry point (pinned host tensors, copies inside the timing)
     e2e = None
     if (rank == 0 or world > 1) and not args.skip_extras and CONFIG == 2:
@@ -576,6 +619,7 @@ def run_ours(args):
         "format_variants": format_variants,
         "attention": attention,
         "small_case": small_case,
+        "decode": decode,
         "clocks": clocks,
         "e2e": e2e,
         # kernels per layer: 2 casts + the GEMM; without the fused entry points the FP4 kernel's operands need

@@ -61,8 +61,9 @@ typedef enum amx_status {
 #define AMX_OUT_BF16 0x0u
 #define AMX_OUT_F32 0x1u
 /* flags for amx_gemm / amx_quant_gemm: kernel choice.  Default (AMX_GEMM_AUTO): group size 32 runs on
- * the tensor cores - the FP4 kernel when M*N*K >= 2^27, the exact bf16-decode kernel below that - and
- * other group sizes on the SIMT kernel. */
+ * the tensor cores - the FP4 kernel when M*N*K >= 2^27, the exact bf16-decode kernel below that and for
+ * at most 64 rows of A against a large weight (decode-like shapes: that kernel then cuts K into slices over
+ * CTAs and adds the partial products in slice order) - and other group sizes on the SIMT kernel. */
 #define AMX_GEMM_AUTO 0x0u
 #define AMX_GEMM_SIMT 0x10u  /* plain CUDA-core kernel: any shape, any supported gs */
 #define AMX_GEMM_TC 0x20u    /* tcgen05 kernel, exact bf16 decode: AMX_ERR_SHAPE if the shape does not fit */

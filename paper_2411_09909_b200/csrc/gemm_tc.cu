@@ -159,13 +159,17 @@ gemm_tc_kernel(const uint8_t* __restrict__ a_codes, const uint8_t* __restrict__ 
                const uint16_t* __restrict__ a_x, int64_t ld_a,
                const uint8_t* __restrict__ w_codes, const uint8_t* __restrict__ w_scales,
                int64_t M, int64_t N, int64_t K, float* __restrict__ C, int64_t ld_c, int vec_store,
-               int* __restrict__ status) {
+               int* __restrict__ status, int kb_per_slice, int64_t slice_stride) {
+    // blockIdx.z: slice of the K range (kb_per_slice K blocks each); slice z writes its partial product to
+    // C + z * slice_stride (one slice: the result itself)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     Control* ctl = reinterpret_cast<Control*>(tiles + kStages * kStageBytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t m0 = (int64_t)blockIdx.y * BM, n0 = (int64_t)blockIdx.x * BN;
-    const int num_kb = (int)((K + BK - 1) / BK);
+    const int kb_begin = (int)blockIdx.z * kb_per_slice;
+    const int num_kb = min((int)((K + BK - 1) / BK) - kb_begin, kb_per_slice);   // K blocks of this slice
+    C += (int64_t)blockIdx.z * slice_stride;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -189,7 +193,7 @@ gemm_tc_kernel(const uint8_t* __restrict__ a_codes, const uint8_t* __restrict__ 
         Task cur[kTasksPerThread], nxt[kTasksPerThread];
         RawGroup raw;
         auto load_all = [&](Task (&t)[kTasksPerThread], int kb) {
-            const int64_t k = (int64_t)kb * BK + half * 32;
+            const int64_t k = (int64_t)(kb_begin + kb) * BK + half * 32;
             if (CAST_A) raw = load_raw(a_x, ld_a, m0 + r, M, K, k);
             else t[0] = load_task(a_codes, a_scales, m0 + r, M, K, k);
 #pragma unroll
@@ -207,9 +211,16 @@ gemm_tc_kernel(const uint8_t* __restrict__ a_codes, const uint8_t* __restrict__ 
             uint8_t* stage = tiles + s * kStageBytes;
 #pragma unroll
             for (int i = 0; i < kTasksPerThread; ++i) {
-                const GroupTables t = make_tables(cur[i].scales);
                 const int row = r + 128 * i;                       // row inside [A tile | B tile]
                 uint8_t* dst = stage + row * 128;                  // A tile is 128 rows: B rows follow it
+                const bool live = i ? (n0 + r + 128 * (i - 1) < N) : (m0 + r < M);
+                if (!live) {                                       // a row past the operand: zeros, no decode
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        *reinterpret_cast<uint4*>(dst + (((half * 4 + j) ^ (row & 7)) << 4)) = make_uint4(0, 0, 0, 0);
+                    continue;
+                }
+                const GroupTables t = make_tables(cur[i].scales);
                 const uint32_t w[4] = {cur[i].codes.x, cur[i].codes.y, cur[i].codes.z, cur[i].codes.w};
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
@@ -282,7 +293,43 @@ bool gemm_tc_supported(int64_t M, int64_t N, int64_t K, int gs) {
     return gs == 32 && M > 0 && N > 0 && K > 0 && K % 32 == 0 && (M + BM - 1) / BM <= 65535;
 }
 
-size_t gemm_tc_workspace_bytes(int64_t, int64_t, int64_t) { return 256; }   // the status word
+namespace {
+
+// Few output tiles and a long K (a handful of token rows against a big weight: the decode phase): the K range is
+// cut into slices that run as separate CTAs, so that the whole machine streams and decodes the weight; the
+// partial products go to the workspace and are added up in slice order (deterministic).  Returns the number of
+// slices (1: none) and the K blocks per slice.
+constexpr int kSmCount = 148;
+int k_slices(int64_t M, int64_t N, int64_t K, int& kb_per_slice) {
+    const int64_t tiles = ((N + BN - 1) / BN) * ((M + BM - 1) / BM);
+    const int num_kb = (int)((K + BK - 1) / BK);
+    kb_per_slice = num_kb;
+    if (tiles >= kSmCount || num_kb < 16) return 1;
+    int want = (int)(2 * kSmCount / tiles);                          // two CTAs per SM, one wave
+    if (want > num_kb / 8) want = num_kb / 8;                        // at least 8 K blocks per slice
+    if (want > 16) want = 16;
+    if (want < 2) return 1;
+    kb_per_slice = (num_kb + want - 1) / want;
+    return (num_kb + kb_per_slice - 1) / kb_per_slice;
+}
+
+// C[m][n] = sum over slices, in slice order.
+__global__ void __launch_bounds__(256)
+reduce_slices_kernel(const float* __restrict__ part, int slices, int64_t M, int64_t N, float* __restrict__ C, int64_t ld_c) {
+    const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (i >= M * N) return;
+    float acc = part[i];
+    for (int z = 1; z < slices; ++z) acc += part[(int64_t)z * M * N + i];
+    C[(i / N) * ld_c + i % N] = acc;
+}
+
+}  // namespace
+
+size_t gemm_tc_workspace_bytes(int64_t M, int64_t N, int64_t K) {   // the status word, then the slices' partial products
+    int kb_per;
+    const int slices = k_slices(M, N, K, kb_per);
+    return 256 + (slices > 1 ? (size_t)slices * M * N * 4 : 0);
+}
 
 namespace {
 
@@ -300,14 +347,22 @@ int launch_tc(const uint8_t* a_codes, const uint8_t* a_scales, const uint16_t* a
     }
     int* status = static_cast<int*>(workspace);
     if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return AMX_ERR_CUDA;
-    dim3 grid((unsigned)((N + BN - 1) / BN), (unsigned)((M + BM - 1) / BM));
-    const int vec_store = aligned(C, 16) && ld_c % 4 == 0;   // else the epilogue stores scalars
+    int kb_per;
+    const int slices = k_slices(M, N, K, kb_per);
+    dim3 grid((unsigned)((N + BN - 1) / BN), (unsigned)((M + BM - 1) / BM), (unsigned)slices);
+    float* part = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 256);
+    float* out = slices > 1 ? part : C;
+    const int64_t ld_out = slices > 1 ? N : ld_c, slice_stride = slices > 1 ? M * N : 0;
+    const int vec_store = aligned(out, 16) && ld_out % 4 == 0;   // else the epilogue stores scalars
     if (a_x)
-        gemm_tc_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(nullptr, nullptr, a_x, ld_a, w_codes, w_scales, M, N, K, C,
-                                                                 ld_c, vec_store, status);
+        gemm_tc_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(nullptr, nullptr, a_x, ld_a, w_codes, w_scales, M, N, K, out,
+                                                                 ld_out, vec_store, status, kb_per, slice_stride);
     else
         gemm_tc_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(a_codes, a_scales, nullptr, 0, w_codes, w_scales, M, N, K,
-                                                                  C, ld_c, vec_store, status);
+                                                                  out, ld_out, vec_store, status, kb_per, slice_stride);
+    int rc = launch_status();
+    if (rc != AMX_OK || slices == 1) return rc;
+    reduce_slices_kernel<<<(unsigned)((M * N + 255) / 256), 256, 0, st>>>(part, slices, M, N, C, ld_c);
     return launch_status();
 }
 

@@ -280,6 +280,26 @@ def test_symmetric_formats(fmt, mode):
     assert rel_fro(amx.gemm_prepared(pa, pw_amx, 300, 520, 1056).cpu().numpy(), oracle.gemm(*qa, *wq, 32)) <= GEMM_TOL
 
 
+@pytest.mark.parametrize("M,N,K", [(1, 12288, 4096), (16, 600, 4096), (130, 300, 2048), (7, 256, 11008)])
+def test_gemm_tc_few_tiles_long_k(M, N, K):
+    """A few token rows against a big weight (decode-like): the bf16-decode kernel cuts K into slices that run as
+    separate CTAs and adds their partial products in slice order; run-to-run identical, padded output untouched,
+    and the cast-in-kernel variant takes the same route."""
+    a_bits = inputs.random_groups(700 + M, M, K, "normal")
+    w_bits = inputs.random_groups(701 + N, N, K, "normal")
+    qa, qw = oracle.quantize(a_bits, 32), oracle.quantize(w_bits, 32)
+    ref = oracle.gemm(*qa, *qw, 32)
+    dev = [torch.from_numpy(t).cuda() for t in (*qa, *qw)]
+    assert amx.lib().amx_workspace_bytes(M, N, K, 32, amx.GEMM_TC) > 256          # slices are in use
+    wide = torch.full((M, N + 12), 5.0, dtype=torch.float32, device="cuda")
+    got = amx.gemm(*dev, 32, amx.GEMM_TC, out=wide[:, :N])
+    assert rel_fro(got.cpu().numpy(), ref) <= 1e-5
+    assert torch.all(wide[:, N:] == 5.0)
+    assert torch.equal(amx.gemm(*dev, 32, amx.GEMM_TC), got.contiguous())
+    fused = amx.quant_gemm(dev_bf16(a_bits), dev[2], dev[3], 32, flags=amx.GEMM_TC | amx.GEMM_CAST_IN_KERNEL)
+    assert torch.equal(fused, got.contiguous())
+
+
 def test_fp4_path_shape_sweep():
     """Seeded sweep of ragged shapes through the fused cast and the FP4 kernel (prepared buffers pre-filled with
     0xFF, padded output), against the oracle on the oracle's own codes."""
