@@ -142,7 +142,11 @@ int amx_gemm(const uint8_t* a_codes, const uint8_t* a_scales,
  *                      offset per row - in a caller-owned buffer of amx_prepared_bytes() bytes
  *                      (256-byte aligned).  is_weight selects the padding of the W (right-hand) operand.
  *   amx_gemm_prepared  multiplies a prepared A [M, K] with a prepared W [N, K]; same result as amx_gemm
- *                      with AMX_GEMM_FP4.  workspace: 256 bytes (status word, see amx_gemm_status).
+ *                      with AMX_GEMM_FP4.  workspace: 256 bytes (status word, see amx_gemm_status) always
+ *                      suffice; with amx_gemm_prepared_workspace_bytes() bytes a product with few output tiles
+ *                      and a long K (a few token rows against a big weight) is cut into K ranges that run as
+ *                      separate CTAs, their partial products added in range order (same result up to fp32
+ *                      summation order, run-to-run identical).
  *   amx_quantize_prepared  amx_quantize (x bf16 [rows, K], contiguous rows, gs = 32) and amx_prepare in one
  *                      go: the cast kernel itself writes the sign planes, so the codes are not read again.
  *                      Writes the canonical codes and scales too.
@@ -159,6 +163,7 @@ int amx_quantize_prepared_fmt(const void* x, int64_t rows, int64_t K, int group_
 size_t amx_prepared_bytes(int64_t rows, int64_t K, int group_size, int is_weight);
 int amx_prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, int group_size,
                 int is_weight, void* prepared, size_t prepared_bytes, void* stream);
+size_t amx_gemm_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size);
 int amx_gemm_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
                       int group_size, float* C, int64_t ld_c, void* workspace, size_t workspace_bytes,
                       void* stream);

@@ -29,7 +29,7 @@ SYMBOLS = (
     "amx_quant_gemm_static", "amx_quant_gemm_static_capacity",
     "amx_attention", "amx_attention_workspace_bytes",
     "amx_prepared_bytes", "amx_prepare", "amx_gemm_prepared", "amx_quantize_prepared", "amx_softmax_quantize",
-    "amx_quantize_fmt", "amx_quantize_prepared_fmt",
+    "amx_quantize_fmt", "amx_quantize_prepared_fmt", "amx_gemm_prepared_workspace_bytes",
 )
 
 
@@ -62,6 +62,8 @@ def lib() -> ctypes.CDLL:
         L.amx_prepare.argtypes = [p, p, i64, i64, i, i, p, sz, p]
         L.amx_quantize_prepared.argtypes = [p, i64, i64, i, i, p, p, p, sz, p]
         L.amx_gemm_prepared.argtypes = [p, p, i64, i64, i64, i, p, i64, p, sz, p]
+        L.amx_gemm_prepared_workspace_bytes.argtypes = [i64, i64, i64, i]
+        L.amx_gemm_prepared_workspace_bytes.restype = sz
         L.amx_softmax_bf16.argtypes = [p, i64, i64, i64, ctypes.c_float, p, i64, p]
         L.amx_softmax_quantize.argtypes = [p, i64, i64, i64, ctypes.c_float, p, p, i, p, sz, p]
         L.amx_linear_host.argtypes = [p, p, i64, i64, i64, i, u32, p, p, sz, p]
@@ -195,7 +197,7 @@ def gemm_prepared(a_prepared: torch.Tensor, w_prepared: torch.Tensor, M: int, N:
     if out is None:
         out = torch.empty((M, N), dtype=torch.float32, device=a_prepared.device)
     if workspace is None:
-        workspace = _ws(256, a_prepared.device)
+        workspace = _ws(lib().amx_gemm_prepared_workspace_bytes(M, N, K, group_size), a_prepared.device)
     _check(lib().amx_gemm_prepared(a_prepared.data_ptr(), w_prepared.data_ptr(), M, N, K, group_size, out.data_ptr(),
                                    out.stride(0), workspace.data_ptr(), workspace.numel(), _stream()), "amx_gemm_prepared")
     return out

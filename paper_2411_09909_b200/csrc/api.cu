@@ -134,6 +134,11 @@ extern "C" int amx_quantize_prepared_fmt(const void* x, int64_t rows, int64_t K,
                                       0, format);
 }
 
+extern "C" size_t amx_gemm_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size) {
+    if (M <= 0 || N <= 0 || !gemm_fp4_supported(M, N, K, group_size)) return 0;
+    return round_up(gemm_fp4_prepared_workspace_bytes(M, N, K));
+}
+
 extern "C" int amx_gemm_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
                                  int group_size, float* C, int64_t ld_c, void* workspace, size_t workspace_bytes,
                                  void* stream) {
@@ -142,7 +147,8 @@ extern "C" int amx_gemm_prepared(const void* a_prepared, const void* w_prepared,
     if (!workspace || workspace_bytes < 256) return AMX_ERR_WORKSPACE;
     if (!aligned(a_prepared, kAlign) || !aligned(w_prepared, kAlign) || !aligned(workspace, kAlign) || !aligned(C, 4))
         return AMX_ERR_ALIGN;
-    return gemm_fp4_prepared(a_prepared, w_prepared, M, N, K, C, ld_c, workspace, static_cast<cudaStream_t>(stream));
+    return gemm_fp4_prepared(a_prepared, w_prepared, M, N, K, C, ld_c, workspace, static_cast<cudaStream_t>(stream),
+                             workspace_bytes);
 }
 
 extern "C" int amx_quant_gemm(const void* A, int64_t ld_a, const uint8_t* w_codes, const uint8_t* w_scales,

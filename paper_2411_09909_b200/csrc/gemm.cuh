@@ -52,7 +52,11 @@ struct Fp4Operand {
     int64_t rows_total, layout_rows, row0;
 };
 int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
-                         int64_t ld_c, void* workspace, cudaStream_t st);
+                         int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes = 256);
+// workspace that lets the kernel cut K into ranges for products with few output tiles (256 bytes otherwise)
+size_t gemm_fp4_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K);
+// C[m][n] = sum over `slices` partial products [slices][M][N], in slice order (defined with the bf16-decode kernel)
+int reduce_slices(const float* part, int slices, int64_t M, int64_t N, float* C, int64_t ld_c, cudaStream_t st);
 // P = softmax(alpha * Q K^T) cast to AMXFP4 (canonical + prepared left-hand operand) without the logits in
 // memory; L % 256 == 0; scratch of gemm_fp4_attn_scratch_bytes(L) bytes.
 size_t gemm_fp4_attn_scratch_bytes(int64_t L);
@@ -61,6 +65,7 @@ int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, in
 int quantize_cols_batched(const void* x, int64_t batch, int64_t R, int64_t C, uint8_t* codes, uint8_t* scales,
                           cudaStream_t st);
 int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
-                      float* C, int64_t ld_c, void* workspace /* 256 B: status word */, cudaStream_t st);
+                      float* C, int64_t ld_c, void* workspace /* 256 B: status word */, cudaStream_t st,
+                      size_t workspace_bytes = 256);
 
 }  // namespace amx

@@ -193,6 +193,8 @@ struct Params {
 
     float* C;
     int nk64, vec_store;
+    int slices;                  // SLICED instantiation: K is cut into this many ranges, each (tile, range) a work item
+    int64_t slice_stride;        //   whose partial product goes to C + range * slice_stride
     int* status;
     // attention epilogues (kEpiStats, kEpiCast): the tile holds logits S = Q K^T; `alpha` scales them
     float alpha;
@@ -222,7 +224,7 @@ __device__ __forceinline__ void store_row16(float* out, const float (&f)[16], bo
     }
 }
 
-template <int BK_, int EPI = kEpiStore>
+template <int BK_, int EPI = kEpiStore, bool SLICED = false>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w, const Params p) {
     using C_ = Cfg<BK_>;
@@ -232,9 +234,12 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     Control* ctl = reinterpret_cast<Control*>(tiles + kStages * kStageBytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int num_kb = (int)((p.K + BK - 1) / BK);
+    // Work items: tile x K range (one range unless SLICED); an item index is tile * S + range, num_kb the K blocks
+    // of one item (the host picks a slice count that divides the K blocks).
+    const int S = SLICED ? p.slices : 1;
+    const int num_kb = (int)((p.K + BK - 1) / BK) / S;
     // Persistent CTA: tiles blockIdx.x, blockIdx.x + gridDim.x, ...; neighbouring tiles share their A rows.
-    const int64_t n_tiles = (p.N + BN - 1) / BN, total_tiles = ((p.M + BM - 1) / BM) * n_tiles;
+    const int64_t n_tiles = (p.N + BN - 1) / BN, total_tiles = ((p.M + BM - 1) / BM) * n_tiles * S;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -258,7 +263,8 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             int it = 0;                                          // K blocks issued so far, over all tiles
             bool ok = true;
             for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int64_t m_blk = tile / n_tiles, n_blk = tile % n_tiles;
+                const int64_t m_blk = (tile / S) / n_tiles, n_blk = (tile / S) % n_tiles;
+                const int kb0 = (int)(tile % S) * num_kb;
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const int s = it % kStages;
                     if (it >= kStages && !mbar_wait(&ctl->empty[s], ((it / kStages) - 1) & 1, &ctl->abort, p.status)) {
@@ -268,8 +274,8 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                     uint8_t* st = tiles + s * kStageBytes;
                     mbar_expect_tx(&ctl->full[s], kStageBytes);
                     // one 3-D tile per operand: {row bytes, rows, both sign planes}
-                    tma_load_3d(st + C_::kOffAp, &tm_a, kb * kRowBytes, (int)(p.a_row0 + m_blk * BM), 0, &ctl->full[s]);
-                    tma_load_3d(st + C_::kOffWp, &tm_w, kb * kRowBytes, (int)(p.w_row0 + n_blk * BN), 0, &ctl->full[s]);
+                    tma_load_3d(st + C_::kOffAp, &tm_a, (kb0 + kb) * kRowBytes, (int)(p.a_row0 + m_blk * BM), 0, &ctl->full[s]);
+                    tma_load_3d(st + C_::kOffWp, &tm_w, (kb0 + kb) * kRowBytes, (int)(p.w_row0 + n_blk * BN), 0, &ctl->full[s]);
                 }
             }
             // after an abort: let the copies already in flight land before shared memory is released
@@ -291,7 +297,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         auto tile_sides = [&](int64_t tile) {
             int bits = 0;
             if (tile < total_tiles) {
-                const int64_t m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
+                const int64_t m0 = ((tile / S) / n_tiles) * BM, n0 = ((tile / S) % n_tiles) * BN;
 #pragma unroll
                 for (int i = 0; i < BM / 32; ++i)
                     if (m0 + i * 32 + lane < p.M) bits |= (__ldg(p.a_exp + m0 + i * 32 + lane) >> 16) & 3;
@@ -364,12 +370,12 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         constexpr int kBlocks = 2 * kSteps * 3;                  // per K block: A (1) + W (2 row blocks), x planes x steps
         uint4 sfv[kBlocks];
         auto fetch = [&](int64_t tile, int kb) {
-            const int64_t m_blk = tile / n_tiles, n_blk = tile % n_tiles;
+            const int64_t m_blk = (tile / S) / n_tiles, n_blk = (tile / S) % n_tiles;
 #pragma unroll
             for (int pl = 0; pl < 2; ++pl)
 #pragma unroll
                 for (int kk = 0; kk < kSteps; ++kk) {
-                    const int64_t c = (int64_t)kb * kSteps + kk;
+                    const int64_t c = ((int64_t)(tile % S) * num_kb + kb) * kSteps + kk;
                     const uint8_t* a = (pl ? p.sfa_neg : p.sfa_pos) + (m_blk * p.nk64 + c) * kSfChunk + lane * 16;
                     const uint8_t* w = (pl ? p.sfb_neg : p.sfb_pos) + ((n_blk * 2) * p.nk64 + c) * kSfChunk + lane * 16;
                     sfv[(pl * kSteps + kk) * 3 + 0] = __ldg(reinterpret_cast<const uint4*>(a));
@@ -416,7 +422,8 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         int t = 0;
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t) {
-            const int64_t m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
+            const int64_t m0 = ((tile / S) / n_tiles) * BM, n0 = ((tile / S) % n_tiles) * BN;
+            float* const C_item = p.C + (SLICED ? (tile % S) * p.slice_stride : 0);
             int* w_exp = ctl->w_exp[t & 1];
             for (int i = tid_e; i < BN; i += kEpilogueWarps * 32) {
                 const int ex = (n0 + i < p.N) ? row_word_exp(p.w_exp[n0 + i]) : 0;
@@ -451,7 +458,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                                 f[j + i] = __uint_as_float(v[buf][j + i]) * __uint_as_float((uint32_t)(sh + 127) << 23);
                             }
                         }
-                        if (m < p.M) store_row16(p.C + m * p.ld_c + n0 + col, f, p.vec_store != 0, p.N - (n0 + col));
+                        if (m < p.M) store_row16(C_item + m * p.ld_c + n0 + col, f, p.vec_store != 0, p.N - (n0 + col));
                     }
                 } else {
                     // The thread's 128 columns come from tensor memory 16 at a time, the next chunk in flight while
@@ -500,7 +507,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                             for (int j = 0; j < 16; ++j) s4[j & 3] += exp2_approx(fmaf(u[j], ra, -nmx));
                             sum += (s4[0] + s4[1]) + (s4[2] + s4[3]);
                         }
-                        if (m < p.M) p.part[m * (2 * n_tiles) + (tile % n_tiles) * 2 + (e >> 2)] = make_float2(mx, sum);
+                        if (m < p.M) p.part[m * (2 * n_tiles) + ((tile / S) % n_tiles) * 2 + (e >> 2)] = make_float2(mx, sum);
                     } else {
                         // Four 32-column groups per thread: normalise with the row's statistics {-max, 1 / sum}, round
                         // to bf16, cast.  P has no negative element: only its positive plane and scale factors exist.
@@ -619,13 +626,13 @@ size_t gemm_fp4_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 
 namespace {
 
-template <int BK_, int EPI = kEpiStore>
+template <int BK_, int EPI = kEpiStore, bool SLICED = false>
 int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, const OperandLayout& ow, int64_t a_rows,
                int64_t w_rows, Params p, int dev, cudaStream_t st) {
     using C_ = Cfg<BK_>;
     static bool configured[64] = {};
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(gemm_fp4_kernel<BK_, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(gemm_fp4_kernel<BK_, EPI, SLICED>, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::kSmemBytes) != cudaSuccess)
             return AMX_ERR_CUDA;
         configured[dev] = true;
     }
@@ -635,9 +642,9 @@ int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, co
     static int sm_count[64] = {};
     if (!sm_count[dev] && cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return AMX_ERR_CUDA;
-    const int64_t tiles = ((p.N + BN - 1) / BN) * ((p.M + BM - 1) / BM);
+    const int64_t tiles = ((p.N + BN - 1) / BN) * ((p.M + BM - 1) / BM) * (SLICED ? p.slices : 1);
     const unsigned grid = (unsigned)(tiles < sm_count[dev] ? tiles : sm_count[dev]);   // one persistent CTA per SM
-    gemm_fp4_kernel<BK_, EPI><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_a, tm_w, p);
+    gemm_fp4_kernel<BK_, EPI, SLICED><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_a, tm_w, p);
     return launch_status();
 }
 
@@ -711,9 +718,27 @@ attn_row_reduce_kernel(const float2* __restrict__ part, int n_parts, int64_t L, 
 }
 }  // namespace
 
+// Few output tiles and a long K (a few token rows against a big weight): K ranges as separate work items, so
+// that more SMs stream the operands; their partial products go to the workspace and are added in range order.
+// Returns the number of ranges (1: none); it divides the 128-element K blocks.
+int gemm_fp4_slices(int64_t M, int64_t N, int64_t K) {
+    const int64_t tiles = ((N + BN - 1) / BN) * ((M + BM - 1) / BM);
+    const int num_kb = (int)((K + 127) / 128);
+    int s = (int)(148 / tiles);
+    if (s > num_kb / 8) s = num_kb / 8;
+    if (s > 8) s = 8;
+    while (s > 1 && num_kb % s) --s;
+    return s < 2 ? 1 : s;
+}
+size_t gemm_fp4_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+    const int s = gemm_fp4_slices(M, N, K);
+    return 256 + (s > 1 ? (size_t)s * M * N * 4 : 0);
+}
+
 // The GEMM proper on two prepared operands (each laid out by operand_layout()), or on row ranges of them.
+// workspace_bytes >= gemm_fp4_prepared_workspace_bytes() enables the K ranges; 256 bytes always suffice.
 int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
-                         int64_t ld_c, void* workspace, cudaStream_t st) {
+                         int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes) {
     Params p;
     OperandLayout oa, ow;
     int dev;
@@ -721,6 +746,17 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
     if (rc != AMX_OK) return rc;
     const uint8_t* pa = static_cast<const uint8_t*>(a.prepared);
     const uint8_t* pw = static_cast<const uint8_t*>(w.prepared);
+    const int slices = gemm_fp4_slices(M, N, K);
+    if (slices > 1 && fp4_block_k() == 128 && workspace_bytes >= gemm_fp4_prepared_workspace_bytes(M, N, K)) {
+        float* part = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 256);
+        p.C = part;
+        p.ld_c = N;
+        p.vec_store = N % 8 == 0;
+        p.slices = slices;
+        p.slice_stride = M * N;
+        const int r2 = launch_fp4<128, kEpiStore, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
+        return r2 != AMX_OK ? r2 : reduce_slices(part, slices, M, N, C, ld_c, st);
+    }
     return fp4_block_k() == 256 ? launch_fp4<256>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st)
                                 : launch_fp4<128>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
 }
@@ -768,8 +804,9 @@ int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, in
 }
 
 int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K, float* C,
-                      int64_t ld_c, void* workspace, cudaStream_t st) {
-    return gemm_fp4_prepared_at({a_prepared, M, M, 0}, {w_prepared, N, N, 0}, M, N, K, C, ld_c, workspace, st);
+                      int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes) {
+    return gemm_fp4_prepared_at({a_prepared, M, M, 0}, {w_prepared, N, N, 0}, M, N, K, C, ld_c, workspace, st,
+                                workspace_bytes);
 }
 
 // Size of a prepared operand: as the A operand (rows padded to 128) or the W operand (rows padded to 256).

@@ -362,11 +362,15 @@ int launch_tc(const uint8_t* a_codes, const uint8_t* a_scales, const uint16_t* a
                                                                   out, ld_out, vec_store, status, kb_per, slice_stride);
     int rc = launch_status();
     if (rc != AMX_OK || slices == 1) return rc;
-    reduce_slices_kernel<<<(unsigned)((M * N + 255) / 256), 256, 0, st>>>(part, slices, M, N, C, ld_c);
-    return launch_status();
+    return reduce_slices(part, slices, M, N, C, ld_c, st);
 }
 
 }  // namespace
+
+int reduce_slices(const float* part, int slices, int64_t M, int64_t N, float* C, int64_t ld_c, cudaStream_t st) {
+    reduce_slices_kernel<<<(unsigned)((M * N + 255) / 256), 256, 0, st>>>(part, slices, M, N, C, ld_c);
+    return launch_status();
+}
 
 int gemm_tc(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes, const uint8_t* w_scales,
             int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {

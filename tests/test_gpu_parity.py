@@ -300,6 +300,27 @@ def test_gemm_tc_few_tiles_long_k(M, N, K):
     assert torch.equal(fused, got.contiguous())
 
 
+@pytest.mark.parametrize("M,N,K", [(16, 1200, 4096), (130, 300, 2048), (1, 256, 11264)])
+def test_gemm_prepared_few_tiles_long_k(M, N, K):
+    """The FP4 kernel on prepared operands with few output tiles and a long K: with the larger workspace the K
+    range is cut into ranges that run as separate work items; partial products are added in range order."""
+    a_bits = inputs.random_groups(800 + M, M, K, "normal")
+    w_bits = inputs.random_groups(801 + N, N, K, "normal")
+    qa, qw = oracle.quantize(a_bits, 32), oracle.quantize(w_bits, 32)
+    ref = oracle.gemm(*qa, *qw, 32)
+    _, _, pa = amx.quantize_prepared(dev_bf16(a_bits), False)
+    _, _, pw = amx.quantize_prepared(dev_bf16(w_bits), True)
+    assert amx.lib().amx_gemm_prepared_workspace_bytes(M, N, K, 32) > 256
+    wide = torch.full((M, N + 12), 5.0, dtype=torch.float32, device="cuda")
+    got = amx.gemm_prepared(pa, pw, M, N, K, out=wide[:, :N])                     # sliced (default workspace)
+    assert rel_fro(got.cpu().numpy(), ref) <= 1e-5
+    assert torch.all(wide[:, N:] == 5.0)
+    assert torch.equal(amx.gemm_prepared(pa, pw, M, N, K), got.contiguous())
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    one = amx.gemm_prepared(pa, pw, M, N, K, workspace=small)                     # 256 bytes: one range
+    assert rel_fro(one.cpu().numpy(), ref) <= 1e-5
+
+
 def test_fp4_path_shape_sweep():
     """Seeded sweep of ragged shapes through the fused cast and the FP4 kernel (prepared buffers pre-filled with
     0xFF, padded output), against the oracle on the oracle's own codes."""
