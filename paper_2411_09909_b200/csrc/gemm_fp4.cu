@@ -193,6 +193,7 @@ struct Params {
 
     float* C;
     int nk64, vec_store;
+    int m_fast;                  // tile order: consecutive tiles walk down M (else along N), see blk_m / blk_n
     int slices;                  // SLICED instantiation: K is cut into this many ranges, each (tile, range) a work item
     int64_t slice_stride;        //   whose partial product goes to C + range * slice_stride
     int* status;
@@ -239,7 +240,12 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     const int S = SLICED ? p.slices : 1;
     const int num_kb = (int)((p.K + BK - 1) / BK) / S;
     // Persistent CTA: tiles blockIdx.x, blockIdx.x + gridDim.x, ...; neighbouring tiles share their A rows.
-    const int64_t n_tiles = (p.N + BN - 1) / BN, total_tiles = ((p.M + BM - 1) / BM) * n_tiles * S;
+    const int64_t n_tiles = (p.N + BN - 1) / BN, m_tiles = (p.M + BM - 1) / BM, total_tiles = m_tiles * n_tiles * S;
+    // Tile order.  The CTAs work on ~148 consecutive tiles at a time; walking down M first keeps that set to a few
+    // row blocks of W (read once from DRAM, shared through L2 by the CTAs of all M blocks) plus all of A, when A is
+    // the smaller operand, and the other way round otherwise.
+    auto blk_m = [&](int64_t tile) { const int64_t t = tile / S; return p.m_fast ? t % m_tiles : t / n_tiles; };
+    auto blk_n = [&](int64_t tile) { const int64_t t = tile / S; return p.m_fast ? t / m_tiles : t % n_tiles; };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -263,7 +269,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             int it = 0;                                          // K blocks issued so far, over all tiles
             bool ok = true;
             for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int64_t m_blk = (tile / S) / n_tiles, n_blk = (tile / S) % n_tiles;
+                const int64_t m_blk = blk_m(tile), n_blk = blk_n(tile);
                 const int kb0 = (int)(tile % S) * num_kb;
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const int s = it % kStages;
@@ -297,7 +303,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         auto tile_sides = [&](int64_t tile) {
             int bits = 0;
             if (tile < total_tiles) {
-                const int64_t m0 = ((tile / S) / n_tiles) * BM, n0 = ((tile / S) % n_tiles) * BN;
+                const int64_t m0 = blk_m(tile) * BM, n0 = blk_n(tile) * BN;
 #pragma unroll
                 for (int i = 0; i < BM / 32; ++i)
                     if (m0 + i * 32 + lane < p.M) bits |= (__ldg(p.a_exp + m0 + i * 32 + lane) >> 16) & 3;
@@ -370,7 +376,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         constexpr int kBlocks = 2 * kSteps * 3;                  // per K block: A (1) + W (2 row blocks), x planes x steps
         uint4 sfv[kBlocks];
         auto fetch = [&](int64_t tile, int kb) {
-            const int64_t m_blk = (tile / S) / n_tiles, n_blk = (tile / S) % n_tiles;
+            const int64_t m_blk = blk_m(tile), n_blk = blk_n(tile);
 #pragma unroll
             for (int pl = 0; pl < 2; ++pl)
 #pragma unroll
@@ -422,7 +428,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         int t = 0;
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t) {
-            const int64_t m0 = ((tile / S) / n_tiles) * BM, n0 = ((tile / S) % n_tiles) * BN;
+            const int64_t m0 = blk_m(tile) * BM, n0 = blk_n(tile) * BN;
             float* const C_item = p.C + (SLICED ? (tile % S) * p.slice_stride : 0);
             int* w_exp = ctl->w_exp[t & 1];
             for (int i = tid_e; i < BN; i += kEpilogueWarps * 32) {
@@ -507,7 +513,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                             for (int j = 0; j < 16; ++j) s4[j & 3] += exp2_approx(fmaf(u[j], ra, -nmx));
                             sum += (s4[0] + s4[1]) + (s4[2] + s4[3]);
                         }
-                        if (m < p.M) p.part[m * (2 * n_tiles) + ((tile / S) % n_tiles) * 2 + (e >> 2)] = make_float2(mx, sum);
+                        if (m < p.M) p.part[m * (2 * n_tiles) + blk_n(tile) * 2 + (e >> 2)] = make_float2(mx, sum);
                     } else {
                         // Four 32-column groups per thread: normalise with the row's statistics {-max, 1 / sum}, round
                         // to bf16, cast.  P has no negative element: only its positive plane and scale factors exist.
@@ -685,6 +691,7 @@ int fill_params(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, 
     p.nk64 = oa.nk64;
     p.vec_store = C && aligned(C, 32) && ld_c % 8 == 0;     // 32-byte stores in the epilogue
     p.status = status;
+    p.m_fast = getenv("AMX_FP4_NFAST") ? 0 : (M <= N);
     return AMX_OK;
 }
 
