@@ -37,7 +37,7 @@ NOMINAL_HBM_GBS = 8000.0
 BYTES_PER_ELEM = 2.0 + 0.5 + 2.0 / 32.0   # bf16 read + 4-bit code + two scale bytes per 32
 # DRAM bytes (read + write) per GEMM launch, mean over the four layer shapes, from the ncu capture summarised
 # in profiles/; None until a capture of the current kernel exists.
-GEMM_DRAM_TRAFFIC_PER_LAUNCH = {"auto": 178.9e6, "fp4": 178.9e6}
+GEMM_DRAM_TRAFFIC_PER_LAUNCH = {"auto": 89.6e6, "fp4": 89.6e6}
 
 
 def measured_peaks():
