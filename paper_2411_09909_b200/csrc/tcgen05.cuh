@@ -44,7 +44,7 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
 }
 // TMA: one 2-D tile (coordinates: x = innermost, in elements of the tensor map) into shared memory;
-// completion is counted in bytes on the mbarrier.  No multicast.
+// completion is counted in bytes on the mbarrier.  Every CTA fetches its own tiles: one destination per copy.
 __device__ __forceinline__ void tma_load_2d(void* smem_dst, const void* tensor_map, int x, int y, uint64_t* b) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
                  ::"r"(smem_u32(smem_dst)), "l"(tensor_map), "r"(smem_u32(b)), "r"(x), "r"(y) : "memory");
