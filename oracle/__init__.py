@@ -52,6 +52,7 @@ def lib() -> ctypes.CDLL:
         L.amx_oracle_gemm.argtypes = [p, p, p, p, i64, i64, i64, ctypes.c_int, p, i64, p]
         L.amx_oracle_fakequant_pot_floor.argtypes = [p, i64, i64, ctypes.c_int, ctypes.c_int, p]
         L.amx_oracle_softmax_bf16.argtypes = [p, i64, i64, dbl, p]
+        L.amx_oracle_softmax_bf16_causal.argtypes = [p, i64, i64, dbl, i64, p]
         L.amx_oracle_num_threads.restype = ctypes.c_int
         _lib = L
     return _lib
@@ -177,10 +178,14 @@ def fakequant_pot_floor(x: np.ndarray, group_size: int, asym: bool) -> np.ndarra
     return out
 
 
-def softmax_bf16(S: np.ndarray, alpha: float) -> np.ndarray:
-    """Row softmax of alpha*S (fp64), rounded to bf16 bit patterns."""
+def softmax_bf16(S: np.ndarray, alpha: float, causal_row0: int | None = None) -> np.ndarray:
+    """Row softmax of alpha*S (fp64), rounded to bf16 bit patterns.  causal_row0: row r is query causal_row0 + r
+    and sees columns 0 .. causal_row0 + r only (the rest get 0)."""
     S = _c(S, np.float32)
     rows, cols = S.shape
     P = np.zeros((rows, cols), np.uint16)
-    lib().amx_oracle_softmax_bf16(_ptr(S), rows, cols, float(alpha), _ptr(P))
+    if causal_row0 is None:
+        lib().amx_oracle_softmax_bf16(_ptr(S), rows, cols, float(alpha), _ptr(P))
+    else:
+        lib().amx_oracle_softmax_bf16_causal(_ptr(S), rows, cols, float(alpha), int(causal_row0), _ptr(P))
     return P

@@ -427,6 +427,30 @@ int amx_oracle_softmax_bf16(const float *S, int64_t rows, int64_t cols, double a
     return 0;
 }
 
+/*
+ * The same with a causal mask: row r is query row0 + r and sees the keys (columns) 0 .. row0 + r only; the
+ * others get probability 0 (bf16 +0).  The paper's decoder-only models attend causally; the mask is applied to
+ * the logits before the softmax, as usual.
+ */
+int amx_oracle_softmax_bf16_causal(const float *S, int64_t rows, int64_t cols, double alpha,
+                                   int64_t row0, uint16_t *P)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        const float *s = S + r * cols;
+        int64_t seen = row0 + r + 1;
+        if (seen > cols) seen = cols;
+        double mx = -INFINITY, sum = 0.0;
+        for (int64_t c = 0; c < seen; ++c)
+            if (alpha * s[c] > mx) mx = alpha * s[c];
+        for (int64_t c = 0; c < seen; ++c)
+            sum += exp(alpha * s[c] - mx);
+        for (int64_t c = 0; c < cols; ++c)
+            P[r * cols + c] = c < seen ? double_to_bf16_rne(exp(alpha * s[c] - mx) / sum) : 0;
+    }
+    return 0;
+}
+
 int amx_oracle_num_threads(void)
 {
     int n = 1;

@@ -104,6 +104,21 @@ def test_softmax_bf16_against_scipy_and_torch_rounding():
     assert np.all(np.abs(p - ref) <= ref * 2.0 ** -8 + 1e-45)
 
 
+def test_causal_softmax_is_the_masked_softmax():
+    rng = np.random.default_rng(9)
+    S = (rng.standard_normal((24, 40)) * 10).astype(np.float32)
+    alpha = 0.25
+    got = inputs.bf16_bits_to_f32(oracle.softmax_bf16(S, alpha, causal_row0=8)).astype(np.float64)
+    masked = np.where(np.arange(40)[None, :] <= (np.arange(24)[:, None] + 8), S.astype(np.float64) * alpha, -np.inf)
+    ref = scipy.special.softmax(masked, axis=1)
+    assert np.all(got[np.isinf(masked)] == 0)
+    assert np.all(np.abs(got - ref) <= ref * 2.0 ** -8 + 1e-45)
+    # the first query (row0 = 0) sees one key only; rows that see every key equal the unmasked softmax
+    first = oracle.softmax_bf16(S[:1], alpha, causal_row0=0)
+    assert first[0, 0] == 0x3F80 and not first[0, 1:].any()
+    assert np.array_equal(oracle.softmax_bf16(S, alpha, causal_row0=39), oracle.softmax_bf16(S, alpha))
+
+
 def test_input_generators_are_seeded_and_shaped():
     a1, a2 = inputs.activation(2, 0, M=8), inputs.activation(2, 0, M=8)
     assert a1.dtype == np.uint16 and a1.shape == (8, 4096) and np.array_equal(a1, a2)
