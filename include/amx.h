@@ -77,6 +77,8 @@ typedef enum amx_status {
  * are what bounds that kernel, so this is slower than the default two launches (measured 1.05x at
  * 128 x 1024 x 1024, 1.25x at 2048 x 12288 x 4096); it is for callers that must not hold the codes. */
 #define AMX_GEMM_CAST_IN_KERNEL 0x80u
+/* extra flag for amx_attention: causal mask */
+#define AMX_ATTN_CAUSAL 0x1000u
 
 /*
  * amx_quantize - direct cast of a bf16 matrix to AMXFP4 (Sections 4.2-4.3; procedure per
@@ -214,6 +216,10 @@ int amx_softmax_quantize(const float* S, int64_t rows, int64_t cols, int64_t ld_
  *       (row sums are then taken tile by tile, so single elements of P may round to the neighbouring bf16
  *       value compared with amx_softmax_quantize on a stored S; O agrees to ~1e-5 relative)
  *   O_h = AMX(P) AMX(V_h)            groups along the key axis (V is quantized down its rows)
+ *   flags    AMX_GEMM_* kernel choice for both products, optionally | AMX_ATTN_CAUSAL: query i sees keys 0..i only
+ *            (the mask is applied to the logits before the softmax; masked entries of P are exactly 0).  On the
+ *            two-pass path the blocks of Q K^T that lie entirely after their queries, and the matching part of
+ *            P V, are not computed at all.
  *   q, k, v  bf16 [heads, L, d] contiguous;  o  out fp32 [heads, L, d]
  *   d % 32 == 0, L % 32 == 0 (group size 32 on both axes)
  *   workspace  at least amx_attention_workspace_bytes(L, d) bytes (reused head after head), 256-aligned

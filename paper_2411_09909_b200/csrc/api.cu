@@ -287,6 +287,8 @@ extern "C" size_t amx_attention_workspace_bytes(int64_t L, int64_t d) {
 
 extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_t heads, int64_t L, int64_t d,
                              uint32_t flags, float* o, void* workspace, size_t workspace_bytes, void* stream) {
+    const int causal = (flags & AMX_ATTN_CAUSAL) ? 1 : 0;
+    flags &= ~AMX_ATTN_CAUSAL;
     if (flags & ~kKernelMask) return AMX_ERR_FLAGS;
     if (heads < 0 || L <= 0 || d <= 0 || L % 32 || d % 32) return AMX_ERR_SHAPE;
     const uint32_t k_qk = pick_kernel(L, L, d, 32, flags), k_pv = pick_kernel(L, d, L, 32, flags);
@@ -334,10 +336,10 @@ extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_
             if (two_pass) {
                 // the logits never reach memory: Q K^T runs twice, its epilogues do the softmax and the cast of P
                 rc = gemm_fp4_attn_scores({w + a.pq, hc * L, chunk * L, i * L}, {w + a.pk, hc * L, chunk * L + 128, i * L}, L, d,
-                                          alpha, S, w + a.pc, w + a.ps, w + a.pp, w + a.gemm, st);
+                                          alpha, S, w + a.pc, w + a.ps, w + a.pp, w + a.gemm, st, causal);
                 if (rc == AMX_OK)
                     rc = gemm_fp4_prepared_at({w + a.pp, L, L, 0}, {w + a.pv, hc * d, chunk * d + 128, i * d}, L, d, L, oh, d,
-                                              w + a.gemm, st);
+                                              w + a.gemm, st, 256, causal);
                 if (rc != AMX_OK) return rc;
                 continue;
             }
@@ -351,13 +353,13 @@ extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_
             if (rc != AMX_OK) return rc;
             // softmax, rounding to bf16 and the cast of P in one kernel; O = AMX(P) AMX(V)
             if (k_pv == AMX_GEMM_FP4) {
-                rc = gemm_fp4_softmax_prepared(S, L, L, L, alpha, false, w + a.pc, w + a.ps, w + a.pp, st);
+                rc = gemm_fp4_softmax_prepared(S, L, L, L, alpha, false, w + a.pc, w + a.ps, w + a.pp, st, causal);
                 if (rc == AMX_OK)
                     rc = gemm_fp4_prepared_at({w + a.pp, L, L, 0}, {w + a.pv, hc * d, chunk * d + 128, i * d}, L, d, L, oh, d,
                                               w + a.gemm, st);
             } else {
                 rc = softmax_cast_rows(S, L, L, L, alpha, w + a.pc, w + a.ps, nullptr, nullptr, nullptr, nullptr, nullptr, 0, L,
-                                       st);
+                                       st, causal);
                 if (rc == AMX_OK)
                     rc = amx_gemm(w + a.pc, w + a.ps, w + a.vc + i * v_codes, w + a.vs + i * v_scales, L, d, L, 32, k_pv, oh,
                                   d, w + a.gemm, gemm_bytes, stream);

@@ -41,9 +41,9 @@ int quantize_rows_prepared(const void* x, int64_t rows, int64_t K, uint8_t* code
 // output only.  gemm_fp4_softmax_prepared lays the prepared operand out like gemm_fp4_quantize_prepared.
 int softmax_cast_rows(const float* S, int64_t rows, int64_t cols, int64_t ld_s, float alpha, uint8_t* codes,
                       uint8_t* scales, void* pos, void* neg, uint8_t* sf_pos, uint8_t* sf_neg, int* row_exp, int nk64,
-                      int64_t padded_rows, cudaStream_t st);
+                      int64_t padded_rows, cudaStream_t st, int causal = 0);
 int gemm_fp4_softmax_prepared(const float* S, int64_t rows, int64_t cols, int64_t ld_s, float alpha, bool is_weight,
-                              uint8_t* codes, uint8_t* scales, void* prepared, cudaStream_t st);
+                              uint8_t* codes, uint8_t* scales, void* prepared, cudaStream_t st, int causal = 0);
 // A prepared operand that stacks several matrices row-wise (rows_total rows, laid out for layout_rows >=
 // rows_total rows) and the first row of the one to multiply; row0 % 128 == 0.  A right-hand operand whose 256-row
 // tiles can reach past rows_total needs layout_rows >= rows_total + 128.
@@ -52,7 +52,8 @@ struct Fp4Operand {
     int64_t rows_total, layout_rows, row0;
 };
 int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
-                         int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes = 256);
+                         int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes = 256,
+                         int causal_pv = 0 /* 1: the product P V of causal attention (A = P, square) */);
 // workspace that lets the kernel cut K into ranges for products with few output tiles (256 bytes otherwise)
 size_t gemm_fp4_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K);
 // C[m][n] = sum over `slices` partial products [slices][M][N], in slice order (defined with the bf16-decode kernel)
@@ -61,7 +62,8 @@ int reduce_slices(const float* part, int slices, int64_t M, int64_t N, float* C,
 // memory; L % 256 == 0; scratch of gemm_fp4_attn_scratch_bytes(L) bytes.
 size_t gemm_fp4_attn_scratch_bytes(int64_t L);
 int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, int64_t d, float alpha, void* scratch,
-                         uint8_t* p_codes, uint8_t* p_scales, void* p_prepared, void* workspace, cudaStream_t st);
+                         uint8_t* p_codes, uint8_t* p_scales, void* p_prepared, void* workspace, cudaStream_t st,
+                         int causal = 0);
 int quantize_cols_batched(const void* x, int64_t batch, int64_t R, int64_t C, uint8_t* codes, uint8_t* scales,
                           cudaStream_t st);
 int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,

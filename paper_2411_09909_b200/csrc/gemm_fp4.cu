@@ -193,6 +193,10 @@ struct Params {
 
     float* C;
     int nk64, vec_store;
+    int causal;                  // attention with a causal mask: 1 = the tile is a block of logits Q K^T (tiles whose
+                                 // keys all lie after their queries are skipped, the epilogue masks the diagonal
+                                 // ones); 2 = the product P V (K blocks after the tile's last query row hold only
+                                 // zeros of P and are skipped)
     int m_fast;                  // tile order: consecutive tiles walk down M (else along N), see blk_m / blk_n
     int slices;                  // SLICED instantiation: K is cut into this many ranges, each (tile, range) a work item
     int64_t slice_stride;        //   whose partial product goes to C + range * slice_stride
@@ -225,7 +229,7 @@ __device__ __forceinline__ void store_row16(float* out, const float (&f)[16], bo
     }
 }
 
-template <int BK_, int EPI = kEpiStore, bool SLICED = false>
+template <int BK_, int EPI = kEpiStore, bool SLICED = false, bool CAUSAL = false>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w, const Params p) {
     using C_ = Cfg<BK_>;
@@ -246,6 +250,13 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     // the smaller operand, and the other way round otherwise.
     auto blk_m = [&](int64_t tile) { const int64_t t = tile / S; return p.m_fast ? t % m_tiles : t / n_tiles; };
     auto blk_n = [&](int64_t tile) { const int64_t t = tile / S; return p.m_fast ? t / m_tiles : t % n_tiles; };
+    // K blocks of a tile (of an item): all of them, fewer or none under a causal mask (see Params::causal)
+    auto nkb_of = [&](int64_t tile) -> int {
+        if (!CAUSAL || p.causal == 0) return num_kb;
+        const int64_t last_row = blk_m(tile) * BM + BM - 1;
+        if (p.causal == 1) return blk_n(tile) * BN > last_row ? 0 : num_kb;
+        return (int)min((int64_t)num_kb, (last_row + BK) / BK);
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -270,8 +281,8 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             bool ok = true;
             for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
                 const int64_t m_blk = blk_m(tile), n_blk = blk_n(tile);
-                const int kb0 = (int)(tile % S) * num_kb;
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                const int kb0 = (int)(tile % S) * num_kb, nkb = nkb_of(tile);
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % kStages;
                     if (it >= kStages && !mbar_wait(&ctl->empty[s], ((it / kStages) - 1) & 1, &ctl->abort, p.status)) {
                         ok = false;
@@ -302,7 +313,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         // next tile are fetched while the current one runs.
         auto tile_sides = [&](int64_t tile) {
             int bits = 0;
-            if (tile < total_tiles) {
+            if (tile < total_tiles && nkb_of(tile) > 0) {            // a skipped tile costs no load latency
                 const int64_t m0 = blk_m(tile) * BM, n0 = blk_n(tile) * BN;
 #pragma unroll
                 for (int i = 0; i < BM / 32; ++i)
@@ -314,9 +325,11 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             return bits;
         };
         int sides_next = tile_sides(blockIdx.x);
-        for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t) {
+        for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
             int sides = __reduce_or_sync(0xFFFFFFFFu, sides_next);   // bit 0/1: A has +/-, bit 2/3: W has +/-
             sides_next = tile_sides(tile + gridDim.x);
+            const int nkb = nkb_of(tile);
+            if (nkb == 0) continue;                              // masked out entirely: no accumulator, no epilogue
             if (!(sides & 3)) sides |= 1;                        // an all-zero operand: one product, which zeroes the tile
             if (!(sides & 12)) sides |= 4;
             const int n_mma = ((sides & 1) + ((sides >> 1) & 1)) * (((sides >> 2) & 1) + ((sides >> 3) & 1)) * kSteps;
@@ -324,7 +337,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             if (t > 0) ok = mbar_wait(&ctl->accum_empty, (t - 1) & 1, &ctl->abort, p.status);
             tc_fence_after();
             uint32_t accumulate = 0;
-            for (int kb = 0; kb < num_kb && ok; ++kb, ++it) {
+            for (int kb = 0; kb < nkb && ok; ++kb, ++it) {
                 const int s = it % kStages;
                 // tiles landed (TMA byte count) and scale factors stored (four warp arrivals); usually already
                 // seen by the poll that was slipped between the previous block's MMAs
@@ -362,6 +375,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             }
             if (ok && elect_one()) mma_commit(&ctl->accum_full);
             __syncwarp();
+            ++t;
         }
     } else if (warp < 2 + kSfWarps) {
         // -------------------------------------------------------------- scale factors
@@ -392,7 +406,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         // this group's K blocks, in order, over all tiles: (tile, kb) with global index it = group, group + 2, ...
         int64_t tile = blockIdx.x;
         int kb = group;
-        while (tile < total_tiles && kb >= num_kb) { kb -= num_kb; tile += gridDim.x; }
+        while (tile < total_tiles && kb >= nkb_of(tile)) { kb -= nkb_of(tile); tile += gridDim.x; }
         int it = group;
         bool ok = true;
         if (tile < total_tiles) fetch(tile, kb);
@@ -412,7 +426,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             // next K block of this group
             it += kSfGroups;
             kb += kSfGroups;
-            while (tile < total_tiles && kb >= num_kb) { kb -= num_kb; tile += gridDim.x; }
+            while (tile < total_tiles && kb >= nkb_of(tile)) { kb -= nkb_of(tile); tile += gridDim.x; }
             if (tile < total_tiles) fetch(tile, kb);             // in flight during the wait below
             tmem_st_wait();
             tc_fence_before();
@@ -427,7 +441,8 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         const int tid_e = threadIdx.x - (2 + kSfWarps) * 32;
         int t = 0;
         bool ok = true;
-        for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t) {
+        for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            if (nkb_of(tile) == 0) continue;
             const int64_t m0 = blk_m(tile) * BM, n0 = blk_n(tile) * BN;
             float* const C_item = p.C + (SLICED ? (tile % S) * p.slice_stride : 0);
             int* w_exp = ctl->w_exp[t & 1];
@@ -486,6 +501,11 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                             u[j + 2] = __uint_as_float(v[buf][j + 2]) * k.z;
                             u[j + 3] = __uint_as_float(v[buf][j + 3]) * k.w;
                         }
+                        if (CAUSAL && p.causal && n0 + col_base + c + 15 > m) {      // keys after this query: masked out
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                if (n0 + col_base + c + j > m) u[j] = -INFINITY;
+                        }
                     };
                     auto exp2_approx = [](float y) {
                         float r;
@@ -506,11 +526,14 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                             for (int j = 4; j < 16; ++j) c4[j & 3] = fmaxf(c4[j & 3], u[j]);
                             const float cm = fmaxf(fmaxf(c4[0], c4[1]), fmaxf(c4[2], c4[3]));
                             const float nmx = fmaxf(mx, cm * ra);
-                            sum *= exp2_approx(mx - nmx);                // 2^(-inf) = 0 on the first chunk
+                            // 2^(-inf) = 0 on the first chunk; a maximum still at -inf (everything masked so far)
+                            // must not meet itself in a difference
+                            const float ref = nmx == -INFINITY ? 0.f : nmx;
+                            sum *= exp2_approx(mx - ref);
                             mx = nmx;
                             float s4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) s4[j & 3] += exp2_approx(fmaf(u[j], ra, -nmx));
+                            for (int j = 0; j < 16; ++j) s4[j & 3] += exp2_approx(fmaf(u[j], ra, -ref));
                             sum += (s4[0] + s4[1]) + (s4[2] + s4[3]);
                         }
                         if (m < p.M) p.part[m * (2 * n_tiles) + blk_n(tile) * 2 + (e >> 2)] = make_float2(mx, sum);
@@ -548,6 +571,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&ctl->accum_empty);
             }
+            ++t;
         }
     }
     tc_fence_before();
@@ -632,13 +656,13 @@ size_t gemm_fp4_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 
 namespace {
 
-template <int BK_, int EPI = kEpiStore, bool SLICED = false>
+template <int BK_, int EPI = kEpiStore, bool SLICED = false, bool CAUSAL = false>
 int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, const OperandLayout& ow, int64_t a_rows,
                int64_t w_rows, Params p, int dev, cudaStream_t st) {
     using C_ = Cfg<BK_>;
     static bool configured[64] = {};
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(gemm_fp4_kernel<BK_, EPI, SLICED>, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(gemm_fp4_kernel<BK_, EPI, SLICED, CAUSAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::kSmemBytes) != cudaSuccess)
             return AMX_ERR_CUDA;
         configured[dev] = true;
     }
@@ -650,7 +674,7 @@ int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, co
         return AMX_ERR_CUDA;
     const int64_t tiles = ((p.N + BN - 1) / BN) * ((p.M + BM - 1) / BM) * (SLICED ? p.slices : 1);
     const unsigned grid = (unsigned)(tiles < sm_count[dev] ? tiles : sm_count[dev]);   // one persistent CTA per SM
-    gemm_fp4_kernel<BK_, EPI, SLICED><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_a, tm_w, p);
+    gemm_fp4_kernel<BK_, EPI, SLICED, CAUSAL><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_a, tm_w, p);
     return launch_status();
 }
 
@@ -698,12 +722,14 @@ int fill_params(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, 
 // One warp per query row: the row's softmax statistics from the per-tile partial ones, and the row word of
 // the cast attention map (its largest element is exp(0) / sum, whose group has the row's largest scale).
 __global__ void __launch_bounds__(256)
-attn_row_reduce_kernel(const float2* __restrict__ part, int n_parts, int64_t L, float2* __restrict__ rowstat,
-                       int* __restrict__ p_kmax, int* __restrict__ p_row_word) {
+attn_row_reduce_kernel(const float2* __restrict__ part, int n_parts_all, int64_t L, int causal,
+                       float2* __restrict__ rowstat, int* __restrict__ p_kmax, int* __restrict__ p_row_word) {
     const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= L) return;
-    const float2* pr = part + row * n_parts;          // {max, sum of 2^(t - max)} per half tile, base-2 units
+    const float2* pr = part + row * n_parts_all;      // {max, sum of 2^(t - max)} per half tile, base-2 units
+    // causal: the half tiles (128 keys each) that start after this query were skipped and hold nothing
+    const int n_parts = causal ? min(n_parts_all, (int)(row / 128) + 1) : n_parts_all;
     float mx = -INFINITY;
     for (int j = lane; j < n_parts; j += 32) mx = fmaxf(mx, pr[j].x);
 #pragma unroll
@@ -745,15 +771,17 @@ size_t gemm_fp4_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 // The GEMM proper on two prepared operands (each laid out by operand_layout()), or on row ranges of them.
 // workspace_bytes >= gemm_fp4_prepared_workspace_bytes() enables the K ranges; 256 bytes always suffice.
 int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
-                         int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes) {
+                         int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes, int causal_pv) {
     Params p;
     OperandLayout oa, ow;
     int dev;
     const int rc = fill_params(a, w, M, N, K, C, ld_c, workspace, st, p, oa, ow, dev);
     if (rc != AMX_OK) return rc;
+    p.causal = causal_pv ? 2 : 0;
     const uint8_t* pa = static_cast<const uint8_t*>(a.prepared);
     const uint8_t* pw = static_cast<const uint8_t*>(w.prepared);
     const int slices = gemm_fp4_slices(M, N, K);
+    if (causal_pv) return launch_fp4<128, kEpiStore, false, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
     if (slices > 1 && fp4_block_k() == 128 && workspace_bytes >= gemm_fp4_prepared_workspace_bytes(M, N, K)) {
         float* part = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 256);
         p.C = part;
@@ -776,7 +804,8 @@ size_t gemm_fp4_attn_scratch_bytes(int64_t L) {
     return up256((size_t)L * (2 * (L / BN)) * sizeof(float2)) + up256((size_t)L * sizeof(float2)) + up256((size_t)L * 4);
 }
 int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, int64_t d, float alpha, void* scratch,
-                         uint8_t* p_codes, uint8_t* p_scales, void* p_prepared, void* workspace, cudaStream_t st) {
+                         uint8_t* p_codes, uint8_t* p_scales, void* p_prepared, void* workspace, cudaStream_t st,
+                         int causal) {
     if (L % BN) return AMX_ERR_SHAPE;
     Params p;
     OperandLayout oq, ok_;
@@ -793,6 +822,7 @@ int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, in
     const OperandLayout op = operand_layout(L, L, BM);
     uint8_t* pp = static_cast<uint8_t*>(p_prepared);
     p.alpha = alpha;
+    p.causal = causal ? 1 : 0;
     p.part = part;
     p.rowstat = rowstat;
     p.p_kmax = p_kmax;
@@ -801,19 +831,21 @@ int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, in
     p.p_pos = reinterpret_cast<uint4*>(pp);
     p.p_sf = pp + 2 * op.plane;
     p.p_nk64 = op.nk64;
-    rc = launch_fp4<128, kEpiStats>(pq, pk, oq, ok_, q.rows_total, k.rows_total, p, dev, st);
+    rc = causal ? launch_fp4<128, kEpiStats, false, true>(pq, pk, oq, ok_, q.rows_total, k.rows_total, p, dev, st)
+                : launch_fp4<128, kEpiStats>(pq, pk, oq, ok_, q.rows_total, k.rows_total, p, dev, st);
     if (rc != AMX_OK) return rc;
-    attn_row_reduce_kernel<<<(unsigned)((L + 7) / 8), 256, 0, st>>>(part, n_parts, L, rowstat, p_kmax,
+    attn_row_reduce_kernel<<<(unsigned)((L + 7) / 8), 256, 0, st>>>(part, n_parts, L, causal, rowstat, p_kmax,
                                                                         reinterpret_cast<int*>(pp + 2 * op.plane + 2 * op.sf));
     rc = launch_status();
     if (rc != AMX_OK) return rc;
-    return launch_fp4<128, kEpiCast>(pq, pk, oq, ok_, q.rows_total, k.rows_total, p, dev, st);
+    return causal ? launch_fp4<128, kEpiCast, false, true>(pq, pk, oq, ok_, q.rows_total, k.rows_total, p, dev, st)
+                  : launch_fp4<128, kEpiCast>(pq, pk, oq, ok_, q.rows_total, k.rows_total, p, dev, st);
 }
 
 int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K, float* C,
                       int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes) {
     return gemm_fp4_prepared_at({a_prepared, M, M, 0}, {w_prepared, N, N, 0}, M, N, K, C, ld_c, workspace, st,
-                                workspace_bytes);
+                                workspace_bytes, 0);
 }
 
 // Size of a prepared operand: as the A operand (rows padded to 128) or the W operand (rows padded to 256).
@@ -832,12 +864,12 @@ int gemm_fp4_quantize_prepared(const void* x, int64_t rows, int64_t K, bool is_w
 }
 
 int gemm_fp4_softmax_prepared(const float* S, int64_t rows, int64_t cols, int64_t ld_s, float alpha, bool is_weight,
-                              uint8_t* codes, uint8_t* scales, void* prepared, cudaStream_t st) {
+                              uint8_t* codes, uint8_t* scales, void* prepared, cudaStream_t st, int causal) {
     const OperandLayout o = operand_layout(rows, cols, is_weight ? BN : BM);
     uint8_t* base = static_cast<uint8_t*>(prepared);
     return softmax_cast_rows(S, rows, cols, ld_s, alpha, codes, scales, base, base + o.plane, base + 2 * o.plane,
                              base + 2 * o.plane + o.sf, reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf), o.nk64,
-                             o.row_blocks * 128, st);
+                             o.row_blocks * 128, st, causal);
 }
 
 int gemm_fp4_prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, bool is_weight,

@@ -192,7 +192,7 @@ cast_prepared_kernel(const uint4* __restrict__ x, int64_t R, int G, uint4* __res
 // CACHED: the row has at most kT groups, so each thread keeps its one group in registers between the passes.
 template <bool CACHED>
 __global__ void __launch_bounds__(softmax::kT)
-softmax_cast_kernel(const float* __restrict__ S, int64_t R, int G, int64_t ld_s, float alpha, int vec,
+softmax_cast_kernel(const float* __restrict__ S, int64_t R, int G, int64_t ld_s, float alpha, int vec, int causal,
                     uint4* __restrict__ codes, uint16_t* __restrict__ scales, uint4* __restrict__ pos,
                     uint4* __restrict__ neg, uint8_t* __restrict__ sf_pos, uint8_t* __restrict__ sf_neg,
                     int* __restrict__ row_exp, int nk64) {
@@ -206,9 +206,10 @@ softmax_cast_kernel(const float* __restrict__ S, int64_t R, int G, int64_t ld_s,
     if (row_live) {
         const float* s = S + row * ld_s;
         const int64_t cols = (int64_t)G * 32, v_row = row * G;
+        const int64_t seen = causal ? min(cols, row + 1) : cols;     // causal: query `row` sees keys 0 .. row
         if (CACHED) {
             float e[32];
-            const float sum = softmax::cached_row_exp(s, G, vec != 0, alpha, sh, e);
+            const float sum = softmax::cached_row_exp(s, G, vec != 0, alpha, sh, e, seen);
             if (gx < G) {
                 uint32_t w[16];
                 softmax::normalised_group_e(e, sum, w);
@@ -217,11 +218,11 @@ softmax_cast_kernel(const float* __restrict__ S, int64_t R, int G, int64_t ld_s,
             }
         } else {
             float mx, sum;
-            softmax::row_stats(s, cols, vec != 0, alpha, sh, mx, sum);
+            softmax::row_stats(s, cols, vec != 0, alpha, sh, mx, sum, seen);
             for (int g = gx; g < G; g += softmax::kT) {
                 float t[32];
                 uint32_t w[16];
-                softmax::load_group(s, g, cols, vec != 0, alpha, t);
+                softmax::load_group(s, g, cols, vec != 0, alpha, t, seen);
                 softmax::normalised_group(t, mx, sum, w);
                 const uint32_t sc = emit_group(w, v_row + g, codes, scales, pos, neg);
                 if (g == gx) sc_first = sc;
@@ -277,12 +278,12 @@ int quantize_rows_prepared(const void* x, int64_t rows, int64_t K, uint8_t* code
 // pos == nullptr only the canonical codes and scales are written.
 int softmax_cast_rows(const float* S, int64_t rows, int64_t cols, int64_t ld_s, float alpha, uint8_t* codes,
                       uint8_t* scales, void* pos, void* neg, uint8_t* sf_pos, uint8_t* sf_neg, int* row_exp, int nk64,
-                      int64_t padded_rows, cudaStream_t st) {
+                      int64_t padded_rows, cudaStream_t st, int causal) {
     const int64_t G = cols / 32, blocks = pos ? padded_rows : rows;
     if (blocks > 0x7FFFFFFF || G > 0x7FFFFFFF / 32) return AMX_ERR_SHAPE;
     const int vec = aligned(S, 16) && ld_s % 4 == 0;
     auto* kernel = G <= softmax::kT ? softmax_cast_kernel<true> : softmax_cast_kernel<false>;
-    kernel<<<(unsigned)blocks, softmax::kT, 0, st>>>(S, rows, (int)G, ld_s, alpha, vec, reinterpret_cast<uint4*>(codes),
+    kernel<<<(unsigned)blocks, softmax::kT, 0, st>>>(S, rows, (int)G, ld_s, alpha, vec, causal, reinterpret_cast<uint4*>(codes),
                                                      reinterpret_cast<uint16_t*>(scales), reinterpret_cast<uint4*>(pos),
                                                      reinterpret_cast<uint4*>(neg), sf_pos, sf_neg, row_exp, nk64);
     return launch_status();

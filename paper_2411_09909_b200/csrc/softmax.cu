@@ -30,7 +30,7 @@ softmax_bf16_cached_kernel(const float* __restrict__ S, int G, int64_t ld_s, flo
                            int64_t ld_p, int vec_in, int vec_out) {
     __shared__ float sh[kT / 32];
     float e[32];
-    const float sum = cached_row_exp(S + (int64_t)blockIdx.x * ld_s, G, vec_in != 0, alpha, sh, e);
+    const float sum = cached_row_exp(S + (int64_t)blockIdx.x * ld_s, G, vec_in != 0, alpha, sh, e, (int64_t)G * 32);
     if ((int)threadIdx.x < G) {
         uint32_t w[16];
         normalised_group_e(e, sum, w);
@@ -45,12 +45,12 @@ softmax_bf16_kernel(const float* __restrict__ S, int64_t cols, int64_t ld_s, flo
     const float* s = S + (int64_t)blockIdx.x * ld_s;
     uint16_t* p = P + (int64_t)blockIdx.x * ld_p;
     float mx, sum;
-    row_stats(s, cols, vec_in != 0, alpha, sh, mx, sum);
+    row_stats(s, cols, vec_in != 0, alpha, sh, mx, sum, cols);
     const int64_t G = (cols + 31) / 32;
     for (int64_t g = threadIdx.x; g < G; g += kT) {
         float t[32];
         uint32_t w[16];
-        load_group(s, g, cols, vec_in != 0, alpha, t);
+        load_group(s, g, cols, vec_in != 0, alpha, t, cols);
         normalised_group(t, mx, sum, w);
         store_group(p, g, cols, vec_out != 0, w);
     }

@@ -43,9 +43,11 @@ __device__ __forceinline__ float exp_rel(float t, float neg_mx_l2e) {
 
 // alpha * s for the 32 columns of group g of a row; -inf past the last column (contributes exp() = 0).
 // vec: the row is 16-byte aligned and holds whole groups, so the group is read with eight 16-byte loads.
+// seen: columns from `seen` on are masked (a causal row sees its own and earlier keys only): -inf as well.
 __device__ __forceinline__ void load_group(const float* __restrict__ s, int64_t g, int64_t cols, bool vec, float alpha,
-                                           float (&t)[32]) {
-    if (vec) {
+                                           float (&t)[32], int64_t seen) {
+    if (seen < cols) cols = seen;
+    if (vec && (g + 1) * 32 <= cols) {
         const float4* p = reinterpret_cast<const float4*>(s + g * 32);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -64,9 +66,9 @@ __device__ __forceinline__ void load_group(const float* __restrict__ s, int64_t 
 // Softmax of a row of at most kT groups with the thread's group kept in registers: on return e holds
 // exp(alpha * s - max) of the thread's own group (zeros for a thread without one); returns the row sum.
 __device__ __forceinline__ float cached_row_exp(const float* __restrict__ s, int G, bool vec, float alpha, float* sh,
-                                                float (&e)[32]) {
+                                                float (&e)[32], int64_t seen) {
     if ((int)threadIdx.x < G) {
-        load_group(s, threadIdx.x, (int64_t)G * 32, vec, alpha, e);
+        load_group(s, threadIdx.x, (int64_t)G * 32, vec, alpha, e, seen);
     } else {
 #pragma unroll
         for (int i = 0; i < 32; ++i) e[i] = -INFINITY;
@@ -86,12 +88,12 @@ __device__ __forceinline__ float cached_row_exp(const float* __restrict__ s, int
 
 // Row maximum and the sum of exp(alpha * s - max) for the row this block owns.
 __device__ __forceinline__ void row_stats(const float* __restrict__ s, int64_t cols, bool vec, float alpha, float* sh,
-                                          float& mx, float& sum) {
+                                          float& mx, float& sum, int64_t seen) {
     const int64_t G = (cols + 31) / 32;
     float t[32];
     mx = -INFINITY;
     for (int64_t g = threadIdx.x; g < G; g += kT) {
-        load_group(s, g, cols, vec, alpha, t);
+        load_group(s, g, cols, vec, alpha, t, seen);
 #pragma unroll
         for (int i = 0; i < 32; ++i) mx = fmaxf(mx, t[i]);
     }
@@ -99,7 +101,7 @@ __device__ __forceinline__ void row_stats(const float* __restrict__ s, int64_t c
     sum = 0.f;
     const float nm = neg_max_log2e(mx);
     for (int64_t g = threadIdx.x; g < G; g += kT) {
-        load_group(s, g, cols, vec, alpha, t);
+        load_group(s, g, cols, vec, alpha, t, seen);
 #pragma unroll
         for (int i = 0; i < 32; ++i) sum += exp_rel(t[i], nm);
     }

@@ -65,6 +65,8 @@ def test_host_detected_argument_errors(L):
     assert L.amx_quant_gemm(fake, 64, fake, fake, 4, 4, 64, 32, 0x80, fake, 4, fake, 4096, None) == -5   # cast-in-kernel
     assert L.amx_quant_gemm(fake, 64, fake, fake, 4, 4, 64, 32, 0xC0, fake, 4, fake, 4096, None) == -5   # needs the TC kernel
     assert L.amx_gemm(fake, fake, fake, fake, 4, 4, 64, 32, 0xA0, fake, 4, None, 0, None) == -5          # not an amx_gemm flag
+    assert L.amx_attention(fake, fake, fake, 1, 64, 64, 0x2000, fake, fake, 1 << 30, None) == -5           # unknown flag
+    assert L.amx_attention(fake, fake, fake, 1, 48, 64, 0x1000, fake, fake, 1 << 30, None) == -2           # L % 32
     assert L.amx_softmax_bf16(fake, 4, 0, 0, 1.0, fake, 0, None) == -2
     assert L.amx_softmax_quantize(fake, 4, 48, 48, ctypes.c_float(1.0), fake, fake, 0, None, 0, None) == -2   # cols % 32
     assert L.amx_softmax_quantize(fake, 4, 64, 32, ctypes.c_float(1.0), fake, fake, 0, None, 0, None) == -2   # ld < cols

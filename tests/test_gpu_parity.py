@@ -527,6 +527,26 @@ def test_attention_all_heads_entry_point_matches_per_head_pipeline(heads, seq, f
             assert torch.equal(O[h], Oh), h
 
 
+@pytest.mark.parametrize("heads,seq,flags", [(2, 192, amx.GEMM_AUTO),        # stored logits, small-product kernel
+                                             (1, 320, amx.GEMM_FP4),         # stored logits, FP4 kernel
+                                             (2, 512, amx.GEMM_FP4),         # two-pass scores, tiles skipped
+                                             (1, 1024, amx.GEMM_AUTO)])
+def test_attention_causal_against_oracle_pipeline(heads, seq, flags):
+    """Causal attention (query i sees keys 0..i) against the all-CPU pipeline with the mask applied before the
+    softmax, every query row; the first query returns V's first row as quantized, times the quantized 1."""
+    qb, kb, vb = inputs.attention_qkv(heads=heads, seq=seq)
+    O = amx.attention_heads(dev_bf16(qb), dev_bf16(kb), dev_bf16(vb), flags=flags | amx.ATTN_CAUSAL).cpu().numpy()
+    assert np.all(np.isfinite(O))
+    for h in range(heads):
+        S = oracle.gemm(*oracle.quantize(qb[h], 32), *oracle.quantize(kb[h], 32), 32)
+        P = oracle.softmax_bf16(S, 128 ** -0.5, causal_row0=0)
+        vq = oracle.quantize(np.ascontiguousarray(vb[h].T), 32)
+        ref = oracle.gemm(*oracle.quantize(P, 32), *vq, 32)
+        assert rel_fro(O[h], ref) <= GEMM_TOL, h
+        # the first query sees one key: P = 1 there, which AMXFP4 stores as 6 x 0.15625 (scale nearest to 1/6)
+        assert np.allclose(O[h][0], 0.9375 * oracle.dequantize(*vq, 32)[:, 0], rtol=1e-6, atol=0)
+
+
 def test_attention_two_pass_against_oracle_pipeline():
     """Attention with the softmax and the cast of P in the epilogue of Q K^T (FP4 kernel, sequence a multiple of
     256): output against the all-CPU pipeline, every query row."""
