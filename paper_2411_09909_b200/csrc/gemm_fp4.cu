@@ -248,8 +248,16 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     // Tile order.  The CTAs work on ~148 consecutive tiles at a time; walking down M first keeps that set to a few
     // row blocks of W (read once from DRAM, shared through L2 by the CTAs of all M blocks) plus all of A, when A is
     // the smaller operand, and the other way round otherwise.
-    auto blk_m = [&](int64_t tile) { const int64_t t = tile / S; return p.m_fast ? t % m_tiles : t / n_tiles; };
-    auto blk_n = [&](int64_t tile) { const int64_t t = tile / S; return p.m_fast ? t / m_tiles : t % n_tiles; };
+    // (one 32-bit division per call: the host rejects products with 2^31 tiles or more)
+    const uint32_t fast_dim = (uint32_t)(p.m_fast ? m_tiles : n_tiles);
+    auto blk_m = [&](int64_t tile) -> int64_t {
+        const uint32_t t = (uint32_t)tile / (uint32_t)S, q = t / fast_dim;
+        return p.m_fast ? t - q * fast_dim : q;
+    };
+    auto blk_n = [&](int64_t tile) -> int64_t {
+        const uint32_t t = (uint32_t)tile / (uint32_t)S, q = t / fast_dim;
+        return p.m_fast ? q : t - q * fast_dim;
+    };
     // K blocks of a tile (of an item): all of them, fewer or none under a causal mask (see Params::causal)
     auto nkb_of = [&](int64_t tile) -> int {
         if (!CAUSAL || p.causal == 0) return num_kb;
@@ -695,6 +703,7 @@ int fill_params(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, 
                 void* workspace, cudaStream_t st, Params& p, OperandLayout& oa, OperandLayout& ow, int& dev) {
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AMX_ERR_CUDA;
     if (a.row0 % 128 || w.row0 % 128) return AMX_ERR_SHAPE;
+    if (((M + BM - 1) / BM) * ((N + BN - 1) / BN) >= (1ll << 27)) return AMX_ERR_SHAPE;   // tile indices are 32-bit
     oa = operand_layout(a.layout_rows, K, BM);
     ow = operand_layout(w.layout_rows, K, BN);
     const uint8_t* pa = static_cast<const uint8_t*>(a.prepared);
