@@ -244,17 +244,33 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     const int S = SLICED ? p.slices : 1;
     const int num_kb = (int)((p.K + BK - 1) / BK) / S;
     // Persistent CTA: tiles blockIdx.x, blockIdx.x + gridDim.x, ...; neighbouring tiles share their A rows.
-    const int64_t n_tiles = (p.N + BN - 1) / BN, m_tiles = (p.M + BM - 1) / BM, total_tiles = m_tiles * n_tiles * S;
+    const int64_t n_tiles = (p.N + BN - 1) / BN, m_tiles = (p.M + BM - 1) / BM;
+    // Causal logits (square, keys after the queries masked): only the tiles on or below the diagonal exist.  Row
+    // block m has the column blocks 0 .. m/2 (a tile is 128 queries x 256 keys), so f(m) = tiles before row
+    // block m is j(j+1) for m = 2j and (j+1)^2 for m = 2j+1; the work items enumerate exactly those tiles, which
+    // keeps the persistent CTAs evenly loaded.
+    const bool compact = CAUSAL && p.causal == 1;
+    const int64_t half = m_tiles / 2;
+    const int64_t total_tiles = compact ? ((m_tiles & 1) ? (half + 1) * (half + 1) : half * (half + 1)) : m_tiles * n_tiles * S;
+    auto compact_mn = [&](uint32_t c, uint32_t& m, uint32_t& n) {
+        uint32_t j = (uint32_t)((sqrtf(4.0f * (float)c + 1.0f) - 1.0f) * 0.5f);
+        while (j * (j + 1) > c) --j;                      // the float estimate can be off by one
+        while ((j + 1) * (j + 2) <= c) ++j;
+        if (c < (j + 1) * (j + 1)) { m = 2 * j; n = c - j * (j + 1); }
+        else { m = 2 * j + 1; n = c - (j + 1) * (j + 1); }
+    };
     // Tile order.  The CTAs work on ~148 consecutive tiles at a time; walking down M first keeps that set to a few
     // row blocks of W (read once from DRAM, shared through L2 by the CTAs of all M blocks) plus all of A, when A is
     // the smaller operand, and the other way round otherwise.
     // (one 32-bit division per call: the host rejects products with 2^31 tiles or more)
     const uint32_t fast_dim = (uint32_t)(p.m_fast ? m_tiles : n_tiles);
     auto blk_m = [&](int64_t tile) -> int64_t {
+        if (compact) { uint32_t m, n; compact_mn((uint32_t)tile, m, n); return m; }
         const uint32_t t = (uint32_t)tile / (uint32_t)S, q = t / fast_dim;
         return p.m_fast ? t - q * fast_dim : q;
     };
     auto blk_n = [&](int64_t tile) -> int64_t {
+        if (compact) { uint32_t m, n; compact_mn((uint32_t)tile, m, n); return n; }
         const uint32_t t = (uint32_t)tile / (uint32_t)S, q = t / fast_dim;
         return p.m_fast ? q : t - q * fast_dim;
     };
@@ -262,7 +278,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     auto nkb_of = [&](int64_t tile) -> int {
         if (!CAUSAL || p.causal == 0) return num_kb;
         const int64_t last_row = blk_m(tile) * BM + BM - 1;
-        if (p.causal == 1) return blk_n(tile) * BN > last_row ? 0 : num_kb;
+        if (p.causal == 1) return num_kb;                 // the enumeration holds no masked tile
         return (int)min((int64_t)num_kb, (last_row + BK) / BK);
     };
 
