@@ -144,7 +144,7 @@ prepare_operand_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restr
         for (int64_t i = threadIdx.x; i < n_vec; i += 256) {
             const uint4 w = __ldg(src + i);
             const uint32_t v[4] = {w.x, w.y, w.z, w.w};
-            const uint32_t keep = unsplit_s[i / G] ? 0u : 0xFFFFFFFFu;
+            const uint32_t keep = unsplit_s[(int)i / (int)G] ? 0u : 0xFFFFFFFFu;   // i < 8 rows x G: 32-bit division
             uint32_t p[4], n[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
