@@ -35,6 +35,7 @@ GS = 32
 NOMINAL_FP4_TFLOPS = 9000.0      # NVIDIA's dense FP4 figure for one B200 (HGX B200 data sheet)
 NOMINAL_HBM_GBS = 8000.0
 BYTES_PER_ELEM = 2.0 + 0.5 + 2.0 / 32.0   # bf16 read + 4-bit code + two scale bytes per 32
+MOVED_BYTES_PER_ELEM = BYTES_PER_ELEM + 1.0 + 4.0 / 32.0   # + two sign planes + four scale-factor bytes per 32
 # DRAM bytes (read + write) per GEMM launch, mean over the four layer shapes, from the ncu capture summarised
 # in profiles/; None until a capture of the current kernel exists.
 GEMM_DRAM_TRAFFIC_PER_LAUNCH = {"auto": 89.6e6, "fp4": 89.6e6}
@@ -651,9 +652,13 @@ def run_ours(args):
         "quantize": {"gb_per_s": quant_gbs, "pct_of_nominal_hbm_8TBs": 100.0 * quant_gbs / NOMINAL_HBM_GBS,
                      "frac_of_measured_copy": quant_gbs / peaks["hbm_gbs"], "bytes_per_element": BYTES_PER_ELEM,
                      "ms_per_step": q_ms / args.steps, "large_tensor": quant_large,
-                     "note": ("GB/s counts the canonical bytes only; the step's casts also write the GEMM-ready sign "
-                              "planes and scale factors (+1.125 B/element) and run the scale-factor kernel; "
-                              "large_tensor is the plain amx_quantize") if fused_prepare else "plain amx_quantize"},
+                     # the step's casts also write the GEMM-ready sign planes and scale factors: bytes actually moved
+                     "bytes_per_element_moved": MOVED_BYTES_PER_ELEM if fused_prepare else BYTES_PER_ELEM,
+                     "gb_per_s_moved": quant_gbs * (MOVED_BYTES_PER_ELEM / BYTES_PER_ELEM if fused_prepare else 1.0),
+                     "note": ("gb_per_s counts the canonical bytes only (2.5625 B/element); the step's casts also write "
+                              "the GEMM-ready sign planes and scale factors in the same pass (gb_per_s_moved); timed by "
+                              "events in a pass of plain launches; large_tensor is the plain amx_quantize")
+                             if fused_prepare else "plain amx_quantize"},
         "gemm": {"useful_tflops": gemm_tflops, "ms_per_step": g_ms / args.steps,
                  # the sign split issues four FP4 products per useful one
                  "issued_tflops": gemm_tflops * (4.0 if "mxf4" in gemm_kernel else 1.0),
