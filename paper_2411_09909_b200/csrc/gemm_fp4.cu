@@ -240,9 +240,11 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     Control* ctl = reinterpret_cast<Control*>(tiles + kStages * kStageBytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // Work items: tile x K range (one range unless SLICED); an item index is tile * S + range, num_kb the K blocks
-    // of one item (the host picks a slice count that divides the K blocks).
+    // of one item when there is one range.
     const int S = SLICED ? p.slices : 1;
-    const int num_kb = (int)((p.K + BK - 1) / BK) / S;
+    const int kb_total = (int)((p.K + BK - 1) / BK);
+    const int num_kb = kb_total / S;                             // per item; SLICED: ranges differ by at most one block
+    auto kb_begin = [&](int64_t tile) -> int { return SLICED ? (int)((int)(tile % S) * kb_total / S) : 0; };
     // Persistent CTA: tiles blockIdx.x, blockIdx.x + gridDim.x, ...; neighbouring tiles share their A rows.
     const int64_t n_tiles = (p.N + BN - 1) / BN, m_tiles = (p.M + BM - 1) / BM;
     // Causal logits (square, keys after the queries masked): only the tiles on or below the diagonal exist.  Row
@@ -276,6 +278,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     };
     // K blocks of a tile (of an item): all of them, fewer or none under a causal mask (see Params::causal)
     auto nkb_of = [&](int64_t tile) -> int {
+        if (SLICED) return (int)(((int)(tile % S) + 1) * kb_total / S) - kb_begin(tile);
         if (!CAUSAL || p.causal == 0) return num_kb;
         const int64_t last_row = blk_m(tile) * BM + BM - 1;
         if (p.causal == 1) return num_kb;                 // the enumeration holds no masked tile
@@ -305,7 +308,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             bool ok = true;
             for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
                 const int64_t m_blk = blk_m(tile), n_blk = blk_n(tile);
-                const int kb0 = (int)(tile % S) * num_kb, nkb = nkb_of(tile);
+                const int kb0 = kb_begin(tile), nkb = nkb_of(tile);
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % kStages;
                     if (it >= kStages && !mbar_wait(&ctl->empty[s], ((it / kStages) - 1) & 1, &ctl->abort, p.status)) {
@@ -419,7 +422,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             for (int pl = 0; pl < 2; ++pl)
 #pragma unroll
                 for (int kk = 0; kk < kSteps; ++kk) {
-                    const int64_t c = ((int64_t)(tile % S) * num_kb + kb) * kSteps + kk;
+                    const int64_t c = ((int64_t)kb_begin(tile) + kb) * kSteps + kk;
                     const uint8_t* a = (pl ? p.sfa_neg : p.sfa_pos) + (m_blk * p.nk64 + c) * kSfChunk + lane * 16;
                     const uint8_t* w = (pl ? p.sfb_neg : p.sfb_pos) + ((n_blk * 2) * p.nk64 + c) * kSfChunk + lane * 16;
                     sfv[(pl * kSteps + kk) * 3 + 0] = __ldg(reinterpret_cast<const uint4*>(a));
@@ -778,14 +781,13 @@ attn_row_reduce_kernel(const float2* __restrict__ part, int n_parts_all, int64_t
 
 // Few output tiles and a long K (a few token rows against a big weight): K ranges as separate work items, so
 // that more SMs stream the operands; their partial products go to the workspace and are added in range order.
-// Returns the number of ranges (1: none); it divides the 128-element K blocks.
+// Returns the number of ranges (1: none); ranges hold the same number of 128-element K blocks up to one.
 int gemm_fp4_slices(int64_t M, int64_t N, int64_t K) {
     const int64_t tiles = ((N + BN - 1) / BN) * ((M + BM - 1) / BM);
     const int num_kb = (int)((K + 127) / 128);
     int s = (int)(148 / tiles);
-    if (s > num_kb / 8) s = num_kb / 8;
+    if (s > num_kb / 6) s = num_kb / 6;                  // at least six K blocks per range
     if (s > 8) s = 8;
-    while (s > 1 && num_kb % s) --s;
     return s < 2 ? 1 : s;
 }
 size_t gemm_fp4_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K) {
