@@ -468,18 +468,45 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         const int tid_e = threadIdx.x - (2 + kSfWarps) * 32;
         int t = 0;
         bool ok = true;
-        for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-            if (nkb_of(tile) == 0) continue;
+        static_assert(kEpilogueWarps * 32 == BN, "one column offset per epilogue thread");
+        // The per-tile constants (this thread's column offset and row offset; in the cast pass the row's softmax
+        // statistics) are fetched one tile ahead, so that their latency is off the path between two tiles.
+        struct TileConsts {
+            int w_ex, a_ex, kmax;
+            float2 rs;
+        };
+        auto next_live = [&](int64_t tl) {
+            while (tl < total_tiles && nkb_of(tl) == 0) tl += gridDim.x;
+            return tl;
+        };
+        auto load_consts = [&](int64_t tl) {
+            TileConsts c = {0, 0, 0, make_float2(0.f, 0.f)};
+            if (tl < total_tiles) {
+                const int64_t n = blk_n(tl) * BN + tid_e, mm = blk_m(tl) * BM + q * 32 + lane;
+                if (n < p.N) c.w_ex = row_word_exp(__ldg(p.w_exp + n));
+                if (mm < p.M) {
+                    c.a_ex = row_word_exp(__ldg(p.a_exp + mm));
+                    if constexpr (EPI == kEpiCast) {
+                        c.rs = p.rowstat[mm];
+                        c.kmax = p.p_kmax[mm];
+                    }
+                }
+            }
+            return c;
+        };
+        int64_t tile = next_live(blockIdx.x);
+        TileConsts nxt = load_consts(tile);
+        while (tile < total_tiles && ok) {
+            const TileConsts cur = nxt;
+            const int64_t tile_after = next_live(tile + gridDim.x);
+            nxt = load_consts(tile_after);                       // in flight while this tile is worked on
             const int64_t m0 = blk_m(tile) * BM, n0 = blk_n(tile) * BN;
             float* const C_item = p.C + (SLICED ? (tile % S) * p.slice_stride : 0);
             int* w_exp = ctl->w_exp[t & 1];
-            for (int i = tid_e; i < BN; i += kEpilogueWarps * 32) {
-                const int ex = (n0 + i < p.N) ? row_word_exp(p.w_exp[n0 + i]) : 0;
-                if constexpr (EPI == kEpiStore) w_exp[i] = ex;
-                else w_exp[i] = __float_as_int(p.alpha * 1.4426950408889634f * __uint_as_float((uint32_t)(ex + 127) << 23));
-            }
+            if constexpr (EPI == kEpiStore) w_exp[tid_e] = cur.w_ex;
+            else w_exp[tid_e] = __float_as_int(p.alpha * 1.4426950408889634f * __uint_as_float((uint32_t)(cur.w_ex + 127) << 23));
             const int64_t m = m0 + q * 32 + lane;
-            const int a_exp = (m < p.M) ? row_word_exp(p.a_exp[m]) : 0;
+            const int a_exp = cur.a_ex;
             ok = mbar_wait(&ctl->accum_full, t & 1, &ctl->abort, p.status);
             tc_fence_after();
             // every epilogue warp has written its part of w_exp (named barrier: the other roles do not join)
@@ -567,8 +594,8 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                     } else {
                         // Four 32-column groups per thread: normalise with the row's statistics {-max, 1 / sum}, round
                         // to bf16, cast.  P has no negative element: only its positive plane and scale factors exist.
-                        const float2 rs = (m < p.M) ? p.rowstat[m] : make_float2(0.f, 0.f);
-                        const int kmax = (m < p.M) ? p.p_kmax[m] : 0;
+                        const float2 rs = cur.rs;
+                        const int kmax = cur.kmax;
                         const int64_t G = p.N / 32, g0 = (n0 + col_base) / 32;
                         const int64_t sf_row = sf_row_offset(m, p.p_nk64);
 #pragma unroll
@@ -599,6 +626,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 if (lane == 0) mbar_arrive(&ctl->accum_empty);
             }
             ++t;
+            tile = tile_after;
         }
     }
     tc_fence_before();
