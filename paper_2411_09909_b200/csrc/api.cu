@@ -338,8 +338,8 @@ extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_
                 rc = gemm_fp4_attn_scores({w + a.pq, hc * L, chunk * L, i * L}, {w + a.pk, hc * L, chunk * L + 128, i * L}, L, d,
                                           alpha, S, w + a.pc, w + a.ps, w + a.pp, w + a.gemm, st, causal);
                 if (rc == AMX_OK)
-                    rc = gemm_fp4_prepared_at({w + a.pp, L, L, 0}, {w + a.pv, hc * d, chunk * d + 128, i * d}, L, d, L, oh, d,
-                                              w + a.gemm, st, 256, causal);
+                    rc = gemm_fp4_prepared_at({w + a.pp, L, L, 0, /*single_plane=*/true}, {w + a.pv, hc * d, chunk * d + 128, i * d},
+                                              L, d, L, oh, d, w + a.gemm, st, 256, causal);
                 if (rc != AMX_OK) return rc;
                 continue;
             }

@@ -50,6 +50,8 @@ int gemm_fp4_softmax_prepared(const float* S, int64_t rows, int64_t cols, int64_
 struct Fp4Operand {
     const void* prepared;
     int64_t rows_total, layout_rows, row0;
+    bool single_plane = false;   // left-hand operand only: its negative plane was never written (the two-pass
+                                 // attention scores write P's positive plane alone) and must not be read
 };
 int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
                          int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes = 256,

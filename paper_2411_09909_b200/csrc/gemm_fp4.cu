@@ -197,6 +197,9 @@ struct Params {
                                  // keys all lie after their queries are skipped, the epilogue masks the diagonal
                                  // ones); 2 = the product P V (K blocks after the tile's last query row hold only
                                  // zeros of P and are skipped)
+    int a_single;                // the left-hand operand has only its positive plane in memory (a cast softmax
+                                 // output): the tensor map's box is one plane deep, the negative plane's products
+                                 // are skipped anyway (row words)
     int m_fast;                  // tile order: consecutive tiles walk down M (else along N), see blk_m / blk_n
     int slices;                  // SLICED instantiation: K is cut into this many ranges, each (tile, range) a work item
     int64_t slice_stride;        //   whose partial product goes to C + range * slice_stride
@@ -316,7 +319,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                         break;
                     }
                     uint8_t* st = tiles + s * kStageBytes;
-                    mbar_expect_tx(&ctl->full[s], kStageBytes);
+                    mbar_expect_tx(&ctl->full[s], kStageBytes - (p.a_single ? C_::kTileA : 0));
                     // one 3-D tile per operand: {row bytes, rows, both sign planes}
                     tma_load_3d(st + C_::kOffAp, &tm_a, (kb0 + kb) * kRowBytes, (int)(p.a_row0 + m_blk * BM), 0, &ctl->full[s]);
                     tma_load_3d(st + C_::kOffWp, &tm_w, (kb0 + kb) * kRowBytes, (int)(p.w_row0 + n_blk * BN), 0, &ctl->full[s]);
@@ -658,12 +661,12 @@ EncodeTiledFn encode_tiled() {
 // Both sign planes of an operand as one 3-D tensor [2][rows][K/2] of bytes (plane_stride bytes apart);
 // box = {row_bytes, box_rows, 2}, 128- or 64-byte swizzle, zero fill outside.
 bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t K, size_t plane_stride, int box_rows,
-              int row_bytes) {
+              int row_bytes, int planes = 2) {
     EncodeTiledFn fn = encode_tiled();
     if (!fn) return false;
     const cuuint64_t dims[3] = {(cuuint64_t)(K / 2), (cuuint64_t)rows, 2};
     const cuuint64_t strides[2] = {(cuuint64_t)(K / 2), (cuuint64_t)plane_stride};
-    const cuuint32_t box[3] = {(cuuint32_t)row_bytes, (cuuint32_t)box_rows, 2};
+    const cuuint32_t box[3] = {(cuuint32_t)row_bytes, (cuuint32_t)box_rows, (cuuint32_t)planes};   // 1: positive plane only
     const cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
@@ -722,7 +725,7 @@ int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, co
         configured[dev] = true;
     }
     CUtensorMap tm_a, tm_w;
-    if (!make_map(&tm_a, pa, a_rows, p.K, oa.plane, BM, C_::kRowBytes) || !make_map(&tm_w, pw, w_rows, p.K, ow.plane, BN, C_::kRowBytes))
+    if (!make_map(&tm_a, pa, a_rows, p.K, oa.plane, BM, C_::kRowBytes, p.a_single ? 1 : 2) || !make_map(&tm_w, pw, w_rows, p.K, ow.plane, BN, C_::kRowBytes))
         return AMX_ERR_CUDA;
     static int sm_count[64] = {};
     if (!sm_count[dev] && cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
@@ -833,6 +836,7 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
     const int rc = fill_params(a, w, M, N, K, C, ld_c, workspace, st, p, oa, ow, dev);
     if (rc != AMX_OK) return rc;
     p.causal = causal_pv ? 2 : 0;
+    p.a_single = a.single_plane ? 1 : 0;
     const uint8_t* pa = static_cast<const uint8_t*>(a.prepared);
     const uint8_t* pw = static_cast<const uint8_t*>(w.prepared);
     const int slices = gemm_fp4_slices(M, N, K);
