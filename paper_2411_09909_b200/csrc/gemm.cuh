@@ -55,7 +55,9 @@ struct Fp4Operand {
 };
 int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
                          int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes = 256,
-                         int causal_pv = 0 /* 1: the product P V of causal attention (A = P, square) */);
+                         int causal_pv = 0 /* 1: the product P V of causal attention (A = P, square) */,
+                         int batch = 1 /* > 1 (N <= 128): a stack of `batch` independent products of M / batch rows */,
+                         int64_t w_batch_rows = 0 /* rows between their right-hand operands in the stacked W */);
 // workspace that lets the kernel cut K into ranges for products with few output tiles (256 bytes otherwise)
 size_t gemm_fp4_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K);
 // C[m][n] = sum over `slices` partial products [slices][M][N], in slice order (defined with the bf16-decode kernel)
@@ -65,7 +67,7 @@ int reduce_slices(const float* part, int slices, int64_t M, int64_t N, float* C,
 size_t gemm_fp4_attn_scratch_bytes(int64_t L);
 int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, int64_t d, float alpha, void* scratch,
                          uint8_t* p_codes, uint8_t* p_scales, void* p_prepared, void* workspace, cudaStream_t st,
-                         int causal = 0);
+                         int causal = 0, int64_t p_layout_rows = 0 /* 0: L */, int64_t p_row0 = 0);
 int quantize_cols_batched(const void* x, int64_t batch, int64_t R, int64_t C, uint8_t* codes, uint8_t* scales,
                           cudaStream_t st);
 int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,

@@ -200,6 +200,9 @@ struct Params {
     int a_single;                // the left-hand operand has only its positive plane in memory (a cast softmax
                                  // output): the tensor map's box is one plane deep, the negative plane's products
                                  // are skipped anyway (row words)
+    int mt_batch;                // half-width instantiation: > 0 = the product is a stack of independent ones, mt_batch
+    int64_t w_batch_rows;        //   row blocks of A each, whose right-hand operands lie w_batch_rows rows apart (a
+                                 //   multiple of 128) in the stacked W; C is the stack of the results
     int m_fast;                  // tile order: consecutive tiles walk down M (else along N), see blk_m / blk_n
     int slices;                  // SLICED instantiation: K is cut into this many ranges, each (tile, range) a work item
     int64_t slice_stride;        //   whose partial product goes to C + range * slice_stride
@@ -232,10 +235,16 @@ __device__ __forceinline__ void store_row16(float* out, const float (&f)[16], bo
     }
 }
 
-template <int BK_, int EPI = kEpiStore, bool SLICED = false, bool CAUSAL = false>
+// NHALF: tiles of 128 x 128 for products with at most 128 columns (the P V product of attention at head
+// dimension 128): the W box, the MMA and the epilogue are half as wide, the stage layout keeps its size.
+template <int BK_, int EPI = kEpiStore, bool SLICED = false, bool CAUSAL = false, bool NHALF = false>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w, const Params p) {
     using C_ = Cfg<BK_>;
+    constexpr int BNT = NHALF ? BN / 2 : BN;                     // tile width
+    static_assert(!NHALF || EPI == kEpiStore, "half-width tiles: plain epilogue only");
+    constexpr int kOffWnT = NHALF ? C_::kOffWp + C_::kTileB / 2 : C_::kOffWn;   // the box packs its two planes
+    constexpr uint32_t kIdescT = (1u << 7) | (1u << 10) | ((uint32_t)(BNT >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
     constexpr int BK = C_::BK, kRowBytes = C_::kRowBytes, kSteps = C_::kSteps, kStages = C_::kStages;
     constexpr int kStageBytes = C_::kStageBytes;
     extern __shared__ uint8_t smem_raw[];
@@ -249,7 +258,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     const int num_kb = kb_total / S;                             // per item; SLICED: ranges differ by at most one block
     auto kb_begin = [&](int64_t tile) -> int { return SLICED ? (int)((int)(tile % S) * kb_total / S) : 0; };
     // Persistent CTA: tiles blockIdx.x, blockIdx.x + gridDim.x, ...; neighbouring tiles share their A rows.
-    const int64_t n_tiles = (p.N + BN - 1) / BN, m_tiles = (p.M + BM - 1) / BM;
+    const int64_t n_tiles = (p.N + BNT - 1) / BNT, m_tiles = (p.M + BM - 1) / BM;
     // Causal logits (square, keys after the queries masked): only the tiles on or below the diagonal exist.  Row
     // block m has the column blocks 0 .. m/2 (a tile is 128 queries x 256 keys), so f(m) = tiles before row
     // block m is j(j+1) for m = 2j and (j+1)^2 for m = 2j+1; the work items enumerate exactly those tiles, which
@@ -279,11 +288,18 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         const uint32_t t = (uint32_t)tile / (uint32_t)S, q = t / fast_dim;
         return p.m_fast ? q : t - q * fast_dim;
     };
+    // rows by which the right-hand operand of row block m_blk is shifted (stack of independent products)
+    auto w_shift = [&](int64_t m_blk) -> int64_t {
+        if (!NHALF || p.mt_batch == 0) return 0;
+        return (int64_t)((uint32_t)m_blk / (uint32_t)p.mt_batch) * p.w_batch_rows;
+    };
     // K blocks of a tile (of an item): all of them, fewer or none under a causal mask (see Params::causal)
     auto nkb_of = [&](int64_t tile) -> int {
         if (SLICED) return (int)(((int)(tile % S) + 1) * kb_total / S) - kb_begin(tile);
         if (!CAUSAL || p.causal == 0) return num_kb;
-        const int64_t last_row = blk_m(tile) * BM + BM - 1;
+        int64_t mb = blk_m(tile);
+        if (NHALF && p.mt_batch) mb = (int64_t)((uint32_t)mb % (uint32_t)p.mt_batch);   // row block inside its product
+        const int64_t last_row = mb * BM + BM - 1;
         if (p.causal == 1) return num_kb;                 // the enumeration holds no masked tile
         return (int)min((int64_t)num_kb, (last_row + BK) / BK);
     };
@@ -319,10 +335,10 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                         break;
                     }
                     uint8_t* st = tiles + s * kStageBytes;
-                    mbar_expect_tx(&ctl->full[s], kStageBytes - (p.a_single ? C_::kTileA : 0));
+                    mbar_expect_tx(&ctl->full[s], kStageBytes - (p.a_single ? C_::kTileA : 0) - (NHALF ? C_::kTileB : 0));
                     // one 3-D tile per operand: {row bytes, rows, both sign planes}
                     tma_load_3d(st + C_::kOffAp, &tm_a, (kb0 + kb) * kRowBytes, (int)(p.a_row0 + m_blk * BM), 0, &ctl->full[s]);
-                    tma_load_3d(st + C_::kOffWp, &tm_w, (kb0 + kb) * kRowBytes, (int)(p.w_row0 + n_blk * BN), 0, &ctl->full[s]);
+                    tma_load_3d(st + C_::kOffWp, &tm_w, (kb0 + kb) * kRowBytes, (int)(p.w_row0 + w_shift(m_blk) + n_blk * BNT), 0, &ctl->full[s]);
                 }
             }
             // after an abort: let the copies already in flight land before shared memory is released
@@ -344,13 +360,14 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         auto tile_sides = [&](int64_t tile) {
             int bits = 0;
             if (tile < total_tiles && nkb_of(tile) > 0) {            // a skipped tile costs no load latency
-                const int64_t m0 = blk_m(tile) * BM, n0 = blk_n(tile) * BN;
+                const int64_t m0 = blk_m(tile) * BM, n0 = blk_n(tile) * BNT;
+                const int* w_words = p.w_exp + w_shift(blk_m(tile));
 #pragma unroll
                 for (int i = 0; i < BM / 32; ++i)
                     if (m0 + i * 32 + lane < p.M) bits |= (__ldg(p.a_exp + m0 + i * 32 + lane) >> 16) & 3;
 #pragma unroll
-                for (int i = 0; i < BN / 32; ++i)
-                    if (n0 + i * 32 + lane < p.N) bits |= ((__ldg(p.w_exp + n0 + i * 32 + lane) >> 16) & 3) << 2;
+                for (int i = 0; i < BNT / 32; ++i)
+                    if (n0 + i * 32 + lane < p.N) bits |= ((__ldg(w_words + n0 + i * 32 + lane) >> 16) & 3) << 2;
             }
             return bits;
         };
@@ -389,7 +406,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                             for (int kk = 0; kk < kSteps; ++kk) {   // 64 elements = 32 bytes along the swizzled row
                                 if (((sides >> pa) & 1) && ((sides >> (2 + pw)) & 1)) {
                                     mma_fp4_block16(tmem, dstage + (((pa ? C_::kOffAn : C_::kOffAp) + kk * 32) >> 4),
-                                                    dstage + (((pw ? C_::kOffWn : C_::kOffWp) + kk * 32) >> 4), kIdesc,
+                                                    dstage + (((pw ? kOffWnT : C_::kOffWp) + kk * 32) >> 4), kIdescT,
                                                     sfa + (pa * kSteps + kk) * 4, sfb + (pw * kSteps + kk) * 8,
                                                     idx ? 1u : accumulate);
                                     // with two MMAs still to go (they keep the pipe busy meanwhile), look whether the
@@ -427,10 +444,11 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 for (int kk = 0; kk < kSteps; ++kk) {
                     const int64_t c = ((int64_t)kb_begin(tile) + kb) * kSteps + kk;
                     const uint8_t* a = (pl ? p.sfa_neg : p.sfa_pos) + (m_blk * p.nk64 + c) * kSfChunk + lane * 16;
-                    const uint8_t* w = (pl ? p.sfb_neg : p.sfb_pos) + ((n_blk * 2) * p.nk64 + c) * kSfChunk + lane * 16;
+                    const uint8_t* w = (pl ? p.sfb_neg : p.sfb_pos) + ((n_blk * (BNT / 128) + w_shift(m_blk) / 128) * p.nk64 + c) * kSfChunk + lane * 16;
                     sfv[(pl * kSteps + kk) * 3 + 0] = __ldg(reinterpret_cast<const uint4*>(a));
                     sfv[(pl * kSteps + kk) * 3 + 1] = __ldg(reinterpret_cast<const uint4*>(w));
-                    sfv[(pl * kSteps + kk) * 3 + 2] = __ldg(reinterpret_cast<const uint4*>(w + (int64_t)p.nk64 * kSfChunk));
+                    sfv[(pl * kSteps + kk) * 3 + 2] =           // second block of 128 rows (none in a half-width tile)
+                        __ldg(reinterpret_cast<const uint4*>(w + (NHALF ? 0 : (int64_t)p.nk64 * kSfChunk)));
                 }
         };
         // this group's K blocks, in order, over all tiles: (tile, kb) with global index it = group, group + 2, ...
@@ -467,11 +485,11 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         // -------------------------------------------------------------- epilogue
         // Eight warps: quarter q = warp % 4 of the lanes (= rows), one half of the columns each.
         const int e = warp - (2 + kSfWarps);                     // 0..7
-        const int q = warp & 3, col_base = (e >> 2) * (BN / 2);
+        const int q = warp & 3, col_base = (e >> 2) * (BNT / 2);
         const int tid_e = threadIdx.x - (2 + kSfWarps) * 32;
         int t = 0;
         bool ok = true;
-        static_assert(kEpilogueWarps * 32 == BN, "one column offset per epilogue thread");
+        static_assert(kEpilogueWarps * 32 == BN, "one column offset per epilogue thread");   // BNT <= BN
         // The per-tile constants (this thread's column offset and row offset; in the cast pass the row's softmax
         // statistics) are fetched one tile ahead, so that their latency is off the path between two tiles.
         struct TileConsts {
@@ -485,8 +503,8 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         auto load_consts = [&](int64_t tl) {
             TileConsts c = {0, 0, 0, make_float2(0.f, 0.f)};
             if (tl < total_tiles) {
-                const int64_t n = blk_n(tl) * BN + tid_e, mm = blk_m(tl) * BM + q * 32 + lane;
-                if (n < p.N) c.w_ex = row_word_exp(__ldg(p.w_exp + n));
+                const int64_t n = blk_n(tl) * BNT + tid_e, mm = blk_m(tl) * BM + q * 32 + lane;
+                if (tid_e < BNT && n < p.N) c.w_ex = row_word_exp(__ldg(p.w_exp + w_shift(blk_m(tl)) + n));
                 if (mm < p.M) {
                     c.a_ex = row_word_exp(__ldg(p.a_exp + mm));
                     if constexpr (EPI == kEpiCast) {
@@ -503,7 +521,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             const TileConsts cur = nxt;
             const int64_t tile_after = next_live(tile + gridDim.x);
             nxt = load_consts(tile_after);                       // in flight while this tile is worked on
-            const int64_t m0 = blk_m(tile) * BM, n0 = blk_n(tile) * BN;
+            const int64_t m0 = blk_m(tile) * BM, n0 = blk_n(tile) * BNT;
             float* const C_item = p.C + (SLICED ? (tile % S) * p.slice_stride : 0);
             int* w_exp = ctl->w_exp[t & 1];
             if constexpr (EPI == kEpiStore) w_exp[tid_e] = cur.w_ex;
@@ -520,10 +538,10 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                     uint32_t v[2][16];
                     tmem_ld16(taddr, v[0]);
 #pragma unroll
-                    for (int c = 0; c < BN / 2; c += 16) {
+                    for (int c = 0; c < BNT / 2; c += 16) {
                         const int buf = (c / 16) & 1;
                         tmem_ld_wait();
-                        if (c + 16 < BN / 2) tmem_ld16(taddr + c + 16, v[buf ^ 1]);   // next chunk loads while this one is stored
+                        if (c + 16 < BNT / 2) tmem_ld16(taddr + c + 16, v[buf ^ 1]);   // next chunk loads while this one is stored
                         const int col = col_base + c;
                         float f[16];
 #pragma unroll
@@ -714,25 +732,26 @@ size_t gemm_fp4_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 
 namespace {
 
-template <int BK_, int EPI = kEpiStore, bool SLICED = false, bool CAUSAL = false>
+template <int BK_, int EPI = kEpiStore, bool SLICED = false, bool CAUSAL = false, bool NHALF = false>
 int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, const OperandLayout& ow, int64_t a_rows,
                int64_t w_rows, Params p, int dev, cudaStream_t st) {
     using C_ = Cfg<BK_>;
+    constexpr int BNT = NHALF ? BN / 2 : BN;
     static bool configured[64] = {};
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(gemm_fp4_kernel<BK_, EPI, SLICED, CAUSAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(gemm_fp4_kernel<BK_, EPI, SLICED, CAUSAL, NHALF>, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::kSmemBytes) != cudaSuccess)
             return AMX_ERR_CUDA;
         configured[dev] = true;
     }
     CUtensorMap tm_a, tm_w;
-    if (!make_map(&tm_a, pa, a_rows, p.K, oa.plane, BM, C_::kRowBytes, p.a_single ? 1 : 2) || !make_map(&tm_w, pw, w_rows, p.K, ow.plane, BN, C_::kRowBytes))
+    if (!make_map(&tm_a, pa, a_rows, p.K, oa.plane, BM, C_::kRowBytes, p.a_single ? 1 : 2) || !make_map(&tm_w, pw, w_rows, p.K, ow.plane, BNT, C_::kRowBytes))
         return AMX_ERR_CUDA;
     static int sm_count[64] = {};
     if (!sm_count[dev] && cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return AMX_ERR_CUDA;
-    const int64_t tiles = ((p.N + BN - 1) / BN) * ((p.M + BM - 1) / BM) * (SLICED ? p.slices : 1);
+    const int64_t tiles = ((p.N + BNT - 1) / BNT) * ((p.M + BM - 1) / BM) * (SLICED ? p.slices : 1);
     const unsigned grid = (unsigned)(tiles < sm_count[dev] ? tiles : sm_count[dev]);   // one persistent CTA per SM
-    gemm_fp4_kernel<BK_, EPI, SLICED, CAUSAL><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_a, tm_w, p);
+    gemm_fp4_kernel<BK_, EPI, SLICED, CAUSAL, NHALF><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_a, tm_w, p);
     return launch_status();
 }
 
@@ -829,7 +848,9 @@ size_t gemm_fp4_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 // The GEMM proper on two prepared operands (each laid out by operand_layout()), or on row ranges of them.
 // workspace_bytes >= gemm_fp4_prepared_workspace_bytes() enables the K ranges; 256 bytes always suffice.
 int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
-                         int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes, int causal_pv) {
+                         int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes, int causal_pv, int batch,
+                         int64_t w_batch_rows) {
+    if (batch > 1 && (N > BN / 2 || M % batch || (M / batch) % BM || w_batch_rows % 128)) return AMX_ERR_SHAPE;
     Params p;
     OperandLayout oa, ow;
     int dev;
@@ -839,8 +860,16 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
     p.a_single = a.single_plane ? 1 : 0;
     const uint8_t* pa = static_cast<const uint8_t*>(a.prepared);
     const uint8_t* pw = static_cast<const uint8_t*>(w.prepared);
-    const int slices = gemm_fp4_slices(M, N, K);
-    if (causal_pv) return launch_fp4<128, kEpiStore, false, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
+    const int slices = batch > 1 ? 1 : gemm_fp4_slices(M, N, K);
+    // at most 128 columns (P V at head dimension 128): tiles of 128 x 128, so that no half of a W tile is padding
+    const bool half = N <= BN / 2 && (batch > 1 || !getenv("AMX_FP4_NO_HALF_TILE"));
+    if (batch > 1) {
+        p.mt_batch = (int)(M / batch / BM);
+        p.w_batch_rows = w_batch_rows;
+    }
+    if (causal_pv)
+        return half ? launch_fp4<128, kEpiStore, false, true, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st)
+                    : launch_fp4<128, kEpiStore, false, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
     if (slices > 1 && fp4_block_k() == 128 && workspace_bytes >= gemm_fp4_prepared_workspace_bytes(M, N, K)) {
         float* part = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 256);
         p.C = part;
@@ -851,8 +880,9 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
         const int r2 = launch_fp4<128, kEpiStore, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
         return r2 != AMX_OK ? r2 : reduce_slices(part, slices, M, N, C, ld_c, st);
     }
-    return fp4_block_k() == 256 ? launch_fp4<256>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st)
-                                : launch_fp4<128>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
+    if (fp4_block_k() == 256 && batch == 1) return launch_fp4<256>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
+    return half ? launch_fp4<128, kEpiStore, false, false, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st)
+                : launch_fp4<128>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
 }
 
 // Attention scores without the logits in memory: P = softmax(alpha * Q K^T) cast to AMXFP4 as the prepared
@@ -864,7 +894,9 @@ size_t gemm_fp4_attn_scratch_bytes(int64_t L) {
 }
 int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, int64_t d, float alpha, void* scratch,
                          uint8_t* p_codes, uint8_t* p_scales, void* p_prepared, void* workspace, cudaStream_t st,
-                         int causal) {
+                         int causal, int64_t p_layout_rows, int64_t p_row0) {
+    if (p_layout_rows == 0) p_layout_rows = L;
+    if (p_row0 % 128 || p_row0 + L > p_layout_rows) return AMX_ERR_SHAPE;
     if (L % BN) return AMX_ERR_SHAPE;
     Params p;
     OperandLayout oq, ok_;
@@ -878,8 +910,11 @@ int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, in
     float2* part = reinterpret_cast<float2*>(sc);
     float2* rowstat = reinterpret_cast<float2*>(sc + up256((size_t)L * n_parts * sizeof(float2)));
     int* p_kmax = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(rowstat) + up256((size_t)L * sizeof(float2)));
-    const OperandLayout op = operand_layout(L, L, BM);
+    const OperandLayout op = operand_layout(p_layout_rows, L, BM);
     uint8_t* pp = static_cast<uint8_t*>(p_prepared);
+    uint8_t* p_plane = pp + (size_t)p_row0 * (L / 2);
+    uint8_t* p_sf = pp + 2 * op.plane + (size_t)(p_row0 / 128) * op.nk64 * kSfChunk;
+    int* p_words = reinterpret_cast<int*>(pp + 2 * op.plane + 2 * op.sf) + p_row0;
     p.alpha = alpha;
     p.causal = causal ? 1 : 0;
     p.part = part;
@@ -887,14 +922,13 @@ int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, in
     p.p_kmax = p_kmax;
     p.p_codes = reinterpret_cast<uint4*>(p_codes);      // not written: the prepared operand is all P V needs
     p.p_scales = reinterpret_cast<uint16_t*>(p_scales);
-    p.p_pos = reinterpret_cast<uint4*>(pp);
-    p.p_sf = pp + 2 * op.plane;
+    p.p_pos = reinterpret_cast<uint4*>(p_plane);
+    p.p_sf = p_sf;
     p.p_nk64 = op.nk64;
     rc = causal ? launch_fp4<128, kEpiStats, false, true>(pq, pk, oq, ok_, q.rows_total, k.rows_total, p, dev, st)
                 : launch_fp4<128, kEpiStats>(pq, pk, oq, ok_, q.rows_total, k.rows_total, p, dev, st);
     if (rc != AMX_OK) return rc;
-    attn_row_reduce_kernel<<<(unsigned)((L + 7) / 8), 256, 0, st>>>(part, n_parts, L, causal, rowstat, p_kmax,
-                                                                        reinterpret_cast<int*>(pp + 2 * op.plane + 2 * op.sf));
+    attn_row_reduce_kernel<<<(unsigned)((L + 7) / 8), 256, 0, st>>>(part, n_parts, L, causal, rowstat, p_kmax, p_words);
     rc = launch_status();
     if (rc != AMX_OK) return rc;
     return causal ? launch_fp4<128, kEpiCast, false, true>(pq, pk, oq, ok_, q.rows_total, k.rows_total, p, dev, st)
