@@ -14,7 +14,7 @@ bool gemm_shape_ok(int64_t M, int64_t N, int64_t K, int gs) {
     return valid_group_size(gs) && M >= 0 && N >= 0 && K > 0 && K % gs == 0 && K % 8 == 0;
 }
 
-constexpr uint32_t kKernelMask = AMX_GEMM_SIMT | AMX_GEMM_TC | AMX_GEMM_FP4;
+constexpr uint32_t kKernelMask = AMX_GEMM_SIMT | AMX_GEMM_TC | AMX_GEMM_FP4 | AMX_GEMM_ROWS;
 
 // The kernel to run (one AMX_GEMM_* bit), or 0 when the flags cannot be honoured for this shape.
 uint32_t pick_kernel(int64_t M, int64_t N, int64_t K, int gs, uint32_t flags) {
@@ -24,11 +24,15 @@ uint32_t pick_kernel(int64_t M, int64_t N, int64_t K, int gs, uint32_t flags) {
     const bool tc = gemm_tc_supported(M, N, K, gs);
     if (want == AMX_GEMM_TC) return tc ? AMX_GEMM_TC : 0;
     if (want == AMX_GEMM_SIMT) return AMX_GEMM_SIMT;
+    const bool rows = gemm_rows_supported(M, N, K, gs);
+    if (want == AMX_GEMM_ROWS) return rows ? AMX_GEMM_ROWS : 0;
     // AMX_GEMM_AUTO: the FP4-pipe kernel for anything that fills the machine (it is about twice as fast as
     // the bf16-decode kernel); the exact bf16-decode kernel for small products, where launch count matters
     // more than throughput; the SIMT kernel for group sizes the tensor-core kernels do not take.
     // A few token rows against a big weight (decode-like): too few 128 x 256 tiles to fill the machine, and the
     // FP4 kernel would have to prepare the whole weight for them; the bf16-decode kernel slices K over CTAs.
+    // At most 16 token rows: the weight-streaming kernel reads the canonical weight once at memory speed.
+    if (rows && K >= 512) return AMX_GEMM_ROWS;
     const int64_t tiles = ((M + 127) / 128) * ((N + 255) / 256);
     if (tc && M <= 64 && tiles < 148 && K >= 1024) return AMX_GEMM_TC;
     if (gemm_fp4_supported(M, N, K, gs) && (double)M * (double)N * (double)K >= 128.0 * 1024.0 * 1024.0) return AMX_GEMM_FP4;
@@ -38,6 +42,7 @@ uint32_t pick_kernel(int64_t M, int64_t N, int64_t K, int gs, uint32_t flags) {
 size_t kernel_workspace(uint32_t kernel, int64_t M, int64_t N, int64_t K) {
     if (kernel == AMX_GEMM_TC) return round_up(gemm_tc_workspace_bytes(M, N, K));
     if (kernel == AMX_GEMM_FP4) return round_up(gemm_fp4_workspace_bytes(M, N, K));
+    if (kernel == AMX_GEMM_ROWS) return round_up(gemm_rows_workspace_bytes(K));
     return 0;
 }
 
@@ -98,6 +103,9 @@ extern "C" int amx_gemm(const uint8_t* a_codes, const uint8_t* a_scales, const u
     if (need && !aligned(workspace, kAlign)) return AMX_ERR_ALIGN;
     if (kernel == AMX_GEMM_FP4)
         return gemm_fp4(a_codes, a_scales, w_codes, w_scales, M, N, K, C, ld_c, workspace, st);
+    if (kernel == AMX_GEMM_ROWS && !aligned(w_scales, 4)) return AMX_ERR_ALIGN;   // 4-byte asynchronous copies
+    if (kernel == AMX_GEMM_ROWS)
+        return gemm_rows(a_codes, a_scales, w_codes, w_scales, M, N, K, C, ld_c, workspace, st);
     return gemm_tc(a_codes, a_scales, w_codes, w_scales, M, N, K, C, ld_c, workspace, st);
 }
 
@@ -177,6 +185,13 @@ extern "C" int amx_quant_gemm(const void* A, int64_t ld_a, const uint8_t* w_code
     }
     uint8_t* a_codes = base + gemm_ws;
     uint8_t* a_scales = a_codes + a.codes;
+    if (pick_kernel(M, N, K, group_size, flags) == AMX_GEMM_ROWS) {
+        // the cast of the few rows writes the decoded operand of the weight-streaming kernel directly: two launches
+        if (!A || !w_codes || !w_scales || !C) return AMX_ERR_NULL;
+        if (!aligned(A, 16) || ld_a % 8 || !aligned(w_codes, 16) || !aligned(w_scales, 4) || !aligned(C, 4))
+            return AMX_ERR_ALIGN;
+        return gemm_rows_cast(A, ld_a, w_codes, w_scales, M, N, K, C, ld_c, base, static_cast<cudaStream_t>(stream));
+    }
     if (pick_kernel(M, N, K, group_size, flags) == AMX_GEMM_FP4 && ld_a == K) {
         // the activation's cast writes the kernel's operand itself (one launch less, the codes are not re-read);
         // same workspace layout as amx_gemm's: status word, prepared A, prepared W

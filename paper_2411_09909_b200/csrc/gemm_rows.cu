@@ -1,0 +1,376 @@
+// AMXFP4 x AMXFP4 -> fp32 for at most 16 rows of A against a large weight (the decode phase of inference):
+// C[m,n] = sum_k Ahat[m,k] * What[n,k] (arXiv 2411.09909, Section 4.3), bound by streaming the 4.5-bit weight
+// from HBM once, not by arithmetic.
+//
+// The weight is read in its canonical layout (codes [N, K/2], scales [N, K/32, 2]); nothing is prepared ahead.
+// The few activation rows are decoded to bf16 once by a small kernel (decoded values are exact in bf16, Eq. 1),
+// already in the order the multiply instruction's fragments want, so that the streaming kernel only copies them.
+//
+// Streaming kernel: warp-level mma.sync m16n8k16 (bf16 in, fp32 accumulate) with the 16 token rows as the M side
+// and 8 weight rows as the N side.  The contraction index may be permuted freely as long as both operands use
+// the same permutation; here lane (g, t) (g = lane / 4, t = lane % 4) owns, for one step of 128 elements of K,
+// the whole 32-element group 4 * step + t of weight row g of each of its two 8-row tiles: 16 bytes of codes and
+// the group's two scales per tile, brought in by asynchronous copies into a per-warp ring in shared memory four
+// steps ahead (no registers are held by loads in flight) and decoded in registers with the group's lookup tables.
+// The matching activation values (rows g and g + 8, same group) come from shared memory in 16-byte pieces.
+// Eight MMAs per tile and step consume four elements per lane each.  What bounds the kernel is instruction
+// issue (decode on the integer/logic pipe), not the tensor cores: the MMAs are a few percent of the instructions.
+//
+// A CTA of eight warps covers 128 weight rows and one range of K; the ranges of K of the same 128 rows are the
+// CTAs of one thread-block cluster (up to 8), which add their partial products over distributed shared memory
+// in rank order - deterministic, no scratch in global memory and no second launch.
+#include <cooperative_groups.h>
+#include <cuda_bf16.h>
+
+#include "cast_math.cuh"
+#include "decode_math.cuh"
+#include "gemm.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace amx {
+namespace {
+
+using namespace decode;
+
+constexpr int kMaxRows = 16;                 // token rows (the M side of one MMA)
+constexpr int kWarps = 8, kThreads = kWarps * 32;
+constexpr int kTiles = 2;                    // 8-row weight tiles per warp
+constexpr int kCtaRows = kWarps * kTiles * 8;   // 128 weight rows per CTA
+constexpr int kStepK = 128;                  // elements of K per step: one group per lane of a quad
+constexpr int kStepBytes = kMaxRows * kStepK * 2;   // activation fragments of one step: 4 KB
+constexpr int kChunkSteps = 4;               // steps of activation fragments in shared memory at a time (16 KB)
+constexpr int kMaxSlices = 8;                // portable cluster size
+constexpr int kPartPitch = 136;              // floats per token row of the partial-product tile (bank spread)
+
+// Fragment order of the decoded activation, per step of 128 elements: [unit j = 0..3][half 0..1][lane 0..31]
+// pieces of 16 bytes; the piece of lane (g, t) holds elements 8j .. 8j+7 of group 4 * step + t of row 8 * half + g
+// (in the pair order and scaling of pair_order_scaled).
+__device__ __forceinline__ int64_t fragment_piece(int64_t step, int j, int half, int g, int t) {
+    return ((step * 4 + j) * 2 + half) * 32 + g * 4 + t;
+}
+
+// The streaming kernel decodes a word of eight weight codes into the bf16 pairs (e0, e4), (e1, e5), (e2, e6),
+// (e3, e7), each value 2^-63 times the true one (see decode_pairs); the activation pieces are stored in the same
+// pair order and multiplied by 2^63, so that every product is the true one.  Both scalings are exact: a decoded
+// value times 2^+-63 stays far inside the bf16 range.
+__device__ __forceinline__ uint4 pair_order_scaled(uint4 o) {      // o: pairs (e0,e1), (e2,e3), (e4,e5), (e6,e7)
+    const uint32_t two63 = 0x5F005F00u;
+    uint4 r;
+    r.x = mul_bf16x2(prmt(o.x, o.z, 0x5410), two63);
+    r.y = mul_bf16x2(prmt(o.x, o.z, 0x7632), two63);
+    r.z = mul_bf16x2(prmt(o.y, o.w, 0x5410), two63);
+    r.w = mul_bf16x2(prmt(o.y, o.w, 0x7632), two63);
+    return r;
+}
+
+// One thread per 32-element group of the 16-row slab: decode (DECODE) or cast then decode (CAST) and write the
+// four 16-byte pieces.  Rows past M are written as zeros.
+template <bool CAST>
+__global__ void __launch_bounds__(128) rows_fragments_kernel(const uint8_t* __restrict__ codes,
+                                                             const uint8_t* __restrict__ scales,
+                                                             const uint16_t* __restrict__ x, int64_t ld_x, int M,
+                                                             int64_t K, uint4* __restrict__ frag) {
+    const int64_t groups = K / 32;
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= groups * kMaxRows) return;
+    const int row = (int)(idx / groups);
+    const int64_t grp = idx % groups;
+    uint4 c = make_uint4(0, 0, 0, 0);
+    uint32_t sc = 0;
+    if (row < M) {
+        if (CAST) {
+            const uint4* p = reinterpret_cast<const uint4*>(x + row * ld_x + grp * 32);
+            uint32_t w[16];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint4 q = __ldg(p + j);
+                w[4 * j] = q.x; w[4 * j + 1] = q.y; w[4 * j + 2] = q.z; w[4 * j + 3] = q.w;
+            }
+            float inv_p, inv_n;
+            sc = cast::group_scales(cast::side_maxima<16>(w), inv_p, inv_n);
+            c.x = cast::encode8(w, inv_p, inv_n);
+            c.y = cast::encode8(w + 4, inv_p, inv_n);
+            c.z = cast::encode8(w + 8, inv_p, inv_n);
+            c.w = cast::encode8(w + 12, inv_p, inv_n);
+        } else {
+            c = __ldg(reinterpret_cast<const uint4*>(codes + (row * groups + grp) * 16));
+            sc = __ldg(reinterpret_cast<const unsigned short*>(scales + (row * groups + grp) * 2));
+        }
+    }
+    const GroupTables tb = make_tables(sc);
+    const int64_t step = grp >> 2;
+    const int t = (int)(grp & 3), g = row & 7, half = row >> 3;
+    const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) frag[fragment_piece(step, j, half, g, t)] = pair_order_scaled(decode_word(w[j], tb));
+}
+
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Decode for the weight stream.  The integer/logic pipe is what bounds this kernel, so the multiplication by
+// the scale is a packed bf16 multiply (FMA pipe) instead of table look-ups:
+//   - a 3-bit E2M1 code placed at bits 8..6 of a bf16 reads as (its value) x 2^-126: codes 0 and 1 are the bf16
+//     subnormals 0 and 2^-127, the others have exponent field 1..3 and the code's mantissa bit;
+//   - one shift and one mask put the codes of elements q and q + 4 of a word there (pair q);
+//   - the element's scale (positive or negative side, the sign folded into the latter) is chosen with a mask that
+//     a byte permute in sign-replicating mode builds from the two sign bits;
+//   - scales are held as bf16 pairs times 2^63 (2^126 would overflow), the activation carries the other 2^63.
+struct GroupScales {
+    uint32_t pos, neg;     // {s_p, s_p} x 2^63 and {-s_n, -s_n} x 2^63 as bf16 pairs
+};
+__device__ __forceinline__ GroupScales make_scales(uint32_t sc) {
+    const float two63 = 9223372036854775808.f;
+    const uint32_t p = __float_as_uint(e5m2_to_float(sc & 0xFFu) * two63);
+    const uint32_t n = __float_as_uint(e5m2_to_float((sc >> 8) & 0xFFu) * -two63);
+    return {prmt(p, p, 0x3232), prmt(n, n, 0x3232)};
+}
+__device__ __forceinline__ uint4 decode_pairs(uint32_t w, const GroupScales& gs) {
+    const uint32_t kMag = 0x01C001C0u, ws = w << 4;
+    const uint32_t m0 = prmt(ws, ws, 0xAA88), m1 = prmt(w, w, 0xAA88);     // 0xFFFF where the element is negative
+    const uint32_t m2 = prmt(ws, ws, 0xBB99), m3 = prmt(w, w, 0xBB99);
+    uint4 o;
+    o.x = mul_bf16x2((w << 6) & kMag, (gs.pos & ~m0) | (gs.neg & m0));
+    o.y = mul_bf16x2((w << 2) & kMag, (gs.pos & ~m1) | (gs.neg & m1));
+    o.z = mul_bf16x2((w >> 2) & kMag, (gs.pos & ~m2) | (gs.neg & m2));
+    o.w = mul_bf16x2((w >> 6) & kMag, (gs.pos & ~m3) | (gs.neg & m3));
+    return o;
+}
+
+// Asynchronous copy of 16 or 4 bytes from global to shared memory (no registers held while in flight).
+__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src));
+}
+__device__ __forceinline__ void cp_async4(void* dst, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Shared memory of a CTA: two buffers of activation fragments (a chunk of steps each), then one ring of kDepth
+// steps per warp for the weight stream.  A ring slot holds, per 8-row tile, the 32 lanes' 16 bytes of codes and
+// 4 bytes of scales (the two groups 4 * step + 2 * (t / 2) + {0, 1}; the lane uses the half t % 2).  Every lane
+// reads back only what its own copies wrote, so the ring needs no barrier, only the lane's own wait.
+constexpr int kDepth = 4;
+constexpr int kSlotCodes = kTiles * 32 * 16, kSlotBytes = kSlotCodes + kTiles * 32 * 4;   // 2560
+constexpr int kRingBytes = kDepth * kSlotBytes;                                            // per warp
+constexpr int kFragBytes = kChunkSteps * kStepBytes;
+constexpr int kSmemBytes = 2 * kFragBytes + kWarps * kRingBytes;
+static_assert(kChunkSteps <= kDepth, "a chunk's fragments are committed with the group of its first step");
+
+__global__ void __launch_bounds__(kThreads, 3) gemm_rows_kernel(const uint4* __restrict__ frag,
+                                                                const uint8_t* __restrict__ w_codes,
+                                                                const uint8_t* __restrict__ w_scales, int M, int64_t N,
+                                                                int64_t K, float* __restrict__ C, int64_t ld_c) {
+    extern __shared__ __align__(16) uint8_t smem[];
+    cg::cluster_group cluster = cg::this_cluster();
+    const int slices = (int)gridDim.y, slice = (int)blockIdx.y;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t = lane & 3;
+    const int64_t groups = K / 32, steps = K / kStepK;
+    const int64_t s_begin = steps * slice / slices;
+    const int n_total = (int)(steps * (slice + 1) / slices - s_begin);
+    const int64_t row0 = (int64_t)blockIdx.x * kCtaRows + warp * (kTiles * 8);
+
+    // this lane's stream positions at step s_begin: codes of group 4 * step + t, scales of the group pair
+    const uint8_t* pc[kTiles];
+    const uint8_t* ps[kTiles];
+#pragma unroll
+    for (int i = 0; i < kTiles; ++i) {
+        int64_t r = row0 + i * 8 + g;
+        r = r < N ? r : N - 1;               // rows past the weight read its last row; their sums are not stored
+        pc[i] = w_codes + (r * groups + s_begin * 4 + t) * 16;
+        ps[i] = w_scales + (r * groups + s_begin * 4 + (t & 2)) * 2;
+    }
+    uint8_t* ring = smem + 2 * kFragBytes + warp * kRingBytes;
+    auto issue = [&](int step) {             // step relative to s_begin; one commit group per call
+        if (step < n_total) {
+            uint8_t* slot = ring + (step % kDepth) * kSlotBytes;
+#pragma unroll
+            for (int i = 0; i < kTiles; ++i) {
+                cp_async16(slot + i * 512 + lane * 16, pc[i] + (int64_t)step * 64);
+                cp_async4(slot + kSlotCodes + i * 128 + lane * 4, ps[i] + (int64_t)step * 8);
+            }
+        }
+        cp_async_commit();
+    };
+    // Activation fragments of a chunk of steps: contiguous in global memory, copied as they are into one of two
+    // buffers.  The copies are not committed on their own: they join the next group of the weight stream, which
+    // is waited for before the chunk's first step.
+    auto issue_fragments = [&](int chunk) {
+        const int first = chunk * kChunkSteps;
+        if (first >= n_total) return;
+        const int n_steps = n_total - first < kChunkSteps ? n_total - first : kChunkSteps;
+        const uint4* src = frag + (s_begin + first) * (kStepBytes / 16);
+        uint4* dst = reinterpret_cast<uint4*>(smem + (chunk & 1) * kFragBytes);
+        for (int i = threadIdx.x; i < n_steps * (kStepBytes / 16); i += kThreads) cp_async16(dst + i, src + i);
+    };
+    issue_fragments(0);
+#pragma unroll
+    for (int d = 0; d < kDepth; ++d) issue(d);
+
+    float acc[kTiles][4];
+#pragma unroll
+    for (int i = 0; i < kTiles; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    for (int step = 0; step < n_total; ++step) {
+        cp_async_wait<kDepth - 1>();                             // this step's group has landed
+        const int chunk = step / kChunkSteps, s = step % kChunkSteps;
+        if (s == 0) {
+            __syncthreads();             // the chunk's fragments are visible; the other buffer is no longer read
+            issue_fragments(chunk + 1);
+        }
+        const uint8_t* slot = ring + (step % kDepth) * kSlotBytes;
+        const uint4* a = reinterpret_cast<const uint4*>(smem + (chunk & 1) * kFragBytes + s * kStepBytes) + lane;
+        uint4 a_lo[4], a_hi[4];                                  // rows g and g + 8, elements 8j .. 8j + 7
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            a_lo[j] = a[(j * 2) * 32];
+            a_hi[j] = a[(j * 2 + 1) * 32];
+        }
+#pragma unroll
+        for (int i = 0; i < kTiles; ++i) {
+            const uint4 cw = *reinterpret_cast<const uint4*>(slot + i * 512 + lane * 16);
+            const uint32_t sw = *reinterpret_cast<const uint32_t*>(slot + kSlotCodes + i * 128 + lane * 4);
+            const GroupScales gs = make_scales((t & 1) ? sw >> 16 : sw & 0xFFFFu);
+            const uint32_t w[4] = {cw.x, cw.y, cw.z, cw.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint4 b = decode_pairs(w[j], gs);
+                mma_bf16(acc[i], a_lo[j].x, a_hi[j].x, a_lo[j].y, a_hi[j].y, b.x, b.y);
+                mma_bf16(acc[i], a_lo[j].z, a_hi[j].z, a_lo[j].w, a_hi[j].w, b.z, b.w);
+            }
+        }
+        issue(step + kDepth);                                    // refill the slot just consumed
+    }
+    cp_async_wait<0>();
+
+    // Partial products of this range of K: [16 token rows][128 weight rows] in shared memory, then every CTA of
+    // the cluster adds its share of the outputs over all ranks, in rank order.
+    __syncthreads();
+    float* part = reinterpret_cast<float*>(smem);
+#pragma unroll
+    for (int i = 0; i < kTiles; ++i) {
+        const int col = warp * (kTiles * 8) + i * 8 + 2 * t;
+        *reinterpret_cast<float2*>(part + g * kPartPitch + col) = make_float2(acc[i][0], acc[i][1]);
+        *reinterpret_cast<float2*>(part + (g + 8) * kPartPitch + col) = make_float2(acc[i][2], acc[i][3]);
+    }
+    cluster.sync();
+    const int per = kMaxRows * kCtaRows / slices;                // outputs this CTA adds up (a multiple of 128)
+    for (int o = slice * per + threadIdx.x; o < (slice + 1) * per; o += kThreads) {
+        const int m = o / kCtaRows, col = o % kCtaRows;
+        float v[kMaxSlices];
+#pragma unroll
+        for (int r = 0; r < kMaxSlices; ++r)                     // all remote reads in flight together
+            v[r] = r < slices ? cluster.map_shared_rank(part, r)[m * kPartPitch + col] : 0.f;
+        float sum = 0.f;
+#pragma unroll
+        for (int r = 0; r < kMaxSlices; ++r) sum += v[r];
+        const int64_t n = (int64_t)blockIdx.x * kCtaRows + col;
+        if (m < M && n < N) C[m * ld_c + n] = sum;
+    }
+    cluster.sync();                                              // no CTA leaves while its tile is still read
+}
+
+// How many clusters of `slices` CTAs the device holds at once (asked once per cluster size; 0 if the query fails).
+int resident_clusters(int slices) {
+    static int cached[kMaxSlices + 1] = {};
+    if (cached[slices]) return cached[slices] > 0 ? cached[slices] : 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(1, (unsigned)slices, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = (unsigned)slices;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_rows_kernel, &cfg) != cudaSuccess || n <= 0) {
+        cudaGetLastError();
+        n = -1;
+    }
+    cached[slices] = n;
+    return n > 0 ? n : 0;
+}
+
+// Ranges of K per 128 weight rows: as many as give every range at least two steps and still let all clusters
+// be resident at once (a second wave of CTAs would start its stream from an empty pipeline).
+int slices_for(int64_t N, int64_t K) {
+    const int64_t steps = K / kStepK, row_blocks = (N + kCtaRows - 1) / kCtaRows;
+    int s = kMaxSlices;
+    while (s > 1 && (steps < 2 * s || row_blocks > resident_clusters(s))) s >>= 1;
+    return s;
+}
+
+int launch_rows(const uint4* frag, const uint8_t* w_codes, const uint8_t* w_scales, int64_t M, int64_t N, int64_t K,
+                float* C, int64_t ld_c, cudaStream_t st) {
+    static bool configured[64] = {};         // the opt-in to > 48 KB of dynamic shared memory is per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AMX_ERR_CUDA;
+    if (!configured[dev]) {
+        if (cudaFuncSetAttribute(gemm_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) {
+            cudaGetLastError();
+            return AMX_ERR_CUDA;
+        }
+        configured[dev] = true;
+    }
+    const int slices = slices_for(N, K);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((N + kCtaRows - 1) / kCtaRows), (unsigned)slices, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = (unsigned)slices;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, gemm_rows_kernel, frag, w_codes, w_scales, (int)M, N, K, C, ld_c) != cudaSuccess) {
+        cudaGetLastError();
+        return AMX_ERR_CUDA;
+    }
+    return AMX_OK;
+}
+
+}  // namespace
+
+bool gemm_rows_supported(int64_t M, int64_t N, int64_t K, int gs) {
+    return gs == 32 && M >= 1 && M <= kMaxRows && N >= 1 && K >= kStepK && K % kStepK == 0 &&
+           (N + kCtaRows - 1) / kCtaRows <= 0x7FFFFFFF;
+}
+
+size_t gemm_rows_workspace_bytes(int64_t K) { return (size_t)kMaxRows * (size_t)K * 2; }
+
+int gemm_rows(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes, const uint8_t* w_scales,
+              int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {
+    uint4* frag = static_cast<uint4*>(workspace);
+    const int64_t threads = kMaxRows * (K / 32);
+    rows_fragments_kernel<false><<<(unsigned)((threads + 127) / 128), 128, 0, st>>>(a_codes, a_scales, nullptr, 0, (int)M,
+                                                                                   K, frag);
+    if (launch_status() != AMX_OK) return AMX_ERR_CUDA;
+    return launch_rows(frag, w_codes, w_scales, M, N, K, C, ld_c, st);
+}
+
+int gemm_rows_cast(const void* x, int64_t ld_x, const uint8_t* w_codes, const uint8_t* w_scales, int64_t M, int64_t N,
+                   int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {
+    uint4* frag = static_cast<uint4*>(workspace);
+    const int64_t threads = kMaxRows * (K / 32);
+    rows_fragments_kernel<true><<<(unsigned)((threads + 127) / 128), 128, 0, st>>>(
+        nullptr, nullptr, static_cast<const uint16_t*>(x), ld_x, (int)M, K, frag);
+    if (launch_status() != AMX_OK) return AMX_ERR_CUDA;
+    return launch_rows(frag, w_codes, w_scales, M, N, K, C, ld_c, st);
+}
+
+}  // namespace amx

@@ -57,7 +57,7 @@ def test_host_detected_argument_errors(L):
     assert L.amx_dequantize(fake, fake, 4, 64, 32, 0, None, 64, None) == -1
     g = L.amx_gemm
     assert g(fake, fake, fake, fake, 4, 4, 64, 32, 0x30, fake, 4, None, 0, None) == -5  # both kernels asked
-    assert g(fake, fake, fake, fake, 4, 4, 64, 32, 0x100, fake, 4, None, 0, None) == -5
+    assert g(fake, fake, fake, fake, 4, 4, 64, 32, 0x200, fake, 4, None, 0, None) == -5
     assert g(fake, fake, fake, fake, 4, 8, 64, 32, 0, fake, 4, None, 0, None) == -2     # ld_c < N
     assert g(None, fake, fake, fake, 4, 4, 64, 32, 0x10, fake, 4, None, 0, None) == -1
     assert g(fake, fake, fake, fake, 0, 4, 64, 32, 0x10, fake, 4, None, 0, None) == 0   # empty

@@ -321,6 +321,52 @@ def test_gemm_prepared_few_tiles_long_k(M, N, K):
     assert rel_fro(one.cpu().numpy(), ref) <= 1e-5
 
 
+@pytest.mark.parametrize("M,N,K,kind", [(16, 4096, 4096, "normal"), (1, 12288, 4096, "normal"), (5, 600, 1024, "wide"),
+                                        (16, 8, 128, "mixed"), (3, 130, 256, "normal"), (7, 256, 11008, "normal"),
+                                        (16, 1030, 11264, "mixed"), (9, 129, 640, "wide")])
+def test_gemm_rows_weight_streaming(M, N, K, kind):
+    """At most 16 token rows against a canonical weight (decode phase): the weight-streaming kernel decodes both
+    operands exactly, cuts K into ranges over a cluster and adds them in rank order: close to the fp64 oracle,
+    run-to-run identical, padded output untouched; AUTO picks it, and amx_quant_gemm (cast of the rows fused with
+    their decode) gives the same bits."""
+    a_bits = inputs.random_groups(900 + M, M, K, kind)
+    w_bits = inputs.random_groups(901 + N, N, K, kind)
+    qa, qw = oracle.quantize(a_bits, 32), oracle.quantize(w_bits, 32)
+    ref = oracle.gemm(*qa, *qw, 32)
+    dev = [torch.from_numpy(t).cuda() for t in (*qa, *qw)]
+    assert amx.lib().amx_gemm_kernel_for(M, N, K, 32, amx.GEMM_ROWS) == amx.GEMM_ROWS
+    wide = torch.full((M, N + 12), 5.0, dtype=torch.float32, device="cuda")
+    got = amx.gemm(*dev, 32, amx.GEMM_ROWS, out=wide[:, :N])
+    g = got.cpu().numpy().astype(np.float64)
+    if kind == "wide":                           # rows differ by many orders of magnitude: row by row
+        for m in range(M):
+            if np.all(np.isfinite(ref[m])) and np.linalg.norm(ref[m]) > 0:
+                assert rel_fro(g[m], ref[m]) <= 1e-5
+    else:
+        assert rel_fro(g, ref) <= 1e-5
+    assert torch.all(wide[:, N:] == 5.0)
+    assert torch.equal(amx.gemm(*dev, 32, amx.GEMM_ROWS), got.contiguous())
+    if K >= 512:
+        assert amx.lib().amx_gemm_kernel_for(M, N, K, 32, amx.GEMM_AUTO) == amx.GEMM_ROWS
+    fused = amx.quant_gemm(dev_bf16(a_bits), dev[2], dev[3], 32, flags=amx.GEMM_ROWS)
+    assert torch.equal(fused, got.contiguous())
+
+
+def test_gemm_rows_exact_on_small_integers():
+    """Integer-valued operands: every product and partial sum is exact in fp32, so any summation order gives the
+    integer result - an independent check of the fragment order and the K ranges."""
+    rng = np.random.default_rng(11)
+    grid = np.array([0, 1, 2, 3, 4, 6], np.float32)
+    def ints(r, k):
+        t = grid[rng.integers(0, 6, size=(r, k))] * rng.choice([-1.0, 1.0], size=(r, k)).astype(np.float32)
+        t[:, ::32], t[:, 1::32] = 6.0, -6.0
+        return t
+    a, w = ints(13, 2304), ints(300, 2304)
+    qa, qw = oracle.quantize(inputs.f32_to_bf16_bits(a), 32), oracle.quantize(inputs.f32_to_bf16_bits(w), 32)
+    got = amx.gemm(*(torch.from_numpy(t).cuda() for t in (*qa, *qw)), 32, amx.GEMM_ROWS).cpu().numpy()
+    assert np.array_equal(got, (a.astype(np.int64) @ w.astype(np.int64).T).astype(np.float32))
+
+
 def test_fp4_path_shape_sweep():
     """Seeded sweep of ragged shapes through the fused cast and the FP4 kernel (prepared buffers pre-filled with
     0xFF, padded output), against the oracle on the oracle's own codes."""
