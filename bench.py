@@ -202,6 +202,119 @@ def time_attention(heads: int, iters: int = 3):
                                            "keys after their queries are skipped in all three products"}}
 
 
+def time_decode(steps: int, A=None, W=None):
+    """Decode-like shape: 16 token rows against the config-2 weights (cast once), amx_quant_gemm per layer, replayed as
+    a CUDA graph.  Bound by streaming the 4.5-bit weights: reports the rate at which they are read."""
+    import torch
+    from paper_2411_09909_b200 import amx, inputs
+    L = amx.lib()
+    peaks = measured_peaks()
+    _, layers = layer_shapes()
+    if A is None:
+        def to_dev(bits):
+            return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+        A = [to_dev(inputs.activation(2, li)[:16]) for li in range(len(layers))]
+        W = [to_dev(inputs.weight(2, li)) for li in range(len(layers))]
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def check(rc):
+        if rc != 0:
+            raise RuntimeError(amx.status_string(rc))
+
+    Md = 16
+    REPS = 3                      # distinct copies of the weights: 3 x 88 MB of codes and scales exceed the L2
+    dd = []
+    for li, (K, N) in enumerate(layers):
+        wc_, ws_ = amx.quantize(W[li], GS)
+        ad = A[li][:Md].contiguous()
+        need = max(L.amx_quant_gemm_workspace_bytes(Md, N, K, GS, 0), 256)
+        dd.append((ad, [(wc_.clone(), ws_.clone()) for _ in range(REPS)],
+                   torch.empty((Md, N), dtype=torch.float32, device="cuda"),
+                   torch.empty(need, dtype=torch.uint8, device="cuda")))
+        del wc_, ws_
+    decode_kernel = L.amx_gemm_kernel_for(Md, layers[0][1], layers[0][0], GS, 0)
+
+    def decode_step(stream, rep=0):
+        for li, (K, N) in enumerate(layers):
+            ad, wq, cd, wsd = dd[li]
+            wc_, ws_ = wq[rep]
+            check(L.amx_quant_gemm(ad.data_ptr(), K, wc_.data_ptr(), ws_.data_ptr(), Md, N, K, GS, 0, cd.data_ptr(), N,
+                                   wsd.data_ptr(), wsd.numel(), stream))
+
+    decode_step(stream)
+    torch.cuda.synchronize()
+    sd = torch.cuda.Stream()
+    sd.wait_stream(torch.cuda.current_stream())
+    gd = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(gd, stream=sd):
+        for rep in range(REPS):
+            decode_step(torch.cuda.current_stream().cuda_stream, rep)
+    for _ in range(3):
+        gd.replay()
+    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    d0.record()
+    for _ in range(steps):
+        gd.replay()
+    d1.record()
+    torch.cuda.synchronize()
+    d_us = d0.elapsed_time(d1) / (steps * REPS) * 1e3
+    w_bytes = sum(N * K for K, N in layers) * (0.5 + 2.0 / 32.0)
+    # the same with the weights prepared once for the FP4 kernel (amx_quantize_prepared + amx_gemm_prepared)
+    dp = []
+    cw_ = [torch.empty((N, K // 2), dtype=torch.uint8, device="cuda") for K, N in layers]
+    cs_ = [torch.empty((N, K // GS, 2), dtype=torch.uint8, device="cuda") for K, N in layers]
+    for li, (K, N) in enumerate(layers):
+        pw_ = torch.empty(L.amx_prepared_bytes(N, K, GS, 1), dtype=torch.uint8, device="cuda")
+        check(L.amx_quantize_prepared(W[li].data_ptr(), N, K, GS, 1, cw_[li].data_ptr(), cs_[li].data_ptr(),
+                                      pw_.data_ptr(), pw_.numel(), stream))
+        dp.append((pw_, torch.empty(L.amx_prepared_bytes(Md, K, GS, 0), dtype=torch.uint8, device="cuda"),
+                   torch.empty((Md, K // 2), dtype=torch.uint8, device="cuda"),
+                   torch.empty((Md, K // GS, 2), dtype=torch.uint8, device="cuda"),
+                   torch.empty(max(L.amx_gemm_prepared_workspace_bytes(Md, N, K, GS), 256), dtype=torch.uint8, device="cuda")))
+
+    def decode_prepared_step(stream):
+        for li, (K, N) in enumerate(layers):
+            ad, _, cd, _ = dd[li]
+            pw_, pa_, ac_, as_, wsp = dp[li]
+            check(L.amx_quantize_prepared(ad.data_ptr(), Md, K, GS, 0, ac_.data_ptr(), as_.data_ptr(), pa_.data_ptr(),
+                                          pa_.numel(), stream))
+            check(L.amx_gemm_prepared(pa_.data_ptr(), pw_.data_ptr(), Md, N, K, GS, cd.data_ptr(), N, wsp.data_ptr(),
+                                      wsp.numel(), stream))
+
+    decode_prepared_step(stream)
+    torch.cuda.synchronize()
+    sp = torch.cuda.Stream()
+    sp.wait_stream(torch.cuda.current_stream())
+    gp = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(gp, stream=sp):
+        decode_prepared_step(torch.cuda.current_stream().cuda_stream)
+    for _ in range(3):
+        gp.replay()
+    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    p0.record()
+    for _ in range(steps):
+        gp.replay()
+    p1.record()
+    torch.cuda.synchronize()
+    dp_us = p0.elapsed_time(p1) / steps * 1e3
+    del dp
+    decode = {"workload": f"{Md} token rows x the four config-2 weights (cast once; {REPS} copies of the weights in turn, "
+                          "so that they come from HBM, not from the L2); amx_quant_gemm per layer, graph replay",
+              "prepared_weights": {"us_per_step": dp_us,
+                                   "what": "weights prepared once for the FP4 kernel (1.06 B/element resident), per layer "
+                                           "amx_quantize_prepared of the rows + amx_gemm_prepared with K ranges",
+                                   "weight_gb_per_s_canonical_bytes": sum(N * K for K, N in layers) * 0.5625 / (dp_us * 1e-6) / 1e9},
+              "us_per_step": d_us, "weight_gb_per_s": w_bytes / (d_us * 1e-6) / 1e9,
+              "frac_of_measured_copy": w_bytes / (d_us * 1e-6) / 1e9 / peaks["hbm_gbs"],
+              "launches_per_step": 2 * len(layers),
+              "kernel": ("weight-streaming kernel (canonical weights read once, exact bf16 decode, mma.sync; K ranges "
+                         "added over a thread-block cluster)" if decode_kernel == amx.GEMM_ROWS
+                         else "tcgen05 kind::f16 (bf16 decode), K cut into slices over CTAs")}
+    return decode
+
+
 def run_ours(args):
     import torch
     from paper_2411_09909_b200 import amx, inputs, build, sharding
@@ -526,100 +639,10 @@ def run_ours(args):
                       "us_per_call": s0.elapsed_time(s1) * 1e3 / 200,
                       "note": "launch-latency-bound (32 output tiles at most): microseconds, not a roofline fraction"}
 
-    # ---- decode-like shape: 16 token rows against the config-2 weights (cast once), amx_quant_gemm per layer,
-    # replayed as a CUDA graph.  Bound by streaming the 4.5-bit weights: report the rate at which they are read.
+    # ---- decode-like shape: 16 token rows against the config-2 weights (see time_decode)
     decode = None
     if not args.layers and not args.skip_extras and world == 1 and CONFIG == 2:
-        Md = 16
-        REPS = 3                      # distinct copies of the weights: 3 x 88 MB of codes and scales exceed the L2
-        dd = []
-        for li, (K, N) in enumerate(layers):
-            wc_, ws_ = amx.quantize(W[li], GS)
-            ad = A[li][:Md].contiguous()
-            need = max(L.amx_quant_gemm_workspace_bytes(Md, N, K, GS, 0), 256)
-            dd.append((ad, [(wc_.clone(), ws_.clone()) for _ in range(REPS)],
-                       torch.empty((Md, N), dtype=torch.float32, device="cuda"),
-                       torch.empty(need, dtype=torch.uint8, device="cuda")))
-            del wc_, ws_
-        decode_kernel = L.amx_gemm_kernel_for(Md, layers[0][1], layers[0][0], GS, 0)
-
-        def decode_step(stream, rep=0):
-            for li, (K, N) in enumerate(layers):
-                ad, wq, cd, wsd = dd[li]
-                wc_, ws_ = wq[rep]
-                check(L.amx_quant_gemm(ad.data_ptr(), K, wc_.data_ptr(), ws_.data_ptr(), Md, N, K, GS, 0, cd.data_ptr(), N,
-                                       wsd.data_ptr(), wsd.numel(), stream))
-
-        decode_step(stream)
-        torch.cuda.synchronize()
-        sd = torch.cuda.Stream()
-        sd.wait_stream(torch.cuda.current_stream())
-        gd = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(gd, stream=sd):
-            for rep in range(REPS):
-                decode_step(torch.cuda.current_stream().cuda_stream, rep)
-        for _ in range(3):
-            gd.replay()
-        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        d0.record()
-        for _ in range(args.steps):
-            gd.replay()
-        d1.record()
-        torch.cuda.synchronize()
-        d_us = d0.elapsed_time(d1) / (args.steps * REPS) * 1e3
-        w_bytes = sum(N * K for K, N in layers) * (0.5 + 2.0 / 32.0)
-        # the same with the weights prepared once for the FP4 kernel (amx_quantize_prepared + amx_gemm_prepared)
-        dp = []
-        for li, (K, N) in enumerate(layers):
-            pw_ = torch.empty(L.amx_prepared_bytes(N, K, GS, 1), dtype=torch.uint8, device="cuda")
-            check(L.amx_quantize_prepared(W[li].data_ptr(), N, K, GS, 1, bufs[li]["wc"].data_ptr(), bufs[li]["ws"].data_ptr(),
-                                          pw_.data_ptr(), pw_.numel(), stream))
-            dp.append((pw_, torch.empty(L.amx_prepared_bytes(Md, K, GS, 0), dtype=torch.uint8, device="cuda"),
-                       torch.empty((Md, K // 2), dtype=torch.uint8, device="cuda"),
-                       torch.empty((Md, K // GS, 2), dtype=torch.uint8, device="cuda"),
-                       torch.empty(max(L.amx_gemm_prepared_workspace_bytes(Md, N, K, GS), 256), dtype=torch.uint8, device="cuda")))
-
-        def decode_prepared_step(stream):
-            for li, (K, N) in enumerate(layers):
-                ad, _, cd, _ = dd[li]
-                pw_, pa_, ac_, as_, wsp = dp[li]
-                check(L.amx_quantize_prepared(ad.data_ptr(), Md, K, GS, 0, ac_.data_ptr(), as_.data_ptr(), pa_.data_ptr(),
-                                              pa_.numel(), stream))
-                check(L.amx_gemm_prepared(pa_.data_ptr(), pw_.data_ptr(), Md, N, K, GS, cd.data_ptr(), N, wsp.data_ptr(),
-                                          wsp.numel(), stream))
-
-        decode_prepared_step(stream)
-        torch.cuda.synchronize()
-        sp = torch.cuda.Stream()
-        sp.wait_stream(torch.cuda.current_stream())
-        gp = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(gp, stream=sp):
-            decode_prepared_step(torch.cuda.current_stream().cuda_stream)
-        for _ in range(3):
-            gp.replay()
-        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        p0.record()
-        for _ in range(args.steps):
-            gp.replay()
-        p1.record()
-        torch.cuda.synchronize()
-        dp_us = p0.elapsed_time(p1) / args.steps * 1e3
-        del dp
-        decode = {"workload": f"{Md} token rows x the four config-2 weights (cast once; {REPS} copies of the weights in turn, "
-                              "so that they come from HBM, not from the L2); amx_quant_gemm per layer, graph replay",
-                  "prepared_weights": {"us_per_step": dp_us,
-                                       "what": "weights prepared once for the FP4 kernel (1.06 B/element resident), per layer "
-                                               "amx_quantize_prepared of the rows + amx_gemm_prepared with K ranges",
-                                       "weight_gb_per_s_canonical_bytes": sum(N * K for K, N in layers) * 0.5625 / (dp_us * 1e-6) / 1e9},
-                  "us_per_step": d_us, "weight_gb_per_s": w_bytes / (d_us * 1e-6) / 1e9,
-                  "frac_of_measured_copy": w_bytes / (d_us * 1e-6) / 1e9 / peaks["hbm_gbs"],
-                  "launches_per_step": 2 * len(layers),
-                  "kernel": ("weight-streaming kernel (canonical weights read once, exact bf16 decode, mma.sync; K ranges "
-                             "added over a thread-block cluster)" if decode_kernel == amx.GEMM_ROWS
-                             else "tcgen05 kind::f16 (bf16 decode), K cut into slices over CTAs")}
-        del dd
+        decode = time_decode(args.steps, A, W)
 
     # ---- end to end through the host-buffer entry point (pinned host tensors, copies inside the timing)
     e2e = None
@@ -734,6 +757,7 @@ def main():
     ap.add_argument("--skip-extras", action="store_true", help="skip the e2e and cpu_baseline legs (profiling aid)")
     ap.add_argument("--attention-only", action="store_true", help="time only the config-5 attention call (profiling aid)")
     ap.add_argument("--heads", type=int, default=32, help="heads for --attention-only")
+    ap.add_argument("--decode-only", action="store_true", help="time only the 16-row decode step (profiling aid)")
     ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4],
                     help="linear-layer workload (default 2, the one the metric is quoted on; 3 and 4 are larger)")
     args = ap.parse_args()
@@ -745,6 +769,12 @@ def main():
         torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
         build.build()
         print(json.dumps({"attention": time_attention(args.heads, iters=1)}))
+    elif args.decode_only:
+        import torch
+        from paper_2411_09909_b200 import build
+        torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+        build.build()
+        print(json.dumps({"decode": time_decode(args.steps)}))
     elif args.impl == "reference":
         run_reference(args)
     else:
