@@ -50,6 +50,7 @@ def lib() -> ctypes.CDLL:
         L.amx_oracle_quantize_f64.argtypes = [p, i64, i64, ctypes.c_int, p, p]
         L.amx_oracle_dequantize.argtypes = [p, p, i64, i64, ctypes.c_int, p]
         L.amx_oracle_gemm.argtypes = [p, p, p, p, i64, i64, i64, ctypes.c_int, p, i64, p]
+        L.amx_oracle_quant_error.argtypes = [p, i64, i64, i64, p, p, ctypes.c_int, p]
         L.amx_oracle_fakequant_pot_floor.argtypes = [p, i64, i64, ctypes.c_int, ctypes.c_int, p]
         L.amx_oracle_softmax_bf16.argtypes = [p, i64, i64, dbl, p]
         L.amx_oracle_softmax_bf16_causal.argtypes = [p, i64, i64, dbl, i64, p]
@@ -145,6 +146,17 @@ def dequantize(codes: np.ndarray, scales: np.ndarray, group_size: int = 32) -> n
     rc = lib().amx_oracle_dequantize(_ptr(codes), _ptr(scales), rows, K, group_size, _ptr(out))
     if rc:
         raise ValueError(f"amx_oracle_dequantize: bad shape (rc={rc})")
+    return out
+
+
+def quant_error(x_bf16_bits: np.ndarray, codes: np.ndarray, scales: np.ndarray, group_size: int = 32) -> np.ndarray:
+    """[sum x^2, sum (x - xhat)^2, its part from clamped elements (|x| > 6 * side scale), their count] in fp64."""
+    x, codes, scales = _c(x_bf16_bits, np.uint16), _c(codes, np.uint8), _c(scales, np.uint8)
+    rows, K = x.shape
+    out = np.zeros(4, np.float64)
+    rc = lib().amx_oracle_quant_error(_ptr(x), rows, K, K, _ptr(codes), _ptr(scales), group_size, _ptr(out))
+    if rc:
+        raise ValueError(f"amx_oracle_quant_error: bad shape (rc={rc})")
     return out
 
 

@@ -300,6 +300,44 @@ int amx_oracle_dequantize(const uint8_t *codes, const uint8_t *scales,
     return 0;
 }
 
+/* --------------------------------------------------- quantization error -- */
+
+/*
+ * Squared error of a quantized tensor against its bf16 source, split the way
+ * the appendix on power-of-two scales (floor vs. round) splits it: an element
+ * whose magnitude exceeds the largest value its side can represent
+ * (|x| > 6 * scale of its side) contributes to the max-clamping error, every
+ * other element to the rounding error.
+ * out[0] = sum x^2, out[1] = sum (x - xhat)^2 over all elements,
+ * out[2] = the part of out[1] from clamped elements, out[3] = their count.
+ * Plain fp64 sums in index order.
+ */
+int amx_oracle_quant_error(const uint16_t *x, int64_t rows, int64_t K, int64_t ld,
+                           const uint8_t *codes, const uint8_t *scales, int gs, double *out)
+{
+    if (gs <= 0 || K % gs != 0 || (K & 1))
+        return -1;
+    int64_t G = K / gs;
+    double sx = 0.0, se = 0.0, sc_err = 0.0, n_clamped = 0.0;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t k = 0; k < K; ++k) {
+            double v = bf16_to_double(x[r * ld + k]);
+            uint8_t byte = codes[r * (K / 2) + k / 2];
+            int c = (k & 1) ? (byte >> 4) : (byte & 15);
+            const uint8_t *sc = scales + (r * G + k / gs) * 2;
+            double s = amx_oracle_e5m2_value((c & 8) ? sc[1] : sc[0]);
+            double e = v - amx_oracle_e2m1_value(c) * s;
+            sx += v * v;
+            se += e * e;
+            if (fabs(v) > 6.0 * s) {
+                sc_err += e * e;
+                n_clamped += 1.0;
+            }
+        }
+    out[0] = sx; out[1] = se; out[2] = sc_err; out[3] = n_clamped;
+    return 0;
+}
+
 /* ---------------------------------------------------------------- GEMM -- */
 
 /*
