@@ -268,12 +268,30 @@ int amx_quant_gemm_static(const void* A, int64_t ld_a,
                           float* C, int64_t ld_c, void* stream);
 size_t amx_quant_gemm_static_capacity(void);
 
+/*
+ * amx_quant_error - squared error of a quantized tensor against its bf16 source, split as the appendix
+ * "Determining PoT Shared Scale: Floor vs. Round" splits the error of a shared scale: elements whose magnitude
+ * exceeds the largest value their side represents (|x| > 6 * scale of the element's side) make up the
+ * max-clamping error, all others the rounding error.
+ *   x, codes, scales   as for amx_quantize / amx_quantize_fmt (any of the formats, group size 16..128);
+ *                      x 16-byte aligned with ld_x % 8 == 0, codes 8-byte aligned
+ *   out        device, 4 doubles: sum x^2, sum (x - xhat)^2, the part of the latter from clamped elements,
+ *              the number of clamped elements.  fp64 sums in a fixed order: the same bits on every run.
+ *   workspace  device scratch of amx_quant_error_workspace_bytes() bytes, 8-byte aligned
+ * Two launches on `stream`; nothing is synchronised.  rows == 0 writes zeros.
+ */
+int amx_quant_error(const void* x, int64_t rows, int64_t K, int64_t ld_x, const uint8_t* codes,
+                    const uint8_t* scales, int group_size, double* out, void* workspace, size_t workspace_bytes,
+                    void* stream);
+size_t amx_quant_error_workspace_bytes(void);
+
 /* Scratch sizes (bytes; 0 is possible).  Return 0 for invalid shapes. */
 size_t amx_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags);
 size_t amx_quant_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags);
 size_t amx_linear_host_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size);
 
-/* Which kernel amx_gemm would run for this shape and flags: AMX_GEMM_SIMT or AMX_GEMM_TC. */
+/* Which kernel amx_gemm would run for this shape and flags: one AMX_GEMM_* kernel bit, or 0 when the flags
+ * cannot be honoured for the shape. */
 uint32_t amx_gemm_kernel_for(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags);
 
 /*

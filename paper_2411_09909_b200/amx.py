@@ -32,6 +32,7 @@ SYMBOLS = (
     "amx_attention", "amx_attention_workspace_bytes",
     "amx_prepared_bytes", "amx_prepare", "amx_gemm_prepared", "amx_quantize_prepared", "amx_softmax_quantize",
     "amx_quantize_fmt", "amx_quantize_prepared_fmt", "amx_gemm_prepared_workspace_bytes",
+    "amx_quant_error", "amx_quant_error_workspace_bytes",
 )
 
 
@@ -52,6 +53,9 @@ def lib() -> ctypes.CDLL:
         L.amx_quantize_prepared_fmt.argtypes = [p, i64, i64, i, i, i, p, p, p, sz, p]
         L.amx_dequantize.argtypes = [p, p, i64, i64, i, u32, p, i64, p]
         L.amx_gemm.argtypes = [p, p, p, p, i64, i64, i64, i, u32, p, i64, p, sz, p]
+        L.amx_quant_error.argtypes = [p, i64, i64, i64, p, p, i, p, p, sz, p]
+        L.amx_quant_error_workspace_bytes.argtypes = []
+        L.amx_quant_error_workspace_bytes.restype = sz
         L.amx_quant_gemm.argtypes = [p, i64, p, p, i64, i64, i64, i, u32, p, i64, p, sz, p]
         L.amx_quant_gemm_static.argtypes = [p, i64, p, p, i64, i64, i64, i, u32, p, i64, p]
         L.amx_quant_gemm_static_capacity.argtypes = []
@@ -142,6 +146,18 @@ def dequantize(codes: torch.Tensor, scales: torch.Tensor, group_size: int = 32, 
     flag = {torch.bfloat16: OUT_BF16, torch.float32: OUT_F32}[dtype]
     _check(lib().amx_dequantize(codes.data_ptr(), scales.data_ptr(), rows, K, group_size, flag,
                                 out.data_ptr(), K, _stream()), "amx_dequantize")
+    return out
+
+
+def quant_error(x: torch.Tensor, codes: torch.Tensor, scales: torch.Tensor, group_size: int = 32) -> torch.Tensor:
+    """Device tensor of 4 doubles: sum x^2, sum (x - xhat)^2, its part from clamped elements, their count."""
+    _dev(x, torch.bfloat16, "x"), _dev(codes, torch.uint8, "codes"), _dev(scales, torch.uint8, "scales")
+    assert x.dim() == 2 and x.stride(1) == 1 and codes.is_contiguous() and scales.is_contiguous()
+    rows, K = x.shape
+    out = torch.empty(4, dtype=torch.float64, device=x.device)
+    ws = torch.empty(lib().amx_quant_error_workspace_bytes(), dtype=torch.uint8, device=x.device)
+    _check(lib().amx_quant_error(x.data_ptr(), rows, K, x.stride(0), codes.data_ptr(), scales.data_ptr(), group_size,
+                                 out.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "amx_quant_error")
     return out
 
 

@@ -367,6 +367,28 @@ def test_gemm_rows_exact_on_small_integers():
     assert np.array_equal(got, (a.astype(np.int64) @ w.astype(np.int64).T).astype(np.float32))
 
 
+@pytest.mark.parametrize("fmt", [amx.FMT_AMXFP4, amx.FMT_SYM_FP8, amx.FMT_MXFP4])
+@pytest.mark.parametrize("gs", [16, 32, 64, 128])
+def test_quant_error_against_oracle(fmt, gs):
+    """Error split (max-clamping / rounding) of every format and group size: the clamped count is exact, the fp64
+    sums agree with the oracle's up to summation order, and two runs give the same bits.  Ragged shape (rows and K
+    not multiples of the block's work), strided rows, inputs with clamping (power-of-two floor) and wide range."""
+    for kind, rows, K in (("normal", 37, 1152), ("mixed", 5, 256), ("normal", 300, 4096)):
+        bits = inputs.random_groups(1200 + gs + rows, rows, K, kind)
+        wide = torch.zeros((rows, K + 64), dtype=torch.bfloat16, device="cuda")
+        wide[:, :K] = dev_bf16(bits)
+        x = wide[:, :K]
+        codes, scales = amx.quantize(x, gs, fmt)
+        ref = oracle.quant_error(bits, codes.cpu().numpy(), scales.cpu().numpy(), gs)
+        got = amx.quant_error(x, codes, scales, gs)
+        g = got.cpu().numpy()
+        assert g[3] == ref[3]
+        assert np.allclose(g[:3], ref[:3], rtol=1e-12, atol=0)
+        assert torch.equal(amx.quant_error(x, codes, scales, gs), got)
+    empty = amx.quant_error(x[:0], codes[:0], scales[:0], gs)
+    assert torch.all(empty == 0)
+
+
 def test_fp4_path_shape_sweep():
     """Seeded sweep of ragged shapes through the fused cast and the FP4 kernel (prepared buffers pre-filled with
     0xFF, padded output), against the oracle on the oracle's own codes."""
