@@ -276,7 +276,9 @@ size_t amx_quant_gemm_static_capacity(void);
  *   x, codes, scales   as for amx_quantize / amx_quantize_fmt (any of the formats, group size 16..128);
  *                      x 16-byte aligned with ld_x % 8 == 0, codes 8-byte aligned
  *   out        device, 4 doubles: sum x^2, sum (x - xhat)^2, the part of the latter from clamped elements,
- *              the number of clamped elements.  fp64 sums in a fixed order: the same bits on every run.
+ *              the number of clamped elements (exact).  Squares are added in fp32 within chunks of 16 consecutive
+ *              elements and in fp64 above (relative error of a sum < 2^-20), in a fixed order: the same bits on
+ *              every run.
  *   workspace  device scratch of amx_quant_error_workspace_bytes() bytes, 8-byte aligned
  * Two launches on `stream`; nothing is synchronised.  rows == 0 writes zeros.
  */

@@ -370,8 +370,9 @@ def test_gemm_rows_exact_on_small_integers():
 @pytest.mark.parametrize("fmt", [amx.FMT_AMXFP4, amx.FMT_SYM_FP8, amx.FMT_MXFP4])
 @pytest.mark.parametrize("gs", [16, 32, 64, 128])
 def test_quant_error_against_oracle(fmt, gs):
-    """Error split (max-clamping / rounding) of every format and group size: the clamped count is exact, the fp64
-    sums agree with the oracle's up to summation order, and two runs give the same bits.  Ragged shape (rows and K
+    """Error split (max-clamping / rounding) of every format and group size: the clamped count is exact, the sums
+    agree with the oracle's fp64 sums to 2^-20 relative (the kernel adds the 16 non-negative squares of a chunk in
+    fp32: at most 16 roundings of 2^-24 each), and two runs give the same bits.  Ragged shape (rows and K
     not multiples of the block's work), strided rows, inputs with clamping (power-of-two floor) and wide range."""
     for kind, rows, K in (("normal", 37, 1152), ("mixed", 5, 256), ("normal", 300, 4096)):
         bits = inputs.random_groups(1200 + gs + rows, rows, K, kind)
@@ -383,7 +384,7 @@ def test_quant_error_against_oracle(fmt, gs):
         got = amx.quant_error(x, codes, scales, gs)
         g = got.cpu().numpy()
         assert g[3] == ref[3]
-        assert np.allclose(g[:3], ref[:3], rtol=1e-12, atol=0)
+        assert np.allclose(g[:3], ref[:3], rtol=2.0 ** -20, atol=0)
         assert torch.equal(amx.quant_error(x, codes, scales, gs), got)
     empty = amx.quant_error(x[:0], codes[:0], scales[:0], gs)
     assert torch.all(empty == 0)
