@@ -100,11 +100,14 @@ def quantize(x_bf16_bits: np.ndarray, group_size: int = 32):
 
 
 SYMMETRIC_FP8, MXFP4 = 1, 2
+AMXFP4_POT, MXFP4_POT_ROUND, AMXFP4_POT_ROUND = 3, 4, 5
 
 
 def quantize_variant(x_bf16_bits: np.ndarray, group_size: int, mode: int):
     """The symmetric comparison formats in AMXFP4's storage layout (both scale bytes equal): mode SYMMETRIC_FP8 =
-    one E5M2 scale per group from max|x| / 6; mode MXFP4 = Algorithm 1's power-of-two floor scale."""
+    one E5M2 scale per group from max|x| / 6; mode MXFP4 = Algorithm 1's power-of-two floor scale.  The per-sign
+    power-of-two variants (AMXFP4_POT: floor; *_POT_ROUND: exponent rounded instead of floored, symmetric or
+    per sign) use the two bytes like AMXFP4."""
     x = _c(x_bf16_bits, np.uint16)
     rows, K = x.shape
     codes = np.zeros((rows, K // 2), np.uint8)

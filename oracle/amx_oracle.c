@@ -216,36 +216,59 @@ int amx_oracle_quantize(const uint16_t *x, int64_t rows, int64_t K, int64_t ld, 
  * Element rounding, sign bit and zero-scale rules are those of the quantizer
  * above.
  */
+/* Scale byte of one side (or of the whole group) from its largest magnitude.
+ * rule 0: E5M2 nearest to max / 6 (Section 4.2);
+ * rule 1: Algorithm 1, 2^(floor(log2 max) - 2);
+ * rule 2: the same with the exponent rounded instead of floored (appendix
+ *         "Determining PoT Shared Scale: Floor vs. Round"), read as
+ *         2^(round(log2 max) - 2): one more than the floor when max is at
+ *         least sqrt(2) times its power of two. */
+static uint8_t variant_scale_byte(double amax, int rule)
+{
+    if (rule == 0)
+        return amx_oracle_e5m2_encode(amax / 6.0);
+    if (!(amax > 0.0))
+        return 0;
+    int e;
+    double f = 2.0 * frexp(amax, &e);          /* amax = f * 2^(e-1), 1 <= f < 2 */
+    int shared_exp = (e - 1) - 2;              /* floor(log2(amax)) - emax_elem */
+    if (rule == 2 && f * f >= 2.0)             /* log2 f >= 1/2 (f*f is exact: f has 8 bits) */
+        shared_exp += 1;
+    if (shared_exp > 15) shared_exp = 15;
+    return shared_exp < -16 ? 0 : amx_oracle_e5m2_encode(ldexp(1.0, shared_exp));
+}
+
+/* modes: 1 symmetric FP8 scale, 2 MXFP4 (power-of-two floor), 3 per-sign
+ * power-of-two floor ("AMXFP4, shared scale PoT" of Appendix B.3), 4 symmetric
+ * power-of-two round, 5 per-sign power-of-two round. */
 int amx_oracle_quantize_variant(const uint16_t *x, int64_t rows, int64_t K, int64_t ld, int gs,
                                 int mode, uint8_t *codes, uint8_t *scales)
 {
-    if (gs <= 0 || K % gs != 0 || (K & 1) || (mode != 1 && mode != 2))
+    if (gs <= 0 || K % gs != 0 || (K & 1) || mode < 1 || mode > 5)
         return -1;
+    const int per_sign = (mode == 3 || mode == 5);
+    const int rule = mode == 1 ? 0 : (mode == 2 || mode == 3) ? 1 : 2;
     int64_t G = K / gs;
 #pragma omp parallel for schedule(static)
     for (int64_t r = 0; r < rows; ++r)
         for (int64_t g = 0; g < G; ++g) {
             const uint16_t *xg = x + r * ld + g * gs;
-            double amax = 0.0;
+            double pmax = 0.0, nmax = 0.0;
             for (int i = 0; i < gs; ++i) {
                 double a = fabs(bf16_to_double(xg[i]));
-                if (a > amax) amax = a;
+                if (xg[i] >> 15) { if (a > nmax) nmax = a; }
+                else             { if (a > pmax) pmax = a; }
             }
-            uint8_t sb;
-            if (mode == 1) {
-                sb = amx_oracle_e5m2_encode(amax / 6.0);
-            } else if (amax > 0.0) {
-                int e;
-                frexp(amax, &e);                       /* amax = f * 2^e, 0.5 <= f < 1 */
-                int shared_exp = (e - 1) - 2;          /* floor(log2(amax)) - emax_elem */
-                if (shared_exp > 15) shared_exp = 15;
-                sb = shared_exp < -16 ? 0 : amx_oracle_e5m2_encode(ldexp(1.0, shared_exp));
+            uint8_t sb[2];
+            if (per_sign) {
+                sb[0] = variant_scale_byte(pmax, rule);
+                sb[1] = variant_scale_byte(nmax, rule);
             } else {
-                sb = 0;
+                sb[0] = sb[1] = variant_scale_byte(pmax > nmax ? pmax : nmax, rule);
             }
-            double sv = amx_oracle_e5m2_value(sb);
             for (int i = 0; i < gs; ++i) {
                 int sign = xg[i] >> 15;
+                double sv = amx_oracle_e5m2_value(sb[sign]);
                 int mag = sv > 0.0 ? amx_oracle_e2m1_encode(fabs(bf16_to_double(xg[i])) / sv) : 0;
                 uint8_t c = (uint8_t)((sign << 3) | mag);
                 int64_t k = g * gs + i;
@@ -253,8 +276,8 @@ int amx_oracle_quantize_variant(const uint16_t *x, int64_t rows, int64_t K, int6
                 if (k & 1) *byte = (uint8_t)((*byte & 0x0F) | (c << 4));
                 else       *byte = (uint8_t)((*byte & 0xF0) | c);
             }
-            scales[(r * G + g) * 2 + 0] = sb;
-            scales[(r * G + g) * 2 + 1] = sb;
+            scales[(r * G + g) * 2 + 0] = sb[0];
+            scales[(r * G + g) * 2 + 1] = sb[1];
         }
     return 0;
 }

@@ -75,3 +75,51 @@ def test_symmetric_formats_lose_to_amxfp4_on_skewed_groups():
                          "mx": oracle.quantize_variant(bits, 32, oracle.MXFP4)}.items():
         err[name] = np.mean((oracle.dequantize(c, s, 32) - xr) ** 2)
     assert err["amx"] < err["sym"] < err["mx"]
+
+
+def test_per_sign_power_of_two_reproduces_the_printed_value_set():
+    """Appendix B.3 prints the values of "AMXFP4 (Shared Scale: PoT)" on linspace(-4.9, 31, 1024) as one group."""
+    path = os.path.join(os.path.dirname(__file__), "golden", "worked_example.txt")
+    printed = next(line.split()[1:] for line in open(path) if line.startswith("amxfp4_pot "))
+    x = _bits(np.linspace(-4.9, 31, 1024, dtype=np.float32))[None, :]
+    c, s = oracle.quantize_variant(x, 1024, oracle.AMXFP4_POT)
+    assert np.unique(oracle.dequantize(c, s, 1024)).tolist() == sorted(float(t) for t in printed)
+    assert oracle.e5m2_value(int(s[0, 0, 0])) == 4.0 and oracle.e5m2_value(int(s[0, 0, 1])) == 1.0
+
+
+def test_per_sign_power_of_two_equals_algorithm1_per_sign():
+    bits = inputs.random_groups(35, 64, 256, "normal")
+    x = inputs.bf16_bits_to_f32(bits).astype(np.float64)
+    c, s = oracle.quantize_variant(bits, 32, oracle.AMXFP4_POT)
+    assert np.array_equal(oracle.dequantize(c, s, 32), oracle.fakequant_pot_floor(x, 32, asym=True))
+
+
+def test_power_of_two_round_scale():
+    """Exponent rounded instead of floored: the scale is 2^(round(log2 max) - 2) (numpy's log2 as the independent
+    route; a tie would need max = sqrt(2) * 2^e, which no bf16 value is), so max / scale lies in [2^1.5, 2^2.5) and
+    never reaches past 6: the clamping error the appendix attributes to the floor is gone.  Elements are rounded as
+    in every other format (checked against the pinned one-scale quantizer run with that scale's group maximum)."""
+    for mode, per_sign in ((oracle.MXFP4_POT_ROUND, False), (oracle.AMXFP4_POT_ROUND, True)):
+        bits = inputs.random_groups(36, 64, 256, "normal")
+        x = inputs.bf16_bits_to_f32(bits).astype(np.float64).reshape(64, 8, 32)
+        c, s = oracle.quantize_variant(bits, 32, mode)
+        sv = s.view(ml_dtypes.float8_e5m2).astype(np.float64)
+        pmax, nmax = np.where(x > 0, x, 0).max(-1), np.where(x < 0, -x, 0).max(-1)
+        tops = (pmax, nmax) if per_sign else (np.maximum(pmax, nmax),) * 2
+        for side, top in enumerate(tops):
+            ok = top > 0
+            assert np.array_equal(sv[..., side][ok], 2.0 ** (np.rint(np.log2(top[ok])) - 2))
+            ratio = top[ok] / sv[..., side][ok]
+            assert np.all(ratio >= 2 ** 1.5) and np.all(ratio < 2 ** 2.5)
+        assert oracle.quant_error(bits, c, s, 32)[3] == 0
+        # floor and round differ exactly where the maximum's mantissa is at least sqrt(2)
+        cf, sf = oracle.quantize_variant(bits, 32, oracle.AMXFP4_POT if per_sign else oracle.MXFP4)
+        svf = sf.view(ml_dtypes.float8_e5m2).astype(np.float64)
+        for side, top in enumerate(tops):
+            ok = top > 0
+            up = top[ok] / 2.0 ** np.floor(np.log2(top[ok])) >= np.sqrt(2.0)
+            assert np.array_equal(sv[..., side][ok] / svf[..., side][ok], np.where(up, 2.0, 1.0))
+        # element codes: a group whose scale did not move has the floor variant's codes
+        same = np.all(sv == svf, axis=-1)
+        c4, cf4 = oracle.unpack_codes(c).reshape(64, 8, 32), oracle.unpack_codes(cf).reshape(64, 8, 32)
+        assert np.array_equal(c4[same], cf4[same]) and same.any() and (~same).any()
