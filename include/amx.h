@@ -56,6 +56,13 @@ typedef enum amx_status {
 #define AMX_FMT_SYM_FP8 1   /* one E5M2 scale per group, nearest to max|x| / 6 (Section 4.2 without the split) */
 #define AMX_FMT_MXFP4 2     /* Algorithm 1: scale 2^(floor(log2 max|x|) - 2), stored as the E5M2 byte of that power
                              * of two; exponents above 15 are stored as 2^15, below -16 as a zero scale */
+/* power-of-two scale variants of the shared-scale ablation (amx_quantize_fmt only; for the FP4 GEMM follow with
+ * amx_prepare, which finds rows whose two scales agree by itself) */
+#define AMX_FMT_AMXFP4_POT 3        /* per-sign scales, each Algorithm 1's power of two ("AMXFP4, shared scale PoT"
+                                     * of the worked example in Appendix B.3) */
+#define AMX_FMT_MXFP4_POT_ROUND 4   /* one scale per group, exponent rounded instead of floored (appendix
+                                     * "Determining PoT Shared Scale: Floor vs. Round"): 2^(round(log2 max|x|) - 2) */
+#define AMX_FMT_AMXFP4_POT_ROUND 5  /* the same per sign */
 
 /* flags for amx_dequantize: output element type (default bf16) */
 #define AMX_OUT_BF16 0x0u

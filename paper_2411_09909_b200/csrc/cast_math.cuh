@@ -90,24 +90,39 @@ __device__ __forceinline__ uint32_t group_scales(uint32_t c, float& inv_p, float
     return sc;
 }
 
-// The same for the symmetric comparison formats, which store their one shared scale in both bytes
-// (FMT: AMX_FMT_AMXFP4 = 0, AMX_FMT_SYM_FP8 = 1, AMX_FMT_MXFP4 = 2):
-//   SYM_FP8  the scale of the larger side maximum, used by both sides;
-//   MXFP4    Algorithm 1: X = 2^(floor(log2 max|x|) - 2), from the exponent field E of the maximum's bf16
-//            pattern: X's E5M2 exponent field is E - 127 - 2 + 15 = E - 114; fields 0 and -1 are the
-//            subnormals 2^-15 (byte 2) and 2^-16 (byte 1), smaller ones store a zero scale, larger than 30
-//            store 2^15.
+// E5M2 byte of the power-of-two scale of Algorithm 1 for a side (or group) maximum given as a non-negative bf16
+// pattern: X = 2^(floor(log2 max) - 2), from the exponent field E of the pattern: X's E5M2 exponent field is
+// E - 127 - 2 + 15 = E - 114; fields 0 and -1 are the subnormals 2^-15 (byte 2) and 2^-16 (byte 1), smaller ones
+// store a zero scale, larger than 30 store 2^15.  ROUND: the exponent is rounded instead of floored (appendix on
+// floor vs. round), i.e. one more when max >= sqrt(2) x its power of two: (128 + m)^2 >= 2 x 128^2 for the 7
+// mantissa bits m, which is m >= 54.
+template <bool ROUND>
+__device__ __forceinline__ uint32_t pot_scale_byte(uint32_t bits) {
+    const int e5 = (int)(bits >> 7) - 114 + ((ROUND && (bits & 0x7Fu) >= 54u) ? 1 : 0);
+    return e5 > 30 ? 0x78u : e5 >= 1 ? (uint32_t)e5 << 2 : e5 == 0 ? 2u : e5 == -1 ? 1u : 0u;
+}
+
+// Whether a format stores one shared scale per group (in both bytes) or one per sign.
+__host__ __device__ constexpr bool format_is_symmetric(int fmt) { return fmt == 1 || fmt == 2 || fmt == 4; }
+
+// Scale bytes and reciprocals for the comparison formats (FMT: AMX_FMT_*):
+//   SYM_FP8 (1)          the FP8 scale of the larger side maximum, used by both sides;
+//   MXFP4 (2)            Algorithm 1's power-of-two floor scale of the group maximum;
+//   AMXFP4_POT (3)       the same per sign;
+//   MXFP4_POT_ROUND (4), AMXFP4_POT_ROUND (5)   exponent rounded instead of floored, per group / per sign.
 template <int FMT>
 __device__ __forceinline__ uint32_t group_scales_fmt(uint32_t c, float& inv_p, float& inv_n) {
     if (FMT == 0) return group_scales(c, inv_p, inv_n);
+    if (FMT == 3 || FMT == 5) {
+        const uint32_t bp = pot_scale_byte<FMT == 5>(c & 0xFFFFu), bn = pot_scale_byte<FMT == 5>(c >> 16);
+        inv_p = inv_scale_up(e5m2_to_float(bp));
+        inv_n = inv_scale_up(e5m2_to_float(bn));
+        return bp | (bn << 8);
+    }
     const uint32_t amax = max(c & 0xFFFFu, c >> 16);              // both halves are non-negative bf16 patterns
     uint32_t b;
-    if (FMT == 1) {
-        b = cvt_e5m2x2(0.0f, trunc12(__uint_as_float(amax << 16) * sixth_up())) & 0xFFu;
-    } else {
-        const int e5 = (int)(amax >> 7) - 114;
-        b = e5 > 30 ? 0x78u : e5 >= 1 ? (uint32_t)e5 << 2 : e5 == 0 ? 2u : e5 == -1 ? 1u : 0u;
-    }
+    if (FMT == 1) b = cvt_e5m2x2(0.0f, trunc12(__uint_as_float(amax << 16) * sixth_up())) & 0xFFu;
+    else b = pot_scale_byte<FMT == 4>(amax);
     inv_p = inv_n = inv_scale_up(e5m2_to_float(b));
     return b | (b << 8);
 }

@@ -336,7 +336,7 @@ extern "C" int amx_quantize(const void* x, int64_t rows, int64_t K, int64_t ld_x
 extern "C" int amx_quantize_fmt(const void* x, int64_t rows, int64_t K, int64_t ld_x, int group_size, int format,
                                 uint8_t* codes, uint8_t* scales, void* stream) {
     using namespace amx;
-    if (format != AMX_FMT_AMXFP4 && format != AMX_FMT_SYM_FP8 && format != AMX_FMT_MXFP4) return AMX_ERR_FLAGS;
+    if (format < AMX_FMT_AMXFP4 || format > AMX_FMT_AMXFP4_POT_ROUND) return AMX_ERR_FLAGS;
     if (!valid_group_size(group_size) || rows < 0 || K <= 0 || K % group_size || K % 8 || ld_x < K)
         return AMX_ERR_SHAPE;
     if (rows == 0) return AMX_OK;
@@ -345,6 +345,9 @@ extern "C" int amx_quantize_fmt(const void* x, int64_t rows, int64_t K, int64_t 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (format == AMX_FMT_SYM_FP8) return launch_rows_gs<1>(x, rows, K, ld_x, group_size, codes, scales, st);
     if (format == AMX_FMT_MXFP4) return launch_rows_gs<2>(x, rows, K, ld_x, group_size, codes, scales, st);
+    if (format == AMX_FMT_AMXFP4_POT) return launch_rows_gs<3>(x, rows, K, ld_x, group_size, codes, scales, st);
+    if (format == AMX_FMT_MXFP4_POT_ROUND) return launch_rows_gs<4>(x, rows, K, ld_x, group_size, codes, scales, st);
+    if (format == AMX_FMT_AMXFP4_POT_ROUND) return launch_rows_gs<5>(x, rows, K, ld_x, group_size, codes, scales, st);
     return launch_rows_gs<0>(x, rows, K, ld_x, group_size, codes, scales, st);
 }
 

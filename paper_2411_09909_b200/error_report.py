@@ -16,7 +16,8 @@ import torch
 from . import amx, build, inputs
 
 FORMATS = (("AMXFP4 (two FP8 scales)", amx.FMT_AMXFP4), ("symmetric, FP8 scale", amx.FMT_SYM_FP8),
-           ("MXFP4 (power-of-two floor)", amx.FMT_MXFP4))
+           ("MXFP4 (power-of-two floor)", amx.FMT_MXFP4), ("per-sign power-of-two floor", amx.FMT_AMXFP4_POT),
+           ("power-of-two round", amx.FMT_MXFP4_POT_ROUND), ("per-sign power-of-two round", amx.FMT_AMXFP4_POT_ROUND))
 TENSORS = (("activation, channel outliers (config 2, 4096 wide)", 2, 0, "a"),
            ("activation, SiLU-skewed (config 3, 14336 wide)", 3, 3, "a"),
            ("weight N(0, 0.02) (config 2, 4096 -> 4096)", 2, 1, "w"))

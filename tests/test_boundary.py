@@ -49,7 +49,7 @@ def test_host_detected_argument_errors(L):
     assert q(fake, 4, 64, 32, 32, fake, fake, None) == -2               # ld < K
     assert q(odd, 4, 64, 64, 32, fake, fake, None) == -3                # alignment
     assert q(fake, 4, 64, 68, 32, fake, fake, None) == -3               # ld % 8
-    assert L.amx_quantize_fmt(fake, 4, 64, 64, 32, 3, fake, fake, None) == -5       # unknown format
+    assert L.amx_quantize_fmt(fake, 4, 64, 64, 32, 6, fake, fake, None) == -5       # unknown format
     assert L.amx_quantize_fmt(fake, 4, 64, 64, 24, 1, fake, fake, None) == -2
     assert L.amx_quantize_prepared_fmt(fake, 4, 64, 32, 0, 7, fake, fake, fake, 1 << 20, None) == -5
     assert L.amx_quantize_t(fake, 48, 8, 8, 32, fake, fake, None) == -2  # R % gs

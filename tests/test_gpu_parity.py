@@ -280,6 +280,44 @@ def test_symmetric_formats(fmt, mode):
     assert rel_fro(amx.gemm_prepared(pa, pw_amx, 300, 520, 1056).cpu().numpy(), oracle.gemm(*qa, *wq, 32)) <= GEMM_TOL
 
 
+@pytest.mark.parametrize("fmt,mode", [(amx.FMT_AMXFP4_POT, oracle.AMXFP4_POT), (amx.FMT_MXFP4_POT_ROUND, oracle.MXFP4_POT_ROUND),
+                                      (amx.FMT_AMXFP4_POT_ROUND, oracle.AMXFP4_POT_ROUND)])
+def test_power_of_two_scale_formats(fmt, mode):
+    """Power-of-two shared scales (per-sign floor; exponent rounded, per group and per sign): codes and scales
+    bit-exact against the oracle for every group size, every bf16 value as a side maximum and as an element; the
+    GEMMs take the stored operands unchanged."""
+    for gs in (16, 32, 64, 128):
+        for kind in ("mixed", "wide"):
+            bits = inputs.random_groups(340 + gs, 96, 512, kind)
+            c, s_ = amx.quantize(dev_bf16(bits), gs, fmt=fmt)
+            oc, os_ = oracle.quantize_variant(bits, gs, mode)
+            assert np.array_equal(c.cpu().numpy(), oc) and np.array_equal(s_.cpu().numpy(), os_), (gs, kind)
+    allv = np.arange(0x7F80, dtype=np.uint16)
+    bits = np.zeros((allv.size, 32), np.uint16)
+    bits[:, 0] = allv
+    bits[:, 1] = allv[::-1] | 0x8000                        # the two sides get different maxima
+    bits[:, 2] = 0x3F80
+    c, s_ = amx.quantize(dev_bf16(bits), 32, fmt=fmt)
+    oc, os_ = oracle.quantize_variant(bits, 32, mode)
+    assert np.array_equal(c.cpu().numpy(), oc) and np.array_equal(s_.cpu().numpy(), os_)
+    bits = np.full((allv.size, 32), 0x0000, np.uint16)
+    bits[:, 0] = 0x4416                                     # 600.0 and -37.0 fix the scales
+    bits[:, 3] = 0xC214
+    bits[:, 1] = allv
+    bits[:, 2] = allv | 0x8000
+    c, s_ = amx.quantize(dev_bf16(bits), 32, fmt=fmt)
+    oc, os_ = oracle.quantize_variant(bits, 32, mode)
+    assert np.array_equal(c.cpu().numpy(), oc) and np.array_equal(s_.cpu().numpy(), os_)
+    a_bits = inputs.random_groups(351, 200, 1056, "normal")
+    w_bits = inputs.random_groups(352, 264, 1056, "normal")
+    qa, qw = oracle.quantize_variant(a_bits, 32, mode), oracle.quantize_variant(w_bits, 32, mode)
+    ref = oracle.gemm(*qa, *qw, 32)
+    ac, as_ = amx.quantize(dev_bf16(a_bits), 32, fmt=fmt)
+    wc, ws = amx.quantize(dev_bf16(w_bits), 32, fmt=fmt)
+    for flags in (amx.GEMM_SIMT, amx.GEMM_TC, amx.GEMM_FP4):
+        assert rel_fro(amx.gemm(ac, as_, wc, ws, 32, flags).cpu().numpy(), ref) <= GEMM_TOL, flags
+
+
 @pytest.mark.parametrize("M,N,K", [(1, 12288, 4096), (16, 600, 4096), (130, 300, 2048), (7, 256, 11008)])
 def test_gemm_tc_few_tiles_long_k(M, N, K):
     """A few token rows against a big weight (decode-like): the bf16-decode kernel cuts K into slices that run as
