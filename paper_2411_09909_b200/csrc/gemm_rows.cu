@@ -12,7 +12,9 @@
 // the whole 32-element group 4 * step + t of weight row g of each of its two 8-row tiles: 16 bytes of codes and
 // the group's two scales per tile, brought in by asynchronous copies into a per-warp ring in shared memory four
 // steps ahead (no registers are held by loads in flight) and decoded in registers with the group's lookup tables.
-// The matching activation values (rows g and g + 8, same group) come from shared memory in 16-byte pieces.
+// The matching activation values (rows g and g + 8, same group) are read from global memory in 16-byte pieces,
+// 512 contiguous bytes per warp and load; every warp of every CTA on an SM reads the same few hundred KB, so they
+// come from the L1 (staging them in shared memory needed a block barrier every few steps and measured slower).
 // Eight MMAs per tile and step consume four elements per lane each.  What bounds the kernel is instruction
 // issue (decode on the integer/logic pipe), not the tensor cores: the MMAs are a few percent of the instructions.
 //
@@ -39,7 +41,6 @@ constexpr int kTiles = 2;                    // 8-row weight tiles per warp
 constexpr int kCtaRows = kWarps * kTiles * 8;   // 128 weight rows per CTA
 constexpr int kStepK = 128;                  // elements of K per step: one group per lane of a quad
 constexpr int kStepBytes = kMaxRows * kStepK * 2;   // activation fragments of one step: 4 KB
-constexpr int kChunkSteps = 4;               // steps of activation fragments in shared memory at a time (16 KB)
 constexpr int kMaxSlices = 8;                // portable cluster size
 constexpr int kPartPitch = 136;              // floats per token row of the partial-product tile (bank spread)
 
@@ -153,18 +154,16 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// Shared memory of a CTA: two buffers of activation fragments (a chunk of steps each), then one ring of kDepth
-// steps per warp for the weight stream.  A ring slot holds, per 8-row tile, the 32 lanes' 16 bytes of codes and
-// 4 bytes of scales (the two groups 4 * step + 2 * (t / 2) + {0, 1}; the lane uses the half t % 2).  Every lane
+// Shared memory of a CTA: one ring of kDepth steps per warp for the weight stream.  A ring slot holds, per 8-row
+// tile, the 32 lanes' 16 bytes of codes and 4 bytes of scales (the two groups 4 * step + 2 * (t / 2) + {0, 1}; the lane uses the half t % 2).  Every lane
 // reads back only what its own copies wrote, so the ring needs no barrier, only the lane's own wait.
 constexpr int kDepth = 4;
-constexpr int kSlotCodes = kTiles * 32 * 16, kSlotBytes = kSlotCodes + kTiles * 32 * 4;   // 2560
+constexpr int kSlotCodes = kTiles * 32 * 16, kSlotBytes = kSlotCodes + kTiles * 32 * 4;
 constexpr int kRingBytes = kDepth * kSlotBytes;                                            // per warp
-constexpr int kFragBytes = kChunkSteps * kStepBytes;
-constexpr int kSmemBytes = 2 * kFragBytes + kWarps * kRingBytes;
-static_assert(kChunkSteps <= kDepth, "a chunk's fragments are committed with the group of its first step");
+constexpr int kSmemBytes = kWarps * kRingBytes;
+static_assert(kMaxRows * kPartPitch * 4 <= kWarps * kRingBytes, "the partial-product tile reuses the rings");
 
-__global__ void __launch_bounds__(kThreads, 3) gemm_rows_kernel(const uint4* __restrict__ frag,
+__global__ void __launch_bounds__(kThreads, 4) gemm_rows_kernel(const uint4* __restrict__ frag,
                                                                 const uint8_t* __restrict__ w_codes,
                                                                 const uint8_t* __restrict__ w_scales, int M, int64_t N,
                                                                 int64_t K, float* __restrict__ C, int64_t ld_c) {
@@ -187,7 +186,7 @@ __global__ void __launch_bounds__(kThreads, 3) gemm_rows_kernel(const uint4* __r
         pc[i] = w_codes + (r * groups + s_begin * 4 + t) * 16;
         ps[i] = w_scales + (r * groups + s_begin * 4 + (t & 2)) * 2;
     }
-    uint8_t* ring = smem + 2 * kFragBytes + warp * kRingBytes;
+    uint8_t* ring = smem + warp * kRingBytes;
     auto issue = [&](int step) {             // step relative to s_begin; one commit group per call
         if (step < n_total) {
             uint8_t* slot = ring + (step % kDepth) * kSlotBytes;
@@ -199,18 +198,6 @@ __global__ void __launch_bounds__(kThreads, 3) gemm_rows_kernel(const uint4* __r
         }
         cp_async_commit();
     };
-    // Activation fragments of a chunk of steps: contiguous in global memory, copied as they are into one of two
-    // buffers.  The copies are not committed on their own: they join the next group of the weight stream, which
-    // is waited for before the chunk's first step.
-    auto issue_fragments = [&](int chunk) {
-        const int first = chunk * kChunkSteps;
-        if (first >= n_total) return;
-        const int n_steps = n_total - first < kChunkSteps ? n_total - first : kChunkSteps;
-        const uint4* src = frag + (s_begin + first) * (kStepBytes / 16);
-        uint4* dst = reinterpret_cast<uint4*>(smem + (chunk & 1) * kFragBytes);
-        for (int i = threadIdx.x; i < n_steps * (kStepBytes / 16); i += kThreads) cp_async16(dst + i, src + i);
-    };
-    issue_fragments(0);
 #pragma unroll
     for (int d = 0; d < kDepth; ++d) issue(d);
 
@@ -221,20 +208,15 @@ __global__ void __launch_bounds__(kThreads, 3) gemm_rows_kernel(const uint4* __r
         for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 
     for (int step = 0; step < n_total; ++step) {
-        cp_async_wait<kDepth - 1>();                             // this step's group has landed
-        const int chunk = step / kChunkSteps, s = step % kChunkSteps;
-        if (s == 0) {
-            __syncthreads();             // the chunk's fragments are visible; the other buffer is no longer read
-            issue_fragments(chunk + 1);
-        }
-        const uint8_t* slot = ring + (step % kDepth) * kSlotBytes;
-        const uint4* a = reinterpret_cast<const uint4*>(smem + (chunk & 1) * kFragBytes + s * kStepBytes) + lane;
+        const uint4* a = frag + (s_begin + step) * (kStepBytes / 16) + lane;
         uint4 a_lo[4], a_hi[4];                                  // rows g and g + 8, elements 8j .. 8j + 7
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            a_lo[j] = a[(j * 2) * 32];
-            a_hi[j] = a[(j * 2 + 1) * 32];
+            a_lo[j] = __ldg(a + (j * 2) * 32);
+            a_hi[j] = __ldg(a + (j * 2 + 1) * 32);
         }
+        cp_async_wait<kDepth - 1>();                             // this step's group has landed
+        const uint8_t* slot = ring + (step % kDepth) * kSlotBytes;
 #pragma unroll
         for (int i = 0; i < kTiles; ++i) {
             const uint4 cw = *reinterpret_cast<const uint4*>(slot + i * 512 + lane * 16);
@@ -252,7 +234,8 @@ __global__ void __launch_bounds__(kThreads, 3) gemm_rows_kernel(const uint4* __r
     }
     cp_async_wait<0>();
 
-    // Partial products of this range of K: [16 token rows][128 weight rows] in shared memory, then every CTA of
+    // Partial products of this range of K: [16 token rows][128 weight rows] in shared memory (over the rings, which
+    // are drained), then every CTA of
     // the cluster adds its share of the outputs over all ranks, in rank order.
     __syncthreads();
     float* part = reinterpret_cast<float*>(smem);
