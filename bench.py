@@ -213,7 +213,7 @@ def time_decode(steps: int, A=None, W=None):
     if A is None:
         def to_dev(bits):
             return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
-        A = [to_dev(inputs.activation(2, li)[:16]) for li in range(len(layers))]
+        A = [to_dev(inputs.activation(2, li, M=64)) for li in range(len(layers))]
         W = [to_dev(inputs.weight(2, li)) for li in range(len(layers))]
     stream = torch.cuda.current_stream().cuda_stream
 
@@ -221,44 +221,52 @@ def time_decode(steps: int, A=None, W=None):
         if rc != 0:
             raise RuntimeError(amx.status_string(rc))
 
-    Md = 16
-    REPS = 3                      # distinct copies of the weights: 3 x 88 MB of codes and scales exceed the L2
-    dd = []
-    for li, (K, N) in enumerate(layers):
-        wc_, ws_ = amx.quantize(W[li], GS)
-        ad = A[li][:Md].contiguous()
-        need = max(L.amx_quant_gemm_workspace_bytes(Md, N, K, GS, 0), 256)
-        dd.append((ad, [(wc_.clone(), ws_.clone()) for _ in range(REPS)],
-                   torch.empty((Md, N), dtype=torch.float32, device="cuda"),
-                   torch.empty(need, dtype=torch.uint8, device="cuda")))
-        del wc_, ws_
-    decode_kernel = L.amx_gemm_kernel_for(Md, layers[0][1], layers[0][0], GS, 0)
+    REPS = 3                          # distinct copies of the weights: 3 x 88 MB of codes and scales exceed the L2
 
-    def decode_step(stream, rep=0):
+    def time_rows(Md):
+        dd = []
         for li, (K, N) in enumerate(layers):
-            ad, wq, cd, wsd = dd[li]
-            wc_, ws_ = wq[rep]
-            check(L.amx_quant_gemm(ad.data_ptr(), K, wc_.data_ptr(), ws_.data_ptr(), Md, N, K, GS, 0, cd.data_ptr(), N,
-                                   wsd.data_ptr(), wsd.numel(), stream))
+            wc_, ws_ = amx.quantize(W[li], GS)
+            ad = A[li][:Md].contiguous()
+            need = max(L.amx_quant_gemm_workspace_bytes(Md, N, K, GS, 0), 256)
+            dd.append((ad, [(wc_.clone(), ws_.clone()) for _ in range(REPS)],
+                       torch.empty((Md, N), dtype=torch.float32, device="cuda"),
+                       torch.empty(need, dtype=torch.uint8, device="cuda")))
+            del wc_, ws_
 
-    decode_step(stream)
-    torch.cuda.synchronize()
-    sd = torch.cuda.Stream()
-    sd.wait_stream(torch.cuda.current_stream())
-    gd = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(gd, stream=sd):
-        for rep in range(REPS):
-            decode_step(torch.cuda.current_stream().cuda_stream, rep)
-    for _ in range(3):
-        gd.replay()
-    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    d0.record()
-    for _ in range(steps):
-        gd.replay()
-    d1.record()
-    torch.cuda.synchronize()
-    d_us = d0.elapsed_time(d1) / (steps * REPS) * 1e3
+        def decode_step(stream, rep=0):
+            for li, (K, N) in enumerate(layers):
+                ad, wq, cd, wsd = dd[li]
+                wc_, ws_ = wq[rep]
+                check(L.amx_quant_gemm(ad.data_ptr(), K, wc_.data_ptr(), ws_.data_ptr(), Md, N, K, GS, 0, cd.data_ptr(), N,
+                                       wsd.data_ptr(), wsd.numel(), stream))
+
+        decode_step(stream)
+        torch.cuda.synchronize()
+        sd = torch.cuda.Stream()
+        sd.wait_stream(torch.cuda.current_stream())
+        gd = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gd, stream=sd):
+            for rep in range(REPS):
+                decode_step(torch.cuda.current_stream().cuda_stream, rep)
+        for _ in range(3):
+            gd.replay()
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        d0.record()
+        for _ in range(steps):
+            gd.replay()
+        d1.record()
+        torch.cuda.synchronize()
+        return d0.elapsed_time(d1) / (steps * REPS) * 1e3, dd
+
+    Md = 16
+    d_us, dd = time_rows(Md)
+    decode_kernel = L.amx_gemm_kernel_for(Md, layers[0][1], layers[0][0], GS, 0)
+    more_rows = {}
+    for rows_ in (32, 64):
+        if all(a.shape[0] >= rows_ for a in A):
+            more_rows[str(rows_)] = time_rows(rows_)[0]
     w_bytes = sum(N * K for K, N in layers) * (0.5 + 2.0 / 32.0)
     # the same with the weights prepared once for the FP4 kernel (amx_quantize_prepared + amx_gemm_prepared)
     dp = []
@@ -309,6 +317,7 @@ def time_decode(steps: int, A=None, W=None):
               "us_per_step": d_us, "weight_gb_per_s": w_bytes / (d_us * 1e-6) / 1e9,
               "frac_of_measured_copy": w_bytes / (d_us * 1e-6) / 1e9 / peaks["hbm_gbs"],
               "launches_per_step": 2 * len(layers),
+              "us_per_step_more_rows": more_rows,
               "kernel": ("weight-streaming kernel (canonical weights read once, exact bf16 decode, mma.sync; K ranges "
                          "added over a thread-block cluster)" if decode_kernel == amx.GEMM_ROWS
                          else "tcgen05 kind::f16 (bf16 decode), K cut into slices over CTAs")}

@@ -70,7 +70,7 @@ typedef enum amx_status {
 /* flags for amx_gemm / amx_quant_gemm: kernel choice.  Default (AMX_GEMM_AUTO): group size 32 runs on
  * the tensor cores - the FP4 kernel when M*N*K >= 2^27, the exact bf16-decode kernel below that and for
  * at most 64 rows of A against a large weight (decode-like shapes: that kernel then cuts K into slices over
- * CTAs and adds the partial products in slice order) - except that at most 16 rows of A with K >= 512 and
+ * CTAs and adds the partial products in slice order) - except that at most 64 rows of A with K >= 512 and
  * K % 128 == 0 go to the weight-streaming kernel (AMX_GEMM_ROWS); other group sizes run on the SIMT kernel. */
 #define AMX_GEMM_AUTO 0x0u
 #define AMX_GEMM_SIMT 0x10u  /* plain CUDA-core kernel: any shape, any supported gs */
@@ -79,7 +79,7 @@ typedef enum amx_status {
                               * than 14 binades below the largest scale of their operand row are flushed to
                               * zero (relative effect < 2^-14 per row); otherwise same result up to fp32
                               * summation order.  Needs the larger workspace amx_workspace_bytes() reports. */
-#define AMX_GEMM_ROWS 0x100u /* weight-streaming kernel for M <= 16 rows of A (decode phase): reads the canonical
+#define AMX_GEMM_ROWS 0x100u /* weight-streaming kernel for M <= 64 rows of A (decode phase): reads the canonical
                               * weight once, exact bf16 decode, K ranges added in a fixed order; gs = 32,
                               * K % 128 == 0, else AMX_ERR_SHAPE; w_scales 4-byte aligned, else AMX_ERR_ALIGN
                               * (also when AMX_GEMM_AUTO picked this kernel) */

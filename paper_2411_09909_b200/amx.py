@@ -17,7 +17,7 @@ _lib = None
 
 OUT_BF16, OUT_F32 = 0x0, 0x1
 GEMM_AUTO, GEMM_SIMT, GEMM_TC, GEMM_FP4 = 0x0, 0x10, 0x20, 0x40
-GEMM_ROWS = 0x100               # weight-streaming kernel for at most 16 rows of A
+GEMM_ROWS = 0x100               # weight-streaming kernel for at most 64 rows of A
 GEMM_CAST_IN_KERNEL = 0x80      # amx_quant_gemm only, together with GEMM_TC
 FMT_AMXFP4, FMT_SYM_FP8, FMT_MXFP4 = 0, 1, 2
 FMT_AMXFP4_POT, FMT_MXFP4_POT_ROUND, FMT_AMXFP4_POT_ROUND = 3, 4, 5   # amx_quantize_fmt only

@@ -31,10 +31,10 @@ uint32_t pick_kernel(int64_t M, int64_t N, int64_t K, int gs, uint32_t flags) {
     // more than throughput; the SIMT kernel for group sizes the tensor-core kernels do not take.
     // A few token rows against a big weight (decode-like): too few 128 x 256 tiles to fill the machine, and the
     // FP4 kernel would have to prepare the whole weight for them; the bf16-decode kernel slices K over CTAs.
-    // At most 16 token rows: the weight-streaming kernel reads the canonical weight once at memory speed.
+    // At most 64 token rows: the weight-streaming kernel reads the canonical weight once.
     if (rows && K >= 512) return AMX_GEMM_ROWS;
     const int64_t tiles = ((M + 127) / 128) * ((N + 255) / 256);
-    if (tc && M <= 64 && tiles < 148 && K >= 1024) return AMX_GEMM_TC;
+    if (tc && M <= 64 && tiles < 148 && K >= 1024) return AMX_GEMM_TC;      // K not a multiple of 128
     if (gemm_fp4_supported(M, N, K, gs) && (double)M * (double)N * (double)K >= 128.0 * 1024.0 * 1024.0) return AMX_GEMM_FP4;
     return tc ? AMX_GEMM_TC : AMX_GEMM_SIMT;
 }
@@ -42,7 +42,7 @@ uint32_t pick_kernel(int64_t M, int64_t N, int64_t K, int gs, uint32_t flags) {
 size_t kernel_workspace(uint32_t kernel, int64_t M, int64_t N, int64_t K) {
     if (kernel == AMX_GEMM_TC) return round_up(gemm_tc_workspace_bytes(M, N, K));
     if (kernel == AMX_GEMM_FP4) return round_up(gemm_fp4_workspace_bytes(M, N, K));
-    if (kernel == AMX_GEMM_ROWS) return round_up(gemm_rows_workspace_bytes(K));
+    if (kernel == AMX_GEMM_ROWS) return round_up(gemm_rows_workspace_bytes(M, K));
     return 0;
 }
 

@@ -20,10 +20,10 @@ int gemm_tc_cast(const void* x, int64_t ld_a, const uint8_t* w_codes, const uint
                  int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st);
 int gemm_tc_status(const void* workspace, cudaStream_t st);
 
-// Weight-streaming kernel for at most 16 rows of A (mma.sync on exactly decoded bf16, K ranges over a cluster):
+// Weight-streaming kernel for at most 64 rows of A (mma.sync on exactly decoded bf16, K ranges over a cluster):
 // the workspace holds the decoded rows; gemm_rows_cast casts the bf16 rows X [M, ld_x] itself.
 bool gemm_rows_supported(int64_t M, int64_t N, int64_t K, int gs);
-size_t gemm_rows_workspace_bytes(int64_t K);
+size_t gemm_rows_workspace_bytes(int64_t M, int64_t K);
 int gemm_rows(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes, const uint8_t* w_scales,
               int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st);
 int gemm_rows_cast(const void* x, int64_t ld_x, const uint8_t* w_codes, const uint8_t* w_scales, int64_t M, int64_t N,

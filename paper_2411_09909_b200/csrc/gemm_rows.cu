@@ -1,4 +1,4 @@
-// AMXFP4 x AMXFP4 -> fp32 for at most 16 rows of A against a large weight (the decode phase of inference):
+// AMXFP4 x AMXFP4 -> fp32 for at most 64 rows of A against a large weight (the decode phase of inference):
 // C[m,n] = sum_k Ahat[m,k] * What[n,k] (arXiv 2411.09909, Section 4.3), bound by streaming the 4.5-bit weight
 // from HBM once, not by arithmetic.
 //
@@ -6,8 +6,8 @@
 // The few activation rows are decoded to bf16 once by a small kernel (decoded values are exact in bf16, Eq. 1),
 // already in the order the multiply instruction's fragments want, so that the streaming kernel only copies them.
 //
-// Streaming kernel: warp-level mma.sync m16n8k16 (bf16 in, fp32 accumulate) with the 16 token rows as the M side
-// and 8 weight rows as the N side.  The contraction index may be permuted freely as long as both operands use
+// Streaming kernel: warp-level mma.sync m16n8k16 (bf16 in, fp32 accumulate) with 16 token rows as the M side
+// and 8 weight rows as the N side (up to four tiles of 16 token rows reuse the decoded weight registers).  The contraction index may be permuted freely as long as both operands use
 // the same permutation; here lane (g, t) (g = lane / 4, t = lane % 4) owns, for one step of 128 elements of K,
 // the whole 32-element group 4 * step + t of weight row g of each of its two 8-row tiles: 16 bytes of codes and
 // the group's two scales per tile, brought in by asynchronous copies into a per-warp ring in shared memory four
@@ -35,7 +35,8 @@ namespace {
 
 using namespace decode;
 
-constexpr int kMaxRows = 16;                 // token rows (the M side of one MMA)
+constexpr int kMaxRows = 16;                 // token rows of one tile (the M side of one MMA)
+constexpr int kMaxRowTiles = 4;              // up to 64 token rows
 constexpr int kWarps = 8, kThreads = kWarps * 32;
 constexpr int kTiles = 2;                    // 8-row weight tiles per warp
 constexpr int kCtaRows = kWarps * kTiles * 8;   // 128 weight rows per CTA
@@ -44,11 +45,11 @@ constexpr int kStepBytes = kMaxRows * kStepK * 2;   // activation fragments of o
 constexpr int kMaxSlices = 8;                // portable cluster size
 constexpr int kPartPitch = 136;              // floats per token row of the partial-product tile (bank spread)
 
-// Fragment order of the decoded activation, per step of 128 elements: [unit j = 0..3][half 0..1][lane 0..31]
-// pieces of 16 bytes; the piece of lane (g, t) holds elements 8j .. 8j+7 of group 4 * step + t of row 8 * half + g
-// (in the pair order and scaling of pair_order_scaled).
-__device__ __forceinline__ int64_t fragment_piece(int64_t step, int j, int half, int g, int t) {
-    return ((step * 4 + j) * 2 + half) * 32 + g * 4 + t;
+// Fragment order of the decoded activation, per step of 128 elements: [row tile mt][unit j = 0..3][half 0..1]
+// [lane 0..31] pieces of 16 bytes; the piece of lane (g, t) holds elements 8j .. 8j+7 of group 4 * step + t of row
+// 16 * mt + 8 * half + g (in the pair order and scaling of pair_order_scaled).  mts = row tiles (1, 2 or 4).
+__device__ __forceinline__ int64_t fragment_piece(int64_t step, int mts, int mt, int j, int half, int g, int t) {
+    return ((((step * mts + mt) * 4 + j) * 2 + half) * 32) + g * 4 + t;
 }
 
 // The streaming kernel decodes a word of eight weight codes into the bf16 pairs (e0, e4), (e1, e5), (e2, e6),
@@ -65,16 +66,16 @@ __device__ __forceinline__ uint4 pair_order_scaled(uint4 o) {      // o: pairs (
     return r;
 }
 
-// One thread per 32-element group of the 16-row slab: decode (DECODE) or cast then decode (CAST) and write the
+// One thread per 32-element group of the slab of 16 * mts rows: decode, or cast then decode (CAST), and write the
 // four 16-byte pieces.  Rows past M are written as zeros.
 template <bool CAST>
 __global__ void __launch_bounds__(128) rows_fragments_kernel(const uint8_t* __restrict__ codes,
                                                              const uint8_t* __restrict__ scales,
                                                              const uint16_t* __restrict__ x, int64_t ld_x, int M,
-                                                             int64_t K, uint4* __restrict__ frag) {
+                                                             int mts, int64_t K, uint4* __restrict__ frag) {
     const int64_t groups = K / 32;
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= groups * kMaxRows) return;
+    if (idx >= groups * kMaxRows * mts) return;
     const int row = (int)(idx / groups);
     const int64_t grp = idx % groups;
     uint4 c = make_uint4(0, 0, 0, 0);
@@ -101,10 +102,11 @@ __global__ void __launch_bounds__(128) rows_fragments_kernel(const uint8_t* __re
     }
     const GroupTables tb = make_tables(sc);
     const int64_t step = grp >> 2;
-    const int t = (int)(grp & 3), g = row & 7, half = row >> 3;
+    const int t = (int)(grp & 3), g = row & 7, half = (row >> 3) & 1, mt = row >> 4;
     const uint32_t w[4] = {c.x, c.y, c.z, c.w};
 #pragma unroll
-    for (int j = 0; j < 4; ++j) frag[fragment_piece(step, j, half, g, t)] = pair_order_scaled(decode_word(w[j], tb));
+    for (int j = 0; j < 4; ++j)
+        frag[fragment_piece(step, mts, mt, j, half, g, t)] = pair_order_scaled(decode_word(w[j], tb));
 }
 
 __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -161,9 +163,11 @@ constexpr int kDepth = 4;
 constexpr int kSlotCodes = kTiles * 32 * 16, kSlotBytes = kSlotCodes + kTiles * 32 * 4;
 constexpr int kRingBytes = kDepth * kSlotBytes;                                            // per warp
 constexpr int kSmemBytes = kWarps * kRingBytes;
-static_assert(kMaxRows * kPartPitch * 4 <= kWarps * kRingBytes, "the partial-product tile reuses the rings");
+static_assert(4 * kMaxRows * kPartPitch * 4 <= kWarps * kRingBytes, "the partial-product tile reuses the rings");
 
-__global__ void __launch_bounds__(kThreads, 4) gemm_rows_kernel(const uint4* __restrict__ frag,
+// MT: tiles of 16 token rows (1, 2 or 4).  The decoded weight registers of a step are used by every row tile.
+template <int MT>
+__global__ void __launch_bounds__(kThreads, MT == 1 ? 4 : 2) gemm_rows_kernel(const uint4* __restrict__ frag,
                                                                 const uint8_t* __restrict__ w_codes,
                                                                 const uint8_t* __restrict__ w_scales, int M, int64_t N,
                                                                 int64_t K, float* __restrict__ C, int64_t ld_c) {
@@ -201,15 +205,17 @@ __global__ void __launch_bounds__(kThreads, 4) gemm_rows_kernel(const uint4* __r
 #pragma unroll
     for (int d = 0; d < kDepth; ++d) issue(d);
 
-    float acc[kTiles][4];
+    float acc[MT][kTiles][4];
 #pragma unroll
-    for (int i = 0; i < kTiles; ++i)
+    for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+        for (int i = 0; i < kTiles; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[mt][i][j] = 0.f;
 
     for (int step = 0; step < n_total; ++step) {
-        const uint4* a = frag + (s_begin + step) * (kStepBytes / 16) + lane;
-        uint4 a_lo[4], a_hi[4];                                  // rows g and g + 8, elements 8j .. 8j + 7
+        const uint4* a = frag + (s_begin + step) * (MT * kStepBytes / 16) + lane;
+        uint4 a_lo[4], a_hi[4];                                  // rows g and g + 8 of a tile, elements 8j .. 8j + 7
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             a_lo[j] = __ldg(a + (j * 2) * 32);
@@ -217,6 +223,7 @@ __global__ void __launch_bounds__(kThreads, 4) gemm_rows_kernel(const uint4* __r
         }
         cp_async_wait<kDepth - 1>();                             // this step's group has landed
         const uint8_t* slot = ring + (step % kDepth) * kSlotBytes;
+        uint4 b[kTiles][4];
 #pragma unroll
         for (int i = 0; i < kTiles; ++i) {
             const uint4 cw = *reinterpret_cast<const uint4*>(slot + i * 512 + lane * 16);
@@ -224,11 +231,24 @@ __global__ void __launch_bounds__(kThreads, 4) gemm_rows_kernel(const uint4* __r
             const GroupScales gs = make_scales((t & 1) ? sw >> 16 : sw & 0xFFFFu);
             const uint32_t w[4] = {cw.x, cw.y, cw.z, cw.w};
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint4 b = decode_pairs(w[j], gs);
-                mma_bf16(acc[i], a_lo[j].x, a_hi[j].x, a_lo[j].y, a_hi[j].y, b.x, b.y);
-                mma_bf16(acc[i], a_lo[j].z, a_hi[j].z, a_lo[j].w, a_hi[j].w, b.z, b.w);
+            for (int j = 0; j < 4; ++j) b[i][j] = decode_pairs(w[j], gs);
+        }
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+            if (mt > 0) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    a_lo[j] = __ldg(a + ((mt * 4 + j) * 2) * 32);
+                    a_hi[j] = __ldg(a + ((mt * 4 + j) * 2 + 1) * 32);
+                }
             }
+#pragma unroll
+            for (int i = 0; i < kTiles; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    mma_bf16(acc[mt][i], a_lo[j].x, a_hi[j].x, a_lo[j].y, a_hi[j].y, b[i][j].x, b[i][j].y);
+                    mma_bf16(acc[mt][i], a_lo[j].z, a_hi[j].z, a_lo[j].w, a_hi[j].w, b[i][j].z, b[i][j].w);
+                }
         }
         issue(step + kDepth);                                    // refill the slot just consumed
     }
@@ -240,13 +260,15 @@ __global__ void __launch_bounds__(kThreads, 4) gemm_rows_kernel(const uint4* __r
     __syncthreads();
     float* part = reinterpret_cast<float*>(smem);
 #pragma unroll
-    for (int i = 0; i < kTiles; ++i) {
-        const int col = warp * (kTiles * 8) + i * 8 + 2 * t;
-        *reinterpret_cast<float2*>(part + g * kPartPitch + col) = make_float2(acc[i][0], acc[i][1]);
-        *reinterpret_cast<float2*>(part + (g + 8) * kPartPitch + col) = make_float2(acc[i][2], acc[i][3]);
-    }
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int i = 0; i < kTiles; ++i) {
+            const int col = warp * (kTiles * 8) + i * 8 + 2 * t;
+            *reinterpret_cast<float2*>(part + (mt * 16 + g) * kPartPitch + col) = make_float2(acc[mt][i][0], acc[mt][i][1]);
+            *reinterpret_cast<float2*>(part + (mt * 16 + g + 8) * kPartPitch + col) = make_float2(acc[mt][i][2], acc[mt][i][3]);
+        }
     cluster.sync();
-    const int per = kMaxRows * kCtaRows / slices;                // outputs this CTA adds up (a multiple of 128)
+    const int per = MT * kMaxRows * kCtaRows / slices;           // outputs this CTA adds up (a multiple of 256)
     for (int o = slice * per + threadIdx.x; o < (slice + 1) * per; o += kThreads) {
         const int m = o / kCtaRows, col = o % kCtaRows;
         float v[kMaxSlices];
@@ -262,36 +284,52 @@ __global__ void __launch_bounds__(kThreads, 4) gemm_rows_kernel(const uint4* __r
     cluster.sync();                                              // no CTA leaves while its tile is still read
 }
 
-// How many clusters of `slices` CTAs the device holds at once (asked once per cluster size; 0 if the query fails).
-int resident_clusters(int slices) {
-    static int cached[kMaxSlices + 1] = {};
-    if (cached[slices]) return cached[slices] > 0 ? cached[slices] : 0;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(1, (unsigned)slices, 1);
+using RowsKernel = void (*)(const uint4*, const uint8_t*, const uint8_t*, int, int64_t, int64_t, float*, int64_t);
+
+// Row tiles for M token rows (1, 2 or 4) and the kernel instantiation for them.
+int row_tiles(int64_t M) { return M <= kMaxRows ? 1 : M <= 2 * kMaxRows ? 2 : 4; }
+RowsKernel kernel_for_tiles(int mts) {
+    return mts == 1 ? gemm_rows_kernel<1> : mts == 2 ? gemm_rows_kernel<2> : gemm_rows_kernel<4>;
+}
+
+void cluster_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, unsigned row_blocks, int slices, cudaStream_t st) {
+    cfg = {};
+    cfg.gridDim = dim3(row_blocks, (unsigned)slices, 1);
     cfg.blockDim = dim3(kThreads, 1, 1);
     cfg.dynamicSmemBytes = kSmemBytes;
-    cudaLaunchAttribute attr[1];
+    cfg.stream = st;
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 1;
     attr[0].val.clusterDim.y = (unsigned)slices;
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+}
+
+// How many clusters of `slices` CTAs the device holds at once (asked once per kernel and cluster size; 0 if the
+// query fails).
+int resident_clusters(int mts, int slices) {
+    static int cached[kMaxRowTiles + 1][kMaxSlices + 1] = {};
+    int& c = cached[mts][slices];
+    if (c) return c > 0 ? c : 0;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    cluster_config(cfg, attr, 1, slices, nullptr);
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, gemm_rows_kernel, &cfg) != cudaSuccess || n <= 0) {
+    if (cudaOccupancyMaxActiveClusters(&n, kernel_for_tiles(mts), &cfg) != cudaSuccess || n <= 0) {
         cudaGetLastError();
         n = -1;
     }
-    cached[slices] = n;
+    c = n;
     return n > 0 ? n : 0;
 }
 
 // Ranges of K per 128 weight rows: as many as give every range at least two steps and still let all clusters
 // be resident at once (a second wave of CTAs would start its stream from an empty pipeline).
-int slices_for(int64_t N, int64_t K) {
+int slices_for(int mts, int64_t N, int64_t K) {
     const int64_t steps = K / kStepK, row_blocks = (N + kCtaRows - 1) / kCtaRows;
     int s = kMaxSlices;
-    while (s > 1 && (steps < 2 * s || row_blocks > resident_clusters(s))) s >>= 1;
+    while (s > 1 && (steps < 2 * s || row_blocks > resident_clusters(mts, s))) s >>= 1;
     return s;
 }
 
@@ -301,58 +339,55 @@ int launch_rows(const uint4* frag, const uint8_t* w_codes, const uint8_t* w_scal
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AMX_ERR_CUDA;
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(gemm_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) {
-            cudaGetLastError();
-            return AMX_ERR_CUDA;
-        }
+        for (int mts = 1; mts <= kMaxRowTiles; mts *= 2)
+            if (cudaFuncSetAttribute(kernel_for_tiles(mts), cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) !=
+                cudaSuccess) {
+                cudaGetLastError();
+                return AMX_ERR_CUDA;
+            }
         configured[dev] = true;
     }
-    const int slices = slices_for(N, K);
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)((N + kCtaRows - 1) / kCtaRows), (unsigned)slices, 1);
-    cfg.blockDim = dim3(kThreads, 1, 1);
-    cfg.dynamicSmemBytes = kSmemBytes;
-    cfg.stream = st;
+    const int mts = row_tiles(M);
+    cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 1;
-    attr[0].val.clusterDim.y = (unsigned)slices;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, gemm_rows_kernel, frag, w_codes, w_scales, (int)M, N, K, C, ld_c) != cudaSuccess) {
+    cluster_config(cfg, attr, (unsigned)((N + kCtaRows - 1) / kCtaRows), slices_for(mts, N, K), st);
+    if (cudaLaunchKernelEx(&cfg, kernel_for_tiles(mts), frag, w_codes, w_scales, (int)M, N, K, C, ld_c) != cudaSuccess) {
         cudaGetLastError();
         return AMX_ERR_CUDA;
     }
     return AMX_OK;
 }
 
+template <bool CAST>
+int launch_fragments(const uint8_t* codes, const uint8_t* scales, const uint16_t* x, int64_t ld_x, int64_t M, int64_t K,
+                     uint4* frag, cudaStream_t st) {
+    const int mts = row_tiles(M);
+    const int64_t threads = (int64_t)kMaxRows * mts * (K / 32);
+    rows_fragments_kernel<CAST><<<(unsigned)((threads + 127) / 128), 128, 0, st>>>(codes, scales, x, ld_x, (int)M, mts, K, frag);
+    return launch_status();
+}
+
 }  // namespace
 
 bool gemm_rows_supported(int64_t M, int64_t N, int64_t K, int gs) {
-    return gs == 32 && M >= 1 && M <= kMaxRows && N >= 1 && K >= kStepK && K % kStepK == 0 &&
+    return gs == 32 && M >= 1 && M <= kMaxRows * kMaxRowTiles && N >= 1 && K >= kStepK && K % kStepK == 0 &&
            (N + kCtaRows - 1) / kCtaRows <= 0x7FFFFFFF;
 }
 
-size_t gemm_rows_workspace_bytes(int64_t K) { return (size_t)kMaxRows * (size_t)K * 2; }
+size_t gemm_rows_workspace_bytes(int64_t M, int64_t K) { return (size_t)kMaxRows * row_tiles(M) * (size_t)K * 2; }
 
 int gemm_rows(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes, const uint8_t* w_scales,
               int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {
     uint4* frag = static_cast<uint4*>(workspace);
-    const int64_t threads = kMaxRows * (K / 32);
-    rows_fragments_kernel<false><<<(unsigned)((threads + 127) / 128), 128, 0, st>>>(a_codes, a_scales, nullptr, 0, (int)M,
-                                                                                   K, frag);
-    if (launch_status() != AMX_OK) return AMX_ERR_CUDA;
+    if (launch_fragments<false>(a_codes, a_scales, nullptr, 0, M, K, frag, st) != AMX_OK) return AMX_ERR_CUDA;
     return launch_rows(frag, w_codes, w_scales, M, N, K, C, ld_c, st);
 }
 
 int gemm_rows_cast(const void* x, int64_t ld_x, const uint8_t* w_codes, const uint8_t* w_scales, int64_t M, int64_t N,
                    int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {
     uint4* frag = static_cast<uint4*>(workspace);
-    const int64_t threads = kMaxRows * (K / 32);
-    rows_fragments_kernel<true><<<(unsigned)((threads + 127) / 128), 128, 0, st>>>(
-        nullptr, nullptr, static_cast<const uint16_t*>(x), ld_x, (int)M, K, frag);
-    if (launch_status() != AMX_OK) return AMX_ERR_CUDA;
+    if (launch_fragments<true>(nullptr, nullptr, static_cast<const uint16_t*>(x), ld_x, M, K, frag, st) != AMX_OK)
+        return AMX_ERR_CUDA;
     return launch_rows(frag, w_codes, w_scales, M, N, K, C, ld_c, st);
 }
 

@@ -361,9 +361,11 @@ def test_gemm_prepared_few_tiles_long_k(M, N, K):
 
 @pytest.mark.parametrize("M,N,K,kind", [(16, 4096, 4096, "normal"), (1, 12288, 4096, "normal"), (5, 600, 1024, "wide"),
                                         (16, 8, 128, "mixed"), (3, 130, 256, "normal"), (7, 256, 11008, "normal"),
-                                        (16, 1030, 11264, "mixed"), (9, 129, 640, "wide")])
+                                        (16, 1030, 11264, "mixed"), (9, 129, 640, "wide"), (17, 300, 1024, "normal"),
+                                        (32, 4096, 4096, "normal"), (33, 200, 2304, "mixed"), (64, 1030, 11008, "normal"),
+                                        (50, 129, 640, "wide")])
 def test_gemm_rows_weight_streaming(M, N, K, kind):
-    """At most 16 token rows against a canonical weight (decode phase): the weight-streaming kernel decodes both
+    """At most 64 token rows against a canonical weight (decode phase): the weight-streaming kernel decodes both
     operands exactly, cuts K into ranges over a cluster and adds them in rank order: close to the fp64 oracle,
     run-to-run identical, padded output untouched; AUTO picks it, and amx_quant_gemm (cast of the rows fused with
     their decode) gives the same bits."""
@@ -390,7 +392,8 @@ def test_gemm_rows_weight_streaming(M, N, K, kind):
     assert torch.equal(fused, got.contiguous())
 
 
-def test_gemm_rows_exact_on_small_integers():
+@pytest.mark.parametrize("rows", [13, 29, 61])
+def test_gemm_rows_exact_on_small_integers(rows):
     """Integer-valued operands: every product and partial sum is exact in fp32, so any summation order gives the
     integer result - an independent check of the fragment order and the K ranges."""
     rng = np.random.default_rng(11)
@@ -399,7 +402,7 @@ def test_gemm_rows_exact_on_small_integers():
         t = grid[rng.integers(0, 6, size=(r, k))] * rng.choice([-1.0, 1.0], size=(r, k)).astype(np.float32)
         t[:, ::32], t[:, 1::32] = 6.0, -6.0
         return t
-    a, w = ints(13, 2304), ints(300, 2304)
+    a, w = ints(rows, 2304), ints(300, 2304)
     qa, qw = oracle.quantize(inputs.f32_to_bf16_bits(a), 32), oracle.quantize(inputs.f32_to_bf16_bits(w), 32)
     got = amx.gemm(*(torch.from_numpy(t).cuda() for t in (*qa, *qw)), 32, amx.GEMM_ROWS).cpu().numpy()
     assert np.array_equal(got, (a.astype(np.int64) @ w.astype(np.int64).T).astype(np.float32))
