@@ -60,6 +60,9 @@ def test_host_detected_argument_errors(L):
     assert g(fake, fake, fake, fake, 4, 4, 64, 32, 0x200, fake, 4, None, 0, None) == -5
     assert g(fake, fake, fake, fake, 4, 8, 64, 32, 0, fake, 4, None, 0, None) == -2     # ld_c < N
     assert g(None, fake, fake, fake, 4, 4, 64, 32, 0x10, fake, 4, None, 0, None) == -1
+    assert g(fake, fake, fake, fake, 4, 4, 64, 32, 0x100, fake, 4, None, 0, None) == -2     # streaming kernel: K % 128
+    assert g(fake, fake, fake, fake, 65, 4, 512, 32, 0x100, fake, 4, None, 0, None) == -2   # and at most 64 rows
+    assert g(fake, fake, fake, ctypes.c_void_p(0x1002), 4, 4, 512, 32, 0x100, fake, 4, fake, 1 << 20, None) == -3
     assert g(fake, fake, fake, fake, 0, 4, 64, 32, 0x10, fake, 4, None, 0, None) == 0   # empty
     assert L.amx_quant_gemm(fake, 64, fake, fake, 4, 4, 64, 32, 0x10, fake, 4, None, 0, None) == -4
     assert L.amx_quant_gemm(fake, 64, fake, fake, 4, 4, 64, 32, 0x80, fake, 4, fake, 4096, None) == -5   # cast-in-kernel
