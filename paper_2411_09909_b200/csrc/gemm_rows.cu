@@ -3,15 +3,16 @@
 // from HBM once, not by arithmetic.
 //
 // The weight is read in its canonical layout (codes [N, K/2], scales [N, K/32, 2]); nothing is prepared ahead.
-// The few activation rows are decoded to bf16 once by a small kernel (decoded values are exact in bf16, Eq. 1),
-// already in the order the multiply instruction's fragments want, so that the streaming kernel only copies them.
+// The few activation rows are cast and decoded to bf16 once by a small kernel (decoded values are exact in bf16,
+// Eq. 1), already in the order the multiply instruction's fragments want.
 //
-// Streaming kernel: warp-level mma.sync m16n8k16 (bf16 in, fp32 accumulate) with 16 token rows as the M side
-// and 8 weight rows as the N side (up to four tiles of 16 token rows reuse the decoded weight registers).  The contraction index may be permuted freely as long as both operands use
-// the same permutation; here lane (g, t) (g = lane / 4, t = lane % 4) owns, for one step of 128 elements of K,
-// the whole 32-element group 4 * step + t of weight row g of each of its two 8-row tiles: 16 bytes of codes and
-// the group's two scales per tile, brought in by asynchronous copies into a per-warp ring in shared memory four
-// steps ahead (no registers are held by loads in flight) and decoded in registers with the group's lookup tables.
+// Streaming kernel: warp-level mma.sync m16n8k16 (bf16 in, fp32 accumulate) with 16 token rows as the M side and
+// 8 weight rows as the N side; up to four tiles of 16 token rows reuse the decoded weight registers of a step.
+// The contraction index may be permuted freely as long as both operands use the same permutation; here lane
+// (g, t) (g = lane / 4, t = lane % 4) owns, for one step of 128 elements of K, the whole 32-element group
+// 4 * step + t of weight row g of each of its two 8-row tiles: 16 bytes of codes and the group's two scales per
+// tile, brought in by asynchronous copies into a per-warp ring in shared memory four steps ahead (no registers
+// are held by loads in flight) and decoded in registers with packed bf16 multiplies (decode_pairs below).
 // The matching activation values (rows g and g + 8, same group) are read from global memory in 16-byte pieces,
 // 512 contiguous bytes per warp and load; every warp of every CTA on an SM reads the same few hundred KB, so they
 // come from the L1 (staging them in shared memory needed a block barrier every few steps and measured slower).
@@ -157,11 +158,12 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // Shared memory of a CTA: one ring of kDepth steps per warp for the weight stream.  A ring slot holds, per 8-row
-// tile, the 32 lanes' 16 bytes of codes and 4 bytes of scales (the two groups 4 * step + 2 * (t / 2) + {0, 1}; the lane uses the half t % 2).  Every lane
-// reads back only what its own copies wrote, so the ring needs no barrier, only the lane's own wait.
+// tile, the 32 lanes' 16 bytes of codes and 4 bytes of scales (the two groups 4 * step + 2 * (t / 2) + {0, 1}; the
+// lane uses the half t % 2).  Every lane reads back only what its own copies wrote, so the ring needs no barrier,
+// only the lane's own wait.
 constexpr int kDepth = 4;
 constexpr int kSlotCodes = kTiles * 32 * 16, kSlotBytes = kSlotCodes + kTiles * 32 * 4;
-constexpr int kRingBytes = kDepth * kSlotBytes;                                            // per warp
+constexpr int kRingBytes = kDepth * kSlotBytes;   // per warp
 constexpr int kSmemBytes = kWarps * kRingBytes;
 static_assert(4 * kMaxRows * kPartPitch * 4 <= kWarps * kRingBytes, "the partial-product tile reuses the rings");
 
