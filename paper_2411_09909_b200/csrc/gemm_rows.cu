@@ -67,8 +67,10 @@ __device__ __forceinline__ uint4 pair_order_scaled(uint4 o) {      // o: pairs (
     return r;
 }
 
-// One thread per 32-element group of the slab of 16 * mts rows: decode, or cast then decode (CAST), and write the
-// four 16-byte pieces.  Rows past M are written as zeros.
+// One thread per 8 elements of the slab of 16 * mts rows (four adjacent lanes share a 32-element group and
+// exchange their side maxima with two shuffles): decode, or cast then decode (CAST), and write one 16-byte piece.
+// Rows past M are written as zeros.  The kernel is a few thousand threads of pure latency, so the work of a group
+// is spread over lanes instead of being one long dependent chain.
 template <bool CAST>
 __global__ void __launch_bounds__(128) rows_fragments_kernel(const uint8_t* __restrict__ codes,
                                                              const uint8_t* __restrict__ scales,
@@ -76,38 +78,33 @@ __global__ void __launch_bounds__(128) rows_fragments_kernel(const uint8_t* __re
                                                              int mts, int64_t K, uint4* __restrict__ frag) {
     const int64_t groups = K / 32;
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= groups * kMaxRows * mts) return;
-    const int row = (int)(idx / groups);
-    const int64_t grp = idx % groups;
-    uint4 c = make_uint4(0, 0, 0, 0);
-    uint32_t sc = 0;
-    if (row < M) {
-        if (CAST) {
-            const uint4* p = reinterpret_cast<const uint4*>(x + row * ld_x + grp * 32);
-            uint32_t w[16];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint4 q = __ldg(p + j);
-                w[4 * j] = q.x; w[4 * j + 1] = q.y; w[4 * j + 2] = q.z; w[4 * j + 3] = q.w;
-            }
-            float inv_p, inv_n;
-            sc = cast::group_scales(cast::side_maxima<16>(w), inv_p, inv_n);
-            c.x = cast::encode8(w, inv_p, inv_n);
-            c.y = cast::encode8(w + 4, inv_p, inv_n);
-            c.z = cast::encode8(w + 8, inv_p, inv_n);
-            c.w = cast::encode8(w + 12, inv_p, inv_n);
-        } else {
-            c = __ldg(reinterpret_cast<const uint4*>(codes + (row * groups + grp) * 16));
-            sc = __ldg(reinterpret_cast<const unsigned short*>(scales + (row * groups + grp) * 2));
+    const bool live = idx < groups * 4 * kMaxRows * mts;           // whole groups: the four lanes agree
+    const int j = (int)(idx & 3);
+    const int64_t gidx = idx >> 2;
+    const int row = live ? (int)(gidx / groups) : M;
+    const int64_t grp = gidx % groups;
+    uint32_t word = 0, sc = 0;
+    if (CAST) {
+        uint32_t w[4] = {0, 0, 0, 0};
+        if (row < M) {
+            const uint4 q = __ldg(reinterpret_cast<const uint4*>(x + row * ld_x + grp * 32) + j);
+            w[0] = q.x; w[1] = q.y; w[2] = q.z; w[3] = q.w;
         }
+        uint32_t c = cast::side_maxima<4>(w);
+        c = __vmaxs2(c, __shfl_xor_sync(0xFFFFFFFFu, c, 1));
+        c = __vmaxs2(c, __shfl_xor_sync(0xFFFFFFFFu, c, 2));
+        float inv_p, inv_n;
+        sc = cast::group_scales(c, inv_p, inv_n);
+        word = cast::encode8(w, inv_p, inv_n);
+    } else if (row < M) {
+        word = __ldg(reinterpret_cast<const uint32_t*>(codes + (row * groups + grp) * 16) + j);
+        sc = __ldg(reinterpret_cast<const unsigned short*>(scales + (row * groups + grp) * 2));
     }
+    if (!live) return;
     const GroupTables tb = make_tables(sc);
     const int64_t step = grp >> 2;
     const int t = (int)(grp & 3), g = row & 7, half = (row >> 3) & 1, mt = row >> 4;
-    const uint32_t w[4] = {c.x, c.y, c.z, c.w};
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-        frag[fragment_piece(step, mts, mt, j, half, g, t)] = pair_order_scaled(decode_word(w[j], tb));
+    frag[fragment_piece(step, mts, mt, j, half, g, t)] = pair_order_scaled(decode_word(word, tb));
 }
 
 __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -364,7 +361,7 @@ template <bool CAST>
 int launch_fragments(const uint8_t* codes, const uint8_t* scales, const uint16_t* x, int64_t ld_x, int64_t M, int64_t K,
                      uint4* frag, cudaStream_t st) {
     const int mts = row_tiles(M);
-    const int64_t threads = (int64_t)kMaxRows * mts * (K / 32);
+    const int64_t threads = (int64_t)kMaxRows * mts * (K / 32) * 4;
     rows_fragments_kernel<CAST><<<(unsigned)((threads + 127) / 128), 128, 0, st>>>(codes, scales, x, ld_x, (int)M, mts, K, frag);
     return launch_status();
 }
