@@ -61,5 +61,45 @@ __device__ __forceinline__ uint4 decode_word(uint32_t w, const GroupTables& t) {
     return o;
 }
 
+// Decode by packed multiplies, for kernels that the integer/logic pipe bounds: the multiplication by the scale
+// is a packed bf16 multiply (FMA pipe) instead of table look-ups, at the price of a fixed permutation of the eight
+// elements of a word (harmless for a contraction whose two operands are decoded the same way) and of a factor
+// 2^-63 on every value (exact; the other operand carries 2^+63):
+//   - a 3-bit E2M1 code placed at bits 8..6 of a bf16 reads as (its value) x 2^-126: codes 0 and 1 are the bf16
+//     subnormals 0 and 2^-127, the others have exponent field 1..3 and the code's mantissa bit;
+//   - one shift and one mask put the codes of elements q and q + 4 of a word there (pair q);
+//   - the element's scale (positive or negative side, the sign folded into the latter) is chosen with a mask that
+//     a byte permute in sign-replicating mode builds from the two sign bits;
+//   - scales are held as bf16 pairs times 2^63 (2^126 would overflow); decode_pairs_up multiplies once more,
+//     by 2^126, for the operand that carries the other 2^63.
+struct GroupScales {
+    uint32_t pos, neg;     // {s_p, s_p} x 2^63 and {-s_n, -s_n} x 2^63 as bf16 pairs
+};
+__device__ __forceinline__ GroupScales make_scales(uint32_t sc) {
+    const float two63 = 9223372036854775808.f;
+    const uint32_t p = __float_as_uint(e5m2_to_float(sc & 0xFFu) * two63);
+    const uint32_t n = __float_as_uint(e5m2_to_float((sc >> 8) & 0xFFu) * -two63);
+    return {prmt(p, p, 0x3232), prmt(n, n, 0x3232)};
+}
+__device__ __forceinline__ uint4 decode_pairs(uint32_t w, const GroupScales& gs) {
+    const uint32_t kMag = 0x01C001C0u, ws = w << 4;
+    const uint32_t m0 = prmt(ws, ws, 0xAA88), m1 = prmt(w, w, 0xAA88);     // 0xFFFF where the element is negative
+    const uint32_t m2 = prmt(ws, ws, 0xBB99), m3 = prmt(w, w, 0xBB99);
+    uint4 o;
+    o.x = mul_bf16x2((w << 6) & kMag, (gs.pos & ~m0) | (gs.neg & m0));
+    o.y = mul_bf16x2((w << 2) & kMag, (gs.pos & ~m1) | (gs.neg & m1));
+    o.z = mul_bf16x2((w >> 2) & kMag, (gs.pos & ~m2) | (gs.neg & m2));
+    o.w = mul_bf16x2((w >> 6) & kMag, (gs.pos & ~m3) | (gs.neg & m3));
+    return o;
+}
+// The same pairs times 2^+63 (true value x 2^63): the other operand of a product with decode_pairs.
+__device__ __forceinline__ uint4 decode_pairs_up(uint32_t w, const GroupScales& gs) {
+    const uint32_t two126 = 0x7E807E80u;
+    uint4 o = decode_pairs(w, gs);
+    o.x = mul_bf16x2(o.x, two126); o.y = mul_bf16x2(o.y, two126);
+    o.z = mul_bf16x2(o.z, two126); o.w = mul_bf16x2(o.w, two126);
+    return o;
+}
+
 }  // namespace decode
 }  // namespace amx

@@ -54,7 +54,7 @@ __device__ __forceinline__ int64_t fragment_piece(int64_t step, int mts, int mt,
 }
 
 // The streaming kernel decodes a word of eight weight codes into the bf16 pairs (e0, e4), (e1, e5), (e2, e6),
-// (e3, e7), each value 2^-63 times the true one (see decode_pairs); the activation pieces are stored in the same
+// (e3, e7), each value 2^-63 times the true one (decode_pairs in decode_math.cuh); the activation pieces are stored in the same
 // pair order and multiplied by 2^63, so that every product is the true one.  Both scalings are exact: a decoded
 // value times 2^+-63 stays far inside the bf16 range.
 __device__ __forceinline__ uint4 pair_order_scaled(uint4 o) {      // o: pairs (e0,e1), (e2,e3), (e4,e5), (e6,e7)
@@ -112,35 +112,6 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-// Decode for the weight stream.  The integer/logic pipe is what bounds this kernel, so the multiplication by
-// the scale is a packed bf16 multiply (FMA pipe) instead of table look-ups:
-//   - a 3-bit E2M1 code placed at bits 8..6 of a bf16 reads as (its value) x 2^-126: codes 0 and 1 are the bf16
-//     subnormals 0 and 2^-127, the others have exponent field 1..3 and the code's mantissa bit;
-//   - one shift and one mask put the codes of elements q and q + 4 of a word there (pair q);
-//   - the element's scale (positive or negative side, the sign folded into the latter) is chosen with a mask that
-//     a byte permute in sign-replicating mode builds from the two sign bits;
-//   - scales are held as bf16 pairs times 2^63 (2^126 would overflow), the activation carries the other 2^63.
-struct GroupScales {
-    uint32_t pos, neg;     // {s_p, s_p} x 2^63 and {-s_n, -s_n} x 2^63 as bf16 pairs
-};
-__device__ __forceinline__ GroupScales make_scales(uint32_t sc) {
-    const float two63 = 9223372036854775808.f;
-    const uint32_t p = __float_as_uint(e5m2_to_float(sc & 0xFFu) * two63);
-    const uint32_t n = __float_as_uint(e5m2_to_float((sc >> 8) & 0xFFu) * -two63);
-    return {prmt(p, p, 0x3232), prmt(n, n, 0x3232)};
-}
-__device__ __forceinline__ uint4 decode_pairs(uint32_t w, const GroupScales& gs) {
-    const uint32_t kMag = 0x01C001C0u, ws = w << 4;
-    const uint32_t m0 = prmt(ws, ws, 0xAA88), m1 = prmt(w, w, 0xAA88);     // 0xFFFF where the element is negative
-    const uint32_t m2 = prmt(ws, ws, 0xBB99), m3 = prmt(w, w, 0xBB99);
-    uint4 o;
-    o.x = mul_bf16x2((w << 6) & kMag, (gs.pos & ~m0) | (gs.neg & m0));
-    o.y = mul_bf16x2((w << 2) & kMag, (gs.pos & ~m1) | (gs.neg & m1));
-    o.z = mul_bf16x2((w >> 2) & kMag, (gs.pos & ~m2) | (gs.neg & m2));
-    o.w = mul_bf16x2((w >> 6) & kMag, (gs.pos & ~m3) | (gs.neg & m3));
-    return o;
 }
 
 // Asynchronous copy of 16 or 4 bytes from global to shared memory (no registers held while in flight).

@@ -15,10 +15,11 @@
 // Two shared-memory stages (48 KB each) cycle through full/empty mbarriers; two CTAs share an SM
 // so that one CTA's epilogue overlaps the other's main loop.
 //
-// Decode: per 32-element group the 2 x 8 possible values (magnitude x side scale) are computed
-// once with packed bf16 multiplies and held as byte-plane lookup tables in registers; elements
-// are then looked up four at a time with byte permutes and the side is chosen with a mask built
-// from the sign bits.
+// Decode (decode_math.cuh): a 3-bit E2M1 code placed at bits 8..6 of a bf16 is the value x 2^-126, so a shift
+// and a mask per element pair, the side's scale chosen by a mask built from the sign bits, and one packed bf16
+// multiply give the decoded pair; the two tiles carry 2^+63 and 2^-63 (exact), and both get the same
+// permutation of a word's eight elements, which a contraction does not see.  (Lookup tables by byte permutes,
+// the earlier form, kept all of this on the integer/logic pipe, which bounds the kernel.)
 //
 // Every wait is bounded: when a limit expires the CTA records AMX_ERR_TIMEOUT in the status word,
 // all roles leave their loops, tensor memory is released and the kernel returns.
@@ -174,12 +175,15 @@ gemm_tc_kernel(const uint8_t* __restrict__ a_codes, const uint8_t* __restrict__ 
                         *reinterpret_cast<uint4*>(dst + (((half * 4 + j) ^ (row & 7)) << 4)) = make_uint4(0, 0, 0, 0);
                     continue;
                 }
-                const GroupTables t = make_tables(cur[i].scales);
+                // packed-multiply decode: both tiles get the same permutation of a word's eight elements, the A
+                // tile holds values x 2^63 and the B tile values x 2^-63 (exact), so every product is the true one
+                const GroupScales gs = make_scales(cur[i].scales);
                 const uint32_t w[4] = {cur[i].codes.x, cur[i].codes.y, cur[i].codes.z, cur[i].codes.w};
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int chunk = half * 4 + j;                // 16-byte chunk inside the 128-byte row
-                    *reinterpret_cast<uint4*>(dst + ((chunk ^ (row & 7)) << 4)) = decode_word(w[j], t);
+                    *reinterpret_cast<uint4*>(dst + ((chunk ^ (row & 7)) << 4)) =
+                        i ? decode_pairs(w[j], gs) : decode_pairs_up(w[j], gs);
                 }
             }
             fence_proxy_async();          // make the generic-proxy stores visible to the tensor core
