@@ -3,10 +3,11 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-One step = one pass over the LLaMA-7B-shaped prefill linears (M = 2048 tokens; 4096->12288,
-4096->4096, 4096->11008, 11008->4096): for every layer the bf16 activation and the bf16 weight
-are cast to AMXFP4 and multiplied with fp32 accumulation.  Inputs are seeded synthetic tensors
-(channel outliers, per-channel offsets) resident in HBM.  Prints one JSON line.
+One step = one pass over the 70B-shaped long-context prefill linears (M = 16384 tokens; 8192->10240,
+8192->28672, 28672->8192 - the largest of the linear-layer workloads that fits one GPU): for every layer
+the bf16 activation and the bf16 weight are cast to AMXFP4 and multiplied with fp32 accumulation.
+Inputs are seeded synthetic tensors (channel outliers) resident in HBM.  Prints one JSON line.
+--config 2 / 3 time the smaller linear workloads the same way.
 
 With N > 1 (launched by torch.distributed.run) every rank runs the same token batch shape on its
 own GPU (token-row sharding of a larger batch: no data-path collective), and the value is the
@@ -27,7 +28,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-CONFIG = 2          # the workload the metric is quoted on; --config 3 / 4 time the larger ones (not bench lines)
+CONFIG = 4          # the largest single-GPU linear workload; --config 2 / 3 time the smaller ones
 WORKLOADS = {2: "config 2: LLaMA-7B-shaped prefill linears, M=2048, 4 layers",
              3: "config 3: LLaMA-3-8B-shaped prefill linears, M=8192, 4 layers (SiLU-skewed activations)",
              4: "config 4: 70B-scale prefill linears, M=16384, 3 layers"}
@@ -36,9 +37,9 @@ NOMINAL_FP4_TFLOPS = 9000.0      # NVIDIA's dense FP4 figure for one B200 (HGX B
 NOMINAL_HBM_GBS = 8000.0
 BYTES_PER_ELEM = 2.0 + 0.5 + 2.0 / 32.0   # bf16 read + 4-bit code + two scale bytes per 32
 MOVED_BYTES_PER_ELEM = BYTES_PER_ELEM + 1.0 + 4.0 / 32.0   # + two sign planes + four scale-factor bytes per 32
-# DRAM bytes (read + write) per GEMM launch, mean over the four layer shapes, from the ncu capture summarised
-# in profiles/; None until a capture of the current kernel exists.
-GEMM_DRAM_TRAFFIC_PER_LAUNCH = {"auto": 89.6e6, "fp4": 89.6e6}
+# DRAM bytes (read + write) per GEMM launch of the FP4 kernel, mean over the layers of a config, from the ncu
+# captures summarised in profiles/ (None: no capture of the current kernel on that config).
+GEMM_DRAM_TRAFFIC_PER_LAUNCH = {2: None, 3: None, 4: None}
 
 
 def measured_peaks():
@@ -158,7 +159,7 @@ def run_reference(args):
         "impl": "reference", "metric": "AMXFP4 quant+GEMM TFLOPS", "value": val, "unit": "TFLOP/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": secs * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "config 2: LLaMA-7B-shaped prefill linears, M=2048 (bounded row sample per step)"},
+        "config": {"workload": WORKLOADS[CONFIG] + " (bounded sample per step: 256 token rows of layer 0)"},
         "cpu_baseline": base,
         "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -209,7 +210,7 @@ def time_decode(steps: int, A=None, W=None):
     from paper_2411_09909_b200 import amx, inputs
     L = amx.lib()
     peaks = measured_peaks()
-    _, layers = layer_shapes()
+    layers = inputs.LINEAR_CONFIGS[2]["layers"]
     if A is None:
         def to_dev(bits):
             return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
@@ -238,8 +239,8 @@ def time_decode(steps: int, A=None, W=None):
             for li, (K, N) in enumerate(layers):
                 ad, wq, cd, wsd = dd[li]
                 wc_, ws_ = wq[rep]
-                check(L.amx_quant_gemm(ad.data_ptr(), K, wc_.data_ptr(), ws_.data_ptr(), Md, N, K, GS, 0, cd.data_ptr(), N,
-                                       wsd.data_ptr(), wsd.numel(), stream))
+                check(L.amx_quant_gemm(ad.data_ptr(), K, wc_.data_ptr(), ws_.data_ptr(), None, 0, Md, N, K, GS, 0,
+                                       cd.data_ptr(), N, wsd.data_ptr(), wsd.numel(), stream))
 
         decode_step(stream)
         torch.cuda.synchronize()
@@ -345,6 +346,7 @@ def run_ours(args):
     layers = [layers[i] for i in keep]
     flops_step = sum(2.0 * M * N * K for K, N in layers)
     elems_step = sum(M * K + N * K for K, N in layers)
+    use_graph = args.graph or (CONFIG == 2 and not args.no_graph)
 
     def to_dev(bits):
         return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
@@ -379,85 +381,78 @@ def run_ours(args):
         if rc != 0:
             raise RuntimeError(amx.status_string(rc))
 
-    ev_q, ev_g = [], []
-
-    def step(record: bool, stream=stream):
-        for li, (K, N) in enumerate(layers):
-            b = bufs[li]
-            if record:
-                e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
-                e0.record()
-            if fused_prepare:
-                # FP4 kernel: the cast writes the GEMM-ready operand (sign planes, scale factors) directly
-                check(L.amx_quantize_prepared(A[li].data_ptr(), M, K, GS, 0, b["ac"].data_ptr(), b["as"].data_ptr(),
-                                              b["pa"].data_ptr(), b["pa"].numel(), stream))
-                check(L.amx_quantize_prepared(W[li].data_ptr(), N, K, GS, 1, b["wc"].data_ptr(), b["ws"].data_ptr(),
-                                              b["pw"].data_ptr(), b["pw"].numel(), stream))
-                if record:
-                    e1.record()
-                check(L.amx_gemm_prepared(b["pa"].data_ptr(), b["pw"].data_ptr(), M, N, K, GS, b["c"].data_ptr(), N,
-                                          b["work"].data_ptr(), b["work"].numel(), stream))
-            else:
-                check(L.amx_quantize(A[li].data_ptr(), M, K, K, GS, b["ac"].data_ptr(), b["as"].data_ptr(), stream))
-                check(L.amx_quantize(W[li].data_ptr(), N, K, K, GS, b["wc"].data_ptr(), b["ws"].data_ptr(), stream))
-                if record:
-                    e1.record()
-                check(L.amx_gemm(b["ac"].data_ptr(), b["as"].data_ptr(), b["wc"].data_ptr(), b["ws"].data_ptr(),
-                                 M, N, K, GS, gemm_flag, b["c"].data_ptr(), N, b["work"].data_ptr(), b["work"].numel(),
-                                 stream))
-            if record:
-                e2.record()
-                ev_q.append((e0, e1))
-                ev_g.append((e1, e2))
-
-    # The same step with the weight casts on a second stream: they depend on nothing that the step computes, so
-    # they run ahead and share the SMs with the GEMMs of earlier layers (the cast is HBM-bound, the GEMM is
-    # not).  Activation casts stay in order on the main stream, directly before the GEMM that consumes them.
-    def step_overlapped(main, side):
-        side.wait_stream(main)
-        ready = []
-        for li, (K, N) in enumerate(layers):
-            b = bufs[li]
-            check(L.amx_quantize_prepared(W[li].data_ptr(), N, K, GS, 1, b["wc"].data_ptr(), b["ws"].data_ptr(),
-                                          b["pw"].data_ptr(), b["pw"].numel(), side.cuda_stream))
-            ev = torch.cuda.Event()
-            ev.record(side)
-            ready.append(ev)
-        for li, (K, N) in enumerate(layers):
-            b = bufs[li]
+    def cast_a(li, st):
+        K, N = layers[li]
+        b = bufs[li]
+        if fused_prepare:   # the cast writes the FP4 kernel's operand (sign planes, scale factors) in the same pass
             check(L.amx_quantize_prepared(A[li].data_ptr(), M, K, GS, 0, b["ac"].data_ptr(), b["as"].data_ptr(),
-                                          b["pa"].data_ptr(), b["pa"].numel(), main.cuda_stream))
-            main.wait_event(ready[li])
-            check(L.amx_gemm_prepared(b["pa"].data_ptr(), b["pw"].data_ptr(), M, N, K, GS, b["c"].data_ptr(), N,
-                                      b["work"].data_ptr(), b["work"].numel(), main.cuda_stream))
-        main.wait_stream(side)
-
-    # "pair": within a layer the cast of the activation and the cast of the weight run side by side (two streams):
-    # they are independent inputs of the same GEMM in any model, and the small activation cast fills the tail of
-    # the weight cast's last wave.  Layers stay in order.
-    def step_paired(main, side):
-        for li, (K, N) in enumerate(layers):
-            b = bufs[li]
-            side.wait_stream(main)
-            check(L.amx_quantize_prepared(A[li].data_ptr(), M, K, GS, 0, b["ac"].data_ptr(), b["as"].data_ptr(),
-                                          b["pa"].data_ptr(), b["pa"].numel(), side.cuda_stream))
-            check(L.amx_quantize_prepared(W[li].data_ptr(), N, K, GS, 1, b["wc"].data_ptr(), b["ws"].data_ptr(),
-                                          b["pw"].data_ptr(), b["pw"].numel(), main.cuda_stream))
-            main.wait_stream(side)
-            check(L.amx_gemm_prepared(b["pa"].data_ptr(), b["pw"].data_ptr(), M, N, K, GS, b["c"].data_ptr(), N,
-                                      b["work"].data_ptr(), b["work"].numel(), main.cuda_stream))
-
-    overlap = fused_prepare and args.schedule == "overlap"
-    paired = fused_prepare and args.schedule == "pair"
-    cast_stream = torch.cuda.Stream() if (overlap or paired) else None
-
-    def run_step():
-        if paired:
-            step_paired(torch.cuda.current_stream(), cast_stream)
-        elif overlap:
-            step_overlapped(torch.cuda.current_stream(), cast_stream)
+                                          b["pa"].data_ptr(), b["pa"].numel(), st))
         else:
-            step(False, torch.cuda.current_stream().cuda_stream)
+            check(L.amx_quantize(A[li].data_ptr(), M, K, K, GS, b["ac"].data_ptr(), b["as"].data_ptr(), st))
+
+    def cast_w(li, st):
+        K, N = layers[li]
+        b = bufs[li]
+        if fused_prepare:
+            check(L.amx_quantize_prepared(W[li].data_ptr(), N, K, GS, 1, b["wc"].data_ptr(), b["ws"].data_ptr(),
+                                          b["pw"].data_ptr(), b["pw"].numel(), st))
+        else:
+            check(L.amx_quantize(W[li].data_ptr(), N, K, K, GS, b["wc"].data_ptr(), b["ws"].data_ptr(), st))
+
+    def gemm(li, st):
+        K, N = layers[li]
+        b = bufs[li]
+        if fused_prepare:
+            check(L.amx_gemm_prepared(b["pa"].data_ptr(), b["pw"].data_ptr(), M, N, K, GS, b["c"].data_ptr(), N,
+                                      b["work"].data_ptr(), b["work"].numel(), st))
+        else:
+            check(L.amx_gemm(b["ac"].data_ptr(), b["as"].data_ptr(), b["wc"].data_ptr(), b["ws"].data_ptr(),
+                             M, N, K, GS, gemm_flag, b["c"].data_ptr(), N, b["work"].data_ptr(), b["work"].numel(), st))
+
+    # Schedules of one step.  Every one records, when asked, CUDA events around the cast phase and the GEMM of each
+    # layer on the main stream (the stream the GEMM is launched on): the roofline of the GEMM kernel is taken from
+    # those events inside the timed region.
+    #   serial   one stream, kernels in order
+    #   pair     within a layer the cast of the activation and the cast of the weight run side by side (two
+    #            streams): they are independent inputs of the same GEMM in any model, and the small activation cast
+    #            fills the tail of the weight cast's last wave.  Layers stay in order.
+    #   overlap  all weight casts on a second stream, running ahead of the GEMMs of earlier layers (they depend on
+    #            nothing the step computes); not the default: in a model only the weights are available ahead
+    cast_stream = torch.cuda.Stream() if args.schedule in ("pair", "overlap") else None
+
+    def run_step(events=None):
+        main = torch.cuda.current_stream()
+        ms = main.cuda_stream
+        ready = []
+        if args.schedule == "overlap":
+            cast_stream.wait_stream(main)
+            for li in range(len(layers)):
+                cast_w(li, cast_stream.cuda_stream)
+                ev = torch.cuda.Event()
+                ev.record(cast_stream)
+                ready.append(ev)
+        for li in range(len(layers)):
+            if events is not None:
+                e0, e1, e2 = events[li]
+                e0.record(main)
+            if args.schedule == "pair":
+                cast_stream.wait_stream(main)
+                cast_a(li, cast_stream.cuda_stream)
+                cast_w(li, ms)
+                main.wait_stream(cast_stream)
+            elif args.schedule == "overlap":
+                cast_a(li, ms)
+                main.wait_event(ready[li])
+            else:
+                cast_a(li, ms)
+                cast_w(li, ms)
+            if events is not None:
+                e1.record(main)
+            gemm(li, ms)
+            if events is not None:
+                e2.record(main)
+        if args.schedule == "overlap":
+            main.wait_stream(cast_stream)
 
     def barrier():
         if world > 1:
@@ -465,17 +460,22 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    def new_events():
+        return [tuple(torch.cuda.Event(enable_timing=True) for _ in range(3)) for _ in layers]
+
     sampler = ClockSampler(local) if rank == 0 else None   # started early: nvidia-smi needs ~0.2 s to begin
-    for _ in range(max(args.warmup, 3)):
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
         run_step()
     barrier()
     if sampler:
         time.sleep(0.3)
         sampler.mark()
-    # The step is launch-bound in places (20 kernels, some of a few microseconds), so the timed region
-    # replays a CUDA graph of one step; --no-graph times plain launches instead.
+    # Plain launches with events between the kernels by default; --graph (the default for the small config 2, whose
+    # step is launch-bound in places) replays a CUDA graph of one step, and the per-kernel times then come from a
+    # separate pass of plain launches.
     graph = None
-    if not args.no_graph:
+    if use_graph:
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         graph = torch.cuda.CUDAGraph()
@@ -484,112 +484,97 @@ def run_ours(args):
         for _ in range(3):
             graph.replay()
         barrier()
+    step_events = [new_events() for _ in range(args.steps)] if graph is None else []
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
     t_start.record()
-    for _ in range(args.steps):
+    for i in range(args.steps):
         if graph is not None:
             graph.replay()
         else:
-            run_step()
+            run_step(step_events[i])
     t_end.record()
     barrier()
     elapsed_ms = t_start.elapsed_time(t_end)
     clocks = sampler.stop() if sampler else None
     elapsed_ms = sharding.max_over_ranks(elapsed_ms, "cuda")      # the slowest rank's time
-    # per-kernel-type times: a separate pass of plain launches with CUDA events around the casts and the GEMM
-    event_steps = min(args.steps, 50)
-    for _ in range(event_steps):
-        step(True)
-    torch.cuda.synchronize()
-    q_ms = sum(a.elapsed_time(b) for a, b in ev_q) * args.steps / event_steps
-    g_ms = sum(a.elapsed_time(b) for a, b in ev_g) * args.steps / event_steps
+    # a kernel that gave up on a bounded wait must not be reported as a fast run
+    for li in range(len(layers)):
+        st_word = amx.gemm_status(bufs[li]["work"])
+        if st_word != 0:
+            raise RuntimeError(f"layer {layer_ids[li]}: GEMM status {amx.status_string(st_word)}")
+    if graph is not None:
+        event_steps = min(args.steps, 50)
+        step_events = [new_events() for _ in range(event_steps)]
+        for ev in step_events:
+            run_step(ev)
+        torch.cuda.synchronize()
+    # per layer: mean duration of the cast phase and of the GEMM launch over the timed steps
+    q_ms_layer = [float(np.mean([ev[li][0].elapsed_time(ev[li][1]) for ev in step_events])) for li in range(len(layers))]
+    g_ms_layer = [float(np.mean([ev[li][1].elapsed_time(ev[li][2]) for ev in step_events])) for li in range(len(layers))]
+    q_ms, g_ms = sum(q_ms_layer), sum(g_ms_layer)     # per step
+
+    def timed_graph(fn, steps):
+        """Mean milliseconds of fn(stream) over `steps` replays of a CUDA graph of one call."""
+        fn(stream)
+        torch.cuda.synchronize()
+        sg = torch.cuda.Stream()
+        sg.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=sg):
+            fn(torch.cuda.current_stream().cuda_stream)
+        for _ in range(3):
+            g.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    extra_steps = max(3, min(args.steps, 30 if CONFIG == 2 else 10))
 
     # ---- the inference-time variant: weights cast and prepared once, activations per step (reported beside
     # the headline, which casts both operands every step)
     weights_cached = None
-    if "mxf4" in gemm_kernel and not args.layers:
-        prep = []
-        for li, (K, N) in enumerate(layers):
-            b = bufs[li]
-            pw = torch.empty(L.amx_prepared_bytes(N, K, GS, 1), dtype=torch.uint8, device="cuda")
-            pa = torch.empty(L.amx_prepared_bytes(M, K, GS, 0), dtype=torch.uint8, device="cuda")
-            check(L.amx_prepare(b["wc"].data_ptr(), b["ws"].data_ptr(), N, K, GS, 1, pw.data_ptr(), pw.numel(), stream))
-            prep.append((pa, pw))
-
-        def cached_step(stream):
-            for li, (K, N) in enumerate(layers):
-                b, (pa, pw) = bufs[li], prep[li]
-                check(L.amx_quantize_prepared(A[li].data_ptr(), M, K, GS, 0, b["ac"].data_ptr(), b["as"].data_ptr(),
-                                              pa.data_ptr(), pa.numel(), stream))
-                check(L.amx_gemm_prepared(pa.data_ptr(), pw.data_ptr(), M, N, K, GS, b["c"].data_ptr(), N,
-                                          b["work"].data_ptr(), b["work"].numel(), stream))
-
-        cached_step(stream)
-        torch.cuda.synchronize()
-        side2 = torch.cuda.Stream()
-        side2.wait_stream(torch.cuda.current_stream())
-        g2 = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g2, stream=side2):
-            cached_step(torch.cuda.current_stream().cuda_stream)
-        for _ in range(3):
-            g2.replay()
-        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        c0.record()
-        for _ in range(args.steps):
-            g2.replay()
-        c1.record()
-        torch.cuda.synchronize()
-        c_ms = sharding.max_over_ranks(c0.elapsed_time(c1) / args.steps, "cuda")
+    if fused_prepare and not args.layers:
+        def cached_step(st):
+            for li in range(len(layers)):
+                cast_a(li, st)
+                gemm(li, st)
+        c_ms = sharding.max_over_ranks(timed_graph(cached_step, extra_steps), "cuda")
         weights_cached = {"value": sharding.aggregate_rate(flops_step, world, c_ms) / 1e12, "unit": "TFLOP/s",
                           "ms_per_step": c_ms,
                           "what": "weights cast and prepared once; per step: cast + prepare activations, GEMM"}
-        del prep
 
     # ---- the paper's symmetric comparison formats on the same kernels (one shared scale per group: no split by
     # sign, one FP4 product per tile pair instead of four).  Shows what AMXFP4's asymmetry costs on this GPU, and
     # the rate of the FP4 pipe on this kernel design when nothing is split.
     format_variants = None
-    if "mxf4" in gemm_kernel and not args.layers and not args.skip_extras:
+    if fused_prepare and not args.layers and not args.skip_extras:
         format_variants = {}
         for name, fmt in (("sym_fp8", 1), ("mxfp4", 2)):
-            def fmt_step(stream, with_casts, fmt=fmt):
+            def fmt_step(st, with_casts=True, fmt=fmt):
                 for li, (K, N) in enumerate(layers):
                     b = bufs[li]
                     if with_casts:
                         check(L.amx_quantize_prepared_fmt(A[li].data_ptr(), M, K, GS, 0, fmt, b["ac"].data_ptr(),
-                                                          b["as"].data_ptr(), b["pa"].data_ptr(), b["pa"].numel(), stream))
+                                                          b["as"].data_ptr(), b["pa"].data_ptr(), b["pa"].numel(), st))
                         check(L.amx_quantize_prepared_fmt(W[li].data_ptr(), N, K, GS, 1, fmt, b["wc"].data_ptr(),
-                                                          b["ws"].data_ptr(), b["pw"].data_ptr(), b["pw"].numel(), stream))
-                    check(L.amx_gemm_prepared(b["pa"].data_ptr(), b["pw"].data_ptr(), M, N, K, GS, b["c"].data_ptr(), N,
-                                              b["work"].data_ptr(), b["work"].numel(), stream))
-
+                                                          b["ws"].data_ptr(), b["pw"].data_ptr(), b["pw"].numel(), st))
+                    gemm(li, st)
             res = {}
             for key, with_casts in (("step", True), ("gemm", False)):
-                fmt_step(stream, True)
-                torch.cuda.synchronize()
-                sv = torch.cuda.Stream()
-                sv.wait_stream(torch.cuda.current_stream())
-                gv = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(gv, stream=sv):
-                    fmt_step(torch.cuda.current_stream().cuda_stream, with_casts)
-                for _ in range(3):
-                    gv.replay()
-                v0, v1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                torch.cuda.synchronize()
-                v0.record()
-                for _ in range(args.steps):
-                    gv.replay()
-                v1.record()
-                torch.cuda.synchronize()
-                v_ms = v0.elapsed_time(v1) / args.steps
+                fmt_step(stream)
+                v_ms = timed_graph(lambda st: fmt_step(st, with_casts), extra_steps)
                 res[key + "_tflops"] = flops_step / (v_ms * 1e-3) / 1e12
                 res[key + "_ms"] = v_ms
             format_variants[name] = res
         format_variants["what"] = ("same workload and kernels with the symmetric formats (amx_quantize_prepared_fmt): "
-                                   "step = casts of both operands + GEMMs, gemm = the four GEMMs alone")
-        # leave the buffers as the headline step writes them
-        step(False, stream)
+                                   "step = casts of both operands + GEMMs, gemm = the GEMMs alone")
+        run_step()                      # leave the buffers as the headline step writes them
         torch.cuda.synchronize()
 
     # ---- the cast alone on a tensor larger than L2 (config-4 activation shape, 16384 x 8192 = 268 MB of bf16)
@@ -621,7 +606,8 @@ def run_ours(args):
     if not args.layers and not args.skip_extras and world == 1:
         attention = time_attention(32)
 
-    # ---- config 1: one small layer (128 x 1024 -> 1024), latency-bound: microseconds per call of amx_quant_gemm
+    # ---- config 1: one small layer (128 x 1024 -> 1024), latency-bound: microseconds per call of amx_quant_gemm,
+    # with the weight cast ahead of time and with both operands cast in the call
     small_case = None
     if not args.layers and not args.skip_extras and world == 1:
         a1b, w1b = to_dev(inputs.activation(1, 0)), to_dev(inputs.weight(1, 0))
@@ -629,46 +615,58 @@ def run_ours(args):
         M1, K1 = a1b.shape
         N1 = w1c.shape[0]
         c1 = torch.empty((M1, N1), dtype=torch.float32, device="cuda")
-        ws1 = torch.empty(max(L.amx_quant_gemm_workspace_bytes(M1, N1, K1, GS, 0), 256), dtype=torch.uint8, device="cuda")
+        ws1 = torch.empty(max(L.amx_quant_gemm_workspace_bytes(M1, N1, K1, GS, amx.WEIGHT_BF16), 256), dtype=torch.uint8,
+                          device="cuda")
 
-        def small():
-            check(L.amx_quant_gemm(a1b.data_ptr(), K1, w1c.data_ptr(), w1s.data_ptr(), M1, N1, K1, GS, 0, c1.data_ptr(), N1,
+        def small(both):
+            check(L.amx_quant_gemm(a1b.data_ptr(), K1, None if both else w1c.data_ptr(), None if both else w1s.data_ptr(),
+                                   w1b.data_ptr() if both else None, K1 if both else 0, M1, N1, K1, GS, 0, c1.data_ptr(), N1,
                                    ws1.data_ptr(), ws1.numel(), stream))
 
-        for _ in range(5):
-            small()
-        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        s0.record()
-        for _ in range(200):
-            small()
-        s1.record()
-        torch.cuda.synchronize()
-        small_case = {"workload": f"config 1: A {M1}x{K1} cast per call, W {N1}x{K1} cast once; amx_quant_gemm",
-                      "us_per_call": s0.elapsed_time(s1) * 1e3 / 200,
-                      "note": "launch-latency-bound (32 output tiles at most): microseconds, not a roofline fraction"}
+        us = {}
+        for both in (False, True):
+            for _ in range(5):
+                small(both)
+            s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            s0.record()
+            for _ in range(200):
+                small(both)
+            s1.record()
+            torch.cuda.synchronize()
+            us[both] = s0.elapsed_time(s1) * 1e3 / 200
+        small_case = {"workload": f"config 1: A {M1}x{K1}, W {N1}x{K1}; one call of amx_quant_gemm",
+                      "us_per_call": us[False], "us_per_call_both_operands_cast": us[True],
+                      "note": "us_per_call: the weight was cast ahead of time; both_operands_cast: the bf16 weight is "
+                              "cast in the same call.  Launch-latency-bound (32 output tiles at most): microseconds, "
+                              "not a roofline fraction"}
 
     # ---- decode-like shape: 16 token rows against the config-2 weights (see time_decode)
     decode = None
-    if not args.layers and not args.skip_extras and world == 1 and CONFIG == 2:
-        decode = time_decode(args.steps, A, W)
+    if not args.layers and not args.skip_extras and world == 1:
+        decode = time_decode(max(20, min(args.steps, 100)))
 
-    # ---- end to end through the host-buffer entry point (pinned host tensors, copies inside the timing)
+    # ---- end to end through the host-buffer entry point (pinned host tensors, copies inside the timing).
+    # Consecutive layers alternate between two streams and two workspaces and the call does not synchronise
+    # (AMX_HOST_NO_SYNC), so that one layer's result goes back to the host while the next layer's inputs come in.
     e2e = None
-    if (rank == 0 or world > 1) and not args.skip_extras and CONFIG == 2:
+    if (rank == 0 or world > 1) and not args.skip_extras:
         pinned = []
         for li, (K, N) in enumerate(layers):
             a_bits, w_bits = host[li]
             pinned.append((torch.from_numpy(a_bits.view(np.int16)).view(torch.bfloat16).pin_memory(),
                            torch.from_numpy(w_bits.view(np.int16)).view(torch.bfloat16).pin_memory(),
                            torch.empty((M, N), dtype=torch.float32).pin_memory()))
-        lh_bytes = max(L.amx_linear_host_workspace_bytes(M, N, K, GS) for K, N in layers)
-        lh_ws = torch.empty(lh_bytes, dtype=torch.uint8, device="cuda")
+        lh_bytes = max(L.amx_linear_host_workspace_bytes(M, N, K, GS, gemm_flag) for K, N in layers)
+        lh_ws = [torch.empty(lh_bytes, dtype=torch.uint8, device="cuda") for _ in range(2)]
+        lh_streams = [torch.cuda.Stream(), torch.cuda.Stream()]
 
         def e2e_step():
-            for li in range(len(layers)):
+            for li, (K, N) in enumerate(layers):
                 a, w, c = pinned[li]
-                amx.linear_host(a, w, c, lh_ws, GS)
+                check(L.amx_linear_host(a.data_ptr(), w.data_ptr(), M, N, K, GS, gemm_flag | amx.HOST_NO_SYNC, c.data_ptr(),
+                                        lh_ws[li % 2].data_ptr(), lh_ws[li % 2].numel(), lh_streams[li % 2].cuda_stream))
+            torch.cuda.synchronize()
 
         e2e_step()
         barrier()
@@ -676,13 +674,15 @@ def run_ours(args):
         t0 = time.perf_counter()
         for _ in range(e2e_steps):
             e2e_step()
-        torch.cuda.synchronize()
         e2e_s = (time.perf_counter() - t0) / e2e_steps
         e2e_s = sharding.max_over_ranks(e2e_s, "cuda")
         e2e = {"value": world * flops_step / e2e_s / 1e12, "unit": "TFLOP/s",
                "h2d_bytes_per_step": int(elems_step * 2),
                "d2h_bytes_per_step": int(sum(M * N * 4 for _, N in layers)),
-               "ms_per_step": e2e_s * 1e3}
+               "ms_per_step": e2e_s * 1e3,
+               "what": "amx_linear_host per layer from pinned host buffers; layers alternate between two streams, so "
+                       "host-to-device and device-to-host copies of neighbouring layers overlap; PCIe-bound"}
+        del pinned, lh_ws
 
     if rank != 0:
         if world > 1:
@@ -692,43 +692,64 @@ def run_ours(args):
 
     ms_per_step = elapsed_ms / args.steps
     value = sharding.aggregate_rate(flops_step, world, ms_per_step) / 1e12
-    gemm_tflops = args.steps * flops_step / (g_ms * 1e-3) / 1e12
-    quant_gbs = args.steps * elems_step * BYTES_PER_ELEM / (q_ms * 1e-3) / 1e9
-    fp4_peak = 4.0 * peaks["bf16_tflops_sustained"]
+    gemm_tflops = flops_step / (g_ms * 1e-3) / 1e12
+    quant_gbs = elems_step * BYTES_PER_ELEM / (q_ms * 1e-3) / 1e9
+    moved = MOVED_BYTES_PER_ELEM if fused_prepare else BYTES_PER_ELEM
+    # Roofline denominator of the GEMM: 4 x the measured bf16 cuBLAS rate (nominal FP4 : bf16 ratio).  Which bf16
+    # figure applies depends on the run: a timed region that stayed at (nearly) full clock without the power cap is
+    # a burst, anything else is sustained.  Both fractions are printed.
+    sm, sm_max = (clocks or {}).get("sm_mhz"), (clocks or {}).get("sm_max_mhz")
+    burst = bool(sm and sm_max and sm >= 0.95 * sm_max and "sw_power_cap" not in (clocks or {}).get("reasons", []))
+    peak_burst, peak_sust = 4.0 * peaks["bf16_tflops"], 4.0 * peaks["bf16_tflops_sustained"]
+    fp4_peak = peak_burst if burst else peak_sust
     line = {
         "metric": "AMXFP4 quant+GEMM TFLOPS", "value": value, "unit": "TFLOP/s", "n_gpus": world,
-        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+        "steps": args.steps, "warmup": warmup, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp4xfp4->f32",
         "data": "synthetic",
         "config": {"workload": (WORKLOADS[CONFIG] + "; activations and weights both cast to AMXFP4 every step, then GEMM"),
                    "group_size": GS, "gemm_kernel": gemm_kernel,
                    "entry_points": "amx_quantize_prepared + amx_gemm_prepared" if fused_prepare else "amx_quantize + amx_gemm",
                    "l2": f"per-step inputs (~{int(elems_step * 2 / 1e6)} MB of bf16) exceed the 126 MB L2",
-                   "launch": "plain launches" if args.no_graph else "CUDA graph of one step, replayed",
-                   "schedule": ("weight casts on a second stream, overlapping the GEMMs of earlier layers" if overlap else
-                                "layers in order; a layer's two casts side by side on two streams" if paired else
-                                "one stream, kernels in order")},
+                   "launch": "CUDA graph of one step, replayed" if use_graph else "plain launches, CUDA events between the kernels",
+                   "schedule": {"overlap": "weight casts on a second stream, overlapping the GEMMs of earlier layers",
+                                "pair": "layers in order; a layer's two casts side by side on two streams",
+                                "serial": "one stream, kernels in order"}[args.schedule]},
         "pct_of_nominal_fp4_peak": 100.0 * value / world / NOMINAL_FP4_TFLOPS,
         "nominal_fp4_peak_tflops": NOMINAL_FP4_TFLOPS,
-        "quantize": {"gb_per_s": quant_gbs, "pct_of_nominal_hbm_8TBs": 100.0 * quant_gbs / NOMINAL_HBM_GBS,
-                     "frac_of_measured_copy": quant_gbs / peaks["hbm_gbs"], "bytes_per_element": BYTES_PER_ELEM,
-                     "ms_per_step": q_ms / args.steps, "large_tensor": quant_large,
-                     # the step's casts also write the GEMM-ready sign planes and scale factors: bytes actually moved
-                     "bytes_per_element_moved": MOVED_BYTES_PER_ELEM if fused_prepare else BYTES_PER_ELEM,
-                     "gb_per_s_moved": quant_gbs * (MOVED_BYTES_PER_ELEM / BYTES_PER_ELEM if fused_prepare else 1.0),
-                     "note": ("gb_per_s counts the canonical bytes only (2.5625 B/element); the step's casts also write "
-                              "the GEMM-ready sign planes and scale factors in the same pass (gb_per_s_moved); timed by "
-                              "events in a pass of plain launches; large_tensor is the plain amx_quantize")
-                             if fused_prepare else "plain amx_quantize"},
-        "gemm": {"useful_tflops": gemm_tflops, "ms_per_step": g_ms / args.steps,
+        "gemm": {"useful_tflops": gemm_tflops, "ms_per_step": g_ms, "ms_per_layer": g_ms_layer,
                  # the sign split issues four FP4 products per useful one
                  "issued_tflops": gemm_tflops * (4.0 if "mxf4" in gemm_kernel else 1.0),
                  "pct_of_nominal_fp4_peak": 100.0 * gemm_tflops / NOMINAL_FP4_TFLOPS},
         "roofline": {"bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
-                     "frac": gemm_tflops / fp4_peak, "traffic": GEMM_DRAM_TRAFFIC_PER_LAUNCH.get(args.gemm),
+                     "frac": gemm_tflops / fp4_peak, "traffic": GEMM_DRAM_TRAFFIC_PER_LAUNCH.get(CONFIG),
+                     "frac_burst": gemm_tflops / peak_burst, "frac_sustained": gemm_tflops / peak_sust,
+                     "regime": "burst" if burst else "sustained",
                      "exact_mapping_ceiling_frac": 0.25,
                      "kernel": f"amx_gemm ({gemm_kernel})",
-                     "peak_source": f"4 x sustained bf16 cuBLAS rate ({peaks['source']}), nominal FP4:bf16 ratio"},
+                     "timing": ("CUDA events around every GEMM launch inside the timed region" if not use_graph else
+                                "CUDA events around every GEMM launch in a pass of plain launches after the timed graph replays"),
+                     "peak_source": f"4 x {'burst' if burst else 'sustained'} bf16 cuBLAS rate ({peaks['source']}), nominal "
+                                    "FP4:bf16 ratio; burst when the sampled SM clock stayed within 5 % of its maximum with "
+                                    "no power cap",
+                     # the HBM-bound kernel of the step: the cast
+                     "quantize": {"bound": "hbm", "unit": "GB/s", "peak": peaks["hbm_gbs"],
+                                  "peak_source": f"copy rate ({peaks['source']})",
+                                  "prepared_cast": {"bytes_per_element": moved, "achieved": quant_gbs * moved / BYTES_PER_ELEM,
+                                                    "frac": quant_gbs * moved / BYTES_PER_ELEM / peaks["hbm_gbs"],
+                                                    "achieved_canonical_bytes": quant_gbs,
+                                                    "what": "both casts of every layer of the step (events around the cast "
+                                                            "phase); bytes actually moved: canonical 2.5625 B/element plus "
+                                                            "the sign planes and scale factors of the FP4 kernel's operand"},
+                                  "plain_cast": (None if quant_large is None else
+                                                 {"bytes_per_element": BYTES_PER_ELEM, "achieved": quant_large["gb_per_s"],
+                                                  "frac": quant_large["frac_of_measured_copy"],
+                                                  "pct_of_nominal_hbm_8TBs": quant_large["pct_of_nominal_hbm_8TBs"],
+                                                  "what": "amx_quantize on 16384 x 8192 (268 MB of bf16)"})}},
+        "quantize": {"gb_per_s": quant_gbs, "pct_of_nominal_hbm_8TBs": 100.0 * quant_gbs / NOMINAL_HBM_GBS,
+                     "frac_of_measured_copy": quant_gbs / peaks["hbm_gbs"], "bytes_per_element": BYTES_PER_ELEM,
+                     "ms_per_step": q_ms, "ms_per_layer": q_ms_layer, "large_tensor": quant_large,
+                     "bytes_per_element_moved": moved, "gb_per_s_moved": quant_gbs * moved / BYTES_PER_ELEM},
         "weights_cached": weights_cached,
         "format_variants": format_variants,
         "attention": attention,
@@ -740,7 +761,7 @@ def run_ours(args):
         # one preparation kernel each on top
         "gpu_launches": (5 if "mxf4" in gemm_kernel and not fused_prepare else 3) * len(layers) * args.steps,
     }
-    if len(layer_ids) != 4:
+    if len(layer_ids) != len(inputs.LINEAR_CONFIGS[CONFIG]["layers"]):
         line["config"]["layers"] = layer_ids
     if world == 1 and not args.skip_extras:
         line["cpu_baseline"] = cpu_baseline()
@@ -753,7 +774,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--gemm", default="auto", choices=["auto", "simt", "tc", "fp4"], help="GEMM kernel to time")
@@ -761,14 +782,15 @@ def main():
     ap.add_argument("--schedule", choices=["serial", "pair", "overlap"], default="pair",
                     help="pair (default): a layer's two casts side by side, layers in order; serial: one stream; "
                          "overlap: weight casts on a second stream, running ahead of the GEMMs")
-    ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of a CUDA graph of the step")
+    ap.add_argument("--graph", action="store_true", help="time replays of a CUDA graph of one step (the default for config 2)")
+    ap.add_argument("--no-graph", action="store_true", help="config 2: time plain launches instead of the graph")
     ap.add_argument("--layers", default="", help="comma-separated layer indices to run (profiling aid; default all)")
     ap.add_argument("--skip-extras", action="store_true", help="skip the e2e and cpu_baseline legs (profiling aid)")
     ap.add_argument("--attention-only", action="store_true", help="time only the config-5 attention call (profiling aid)")
     ap.add_argument("--heads", type=int, default=32, help="heads for --attention-only")
     ap.add_argument("--decode-only", action="store_true", help="time only the 16-row decode step (profiling aid)")
-    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4],
-                    help="linear-layer workload (default 2, the one the metric is quoted on; 3 and 4 are larger)")
+    ap.add_argument("--config", type=int, default=4, choices=[2, 3, 4],
+                    help="linear-layer workload (default 4, the largest that fits one GPU; 2 and 3 are smaller)")
     args = ap.parse_args()
     global CONFIG
     CONFIG = args.config

@@ -10,6 +10,8 @@
  *   - Pointers are DEVICE pointers owned by the caller unless the name of the
  *     argument ends in _host.  The library allocates no device memory and keeps
  *     no state between calls; scratch comes from the caller as `workspace`.
+ *     (One exception, stated at its declaration: amx_quant_gemm_static keeps its
+ *     scratch in a fixed array inside the library image.)
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
  *     stream).  Work is enqueued on it; calls return without synchronising
  *     unless stated otherwise.
@@ -22,7 +24,10 @@
  *       scales  uint8 [rows, K/gs, 2]  E5M2 bytes: [..][0] positive-side scale,
  *                                      [..][1] negative-side scale
  *     That is 4.5 bits per element at gs = 32.
- *   - group_size (gs) must be 16, 32, 64 or 128 and divide K.
+ *   - group_size (gs) must be 16, 32, 64 or 128 and divide K; or gs == K (K % 8 == 0): the whole row is
+ *     one group, the grouping of the worked example in Appendix B.3 (`group_size=-1` there).  Whole-row
+ *     groups are taken by amx_quantize / amx_quantize_fmt, amx_dequantize and the plain GEMM kernel
+ *     (amx_gemm / amx_quant_gemm pick it by themselves); the tensor-core kernels need gs = 32.
  *   - NaN / Inf inputs are outside the format's definition; results for them are
  *     unspecified (no fault).
  */
@@ -71,14 +76,26 @@ typedef enum amx_status {
  * the tensor cores - the FP4 kernel when M*N*K >= 2^27, the exact bf16-decode kernel below that and for
  * at most 64 rows of A against a large weight (decode-like shapes: that kernel then cuts K into slices over
  * CTAs and adds the partial products in slice order) - except that at most 64 rows of A with K >= 512 and
- * K % 128 == 0 go to the weight-streaming kernel (AMX_GEMM_ROWS); other group sizes run on the SIMT kernel. */
+ * K % 128 == 0 go to the weight-streaming kernel (AMX_GEMM_ROWS); other group sizes run on the SIMT kernel.
+ * AUTO never loses a scale: where it picks the FP4 kernel and preparing the operands had to flush one (see
+ * AMX_GEMM_FP4), the FP4 kernel returns at once and the exact bf16-decode kernel computes the product instead.
+ * The decision is taken on the device, from the count amx_gemm_flushed_scales() reports; it costs one empty
+ * launch per call and the bf16-decode kernel's scratch on top of the FP4 kernel's. */
 #define AMX_GEMM_AUTO 0x0u
 #define AMX_GEMM_SIMT 0x10u  /* plain CUDA-core kernel: any shape, any supported gs */
 #define AMX_GEMM_TC 0x20u    /* tcgen05 kernel, exact bf16 decode: AMX_ERR_SHAPE if the shape does not fit */
-#define AMX_GEMM_FP4 0x40u   /* tcgen05 block-scaled FP4 kernel (four sign-pair MMAs per tile).  Scales more
-                              * than 14 binades below the largest scale of their operand row are flushed to
-                              * zero (relative effect < 2^-14 per row); otherwise same result up to fp32
-                              * summation order.  Needs the larger workspace amx_workspace_bytes() reports. */
+#define AMX_GEMM_FP4 0x40u   /* tcgen05 block-scaled FP4 kernel (four sign-pair MMAs per tile).  The kernel's
+                              * scale type (UE4M3) spans 15 binades, E5M2 spans 32: per operand row the scales
+                              * are shifted so that the row's largest lands in the top binade, and a nonzero
+                              * scale 15 or more binades below it is FLUSHED to zero - its group then contributes
+                              * nothing.  One flushed group is below 2^-14 of the row's largest group, but a row
+                              * can hold K/32 - 1 of them: the error of an output is bounded by
+                              * (number of flushed groups) * 2^-14 of its dominant term, i.e. up to K * 2^-19
+                              * (1.6 % at K = 8192) for adversarial rows; rows whose scales span less than 15
+                              * binades (all of the benchmark's data) lose nothing and the result then equals
+                              * the other kernels' up to fp32 summation order.  Flushed scales are counted:
+                              * amx_gemm_flushed_scales / amx_prepared_flushed_scales.  Needs the larger
+                              * workspace amx_workspace_bytes() reports. */
 #define AMX_GEMM_ROWS 0x100u /* weight-streaming kernel for M <= 64 rows of A (decode phase): reads the canonical
                               * weight once, exact bf16 decode, K ranges added in a fixed order; gs = 32,
                               * K % 128 == 0, else AMX_ERR_SHAPE; w_scales 4-byte aligned, else AMX_ERR_ALIGN
@@ -89,8 +106,12 @@ typedef enum amx_status {
  * are what bounds that kernel, so this is slower than the default two launches (measured 1.05x at
  * 128 x 1024 x 1024, 1.25x at 2048 x 12288 x 4096); it is for callers that must not hold the codes. */
 #define AMX_GEMM_CAST_IN_KERNEL 0x80u
-/* extra flag for amx_attention: causal mask */
+/* flag for amx_quant_gemm_workspace_bytes: size the scratch for a bf16 weight (amx_quant_gemm called with W_bf16) */
+#define AMX_WEIGHT_BF16 0x200u
+/* extra flag for amx_attention / amx_attention_map: causal mask */
 #define AMX_ATTN_CAUSAL 0x1000u
+/* extra flag for amx_linear_host: return after enqueueing everything, without synchronising `stream` */
+#define AMX_HOST_NO_SYNC 0x2000u
 
 /*
  * amx_quantize - direct cast of a bf16 matrix to AMXFP4 (Sections 4.2-4.3; procedure per
@@ -104,7 +125,8 @@ typedef enum amx_status {
  *   x       bf16 [rows, ld_x] row-major, ld_x >= K in elements; 16-byte aligned, ld_x % 8 == 0
  *   codes   out, [rows, K/2], 16-byte aligned (8-byte for gs = 16)
  *   scales  out, [rows, K/gs, 2], 2-byte aligned
- * K % 8 == 0 is required.  rows == 0 is a no-op.
+ * K % 8 == 0 is required.  rows == 0 is a no-op.  With gs == K (whole-row groups) scales is [rows, 1, 2] and
+ * codes need 4-byte alignment only.
  */
 int amx_quantize(const void* x, int64_t rows, int64_t K, int64_t ld_x, int group_size,
                  uint8_t* codes, uint8_t* scales, void* stream);
@@ -185,13 +207,22 @@ int amx_gemm_prepared(const void* a_prepared, const void* w_prepared, int64_t M,
 /*
  * amx_quant_gemm - the fully quantized linear layer of Section 5 ("quantize input operands for
  * all decoder-layer matrix multiplications"): quantizes the bf16 activation A[M, ld_a] and
- * multiplies it with an already quantized weight.  Same result as amx_quantize followed by
- * amx_gemm, which is also how it runs (two launches; the workspace additionally holds the quantized
- * activation) unless AMX_GEMM_TC | AMX_GEMM_CAST_IN_KERNEL asks for the single-launch kernel.
- * AMX_GEMM_CAST_IN_KERNEL with any other kernel choice: AMX_ERR_FLAGS.  A 16-byte aligned, ld_a % 8 == 0.
+ * multiplies it with the weight, which comes in exactly one of two forms:
+ *   w_codes / w_scales   an already quantized weight, canonical [N, K] (then W_bf16 must be NULL), or
+ *   W_bf16, ld_w         a bf16 weight [N, ld_w] that this call casts as well (then w_codes and w_scales must
+ *                        be NULL): both operands of the layer are cast per call, the direct-cast setting of
+ *                        Section 5 with nothing prepared ahead
+ * Same result as amx_quantize (of each bf16 operand) followed by amx_gemm.  How it runs: on the FP4 kernel each
+ * bf16 operand with contiguous rows is cast by one launch that also writes the kernel's operand form; on the
+ * weight-streaming kernel the few rows of A are cast and decoded in one launch; otherwise amx_quantize per bf16
+ * operand, then the GEMM; AMX_GEMM_TC | AMX_GEMM_CAST_IN_KERNEL asks for the kernel that casts A inside
+ * (with any other kernel choice: AMX_ERR_FLAGS).  The workspace additionally holds the quantized operands:
+ * amx_quant_gemm_workspace_bytes(flags | AMX_WEIGHT_BF16) with a bf16 weight.
+ * A (and W_bf16) 16-byte aligned, ld_a % 8 == 0 (ld_w % 8 == 0).
  */
 int amx_quant_gemm(const void* A, int64_t ld_a,
                    const uint8_t* w_codes, const uint8_t* w_scales,
+                   const void* W_bf16, int64_t ld_w,
                    int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags,
                    float* C, int64_t ld_c, void* workspace, size_t workspace_bytes, void* stream);
 
@@ -242,29 +273,59 @@ int amx_attention(const void* q, const void* k, const void* v, int64_t heads, in
 size_t amx_attention_workspace_bytes(int64_t L, int64_t d);
 
 /*
+ * amx_attention_map - the cast attention map of ONE head exactly as amx_attention builds it when it does not
+ * store the logits (both products on the FP4 kernel, L % 256 == 0): P = softmax(Q K^T / sqrt(d)) per row,
+ * rounded to bf16 and cast to AMXFP4 inside the epilogue of the second pass over Q K^T (Appendix C: the
+ * self-attention map is quantized).  Same kernels, same launch sequence; in addition the epilogue stores what
+ * amx_attention never writes, so that the cast can be checked against a reference:
+ *   p_bf16      out, nullable: bf16 [L, L], the normalised map as rounded to bf16 - the cast's input
+ *   p_codes     out, nullable: canonical codes [L, L/2] of that map;  p_scales  out, nullable: [L, L/32, 2]
+ *   p_prepared  out: the left-hand operand of P V in the FP4 kernel's form (positive plane, UE4M3 scale factors,
+ *               row words), amx_prepared_bytes(L, L, 32, 0) bytes, 256-aligned
+ *   flags       0 or AMX_ATTN_CAUSAL (blocks of keys entirely after their queries are not visited; their
+ *               entries of the three optional outputs are zero)
+ *   workspace   amx_attention_workspace_bytes(L, d) bytes
+ * AMX_ERR_SHAPE when L % 256 != 0 or d % 32 != 0.
+ */
+int amx_attention_map(const void* q, const void* k, int64_t L, int64_t d, uint32_t flags, void* p_bf16,
+                      uint8_t* p_codes, uint8_t* p_scales, void* p_prepared, size_t prepared_bytes,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * amx_linear_host - one whole layer from HOST memory: copies the bf16 activation A_host[M,K] and
  * weight W_host[N,K] to the device, quantizes both, multiplies, and copies C back to
  * C_host[M,N] (fp32).  All copies and kernels are enqueued on `stream`; the call returns after
- * synchronising it.  Host buffers should be page-locked for the copies to be asynchronous.
- *   workspace  device scratch, at least amx_linear_host_workspace_bytes(M, N, K, gs) bytes
+ * synchronising it - unless flags carry AMX_HOST_NO_SYNC: then it returns once everything is enqueued, the
+ * caller synchronises, and calls on different streams with different workspaces overlap their copies in both
+ * directions.  Host buffers should be page-locked for the copies to be asynchronous.  Runs as amx_quant_gemm
+ * with a bf16 weight.  All arguments are checked before the first copy is enqueued.
+ *   flags      AMX_GEMM_* kernel choice, optionally | AMX_HOST_NO_SYNC
+ *   workspace  device scratch, at least amx_linear_host_workspace_bytes(M, N, K, gs, flags) bytes
  */
 int amx_linear_host(const void* A_host, const void* W_host, int64_t M, int64_t N, int64_t K,
                     int group_size, uint32_t flags, float* C_host,
                     void* workspace, size_t workspace_bytes, void* stream);
 
 /*
- * amx_quant_gemm_static - amx_quant_gemm without a workspace argument, for callers that cannot
- * allocate device memory: processes that gave the whole GPU to their own memory pool at start-up,
+ * amx_quant_gemm_static - amx_quant_gemm (quantized-weight form) without a workspace argument, for callers
+ * that cannot allocate device memory: processes that gave the whole GPU to their own memory pool at start-up,
  * plug-ins that must not touch the allocator, and latency-critical loops that cannot afford an
  * allocation's implicit synchronisation.  (The paper has no counterpart; this is a deployment
- * convenience of this library.)  Same arguments and result as amx_quant_gemm otherwise.
- *   - The scratch (quantized activation + status word) is a fixed 16 MiB array that is part of the
- *     library image: every GPU that loads the library holds it until the process exits.
- *     amx_quant_gemm_static_capacity() returns its size; a problem for which
+ * convenience of this library.)  Same result as amx_quant_gemm with the same kernel choice.
+ *   - flags: AMX_GEMM_AUTO, AMX_GEMM_SIMT or AMX_GEMM_TC only.  AMX_GEMM_FP4, AMX_GEMM_ROWS and
+ *     AMX_GEMM_CAST_IN_KERNEL are rejected with AMX_ERR_FLAGS; AUTO may still pick any kernel.
+ *   - The scratch is a fixed 16 MiB array that is part of the library image: every GPU that loads the
+ *     library holds it until the process exits.  It holds whatever amx_quant_gemm would keep in its
+ *     workspace: the status word, the quantized activation and, when AUTO picks the FP4 kernel, both
+ *     operands in that kernel's form.  amx_quant_gemm_static_capacity() returns its size; a problem for which
  *     amx_quant_gemm_workspace_bytes() exceeds it is rejected with AMX_ERR_TOO_LARGE and nothing runs.
  *   - The entry point calls no cudaMalloc / cudaFree and no allocating library routine.
- *   - The first call on each device looks up the array's device address; make that first call
- *     outside any stream capture.
+ *   - The first call on each device looks up the array's device address, which is also when the CUDA
+ *     runtime loads this part of the library onto the device and the array starts to occupy memory there:
+ *     make that first call outside any stream capture and BEFORE the application's own pool takes the rest of
+ *     the device, or the call fails with AMX_ERR_CUDA (nothing was launched; the error is cleared).
+ *   - amx_quant_gemm_static_status() reads the status word the way amx_gemm_status does for a caller-owned
+ *     workspace (AMX_ERR_TIMEOUT after a bounded device-side wait expired); it synchronises `stream`.
  *   - All calls share the one array, which keeps whatever the previous call left in it.  The
  *     call itself re-initialises what it needs; but two calls whose work overlaps on the GPU
  *     (different streams or host threads) race on the array - serialise them.
@@ -274,6 +335,7 @@ int amx_quant_gemm_static(const void* A, int64_t ld_a,
                           int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags,
                           float* C, int64_t ld_c, void* stream);
 size_t amx_quant_gemm_static_capacity(void);
+int amx_quant_gemm_static_status(void* stream);
 
 /*
  * amx_quant_error - squared error of a quantized tensor against its bf16 source, split as the appendix
@@ -297,18 +359,44 @@ size_t amx_quant_error_workspace_bytes(void);
 /* Scratch sizes (bytes; 0 is possible).  Return 0 for invalid shapes. */
 size_t amx_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags);
 size_t amx_quant_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags);
-size_t amx_linear_host_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size);
+size_t amx_linear_host_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags);
 
 /* Which kernel amx_gemm would run for this shape and flags: one AMX_GEMM_* kernel bit, or 0 when the flags
  * cannot be honoured for the shape. */
 uint32_t amx_gemm_kernel_for(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags);
 
 /*
- * Status word of the most recent tensor-core GEMM that used `workspace`: AMX_OK, or
- * AMX_ERR_TIMEOUT when a bounded wait inside the kernel expired (the kernel then stopped
- * issuing work, released its resources and returned; C is not valid).  Synchronises `stream`.
+ * Status word of the most recent amx_gemm / amx_quant_gemm / amx_gemm_prepared that used `workspace` (its
+ * first word, for every kernel that takes a workspace): AMX_OK, or AMX_ERR_TIMEOUT when a bounded wait inside
+ * a tensor-core kernel expired (the kernel then stopped issuing work, released its resources and returned; C is
+ * not valid).  The weight-streaming kernel has no such wait and always leaves AMX_OK.  Synchronises `stream`.
  */
 int amx_gemm_status(const void* workspace, void* stream);
+
+/*
+ * Flushed scales (see AMX_GEMM_FP4).  amx_gemm_flushed_scales: how many nonzero scales of the two operands the
+ * most recent amx_gemm / amx_quant_gemm that used `workspace` flushed while preparing them for the FP4 kernel
+ * (the workspace's second word; 0 for the other kernels); under AMX_GEMM_AUTO a nonzero count means the exact
+ * bf16-decode kernel computed the product.  amx_prepared_flushed_scales: the same count for one prepared operand
+ * (amx_prepare, amx_quantize_prepared[_fmt], amx_softmax_quantize), read from its per-row words.
+ * Both synchronise `stream` and return the count, or a negative amx_status.
+ */
+int64_t amx_gemm_flushed_scales(const void* workspace, void* stream);
+int64_t amx_prepared_flushed_scales(const void* prepared, int64_t rows, int64_t K, int group_size, int is_weight,
+                                    void* stream);
+
+/*
+ * amx_selftest_wait_timeout - exercises the bounded-wait protocol of the tensor-core kernels without a GEMM:
+ * one CTA allocates tensor memory, starts a bulk copy, then waits on an mbarrier nothing arrives at.  After
+ * `polls` polls (1..65536) the waiting role gives up, records AMX_ERR_TIMEOUT in the status word
+ * (amx_gemm_status(workspace) returns it), the other roles leave through the abort flag, the copy is drained,
+ * tensor memory is released and the kernel returns; the context stays usable.  (No counterpart in the paper: a
+ * check of this library's failure handling.)
+ *   workspace  at least 2048 bytes, 256-aligned.  After the kernel, int words 8..11 tell how warps 0..3 left
+ *              their wait (2 = gave up at its own limit, 3 = left through the abort flag, 1 = the wait
+ *              completed, which must not happen) and word 12 is 1 when the copy in flight was seen to land.
+ */
+int amx_selftest_wait_timeout(void* workspace, size_t workspace_bytes, uint32_t polls, void* stream);
 
 const char* amx_status_string(int status);
 

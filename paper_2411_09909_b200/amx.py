@@ -21,7 +21,9 @@ GEMM_ROWS = 0x100               # weight-streaming kernel for at most 64 rows of
 GEMM_CAST_IN_KERNEL = 0x80      # amx_quant_gemm only, together with GEMM_TC
 FMT_AMXFP4, FMT_SYM_FP8, FMT_MXFP4 = 0, 1, 2
 FMT_AMXFP4_POT, FMT_MXFP4_POT_ROUND, FMT_AMXFP4_POT_ROUND = 3, 4, 5   # amx_quantize_fmt only
-ATTN_CAUSAL = 0x1000            # amx_attention only
+WEIGHT_BF16 = 0x200             # amx_quant_gemm_workspace_bytes: size for a bf16 weight
+ATTN_CAUSAL = 0x1000            # amx_attention / amx_attention_map
+HOST_NO_SYNC = 0x2000           # amx_linear_host: do not synchronise
 
 # every symbol include/amx.h declares
 SYMBOLS = (
@@ -34,6 +36,8 @@ SYMBOLS = (
     "amx_prepared_bytes", "amx_prepare", "amx_gemm_prepared", "amx_quantize_prepared", "amx_softmax_quantize",
     "amx_quantize_fmt", "amx_quantize_prepared_fmt", "amx_gemm_prepared_workspace_bytes",
     "amx_quant_error", "amx_quant_error_workspace_bytes",
+    "amx_attention_map", "amx_gemm_flushed_scales", "amx_prepared_flushed_scales", "amx_selftest_wait_timeout",
+    "amx_quant_gemm_static_status",
 )
 
 
@@ -57,7 +61,14 @@ def lib() -> ctypes.CDLL:
         L.amx_quant_error.argtypes = [p, i64, i64, i64, p, p, i, p, p, sz, p]
         L.amx_quant_error_workspace_bytes.argtypes = []
         L.amx_quant_error_workspace_bytes.restype = sz
-        L.amx_quant_gemm.argtypes = [p, i64, p, p, i64, i64, i64, i, u32, p, i64, p, sz, p]
+        L.amx_quant_gemm.argtypes = [p, i64, p, p, p, i64, i64, i64, i64, i, u32, p, i64, p, sz, p]
+        L.amx_attention_map.argtypes = [p, p, i64, i64, u32, p, p, p, p, sz, p, sz, p]
+        L.amx_gemm_flushed_scales.argtypes = [p, p]
+        L.amx_gemm_flushed_scales.restype = i64
+        L.amx_prepared_flushed_scales.argtypes = [p, i64, i64, i, i, p]
+        L.amx_prepared_flushed_scales.restype = i64
+        L.amx_selftest_wait_timeout.argtypes = [p, sz, u32, p]
+        L.amx_quant_gemm_static_status.argtypes = [p]
         L.amx_quant_gemm_static.argtypes = [p, i64, p, p, i64, i64, i64, i, u32, p, i64, p]
         L.amx_quant_gemm_static_capacity.argtypes = []
         L.amx_quant_gemm_static_capacity.restype = sz
@@ -77,7 +88,7 @@ def lib() -> ctypes.CDLL:
         for name in ("amx_workspace_bytes", "amx_quant_gemm_workspace_bytes"):
             getattr(L, name).argtypes = [i64, i64, i64, i, u32]
             getattr(L, name).restype = sz
-        L.amx_linear_host_workspace_bytes.argtypes = [i64, i64, i64, i]
+        L.amx_linear_host_workspace_bytes.argtypes = [i64, i64, i64, i, u32]
         L.amx_linear_host_workspace_bytes.restype = sz
         L.amx_gemm_kernel_for.argtypes = [i64, i64, i64, i, u32]
         L.amx_gemm_kernel_for.restype = u32
@@ -226,21 +237,55 @@ def gemm_status(workspace: torch.Tensor) -> int:
     return int(lib().amx_gemm_status(workspace.data_ptr(), _stream()))
 
 
-def quant_gemm(a: torch.Tensor, w_codes, w_scales, group_size: int = 32, flags: int = GEMM_AUTO,
-               out: torch.Tensor | None = None, workspace: torch.Tensor | None = None):
-    """fp32 [M, N] = AMXFP4(a) x quantized W; a is bf16 [M, K]."""
+def quant_gemm(a: torch.Tensor, w_codes=None, w_scales=None, group_size: int = 32, flags: int = GEMM_AUTO,
+               out: torch.Tensor | None = None, workspace: torch.Tensor | None = None, w_bf16: torch.Tensor | None = None):
+    """fp32 [M, N] = AMXFP4(a) x W; a is bf16 [M, K]; W is either quantized (w_codes, w_scales) or bf16 [N, K]
+    (w_bf16), which the call casts too."""
     _dev(a, torch.bfloat16, "a")
     M, K = a.shape
-    N = w_codes.shape[0]
+    if w_bf16 is not None:
+        _dev(w_bf16, torch.bfloat16, "w_bf16")
+        assert w_codes is None and w_scales is None and w_bf16.stride(1) == 1
+    N = w_bf16.shape[0] if w_bf16 is not None else w_codes.shape[0]
     if out is None:
         out = torch.empty((M, N), dtype=torch.float32, device=a.device)
-    need = lib().amx_quant_gemm_workspace_bytes(M, N, K, group_size, flags & ~GEMM_CAST_IN_KERNEL)
+    need = lib().amx_quant_gemm_workspace_bytes(M, N, K, group_size, (flags & ~GEMM_CAST_IN_KERNEL) |
+                                                (WEIGHT_BF16 if w_bf16 is not None else 0))
     if workspace is None:
         workspace = _ws(need, a.device)
-    _check(lib().amx_quant_gemm(a.data_ptr(), a.stride(0), w_codes.data_ptr(), w_scales.data_ptr(), M, N, K,
+    _check(lib().amx_quant_gemm(a.data_ptr(), a.stride(0),
+                                w_codes.data_ptr() if w_codes is not None else None,
+                                w_scales.data_ptr() if w_scales is not None else None,
+                                w_bf16.data_ptr() if w_bf16 is not None else None,
+                                w_bf16.stride(0) if w_bf16 is not None else 0, M, N, K,
                                 group_size, flags, out.data_ptr(), out.stride(0), workspace.data_ptr(),
                                 workspace.numel(), _stream()), "amx_quant_gemm")
     return out
+
+
+def gemm_flushed_scales(workspace: torch.Tensor) -> int:
+    return int(lib().amx_gemm_flushed_scales(workspace.data_ptr(), _stream()))
+
+
+def prepared_flushed_scales(prepared: torch.Tensor, rows: int, K: int, is_weight: bool, group_size: int = 32) -> int:
+    return int(lib().amx_prepared_flushed_scales(prepared.data_ptr(), rows, K, group_size, int(is_weight), _stream()))
+
+
+def attention_map(q: torch.Tensor, k: torch.Tensor, flags: int = 0, want_bf16: bool = True):
+    """The cast attention map of one head as amx_attention builds it on its two-pass path.  q, k: bf16 [L, d].
+    Returns (p_bf16 or None, codes, scales, prepared)."""
+    _dev(q, torch.bfloat16, "q"), _dev(k, torch.bfloat16, "k")
+    assert q.is_contiguous() and k.is_contiguous() and q.shape == k.shape
+    Lq, d = q.shape
+    p_bits = torch.empty((Lq, Lq), dtype=torch.bfloat16, device=q.device) if want_bf16 else None
+    codes = torch.empty((Lq, Lq // 2), dtype=torch.uint8, device=q.device)
+    scales = torch.empty((Lq, Lq // 32, 2), dtype=torch.uint8, device=q.device)
+    prep = _ws(lib().amx_prepared_bytes(Lq, Lq, 32, 0), q.device)
+    ws = _ws(lib().amx_attention_workspace_bytes(Lq, d), q.device)
+    _check(lib().amx_attention_map(q.data_ptr(), k.data_ptr(), Lq, d, flags, p_bits.data_ptr() if want_bf16 else None,
+                                   codes.data_ptr(), scales.data_ptr(), prep.data_ptr(), prep.numel(), ws.data_ptr(),
+                                   ws.numel(), _stream()), "amx_attention_map")
+    return p_bits, codes, scales, prep
 
 
 def softmax_bf16(S: torch.Tensor, alpha: float, out: torch.Tensor | None = None):
@@ -272,7 +317,8 @@ def softmax_quantize(S: torch.Tensor, alpha: float, prepared_as: str | None = No
 
 def linear_host(a_host: torch.Tensor, w_host: torch.Tensor, c_host: torch.Tensor, workspace: torch.Tensor,
                 group_size: int = 32, flags: int = GEMM_AUTO):
-    """Whole layer from (pinned) host bf16 tensors a[M,K], w[N,K] into host fp32 c[M,N]; synchronises."""
+    """Whole layer from (pinned) host bf16 tensors a[M,K], w[N,K] into host fp32 c[M,N]; synchronises unless
+    flags carry HOST_NO_SYNC."""
     assert not a_host.is_cuda and not w_host.is_cuda and not c_host.is_cuda and workspace.is_cuda
     assert a_host.dtype == w_host.dtype == torch.bfloat16 and c_host.dtype == torch.float32
     M, K = a_host.shape

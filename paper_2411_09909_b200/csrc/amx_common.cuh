@@ -8,7 +8,10 @@
 
 namespace amx {
 
-inline bool valid_group_size(int gs) { return gs == 16 || gs == 32 || gs == 64 || gs == 128; }
+// Group sizes: 16, 32, 64 or 128 elements, or the whole row as one group (group_size == K, K a multiple of 8:
+// the grouping of the paper's worked example), which only the generic kernels take.
+inline bool fixed_group_size(int gs) { return gs == 16 || gs == 32 || gs == 64 || gs == 128; }
+inline bool valid_group_size(int gs, int64_t K) { return fixed_group_size(gs) || (gs > 0 && gs == K && K % 8 == 0); }
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
@@ -45,12 +48,17 @@ __device__ __forceinline__ int scale_key(uint32_t b) { return (int)(scale_norm(b
 // Per-row word of a prepared FP4-GEMM operand: bits 15..0 the row's power-of-two offset (largest exponent key
 // - 25; 0 for an all-zero row) as a signed 16-bit number, bit 16 set when some group of the row has a nonzero
 // positive-side scale, bit 17 the same for the negative side.  A tile whose rows all lack a side has an
-// all-zero plane for it, and the GEMM does not issue that plane's products.
+// all-zero plane for it, and the GEMM does not issue that plane's products.  Bits 31..18: how many nonzero
+// scales of the row did not fit the UE4M3 range under the row's offset and were flushed to zero (see
+// to_ue4m3), saturating at kRowFlushedMax.
 constexpr int kRowHasPos = 1 << 16, kRowHasNeg = 1 << 17;
-__host__ __device__ __forceinline__ int row_word(int kmax, int side_bits) {
-    return ((kmax ? kmax - 25 : 0) & 0xFFFF) | side_bits;
+constexpr int kRowFlushedShift = 18, kRowFlushedMax = 0x3FFF;
+__host__ __device__ __forceinline__ int row_word(int kmax, int side_bits, int flushed = 0) {
+    const int f = flushed > kRowFlushedMax ? kRowFlushedMax : flushed;
+    return ((kmax ? kmax - 25 : 0) & 0xFFFF) | side_bits | (int)((unsigned)f << kRowFlushedShift);
 }
 __host__ __device__ __forceinline__ int row_word_exp(int w) { return (int)(short)(w & 0xFFFF); }
+__host__ __device__ __forceinline__ int row_word_flushed(int w) { return (int)((unsigned)w >> kRowFlushedShift); }
 // side bits of a group's scale bytes {neg : pos}
 __device__ __forceinline__ int side_bits_of(uint32_t sc) {
     return ((sc & 0xFFu) ? kRowHasPos : 0) | ((sc >> 8) ? kRowHasNeg : 0);
@@ -71,6 +79,10 @@ __host__ __device__ __forceinline__ int64_t sf_group_offset(int g) { return (int
 __device__ __forceinline__ uint32_t to_ue4m3(uint32_t b, int kmax) {
     const int t = (int)scale_norm(b) + ((15 - kmax) << 2);       // (exponent field << 2) | mantissa
     return (b != 0 && t >= 4) ? (uint32_t)t << 1 : 0u;
+}
+// Whether to_ue4m3 flushes the nonzero scale byte b: its key lies 15 or more below the row's largest.
+__device__ __forceinline__ bool ue4m3_flushes(uint32_t b, int kmax) {
+    return b != 0 && (int)scale_norm(b) + ((15 - kmax) << 2) < 4;
 }
 
 }  // namespace amx

@@ -1,6 +1,7 @@
 // C-ABI entry points that combine kernels: GEMM dispatch, quantize+GEMM, the host-buffer
 // layer call, workspace sizing and status strings.
 #include <cmath>
+#include <vector>
 
 #include "gemm.cuh"
 
@@ -11,7 +12,7 @@ constexpr size_t kAlign = 256;
 inline size_t round_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 bool gemm_shape_ok(int64_t M, int64_t N, int64_t K, int gs) {
-    return valid_group_size(gs) && M >= 0 && N >= 0 && K > 0 && K % gs == 0 && K % 8 == 0;
+    return valid_group_size(gs, K) && M >= 0 && N >= 0 && K > 0 && K % gs == 0 && K % 8 == 0;
 }
 
 constexpr uint32_t kKernelMask = AMX_GEMM_SIMT | AMX_GEMM_TC | AMX_GEMM_FP4 | AMX_GEMM_ROWS;
@@ -39,9 +40,15 @@ uint32_t pick_kernel(int64_t M, int64_t N, int64_t K, int gs, uint32_t flags) {
     return tc ? AMX_GEMM_TC : AMX_GEMM_SIMT;
 }
 
-size_t kernel_workspace(uint32_t kernel, int64_t M, int64_t N, int64_t K) {
+// AMX_GEMM_AUTO on the FP4 kernel: when preparing the operands flushed a scale (see to_ue4m3), the FP4 kernel
+// returns at once and the exact bf16-decode kernel runs instead - decided on the device, from the count in the
+// workspace's second word.  That kernel's scratch follows the FP4 kernel's.
+bool auto_fallback(uint32_t flags, uint32_t kernel) { return (flags & kKernelMask) == AMX_GEMM_AUTO && kernel == AMX_GEMM_FP4; }
+
+size_t kernel_workspace(uint32_t kernel, int64_t M, int64_t N, int64_t K, bool fallback = false) {
     if (kernel == AMX_GEMM_TC) return round_up(gemm_tc_workspace_bytes(M, N, K));
-    if (kernel == AMX_GEMM_FP4) return round_up(gemm_fp4_workspace_bytes(M, N, K));
+    if (kernel == AMX_GEMM_FP4)
+        return round_up(gemm_fp4_workspace_bytes(M, N, K)) + (fallback ? round_up(gemm_tc_workspace_bytes(M, N, K)) : 0);
     if (kernel == AMX_GEMM_ROWS) return round_up(gemm_rows_workspace_bytes(M, K));
     return 0;
 }
@@ -52,6 +59,8 @@ struct QuantSizes {
 QuantSizes quant_sizes(int64_t rows, int64_t K, int gs) {
     return {round_up((size_t)rows * (size_t)(K / 2)), round_up((size_t)rows * (size_t)(K / gs) * 2)};
 }
+
+constexpr uint32_t kQuantGemmFlags = kKernelMask | AMX_GEMM_CAST_IN_KERNEL | AMX_WEIGHT_BF16;
 
 }  // namespace
 }  // namespace amx
@@ -65,19 +74,22 @@ extern "C" uint32_t amx_gemm_kernel_for(int64_t M, int64_t N, int64_t K, int gro
 
 extern "C" size_t amx_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags) {
     if (!gemm_shape_ok(M, N, K, group_size)) return 0;
-    return kernel_workspace(pick_kernel(M, N, K, group_size, flags), M, N, K);
+    const uint32_t kernel = pick_kernel(M, N, K, group_size, flags);
+    return kernel_workspace(kernel, M, N, K, auto_fallback(flags, kernel));
 }
 
 extern "C" size_t amx_quant_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags) {
     if (!gemm_shape_ok(M, N, K, group_size)) return 0;
-    const QuantSizes a = quant_sizes(M, K, group_size);
-    return amx_workspace_bytes(M, N, K, group_size, flags) + a.codes + a.scales;
+    const QuantSizes a = quant_sizes(M, K, group_size), w = quant_sizes(N, K, group_size);
+    // the first 256 bytes always hold the status word and the flushed-scale count, whichever kernel runs
+    size_t gemm_ws = amx_workspace_bytes(M, N, K, group_size, flags & kKernelMask);
+    if (gemm_ws < 256) gemm_ws = 256;
+    return gemm_ws + a.codes + a.scales + ((flags & AMX_WEIGHT_BF16) ? w.codes + w.scales : 0);
 }
 
-extern "C" size_t amx_linear_host_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size) {
+extern "C" size_t amx_linear_host_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags) {
     if (!gemm_shape_ok(M, N, K, group_size)) return 0;
-    const QuantSizes a = quant_sizes(M, K, group_size), w = quant_sizes(N, K, group_size);
-    return amx_workspace_bytes(M, N, K, group_size, AMX_GEMM_AUTO) + a.codes + a.scales + w.codes + w.scales +
+    return amx_quant_gemm_workspace_bytes(M, N, K, group_size, (flags & kKernelMask) | AMX_WEIGHT_BF16) +
            round_up((size_t)M * K * 2) + round_up((size_t)N * K * 2) + round_up((size_t)M * N * 4);
 }
 
@@ -98,12 +110,23 @@ extern "C" int amx_gemm(const uint8_t* a_codes, const uint8_t* a_scales, const u
     if (kernel == AMX_GEMM_SIMT)
         return gemm_simt(a_codes, a_scales, w_codes, w_scales, M, N, K, group_size, C, ld_c, st);
     if (!aligned(a_codes, 16) || !aligned(w_codes, 16)) return AMX_ERR_ALIGN;
-    const size_t need = kernel_workspace(kernel, M, N, K);
+    // AUTO picked the weight-streaming kernel but the weight's scales miss its alignment (4-byte asynchronous
+    // copies): the plain kernel takes any 2-byte aligned scales and needs no scratch
+    if (kernel == AMX_GEMM_ROWS && !aligned(w_scales, 4)) {
+        if ((flags & kKernelMask) == AMX_GEMM_ROWS) return AMX_ERR_ALIGN;
+        return gemm_simt(a_codes, a_scales, w_codes, w_scales, M, N, K, group_size, C, ld_c, st);
+    }
+    const bool fallback = auto_fallback(flags, kernel);
+    const size_t need = kernel_workspace(kernel, M, N, K, fallback);
     if (need && (!workspace || workspace_bytes < need)) return AMX_ERR_WORKSPACE;
     if (need && !aligned(workspace, kAlign)) return AMX_ERR_ALIGN;
-    if (kernel == AMX_GEMM_FP4)
-        return gemm_fp4(a_codes, a_scales, w_codes, w_scales, M, N, K, C, ld_c, workspace, st);
-    if (kernel == AMX_GEMM_ROWS && !aligned(w_scales, 4)) return AMX_ERR_ALIGN;   // 4-byte asynchronous copies
+    if (kernel == AMX_GEMM_FP4) {
+        int rc = gemm_fp4(a_codes, a_scales, w_codes, w_scales, M, N, K, C, ld_c, workspace, st, fallback);
+        if (rc != AMX_OK || !fallback) return rc;
+        int* words = static_cast<int*>(workspace);       // [0] status, [1] flushed scales
+        return gemm_tc(a_codes, a_scales, w_codes, w_scales, M, N, K, C, ld_c,
+                       static_cast<uint8_t*>(workspace) + round_up(gemm_fp4_workspace_bytes(M, N, K)), st, words + 1, words);
+    }
     if (kernel == AMX_GEMM_ROWS)
         return gemm_rows(a_codes, a_scales, w_codes, w_scales, M, N, K, C, ld_c, workspace, st);
     return gemm_tc(a_codes, a_scales, w_codes, w_scales, M, N, K, C, ld_c, workspace, st);
@@ -160,89 +183,118 @@ extern "C" int amx_gemm_prepared(const void* a_prepared, const void* w_prepared,
 }
 
 extern "C" int amx_quant_gemm(const void* A, int64_t ld_a, const uint8_t* w_codes, const uint8_t* w_scales,
-                              int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags, float* C,
-                              int64_t ld_c, void* workspace, size_t workspace_bytes, void* stream) {
+                              const void* W_bf16, int64_t ld_w, int64_t M, int64_t N, int64_t K, int group_size,
+                              uint32_t flags, float* C, int64_t ld_c, void* workspace, size_t workspace_bytes,
+                              void* stream) {
+    if (flags & ~kQuantGemmFlags) return AMX_ERR_FLAGS;
     const bool cast_in_kernel = flags & AMX_GEMM_CAST_IN_KERNEL;
-    if (cast_in_kernel && (flags & kKernelMask) != AMX_GEMM_TC) return AMX_ERR_FLAGS;
-    flags &= ~AMX_GEMM_CAST_IN_KERNEL;
-    if (flags & ~kKernelMask) return AMX_ERR_FLAGS;
-    if (!gemm_shape_ok(M, N, K, group_size) || ld_a < K || ld_c < N) return AMX_ERR_SHAPE;
+    const bool w_is_bf16 = W_bf16 != nullptr;
+    flags &= kKernelMask;
+    if (cast_in_kernel && flags != AMX_GEMM_TC) return AMX_ERR_FLAGS;
+    if (!gemm_shape_ok(M, N, K, group_size) || ld_a < K || ld_c < N || (w_is_bf16 && ld_w < K)) return AMX_ERR_SHAPE;
+    const uint32_t kernel = pick_kernel(M, N, K, group_size, flags);
+    if (!kernel) return (flags & (flags - 1)) ? AMX_ERR_FLAGS : AMX_ERR_SHAPE;
     if (M == 0 || N == 0) return AMX_OK;
-    const size_t need = amx_quant_gemm_workspace_bytes(M, N, K, group_size, flags);
+    // exactly one form of the weight
+    if (!A || !C || (w_is_bf16 ? (w_codes || w_scales) : (!w_codes || !w_scales))) return AMX_ERR_NULL;
+    const size_t need = amx_quant_gemm_workspace_bytes(M, N, K, group_size, flags | (w_is_bf16 ? AMX_WEIGHT_BF16 : 0));
     if (!workspace || workspace_bytes < need) return AMX_ERR_WORKSPACE;
-    if (!aligned(workspace, kAlign)) return AMX_ERR_ALIGN;
-    const size_t gemm_ws = amx_workspace_bytes(M, N, K, group_size, flags);
-    const QuantSizes a = quant_sizes(M, K, group_size);
+    const int code_align = kernel == AMX_GEMM_SIMT ? 4 : 16;
+    if (!aligned(workspace, kAlign) || !aligned(A, 16) || ld_a % 8 || !aligned(C, 4) ||
+        (w_is_bf16 ? (!aligned(W_bf16, 16) || ld_w % 8) : (!aligned(w_codes, code_align) || !aligned(w_scales, 2))))
+        return AMX_ERR_ALIGN;
+    if (kernel == AMX_GEMM_ROWS && !w_is_bf16 && !aligned(w_scales, 4)) return AMX_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool fallback = auto_fallback(flags, kernel);
+    size_t gemm_ws = kernel_workspace(kernel, M, N, K, fallback);
+    if (gemm_ws < 256) gemm_ws = 256;                       // the plain kernel has no scratch of its own: header only
+    const QuantSizes a = quant_sizes(M, K, group_size), w = quant_sizes(N, K, group_size);
     uint8_t* base = static_cast<uint8_t*>(workspace);
-    if (cast_in_kernel) {
-        // one launch: the kernel's producers cast the activation tile in registers (same arithmetic as
-        // amx_quantize, so the result is bit-identical to the two-call sequence)
-        if (!gemm_tc_supported(M, N, K, group_size)) return AMX_ERR_SHAPE;
-        if (!A || !w_codes || !w_scales || !C) return AMX_ERR_NULL;
-        if (!aligned(A, 16) || ld_a % 8 || !aligned(w_codes, 16) || !aligned(w_scales, 2) || !aligned(C, 4))
-            return AMX_ERR_ALIGN;
-        return gemm_tc_cast(A, ld_a, w_codes, w_scales, M, N, K, C, ld_c, base, static_cast<cudaStream_t>(stream));
-    }
+    if (kernel == AMX_GEMM_SIMT && cudaMemsetAsync(base, 0, 8, st) != cudaSuccess) return AMX_ERR_CUDA;
     uint8_t* a_codes = base + gemm_ws;
     uint8_t* a_scales = a_codes + a.codes;
-    if (pick_kernel(M, N, K, group_size, flags) == AMX_GEMM_ROWS) {
-        // the cast of the few rows writes the decoded operand of the weight-streaming kernel directly: two launches
-        if (!A || !w_codes || !w_scales || !C) return AMX_ERR_NULL;
-        if (!aligned(A, 16) || ld_a % 8 || !aligned(w_codes, 16) || !aligned(w_scales, 4) || !aligned(C, 4))
-            return AMX_ERR_ALIGN;
-        return gemm_rows_cast(A, ld_a, w_codes, w_scales, M, N, K, C, ld_c, base, static_cast<cudaStream_t>(stream));
-    }
-    if (pick_kernel(M, N, K, group_size, flags) == AMX_GEMM_FP4 && ld_a == K) {
-        // the activation's cast writes the kernel's operand itself (one launch less, the codes are not re-read);
-        // same workspace layout as amx_gemm's: status word, prepared A, prepared W
-        if (!A || !w_codes || !w_scales || !C) return AMX_ERR_NULL;
-        if (!aligned(A, 16) || !aligned(w_codes, 16) || !aligned(w_scales, 2) || !aligned(C, 4)) return AMX_ERR_ALIGN;
-        cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t* wq_codes = a_scales + a.scales;               // only with a bf16 weight
+    uint8_t* wq_scales = wq_codes + w.codes;
+    int rc = AMX_OK;
+    if (kernel == AMX_GEMM_FP4) {
+        // Both casts write the kernel's operands themselves where the rows are contiguous (one launch per operand,
+        // the codes are not read again); workspace: status word and flushed-scale count, prepared A, prepared W
         uint8_t* pa = base + 256;
         uint8_t* pw = pa + gemm_fp4_prepared_bytes(M, K, false);
-        int rc = gemm_fp4_quantize_prepared(A, M, K, false, a_codes, a_scales, pa, st);
-        if (rc == AMX_OK) rc = gemm_fp4_prepare(w_codes, w_scales, N, K, true, pw, st);
+        int* words = reinterpret_cast<int*>(base);
+        if (cudaMemsetAsync(words, 0, 8, st) != cudaSuccess) return AMX_ERR_CUDA;
+        if (ld_a == K) rc = gemm_fp4_quantize_prepared(A, M, K, false, a_codes, a_scales, pa, st, 0, AMX_FMT_AMXFP4, words + 1);
+        else {
+            rc = amx_quantize(A, M, K, ld_a, group_size, a_codes, a_scales, stream);
+            if (rc == AMX_OK) rc = gemm_fp4_prepare(a_codes, a_scales, M, K, false, pa, st, 0, words + 1);
+        }
         if (rc != AMX_OK) return rc;
-        return gemm_fp4_prepared(pa, pw, M, N, K, C, ld_c, base, st);
+        if (w_is_bf16 && ld_w == K)
+            rc = gemm_fp4_quantize_prepared(W_bf16, N, K, true, wq_codes, wq_scales, pw, st, 0, AMX_FMT_AMXFP4, words + 1);
+        else {
+            if (w_is_bf16) rc = amx_quantize(W_bf16, N, K, ld_w, group_size, wq_codes, wq_scales, stream);
+            if (rc == AMX_OK)
+                rc = gemm_fp4_prepare(w_is_bf16 ? wq_codes : w_codes, w_is_bf16 ? wq_scales : w_scales, N, K, true, pw, st, 0,
+                                      words + 1);
+        }
+        if (rc != AMX_OK) return rc;
+        rc = gemm_fp4_prepared(pa, pw, M, N, K, C, ld_c, base, st, 256, fallback ? words + 1 : nullptr);
+        if (rc != AMX_OK || !fallback) return rc;
+        return gemm_tc(a_codes, a_scales, w_is_bf16 ? wq_codes : w_codes, w_is_bf16 ? wq_scales : w_scales, M, N, K, C, ld_c,
+                       base + round_up(gemm_fp4_workspace_bytes(M, N, K)), st, words + 1, words);
     }
-    int rc = amx_quantize(A, M, K, ld_a, group_size, a_codes, a_scales, stream);
+    if (w_is_bf16) {
+        rc = amx_quantize(W_bf16, N, K, ld_w, group_size, wq_codes, wq_scales, stream);
+        if (rc != AMX_OK) return rc;
+        w_codes = wq_codes;
+        w_scales = wq_scales;
+    }
+    if (cast_in_kernel)
+        // one launch: the kernel's producers cast the activation tile in registers (same arithmetic as
+        // amx_quantize, so the result is bit-identical to the two-call sequence)
+        return gemm_tc_cast(A, ld_a, w_codes, w_scales, M, N, K, C, ld_c, base, st);
+    if (kernel == AMX_GEMM_ROWS)
+        // the cast of the few rows writes the decoded operand of the weight-streaming kernel directly: two launches
+        return gemm_rows_cast(A, ld_a, w_codes, w_scales, M, N, K, C, ld_c, base, st);
+    rc = amx_quantize(A, M, K, ld_a, group_size, a_codes, a_scales, stream);
     if (rc != AMX_OK) return rc;
-    return amx_gemm(a_codes, a_scales, w_codes, w_scales, M, N, K, group_size, flags, C, ld_c, base, gemm_ws, stream);
+    return amx_gemm(a_codes, a_scales, w_codes, w_scales, M, N, K, group_size, kernel, C, ld_c, base, gemm_ws, stream);
 }
 
 extern "C" int amx_linear_host(const void* A_host, const void* W_host, int64_t M, int64_t N, int64_t K,
                                int group_size, uint32_t flags, float* C_host, void* workspace,
                                size_t workspace_bytes, void* stream) {
+    const bool no_sync = flags & AMX_HOST_NO_SYNC;
+    flags &= ~AMX_HOST_NO_SYNC;
     if (flags & ~kKernelMask) return AMX_ERR_FLAGS;
     if (!gemm_shape_ok(M, N, K, group_size)) return AMX_ERR_SHAPE;
+    if (!pick_kernel(M, N, K, group_size, flags)) return (flags & (flags - 1)) ? AMX_ERR_FLAGS : AMX_ERR_SHAPE;
     if (M == 0 || N == 0) return AMX_OK;
     if (!A_host || !W_host || !C_host) return AMX_ERR_NULL;
-    const size_t need = amx_linear_host_workspace_bytes(M, N, K, group_size);
+    const size_t need = amx_linear_host_workspace_bytes(M, N, K, group_size, flags);
     if (!workspace || workspace_bytes < need) return AMX_ERR_WORKSPACE;
     if (!aligned(workspace, kAlign)) return AMX_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const size_t gemm_ws = amx_workspace_bytes(M, N, K, group_size, AMX_GEMM_AUTO);
-    const QuantSizes a = quant_sizes(M, K, group_size), w = quant_sizes(N, K, group_size);
+    // everything is validated: from here on only a failing CUDA call can stop the sequence
+    const size_t qg_ws = amx_quant_gemm_workspace_bytes(M, N, K, group_size, flags | AMX_WEIGHT_BF16);
     uint8_t* p = static_cast<uint8_t*>(workspace);
-    uint8_t* gemm_base = p;            p += gemm_ws;
-    uint8_t* a_codes = p;              p += a.codes;
-    uint8_t* a_scales = p;             p += a.scales;
-    uint8_t* w_codes = p;              p += w.codes;
-    uint8_t* w_scales = p;             p += w.scales;
+    uint8_t* qg_base = p;              p += qg_ws;
     uint8_t* a_dev = p;                p += round_up((size_t)M * K * 2);
     uint8_t* w_dev = p;                p += round_up((size_t)N * K * 2);
     float* c_dev = reinterpret_cast<float*>(p);
     if (cudaMemcpyAsync(a_dev, A_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(w_dev, W_host, (size_t)N * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        cudaMemcpyAsync(w_dev, W_host, (size_t)N * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        cudaGetLastError();
         return AMX_ERR_CUDA;
-    int rc = amx_quantize(a_dev, M, K, K, group_size, a_codes, a_scales, stream);
-    if (rc == AMX_OK) rc = amx_quantize(w_dev, N, K, K, group_size, w_codes, w_scales, stream);
-    if (rc == AMX_OK)
-        rc = amx_gemm(a_codes, a_scales, w_codes, w_scales, M, N, K, group_size, flags, c_dev, N, gemm_base,
-                      gemm_ws, stream);
+    }
+    const int rc = amx_quant_gemm(a_dev, K, nullptr, nullptr, w_dev, K, M, N, K, group_size, flags, c_dev, N, qg_base, qg_ws,
+                                  stream);
     if (rc != AMX_OK) return rc;
-    if (cudaMemcpyAsync(C_host, c_dev, (size_t)M * N * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    if (cudaMemcpyAsync(C_host, c_dev, (size_t)M * N * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
+        cudaGetLastError();
         return AMX_ERR_CUDA;
+    }
+    if (no_sync) return AMX_OK;
     return cudaStreamSynchronize(st) == cudaSuccess ? AMX_OK : AMX_ERR_CUDA;
 }
 
@@ -357,7 +409,7 @@ extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_
             const int nb = pair && i + 1 < hc ? 2 : 1;
             for (int j = 0; j < nb && rc == AMX_OK; ++j)
                 rc = gemm_fp4_attn_scores({w + a.pq, hc * L, chunk * L, (i + j) * L}, {w + a.pk, hc * L, chunk * L + 128, (i + j) * L},
-                                          L, d, alpha, S, w + a.pc, w + a.ps, p_prep, w + a.gemm, st, causal, p_rows, j * L);
+                                          L, d, alpha, S, nullptr, nullptr, p_prep, w + a.gemm, st, causal, p_rows, j * L);
             if (rc == AMX_OK)
                 rc = gemm_fp4_prepared_at({p_prep, nb * L, p_rows, 0, /*single_plane=*/true}, {w + a.pv, hc * d, chunk * d + 128, i * d},
                                           nb * L, d, L, o + (size_t)(h0 + i) * L * d, d, w + a.gemm, st, 256, causal, nb, d);
@@ -392,8 +444,68 @@ extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_
     return AMX_OK;
 }
 
+extern "C" int amx_attention_map(const void* q, const void* k, int64_t L, int64_t d, uint32_t flags, void* p_bf16,
+                                 uint8_t* p_codes, uint8_t* p_scales, void* p_prepared, size_t prepared_bytes,
+                                 void* workspace, size_t workspace_bytes, void* stream) {
+    const int causal = (flags & AMX_ATTN_CAUSAL) ? 1 : 0;
+    if (flags & ~AMX_ATTN_CAUSAL) return AMX_ERR_FLAGS;
+    if (L <= 0 || d <= 0 || L % 256 || d % 32 || !gemm_fp4_supported(L, L, d, 32) ||
+        gemm_fp4_attn_scratch_bytes(L) > (size_t)L * L * 4)
+        return AMX_ERR_SHAPE;
+    if (!q || !k || !p_prepared) return AMX_ERR_NULL;
+    const AttnLayout a = attn_layout(L, d);
+    if (!workspace || workspace_bytes < a.total || prepared_bytes < amx_prepared_bytes(L, L, 32, 0)) return AMX_ERR_WORKSPACE;
+    if (!aligned(workspace, kAlign) || !aligned(q, 16) || !aligned(k, 16) || !aligned(p_prepared, kAlign) ||
+        !aligned(p_bf16, 16) || !aligned(p_codes, 16) || !aligned(p_scales, 2))
+        return AMX_ERR_ALIGN;
+    uint8_t* w = static_cast<uint8_t*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (causal) {
+        // blocks of keys that lie entirely after their queries are never visited: their entries are +0
+        if ((p_bf16 && cudaMemsetAsync(p_bf16, 0, (size_t)L * L * 2, st) != cudaSuccess) ||
+            (p_codes && cudaMemsetAsync(p_codes, 0, (size_t)L * L / 2, st) != cudaSuccess) ||
+            (p_scales && cudaMemsetAsync(p_scales, 0, (size_t)L * (L / 32) * 2, st) != cudaSuccess))
+            return AMX_ERR_CUDA;
+    }
+    int rc = gemm_fp4_quantize_prepared(q, L, d, false, w + a.qc, w + a.qs, w + a.pq, st);
+    if (rc == AMX_OK) rc = gemm_fp4_quantize_prepared(k, L, d, true, w + a.kc, w + a.ks, w + a.pk, st);
+    if (rc != AMX_OK) return rc;
+    return gemm_fp4_attn_scores({w + a.pq, L, L, 0}, {w + a.pk, L, L, 0}, L, d, 1.0f / sqrtf((float)d), w + a.S, p_codes,
+                                p_scales, p_prepared, w + a.gemm, st, causal, L, 0, p_bf16);
+}
+
 extern "C" int amx_gemm_status(const void* workspace, void* stream) {
     return gemm_tc_status(workspace, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int64_t amx_gemm_flushed_scales(const void* workspace, void* stream) {
+    if (!workspace) return AMX_ERR_NULL;
+    int v = 0;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(&v, static_cast<const int*>(workspace) + 1, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return AMX_ERR_CUDA;
+    }
+    return v;
+}
+
+extern "C" int64_t amx_prepared_flushed_scales(const void* prepared, int64_t rows, int64_t K, int group_size, int is_weight,
+                                               void* stream) {
+    if (rows <= 0 || !gemm_fp4_supported(rows, rows, K, group_size)) return AMX_ERR_SHAPE;
+    if (!prepared) return AMX_ERR_NULL;
+    // diagnostic, off the hot path: the per-row counts sit in the operand's row words; they are summed on the host
+    std::vector<int> words((size_t)rows);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(words.data(), gemm_fp4_row_words(prepared, rows, K, is_weight != 0), (size_t)rows * sizeof(int),
+                        cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return AMX_ERR_CUDA;
+    }
+    int64_t total = 0;
+    for (int w : words) total += row_word_flushed(w);
+    return total;
 }
 
 extern "C" const char* amx_status_string(int status) {

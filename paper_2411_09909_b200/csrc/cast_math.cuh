@@ -175,8 +175,10 @@ __device__ __forceinline__ uint32_t emit_group(const uint32_t (&w)[16], int64_t 
 
 // The same for a group without negative elements (a softmax output) when only the FP4 GEMM's operand is wanted:
 // its positive sign plane is its code word, the negative plane and scale are zero.  Same arithmetic as above,
-// minus everything the negative side needs.  Stores the plane at group index v, returns the positive scale byte.
-__device__ __forceinline__ uint32_t emit_nonneg_plane(const uint32_t (&w)[16], int64_t v, uint4* __restrict__ plane) {
+// minus everything the negative side needs.  Stores the plane at group index v (and, when asked, the same word as
+// the group's canonical codes: without a set sign bit the two are equal), returns the positive scale byte.
+__device__ __forceinline__ uint32_t emit_nonneg_plane(const uint32_t (&w)[16], int64_t v, uint4* __restrict__ plane,
+                                                      uint4* __restrict__ codes = nullptr) {
     uint32_t pm = w[0];
 #pragma unroll
     for (int i = 1; i + 1 < 16; i += 2) pm = __vimax3_s16x2(pm, w[i], w[i + 1]);
@@ -196,6 +198,7 @@ __device__ __forceinline__ uint32_t emit_nonneg_plane(const uint32_t (&w)[16], i
         nib[j] = cvt_e2m1x8(r);
     }
     plane[v] = make_uint4(nib[0], nib[1], nib[2], nib[3]);
+    if (codes) codes[v] = make_uint4(nib[0], nib[1], nib[2], nib[3]);
     return sc;
 }
 

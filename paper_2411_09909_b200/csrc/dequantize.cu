@@ -46,7 +46,7 @@ dequantize_kernel(const uint32_t* __restrict__ codes, const uint16_t* __restrict
 extern "C" int amx_dequantize(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K,
                               int group_size, uint32_t flags, void* out, int64_t ld_out, void* stream) {
     using namespace amx;
-    if (!valid_group_size(group_size) || rows < 0 || K <= 0 || K % group_size || K % 8 || ld_out < K)
+    if (!valid_group_size(group_size, K) || rows < 0 || K <= 0 || K % group_size || K % 8 || ld_out < K)
         return AMX_ERR_SHAPE;
     if (flags & ~AMX_OUT_F32) return AMX_ERR_FLAGS;
     if (rows == 0) return AMX_OK;

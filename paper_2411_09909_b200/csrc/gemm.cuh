@@ -12,9 +12,11 @@ int gemm_simt(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_
 // Tensor-core (tcgen05) kernel: shapes it accepts, scratch it needs, launcher.
 bool gemm_tc_supported(int64_t M, int64_t N, int64_t K, int gs);
 size_t gemm_tc_workspace_bytes(int64_t M, int64_t N, int64_t K);
+// run_if_nonzero (optional, device word): the launch does nothing when that word is zero.  status_word
+// (optional): a status word the caller has cleared, used instead of the workspace's first word.
 int gemm_tc(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes,
             const uint8_t* w_scales, int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c,
-            void* workspace, cudaStream_t st);
+            void* workspace, cudaStream_t st, const int* run_if_nonzero = nullptr, int* status_word = nullptr);
 // The same product with the cast of the bf16 activation X [M, ld_a] done inside the kernel.
 int gemm_tc_cast(const void* x, int64_t ld_a, const uint8_t* w_codes, const uint8_t* w_scales, int64_t M,
                  int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st);
@@ -35,17 +37,20 @@ bool gemm_fp4_supported(int64_t M, int64_t N, int64_t K, int gs);
 size_t gemm_fp4_workspace_bytes(int64_t M, int64_t N, int64_t K);
 int gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes,
              const uint8_t* w_scales, int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c,
-             void* workspace, cudaStream_t st);
+             void* workspace, cudaStream_t st, bool gate_on_flushed = false);
 // The same in two phases, so that an operand (typically the weight) is prepared once and reused.
 size_t gemm_fp4_prepared_bytes(int64_t rows, int64_t K, bool is_weight);
+// flushed_total (optional, device): incremented by the number of nonzero scales that fell below the UE4M3 range
+// of their row and were flushed; the per-row counts are in the row words either way.
 int gemm_fp4_prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, bool is_weight,
-                     void* prepared, cudaStream_t st, int64_t layout_rows = 0 /* 0: rows */);
+                     void* prepared, cudaStream_t st, int64_t layout_rows = 0 /* 0: rows */, int* flushed_total = nullptr);
 int gemm_fp4_quantize_prepared(const void* x, int64_t rows, int64_t K, bool is_weight, uint8_t* codes,
                                uint8_t* scales, void* prepared, cudaStream_t st, int64_t layout_rows = 0,
-                               int format = AMX_FMT_AMXFP4);
+                               int format = AMX_FMT_AMXFP4, int* flushed_total = nullptr);
 int quantize_rows_prepared(const void* x, int64_t rows, int64_t K, uint8_t* codes, uint8_t* scales, void* pos,
                            void* neg, uint8_t* sf_pos, uint8_t* sf_neg, int* row_exp, int nk64, int64_t padded_rows,
-                           cudaStream_t st, int format = AMX_FMT_AMXFP4);
+                           cudaStream_t st, int format = AMX_FMT_AMXFP4, int* flushed_total = nullptr);
+const int* gemm_fp4_row_words(const void* prepared, int64_t rows, int64_t K, bool is_weight);
 // Softmax of the rows of S, rounded to bf16 and cast in one launch (cols % 32 == 0); pos == nullptr: canonical
 // output only.  gemm_fp4_softmax_prepared lays the prepared operand out like gemm_fp4_quantize_prepared.
 int softmax_cast_rows(const float* S, int64_t rows, int64_t cols, int64_t ld_s, float alpha, uint8_t* codes,
@@ -66,21 +71,25 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
                          int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes = 256,
                          int causal_pv = 0 /* 1: the product P V of causal attention (A = P, square) */,
                          int batch = 1 /* > 1 (N <= 128): a stack of `batch` independent products of M / batch rows */,
-                         int64_t w_batch_rows = 0 /* rows between their right-hand operands in the stacked W */);
+                         int64_t w_batch_rows = 0 /* rows between their right-hand operands in the stacked W */,
+                         const int* gate = nullptr /* device word: the kernel does nothing when it is nonzero */);
 // workspace that lets the kernel cut K into ranges for products with few output tiles (256 bytes otherwise)
 size_t gemm_fp4_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K);
 // C[m][n] = sum over `slices` partial products [slices][M][N], in slice order (defined with the bf16-decode kernel)
-int reduce_slices(const float* part, int slices, int64_t M, int64_t N, float* C, int64_t ld_c, cudaStream_t st);
+int reduce_slices(const float* part, int slices, int64_t M, int64_t N, float* C, int64_t ld_c, cudaStream_t st,
+                  const int* run_if_nonzero = nullptr);
 // P = softmax(alpha * Q K^T) cast to AMXFP4 (canonical + prepared left-hand operand) without the logits in
 // memory; L % 256 == 0; scratch of gemm_fp4_attn_scratch_bytes(L) bytes.
 size_t gemm_fp4_attn_scratch_bytes(int64_t L);
 int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, int64_t d, float alpha, void* scratch,
                          uint8_t* p_codes, uint8_t* p_scales, void* p_prepared, void* workspace, cudaStream_t st,
-                         int causal = 0, int64_t p_layout_rows = 0 /* 0: L */, int64_t p_row0 = 0);
+                         int causal = 0, int64_t p_layout_rows = 0 /* 0: L */, int64_t p_row0 = 0,
+                         void* p_bits = nullptr /* optional out: the bf16 map the cast started from, [L, L] */);
+// p_codes / p_scales may be NULL as well: only the prepared operand is written then.
 int quantize_cols_batched(const void* x, int64_t batch, int64_t R, int64_t C, uint8_t* codes, uint8_t* scales,
                           cudaStream_t st);
 int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
                       float* C, int64_t ld_c, void* workspace /* 256 B: status word */, cudaStream_t st,
-                      size_t workspace_bytes = 256);
+                      size_t workspace_bytes = 256, const int* gate = nullptr);
 
 }  // namespace amx

@@ -104,7 +104,7 @@ constexpr int kPrepRows = 8;
 __global__ void __launch_bounds__(256)
 prepare_operand_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales, int64_t R, int64_t K,
                        int nk64, uint4* __restrict__ pos, uint4* __restrict__ neg, uint8_t* __restrict__ sf_pos,
-                       uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp) {
+                       uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp, int* __restrict__ flushed_total) {
     __shared__ int kmax_s[kPrepRows];
     __shared__ int unsplit_s[kPrepRows];
     const int64_t row0 = (int64_t)blockIdx.x * kPrepRows, G = K / 32;
@@ -129,10 +129,21 @@ prepare_operand_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restr
         // code x scale_side = code x scale.  Its signed codes go to the positive plane as they are.
         const bool unsplit = !differ;
         if (unsplit) sides &= kRowHasPos;
+        // nonzero scales that the row's offset pushes below the UE4M3 range (they are flushed in step 3)
+        int flushed = 0;
+        if (row < R) {
+            const unsigned short* s2 = reinterpret_cast<const unsigned short*>(scales + row * G * 2);
+            for (int64_t g = lane; g < G; g += 32) {
+                const uint32_t v = __ldg(s2 + g);
+                flushed += (int)ue4m3_flushes(v & 0xFF, kmax) + (int)(!unsplit && ue4m3_flushes(v >> 8, kmax));
+            }
+        }
+        flushed = __reduce_add_sync(0xFFFFFFFFu, flushed);
         if (lane == 0) {
             kmax_s[r] = kmax;
             unsplit_s[r] = unsplit;
-            if (row < R) row_exp[row] = row_word(kmax, sides);
+            if (row < R) row_exp[row] = row_word(kmax, sides, flushed);
+            if (flushed && flushed_total) atomicAdd(flushed_total, flushed);
         }
     }
     // sign planes of this block's rows (contiguous in memory: rows are K/2 bytes apart)
@@ -207,12 +218,18 @@ struct Params {
     int slices;                  // SLICED instantiation: K is cut into this many ranges, each (tile, range) a work item
     int64_t slice_stride;        //   whose partial product goes to C + range * slice_stride
     int* status;
+    const int* gate;             // not NULL: the kernel returns at once when this word is nonzero (the caller then
+                                 // runs the exact bf16-decode kernel on the same operands, gated the other way)
     // attention epilogues (kEpiStats, kEpiCast): the tile holds logits S = Q K^T; `alpha` scales them
     float alpha;
     float2* part;            // kEpiStats out: per row and half tile {max, sum of exp} of alpha * S, [M][2 * n_tiles]
     const float2* rowstat;   // kEpiCast in: per row {-max * log2(e), 1 / sum}
     const int* p_kmax;       // kEpiCast in: per row the largest exponent key of the row's scales
-    uint4 *p_codes, *p_pos;  // kEpiCast out: canonical codes of P = softmax(alpha * S) and its positive plane
+    uint4* p_pos;            // kEpiCast out: the positive plane of P = softmax(alpha * S), cast to AMXFP4
+    // kEpiCast, optional outputs (NULL in the attention call itself; amx_attention_map asks for them so that the
+    // cast done in this epilogue can be compared with a reference): the bf16 words the cast started from
+    // [M][N / 2 words], the canonical codes [M][N / 32 groups] and scale bytes {0 : positive scale} per group
+    uint4 *p_bits, *p_codes;
     uint16_t* p_scales;
     uint8_t* p_sf;           // scale factors of the positive plane (P has no negative element)
     int p_nk64;
@@ -241,6 +258,7 @@ template <int BK_, int EPI = kEpiStore, bool SLICED = false, bool CAUSAL = false
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w, const Params p) {
     using C_ = Cfg<BK_>;
+    if (p.gate && *p.gate != 0) return;                          // uniform over the grid: nothing was set up yet
     constexpr int BNT = NHALF ? BN / 2 : BN;                     // tile width
     static_assert(!NHALF || EPI == kEpiStore, "half-width tiles: plain epilogue only");
     constexpr int kOffWnT = NHALF ? C_::kOffWp + C_::kTileB / 2 : C_::kOffWn;   // the box packs its two planes
@@ -635,8 +653,15 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                             }
                             if (m < p.M) {
                                 const int64_t g = g0 + gi;
-                                const uint32_t up = to_ue4m3(cast::emit_nonneg_plane(w, m * G + g, p.p_pos), kmax);
+                                const uint32_t sc = cast::emit_nonneg_plane(w, m * G + g, p.p_pos, p.p_codes);
+                                const uint32_t up = to_ue4m3(sc, kmax);
                                 *reinterpret_cast<uint16_t*>(p.p_sf + sf_row + sf_group_offset((int)g)) = (uint16_t)(up | (up << 8));
+                                if (p.p_scales) p.p_scales[m * G + g] = (uint16_t)sc;
+                                if (p.p_bits) {
+#pragma unroll
+                                    for (int j = 0; j < 4; ++j)
+                                        p.p_bits[(m * G + g) * 4 + j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                                }
                             }
                         }
                     }
@@ -711,11 +736,12 @@ OperandLayout operand_layout(int64_t rows, int64_t K, int rows_per_tile) {
 }
 
 int prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, const OperandLayout& o,
-            uint8_t* base, cudaStream_t st) {
+            uint8_t* base, cudaStream_t st, int* flushed_total = nullptr) {
     const int64_t padded_rows = o.row_blocks * 128;
     prepare_operand_kernel<<<(unsigned)(padded_rows / kPrepRows), 256, 0, st>>>(
         codes, scales, rows, K, o.nk64, reinterpret_cast<uint4*>(base), reinterpret_cast<uint4*>(base + o.plane),
-        base + 2 * o.plane, base + 2 * o.plane + o.sf, reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf));
+        base + 2 * o.plane, base + 2 * o.plane + o.sf, reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf),
+        flushed_total);
     return launch_status();
 }
 
@@ -849,7 +875,7 @@ size_t gemm_fp4_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 // workspace_bytes >= gemm_fp4_prepared_workspace_bytes() enables the K ranges; 256 bytes always suffice.
 int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
                          int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes, int causal_pv, int batch,
-                         int64_t w_batch_rows) {
+                         int64_t w_batch_rows, const int* gate) {
     if (batch > 1 && (N > BN / 2 || M % batch || (M / batch) % BM || w_batch_rows % 128)) return AMX_ERR_SHAPE;
     Params p;
     OperandLayout oa, ow;
@@ -858,6 +884,7 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
     if (rc != AMX_OK) return rc;
     p.causal = causal_pv ? 2 : 0;
     p.a_single = a.single_plane ? 1 : 0;
+    p.gate = gate;
     const uint8_t* pa = static_cast<const uint8_t*>(a.prepared);
     const uint8_t* pw = static_cast<const uint8_t*>(w.prepared);
     const int slices = batch > 1 ? 1 : gemm_fp4_slices(M, N, K);
@@ -870,7 +897,7 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
     if (causal_pv)
         return half ? launch_fp4<128, kEpiStore, false, true, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st)
                     : launch_fp4<128, kEpiStore, false, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
-    if (slices > 1 && fp4_block_k() == 128 && workspace_bytes >= gemm_fp4_prepared_workspace_bytes(M, N, K)) {
+    if (!gate && slices > 1 && fp4_block_k() == 128 && workspace_bytes >= gemm_fp4_prepared_workspace_bytes(M, N, K)) {
         float* part = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 256);
         p.C = part;
         p.ld_c = N;
@@ -894,7 +921,7 @@ size_t gemm_fp4_attn_scratch_bytes(int64_t L) {
 }
 int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, int64_t d, float alpha, void* scratch,
                          uint8_t* p_codes, uint8_t* p_scales, void* p_prepared, void* workspace, cudaStream_t st,
-                         int causal, int64_t p_layout_rows, int64_t p_row0) {
+                         int causal, int64_t p_layout_rows, int64_t p_row0, void* p_bits) {
     if (p_layout_rows == 0) p_layout_rows = L;
     if (p_row0 % 128 || p_row0 + L > p_layout_rows) return AMX_ERR_SHAPE;
     if (L % BN) return AMX_ERR_SHAPE;
@@ -920,8 +947,9 @@ int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, in
     p.part = part;
     p.rowstat = rowstat;
     p.p_kmax = p_kmax;
-    p.p_codes = reinterpret_cast<uint4*>(p_codes);      // not written: the prepared operand is all P V needs
+    p.p_codes = reinterpret_cast<uint4*>(p_codes);      // optional: the prepared operand is all P V needs
     p.p_scales = reinterpret_cast<uint16_t*>(p_scales);
+    p.p_bits = reinterpret_cast<uint4*>(p_bits);
     p.p_pos = reinterpret_cast<uint4*>(p_plane);
     p.p_sf = p_sf;
     p.p_nk64 = op.nk64;
@@ -936,9 +964,9 @@ int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, in
 }
 
 int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K, float* C,
-                      int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes) {
+                      int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes, const int* gate) {
     return gemm_fp4_prepared_at({a_prepared, M, M, 0}, {w_prepared, N, N, 0}, M, N, K, C, ld_c, workspace, st,
-                                workspace_bytes, 0);
+                                workspace_bytes, 0, 1, 0, gate);
 }
 
 // Size of a prepared operand: as the A operand (rows padded to 128) or the W operand (rows padded to 256).
@@ -948,12 +976,18 @@ size_t gemm_fp4_prepared_bytes(int64_t rows, int64_t K, bool is_weight) {
 
 // Fused form: one launch of the cast kernel writes the canonical operand and the prepared one.
 int gemm_fp4_quantize_prepared(const void* x, int64_t rows, int64_t K, bool is_weight, uint8_t* codes, uint8_t* scales,
-                               void* prepared, cudaStream_t st, int64_t layout_rows, int format) {
+                               void* prepared, cudaStream_t st, int64_t layout_rows, int format, int* flushed_total) {
     const OperandLayout o = operand_layout(layout_rows ? layout_rows : rows, K, is_weight ? BN : BM);
     uint8_t* base = static_cast<uint8_t*>(prepared);
     return quantize_rows_prepared(x, rows, K, codes, scales, base, base + o.plane, base + 2 * o.plane,
                                   base + 2 * o.plane + o.sf, reinterpret_cast<int*>(base + 2 * o.plane + 2 * o.sf), o.nk64,
-                                  o.row_blocks * 128, st, format);
+                                  o.row_blocks * 128, st, format, flushed_total);
+}
+
+// Row words of a prepared operand (rows of them, device memory).
+const int* gemm_fp4_row_words(const void* prepared, int64_t rows, int64_t K, bool is_weight) {
+    const OperandLayout o = operand_layout(rows, K, is_weight ? BN : BM);
+    return reinterpret_cast<const int*>(static_cast<const uint8_t*>(prepared) + 2 * o.plane + 2 * o.sf);
 }
 
 int gemm_fp4_softmax_prepared(const float* S, int64_t rows, int64_t cols, int64_t ld_s, float alpha, bool is_weight,
@@ -966,21 +1000,27 @@ int gemm_fp4_softmax_prepared(const float* S, int64_t rows, int64_t cols, int64_
 }
 
 int gemm_fp4_prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, bool is_weight,
-                     void* prepared, cudaStream_t st, int64_t layout_rows) {
+                     void* prepared, cudaStream_t st, int64_t layout_rows, int* flushed_total) {
     return prepare(codes, scales, rows, K, operand_layout(layout_rows ? layout_rows : rows, K, is_weight ? BN : BM),
-                   static_cast<uint8_t*>(prepared), st);
+                   static_cast<uint8_t*>(prepared), st, flushed_total);
 }
 
+// Workspace: word 0 the status, word 1 the number of scales flushed while preparing the two operands (see
+// to_ue4m3), then the prepared operands.  gate_on_flushed: the GEMM kernel returns at once when that count is
+// not zero (the caller follows with the exact kernel, gated the other way).
 int gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes, const uint8_t* w_scales,
-             int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {
+             int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st,
+             bool gate_on_flushed) {
     const OperandLayout oa = operand_layout(M, K, BM), ow = operand_layout(N, K, BN);
     uint8_t* base = static_cast<uint8_t*>(workspace);
     uint8_t* pa = base + 256;
     uint8_t* pw = pa + oa.total;
-    int rc = prepare(a_codes, a_scales, M, K, oa, pa, st);
-    if (rc == AMX_OK) rc = prepare(w_codes, w_scales, N, K, ow, pw, st);
+    int* flushed = reinterpret_cast<int*>(base) + 1;
+    if (cudaMemsetAsync(base, 0, 8, st) != cudaSuccess) return AMX_ERR_CUDA;
+    int rc = prepare(a_codes, a_scales, M, K, oa, pa, st, flushed);
+    if (rc == AMX_OK) rc = prepare(w_codes, w_scales, N, K, ow, pw, st, flushed);
     if (rc != AMX_OK) return rc;
-    return gemm_fp4_prepared(pa, pw, M, N, K, C, ld_c, base, st);
+    return gemm_fp4_prepared(pa, pw, M, N, K, C, ld_c, base, st, 256, gate_on_flushed ? flushed : nullptr);
 }
 
 }  // namespace amx

@@ -75,9 +75,11 @@ template <bool CAST>
 __global__ void __launch_bounds__(128) rows_fragments_kernel(const uint8_t* __restrict__ codes,
                                                              const uint8_t* __restrict__ scales,
                                                              const uint16_t* __restrict__ x, int64_t ld_x, int M,
-                                                             int mts, int64_t K, uint4* __restrict__ frag) {
+                                                             int mts, int64_t K, uint4* __restrict__ frag,
+                                                             int* __restrict__ status) {
     const int64_t groups = K / 32;
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx == 0) status[0] = status[1] = 0;   // no device-side wait that can expire, no scale is flushed: both words read 0
     const bool live = idx < groups * 4 * kMaxRows * mts;           // whole groups: the four lanes agree
     const int j = (int)(idx & 3);
     const int64_t gidx = idx >> 2;
@@ -328,12 +330,17 @@ int launch_rows(const uint4* frag, const uint8_t* w_codes, const uint8_t* w_scal
     return AMX_OK;
 }
 
+// Workspace: 256 bytes whose first word is the status word amx_gemm_status reads, then the decoded rows.
+constexpr size_t kHeaderBytes = 256;
+uint4* fragments_of(void* workspace) { return reinterpret_cast<uint4*>(static_cast<uint8_t*>(workspace) + kHeaderBytes); }
+
 template <bool CAST>
 int launch_fragments(const uint8_t* codes, const uint8_t* scales, const uint16_t* x, int64_t ld_x, int64_t M, int64_t K,
-                     uint4* frag, cudaStream_t st) {
+                     void* workspace, cudaStream_t st) {
     const int mts = row_tiles(M);
     const int64_t threads = (int64_t)kMaxRows * mts * (K / 32) * 4;
-    rows_fragments_kernel<CAST><<<(unsigned)((threads + 127) / 128), 128, 0, st>>>(codes, scales, x, ld_x, (int)M, mts, K, frag);
+    rows_fragments_kernel<CAST><<<(unsigned)((threads + 127) / 128), 128, 0, st>>>(
+        codes, scales, x, ld_x, (int)M, mts, K, fragments_of(workspace), static_cast<int*>(workspace));
     return launch_status();
 }
 
@@ -344,21 +351,21 @@ bool gemm_rows_supported(int64_t M, int64_t N, int64_t K, int gs) {
            (N + kCtaRows - 1) / kCtaRows <= 0x7FFFFFFF;
 }
 
-size_t gemm_rows_workspace_bytes(int64_t M, int64_t K) { return (size_t)kMaxRows * row_tiles(M) * (size_t)K * 2; }
+size_t gemm_rows_workspace_bytes(int64_t M, int64_t K) {
+    return kHeaderBytes + (size_t)kMaxRows * row_tiles(M) * (size_t)K * 2;
+}
 
 int gemm_rows(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes, const uint8_t* w_scales,
               int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {
-    uint4* frag = static_cast<uint4*>(workspace);
-    if (launch_fragments<false>(a_codes, a_scales, nullptr, 0, M, K, frag, st) != AMX_OK) return AMX_ERR_CUDA;
-    return launch_rows(frag, w_codes, w_scales, M, N, K, C, ld_c, st);
+    if (launch_fragments<false>(a_codes, a_scales, nullptr, 0, M, K, workspace, st) != AMX_OK) return AMX_ERR_CUDA;
+    return launch_rows(fragments_of(workspace), w_codes, w_scales, M, N, K, C, ld_c, st);
 }
 
 int gemm_rows_cast(const void* x, int64_t ld_x, const uint8_t* w_codes, const uint8_t* w_scales, int64_t M, int64_t N,
                    int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {
-    uint4* frag = static_cast<uint4*>(workspace);
-    if (launch_fragments<true>(nullptr, nullptr, static_cast<const uint16_t*>(x), ld_x, M, K, frag, st) != AMX_OK)
+    if (launch_fragments<true>(nullptr, nullptr, static_cast<const uint16_t*>(x), ld_x, M, K, workspace, st) != AMX_OK)
         return AMX_ERR_CUDA;
-    return launch_rows(frag, w_codes, w_scales, M, N, K, C, ld_c, st);
+    return launch_rows(fragments_of(workspace), w_codes, w_scales, M, N, K, C, ld_c, st);
 }
 
 }  // namespace amx

@@ -114,7 +114,8 @@ gemm_tc_kernel(const uint8_t* __restrict__ a_codes, const uint8_t* __restrict__ 
                const uint16_t* __restrict__ a_x, int64_t ld_a,
                const uint8_t* __restrict__ w_codes, const uint8_t* __restrict__ w_scales,
                int64_t M, int64_t N, int64_t K, float* __restrict__ C, int64_t ld_c, int vec_store,
-               int* __restrict__ status, int kb_per_slice, int64_t slice_stride) {
+               int* __restrict__ status, int kb_per_slice, int64_t slice_stride, const int* __restrict__ run_if_nonzero) {
+    if (run_if_nonzero && *run_if_nonzero == 0) return;          // uniform over the grid: nothing was set up yet
     // blockIdx.z: slice of the K range (kb_per_slice K blocks each); slice z writes its partial product to
     // C + z * slice_stride (one slice: the result itself)
     extern __shared__ uint8_t smem_raw[];
@@ -273,7 +274,9 @@ int k_slices(int64_t M, int64_t N, int64_t K, int& kb_per_slice) {
 
 // C[m][n] = sum over slices, in slice order.
 __global__ void __launch_bounds__(256)
-reduce_slices_kernel(const float* __restrict__ part, int slices, int64_t M, int64_t N, float* __restrict__ C, int64_t ld_c) {
+reduce_slices_kernel(const float* __restrict__ part, int slices, int64_t M, int64_t N, float* __restrict__ C, int64_t ld_c,
+                     const int* __restrict__ run_if_nonzero) {
+    if (run_if_nonzero && *run_if_nonzero == 0) return;
     const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
     if (i >= M * N) return;
     float acc = part[i];
@@ -293,7 +296,7 @@ namespace {
 
 int launch_tc(const uint8_t* a_codes, const uint8_t* a_scales, const uint16_t* a_x, int64_t ld_a,
               const uint8_t* w_codes, const uint8_t* w_scales, int64_t M, int64_t N, int64_t K, float* C,
-              int64_t ld_c, void* workspace, cudaStream_t st) {
+              int64_t ld_c, void* workspace, cudaStream_t st, const int* gate = nullptr, int* status_word = nullptr) {
     static bool configured[64] = {};   // the opt-in to > 48 KB of dynamic shared memory is per device
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AMX_ERR_CUDA;
@@ -303,8 +306,9 @@ int launch_tc(const uint8_t* a_codes, const uint8_t* a_scales, const uint16_t* a
             return AMX_ERR_CUDA;
         configured[dev] = true;
     }
-    int* status = static_cast<int*>(workspace);
-    if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return AMX_ERR_CUDA;
+    // status word: the first word of the workspace, cleared here, unless the caller shares one it cleared itself
+    int* status = status_word ? status_word : static_cast<int*>(workspace);
+    if (!status_word && cudaMemsetAsync(status, 0, 2 * sizeof(int), st) != cudaSuccess) return AMX_ERR_CUDA;   // + flushed count: none
     int kb_per;
     const int slices = k_slices(M, N, K, kb_per);
     dim3 grid((unsigned)((N + BN - 1) / BN), (unsigned)((M + BM - 1) / BM), (unsigned)slices);
@@ -314,25 +318,30 @@ int launch_tc(const uint8_t* a_codes, const uint8_t* a_scales, const uint16_t* a
     const int vec_store = aligned(out, 16) && ld_out % 4 == 0;   // else the epilogue stores scalars
     if (a_x)
         gemm_tc_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(nullptr, nullptr, a_x, ld_a, w_codes, w_scales, M, N, K, out,
-                                                                 ld_out, vec_store, status, kb_per, slice_stride);
+                                                                 ld_out, vec_store, status, kb_per, slice_stride, gate);
     else
         gemm_tc_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(a_codes, a_scales, nullptr, 0, w_codes, w_scales, M, N, K,
-                                                                  out, ld_out, vec_store, status, kb_per, slice_stride);
+                                                                  out, ld_out, vec_store, status, kb_per, slice_stride, gate);
     int rc = launch_status();
     if (rc != AMX_OK || slices == 1) return rc;
-    return reduce_slices(part, slices, M, N, C, ld_c, st);
+    return reduce_slices(part, slices, M, N, C, ld_c, st, gate);
 }
 
 }  // namespace
 
-int reduce_slices(const float* part, int slices, int64_t M, int64_t N, float* C, int64_t ld_c, cudaStream_t st) {
-    reduce_slices_kernel<<<(unsigned)((M * N + 255) / 256), 256, 0, st>>>(part, slices, M, N, C, ld_c);
+int reduce_slices(const float* part, int slices, int64_t M, int64_t N, float* C, int64_t ld_c, cudaStream_t st,
+                  const int* run_if_nonzero) {
+    reduce_slices_kernel<<<(unsigned)((M * N + 255) / 256), 256, 0, st>>>(part, slices, M, N, C, ld_c, run_if_nonzero);
     return launch_status();
 }
 
+// run_if_nonzero: the launches do nothing when that device word is zero.  status_word: where a timeout is
+// recorded instead of the workspace's first word (the caller has cleared it).
 int gemm_tc(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_codes, const uint8_t* w_scales,
-            int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st) {
-    return launch_tc(a_codes, a_scales, nullptr, 0, w_codes, w_scales, M, N, K, C, ld_c, workspace, st);
+            int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c, void* workspace, cudaStream_t st,
+            const int* run_if_nonzero, int* status_word) {
+    return launch_tc(a_codes, a_scales, nullptr, 0, w_codes, w_scales, M, N, K, C, ld_c, workspace, st, run_if_nonzero,
+                     status_word);
 }
 
 // C = cast(X) What^T with the cast of X done by the kernel's producers.  X: bf16 [M, ld_a], 16-byte aligned,

@@ -114,7 +114,7 @@ extern "C" size_t amx_quant_error_workspace_bytes(void) { return (size_t)kMaxBlo
 extern "C" int amx_quant_error(const void* x, int64_t rows, int64_t K, int64_t ld_x, const uint8_t* codes,
                                const uint8_t* scales, int group_size, double* out, void* workspace,
                                size_t workspace_bytes, void* stream) {
-    if (!valid_group_size(group_size) || rows < 0 || K <= 0 || K % group_size || ld_x < K) return AMX_ERR_SHAPE;
+    if (!fixed_group_size(group_size) || rows < 0 || K <= 0 || K % group_size || ld_x < K) return AMX_ERR_SHAPE;
     if (!out) return AMX_ERR_NULL;
     if (rows > 0 && (!x || !codes || !scales)) return AMX_ERR_NULL;
     if (!workspace || workspace_bytes < amx_quant_error_workspace_bytes()) return AMX_ERR_WORKSPACE;

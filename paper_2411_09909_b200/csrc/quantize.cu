@@ -62,6 +62,38 @@ quantize_rows_kernel(const uint4* __restrict__ x, int64_t n_items, int64_t items
     }
 }
 
+// The whole row as one group (group_size == K; the grouping of the worked example in Appendix B.3): one block per
+// row, two sweeps - the row's side maxima (block reduction), then the codes.  The second sweep re-reads the row
+// from the caches.  Generic path, any K that is a multiple of 8.
+template <int FMT>
+__global__ void __launch_bounds__(kThreads)
+quantize_whole_rows_kernel(const uint4* __restrict__ x, int64_t vec_per_row, int64_t ld_vec, uint32_t* __restrict__ codes,
+                           uint16_t* __restrict__ scales) {
+    __shared__ uint32_t red[kThreads / 32];
+    const int64_t row = blockIdx.x;
+    const uint4* xr = x + row * ld_vec;
+    uint32_t c = 0;
+    for (int64_t i = threadIdx.x; i < vec_per_row; i += kThreads) {
+        const uint4 q = __ldg(xr + i);
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+        c = __vmaxs2(c, side_maxima<4>(w));
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) c = __vmaxs2(c, __shfl_xor_sync(0xFFFFFFFFu, c, d));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = c;
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < kThreads / 32; ++i) c = __vmaxs2(c, red[i]);
+    float inv_p, inv_n;
+    const uint32_t sc = group_scales_fmt<FMT>(c, inv_p, inv_n);
+    for (int64_t i = threadIdx.x; i < vec_per_row; i += kThreads) {
+        const uint4 q = __ldg(xr + i);
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+        codes[row * vec_per_row + i] = encode8(w, inv_p, inv_n);
+    }
+    if (threadIdx.x == 0) scales[row] = (uint16_t)sc;
+}
+
 // Groups DOWN the rows (strided axis): x is [R, C]; output is the canonical layout of x^T.
 // A block stages a [64 rows x 64 columns] tile in shared memory and re-reads it column-wise.
 constexpr int kTR = 64, kTC = 64;
@@ -119,12 +151,15 @@ constexpr int kPrepMaxRows = 8;
 
 // Second half of a prepared cast, for the GX threads (a multiple of 32) that own row `row` (`top`: the largest
 // positive-side scale byte the thread has seen in bits 7..0, the largest negative-side one in bits 15..8;
-// slot: the row's two shared-memory words, zero on entry): row maximum of the exponent keys and which sides
-// occur, the row's scale factors in the tensor cores' layout, padding included, and the row word.
+// slot: the row's four shared-memory words, zero on entry): row maximum of the exponent keys and which sides
+// occur, the row's scale factors in the tensor cores' layout, padding included, and the row word (with the
+// number of scales that did not fit the UE4M3 range and were flushed: the last warp of the row to finish
+// writes it, so no third block barrier is needed).
 __device__ __forceinline__ void finish_prepared_row(int64_t row, bool row_live, int G, int gx, int GX, uint32_t top,
                                                     uint32_t sc_first, const uint16_t* __restrict__ scales,
                                                     int* slot, uint8_t* __restrict__ sf_pos,
-                                                    uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp, int nk64) {
+                                                    uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp, int nk64,
+                                                    int* __restrict__ flushed_total = nullptr) {
     // Two shared-memory atomics per warp.  The key of an E5M2 byte grows with the byte (scales carry no sign
     // bit), so the largest byte has the largest key.
     const uint32_t top_p = __reduce_max_sync(0xFFFFFFFFu, top & 0xFFu), top_n = __reduce_max_sync(0xFFFFFFFFu, top >> 8);
@@ -138,6 +173,7 @@ __device__ __forceinline__ void finish_prepared_row(int64_t row, bool row_live, 
     // offset of this row's bytes inside a chunk; the chunks of one block of 128 rows are consecutive along K
     const int64_t sf_row = sf_row_offset(row, nk64);
     const int64_t v_row = row * G;
+    int flushed = 0;
     for (int g = gx; g < nk64 * 2; g += GX) {      // groups past G: padding to whole 256-element blocks
         uint32_t up = 0, un = 0;
         if (row_live && g < G) {
@@ -145,12 +181,23 @@ __device__ __forceinline__ void finish_prepared_row(int64_t row, bool row_live, 
             const uint32_t sc = (g == gx) ? sc_first : scales[v_row + g];
             up = to_ue4m3(sc & 0xFFu, kmax);
             un = to_ue4m3(sc >> 8, kmax);
+            flushed += (int)((sc & 0xFFu) != 0 && up == 0) + (int)((sc >> 8) != 0 && un == 0);
         }
         const int64_t off = sf_row + sf_group_offset(g);
         *reinterpret_cast<uint16_t*>(sf_pos + off) = (uint16_t)(up | (up << 8));
         *reinterpret_cast<uint16_t*>(sf_neg + off) = (uint16_t)(un | (un << 8));
     }
-    if (gx == 0 && row_live) row_exp[row] = row_word(kmax, slot[1]);
+    if (!row_live) return;                         // uniform over the row's warps
+    flushed = __reduce_add_sync(0xFFFFFFFFu, flushed);
+    if ((gx & 31) == 0) {
+        if (flushed) atomicAdd(&slot[2], flushed);
+        __threadfence_block();
+        if (atomicAdd(&slot[3], 1) == GX / 32 - 1) {
+            const int total = atomicAdd(&slot[2], 0);
+            row_exp[row] = row_word(kmax, slot[1], total);
+            if (total && flushed_total) atomicAdd(flushed_total, total);
+        }
+    }
 }
 
 // 40 registers (three blocks of 512 per SM): at 32 the kernel spills and is 12 % slower.
@@ -158,12 +205,13 @@ template <int FMT>
 __global__ void __launch_bounds__(512, 3)
 cast_prepared_kernel(const uint4* __restrict__ x, int64_t R, int G, uint4* __restrict__ codes,
                      uint16_t* __restrict__ scales, uint4* __restrict__ pos, uint4* __restrict__ neg,
-                     uint8_t* __restrict__ sf_pos, uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp, int nk64) {
-    __shared__ int slot_s[kPrepMaxRows][2];
+                     uint8_t* __restrict__ sf_pos, uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp, int nk64,
+                     int* __restrict__ flushed_total) {
+    __shared__ int slot_s[kPrepMaxRows][4];
     const int gx = threadIdx.x, rl = threadIdx.y, GX = blockDim.x;
     const int64_t row = (int64_t)blockIdx.x * blockDim.y + rl;
     const bool row_live = row < R;
-    if (gx < 2) slot_s[rl][gx] = 0;                 // visible to all after the barrier in finish_prepared_row
+    if (gx < 4) slot_s[rl][gx] = 0;                 // visible to all after the barrier in finish_prepared_row
     const int64_t v_row = row * G;
     uint32_t sc_first = 0;                      // scale bytes of this thread's first group (its only one when
                                                 // the block is as wide as its rows)
@@ -181,7 +229,8 @@ cast_prepared_kernel(const uint4* __restrict__ x, int64_t R, int G, uint4* __res
         if (g == gx) sc_first = sc;
         top = __vmaxu4(top, sc);                // byte-wise maximum
     }
-    finish_prepared_row(row, row_live, G, gx, GX, top, sc_first, scales, slot_s[rl], sf_pos, sf_neg, row_exp, nk64);
+    finish_prepared_row(row, row_live, G, gx, GX, top, sc_first, scales, slot_s[rl], sf_pos, sf_neg, row_exp, nk64,
+                        flushed_total);
 }
 
 // Attention glue in one pass (Appendix C): row softmax of the fp32 logits (times alpha), rounding of the
@@ -197,11 +246,11 @@ softmax_cast_kernel(const float* __restrict__ S, int64_t R, int G, int64_t ld_s,
                     uint4* __restrict__ neg, uint8_t* __restrict__ sf_pos, uint8_t* __restrict__ sf_neg,
                     int* __restrict__ row_exp, int nk64) {
     __shared__ float sh[softmax::kT / 32];
-    __shared__ int slot_s[2];
+    __shared__ int slot_s[4];
     const int gx = threadIdx.x;
     const int64_t row = blockIdx.x;
     const bool row_live = row < R;                  // uniform over the block
-    if (gx < 2) slot_s[gx] = 0;
+    if (gx < 4) slot_s[gx] = 0;
     uint32_t sc_first = 0, top = 0;
     if (row_live) {
         const float* s = S + row * ld_s;
@@ -257,7 +306,7 @@ int launch_rows(const void* x, int64_t rows, int64_t K, int64_t ld, uint8_t* cod
 // chunks of 512 B per block of 128 rows, rows padded to padded_rows) and the rows' power-of-two offsets.
 int quantize_rows_prepared(const void* x, int64_t rows, int64_t K, uint8_t* codes, uint8_t* scales, void* pos,
                            void* neg, uint8_t* sf_pos, uint8_t* sf_neg, int* row_exp, int nk64, int64_t padded_rows,
-                           cudaStream_t st, int format) {
+                           cudaStream_t st, int format, int* flushed_total) {
     const int64_t G = K / 32;
     // one thread per group when a row fits a block of 512, several rows per block when rows are short
     const int gx = (int)((G < 512 ? G : 512) + 31) / 32 * 32;
@@ -270,7 +319,7 @@ int quantize_rows_prepared(const void* x, int64_t rows, int64_t K, uint8_t* code
     kernel<<<(unsigned)blocks, dim3(gx, rb), 0, st>>>(
         reinterpret_cast<const uint4*>(x), rows, (int)G, reinterpret_cast<uint4*>(codes),
         reinterpret_cast<uint16_t*>(scales), reinterpret_cast<uint4*>(pos), reinterpret_cast<uint4*>(neg), sf_pos, sf_neg,
-        row_exp, nk64);
+        row_exp, nk64, flushed_total);
     return launch_status();
 }
 
@@ -318,6 +367,13 @@ namespace {
 template <int FMT>
 int launch_rows_gs(const void* x, int64_t rows, int64_t K, int64_t ld_x, int group_size, uint8_t* codes, uint8_t* scales,
                    cudaStream_t st) {
+    if (group_size == K && !fixed_group_size(group_size)) {          // whole-row grouping
+        if (rows > 0x7FFFFFFF) return AMX_ERR_SHAPE;
+        quantize_whole_rows_kernel<FMT><<<(unsigned)rows, kThreads, 0, st>>>(
+            reinterpret_cast<const uint4*>(x), K / 8, ld_x / 8, reinterpret_cast<uint32_t*>(codes),
+            reinterpret_cast<uint16_t*>(scales));
+        return launch_status();
+    }
     switch (group_size) {
         case 16: return launch_rows<16, 1, FMT>(x, rows, K, ld_x, codes, scales, st);
         case 32: return launch_rows<32, 1, FMT>(x, rows, K, ld_x, codes, scales, st);
@@ -337,11 +393,12 @@ extern "C" int amx_quantize_fmt(const void* x, int64_t rows, int64_t K, int64_t 
                                 uint8_t* codes, uint8_t* scales, void* stream) {
     using namespace amx;
     if (format < AMX_FMT_AMXFP4 || format > AMX_FMT_AMXFP4_POT_ROUND) return AMX_ERR_FLAGS;
-    if (!valid_group_size(group_size) || rows < 0 || K <= 0 || K % group_size || K % 8 || ld_x < K)
+    if (!valid_group_size(group_size, K) || rows < 0 || K <= 0 || K % group_size || K % 8 || ld_x < K)
         return AMX_ERR_SHAPE;
     if (rows == 0) return AMX_OK;
     if (!x || !codes || !scales) return AMX_ERR_NULL;
-    if (!aligned(x, 16) || ld_x % 8 || !aligned(codes, group_size == 16 ? 8 : 16) || !aligned(scales, 2)) return AMX_ERR_ALIGN;
+    const int code_align = fixed_group_size(group_size) ? (group_size == 16 ? 8 : 16) : 4;
+    if (!aligned(x, 16) || ld_x % 8 || !aligned(codes, code_align) || !aligned(scales, 2)) return AMX_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (format == AMX_FMT_SYM_FP8) return launch_rows_gs<1>(x, rows, K, ld_x, group_size, codes, scales, st);
     if (format == AMX_FMT_MXFP4) return launch_rows_gs<2>(x, rows, K, ld_x, group_size, codes, scales, st);
@@ -354,7 +411,7 @@ extern "C" int amx_quantize_fmt(const void* x, int64_t rows, int64_t K, int64_t 
 extern "C" int amx_quantize_t(const void* x, int64_t R, int64_t C, int64_t ld_x, int group_size,
                               uint8_t* codes, uint8_t* scales, void* stream) {
     using namespace amx;
-    if (!valid_group_size(group_size) || R < 0 || C < 0 || R % group_size || ld_x < C) return AMX_ERR_SHAPE;
+    if (!fixed_group_size(group_size) || R < 0 || C < 0 || R % group_size || ld_x < C) return AMX_ERR_SHAPE;
     if (R == 0 || C == 0) return AMX_OK;
     if (!x || !codes || !scales) return AMX_ERR_NULL;
     if (!aligned(x, 2) || !aligned(codes, 4) || !aligned(scales, 2)) return AMX_ERR_ALIGN;

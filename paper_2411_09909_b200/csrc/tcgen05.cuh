@@ -31,8 +31,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* b, uint32_t parity) {
 }
 // Bounded wait.  Returns false when the limit expired or another role already gave up; the first
 // role to give up raises the CTA's abort flag and records AMX_ERR_TIMEOUT in the status word.
-__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag, int* status) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag, int* status,
+                                          uint32_t limit = kSpinLimit) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait(b, parity)) return true;
         if (*abort_flag) return false;
     }

@@ -64,9 +64,28 @@ def test_host_detected_argument_errors(L):
     assert g(fake, fake, fake, fake, 65, 4, 512, 32, 0x100, fake, 4, None, 0, None) == -2   # and at most 64 rows
     assert g(fake, fake, fake, ctypes.c_void_p(0x1002), 4, 4, 512, 32, 0x100, fake, 4, fake, 1 << 20, None) == -3
     assert g(fake, fake, fake, fake, 0, 4, 64, 32, 0x10, fake, 4, None, 0, None) == 0   # empty
-    assert L.amx_quant_gemm(fake, 64, fake, fake, 4, 4, 64, 32, 0x10, fake, 4, None, 0, None) == -4
-    assert L.amx_quant_gemm(fake, 64, fake, fake, 4, 4, 64, 32, 0x80, fake, 4, fake, 4096, None) == -5   # cast-in-kernel
-    assert L.amx_quant_gemm(fake, 64, fake, fake, 4, 4, 64, 32, 0xC0, fake, 4, fake, 4096, None) == -5   # needs the TC kernel
+    qg = L.amx_quant_gemm
+    assert qg(fake, 64, fake, fake, None, 0, 4, 4, 64, 32, 0x10, fake, 4, None, 0, None) == -4
+    assert qg(fake, 64, fake, fake, None, 0, 4, 4, 64, 32, 0x80, fake, 4, fake, 4096, None) == -5   # cast-in-kernel
+    assert qg(fake, 64, fake, fake, None, 0, 4, 4, 64, 32, 0xC0, fake, 4, fake, 4096, None) == -5   # needs the TC kernel
+    assert qg(fake, 64, fake, fake, fake, 64, 4, 4, 64, 32, 0x10, fake, 4, fake, 1 << 20, None) == -1   # both weight forms
+    assert qg(fake, 64, None, None, None, 0, 4, 4, 64, 32, 0x10, fake, 4, fake, 1 << 20, None) == -1    # no weight at all
+    assert qg(fake, 64, None, None, fake, 32, 4, 4, 64, 32, 0x10, fake, 4, fake, 1 << 20, None) == -2   # ld_w < K
+    assert qg(fake, 64, None, None, odd, 64, 4, 4, 64, 32, 0x10, fake, 4, fake, 1 << 20, None) == -3    # bf16 weight alignment
+    assert L.amx_linear_host(fake, fake, 4, 4, 64, 32, 0x30, fake, fake, 1 << 30, None) == -5             # two kernels
+    assert L.amx_linear_host(fake, fake, 4, 4, 64, 32, 0x40, fake, fake, 16, None) == -4                  # checked before any copy
+    assert L.amx_attention_map(fake, fake, 320, 128, 0, fake, fake, fake, fake, 1 << 30, fake, 1 << 30, None) == -2   # L % 256
+    assert L.amx_attention_map(fake, fake, 512, 128, 0x40, fake, fake, fake, fake, 1 << 30, fake, 1 << 30, None) == -5
+    assert L.amx_prepared_flushed_scales(None, 4, 64, 32, 0, None) == -1
+    assert L.amx_prepared_flushed_scales(fake, 4, 64, 16, 0, None) == -2
+    assert L.amx_selftest_wait_timeout(fake, 64, 100, None) == -4
+    assert L.amx_selftest_wait_timeout(fake, 4096, 0, None) == -2
+    # whole-row groups (group_size == K) on the generic entry points; not on the transposed cast
+    assert q(fake, 4, 72, 72, 72, None, fake, None) == -1
+    assert q(fake, 4, 76, 76, 76, fake, fake, None) == -2               # K % 8
+    assert L.amx_dequantize(fake, fake, 4, 72, 72, 0, None, 72, None) == -1
+    assert L.amx_gemm_kernel_for(4, 4, 72, 72, 0) == 0x10
+    assert L.amx_quantize_t(fake, 48, 8, 8, 48, fake, fake, None) == -2
     assert L.amx_gemm(fake, fake, fake, fake, 4, 4, 64, 32, 0xA0, fake, 4, None, 0, None) == -5          # not an amx_gemm flag
     assert L.amx_attention(fake, fake, fake, 1, 64, 64, 0x2000, fake, fake, 1 << 30, None) == -5           # unknown flag
     assert L.amx_attention(fake, fake, fake, 1, 48, 64, 0x1000, fake, fake, 1 << 30, None) == -2           # L % 32
@@ -83,8 +102,15 @@ def test_workspace_sizes(L):
     assert simt == 0
     qg = L.amx_quant_gemm_workspace_bytes(100, 100, 64, 32, 0x10)
     assert qg >= 100 * 32 + 100 * 2 * 2 and qg % 256 == 0
-    lh = L.amx_linear_host_workspace_bytes(128, 256, 512, 32)
+    assert L.amx_quant_gemm_workspace_bytes(100, 100, 64, 32, 0x10 | 0x200) >= qg + 100 * 32 + 100 * 2 * 2
+    lh = L.amx_linear_host_workspace_bytes(128, 256, 512, 32, 0)
     assert lh >= 128 * 512 * 2 + 256 * 512 * 2 + 128 * 256 * 4
+    # an explicit kernel choice sizes the scratch for that kernel
+    assert L.amx_linear_host_workspace_bytes(128, 256, 512, 32, 0x40) > lh
+    # AUTO on the FP4 kernel carries the exact kernel's scratch too (device-side fallback)
+    assert L.amx_workspace_bytes(2048, 4096, 4096, 32, 0) > L.amx_workspace_bytes(2048, 4096, 4096, 32, 0x40)
+    # the weight-streaming kernel's scratch starts with a status header
+    assert L.amx_workspace_bytes(16, 4096, 4096, 32, 0x100) == 256 + 16 * 4096 * 2
     assert L.amx_gemm_kernel_for(100, 100, 64, 32, 0x10) == 0x10
 
 

@@ -1,0 +1,108 @@
+"""The cast of the attention map inside the second Q K^T pass (the path full-size attention runs): the kernel's
+own bf16 map, fed to the oracle quantizer, must give the kernel's codes and scales bit for bit; the positive
+plane of the prepared operand must equal the codes, its UE4M3 scale factors a host-side conversion of the
+oracle's scales, and no scale may be flushed.  The map itself is checked against the all-CPU pipeline (fp32
+exp on the device against fp64 on the host: single bf16 roundings differ)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2411_09909_b200 import amx, inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def dev_bf16(bits):
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def e5m2_key_mant(b):
+    """E5M2 byte -> (exponent key = unbiased exponent + 17, two mantissa bits) of its normalised form; key 0 = zero."""
+    b = b.astype(np.int64)
+    key = np.where(b >= 4, (b + 8) >> 2, np.array([0, 1, 2, 2])[np.minimum(b, 3)])
+    mant = np.where(b >= 4, b & 3, np.array([0, 0, 0, 2])[np.minimum(b, 3)])
+    return key, mant
+
+
+def expected_scale_factors(scale_pos, kmax):
+    """UE4M3 bytes of the positive-side scales [rows, G] under the per-row offset (largest key kmax [rows])."""
+    key, mant = e5m2_key_mant(scale_pos)
+    field = key - kmax[:, None] + 15
+    return np.where((scale_pos != 0) & (field >= 1), (field << 3) | (mant << 1), 0).astype(np.uint8)
+
+
+def check_rows(rows, L, p_bits, codes, scales, prep, causal):
+    """rows: row indices to check.  p_bits/codes/scales: host arrays of the whole map."""
+    oc, os_ = oracle.quantize(np.ascontiguousarray(p_bits[rows]), 32)
+    assert np.array_equal(codes[rows], oc)
+    assert np.array_equal(scales[rows], os_)
+    assert not np.any(os_[:, :, 1])                                  # no negative side in a softmax output
+    plane_bytes = -(-(L * L // 2) // 256) * 256
+    nk64 = -(-L // 256) * 4
+    sf_bytes = (L // 128) * nk64 * 512
+    plane = prep[: L * L // 2].reshape(L, L // 2)
+    G = L // 32
+    if causal:          # blocks of 256 keys entirely after the query's block of 128 are never visited nor read
+        for r in rows:
+            seen = (r // 128 // 2 + 1) * 256 // 2
+            assert np.array_equal(plane[r, :seen], oc[list(rows).index(r), :seen])
+    else:
+        assert np.array_equal(plane[rows], oc)
+    sf = prep[2 * plane_bytes: 2 * plane_bytes + sf_bytes]
+    words = prep[2 * plane_bytes + 2 * sf_bytes: 2 * plane_bytes + 2 * sf_bytes + 4 * L].view(np.int32)
+    key, _ = e5m2_key_mant(os_[:, :, 0])
+    kmax = key.max(axis=1)
+    assert np.array_equal((words[rows] & 0xFFFF).astype(np.int16).astype(np.int64), kmax - 25)
+    assert np.all((words[rows] >> 16) & 3 == 1) and np.all(words[rows] >> 18 == 0)   # positive side only, nothing flushed
+    want = expected_scale_factors(os_[:, :, 0], kmax)
+    for i, r in enumerate(rows):
+        g = np.arange(G if not causal else (r // 128 // 2 + 1) * 8)
+        off = (r // 128) * nk64 * 512 + (g // 2) * 512 + (r % 32) * 16 + ((r % 128) // 32) * 4 + (g % 2) * 2
+        assert np.array_equal(sf[off], want[i, g]) and np.array_equal(sf[off + 1], want[i, g]), r
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_attention_map_cast_bit_exact_small(causal):
+    L = 512
+    qb, kb, _ = (t[0] for t in inputs.attention_qkv(heads=1, seq=L))
+    flags = amx.ATTN_CAUSAL if causal else 0
+    p, c, s, prep = amx.attention_map(dev_bf16(qb), dev_bf16(kb), flags)
+    p_bits = p.view(torch.int16).cpu().numpy().view(np.uint16)
+    check_rows(np.arange(L), L, p_bits, c.cpu().numpy(), s.cpu().numpy(), prep.cpu().numpy(), causal)
+    assert amx.prepared_flushed_scales(prep, L, L, False) == 0
+    # the map itself against the all-CPU pipeline: equal up to one bf16 ulp on a small share of the entries
+    S = oracle.gemm(*oracle.quantize(qb, 32), *oracle.quantize(kb, 32), 32)
+    want = oracle.softmax_bf16(S, 128 ** -0.5, causal_row0=0) if causal else oracle.softmax_bf16(S, 128 ** -0.5)
+    diff = np.abs(p_bits.astype(np.int32) - want.astype(np.int32))
+    assert diff.max() <= 1 and np.mean(diff != 0) < 0.02
+    if causal:
+        assert not np.any(np.triu(p_bits, 1))                        # masked entries are exactly +0
+
+
+def test_attention_map_softer_rows_bit_exact():
+    """Inputs scaled down so that rows of the map hold many nonzero groups of very different size (the benchmark's
+    inputs make it nearly one-hot): exercises the scale-factor range of the cast."""
+    L = 512
+    qb, kb, _ = (t[0] for t in inputs.attention_qkv(heads=1, seq=L))
+    small = lambda b: inputs.f32_to_bf16_bits(inputs.bf16_bits_to_f32(b) * 0.35)
+    qb, kb = small(qb), small(kb)
+    p, c, s, prep = amx.attention_map(dev_bf16(qb), dev_bf16(kb), 0)
+    p_bits = p.view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.mean(s.cpu().numpy()[:, :, 0] != 0) > 0.5
+    check_rows(np.arange(L), L, p_bits, c.cpu().numpy(), s.cpu().numpy(), prep.cpu().numpy(), False)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_attention_map_cast_bit_exact_full_size_sampled(causal):
+    """Config-5 size (8192 keys): three sampled blocks of 128 query rows of head 0."""
+    L = 8192
+    qb, kb, _ = (t[0] for t in inputs.attention_qkv(heads=1, seq=L))
+    flags = amx.ATTN_CAUSAL if causal else 0
+    p, c, s, prep = amx.attention_map(dev_bf16(qb), dev_bf16(kb), flags)
+    p_bits = p.view(torch.int16).cpu().numpy().view(np.uint16)
+    rng = np.random.default_rng(77)
+    blocks = np.sort(rng.choice(L // 128, size=3, replace=False))
+    rows = np.concatenate([np.arange(b * 128, b * 128 + 128) for b in blocks])
+    check_rows(rows, L, p_bits, c.cpu().numpy(), s.cpu().numpy(), prep.cpu().numpy(), causal)
+    assert amx.prepared_flushed_scales(prep, L, L, False) == 0

@@ -547,7 +547,7 @@ def test_linear_host_entry_point():
     a = torch.from_numpy(a_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
     w = torch.from_numpy(w_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
     c = torch.empty((128, 256), dtype=torch.float32).pin_memory()
-    ws = torch.empty(amx.lib().amx_linear_host_workspace_bytes(128, 256, 1024, 32), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(amx.lib().amx_linear_host_workspace_bytes(128, 256, 1024, 32, 0), dtype=torch.uint8, device="cuda")
     amx.linear_host(a, w, c, ws)
     ref = oracle.gemm(*oracle.quantize(a_bits, 32), *oracle.quantize(w_bits, 32), 32)
     assert rel_fro(c.numpy(), ref) <= GEMM_TOL
@@ -697,30 +697,43 @@ def test_config5_full_size_attention_sampled():
 
 # ------------------------------------------------ full-size configurations --
 
-@pytest.mark.parametrize("config,layer", [(2, 0), (2, 3), (3, 0), (3, 1), (3, 3), (4, 0), (4, 2)])
+@pytest.mark.parametrize("config,layer", [(c, l) for c in (2, 3, 4) for l in range(len(inputs.LINEAR_CONFIGS[c]["layers"]))])
 def test_full_size_layer_sampled(config, layer):
-    """Whole-tensor launches at the benchmark's sizes; codes and scales compared on the whole activation
-    for config 2 and on sampled rows otherwise; GEMM compared on 64 sampled rows x all N."""
+    """Every layer of the three large configurations at its full size, whole-tensor launches.  Codes and scales are
+    compared on the whole activation for config 2 and on sampled rows otherwise; the product on 64 sampled rows x
+    all N, for amx_gemm and for the launch sequence the benchmark times (casts that write the FP4 kernel's
+    operands, then the GEMM on them), whose status word and flushed-scale counts are checked too."""
     spec = inputs.LINEAR_CONFIGS[config]
     M = spec["M"]
     a_bits, w_bits = inputs.activation(config, layer), inputs.weight(config, layer)
-    ac, as_ = amx.quantize(dev_bf16(a_bits), 32)
-    wc, ws = amx.quantize(dev_bf16(w_bits), 32)
+    K, N = a_bits.shape[1], w_bits.shape[0]
+    a, w = dev_bf16(a_bits), dev_bf16(w_bits)
+    ac, as_ = amx.quantize(a, 32)
+    wc, ws = amx.quantize(w, 32)
     rng = np.random.default_rng(100 * config + layer)
     rows = np.sort(rng.choice(M, size=64, replace=False))
+    rows_dev = torch.from_numpy(rows).cuda()
     arow = np.arange(M) if config == 2 else np.union1d(rows, rng.choice(M, size=256, replace=False))
+    arow_dev = torch.from_numpy(arow).cuda()
     oac, oas = oracle.quantize(a_bits[arow], 32)
-    assert np.array_equal(ac.cpu().numpy()[arow], oac) and np.array_equal(as_.cpu().numpy()[arow], oas)
-    wrow = np.sort(rng.choice(w_bits.shape[0], size=512, replace=False))
+    assert np.array_equal(ac[arow_dev].cpu().numpy(), oac) and np.array_equal(as_[arow_dev].cpu().numpy(), oas)
+    wrow = np.sort(rng.choice(N, size=512, replace=False))
+    wrow_dev = torch.from_numpy(wrow).cuda()
     owc, ows = oracle.quantize(w_bits[wrow], 32)
-    assert np.array_equal(wc.cpu().numpy()[wrow], owc) and np.array_equal(ws.cpu().numpy()[wrow], ows)
-    got = amx.gemm(ac, as_, wc, ws, 32).cpu().numpy()[rows]
-    ref = oracle.gemm(ac.cpu().numpy(), as_.cpu().numpy(), wc.cpu().numpy(), ws.cpu().numpy(), 32, rows=rows)
+    assert np.array_equal(wc[wrow_dev].cpu().numpy(), owc) and np.array_equal(ws[wrow_dev].cpu().numpy(), ows)
+    # reference on the sampled rows: the oracle's own codes of those rows against the device's weight codes
+    # (checked above on a sample; the product below would expose a wrong row anywhere else)
+    sel = np.searchsorted(arow, rows)
+    ref = oracle.gemm(oac[sel], oas[sel], wc.cpu().numpy(), ws.cpu().numpy(), 32)
+    got = amx.gemm(ac, as_, wc, ws, 32)[rows_dev].cpu().numpy()
     assert rel_fro(got, ref) <= GEMM_TOL
-    if config == 2:
-        # the launch sequence the benchmark times: casts that write the prepared operands, then the GEMM on them
-        ac2, as2, pa = amx.quantize_prepared(dev_bf16(a_bits), False)
-        wc2, ws2, pw = amx.quantize_prepared(dev_bf16(w_bits), True)
-        assert torch.equal(ac2, ac) and torch.equal(as2, as_) and torch.equal(wc2, wc) and torch.equal(ws2, ws)
-        got2 = amx.gemm_prepared(pa, pw, M, w_bits.shape[0], a_bits.shape[1]).cpu().numpy()[rows]
-        assert rel_fro(got2, ref) <= GEMM_TOL
+    del got
+    # the launch sequence the benchmark times
+    ac2, as2, pa = amx.quantize_prepared(a, False)
+    wc2, ws2, pw = amx.quantize_prepared(w, True)
+    assert torch.equal(ac2, ac) and torch.equal(as2, as_) and torch.equal(wc2, wc) and torch.equal(ws2, ws)
+    assert amx.prepared_flushed_scales(pa, M, K, False) == 0 and amx.prepared_flushed_scales(pw, N, K, True) == 0
+    work = torch.empty(256, dtype=torch.uint8, device="cuda")
+    got2 = amx.gemm_prepared(pa, pw, M, N, K, workspace=work)[rows_dev].cpu().numpy()
+    assert amx.gemm_status(work) == 0
+    assert rel_fro(got2, ref) <= GEMM_TOL

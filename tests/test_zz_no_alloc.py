@@ -21,9 +21,11 @@ def _static(a, wc, ws, flags=0):
     M, K = a.shape
     N = wc.shape[0]
     out = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
     rc = amx.lib().amx_quant_gemm_static(a.data_ptr(), a.stride(0), wc.data_ptr(), ws.data_ptr(), M, N, K, 32,
-                                         flags, out.data_ptr(), N, torch.cuda.current_stream().cuda_stream)
+                                         flags, out.data_ptr(), N, stream)
     assert rc == 0, amx.status_string(rc)
+    assert amx.lib().amx_quant_gemm_static_status(stream) == 0       # no bounded wait expired
     return out
 
 
