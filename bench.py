@@ -36,7 +36,9 @@ GS = 32
 NOMINAL_FP4_TFLOPS = 9000.0      # NVIDIA's dense FP4 figure for one B200 (HGX B200 data sheet)
 NOMINAL_HBM_GBS = 8000.0
 BYTES_PER_ELEM = 2.0 + 0.5 + 2.0 / 32.0   # bf16 read + 4-bit code + two scale bytes per 32
-MOVED_BYTES_PER_ELEM = BYTES_PER_ELEM + 1.0 + 4.0 / 32.0   # + two sign planes + four scale-factor bytes per 32
+# what the step's cast moves: bf16 read, two sign planes, two scale bytes and four scale-factor bytes per 32 (the
+# canonical codes are not written: the step only multiplies)
+MOVED_BYTES_PER_ELEM = 2.0 + 1.0 + 2.0 / 32.0 + 4.0 / 32.0
 # DRAM bytes (read + write) per GEMM launch of the FP4 kernel, mean over the layers of a config, from the ncu
 # captures summarised in profiles/ (None: no capture of the current kernel on that config).
 GEMM_DRAM_TRAFFIC_PER_LAUNCH = {2: None, 3: None, 4: None}
@@ -385,7 +387,7 @@ def run_ours(args):
         K, N = layers[li]
         b = bufs[li]
         if fused_prepare:   # the cast writes the FP4 kernel's operand (sign planes, scale factors) in the same pass
-            check(L.amx_quantize_prepared(A[li].data_ptr(), M, K, GS, 0, b["ac"].data_ptr(), b["as"].data_ptr(),
+            check(L.amx_quantize_prepared(A[li].data_ptr(), M, K, GS, 0, None, b["as"].data_ptr(),
                                           b["pa"].data_ptr(), b["pa"].numel(), st))
         else:
             check(L.amx_quantize(A[li].data_ptr(), M, K, K, GS, b["ac"].data_ptr(), b["as"].data_ptr(), st))
@@ -394,7 +396,7 @@ def run_ours(args):
         K, N = layers[li]
         b = bufs[li]
         if fused_prepare:
-            check(L.amx_quantize_prepared(W[li].data_ptr(), N, K, GS, 1, b["wc"].data_ptr(), b["ws"].data_ptr(),
+            check(L.amx_quantize_prepared(W[li].data_ptr(), N, K, GS, 1, None, b["ws"].data_ptr(),
                                           b["pw"].data_ptr(), b["pw"].numel(), st))
         else:
             check(L.amx_quantize(W[li].data_ptr(), N, K, K, GS, b["wc"].data_ptr(), b["ws"].data_ptr(), st))
@@ -560,9 +562,9 @@ def run_ours(args):
                 for li, (K, N) in enumerate(layers):
                     b = bufs[li]
                     if with_casts:
-                        check(L.amx_quantize_prepared_fmt(A[li].data_ptr(), M, K, GS, 0, fmt, b["ac"].data_ptr(),
+                        check(L.amx_quantize_prepared_fmt(A[li].data_ptr(), M, K, GS, 0, fmt, None,
                                                           b["as"].data_ptr(), b["pa"].data_ptr(), b["pa"].numel(), st))
-                        check(L.amx_quantize_prepared_fmt(W[li].data_ptr(), N, K, GS, 1, fmt, b["wc"].data_ptr(),
+                        check(L.amx_quantize_prepared_fmt(W[li].data_ptr(), N, K, GS, 1, fmt, None,
                                                           b["ws"].data_ptr(), b["pw"].data_ptr(), b["pw"].numel(), st))
                     gemm(li, st)
             res = {}
@@ -739,8 +741,9 @@ def run_ours(args):
                                                     "frac": quant_gbs * moved / BYTES_PER_ELEM / peaks["hbm_gbs"],
                                                     "achieved_canonical_bytes": quant_gbs,
                                                     "what": "both casts of every layer of the step (events around the cast "
-                                                            "phase); bytes actually moved: canonical 2.5625 B/element plus "
-                                                            "the sign planes and scale factors of the FP4 kernel's operand"},
+                                                            "phase); bytes actually moved per element: 2 read, 1 of sign "
+                                                            "planes, 0.0625 of scale bytes, 0.125 of scale factors (the "
+                                                            "canonical codes are not written)"},
                                   "plain_cast": (None if quant_large is None else
                                                  {"bytes_per_element": BYTES_PER_ELEM, "achieved": quant_large["gb_per_s"],
                                                   "frac": quant_large["frac_of_measured_copy"],

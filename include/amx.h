@@ -185,7 +185,8 @@ int amx_gemm(const uint8_t* a_codes, const uint8_t* a_scales,
  *                      summation order, run-to-run identical).
  *   amx_quantize_prepared  amx_quantize (x bf16 [rows, K], contiguous rows, gs = 32) and amx_prepare in one
  *                      go: the cast kernel itself writes the sign planes, so the codes are not read again.
- *                      Writes the canonical codes and scales too.
+ *                      Writes the canonical scales too, and the canonical codes unless `codes` is NULL (a caller
+ *                      that only multiplies does not need them: 0.5 of 3.7 bytes per element less to write).
  * This is how Section 4.3's product runs when the weights were cast once ahead of time.
  */
 int amx_quantize_prepared(const void* x, int64_t rows, int64_t K, int group_size, int is_weight,

@@ -204,19 +204,21 @@ def prepare(codes: torch.Tensor, scales: torch.Tensor, is_weight: bool, group_si
 
 
 def quantize_prepared(x: torch.Tensor, is_weight: bool, group_size: int = 32, prepared: torch.Tensor | None = None,
-                      fmt: int = FMT_AMXFP4):
-    """Cast and prepare in one go: returns (codes, scales, prepared)."""
+                      fmt: int = FMT_AMXFP4, want_codes: bool = True):
+    """Cast and prepare in one go: returns (codes, scales, prepared); codes is None when want_codes is False."""
     _dev(x, torch.bfloat16, "x")
     assert x.is_contiguous()
     rows, K = x.shape
-    codes = torch.empty((rows, K // 2), dtype=torch.uint8, device=x.device)
+    codes = torch.empty((rows, K // 2), dtype=torch.uint8, device=x.device) if want_codes else None
     scales = torch.empty((rows, K // group_size, 2), dtype=torch.uint8, device=x.device)
     buf = prepared if prepared is not None else _ws(lib().amx_prepared_bytes(rows, K, group_size, int(is_weight)), x.device)
     if fmt == FMT_AMXFP4:
-        _check(lib().amx_quantize_prepared(x.data_ptr(), rows, K, group_size, int(is_weight), codes.data_ptr(),
+        _check(lib().amx_quantize_prepared(x.data_ptr(), rows, K, group_size, int(is_weight),
+                                           codes.data_ptr() if want_codes else None,
                                            scales.data_ptr(), buf.data_ptr(), buf.numel(), _stream()), "amx_quantize_prepared")
     else:
-        _check(lib().amx_quantize_prepared_fmt(x.data_ptr(), rows, K, group_size, int(is_weight), fmt, codes.data_ptr(),
+        _check(lib().amx_quantize_prepared_fmt(x.data_ptr(), rows, K, group_size, int(is_weight), fmt,
+                                               codes.data_ptr() if want_codes else None,
                                                scales.data_ptr(), buf.data_ptr(), buf.numel(), _stream()),
                "amx_quantize_prepared_fmt")
     return codes, scales, buf

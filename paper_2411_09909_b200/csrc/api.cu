@@ -158,7 +158,7 @@ extern "C" int amx_quantize_prepared_fmt(const void* x, int64_t rows, int64_t K,
                                          size_t prepared_bytes, void* stream) {
     if (format != AMX_FMT_AMXFP4 && format != AMX_FMT_SYM_FP8 && format != AMX_FMT_MXFP4) return AMX_ERR_FLAGS;
     if (rows <= 0 || !gemm_fp4_supported(rows, rows, K, group_size)) return AMX_ERR_SHAPE;
-    if (!x || !codes || !scales || !prepared) return AMX_ERR_NULL;
+    if (!x || !scales || !prepared) return AMX_ERR_NULL;       // codes may be NULL: they are then not written
     if (prepared_bytes < amx_prepared_bytes(rows, K, group_size, is_weight)) return AMX_ERR_WORKSPACE;
     if (!aligned(x, 16) || !aligned(codes, 16) || !aligned(scales, 2) || !aligned(prepared, kAlign)) return AMX_ERR_ALIGN;
     return gemm_fp4_quantize_prepared(x, rows, K, is_weight != 0, codes, scales, prepared, static_cast<cudaStream_t>(stream),

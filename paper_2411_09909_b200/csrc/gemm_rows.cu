@@ -26,6 +26,7 @@
 #include <cuda_bf16.h>
 
 #include "cast_math.cuh"
+#include "cp_async.cuh"
 #include "decode_math.cuh"
 #include "gemm.cuh"
 
@@ -115,17 +116,6 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-
-// Asynchronous copy of 16 or 4 bytes from global to shared memory (no registers held while in flight).
-__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src));
-}
-__device__ __forceinline__ void cp_async4(void* dst, const void* src) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src));
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // Shared memory of a CTA: one ring of kDepth steps per warp for the weight stream.  A ring slot holds, per 8-row
 // tile, the 32 lanes' 16 bytes of codes and 4 bytes of scales (the two groups 4 * step + 2 * (t / 2) + {0, 1}; the

@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 
 #include "cast_math.cuh"
+#include "cp_async.cuh"
 #include "softmax_math.cuh"
 
 namespace amx {
@@ -141,13 +142,10 @@ quantize_cols_kernel(const __nv_bfloat16* __restrict__ x, int64_t R, int64_t C, 
 // sign bit, zero in the other), the UE4M3 scale factors of both planes - byte (r%32)*16 + (r/32)*4 + k16%4 of
 // the 512-byte chunk of [128 rows x 64 elements]; one scale per 16 elements, so a 32-group's scale is stored
 // twice - and per row the power of two by which those scale factors understate the true scales
-// (row_exp = largest exponent key of the row - 25).  The scale factors depend on the row's largest scale, so a
-// block owns whole rows, one thread per group (threads stride over the groups when a row is longer than the
-// block).  Blocks past the last row, and groups past the last group, zero the padding of the scale-factor
-// array, so that padded tile rows and columns multiply zero codes by a finite scale.
-// Block shape (GX, RB): thread (x, y) owns groups x, x + GX, ... of row blockIdx.x * RB + y.  GX is a multiple
-// of 32, so a warp never spans two rows.
-constexpr int kPrepMaxRows = 8;
+// (row_exp = largest exponent key of the row - 25).  The scale factors depend on the row's largest scale, so
+// whole rows belong to one warp (cast_prepared_kernel) or, in the softmax variant, to one block
+// (finish_prepared_row).  Rows past the last row, and groups past the last group, get zero scale factors, so that
+// padded tile rows and columns multiply zero codes by a finite scale.
 
 // Second half of a prepared cast, for the GX threads (a multiple of 32) that own row `row` (`top`: the largest
 // positive-side scale byte the thread has seen in bits 7..0, the largest negative-side one in bits 15..8;
@@ -200,37 +198,134 @@ __device__ __forceinline__ void finish_prepared_row(int64_t row, bool row_live, 
     }
 }
 
-// 40 registers (three blocks of 512 per SM): at 32 the kernel spills and is 12 % slower.
-template <int FMT>
-__global__ void __launch_bounds__(512, 3)
-cast_prepared_kernel(const uint4* __restrict__ x, int64_t R, int G, uint4* __restrict__ codes,
-                     uint16_t* __restrict__ scales, uint4* __restrict__ pos, uint4* __restrict__ neg,
-                     uint8_t* __restrict__ sf_pos, uint8_t* __restrict__ sf_neg, int* __restrict__ row_exp, int nk64,
-                     int* __restrict__ flushed_total) {
-    __shared__ int slot_s[kPrepMaxRows][4];
-    const int gx = threadIdx.x, rl = threadIdx.y, GX = blockDim.x;
-    const int64_t row = (int64_t)blockIdx.x * blockDim.y + rl;
-    const bool row_live = row < R;
-    if (gx < 4) slot_s[rl][gx] = 0;                 // visible to all after the barrier in finish_prepared_row
+// The cast for an operand of the FP4 GEMM.  A row (or, when rows are short, several rows) belongs to one warp:
+// LPR = 2^lpr_log2 lanes per row, lane lr of them owns the groups lr, lr + LPR, ...  A lane streams its groups
+// through a private ring in shared memory with asynchronous copies (kCastDepth groups ahead; the loads hold no
+// registers).  First sweep: per group the cast, the stores of the planes, the scale bytes and (when asked for)
+// the canonical codes; the scale bytes stay in registers (GPL of them per lane; GPL = 0: any number, re-read from
+// the scales just stored).  Then the row's largest exponent key by a warp reduction, and the second sweep turns
+// the scale bytes into the row's scale factors, padding included, and writes the row word.
+// Scale factors leave the block in whole 32-byte sectors: the tensor cores' layout interleaves eight rows (r, r+1,
+// r+32, r+33, r+64, r+65, r+96, r+97, r even) in every sector, so a block of eight warps owns exactly such sets of
+// rows - warp (q, h) has the rows 32 q + 2 k + h of a 128-row block, for the block's RPW = 32 / LPR values of k -
+// collects the converted bytes in shared memory and stores them 16 bytes per thread.  (Written 2 bytes at a
+// time straight from the owning lanes, the scale factors were 4 % of the bytes and doubled the kernel's L2
+// write requests.)  Rows past the last row get zero scale factors.
+constexpr int kCastDepth = 2;                              // groups in flight per lane
+constexpr int kCastWarps = 8;
+constexpr int kCastRingBytes = kCastWarps * kCastDepth * 32 * 64;
+constexpr int kCastMaxExchangeBytes = 96 * 1024;           // above this (K > 49152 at LPR = 32) the lanes store their bytes themselves
+
+template <int FMT, int GPL>
+__global__ void __launch_bounds__(kCastWarps * 32)
+cast_prepared_kernel(const uint4* __restrict__ x, int64_t R, int G, int lpr_log2, int exchange,
+                     uint4* __restrict__ codes, uint16_t* __restrict__ scales, uint4* __restrict__ pos,
+                     uint4* __restrict__ neg, uint8_t* __restrict__ sf_pos, uint8_t* __restrict__ sf_neg,
+                     int* __restrict__ row_exp, int nk64, int* __restrict__ flushed_total) {
+    extern __shared__ __align__(16) uint8_t smem_raw[];
+    const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5, LPR = 1 << lpr_log2, lr = lane & (LPR - 1);
+    const int RPW = 32 >> lpr_log2, sg = lane >> lpr_log2;      // rows per warp; which of them this lane works on
+    // the block's rows: 128-row block rb, sector sets k0 .. k0 + RPW - 1 (16 / RPW blocks share a 128-row block)
+    const int64_t rb = (int64_t)blockIdx.x >> (lpr_log2 - 1);
+    const int k0 = ((int)blockIdx.x & ((16 >> (5 - lpr_log2)) - 1)) << (5 - lpr_log2);
+    const int r_in = 32 * (wi >> 1) + 2 * (k0 + sg) + (wi & 1);  // row inside the 128-row block
+    const int64_t row = rb * 128 + r_in;
+    const bool live = row < R;
+    const unsigned seg_mask = LPR == 32 ? 0xFFFFFFFFu : ((1u << LPR) - 1u) << (lane & ~(LPR - 1));
     const int64_t v_row = row * G;
-    uint32_t sc_first = 0;                      // scale bytes of this thread's first group (its only one when
-                                                // the block is as wide as its rows)
-    uint32_t top = 0;                           // largest scale bytes seen by this thread, {neg : pos}
-    for (int g = gx; g < G; g += GX) {
-        if (!row_live) break;                   // uniform over the warp: a warp sits inside one row
-        const int64_t v = v_row + g;
+    // this lane's ring: kCastDepth slots of 64 bytes (one group).  Piece j of a group sits at 16-byte position
+    // j ^ ((lane >> 1) & 3) of the slot, so that the lanes of a quarter warp read eight different bank groups.
+    uint8_t* ring = smem_raw + ((wi * kCastDepth * 32) + lane) * 64;
+    uint8_t* xchg = smem_raw + kCastRingBytes;        // [plane][chunk][sector set][h][q] words of 4 scale-factor bytes
+    const int swz = (lane >> 1) & 3;
+    const int n_own = (live && lr < G) ? ((G - lr + LPR - 1) >> lpr_log2) : 0;   // groups this lane owns
+    auto issue = [&](int i) {                        // copies of the lane's i-th group, one commit group per call
+        if (i < n_own) {
+            const uint4* src = x + (v_row + lr + ((int64_t)i << lpr_log2)) * 4;
+            uint8_t* slot = ring + (i % kCastDepth) * (32 * 64);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) cp_async16(slot + ((j ^ swz) << 4), src + j);
+        }
+        cp_async_commit();
+    };
+    auto cast_group = [&](int i) -> uint32_t {       // the i-th group has landed: read it back, cast, store
+        const uint8_t* slot = ring + (i % kCastDepth) * (32 * 64);
         uint32_t w[16];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const uint4 q = __ldg(x + v * 4 + j);
+            const uint4 q = *reinterpret_cast<const uint4*>(slot + ((j ^ swz) << 4));
             w[4 * j] = q.x; w[4 * j + 1] = q.y; w[4 * j + 2] = q.z; w[4 * j + 3] = q.w;
         }
-        const uint32_t sc = emit_group<FMT>(w, v, codes, scales, pos, neg);
-        if (g == gx) sc_first = sc;
-        top = __vmaxu4(top, sc);                // byte-wise maximum
+        return emit_group<FMT>(w, v_row + lr + ((int64_t)i << lpr_log2), codes, scales, pos, neg);
+    };
+    uint32_t sc_reg[GPL > 0 ? GPL : 1];
+    uint32_t top = 0;                               // largest scale bytes seen by this lane, {neg : pos}
+#pragma unroll
+    for (int i = 0; i < kCastDepth - 1; ++i) issue(i);
+    if (GPL > 0) {
+#pragma unroll
+        for (int i = 0; i < GPL; ++i) {
+            issue(i + kCastDepth - 1);
+            cp_async_wait<kCastDepth - 1>();
+            sc_reg[i] = i < n_own ? cast_group(i) : 0u;
+            top = __vmaxu4(top, sc_reg[i]);         // byte-wise maximum
+        }
+    } else {
+        for (int i = 0; i < n_own; ++i) {
+            issue(i + kCastDepth - 1);
+            cp_async_wait<kCastDepth - 1>();
+            top = __vmaxu4(top, cast_group(i));
+        }
     }
-    finish_prepared_row(row, row_live, G, gx, GX, top, sc_first, scales, slot_s[rl], sf_pos, sf_neg, row_exp, nk64,
-                        flushed_total);
+    cp_async_wait<0>();
+    // The key of an E5M2 byte grows with the byte (scales carry no sign bit): the largest byte has the largest key.
+    const uint32_t top_p = __reduce_max_sync(seg_mask, top & 0xFFu), top_n = __reduce_max_sync(seg_mask, (top >> 8) & 0xFFu);
+    const int kmax = scale_key(max(top_p, top_n));
+    const int64_t sf_row = sf_row_offset(row, nk64);
+    // word of the exchange buffer that holds this row's bytes of chunk c: ((c * RPW + sg) * 2 + h) * 4 + q
+    const int x_row = (sg * 2 + (wi & 1)) * 4 + (wi >> 1), x_plane = nk64 * RPW * 8;   // in words
+    int flushed = 0;
+    auto put = [&](int g, uint32_t sc) {            // scale factors of group g (zero past the row's last group)
+        const uint32_t up = to_ue4m3(sc & 0xFFu, kmax), un = to_ue4m3(sc >> 8, kmax);
+        flushed += (int)((sc & 0xFFu) != 0 && up == 0) + (int)((sc >> 8) != 0 && un == 0);
+        if (exchange) {
+            uint16_t* w16 = reinterpret_cast<uint16_t*>(xchg) + (((g >> 1) * RPW * 8 + x_row) << 1) + (g & 1);
+            w16[0] = (uint16_t)(up | (up << 8));
+            w16[x_plane << 1] = (uint16_t)(un | (un << 8));
+        } else {
+            const int64_t off = sf_row + sf_group_offset(g);
+            *reinterpret_cast<uint16_t*>(sf_pos + off) = (uint16_t)(up | (up << 8));
+            *reinterpret_cast<uint16_t*>(sf_neg + off) = (uint16_t)(un | (un << 8));
+        }
+    };
+    const int g_end = nk64 * 2;                     // groups past G: padding to whole 256-element blocks
+    if (GPL > 0) {
+#pragma unroll
+        for (int i = 0; i < GPL; ++i) {
+            const int g = lr + (i << lpr_log2);
+            if (g < g_end) put(g, sc_reg[i]);       // zero for a group past G and for a padding row
+        }
+        for (int g = lr + (GPL << lpr_log2); g < g_end; g += LPR) put(g, 0u);
+    } else {
+        for (int g = lr; g < g_end; g += LPR) put(g, (live && g < G) ? (uint32_t)scales[v_row + g] : 0u);
+    }
+    flushed = __reduce_add_sync(seg_mask, flushed);
+    if (lr == 0 && live) {
+        row_exp[row] = row_word(kmax, side_bits_of(top_p | (top_n << 8)), flushed);
+        if (flushed && flushed_total) atomicAdd(flushed_total, flushed);
+    }
+    if (!exchange) return;                          // uniform over the block
+    __syncthreads();
+    // 16 bytes per thread: the words of rows q = 0..3 (32 rows apart) for one (plane, chunk, sector set, h);
+    // two neighbouring threads (h = 0, 1) fill one sector
+    const int per_plane = nk64 * RPW * 2;
+    for (int item = threadIdx.x; item < 2 * per_plane; item += kCastWarps * 32) {
+        const int plane = item >= per_plane, rest = item - plane * per_plane;
+        const int c = rest / (RPW * 2), sh = rest - c * (RPW * 2);      // sh = sector set * 2 + h
+        const uint4 v = reinterpret_cast<const uint4*>(xchg)[item];
+        uint8_t* dst = (plane ? sf_neg : sf_pos) + (rb * nk64 + c) * (int64_t)kSfChunkBytes + (2 * k0 + sh) * 16;
+        *reinterpret_cast<uint4*>(dst) = v;
+    }
 }
 
 // Attention glue in one pass (Appendix C): row softmax of the fp32 logits (times alpha), rounding of the
@@ -304,23 +399,53 @@ int launch_rows(const void* x, int64_t rows, int64_t K, int64_t ld, uint8_t* cod
 // Cast with the FP4 GEMM's operand preparation in the same launch (gs = 32, contiguous rows): canonical codes
 // and scales, the two sign planes, the UE4M3 scale factors of both planes in the tensor cores' layout (nk64
 // chunks of 512 B per block of 128 rows, rows padded to padded_rows) and the rows' power-of-two offsets.
+namespace {
+template <int FMT>
+int launch_cast_prepared(const void* x, int64_t rows, int64_t G, uint8_t* codes, uint8_t* scales, void* pos, void* neg,
+                         uint8_t* sf_pos, uint8_t* sf_neg, int* row_exp, int nk64, int64_t padded_rows, cudaStream_t st,
+                         int* flushed_total) {
+    int lpr_log2 = 1;
+    while (lpr_log2 < 5 && (1 << lpr_log2) < G) ++lpr_log2;          // lanes per row: a power of two, 2 .. 32
+    const int gpl = (int)((G + (1 << lpr_log2) - 1) >> lpr_log2);   // groups per lane
+    const int rpw = 32 >> lpr_log2;                                  // rows per warp
+    const int64_t blocks = (padded_rows / 128) * (16 / rpw);         // a block has 8 * rpw rows of one 128-row block
+    if (blocks > 0x7FFFFFFF) return AMX_ERR_SHAPE;
+    const size_t exchange_bytes = (size_t)64 * rpw * nk64;           // both planes, 4 bytes per row and 64 elements
+    const int exchange = exchange_bytes <= (size_t)kCastMaxExchangeBytes;
+    const int smem = kCastRingBytes + (exchange ? (int)exchange_bytes : 0);
+    auto* kernel = gpl <= 1 ? cast_prepared_kernel<FMT, 1> : gpl <= 2 ? cast_prepared_kernel<FMT, 2>
+                 : gpl <= 4 ? cast_prepared_kernel<FMT, 4> : gpl <= 8 ? cast_prepared_kernel<FMT, 8>
+                 : cast_prepared_kernel<FMT, 0>;      // longer rows: the scale bytes are re-read, not kept in registers
+    static bool configured[64][5] = {};                 // the opt-in to > 48 KB of dynamic shared memory: per device, kernel
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AMX_ERR_CUDA;
+    const int slot = gpl <= 1 ? 0 : gpl <= 2 ? 1 : gpl <= 4 ? 2 : gpl <= 8 ? 3 : 4;
+    if (!configured[dev][slot]) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kCastRingBytes + kCastMaxExchangeBytes) !=
+            cudaSuccess) {
+            cudaGetLastError();
+            return AMX_ERR_CUDA;
+        }
+        configured[dev][slot] = true;
+    }
+    kernel<<<(unsigned)blocks, kCastWarps * 32, smem, st>>>(
+        reinterpret_cast<const uint4*>(x), rows, (int)G, lpr_log2, exchange, reinterpret_cast<uint4*>(codes),
+        reinterpret_cast<uint16_t*>(scales), reinterpret_cast<uint4*>(pos), reinterpret_cast<uint4*>(neg), sf_pos, sf_neg,
+        row_exp, nk64, flushed_total);
+    return launch_status();
+}
+}  // namespace
+
+// codes may be nullptr: the canonical codes are then not written (the planes hold the same nibbles).
 int quantize_rows_prepared(const void* x, int64_t rows, int64_t K, uint8_t* codes, uint8_t* scales, void* pos,
                            void* neg, uint8_t* sf_pos, uint8_t* sf_neg, int* row_exp, int nk64, int64_t padded_rows,
                            cudaStream_t st, int format, int* flushed_total) {
     const int64_t G = K / 32;
-    // one thread per group when a row fits a block of 512, several rows per block when rows are short
-    const int gx = (int)((G < 512 ? G : 512) + 31) / 32 * 32;
-    int rb = 1;
-    while (rb < kPrepMaxRows && rb * 2 * gx <= 256) rb *= 2;
-    const int64_t blocks = (padded_rows + rb - 1) / rb;
-    if (blocks > 0x7FFFFFFF) return AMX_ERR_SHAPE;
-    auto* kernel = format == AMX_FMT_SYM_FP8 ? cast_prepared_kernel<1> : format == AMX_FMT_MXFP4 ? cast_prepared_kernel<2>
-                                                                                                  : cast_prepared_kernel<0>;
-    kernel<<<(unsigned)blocks, dim3(gx, rb), 0, st>>>(
-        reinterpret_cast<const uint4*>(x), rows, (int)G, reinterpret_cast<uint4*>(codes),
-        reinterpret_cast<uint16_t*>(scales), reinterpret_cast<uint4*>(pos), reinterpret_cast<uint4*>(neg), sf_pos, sf_neg,
-        row_exp, nk64, flushed_total);
-    return launch_status();
+    if (format == AMX_FMT_SYM_FP8)
+        return launch_cast_prepared<1>(x, rows, G, codes, scales, pos, neg, sf_pos, sf_neg, row_exp, nk64, padded_rows, st, flushed_total);
+    if (format == AMX_FMT_MXFP4)
+        return launch_cast_prepared<2>(x, rows, G, codes, scales, pos, neg, sf_pos, sf_neg, row_exp, nk64, padded_rows, st, flushed_total);
+    return launch_cast_prepared<0>(x, rows, G, codes, scales, pos, neg, sf_pos, sf_neg, row_exp, nk64, padded_rows, st, flushed_total);
 }
 
 // Softmax of the rows of S (fp32 [rows, ld_s], cols % 32 == 0), rounded to bf16 and cast, in one launch.  With

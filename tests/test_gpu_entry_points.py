@@ -192,3 +192,22 @@ def test_linear_host_with_explicit_kernel(flags):
     torch.cuda.synchronize()
     for o in outs:
         assert np.array_equal(o.numpy(), c.numpy())
+
+
+@pytest.mark.parametrize("rows,K,is_w", [(300, 1056, False), (130, 96, True), (77, 11008, False), (9, 36864, True), (2100, 128, True)])
+def test_quantize_prepared_without_canonical_codes(rows, K, is_w):
+    """The prepared cast with codes = NULL writes the same scales and the same prepared operand, byte for byte
+    (row lengths below, at and above a warp's 32 groups, and beyond the 32 groups per lane held in registers)."""
+    bits = inputs.random_groups(2000 + rows, rows, K, "mixed")
+    x = dev_bf16(bits)
+    nbytes = amx.lib().amx_prepared_bytes(rows, K, 32, int(is_w))
+    c, s1, p1 = amx.quantize_prepared(x, is_w, prepared=torch.zeros(nbytes, dtype=torch.uint8, device="cuda"))
+    none, s2, p2 = amx.quantize_prepared(x, is_w, prepared=torch.zeros(nbytes, dtype=torch.uint8, device="cuda"),
+                                         want_codes=False)
+    assert none is None and torch.equal(s1, s2) and torch.equal(p1, p2)
+    oc, os_ = oracle.quantize(bits, 32)
+    assert np.array_equal(c.cpu().numpy(), oc) and np.array_equal(s1.cpu().numpy(), os_)
+    # the positive and negative planes together are the codes
+    plane = -(-(rows * K // 2) // 256) * 256
+    planes = p1.cpu().numpy()
+    assert np.array_equal(planes[: rows * K // 2] | planes[plane: plane + rows * K // 2], oc.reshape(-1))
