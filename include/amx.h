@@ -255,8 +255,9 @@ int amx_softmax_quantize(const float* S, int64_t rows, int64_t cols, int64_t ld_
  * leave in 16 bits).  Per head h:
  *   S = AMX(Q_h) AMX(K_h)^T          groups along head_dim
  *   P = softmax(S / sqrt(d)) per row, fp32, rounded to bf16; no mask.  P itself is never stored.  When both
- *       products run on the FP4 kernel and L % 256 == 0, S is not stored either: Q K^T runs twice, the first
- *       pass keeps per-row softmax statistics, the second normalises and casts each tile in its epilogue
+ *       products run on the FP4 kernel, S is not stored either if d == 128 and L % 128 == 0 (one kernel per
+ *       pass does both products and the softmax) or L % 256 == 0: Q K^T runs twice, the first pass keeps
+ *       per-row softmax statistics, the second normalises and casts each tile in registers
  *       (row sums are then taken tile by tile, so single elements of P may round to the neighbouring bf16
  *       value compared with amx_softmax_quantize on a stored S; O agrees to ~1e-5 relative)
  *   O_h = AMX(P) AMX(V_h)            groups along the key axis (V is quantized down its rows)
@@ -274,22 +275,24 @@ int amx_attention(const void* q, const void* k, const void* v, int64_t heads, in
 size_t amx_attention_workspace_bytes(int64_t L, int64_t d);
 
 /*
- * amx_attention_map - the cast attention map of ONE head exactly as amx_attention builds it when it does not
- * store the logits (both products on the FP4 kernel, L % 256 == 0): P = softmax(Q K^T / sqrt(d)) per row,
- * rounded to bf16 and cast to AMXFP4 inside the epilogue of the second pass over Q K^T (Appendix C: the
- * self-attention map is quantized).  Same kernels, same launch sequence; in addition the epilogue stores what
- * amx_attention never writes, so that the cast can be checked against a reference:
+ * amx_attention_map - ONE head through the launch sequence amx_attention uses at head dimension 128 (both products
+ * on the FP4 kernel, logits and attention map never stored), with the intermediate the library otherwise never
+ * writes: the cast attention map.  P = softmax(Q K^T / sqrt(d)) per row, rounded to bf16 and cast to AMXFP4 in
+ * registers inside the second pass over Q K^T (Appendix C: the self-attention map is quantized), then multiplied
+ * with the cast V on the tensor cores in the same kernel.  Same kernels and launch sequence as amx_attention; in
+ * addition the second pass stores, so that the cast can be checked against a reference:
+ *   q, k, v     bf16 [L, d], d == 128, L % 128 == 0 (else AMX_ERR_SHAPE)
+ *   o           out fp32 [L, d]: the head's attention output, as amx_attention computes it
  *   p_bf16      out, nullable: bf16 [L, L], the normalised map as rounded to bf16 - the cast's input
  *   p_codes     out, nullable: canonical codes [L, L/2] of that map;  p_scales  out, nullable: [L, L/32, 2]
- *   p_prepared  out: the left-hand operand of P V in the FP4 kernel's form (positive plane, UE4M3 scale factors,
- *               row words), amx_prepared_bytes(L, L, 32, 0) bytes, 256-aligned
- *   flags       0 or AMX_ATTN_CAUSAL (blocks of keys entirely after their queries are not visited; their
- *               entries of the three optional outputs are zero)
+ *   p_prepared  out: P in the FP4 kernels' operand form as the kernel feeds it to the tensor cores (positive
+ *               plane, UE4M3 scale factors, row words), amx_prepared_bytes(L, L, 32, 0) bytes, 256-aligned
+ *   flags       0 or AMX_ATTN_CAUSAL (blocks of 128 keys entirely after their block of 128 queries are not visited;
+ *               their entries of the optional outputs are zero, those of p_prepared are not written)
  *   workspace   amx_attention_workspace_bytes(L, d) bytes
- * AMX_ERR_SHAPE when L % 256 != 0 or d % 32 != 0.
  */
-int amx_attention_map(const void* q, const void* k, int64_t L, int64_t d, uint32_t flags, void* p_bf16,
-                      uint8_t* p_codes, uint8_t* p_scales, void* p_prepared, size_t prepared_bytes,
+int amx_attention_map(const void* q, const void* k, const void* v, int64_t L, int64_t d, uint32_t flags, float* o,
+                      void* p_bf16, uint8_t* p_codes, uint8_t* p_scales, void* p_prepared, size_t prepared_bytes,
                       void* workspace, size_t workspace_bytes, void* stream);
 
 /*

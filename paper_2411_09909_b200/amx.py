@@ -62,7 +62,7 @@ def lib() -> ctypes.CDLL:
         L.amx_quant_error_workspace_bytes.argtypes = []
         L.amx_quant_error_workspace_bytes.restype = sz
         L.amx_quant_gemm.argtypes = [p, i64, p, p, p, i64, i64, i64, i64, i, u32, p, i64, p, sz, p]
-        L.amx_attention_map.argtypes = [p, p, i64, i64, u32, p, p, p, p, sz, p, sz, p]
+        L.amx_attention_map.argtypes = [p, p, p, i64, i64, u32, p, p, p, p, p, sz, p, sz, p]
         L.amx_gemm_flushed_scales.argtypes = [p, p]
         L.amx_gemm_flushed_scales.restype = i64
         L.amx_prepared_flushed_scales.argtypes = [p, i64, i64, i, i, p]
@@ -273,21 +273,23 @@ def prepared_flushed_scales(prepared: torch.Tensor, rows: int, K: int, is_weight
     return int(lib().amx_prepared_flushed_scales(prepared.data_ptr(), rows, K, group_size, int(is_weight), _stream()))
 
 
-def attention_map(q: torch.Tensor, k: torch.Tensor, flags: int = 0, want_bf16: bool = True):
-    """The cast attention map of one head as amx_attention builds it on its two-pass path.  q, k: bf16 [L, d].
-    Returns (p_bf16 or None, codes, scales, prepared)."""
-    _dev(q, torch.bfloat16, "q"), _dev(k, torch.bfloat16, "k")
-    assert q.is_contiguous() and k.is_contiguous() and q.shape == k.shape
+def attention_map(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, flags: int = 0, want_bf16: bool = True):
+    """One head through the attention kernels, with the cast attention map they otherwise never store.
+    q, k, v: bf16 [L, 128].  Returns (O fp32 [L, 128], p_bf16 or None, codes, scales, prepared)."""
+    for t in (q, k, v):
+        _dev(t, torch.bfloat16, "q/k/v")
+        assert t.is_contiguous() and t.shape == q.shape
     Lq, d = q.shape
+    out = torch.empty((Lq, d), dtype=torch.float32, device=q.device)
     p_bits = torch.empty((Lq, Lq), dtype=torch.bfloat16, device=q.device) if want_bf16 else None
     codes = torch.empty((Lq, Lq // 2), dtype=torch.uint8, device=q.device)
     scales = torch.empty((Lq, Lq // 32, 2), dtype=torch.uint8, device=q.device)
-    prep = _ws(lib().amx_prepared_bytes(Lq, Lq, 32, 0), q.device)
+    prep = torch.zeros(max(lib().amx_prepared_bytes(Lq, Lq, 32, 0), 256), dtype=torch.uint8, device=q.device)
     ws = _ws(lib().amx_attention_workspace_bytes(Lq, d), q.device)
-    _check(lib().amx_attention_map(q.data_ptr(), k.data_ptr(), Lq, d, flags, p_bits.data_ptr() if want_bf16 else None,
-                                   codes.data_ptr(), scales.data_ptr(), prep.data_ptr(), prep.numel(), ws.data_ptr(),
-                                   ws.numel(), _stream()), "amx_attention_map")
-    return p_bits, codes, scales, prep
+    _check(lib().amx_attention_map(q.data_ptr(), k.data_ptr(), v.data_ptr(), Lq, d, flags, out.data_ptr(),
+                                   p_bits.data_ptr() if want_bf16 else None, codes.data_ptr(), scales.data_ptr(),
+                                   prep.data_ptr(), prep.numel(), ws.data_ptr(), ws.numel(), _stream()), "amx_attention_map")
+    return out, p_bits, codes, scales, prep
 
 
 def softmax_bf16(S: torch.Tensor, alpha: float, out: torch.Tensor | None = None):

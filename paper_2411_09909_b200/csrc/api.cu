@@ -320,11 +320,14 @@ namespace {
 // scales of the chunk's Q, K and V^T and of one head's P, the logits S of one head, then either the prepared
 // operands of the FP4 kernel (Q and P as left-hand, K and V^T as right-hand operands) or the other kernels' own
 // scratch, and the status word.
-constexpr int64_t kAttnChunk = 8;
-int64_t attn_chunk(int64_t L, int64_t d) { return (L % 128 == 0 && d % 128 == 0) ? kAttnChunk : 1; }
+constexpr int64_t kAttnChunk = 8, kAttnChunkFused = 16;
+int64_t attn_chunk(int64_t L, int64_t d) {
+    if (attn_fused_supported(L, d)) return kAttnChunkFused;   // 16 x (L / 128) items: an even load for 148 persistent CTAs
+    return (L % 128 == 0 && d % 128 == 0) ? kAttnChunk : 1;
+}
 
 struct AttnLayout {
-    size_t qc, qs, kc, ks, vc, vs, pc, ps, S, pq, pk, pv, pp, gemm, total;
+    size_t qc, qs, kc, ks, vc, vs, pc, ps, S, pq, pk, pv, pp, stats, gemm, total;
 };
 AttnLayout attn_layout(int64_t L, int64_t d) {
     AttnLayout a;
@@ -340,6 +343,7 @@ AttnLayout attn_layout(int64_t L, int64_t d) {
     a.pk = take(gemm_fp4_prepared_bytes(hc * L + 128, d, true));
     a.pv = take(gemm_fp4_prepared_bytes(hc * d + 128, L, true));
     a.pp = take(gemm_fp4_prepared_bytes(L, L, false));
+    a.stats = take(attn_fused_supported(L, d) ? attn_fused_scratch_bytes(hc, L) : 0);
     a.gemm = off;
     const size_t g1 = amx_workspace_bytes(L, L, d, 32, AMX_GEMM_TC), g2 = amx_workspace_bytes(L, d, L, 32, AMX_GEMM_TC);
     a.total = off + (g1 > g2 ? g1 : g2) + 256;
@@ -374,7 +378,8 @@ extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_
     const int64_t chunk = attn_chunk(L, d);
     // both products on the FP4 kernel and whole 256-column tiles: softmax and cast run in the first product's
     // epilogue (the S region of the workspace then only holds the per-tile row statistics)
-    const bool two_pass = k_qk == AMX_GEMM_FP4 && k_pv == AMX_GEMM_FP4 && L % 256 == 0 &&
+    const bool fused = k_qk == AMX_GEMM_FP4 && k_pv == AMX_GEMM_FP4 && attn_fused_supported(L, d);
+    const bool two_pass = !fused && k_qk == AMX_GEMM_FP4 && k_pv == AMX_GEMM_FP4 && L % 256 == 0 &&
                           gemm_fp4_attn_scratch_bytes(L) <= (size_t)L * L * 4;
     // At head dimension 128 one head's P V has only L / 128 tiles: two heads' attention maps are cast into one
     // stacked operand (in the unused part of the S region, behind the statistics) and multiplied in one launch.
@@ -393,9 +398,9 @@ extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_
         // casts of the chunk's heads, stacked row-wise: Q and K along head_dim, V along the sequence (V^T)
         int rc;
         if (k_qk == AMX_GEMM_FP4) {
-            rc = gemm_fp4_quantize_prepared(qh, hc * L, d, false, w + a.qc, w + a.qs, w + a.pq, st, chunk * L);
+            rc = gemm_fp4_quantize_prepared(qh, hc * L, d, false, nullptr, w + a.qs, w + a.pq, st, chunk * L);
             if (rc == AMX_OK)
-                rc = gemm_fp4_quantize_prepared(kh, hc * L, d, true, w + a.kc, w + a.ks, w + a.pk, st, chunk * L + 128);
+                rc = gemm_fp4_quantize_prepared(kh, hc * L, d, true, nullptr, w + a.ks, w + a.pk, st, chunk * L + 128);
         } else {
             rc = amx_quantize(qh, hc * L, d, d, 32, w + a.qc, w + a.qs, stream);
             if (rc == AMX_OK) rc = amx_quantize(kh, hc * L, d, d, 32, w + a.kc, w + a.ks, stream);
@@ -404,6 +409,14 @@ extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_
         if (rc == AMX_OK && k_pv == AMX_GEMM_FP4)
             rc = gemm_fp4_prepare(w + a.vc, w + a.vs, hc * d, L, true, w + a.pv, st, chunk * d + 128);
         if (rc != AMX_OK) return rc;
+        if (fused) {
+            // head dimension 128: both products and the softmax of all the chunk's heads in two launches
+            rc = attn_fused({w + a.pq, hc * L, chunk * L, 0}, {w + a.pk, hc * L, chunk * L + 128, 0},
+                            {w + a.pv, hc * d, chunk * d + 128, 0}, (int)hc, L, alpha, causal, w + a.stats,
+                            o + (size_t)h0 * L * d, w + a.gemm, st);
+            if (rc != AMX_OK) return rc;
+            continue;
+        }
         for (int64_t i = 0; two_pass && i < hc; i += pair ? 2 : 1) {
             // the logits never reach memory: Q K^T runs twice, its epilogues do the softmax and the cast of P
             const int nb = pair && i + 1 < hc ? 2 : 1;
@@ -444,19 +457,17 @@ extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_
     return AMX_OK;
 }
 
-extern "C" int amx_attention_map(const void* q, const void* k, int64_t L, int64_t d, uint32_t flags, void* p_bf16,
-                                 uint8_t* p_codes, uint8_t* p_scales, void* p_prepared, size_t prepared_bytes,
-                                 void* workspace, size_t workspace_bytes, void* stream) {
+extern "C" int amx_attention_map(const void* q, const void* k, const void* v, int64_t L, int64_t d, uint32_t flags,
+                                 float* o, void* p_bf16, uint8_t* p_codes, uint8_t* p_scales, void* p_prepared,
+                                 size_t prepared_bytes, void* workspace, size_t workspace_bytes, void* stream) {
     const int causal = (flags & AMX_ATTN_CAUSAL) ? 1 : 0;
     if (flags & ~AMX_ATTN_CAUSAL) return AMX_ERR_FLAGS;
-    if (L <= 0 || d <= 0 || L % 256 || d % 32 || !gemm_fp4_supported(L, L, d, 32) ||
-        gemm_fp4_attn_scratch_bytes(L) > (size_t)L * L * 4)
-        return AMX_ERR_SHAPE;
-    if (!q || !k || !p_prepared) return AMX_ERR_NULL;
+    if (L <= 0 || d <= 0 || !attn_fused_supported(L, d)) return AMX_ERR_SHAPE;
+    if (!q || !k || !v || !o || !p_prepared) return AMX_ERR_NULL;
     const AttnLayout a = attn_layout(L, d);
     if (!workspace || workspace_bytes < a.total || prepared_bytes < amx_prepared_bytes(L, L, 32, 0)) return AMX_ERR_WORKSPACE;
-    if (!aligned(workspace, kAlign) || !aligned(q, 16) || !aligned(k, 16) || !aligned(p_prepared, kAlign) ||
-        !aligned(p_bf16, 16) || !aligned(p_codes, 16) || !aligned(p_scales, 2))
+    if (!aligned(workspace, kAlign) || !aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16) ||
+        !aligned(p_prepared, kAlign) || !aligned(p_bf16, 16) || !aligned(p_codes, 16) || !aligned(p_scales, 2))
         return AMX_ERR_ALIGN;
     uint8_t* w = static_cast<uint8_t*>(workspace);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -467,11 +478,15 @@ extern "C" int amx_attention_map(const void* q, const void* k, int64_t L, int64_
             (p_scales && cudaMemsetAsync(p_scales, 0, (size_t)L * (L / 32) * 2, st) != cudaSuccess))
             return AMX_ERR_CUDA;
     }
-    int rc = gemm_fp4_quantize_prepared(q, L, d, false, w + a.qc, w + a.qs, w + a.pq, st);
-    if (rc == AMX_OK) rc = gemm_fp4_quantize_prepared(k, L, d, true, w + a.kc, w + a.ks, w + a.pk, st);
+    // one head through the launch sequence of amx_attention: casts of Q, K (along head_dim) and V (along the
+    // sequence), then the two passes
+    int rc = gemm_fp4_quantize_prepared(q, L, d, false, nullptr, w + a.qs, w + a.pq, st);
+    if (rc == AMX_OK) rc = gemm_fp4_quantize_prepared(k, L, d, true, nullptr, w + a.ks, w + a.pk, st);
+    if (rc == AMX_OK) rc = quantize_cols_batched(v, 1, L, d, w + a.vc, w + a.vs, st);
+    if (rc == AMX_OK) rc = gemm_fp4_prepare(w + a.vc, w + a.vs, d, L, true, w + a.pv, st);
     if (rc != AMX_OK) return rc;
-    return gemm_fp4_attn_scores({w + a.pq, L, L, 0}, {w + a.pk, L, L, 0}, L, d, 1.0f / sqrtf((float)d), w + a.S, p_codes,
-                                p_scales, p_prepared, w + a.gemm, st, causal, L, 0, p_bf16);
+    return attn_fused({w + a.pq, L, L, 0}, {w + a.pk, L, L, 0}, {w + a.pv, d, d, 0}, 1, L, 1.0f / sqrtf((float)d), causal,
+                      w + a.stats, o, w + a.gemm, st, p_bf16, p_codes, p_scales, p_prepared);
 }
 
 extern "C" int amx_gemm_status(const void* workspace, void* stream) {

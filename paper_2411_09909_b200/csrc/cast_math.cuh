@@ -129,6 +129,17 @@ __device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b) {
     asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+    uint32_t l, h;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(l), "=r"(h) : "l"(v));
+    lo = __uint_as_float(l);
+    hi = __uint_as_float(h);
+}
 // Four packed pairs of quotients -> eight E2M1 nibbles; element i lands in nibble i.
 __device__ __forceinline__ uint32_t cvt_e2m1x8(uint64_t q0, uint64_t q1, uint64_t q2, uint64_t q3) {
     uint32_t d;
@@ -221,12 +232,10 @@ __device__ __forceinline__ uint32_t emit_group(const uint32_t (&w)[16], int64_t 
     return FMT ? (sc & 0xFFu) : sc;
 }
 
-// The same for a group without negative elements (a softmax output) when only the FP4 GEMM's operand is wanted:
+// The cast of a group without negative elements (a softmax output) when only the FP4 kernels' operand is wanted:
 // its positive sign plane is its code word, the negative plane and scale are zero.  Same arithmetic as above,
-// minus everything the negative side needs.  Stores the plane at group index v (and, when asked, the same word as
-// the group's canonical codes: without a set sign bit the two are equal), returns the positive scale byte.
-__device__ __forceinline__ uint32_t emit_nonneg_plane(const uint32_t (&w)[16], int64_t v, uint4* __restrict__ plane,
-                                                      uint4* __restrict__ codes = nullptr) {
+// minus everything the negative side needs.  nib: the group's 32 codes; returns the positive scale byte.
+__device__ __forceinline__ uint32_t cast_nonneg_group(const uint32_t (&w)[16], uint32_t (&nib)[4]) {
     uint32_t pm = w[0];
 #pragma unroll
     for (int i = 1; i + 1 < 16; i += 2) pm = __vimax3_s16x2(pm, w[i], w[i + 1]);
@@ -235,9 +244,16 @@ __device__ __forceinline__ uint32_t emit_nonneg_plane(const uint32_t (&w)[16], i
     const uint32_t sc = cvt_e5m2x2(0.0f, trunc12(__uint_as_float(pm << 16) * sixth_up())) & 0xFFu;
     const uint32_t inv = __float_as_uint(inv_scale(sc));
     const uint64_t inv2 = pack_f32x2(inv, inv);
-    uint32_t nib[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) nib[j] = encode8_one(w + 4 * j, inv2);
+    return sc;
+}
+// Stores the plane at group index v (and, when asked, the same word as the group's canonical codes: without a set
+// sign bit the two are equal), returns the positive scale byte.
+__device__ __forceinline__ uint32_t emit_nonneg_plane(const uint32_t (&w)[16], int64_t v, uint4* __restrict__ plane,
+                                                      uint4* __restrict__ codes = nullptr) {
+    uint32_t nib[4];
+    const uint32_t sc = cast_nonneg_group(w, nib);
     plane[v] = make_uint4(nib[0], nib[1], nib[2], nib[3]);
     if (codes) codes[v] = make_uint4(nib[0], nib[1], nib[2], nib[3]);
     return sc;

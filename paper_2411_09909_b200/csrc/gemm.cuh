@@ -86,6 +86,13 @@ int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, in
                          int causal = 0, int64_t p_layout_rows = 0 /* 0: L */, int64_t p_row0 = 0,
                          void* p_bits = nullptr /* optional out: the bf16 map the cast started from, [L, L] */);
 // p_codes / p_scales may be NULL as well: only the prepared operand is written then.
+// Fused attention for head dimension 128 (attention_fp4.cu): both products and the softmax in two launches, logits
+// and attention map never in global memory.  Operands prepared ahead, heads stacked row-wise.
+bool attn_fused_supported(int64_t L, int64_t d);
+size_t attn_fused_scratch_bytes(int64_t heads, int64_t L);
+int attn_fused(const Fp4Operand& q, const Fp4Operand& k, const Fp4Operand& vt, int heads, int64_t L, float alpha, int causal,
+               void* scratch, float* O, void* workspace /* 256 B: status word */, cudaStream_t st, void* dbg_bits = nullptr,
+               uint8_t* dbg_codes = nullptr, uint8_t* dbg_scales = nullptr, void* dbg_prepared = nullptr);
 int quantize_cols_batched(const void* x, int64_t batch, int64_t R, int64_t C, uint8_t* codes, uint8_t* scales,
                           cudaStream_t st);
 int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,

@@ -29,12 +29,10 @@
 // A preparation kernel per operand derives the planes, the UE4M3 scale-factor
 // blocks in the 128 x 4 interleaved layout the MMA reads, and the row offsets from the canonical
 // codes and scales.  Every device-side wait is bounded.
-#include <cuda.h>
-
 #include <cstdlib>
-#include <mutex>
 
 #include "cast_math.cuh"
+#include "fp4_operand.cuh"
 #include "gemm.cuh"
 #include "softmax_math.cuh"
 #include "tcgen05.cuh"
@@ -43,11 +41,11 @@ namespace amx {
 namespace {
 
 using namespace tc;
+using namespace fp4;
 
 constexpr int BM = 128, BN = 256;
 constexpr int kSfGroups = 2, kSfWarps = 4 * kSfGroups, kEpilogueWarps = 8;
 constexpr int kThreads = (2 + kSfWarps + kEpilogueWarps) * 32;
-constexpr int kSfChunk = 512;           // scale factors of 128 rows x 64 elements (4 per row)
 constexpr int kTmemCols = 512;
 constexpr uint32_t kTmemSf = 256;      // scale-factor columns follow the 256 accumulator columns
 
@@ -684,57 +682,6 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 }
 
 // ---------------------------------------------------------------------------------- host --
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled() {
-    static EncodeTiledFn fn = nullptr;
-    static std::once_flag once;
-    std::call_once(once, [] {
-        void* f = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(f);
-    });
-    return fn;
-}
-
-// Both sign planes of an operand as one 3-D tensor [2][rows][K/2] of bytes (plane_stride bytes apart);
-// box = {row_bytes, box_rows, 2}, 128- or 64-byte swizzle, zero fill outside.
-bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t K, size_t plane_stride, int box_rows,
-              int row_bytes, int planes = 2) {
-    EncodeTiledFn fn = encode_tiled();
-    if (!fn) return false;
-    const cuuint64_t dims[3] = {(cuuint64_t)(K / 2), (cuuint64_t)rows, 2};
-    const cuuint64_t strides[2] = {(cuuint64_t)(K / 2), (cuuint64_t)plane_stride};
-    const cuuint32_t box[3] = {(cuuint32_t)row_bytes, (cuuint32_t)box_rows, (cuuint32_t)planes};   // 1: positive plane only
-    const cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-inline size_t up256(size_t v) { return (v + 255) / 256 * 256; }
-
-struct OperandLayout {      // offsets inside the workspace of one prepared operand
-    size_t plane, sf, exps, total;
-    int64_t row_blocks;
-    int nk64;
-};
-OperandLayout operand_layout(int64_t rows, int64_t K, int rows_per_tile) {
-    OperandLayout o;
-    o.row_blocks = (rows + rows_per_tile - 1) / rows_per_tile * (rows_per_tile / 128);
-    o.nk64 = (int)((K + 255) / 256) * 4;    // padded to whole 256-element blocks
-    o.plane = up256((size_t)rows * (K / 2));
-    o.sf = up256((size_t)o.row_blocks * o.nk64 * kSfChunk);
-    o.exps = up256((size_t)rows * 4);      // row offsets
-    o.total = 2 * o.plane + 2 * o.sf + o.exps;
-    return o;
-}
-
 int prepare(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K, const OperandLayout& o,
             uint8_t* base, cudaStream_t st, int* flushed_total = nullptr) {
     const int64_t padded_rows = o.row_blocks * 128;

@@ -74,8 +74,11 @@ def test_host_detected_argument_errors(L):
     assert qg(fake, 64, None, None, odd, 64, 4, 4, 64, 32, 0x10, fake, 4, fake, 1 << 20, None) == -3    # bf16 weight alignment
     assert L.amx_linear_host(fake, fake, 4, 4, 64, 32, 0x30, fake, fake, 1 << 30, None) == -5             # two kernels
     assert L.amx_linear_host(fake, fake, 4, 4, 64, 32, 0x40, fake, fake, 16, None) == -4                  # checked before any copy
-    assert L.amx_attention_map(fake, fake, 320, 128, 0, fake, fake, fake, fake, 1 << 30, fake, 1 << 30, None) == -2   # L % 256
-    assert L.amx_attention_map(fake, fake, 512, 128, 0x40, fake, fake, fake, fake, 1 << 30, fake, 1 << 30, None) == -5
+    am = L.amx_attention_map
+    assert am(fake, fake, fake, 320, 128, 0, fake, fake, fake, fake, fake, 1 << 30, fake, 1 << 30, None) == -2   # L % 128
+    assert am(fake, fake, fake, 512, 64, 0, fake, fake, fake, fake, fake, 1 << 30, fake, 1 << 30, None) == -2    # d != 128
+    assert am(fake, fake, fake, 512, 128, 0x40, fake, fake, fake, fake, fake, 1 << 30, fake, 1 << 30, None) == -5
+    assert am(fake, fake, None, 512, 128, 0, fake, fake, fake, fake, fake, 1 << 30, fake, 1 << 30, None) == -1
     assert L.amx_prepared_flushed_scales(None, 4, 64, 32, 0, None) == -1
     assert L.amx_prepared_flushed_scales(fake, 4, 64, 16, 0, None) == -2
     assert L.amx_selftest_wait_timeout(fake, 64, 100, None) == -4

@@ -1,8 +1,10 @@
-"""The cast of the attention map inside the second Q K^T pass (the path full-size attention runs): the kernel's
-own bf16 map, fed to the oracle quantizer, must give the kernel's codes and scales bit for bit; the positive
-plane of the prepared operand must equal the codes, its UE4M3 scale factors a host-side conversion of the
-oracle's scales, and no scale may be flushed.  The map itself is checked against the all-CPU pipeline (fp32
-exp on the device against fp64 on the host: single bf16 roundings differ)."""
+"""The cast of the attention map inside the fused attention kernel (the path full-size attention runs): the
+kernel's own bf16 map, fed to the oracle quantizer, must give the kernel's codes and scales bit for bit; the
+positive plane it feeds to the tensor cores must equal the codes, its UE4M3 scale factors a host-side conversion
+of the oracle's scales, and no scale may be flushed.  The map itself is checked against the all-CPU pipeline
+(fp32 exp on the device against fp64 on the host: single bf16 roundings differ), and the output O - computed by
+the same kernel from the map it never stores - against the oracle's product of the kernel's own quantized map
+with the quantized V."""
 import numpy as np
 import pytest
 import torch
@@ -43,10 +45,10 @@ def check_rows(rows, L, p_bits, codes, scales, prep, causal):
     sf_bytes = (L // 128) * nk64 * 512
     plane = prep[: L * L // 2].reshape(L, L // 2)
     G = L // 32
-    if causal:          # blocks of 256 keys entirely after the query's block of 128 are never visited nor read
-        for r in rows:
-            seen = (r // 128 // 2 + 1) * 256 // 2
-            assert np.array_equal(plane[r, :seen], oc[list(rows).index(r), :seen])
+    if causal:          # blocks of 128 keys entirely after the query's block of 128 are never visited nor read
+        for i, r in enumerate(rows):
+            seen = (r // 128 + 1) * 128 // 2
+            assert np.array_equal(plane[r, :seen], oc[i, :seen])
     else:
         assert np.array_equal(plane[rows], oc)
     sf = prep[2 * plane_bytes: 2 * plane_bytes + sf_bytes]
@@ -57,20 +59,32 @@ def check_rows(rows, L, p_bits, codes, scales, prep, causal):
     assert np.all((words[rows] >> 16) & 3 == 1) and np.all(words[rows] >> 18 == 0)   # positive side only, nothing flushed
     want = expected_scale_factors(os_[:, :, 0], kmax)
     for i, r in enumerate(rows):
-        g = np.arange(G if not causal else (r // 128 // 2 + 1) * 8)
+        g = np.arange(G if not causal else (r // 128 + 1) * 4)
         off = (r // 128) * nk64 * 512 + (g // 2) * 512 + (r % 32) * 16 + ((r % 128) // 32) * 4 + (g % 2) * 2
         assert np.array_equal(sf[off], want[i, g]) and np.array_equal(sf[off + 1], want[i, g]), r
 
 
+def check_output(o, rows, codes, scales, vb):
+    """O of the sampled rows against the oracle's product of the kernel's own quantized map with the quantized V."""
+    vq = oracle.quantize(np.ascontiguousarray(vb.T), 32)
+    ref = oracle.gemm(np.ascontiguousarray(codes[rows]), np.ascontiguousarray(scales[rows]), *vq, 32)
+    got = o[rows].astype(np.float64)
+    assert np.linalg.norm(got - ref) <= 1e-5 * np.linalg.norm(ref)
+
+
+@pytest.mark.parametrize("L", [128, 384, 512])
 @pytest.mark.parametrize("causal", [False, True])
-def test_attention_map_cast_bit_exact_small(causal):
-    L = 512
-    qb, kb, _ = (t[0] for t in inputs.attention_qkv(heads=1, seq=L))
+def test_attention_map_cast_bit_exact_small(L, causal):
+    qb, kb, vb = (t[0] for t in inputs.attention_qkv(heads=1, seq=L))
     flags = amx.ATTN_CAUSAL if causal else 0
-    p, c, s, prep = amx.attention_map(dev_bf16(qb), dev_bf16(kb), flags)
+    o, p, c, s, prep = amx.attention_map(dev_bf16(qb), dev_bf16(kb), dev_bf16(vb), flags)
     p_bits = p.view(torch.int16).cpu().numpy().view(np.uint16)
     check_rows(np.arange(L), L, p_bits, c.cpu().numpy(), s.cpu().numpy(), prep.cpu().numpy(), causal)
+    check_output(o.cpu().numpy(), np.arange(L), c.cpu().numpy(), s.cpu().numpy(), vb)
     assert amx.prepared_flushed_scales(prep, L, L, False) == 0
+    # amx_attention gives the same output for the head (same kernels)
+    heads = amx.attention_heads(dev_bf16(qb)[None], dev_bf16(kb)[None], dev_bf16(vb)[None], flags=flags | amx.GEMM_FP4)
+    assert torch.equal(heads[0], o)
     # the map itself against the all-CPU pipeline: equal up to one bf16 ulp on a small share of the entries
     S = oracle.gemm(*oracle.quantize(qb, 32), *oracle.quantize(kb, 32), 32)
     want = oracle.softmax_bf16(S, 128 ** -0.5, causal_row0=0) if causal else oracle.softmax_bf16(S, 128 ** -0.5)
@@ -84,25 +98,28 @@ def test_attention_map_softer_rows_bit_exact():
     """Inputs scaled down so that rows of the map hold many nonzero groups of very different size (the benchmark's
     inputs make it nearly one-hot): exercises the scale-factor range of the cast."""
     L = 512
-    qb, kb, _ = (t[0] for t in inputs.attention_qkv(heads=1, seq=L))
+    qb, kb, vb = (t[0] for t in inputs.attention_qkv(heads=1, seq=L))
     small = lambda b: inputs.f32_to_bf16_bits(inputs.bf16_bits_to_f32(b) * 0.35)
     qb, kb = small(qb), small(kb)
-    p, c, s, prep = amx.attention_map(dev_bf16(qb), dev_bf16(kb), 0)
+    o, p, c, s, prep = amx.attention_map(dev_bf16(qb), dev_bf16(kb), dev_bf16(vb), 0)
     p_bits = p.view(torch.int16).cpu().numpy().view(np.uint16)
     assert np.mean(s.cpu().numpy()[:, :, 0] != 0) > 0.5
     check_rows(np.arange(L), L, p_bits, c.cpu().numpy(), s.cpu().numpy(), prep.cpu().numpy(), False)
+    check_output(o.cpu().numpy(), np.arange(L), c.cpu().numpy(), s.cpu().numpy(), vb)
 
 
 @pytest.mark.parametrize("causal", [False, True])
 def test_attention_map_cast_bit_exact_full_size_sampled(causal):
     """Config-5 size (8192 keys): three sampled blocks of 128 query rows of head 0."""
     L = 8192
-    qb, kb, _ = (t[0] for t in inputs.attention_qkv(heads=1, seq=L))
+    qb, kb, vb = (t[0] for t in inputs.attention_qkv(heads=1, seq=L))
     flags = amx.ATTN_CAUSAL if causal else 0
-    p, c, s, prep = amx.attention_map(dev_bf16(qb), dev_bf16(kb), flags)
+    o, p, c, s, prep = amx.attention_map(dev_bf16(qb), dev_bf16(kb), dev_bf16(vb), flags)
     p_bits = p.view(torch.int16).cpu().numpy().view(np.uint16)
     rng = np.random.default_rng(77)
     blocks = np.sort(rng.choice(L // 128, size=3, replace=False))
     rows = np.concatenate([np.arange(b * 128, b * 128 + 128) for b in blocks])
-    check_rows(rows, L, p_bits, c.cpu().numpy(), s.cpu().numpy(), prep.cpu().numpy(), causal)
+    c_np, s_np = c.cpu().numpy(), s.cpu().numpy()
+    check_rows(rows, L, p_bits, c_np, s_np, prep.cpu().numpy(), causal)
+    check_output(o.cpu().numpy(), rows[::4], c_np, s_np, vb)
     assert amx.prepared_flushed_scales(prep, L, L, False) == 0

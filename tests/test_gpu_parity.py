@@ -626,7 +626,7 @@ def test_attention_small_head_against_oracle_pipeline():
 def test_attention_all_heads_entry_point_matches_per_head_pipeline(heads, seq, flags):
     q, k, v = (dev_bf16(t) for t in inputs.attention_qkv(heads=heads, seq=seq))
     O = amx.attention_heads(q, k, v, flags=flags)
-    two_pass = seq % 256 == 0 and amx.lib().amx_gemm_kernel_for(seq, seq, 128, 32, flags) == amx.GEMM_FP4
+    two_pass = seq % 128 == 0 and amx.lib().amx_gemm_kernel_for(seq, seq, 128, 32, flags) == amx.GEMM_FP4
     for h in range(heads):
         Oh, _ = amx.attention(q[h], k[h], v[h], flags=flags)
         if two_pass:
