@@ -14,12 +14,15 @@
 // One persistent CTA per SM walks over (head, block of 128 queries) items; per item it loops over the key tiles:
 //   warp 0      TMA: the item's Q tile; per key tile the K tile and (pass 2) the V^T tile, {+, -} planes each, into a
 //               ring of kStages stages
-//   warp 1      issues the MMAs one key tile ahead: S(j+1) is issued before the wait for P(j), so the tensor cores
+//   warp 1      issues the MMAs two key tiles ahead: S(j+2) is issued before the wait for P(j), so the tensor cores
 //               work on the next logits while the epilogue warps turn the current ones into P
 //   warps 2-5   scale factors of Q, K, V^T: global -> registers -> tensor memory (tcgen05.st), and the per-key column
 //               factors alpha * log2(e) * 2^(K row offset) of the tile
-//   warps 6-21  epilogue: thread = (query row, one group of 32 keys); tensor memory -> registers (two S accumulators
-//               alternate; released right after the load), softmax arithmetic, the cast, stores to shared memory
+//   warps 6-21  epilogue, two groups of eight warps: group g takes the key tiles with (tile count) % 2 == g from the S
+//               accumulator g, so the two groups are in different phases of their tiles (tensor-memory loads and
+//               maxima in one, exponentials in the other) and keep both the issue slots and the special-function
+//               unit busy; a thread owns one query row and 64 keys of its tiles: tensor memory -> registers (the
+//               accumulator is released right after the loads), softmax arithmetic, the cast, stores to shared memory
 //   after the last key tile of an item the epilogue warps read out O, rescale by the rows' powers of two and store.
 // Tensor memory: S0, S1, O (128 columns each), scale factors of Q (16), of kStages K/V^T stages (32 each), of the
 // two P tiles (8 each): 512 columns.  Every wait is bounded; on a timeout all roles run their loops out without
@@ -39,6 +42,9 @@ using namespace fp4;
 
 constexpr int BM = 128, BNK = 128, HD = 128;         // queries per item, keys per tile, head dimension
 constexpr int kStages = 3;
+// Ring of the per-tile column factors: its writers (scale-factor warps) run at most kStages tiles ahead of the MMAs
+// and those at most 2 tiles ahead of the readers (epilogue), so 8 slots never collide and need no barrier of their own.
+constexpr int kKcRing = 8;
 constexpr int kSfWarps = 4, kEpiWarps = 16;
 constexpr int kThreads = (2 + kSfWarps + kEpiWarps) * 32;
 constexpr int kPlane = 128 * 64;                      // one sign plane of a 128 x 128 tile: 64-byte rows
@@ -62,7 +68,7 @@ struct Smem {
     static constexpr int kOffP = kOffKV + kStages * kStageBytes;                  // two P planes (pass 2)
     static constexpr int kOffSfP = kOffP + (PASS == 2 ? 2 * kPlane : 0);          // two buffers x two 512-byte chunks
     static constexpr int kOffKc = kOffSfP + (PASS == 2 ? 2 * 2 * 512 : 0);        // per stage: 128 column factors
-    static constexpr int kOffCtl = kOffKc + kStages * 512;
+    static constexpr int kOffCtl = kOffKc + kKcRing * 512;
     static constexpr int kBytes = kOffCtl + 512 + 1024;                           // + Control + alignment slack
 };
 static_assert(sizeof(Control) <= 512, "Control must fit its reserved space");
@@ -118,13 +124,12 @@ attention_fp4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         mbar_init(&ctl->q_empty, 1);
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&ctl->kv_full[s], 1 + kSfWarps);
-            // pass 1: the stage (its column factors) is also released by the epilogue warps that read them
-            mbar_init(&ctl->kv_empty[s], PASS == 1 ? 1 + kEpiWarps : 1);
+            mbar_init(&ctl->kv_empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&ctl->s_full[b], 1);
-            mbar_init(&ctl->s_empty[b], kEpiWarps);
-            mbar_init(&ctl->p_full[b], kEpiWarps);
+            mbar_init(&ctl->s_empty[b], kEpiWarps / 2);          // the accumulator's own epilogue group
+            mbar_init(&ctl->p_full[b], kEpiWarps / 2);
             mbar_init(&ctl->p_empty[b], 1);
         }
         mbar_init(&ctl->o_full, 1);
@@ -234,12 +239,18 @@ attention_fp4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         for (int id = blockIdx.x; id < n_items; id += gridDim.x, ++ii) {
             const int T = tiles_of(item_m(id));
             if (ok) ok = mbar_wait(&ctl->q_full, ii & 1, &ctl->abort, p.status);
-            issue_s(it_s++);
-            for (int j = 0; j < T; ++j) {
-                if (j + 1 < T) issue_s(it_s++);
-                else if (ok && elect_one()) mma_commit(&ctl->q_empty);       // all logits MMAs of the item are issued
+            // the logits run two key tiles ahead of P V (both accumulators in use); after the item's last S the Q
+            // tile is free for the next item
+            auto next_s = [&](int j) {
+                if (j < T) issue_s(it_s++);
+                if (j == T - 1 && ok && elect_one()) mma_commit(&ctl->q_empty);
                 __syncwarp();
+            };
+            next_s(0);
+            next_s(1);
+            for (int j = 0; j < T; ++j) {
                 if (PASS == 2) issue_pv(it_p++, j == 0);
+                next_s(j + 2);
             }
             if (PASS == 2 && ok && elect_one()) mma_commit(&ctl->o_full);
             __syncwarp();
@@ -287,7 +298,7 @@ attention_fp4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (ok && it >= kStages) ok = mbar_wait(&ctl->kv_empty[s], ((it / kStages) - 1) & 1, &ctl->abort, p.status);
                 if (!ok) continue;
                 tc_fence_after();
-                kc_all[s * 128 + t] = p.alpha * 1.4426950408889634f * __uint_as_float((uint32_t)(kw + 127) << 23);
+                kc_all[(it % kKcRing) * 128 + t] = p.alpha * 1.4426950408889634f * __uint_as_float((uint32_t)(kw + 127) << 23);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) tmem_st4(tq + kColSfKV + s * 32 + i * 4, vk[i].x, vk[i].y, vk[i].z, vk[i].w);
                 if (PASS == 2) {
@@ -302,9 +313,10 @@ attention_fp4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         }
     } else {
         // ---------------------------------------------------------------------------------- epilogue
-        // Warp e: lane quarter q = warp % 4 (its rows), key group cg = e / 4 of the tile (32 columns): a thread owns
-        // one query row and one 32-key group per key tile.
-        const int e = warp - (2 + kSfWarps), q = warp & 3, cg = e >> 2;
+        // Warp e: group g = e / 8 (the key tiles whose global count is g modulo 2, accumulator g), lane quarter
+        // q = warp % 4 (its rows), half = (e / 4) % 2 of the tile's 128 keys: a thread owns one query row and two
+        // 32-key groups (64 columns) of each of its group's tiles.  For reading out O every warp takes 32 columns.
+        const int e = warp - (2 + kSfWarps), q = warp & 3, grp = e >> 3, half = (e >> 2) & 1, cg_o = e >> 2;
         const int r = q * 32 + lane;                                 // row inside the item = tensor-memory lane
         const uint32_t tq = tmem + ((uint32_t)(q * 32) << 16);
         int it = 0, ii = 0;
@@ -337,102 +349,130 @@ attention_fp4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 float ip, in;
                 const uint32_t sc = cast::group_scales((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(inv)), ip, in);
                 kmax = scale_key(sc & 0xFFu);
-                if (p.p_words && h == 0 && cg == 0) p.p_words[m] = row_word(kmax, kRowHasPos);
+                if (p.p_words && h == 0 && (e >> 2) == 0) p.p_words[m] = row_word(kmax, kRowHasPos);
             }
-            float run_mx = -INFINITY, run_sum = 0.f;                  // pass 1
+            float run_mx = -INFINITY, run_sum = 0.f;                  // pass 1: over this thread's columns of its tiles
             const int T = tiles_of(m_blk);
             for (int j = 0; j < T; ++j, ++it) {
-                const int s = it % kStages, b = it & 1;
+                if ((it & 1) != grp) continue;                        // the other group's tile
+                const int b = grp;
                 if (ok) ok = mbar_wait(&ctl->s_full[b], (it >> 1) & 1, &ctl->abort, p.status);
                 if (!ok) continue;
                 tc_fence_after();
-                uint32_t acc[32];
-                tmem_ld32(tq + kColS + b * 128 + cg * 32, acc);
-                tmem_ld_wait();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&ctl->s_empty[b]);       // the accumulator may be overwritten
-                // the stage's column factors were stored before the scale-factor warps arrived on its barrier
-                // (complete since before the MMAs): acquire them
-                mbar_wait(&ctl->kv_full[s], (it / kStages) & 1, &ctl->abort, p.status);
-                const float4* kc4 = reinterpret_cast<const float4*>(kc_all + s * 128 + cg * 32);
-                // u = accumulator x (alpha log2(e) 2^(K row offset)): the logit in base-2 units up to the query
-                // row's power of two ra, by which multiplying is exact: t = u ra
-                float u[32];
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const float4 k4 = kc4[c];
-                    cast::unpack_f32x2(cast::mul_f32x2(cast::pack_f32x2(acc[4 * c], acc[4 * c + 1]),
-                                                       cast::pack_f32x2(__float_as_uint(k4.x), __float_as_uint(k4.y))),
-                                       u[4 * c], u[4 * c + 1]);
-                    cast::unpack_f32x2(cast::mul_f32x2(cast::pack_f32x2(acc[4 * c + 2], acc[4 * c + 3]),
-                                                       cast::pack_f32x2(__float_as_uint(k4.z), __float_as_uint(k4.w))),
-                                       u[4 * c + 2], u[4 * c + 3]);
-                }
-                if (PASS == 1) {                                      // the column factors are in registers: release the stage
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&ctl->kv_empty[s]);
-                }
-                if (CAUSAL && p.causal && j == m_blk) {                // the diagonal tile: keys after the query are masked
-                    const int n_local = (int)(m - (int64_t)j * BNK) - cg * 32;   // last visible column of this group
-#pragma unroll
-                    for (int c = 0; c < 32; ++c)
-                        if (c > n_local) u[c] = -INFINITY;
-                }
-                if (PASS == 1) {
-                    float c4[4] = {u[0], u[1], u[2], u[3]};
-#pragma unroll
-                    for (int c = 4; c < 32; ++c) c4[c & 3] = fmaxf(c4[c & 3], u[c]);
-                    const float cm = fmaxf(fmaxf(c4[0], c4[1]), fmaxf(c4[2], c4[3]));
-                    const float nmx = fmaxf(run_mx, cm * ra);
-                    // 2^(-inf) = 0 on the first tile; a maximum still at -inf (everything masked so far) must not
-                    // meet itself in a difference
-                    const float ref = nmx == -INFINITY ? 0.f : nmx;
-                    run_sum *= exp2_approx(run_mx - ref);
-                    run_mx = nmx;
-                    float s4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) s4[c & 3] += exp2_approx(fmaf(u[c], ra, -ref));
-                    run_sum += (s4[0] + s4[1]) + (s4[2] + s4[3]);
-                } else {
-                    // normalise, round to bf16, cast (P has no negative element: one plane)
-                    uint32_t w[16];
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        const __nv_bfloat162 pr = __floats2bfloat162_rn(exp2_approx(fmaf(u[2 * c], ra, neg_mx)) * inv,
-                                                                        exp2_approx(fmaf(u[2 * c + 1], ra, neg_mx)) * inv);
-                        w[c] = *reinterpret_cast<const uint32_t*>(&pr);
-                    }
-                    uint32_t nib[4];
-                    const uint32_t sc = cast::cast_nonneg_group(w, nib);
-                    const uint32_t up = to_ue4m3(sc, kmax);
-                    // the previous P in this buffer has been multiplied
-                    if (it >= 2) ok = mbar_wait(&ctl->p_empty[b], ((it >> 1) - 1) & 1, &ctl->abort, p.status);
+                // (the tile's column factors were stored before the scale-factor warps arrived on the stage's barrier,
+                // which the MMA warp waited for before it issued what s_full reports as complete)
+                if (PASS == 2 && it >= 2) {                           // the previous P in this buffer has been multiplied
+                    ok = mbar_wait(&ctl->p_empty[b], ((it >> 1) - 1) & 1, &ctl->abort, p.status);
                     if (!ok) continue;
-                    // plane: row r, 16-byte piece cg of its 64 bytes, 64-byte swizzle; scale factors: chunk of the
-                    // K step cg / 2, byte (r % 32) * 16 + (r / 32) * 4 + (cg % 2) * 2, each scale twice (blocks of 16)
-                    *reinterpret_cast<uint4*>(sm + S_::kOffP + b * kPlane + r * 64 + ((cg ^ ((r >> 1) & 3)) << 4)) =
-                        make_uint4(nib[0], nib[1], nib[2], nib[3]);
-                    *reinterpret_cast<uint16_t*>(sm + S_::kOffSfP + (b * 2 + (cg >> 1)) * 512 + (r & 31) * 16 + (r >> 5) * 4 +
-                                                 (cg & 1) * 2) = (uint16_t)(up | (up << 8));
+                }
+                // u = accumulator x (alpha log2(e) 2^(K row offset)): the logit in base-2 units up to the query row's
+                // power of two ra, by which multiplying is exact: t = u ra.  (Packed fp32 pairs: same roundings as the
+                // scalar operations, half the instructions.)
+                uint32_t acc[32];
+                uint64_t u2[16];
+                auto scale_columns = [&](int cg) {
+                    const ulonglong2* kc2 = reinterpret_cast<const ulonglong2*>(kc_all + (it % kKcRing) * 128 + cg * 32);
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const ulonglong2 k2 = kc2[c];                 // four column factors
+                        u2[2 * c] = cast::mul_f32x2(cast::pack_f32x2(acc[4 * c], acc[4 * c + 1]), k2.x);
+                        u2[2 * c + 1] = cast::mul_f32x2(cast::pack_f32x2(acc[4 * c + 2], acc[4 * c + 3]), k2.y);
+                    }
+                    if (CAUSAL && p.causal && j == m_blk) {            // the diagonal tile: keys after the query are masked
+                        const int n_local = (int)(m - (int64_t)j * BNK) - cg * 32;   // last visible column of this group
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            float lo, hi;
+                            cast::unpack_f32x2(u2[c], lo, hi);
+                            if (2 * c > n_local) lo = -INFINITY;
+                            if (2 * c + 1 > n_local) hi = -INFINITY;
+                            u2[c] = cast::pack_f32x2(__float_as_uint(lo), __float_as_uint(hi));
+                        }
+                    }
+                };
+                const uint64_t ra2 = cast::pack_f32x2(__float_as_uint(ra), __float_as_uint(ra));
+                auto work = [&](int cg) {                             // one 32-key group, from u2
+                    if (PASS == 1) {
+                        float u[32];
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) cast::unpack_f32x2(u2[c], u[2 * c], u[2 * c + 1]);
+                        float c4[4] = {u[0], u[1], u[2], u[3]};
+#pragma unroll
+                        for (int c = 4; c < 32; ++c) c4[c & 3] = fmaxf(c4[c & 3], u[c]);
+                        const float cm = fmaxf(fmaxf(c4[0], c4[1]), fmaxf(c4[2], c4[3]));
+                        const float nmx = fmaxf(run_mx, cm * ra);
+                        // 2^(-inf) = 0 on the first tile; a maximum still at -inf (everything masked so far) must
+                        // not meet itself in a difference
+                        const float ref = nmx == -INFINITY ? 0.f : nmx;
+                        run_sum *= exp2_approx(run_mx - ref);
+                        run_mx = nmx;
+                        const uint64_t nref2 = cast::pack_f32x2(__float_as_uint(-ref), __float_as_uint(-ref));
+                        float s4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            float t0, t1;
+                            cast::unpack_f32x2(cast::fma_f32x2(u2[c], ra2, nref2), t0, t1);
+                            s4[(2 * c) & 3] += exp2_approx(t0);
+                            s4[(2 * c + 1) & 3] += exp2_approx(t1);
+                        }
+                        run_sum += (s4[0] + s4[1]) + (s4[2] + s4[3]);
+                    } else {
+                        // normalise, round to bf16, cast (P has no negative element: one plane)
+                        const uint64_t nm2 = cast::pack_f32x2(__float_as_uint(neg_mx), __float_as_uint(neg_mx));
+                        const uint64_t inv2 = cast::pack_f32x2(__float_as_uint(inv), __float_as_uint(inv));
+                        uint32_t w[16];
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            float t0, t1, p0, p1;
+                            cast::unpack_f32x2(cast::fma_f32x2(u2[c], ra2, nm2), t0, t1);
+                            cast::unpack_f32x2(cast::mul_f32x2(cast::pack_f32x2(__float_as_uint(exp2_approx(t0)),
+                                                                                __float_as_uint(exp2_approx(t1))), inv2), p0, p1);
+                            const __nv_bfloat162 pr = __floats2bfloat162_rn(p0, p1);
+                            w[c] = *reinterpret_cast<const uint32_t*>(&pr);
+                        }
+                        uint32_t nib[4];
+                        const uint32_t sc = cast::cast_nonneg_group(w, nib);
+                        const uint32_t up = to_ue4m3(sc, kmax);
+                        // plane: row r, 16-byte piece cg of its 64 bytes, 64-byte swizzle; scale factors: chunk of the
+                        // K step cg / 2, byte (r % 32) * 16 + (r / 32) * 4 + (cg % 2) * 2, each scale twice (blocks of 16)
+                        *reinterpret_cast<uint4*>(sm + S_::kOffP + b * kPlane + r * 64 + ((cg ^ ((r >> 1) & 3)) << 4)) =
+                            make_uint4(nib[0], nib[1], nib[2], nib[3]);
+                        *reinterpret_cast<uint16_t*>(sm + S_::kOffSfP + (b * 2 + (cg >> 1)) * 512 + (r & 31) * 16 + (r >> 5) * 4 +
+                                                     (cg & 1) * 2) = (uint16_t)(up | (up << 8));
+                        if (p.p_plane && h == 0) {                    // verification outputs (head 0 of the launch)
+                            const int64_t g = (int64_t)j * 4 + cg, v = m * (p.L / 32) + g;
+                            p.p_plane[v] = make_uint4(nib[0], nib[1], nib[2], nib[3]);
+                            *reinterpret_cast<uint16_t*>(p.p_sf + sf_row_offset(m, p.p_nk64) + sf_group_offset((int)g)) = (uint16_t)(up | (up << 8));
+                            if (p.p_codes) p.p_codes[v] = make_uint4(nib[0], nib[1], nib[2], nib[3]);
+                            if (p.p_scales) p.p_scales[v] = (uint16_t)sc;
+                            if (p.p_bits) {
+#pragma unroll
+                                for (int c = 0; c < 4; ++c) p.p_bits[v * 4 + c] = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+                            }
+                        }
+                    }
+                };
+                // the second group's tensor-memory load is in flight while the first group is worked on
+                const int cg0 = half * 2;
+                tmem_ld32(tq + kColS + b * 128 + cg0 * 32, acc);
+                tmem_ld_wait();
+                scale_columns(cg0);
+                tmem_ld32(tq + kColS + b * 128 + (cg0 + 1) * 32, acc);
+                work(cg0);
+                tmem_ld_wait();
+                tc_fence_before();                                    // both halves are in registers: release the accumulator
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->s_empty[b]);
+                scale_columns(cg0 + 1);
+                work(cg0 + 1);
+                if (PASS == 2) {
                     fence_proxy_async();                              // visible to the tensor core's reads
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&ctl->p_full[b]);
-                    if (p.p_plane && h == 0) {                        // verification outputs (head 0 of the launch)
-                        const int64_t g = (int64_t)j * 4 + cg, v = m * (p.L / 32) + g;
-                        p.p_plane[v] = make_uint4(nib[0], nib[1], nib[2], nib[3]);
-                        *reinterpret_cast<uint16_t*>(p.p_sf + sf_row_offset(m, p.p_nk64) + sf_group_offset((int)g)) = (uint16_t)(up | (up << 8));
-                        if (p.p_codes) p.p_codes[v] = make_uint4(nib[0], nib[1], nib[2], nib[3]);
-                        if (p.p_scales) p.p_scales[v] = (uint16_t)sc;
-                        if (p.p_bits) {
-#pragma unroll
-                            for (int c = 0; c < 4; ++c) p.p_bits[v * 4 + c] = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
-                        }
-                    }
                 }
             }
             if (PASS == 1) {
-                if (ok) p.part[grow * 4 + cg] = make_float2(run_mx, run_sum);
+                if (ok) p.part[grow * 4 + grp * 2 + half] = make_float2(run_mx, run_sum);
             } else {
                 // O of the item: rows x (32 columns of the head dimension per thread), rescaled by 2^(row offset of P
                 // + row offset of V^T) - exact - and stored
@@ -440,13 +480,13 @@ attention_fp4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (!ok) continue;
                 tc_fence_after();
                 uint32_t acc[32];
-                tmem_ld32(tq + kColO + cg * 32, acc);
+                tmem_ld32(tq + kColO + cg_o * 32, acc);
                 tmem_ld_wait();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&ctl->o_empty);
-                const int4* vw = reinterpret_cast<const int4*>(p.v_words + p.v_row0 + (int64_t)h * HD + cg * 32);
-                float* out = p.O + ((int64_t)h * p.L + m) * HD + cg * 32;
+                const int4* vw = reinterpret_cast<const int4*>(p.v_words + p.v_row0 + (int64_t)h * HD + cg_o * 32);
+                float* out = p.O + ((int64_t)h * p.L + m) * HD + cg_o * 32;
                 const int p_exp = kmax ? kmax - 25 : 0;
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {

@@ -235,6 +235,8 @@ __device__ __forceinline__ uint32_t emit_group(const uint32_t (&w)[16], int64_t 
 // The cast of a group without negative elements (a softmax output) when only the FP4 kernels' operand is wanted:
 // its positive sign plane is its code word, the negative plane and scale are zero.  Same arithmetic as above,
 // minus everything the negative side needs.  nib: the group's 32 codes; returns the positive scale byte.
+// (The bf16 pairs are split with a shift and a mask here: this runs in the attention epilogue, where the logic pipe
+// has room and instruction issue is what counts.)
 __device__ __forceinline__ uint32_t cast_nonneg_group(const uint32_t (&w)[16], uint32_t (&nib)[4]) {
     uint32_t pm = w[0];
 #pragma unroll
@@ -245,7 +247,12 @@ __device__ __forceinline__ uint32_t cast_nonneg_group(const uint32_t (&w)[16], u
     const uint32_t inv = __float_as_uint(inv_scale(sc));
     const uint64_t inv2 = pack_f32x2(inv, inv);
 #pragma unroll
-    for (int j = 0; j < 4; ++j) nib[j] = encode8_one(w + 4 * j, inv2);
+    for (int j = 0; j < 4; ++j) {
+        uint64_t q[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) q[i] = mul_f32x2(pack_f32x2(w[4 * j + i] << 16, w[4 * j + i] & 0xFFFF0000u), inv2);
+        nib[j] = cvt_e2m1x8(q[0], q[1], q[2], q[3]);
+    }
     return sc;
 }
 // Stores the plane at group index v (and, when asked, the same word as the group's canonical codes: without a set
