@@ -54,6 +54,13 @@ def lib() -> ctypes.CDLL:
         L.amx_oracle_fakequant_pot_floor.argtypes = [p, i64, i64, ctypes.c_int, ctypes.c_int, p]
         L.amx_oracle_softmax_bf16.argtypes = [p, i64, i64, dbl, p]
         L.amx_oracle_softmax_bf16_causal.argtypes = [p, i64, i64, dbl, i64, p]
+        L.amx_oracle_e4m3_value.restype = dbl
+        L.amx_oracle_e4m3_value.argtypes = [ctypes.c_uint8]
+        L.amx_oracle_e4m3_encode.restype = ctypes.c_uint8
+        L.amx_oracle_e4m3_encode.argtypes = [dbl]
+        L.amx_oracle_quantize_nv.argtypes = [p, i64, i64, i64, ctypes.c_int, p, p, p]
+        L.amx_oracle_dequantize_nv.argtypes = [p, p, ctypes.c_float, i64, i64, p]
+        L.amx_oracle_gemm_nv.argtypes = [p, p, ctypes.c_float, p, p, ctypes.c_float, i64, i64, i64, p, i64, p]
         L.amx_oracle_num_threads.restype = ctypes.c_int
         _lib = L
     return _lib
@@ -204,3 +211,56 @@ def softmax_bf16(S: np.ndarray, alpha: float, causal_row0: int | None = None) ->
     else:
         lib().amx_oracle_softmax_bf16_causal(_ptr(S), rows, cols, float(alpha), int(causal_row0), _ptr(P))
     return P
+
+
+# ---- NVFP4 / ANVFP4 (group 16, E4M3 group scales, one fp32 tensor scale) ----
+
+def e4m3_value(code: int) -> float:
+    return float(lib().amx_oracle_e4m3_value(int(code)))
+
+
+def e4m3_encode(q: float) -> int:
+    return int(lib().amx_oracle_e4m3_encode(float(q)))
+
+
+def quantize_nv(x_bf16_bits: np.ndarray, asym: bool):
+    """bf16 bit patterns [rows, K] -> (codes u8 [rows, K/2], E4M3 scales u8 [rows, K/16, 2], tensor scale float32).
+    asym False: NVFP4 (the group's one scale in both bytes); True: ANVFP4 (positive-side, negative-side scale)."""
+    x = _c(x_bf16_bits, np.uint16)
+    rows, K = x.shape
+    codes = np.zeros((rows, K // 2), np.uint8)
+    scales = np.zeros((rows, K // 16, 2), np.uint8)
+    t = np.zeros(1, np.float32)
+    rc = lib().amx_oracle_quantize_nv(_ptr(x), rows, K, K, int(asym), _ptr(codes), _ptr(scales), _ptr(t))
+    if rc:
+        raise ValueError("amx_oracle_quantize_nv: K must be a multiple of 16")
+    return codes, scales, np.float32(t[0])
+
+
+def dequantize_nv(codes: np.ndarray, scales: np.ndarray, tensor_scale) -> np.ndarray:
+    codes, scales = _c(codes, np.uint8), _c(scales, np.uint8)
+    rows, K = codes.shape[0], codes.shape[1] * 2
+    out = np.zeros((rows, K), np.float64)
+    rc = lib().amx_oracle_dequantize_nv(_ptr(codes), _ptr(scales), float(tensor_scale), rows, K, _ptr(out))
+    if rc:
+        raise ValueError("amx_oracle_dequantize_nv: bad shape")
+    return out
+
+
+def gemm_nv(codesA, scalesA, tA, codesW, scalesW, tW, rows=None) -> np.ndarray:
+    codesA, scalesA = _c(codesA, np.uint8), _c(scalesA, np.uint8)
+    codesW, scalesW = _c(codesW, np.uint8), _c(scalesW, np.uint8)
+    M, K = codesA.shape[0], codesA.shape[1] * 2
+    N = codesW.shape[0]
+    assert codesW.shape[1] * 2 == K
+    if rows is None:
+        idx, n_rows, idx_p = None, M, None
+    else:
+        idx = _c(rows, np.int64)
+        n_rows, idx_p = idx.shape[0], _ptr(idx)
+    C = np.zeros((n_rows, N), np.float32)
+    rc = lib().amx_oracle_gemm_nv(_ptr(codesA), _ptr(scalesA), float(tA), _ptr(codesW), _ptr(scalesW), float(tW),
+                                  M, N, K, idx_p, n_rows, _ptr(C))
+    if rc:
+        raise ValueError(f"amx_oracle_gemm_nv failed (rc={rc})")
+    return C

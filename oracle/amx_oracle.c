@@ -512,6 +512,208 @@ int amx_oracle_softmax_bf16_causal(const float *S, int64_t rows, int64_t cols, d
     return 0;
 }
 
+/* ------------------------------------------------- NVFP4 / ANVFP4 -- */
+
+/*
+ * The "recently deployed commercial" format the paper compares with in Section 5
+ * (table of NVFP4 / ANVFP4 results): FP4 E2M1 elements in groups of 16 with a
+ * double scaling - one FP32 scale for the whole tensor and one FP8 E4M3 scale per
+ * group.  ANVFP4 is the paper's asymmetric variant: two E4M3 scales per group, one
+ * per sign, as in AMXFP4.  The paper names the parts but no arithmetic; the reading
+ * used here (recorded in the design notes):
+ *   tensor scale  t = max|x| / (448 * 6): the largest group scale then sits at the
+ *                 top of the E4M3 range (448) and the largest element at 6;
+ *                 t = 1 for an all-zero tensor;
+ *   group scale   E4M3 nearest (ties to even, saturating at 448, with subnormals)
+ *                 to (max_side / 6) / t;
+ *   element       E2M1 nearest (ties to even, clamped at 6) to x / (scale * t);
+ *                 sign bit = the input's sign bit; magnitude 0 under a zero scale;
+ *   decoded value (-1)^s * E2M1 * E4M3(scale_s) * t.
+ * Precision of the DECISIONS: with a 24-bit tensor scale the quotients above are not
+ * exactly representable and can lie within 2^-30 of a rounding boundary, which no
+ * fp32 arithmetic resolves.  So that a device implementation can take every
+ * decision exactly as this reference does, the decisions are taken in IEEE fp32,
+ * in this order (each operation rounded to nearest even):
+ *     t     = amax / 2688
+ *     rt    = 1 / t
+ *     g     = (max_side * fl(1/6)) * rt              -> E4M3 byte
+ *     d     = E4M3(byte) * t,   rd = 1 / d
+ *     q     = x * rd                                  -> E2M1 code
+ * The tests pin this against exact rational arithmetic: the two agree except for
+ * quotients within 2^-20 (relative) of a boundary, and agree everywhere on inputs
+ * for which the fp32 operations are exact.
+ */
+
+/* Value of an E4M3 byte (OCP FP8 E4M3: bias 7, no infinities, 0x7F / 0xFF = NaN). */
+double amx_oracle_e4m3_value(uint8_t code)
+{
+    int e = (code >> 3) & 15, m = code & 7;
+    double v;
+    if (e == 15 && m == 7)
+        v = NAN;
+    else if (e == 0)
+        v = ldexp((double)m, -9);             /* subnormal: m/8 * 2^-6 */
+    else
+        v = ldexp(1.0 + m / 8.0, e - 7);
+    return (code & 0x80) ? -v : v;
+}
+
+/* E4M3 byte nearest to q >= 0; ties to even; saturate at 448 (0x7E). */
+uint8_t amx_oracle_e4m3_encode(double q)
+{
+    if (!(q > 0.0))
+        return 0;
+    int ex;
+    (void)frexp(q, &ex);
+    int e = ex - 1;                           /* floor(log2 q) */
+    if (e < -6)
+        e = -6;                               /* subnormal spacing below 2^-6 */
+    double quantum = ldexp(1.0, e - 3);
+    double t = q / quantum;                   /* exact: power-of-two divisor */
+    double lo = floor(t), frac = t - lo, n = lo;
+    if (frac > 0.5 || (frac == 0.5 && fmod(lo, 2.0) == 1.0))
+        n = lo + 1.0;
+    if (n == 16.0) {
+        n = 8.0;
+        e += 1;
+    }
+    if (e > 8 || (e == 8 && n > 14.0))
+        return 0x7E;                          /* 1.75 * 2^8 = 448 */
+    if (n < 8.0)                              /* only possible with e == -6 */
+        return (uint8_t)n;
+    return (uint8_t)(((e + 7) << 3) | ((int)n - 8));
+}
+
+static float bf16_to_float(uint16_t b)
+{
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+/*
+ * x: bf16 bit patterns [rows][ld]; groups of 16 along K (K % 16 == 0).
+ * asym = 0: NVFP4 (one scale per group, stored in both bytes); 1: ANVFP4.
+ * codes [rows][K/2], scales [rows][K/16][2] (E4M3 bytes: positive side, negative
+ * side), *tensor_scale = t.
+ */
+int amx_oracle_quantize_nv(const uint16_t *x, int64_t rows, int64_t K, int64_t ld, int asym,
+                           uint8_t *codes, uint8_t *scales, float *tensor_scale)
+{
+    if (K <= 0 || K % 16 != 0)
+        return -1;
+    float amax = 0.0f;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t k = 0; k < K; ++k) {
+            float a = fabsf(bf16_to_float(x[r * ld + k]));
+            if (a > amax) amax = a;
+        }
+    const volatile float t = amax > 0.0f ? amax / 2688.0f : 1.0f;
+    const volatile float rt = 1.0f / t;
+    const volatile float sixth = 1.0f / 6.0f;
+    *tensor_scale = t;
+    int64_t G = K / 16;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t g = 0; g < G; ++g) {
+            const uint16_t *xg = x + r * ld + g * 16;
+            float pmax = 0.0f, nmax = 0.0f;
+            for (int i = 0; i < 16; ++i) {
+                float a = fabsf(bf16_to_float(xg[i]));
+                if (xg[i] >> 15) { if (a > nmax) nmax = a; }
+                else             { if (a > pmax) pmax = a; }
+            }
+            if (!asym)
+                pmax = nmax = (pmax > nmax ? pmax : nmax);
+            uint8_t byte[2];
+            float rd[2];
+            for (int side = 0; side < 2; ++side) {
+                volatile float g1 = (side ? nmax : pmax) * sixth;   /* every product rounded to fp32 */
+                volatile float g2 = g1 * rt;
+                byte[side] = amx_oracle_e4m3_encode((double)g2);
+                volatile float d = (float)amx_oracle_e4m3_value(byte[side]) * t;
+                volatile float inv = 1.0f / d;
+                rd[side] = byte[side] ? inv : 0.0f;
+            }
+            for (int i = 0; i < 16; ++i) {
+                int sgn = xg[i] >> 15;
+                volatile float q = fabsf(bf16_to_float(xg[i])) * rd[sgn];
+                int mag = byte[sgn] ? amx_oracle_e2m1_encode((double)q) : 0;
+                uint8_t c = (uint8_t)((sgn << 3) | mag);
+                int64_t k = g * 16 + i;
+                uint8_t *b = codes + r * (K / 2) + k / 2;
+                if (k & 1) *b = (uint8_t)((*b & 0x0F) | (c << 4));
+                else       *b = (uint8_t)((*b & 0xF0) | c);
+            }
+            scales[(r * G + g) * 2 + 0] = byte[0];
+            scales[(r * G + g) * 2 + 1] = byte[1];
+        }
+    return 0;
+}
+
+/* out[r][k] = (-1)^s * E2M1 * E4M3(scale_s) * t, in fp64 (the first product is exact). */
+int amx_oracle_dequantize_nv(const uint8_t *codes, const uint8_t *scales, float tensor_scale,
+                             int64_t rows, int64_t K, double *out)
+{
+    if (K <= 0 || K % 16 != 0)
+        return -1;
+    int64_t G = K / 16;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t k = 0; k < K; ++k) {
+            uint8_t byte = codes[r * (K / 2) + k / 2];
+            int c = (k & 1) ? (byte >> 4) : (byte & 15);
+            double s = amx_oracle_e4m3_value(scales[(r * G + k / 16) * 2 + ((c >> 3) & 1)]);
+            out[r * K + k] = amx_oracle_e2m1_value(c) * s * (double)tensor_scale;
+        }
+    return 0;
+}
+
+/*
+ * C[i][n] = tA * tW * sum_k (E2M1 * E4M3)_A[rows[i]][k] * (E2M1 * E4M3)_W[n][k], fp64 sums,
+ * rounded once to fp32.  rows == NULL: all M rows.
+ */
+int amx_oracle_gemm_nv(const uint8_t *codesA, const uint8_t *scalesA, float tA,
+                       const uint8_t *codesW, const uint8_t *scalesW, float tW,
+                       int64_t M, int64_t N, int64_t K, const int64_t *rows, int64_t n_rows, float *C)
+{
+    if (K <= 0 || K % 16 != 0)
+        return -1;
+    int64_t G = K / 16;
+    double *w = (double *)malloc(sizeof(double) * (size_t)N * (size_t)K);
+    if (!w)
+        return -2;
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < N; ++n)
+        for (int64_t k = 0; k < K; ++k) {
+            uint8_t byte = codesW[n * (K / 2) + k / 2];
+            int c = (k & 1) ? (byte >> 4) : (byte & 15);
+            w[n * K + k] = amx_oracle_e2m1_value(c) * amx_oracle_e4m3_value(scalesW[(n * G + k / 16) * 2 + ((c >> 3) & 1)]);
+        }
+#pragma omp parallel
+    {
+        double *a = (double *)malloc(sizeof(double) * (size_t)K);
+#pragma omp for schedule(static)
+        for (int64_t i = 0; i < n_rows; ++i) {
+            int64_t m = rows ? rows[i] : i;
+            if (m < 0 || m >= M) continue;
+            for (int64_t k = 0; k < K; ++k) {
+                uint8_t byte = codesA[m * (K / 2) + k / 2];
+                int c = (k & 1) ? (byte >> 4) : (byte & 15);
+                a[k] = amx_oracle_e2m1_value(c) * amx_oracle_e4m3_value(scalesA[(m * G + k / 16) * 2 + ((c >> 3) & 1)]);
+            }
+            for (int64_t n = 0; n < N; ++n) {
+                double acc = 0.0;
+                for (int64_t k = 0; k < K; ++k) acc += a[k] * w[n * K + k];
+                C[i * N + n] = (float)(acc * (double)tA * (double)tW);
+            }
+        }
+        free(a);
+    }
+    free(w);
+    return 0;
+}
+
 int amx_oracle_num_threads(void)
 {
     int n = 1;
