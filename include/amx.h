@@ -342,6 +342,38 @@ size_t amx_quant_gemm_static_capacity(void);
 int amx_quant_gemm_static_status(void* stream);
 
 /*
+ * NVFP4 and ANVFP4 - the format the paper compares AMXFP4 with in Section 5 (its table of NVFP4 / ANVFP4 results):
+ * E2M1 elements in groups of 16, one FP8 E4M3 scale per group - ANVFP4: one per sign, as in AMXFP4 - and one fp32
+ * scale for the whole tensor.  The paper names the parts, not the arithmetic; implemented (every step an IEEE fp32
+ * operation, in this order, so that the CPU reference takes the same decisions):
+ *   t = max|x| / 2688 (1 for an all-zero tensor);  group scale byte = E4M3 nearest (ties to even, saturating at 448)
+ *   to (max_side * fl(1/6)) * (1/t);  element = E2M1 nearest (ties to even, clamped at 6) to x * (1 / (E4M3(byte) * t)),
+ *   sign bit = sign of x;  decoded value = (-1)^s * E2M1 * E4M3(scale_s) * t.
+ * amx_quantize_nvfp4  two launches (the tensor maximum, then the cast).
+ *   x             bf16 [rows, ld_x], 16-byte aligned, ld_x % 8 == 0, K % 64 == 0
+ *   flags         0 (NVFP4: the group's one scale is stored in both scale bytes) or AMX_NV_ASYMMETRIC (ANVFP4)
+ *   codes         out, nullable: [rows, K/2] as for AMXFP4;  scales  out, nullable: E4M3 bytes [rows, K/16, 2]
+ *   tensor_scale  out: TWO floats, 8-byte aligned: [0] = t, [1] = max|x|
+ *   prepared      out, nullable: the operand in the FP4 tensor-core kernel's form (amx_nvfp4_prepared_bytes() bytes,
+ *                 256-aligned; is_weight selects the right-hand operand's padding).  Group size 16 and E4M3 are that
+ *                 kernel's native scale block and type: the scale bytes go in as they are, nothing is shifted or
+ *                 flushed, and a symmetric operand is one plane.
+ * amx_dequantize_nvfp4  the decoded values, fp32 (AMX_OUT_F32) or bf16 (the fp32 value rounded to nearest even).
+ * amx_gemm_nvfp4  C = decoded A x decoded W^T for two prepared operands; fp32 accumulation, every result multiplied by
+ *   the product of the two tensor scales.  NVFP4 x NVFP4 issues one block-scaled MMA per tile pair, ANVFP4 four.
+ *   workspace: 256 bytes (status word, see amx_gemm_status).
+ */
+#define AMX_NV_ASYMMETRIC 0x1u
+int amx_quantize_nvfp4(const void* x, int64_t rows, int64_t K, int64_t ld_x, uint32_t flags, uint8_t* codes,
+                       uint8_t* scales, float* tensor_scale, int is_weight, void* prepared, size_t prepared_bytes,
+                       void* stream);
+size_t amx_nvfp4_prepared_bytes(int64_t rows, int64_t K, int is_weight);
+int amx_dequantize_nvfp4(const uint8_t* codes, const uint8_t* scales, const float* tensor_scale, int64_t rows, int64_t K,
+                         uint32_t flags, void* out, int64_t ld_out, void* stream);
+int amx_gemm_nvfp4(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K, float* C,
+                   int64_t ld_c, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * amx_quant_error - squared error of a quantized tensor against its bf16 source, split as the appendix
  * "Determining PoT Shared Scale: Floor vs. Round" splits the error of a shared scale: elements whose magnitude
  * exceeds the largest value their side represents (|x| > 6 * scale of the element's side) make up the

@@ -38,6 +38,7 @@ SYMBOLS = (
     "amx_quant_error", "amx_quant_error_workspace_bytes",
     "amx_attention_map", "amx_gemm_flushed_scales", "amx_prepared_flushed_scales", "amx_selftest_wait_timeout",
     "amx_quant_gemm_static_status",
+    "amx_quantize_nvfp4", "amx_nvfp4_prepared_bytes", "amx_dequantize_nvfp4", "amx_gemm_nvfp4",
 )
 
 
@@ -69,6 +70,11 @@ def lib() -> ctypes.CDLL:
         L.amx_prepared_flushed_scales.restype = i64
         L.amx_selftest_wait_timeout.argtypes = [p, sz, u32, p]
         L.amx_quant_gemm_static_status.argtypes = [p]
+        L.amx_quantize_nvfp4.argtypes = [p, i64, i64, i64, u32, p, p, p, i, p, sz, p]
+        L.amx_nvfp4_prepared_bytes.argtypes = [i64, i64, i]
+        L.amx_nvfp4_prepared_bytes.restype = sz
+        L.amx_dequantize_nvfp4.argtypes = [p, p, p, i64, i64, u32, p, i64, p]
+        L.amx_gemm_nvfp4.argtypes = [p, p, i64, i64, i64, p, i64, p, sz, p]
         L.amx_quant_gemm_static.argtypes = [p, i64, p, p, i64, i64, i64, i, u32, p, i64, p]
         L.amx_quant_gemm_static_capacity.argtypes = []
         L.amx_quant_gemm_static_capacity.restype = sz
@@ -317,6 +323,45 @@ def softmax_quantize(S: torch.Tensor, alpha: float, prepared_as: str | None = No
                                       scales.data_ptr(), is_w, buf.data_ptr() if buf is not None else None, nbytes,
                                       _stream()), "amx_softmax_quantize")
     return (codes, scales) if buf is None else (codes, scales, buf)
+
+
+NV_ASYMMETRIC = 0x1
+
+
+def quantize_nvfp4(x: torch.Tensor, asym: bool, prepared_as: str | None = None):
+    """bf16 [rows, K] -> (codes, E4M3 scales [rows, K/16, 2], tensor_scale (2 floats: t, max|x|)[, prepared])."""
+    _dev(x, torch.bfloat16, "x")
+    assert x.dim() == 2 and x.stride(1) == 1
+    rows, K = x.shape
+    codes = torch.empty((rows, K // 2), dtype=torch.uint8, device=x.device)
+    scales = torch.empty((rows, K // 16, 2), dtype=torch.uint8, device=x.device)
+    ts = torch.empty(2, dtype=torch.float32, device=x.device)
+    is_w = int(prepared_as == "w")
+    prep = None
+    if prepared_as is not None:
+        prep = torch.full((lib().amx_nvfp4_prepared_bytes(rows, K, is_w),), 0xFF, dtype=torch.uint8, device=x.device)
+    _check(lib().amx_quantize_nvfp4(x.data_ptr(), rows, K, x.stride(0), NV_ASYMMETRIC if asym else 0, codes.data_ptr(),
+                                    scales.data_ptr(), ts.data_ptr(), is_w, prep.data_ptr() if prep is not None else None,
+                                    prep.numel() if prep is not None else 0, _stream()), "amx_quantize_nvfp4")
+    return (codes, scales, ts) if prep is None else (codes, scales, ts, prep)
+
+
+def dequantize_nvfp4(codes: torch.Tensor, scales: torch.Tensor, ts: torch.Tensor, dtype=torch.float32):
+    rows, K = codes.shape[0], codes.shape[1] * 2
+    out = torch.empty((rows, K), dtype=dtype, device=codes.device)
+    flag = {torch.bfloat16: OUT_BF16, torch.float32: OUT_F32}[dtype]
+    _check(lib().amx_dequantize_nvfp4(codes.data_ptr(), scales.data_ptr(), ts.data_ptr(), rows, K, flag, out.data_ptr(), K,
+                                      _stream()), "amx_dequantize_nvfp4")
+    return out
+
+
+def gemm_nvfp4(a_prepared: torch.Tensor, w_prepared: torch.Tensor, M: int, N: int, K: int, workspace: torch.Tensor | None = None):
+    out = torch.empty((M, N), dtype=torch.float32, device=a_prepared.device)
+    if workspace is None:
+        workspace = _ws(256, a_prepared.device)
+    _check(lib().amx_gemm_nvfp4(a_prepared.data_ptr(), w_prepared.data_ptr(), M, N, K, out.data_ptr(), N, workspace.data_ptr(),
+                                workspace.numel(), _stream()), "amx_gemm_nvfp4")
+    return out
 
 
 def linear_host(a_host: torch.Tensor, w_host: torch.Tensor, c_host: torch.Tensor, workspace: torch.Tensor,

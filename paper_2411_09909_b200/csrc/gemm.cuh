@@ -72,7 +72,9 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
                          int causal_pv = 0 /* 1: the product P V of causal attention (A = P, square) */,
                          int batch = 1 /* > 1 (N <= 128): a stack of `batch` independent products of M / batch rows */,
                          int64_t w_batch_rows = 0 /* rows between their right-hand operands in the stacked W */,
-                         const int* gate = nullptr /* device word: the kernel does nothing when it is nonzero */);
+                         const int* gate = nullptr /* device word: the kernel does nothing when it is nonzero */,
+                         const float* scale_a = nullptr, const float* scale_w = nullptr /* device: one factor per
+                         operand; every result is multiplied by their product (NVFP4 tensor scales) */);
 // workspace that lets the kernel cut K into ranges for products with few output tiles (256 bytes otherwise)
 size_t gemm_fp4_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K);
 // C[m][n] = sum over `slices` partial products [slices][M][N], in slice order (defined with the bf16-decode kernel)

@@ -216,6 +216,8 @@ struct Params {
     int slices;                  // SLICED instantiation: K is cut into this many ranges, each (tile, range) a work item
     int64_t slice_stride;        //   whose partial product goes to C + range * slice_stride
     int* status;
+    const float *scale_a, *scale_w;   // not NULL: one fp32 factor per operand (the tensor scales of NVFP4 operands);
+                                 // the store epilogue multiplies every result by their product
     const int* gate;             // not NULL: the kernel returns at once when this word is nonzero (the caller then
                                  // runs the exact bf16-decode kernel on the same operands, gated the other way)
     // attention epilogues (kEpiStats, kEpiCast): the tile holds logits S = Q K^T; `alpha` scales them
@@ -531,6 +533,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             }
             return c;
         };
+        const float out_scale = (EPI == kEpiStore && p.scale_a) ? __ldg(p.scale_a) * __ldg(p.scale_w) : 1.0f;
         int64_t tile = next_live(blockIdx.x);
         TileConsts nxt = load_consts(tile);
         while (tile < total_tiles && ok) {
@@ -567,7 +570,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
                                 const int sh = min(127, max(-126, a_exp + ex[i]));
-                                f[j + i] = __uint_as_float(v[buf][j + i]) * __uint_as_float((uint32_t)(sh + 127) << 23);
+                                f[j + i] = __uint_as_float(v[buf][j + i]) * __uint_as_float((uint32_t)(sh + 127) << 23) * out_scale;
                             }
                         }
                         if (m < p.M) store_row16(C_item + m * p.ld_c + n0 + col, f, p.vec_store != 0, p.N - (n0 + col));
@@ -822,7 +825,7 @@ size_t gemm_fp4_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 // workspace_bytes >= gemm_fp4_prepared_workspace_bytes() enables the K ranges; 256 bytes always suffice.
 int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
                          int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes, int causal_pv, int batch,
-                         int64_t w_batch_rows, const int* gate) {
+                         int64_t w_batch_rows, const int* gate, const float* scale_a, const float* scale_w) {
     if (batch > 1 && (N > BN / 2 || M % batch || (M / batch) % BM || w_batch_rows % 128)) return AMX_ERR_SHAPE;
     Params p;
     OperandLayout oa, ow;
@@ -832,6 +835,8 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
     p.causal = causal_pv ? 2 : 0;
     p.a_single = a.single_plane ? 1 : 0;
     p.gate = gate;
+    p.scale_a = scale_a;
+    p.scale_w = scale_w;
     const uint8_t* pa = static_cast<const uint8_t*>(a.prepared);
     const uint8_t* pw = static_cast<const uint8_t*>(w.prepared);
     const int slices = batch > 1 ? 1 : gemm_fp4_slices(M, N, K);
@@ -844,7 +849,7 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
     if (causal_pv)
         return half ? launch_fp4<128, kEpiStore, false, true, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st)
                     : launch_fp4<128, kEpiStore, false, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
-    if (!gate && slices > 1 && fp4_block_k() == 128 && workspace_bytes >= gemm_fp4_prepared_workspace_bytes(M, N, K)) {
+    if (!gate && !scale_a && slices > 1 && fp4_block_k() == 128 && workspace_bytes >= gemm_fp4_prepared_workspace_bytes(M, N, K)) {
         float* part = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 256);
         p.C = part;
         p.ld_c = N;
