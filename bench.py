@@ -574,8 +574,37 @@ def run_ours(args):
                 res[key + "_tflops"] = flops_step / (v_ms * 1e-3) / 1e12
                 res[key + "_ms"] = v_ms
             format_variants[name] = res
-        format_variants["what"] = ("same workload and kernels with the symmetric formats (amx_quantize_prepared_fmt): "
-                                   "step = casts of both operands + GEMMs, gemm = the GEMMs alone")
+        # NVFP4 / ANVFP4 (group 16, E4M3 group scales + fp32 tensor scale: Section 5's comparison format): the scale
+        # bytes are the tensor cores' native type, NVFP4 is one product per tile pair, ANVFP4 four
+        nv = []
+        for li, (K, N) in enumerate(layers):
+            nv.append((torch.empty(L.amx_nvfp4_prepared_bytes(M, K, 0), dtype=torch.uint8, device="cuda"),
+                       torch.empty(L.amx_nvfp4_prepared_bytes(N, K, 1), dtype=torch.uint8, device="cuda"),
+                       torch.empty(2, dtype=torch.float32, device="cuda"), torch.empty(2, dtype=torch.float32, device="cuda")))
+        for name, flag in (("nvfp4", 0), ("anvfp4", 1)):
+            def nv_step(st, with_casts=True, flag=flag):
+                for li, (K, N) in enumerate(layers):
+                    pa, pw, ta, tw = nv[li]
+                    b = bufs[li]
+                    if with_casts:
+                        check(L.amx_quantize_nvfp4(A[li].data_ptr(), M, K, K, flag, None, None, ta.data_ptr(), 0, pa.data_ptr(),
+                                                   pa.numel(), st))
+                        check(L.amx_quantize_nvfp4(W[li].data_ptr(), N, K, K, flag, None, None, tw.data_ptr(), 1, pw.data_ptr(),
+                                                   pw.numel(), st))
+                    check(L.amx_gemm_nvfp4(pa.data_ptr(), pw.data_ptr(), M, N, K, b["c"].data_ptr(), N, b["work"].data_ptr(),
+                                           b["work"].numel(), st))
+            res = {}
+            for key, with_casts in (("step", True), ("gemm", False)):
+                nv_step(stream)
+                v_ms = timed_graph(lambda st: nv_step(st, with_casts), extra_steps)
+                res[key + "_tflops"] = flops_step / (v_ms * 1e-3) / 1e12
+                res[key + "_ms"] = v_ms
+            format_variants[name] = res
+        del nv
+        format_variants["what"] = ("same workload and GEMM kernel with other formats: sym_fp8 / mxfp4 = the paper's symmetric "
+                                   "comparison formats (amx_quantize_prepared_fmt), nvfp4 / anvfp4 = group 16 with E4M3 scales "
+                                   "and a tensor scale (amx_quantize_nvfp4: two launches, the tensor maximum first); step = "
+                                   "casts of both operands + GEMMs, gemm = the GEMMs alone")
         run_step()                      # leave the buffers as the headline step writes them
         torch.cuda.synchronize()
 

@@ -73,7 +73,7 @@ typedef enum amx_status {
 #define AMX_OUT_BF16 0x0u
 #define AMX_OUT_F32 0x1u
 /* flags for amx_gemm / amx_quant_gemm: kernel choice.  Default (AMX_GEMM_AUTO): group size 32 runs on
- * the tensor cores - the FP4 kernel when M*N*K >= 2^27, the exact bf16-decode kernel below that and for
+ * the tensor cores - the FP4 kernel when M*N*K >= 2^28, the exact bf16-decode kernel below that and for
  * at most 64 rows of A against a large weight (decode-like shapes: that kernel then cuts K into slices over
  * CTAs and adds the partial products in slice order) - except that at most 64 rows of A with K >= 512 and
  * K % 128 == 0 go to the weight-streaming kernel (AMX_GEMM_ROWS); other group sizes run on the SIMT kernel.

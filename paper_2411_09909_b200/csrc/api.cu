@@ -28,15 +28,16 @@ uint32_t pick_kernel(int64_t M, int64_t N, int64_t K, int gs, uint32_t flags) {
     const bool rows = gemm_rows_supported(M, N, K, gs);
     if (want == AMX_GEMM_ROWS) return rows ? AMX_GEMM_ROWS : 0;
     // AMX_GEMM_AUTO: the FP4-pipe kernel for anything that fills the machine (it is about twice as fast as
-    // the bf16-decode kernel); the exact bf16-decode kernel for small products, where launch count matters
-    // more than throughput; the SIMT kernel for group sizes the tensor-core kernels do not take.
+    // the bf16-decode kernel); the exact bf16-decode kernel for small products (below 2^28 multiply-adds), where
+    // launch count matters more than throughput - the FP4 route costs two launches more: one preparation per
+    // operand, and under AUTO the gated exact kernel behind it; the SIMT kernel for group sizes the tensor-core kernels do not take.
     // A few token rows against a big weight (decode-like): too few 128 x 256 tiles to fill the machine, and the
     // FP4 kernel would have to prepare the whole weight for them; the bf16-decode kernel slices K over CTAs.
     // At most 64 token rows: the weight-streaming kernel reads the canonical weight once.
     if (rows && K >= 512) return AMX_GEMM_ROWS;
     const int64_t tiles = ((M + 127) / 128) * ((N + 255) / 256);
     if (tc && M <= 64 && tiles < 148 && K >= 1024) return AMX_GEMM_TC;      // K not a multiple of 128
-    if (gemm_fp4_supported(M, N, K, gs) && (double)M * (double)N * (double)K >= 128.0 * 1024.0 * 1024.0) return AMX_GEMM_FP4;
+    if (gemm_fp4_supported(M, N, K, gs) && (double)M * (double)N * (double)K >= 256.0 * 1024.0 * 1024.0) return AMX_GEMM_FP4;
     return tc ? AMX_GEMM_TC : AMX_GEMM_SIMT;
 }
 

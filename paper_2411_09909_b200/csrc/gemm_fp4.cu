@@ -212,7 +212,7 @@ struct Params {
     int mt_batch;                // half-width instantiation: > 0 = the product is a stack of independent ones, mt_batch
     int64_t w_batch_rows;        //   row blocks of A each, whose right-hand operands lie w_batch_rows rows apart (a
                                  //   multiple of 128) in the stacked W; C is the stack of the results
-    int m_fast;                  // tile order: consecutive tiles walk down M (else along N), see blk_m / blk_n
+    int band;                    // tile order: row blocks of A per band, see blk_m / blk_n
     int slices;                  // SLICED instantiation: K is cut into this many ranges, each (tile, range) a work item
     int64_t slice_stride;        //   whose partial product goes to C + range * slice_stride
     int* status;
@@ -291,20 +291,32 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         if (c < (j + 1) * (j + 1)) { m = 2 * j; n = c - j * (j + 1); }
         else { m = 2 * j + 1; n = c - (j + 1) * (j + 1); }
     };
-    // Tile order.  The CTAs work on ~148 consecutive tiles at a time; walking down M first keeps that set to a few
-    // row blocks of W (read once from DRAM, shared through L2 by the CTAs of all M blocks) plus all of A, when A is
-    // the smaller operand, and the other way round otherwise.
-    // (one 32-bit division per call: the host rejects products with 2^31 tiles or more)
-    const uint32_t fast_dim = (uint32_t)(p.m_fast ? m_tiles : n_tiles);
+    // Tile order.  The CTAs work on ~148 consecutive tiles at a time and advance through K roughly together, so what
+    // they read from DRAM per wave is the operand rows the wave touches, once.  Tiles are ordered in bands of
+    // p.band row blocks of A: inside a band the tile index walks down the band's row blocks first, then along N.
+    // A wave then touches band x 128 rows of A and (148 / band) x 256 rows of W (with 16: 2048 + 2368 rows, near
+    // the minimum), and consecutive waves of a band share its rows of A in L2.  Walking along N first, a wave of a
+    // tall product touched a few row blocks of A and ALL of W: 3.6 GB of DRAM reads for 0.23 GB of operands at
+    // 16384 x 10240 x 8192.  A band as tall as the matrix is the plain "down M first" order (small M).
+    // (two 32-bit divisions per call: the host rejects products with 2^31 tiles or more)
+    const uint32_t band = (uint32_t)p.band, per_band = band * (uint32_t)n_tiles;
+    auto banded = [&](int64_t tile, uint32_t& m, uint32_t& n) {
+        const uint32_t t = (uint32_t)tile / (uint32_t)S, b = t / per_band, r = t - b * per_band;
+        const uint32_t rows_here = min(band, (uint32_t)m_tiles - b * band);      // the last band may be shorter
+        n = r / rows_here;
+        m = b * band + (r - n * rows_here);
+    };
     auto blk_m = [&](int64_t tile) -> int64_t {
-        if (compact) { uint32_t m, n; compact_mn((uint32_t)tile, m, n); return m; }
-        const uint32_t t = (uint32_t)tile / (uint32_t)S, q = t / fast_dim;
-        return p.m_fast ? t - q * fast_dim : q;
+        uint32_t m, n;
+        if (compact) compact_mn((uint32_t)tile, m, n);
+        else banded(tile, m, n);
+        return m;
     };
     auto blk_n = [&](int64_t tile) -> int64_t {
-        if (compact) { uint32_t m, n; compact_mn((uint32_t)tile, m, n); return n; }
-        const uint32_t t = (uint32_t)tile / (uint32_t)S, q = t / fast_dim;
-        return p.m_fast ? q : t - q * fast_dim;
+        uint32_t m, n;
+        if (compact) compact_mn((uint32_t)tile, m, n);
+        else banded(tile, m, n);
+        return n;
     };
     // rows by which the right-hand operand of row block m_blk is shifted (stack of independent products)
     auto w_shift = [&](int64_t m_blk) -> int64_t {
@@ -769,7 +781,11 @@ int fill_params(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, 
     p.nk64 = oa.nk64;
     p.vec_store = C && aligned(C, 32) && ld_c % 8 == 0;     // 32-byte stores in the epilogue
     p.status = status;
-    p.m_fast = getenv("AMX_FP4_NFAST") ? 0 : (M <= N);
+    {
+        const char* e = getenv("AMX_FP4_BAND");              // row blocks of A per band of the tile order (default 16)
+        const int64_t want = e && atoi(e) > 0 ? atoi(e) : 16, m_tiles = (M + BM - 1) / BM;
+        p.band = (int)(want < m_tiles ? want : m_tiles);
+    }
     return AMX_OK;
 }
 
