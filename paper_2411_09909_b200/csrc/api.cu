@@ -377,17 +377,8 @@ extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_
     const float alpha = 1.0f / sqrtf((float)d);
     float* S = reinterpret_cast<float*>(w + a.S);
     const int64_t chunk = attn_chunk(L, d);
-    // both products on the FP4 kernel and whole 256-column tiles: softmax and cast run in the first product's
-    // epilogue (the S region of the workspace then only holds the per-tile row statistics)
+    // both products on the FP4 kernel at head dimension 128: one fused kernel, logits and attention map stay on chip
     const bool fused = k_qk == AMX_GEMM_FP4 && k_pv == AMX_GEMM_FP4 && attn_fused_supported(L, d);
-    const bool two_pass = !fused && k_qk == AMX_GEMM_FP4 && k_pv == AMX_GEMM_FP4 && L % 256 == 0 &&
-                          gemm_fp4_attn_scratch_bytes(L) <= (size_t)L * L * 4;
-    // At head dimension 128 one head's P V has only L / 128 tiles: two heads' attention maps are cast into one
-    // stacked operand (in the unused part of the S region, behind the statistics) and multiplied in one launch.
-    const size_t stats_bytes = round_up(gemm_fp4_attn_scratch_bytes(L));
-    const bool pair = two_pass && d == 128 && stats_bytes + gemm_fp4_prepared_bytes(2 * L, L, false) <= (size_t)L * L * 4;
-    uint8_t* p_prep = pair ? w + a.S + stats_bytes : w + a.pp;
-    const int64_t p_rows = pair ? 2 * L : L;
     const size_t head_in = (size_t)L * d * 2;                       // bytes of one head of q, k or v
     const size_t qk_codes = (size_t)L * d / 2, qk_scales = (size_t)L * (d / 32) * 2;   // one head of Q or K, canonical
     const size_t v_codes = (size_t)d * L / 2, v_scales = (size_t)d * (L / 32) * 2;     // one head of V^T
@@ -418,18 +409,7 @@ extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_
             if (rc != AMX_OK) return rc;
             continue;
         }
-        for (int64_t i = 0; two_pass && i < hc; i += pair ? 2 : 1) {
-            // the logits never reach memory: Q K^T runs twice, its epilogues do the softmax and the cast of P
-            const int nb = pair && i + 1 < hc ? 2 : 1;
-            for (int j = 0; j < nb && rc == AMX_OK; ++j)
-                rc = gemm_fp4_attn_scores({w + a.pq, hc * L, chunk * L, (i + j) * L}, {w + a.pk, hc * L, chunk * L + 128, (i + j) * L},
-                                          L, d, alpha, S, nullptr, nullptr, p_prep, w + a.gemm, st, causal, p_rows, j * L);
-            if (rc == AMX_OK)
-                rc = gemm_fp4_prepared_at({p_prep, nb * L, p_rows, 0, /*single_plane=*/true}, {w + a.pv, hc * d, chunk * d + 128, i * d},
-                                          nb * L, d, L, o + (size_t)(h0 + i) * L * d, d, w + a.gemm, st, 256, causal, nb, d);
-            if (rc != AMX_OK) return rc;
-        }
-        for (int64_t i = 0; !two_pass && i < hc; ++i) {
+        for (int64_t i = 0; i < hc; ++i) {
             float* oh = o + (size_t)(h0 + i) * L * d;
             // S = AMX(Q) AMX(K)^T
             if (k_qk == AMX_GEMM_FP4)

@@ -64,14 +64,9 @@ int gemm_fp4_softmax_prepared(const float* S, int64_t rows, int64_t cols, int64_
 struct Fp4Operand {
     const void* prepared;
     int64_t rows_total, layout_rows, row0;
-    bool single_plane = false;   // left-hand operand only: its negative plane was never written (the two-pass
-                                 // attention scores write P's positive plane alone) and must not be read
 };
 int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
                          int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes = 256,
-                         int causal_pv = 0 /* 1: the product P V of causal attention (A = P, square) */,
-                         int batch = 1 /* > 1 (N <= 128): a stack of `batch` independent products of M / batch rows */,
-                         int64_t w_batch_rows = 0 /* rows between their right-hand operands in the stacked W */,
                          const int* gate = nullptr /* device word: the kernel does nothing when it is nonzero */,
                          const float* scale_a = nullptr, const float* scale_w = nullptr /* device: one factor per
                          operand; every result is multiplied by their product (NVFP4 tensor scales) */);
@@ -80,14 +75,6 @@ size_t gemm_fp4_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K);
 // C[m][n] = sum over `slices` partial products [slices][M][N], in slice order (defined with the bf16-decode kernel)
 int reduce_slices(const float* part, int slices, int64_t M, int64_t N, float* C, int64_t ld_c, cudaStream_t st,
                   const int* run_if_nonzero = nullptr);
-// P = softmax(alpha * Q K^T) cast to AMXFP4 (canonical + prepared left-hand operand) without the logits in
-// memory; L % 256 == 0; scratch of gemm_fp4_attn_scratch_bytes(L) bytes.
-size_t gemm_fp4_attn_scratch_bytes(int64_t L);
-int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, int64_t d, float alpha, void* scratch,
-                         uint8_t* p_codes, uint8_t* p_scales, void* p_prepared, void* workspace, cudaStream_t st,
-                         int causal = 0, int64_t p_layout_rows = 0 /* 0: L */, int64_t p_row0 = 0,
-                         void* p_bits = nullptr /* optional out: the bf16 map the cast started from, [L, L] */);
-// p_codes / p_scales may be NULL as well: only the prepared operand is written then.
 // Fused attention for head dimension 128 (attention_fp4.cu): both products and the softmax in two launches, logits
 // and attention map never in global memory.  Operands prepared ahead, heads stacked row-wise.
 bool attn_fused_supported(int64_t L, int64_t d);

@@ -31,10 +31,8 @@
 // codes and scales.  Every device-side wait is bounded.
 #include <cstdlib>
 
-#include "cast_math.cuh"
 #include "fp4_operand.cuh"
 #include "gemm.cuh"
-#include "softmax_math.cuh"
 #include "tcgen05.cuh"
 
 namespace amx {
@@ -72,7 +70,7 @@ struct __align__(16) Control {
     uint64_t full[kMaxStages], empty[kMaxStages], accum_full, accum_empty;
     uint32_t tmem_base;
     volatile int abort;
-    alignas(16) int w_exp[2][BN];   // read as int4 in the epilogue (as float4 column factors in the attention modes)
+    alignas(16) int w_exp[2][BN];   // read as int4 in the epilogue
 };
 static_assert(sizeof(Control) <= 2048 + 256, "Control must fit its reserved space");
 
@@ -202,16 +200,6 @@ struct Params {
 
     float* C;
     int nk64, vec_store;
-    int causal;                  // attention with a causal mask: 1 = the tile is a block of logits Q K^T (tiles whose
-                                 // keys all lie after their queries are skipped, the epilogue masks the diagonal
-                                 // ones); 2 = the product P V (K blocks after the tile's last query row hold only
-                                 // zeros of P and are skipped)
-    int a_single;                // the left-hand operand has only its positive plane in memory (a cast softmax
-                                 // output): the tensor map's box is one plane deep, the negative plane's products
-                                 // are skipped anyway (row words)
-    int mt_batch;                // half-width instantiation: > 0 = the product is a stack of independent ones, mt_batch
-    int64_t w_batch_rows;        //   row blocks of A each, whose right-hand operands lie w_batch_rows rows apart (a
-                                 //   multiple of 128) in the stacked W; C is the stack of the results
     int band;                    // tile order: row blocks of A per band, see blk_m / blk_n
     int slices;                  // SLICED instantiation: K is cut into this many ranges, each (tile, range) a work item
     int64_t slice_stride;        //   whose partial product goes to C + range * slice_stride
@@ -220,24 +208,7 @@ struct Params {
                                  // the store epilogue multiplies every result by their product
     const int* gate;             // not NULL: the kernel returns at once when this word is nonzero (the caller then
                                  // runs the exact bf16-decode kernel on the same operands, gated the other way)
-    // attention epilogues (kEpiStats, kEpiCast): the tile holds logits S = Q K^T; `alpha` scales them
-    float alpha;
-    float2* part;            // kEpiStats out: per row and half tile {max, sum of exp} of alpha * S, [M][2 * n_tiles]
-    const float2* rowstat;   // kEpiCast in: per row {-max * log2(e), 1 / sum}
-    const int* p_kmax;       // kEpiCast in: per row the largest exponent key of the row's scales
-    uint4* p_pos;            // kEpiCast out: the positive plane of P = softmax(alpha * S), cast to AMXFP4
-    // kEpiCast, optional outputs (NULL in the attention call itself; amx_attention_map asks for them so that the
-    // cast done in this epilogue can be compared with a reference): the bf16 words the cast started from
-    // [M][N / 2 words], the canonical codes [M][N / 32 groups] and scale bytes {0 : positive scale} per group
-    uint4 *p_bits, *p_codes;
-    uint16_t* p_scales;
-    uint8_t* p_sf;           // scale factors of the positive plane (P has no negative element)
-    int p_nk64;
 };
-// What the epilogue does with a finished tile: store it as fp32; or, when the tile is a block of attention
-// logits, reduce it to per-row softmax statistics; or turn it into the AMXFP4 cast of the normalised map.
-constexpr int kEpiStore = 0, kEpiStats = 1, kEpiCast = 2;
-
 // 16 consecutive fp32 results of one row -> global memory, as two 32-byte stores when allowed.
 __device__ __forceinline__ void store_row16(float* out, const float (&f)[16], bool vec, int64_t n_left) {
     if (vec && n_left >= 16) {
@@ -252,15 +223,14 @@ __device__ __forceinline__ void store_row16(float* out, const float (&f)[16], bo
     }
 }
 
-// NHALF: tiles of 128 x 128 for products with at most 128 columns (the P V product of attention at head
-// dimension 128): the W box, the MMA and the epilogue are half as wide, the stage layout keeps its size.
-template <int BK_, int EPI = kEpiStore, bool SLICED = false, bool CAUSAL = false, bool NHALF = false>
+// NHALF: tiles of 128 x 128 for products with at most 128 columns: the W box, the MMA and the epilogue are half as
+// wide, the stage layout keeps its size.
+template <int BK_, bool SLICED = false, bool NHALF = false>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w, const Params p) {
     using C_ = Cfg<BK_>;
     if (p.gate && *p.gate != 0) return;                          // uniform over the grid: nothing was set up yet
     constexpr int BNT = NHALF ? BN / 2 : BN;                     // tile width
-    static_assert(!NHALF || EPI == kEpiStore, "half-width tiles: plain epilogue only");
     constexpr int kOffWnT = NHALF ? C_::kOffWp + C_::kTileB / 2 : C_::kOffWn;   // the box packs its two planes
     constexpr uint32_t kIdescT = (1u << 7) | (1u << 10) | ((uint32_t)(BNT >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
     constexpr int BK = C_::BK, kRowBytes = C_::kRowBytes, kSteps = C_::kSteps, kStages = C_::kStages;
@@ -277,20 +247,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     auto kb_begin = [&](int64_t tile) -> int { return SLICED ? (int)((int)(tile % S) * kb_total / S) : 0; };
     // Persistent CTA: tiles blockIdx.x, blockIdx.x + gridDim.x, ...; neighbouring tiles share their A rows.
     const int64_t n_tiles = (p.N + BNT - 1) / BNT, m_tiles = (p.M + BM - 1) / BM;
-    // Causal logits (square, keys after the queries masked): only the tiles on or below the diagonal exist.  Row
-    // block m has the column blocks 0 .. m/2 (a tile is 128 queries x 256 keys), so f(m) = tiles before row
-    // block m is j(j+1) for m = 2j and (j+1)^2 for m = 2j+1; the work items enumerate exactly those tiles, which
-    // keeps the persistent CTAs evenly loaded.
-    const bool compact = CAUSAL && p.causal == 1;
-    const int64_t half = m_tiles / 2;
-    const int64_t total_tiles = compact ? ((m_tiles & 1) ? (half + 1) * (half + 1) : half * (half + 1)) : m_tiles * n_tiles * S;
-    auto compact_mn = [&](uint32_t c, uint32_t& m, uint32_t& n) {
-        uint32_t j = (uint32_t)((sqrtf(4.0f * (float)c + 1.0f) - 1.0f) * 0.5f);
-        while (j * (j + 1) > c) --j;                      // the float estimate can be off by one
-        while ((j + 1) * (j + 2) <= c) ++j;
-        if (c < (j + 1) * (j + 1)) { m = 2 * j; n = c - j * (j + 1); }
-        else { m = 2 * j + 1; n = c - (j + 1) * (j + 1); }
-    };
+    const int64_t total_tiles = m_tiles * n_tiles * S;
     // Tile order.  The CTAs work on ~148 consecutive tiles at a time and advance through K roughly together, so what
     // they read from DRAM per wave is the operand rows the wave touches, once.  Tiles are ordered in bands of
     // p.band row blocks of A: inside a band the tile index walks down the band's row blocks first, then along N.
@@ -308,30 +265,18 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     };
     auto blk_m = [&](int64_t tile) -> int64_t {
         uint32_t m, n;
-        if (compact) compact_mn((uint32_t)tile, m, n);
-        else banded(tile, m, n);
+        banded(tile, m, n);
         return m;
     };
     auto blk_n = [&](int64_t tile) -> int64_t {
         uint32_t m, n;
-        if (compact) compact_mn((uint32_t)tile, m, n);
-        else banded(tile, m, n);
+        banded(tile, m, n);
         return n;
     };
-    // rows by which the right-hand operand of row block m_blk is shifted (stack of independent products)
-    auto w_shift = [&](int64_t m_blk) -> int64_t {
-        if (!NHALF || p.mt_batch == 0) return 0;
-        return (int64_t)((uint32_t)m_blk / (uint32_t)p.mt_batch) * p.w_batch_rows;
-    };
-    // K blocks of a tile (of an item): all of them, fewer or none under a causal mask (see Params::causal)
+    // K blocks of a tile (of an item)
     auto nkb_of = [&](int64_t tile) -> int {
         if (SLICED) return (int)(((int)(tile % S) + 1) * kb_total / S) - kb_begin(tile);
-        if (!CAUSAL || p.causal == 0) return num_kb;
-        int64_t mb = blk_m(tile);
-        if (NHALF && p.mt_batch) mb = (int64_t)((uint32_t)mb % (uint32_t)p.mt_batch);   // row block inside its product
-        const int64_t last_row = mb * BM + BM - 1;
-        if (p.causal == 1) return num_kb;                 // the enumeration holds no masked tile
-        return (int)min((int64_t)num_kb, (last_row + BK) / BK);
+        return num_kb;
     };
 
     if (threadIdx.x == 0) {
@@ -365,10 +310,10 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                         break;
                     }
                     uint8_t* st = tiles + s * kStageBytes;
-                    mbar_expect_tx(&ctl->full[s], kStageBytes - (p.a_single ? C_::kTileA : 0) - (NHALF ? C_::kTileB : 0));
+                    mbar_expect_tx(&ctl->full[s], kStageBytes - (NHALF ? C_::kTileB : 0));
                     // one 3-D tile per operand: {row bytes, rows, both sign planes}
                     tma_load_3d(st + C_::kOffAp, &tm_a, (kb0 + kb) * kRowBytes, (int)(p.a_row0 + m_blk * BM), 0, &ctl->full[s]);
-                    tma_load_3d(st + C_::kOffWp, &tm_w, (kb0 + kb) * kRowBytes, (int)(p.w_row0 + w_shift(m_blk) + n_blk * BNT), 0, &ctl->full[s]);
+                    tma_load_3d(st + C_::kOffWp, &tm_w, (kb0 + kb) * kRowBytes, (int)(p.w_row0 + n_blk * BNT), 0, &ctl->full[s]);
                 }
             }
             // after an abort: let the copies already in flight land before shared memory is released
@@ -389,9 +334,9 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         // next tile are fetched while the current one runs.
         auto tile_sides = [&](int64_t tile) {
             int bits = 0;
-            if (tile < total_tiles && nkb_of(tile) > 0) {            // a skipped tile costs no load latency
+            if (tile < total_tiles) {
                 const int64_t m0 = blk_m(tile) * BM, n0 = blk_n(tile) * BNT;
-                const int* w_words = p.w_exp + w_shift(blk_m(tile));
+                const int* w_words = p.w_exp;
 #pragma unroll
                 for (int i = 0; i < BM / 32; ++i)
                     if (m0 + i * 32 + lane < p.M) bits |= (__ldg(p.a_exp + m0 + i * 32 + lane) >> 16) & 3;
@@ -406,7 +351,6 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             int sides = __reduce_or_sync(0xFFFFFFFFu, sides_next);   // bit 0/1: A has +/-, bit 2/3: W has +/-
             sides_next = tile_sides(tile + gridDim.x);
             const int nkb = nkb_of(tile);
-            if (nkb == 0) continue;                              // masked out entirely: no accumulator, no epilogue
             if (!(sides & 3)) sides |= 1;                        // an all-zero operand: one product, which zeroes the tile
             if (!(sides & 12)) sides |= 4;
             const int n_mma = ((sides & 1) + ((sides >> 1) & 1)) * (((sides >> 2) & 1) + ((sides >> 3) & 1)) * kSteps;
@@ -474,7 +418,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 for (int kk = 0; kk < kSteps; ++kk) {
                     const int64_t c = ((int64_t)kb_begin(tile) + kb) * kSteps + kk;
                     const uint8_t* a = (pl ? p.sfa_neg : p.sfa_pos) + (m_blk * p.nk64 + c) * kSfChunk + lane * 16;
-                    const uint8_t* w = (pl ? p.sfb_neg : p.sfb_pos) + ((n_blk * (BNT / 128) + w_shift(m_blk) / 128) * p.nk64 + c) * kSfChunk + lane * 16;
+                    const uint8_t* w = (pl ? p.sfb_neg : p.sfb_pos) + (n_blk * (BNT / 128) * p.nk64 + c) * kSfChunk + lane * 16;
                     sfv[(pl * kSteps + kk) * 3 + 0] = __ldg(reinterpret_cast<const uint4*>(a));
                     sfv[(pl * kSteps + kk) * 3 + 1] = __ldg(reinterpret_cast<const uint4*>(w));
                     sfv[(pl * kSteps + kk) * 3 + 2] =           // second block of 128 rows (none in a half-width tile)
@@ -520,43 +464,31 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         int t = 0;
         bool ok = true;
         static_assert(kEpilogueWarps * 32 == BN, "one column offset per epilogue thread");   // BNT <= BN
-        // The per-tile constants (this thread's column offset and row offset; in the cast pass the row's softmax
-        // statistics) are fetched one tile ahead, so that their latency is off the path between two tiles.
+        // The per-tile constants (this thread's column offset and row offset) are fetched one tile ahead, so that
+        // their latency is off the path between two tiles.
         struct TileConsts {
-            int w_ex, a_ex, kmax;
-            float2 rs;
-        };
-        auto next_live = [&](int64_t tl) {
-            while (tl < total_tiles && nkb_of(tl) == 0) tl += gridDim.x;
-            return tl;
+            int w_ex, a_ex;
         };
         auto load_consts = [&](int64_t tl) {
-            TileConsts c = {0, 0, 0, make_float2(0.f, 0.f)};
+            TileConsts c = {0, 0};
             if (tl < total_tiles) {
                 const int64_t n = blk_n(tl) * BNT + tid_e, mm = blk_m(tl) * BM + q * 32 + lane;
-                if (tid_e < BNT && n < p.N) c.w_ex = row_word_exp(__ldg(p.w_exp + w_shift(blk_m(tl)) + n));
-                if (mm < p.M) {
-                    c.a_ex = row_word_exp(__ldg(p.a_exp + mm));
-                    if constexpr (EPI == kEpiCast) {
-                        c.rs = p.rowstat[mm];
-                        c.kmax = p.p_kmax[mm];
-                    }
-                }
+                if (tid_e < BNT && n < p.N) c.w_ex = row_word_exp(__ldg(p.w_exp + n));
+                if (mm < p.M) c.a_ex = row_word_exp(__ldg(p.a_exp + mm));
             }
             return c;
         };
-        const float out_scale = (EPI == kEpiStore && p.scale_a) ? __ldg(p.scale_a) * __ldg(p.scale_w) : 1.0f;
-        int64_t tile = next_live(blockIdx.x);
+        const float out_scale = p.scale_a ? __ldg(p.scale_a) * __ldg(p.scale_w) : 1.0f;
+        int64_t tile = blockIdx.x;
         TileConsts nxt = load_consts(tile);
         while (tile < total_tiles && ok) {
             const TileConsts cur = nxt;
-            const int64_t tile_after = next_live(tile + gridDim.x);
+            const int64_t tile_after = tile + gridDim.x;
             nxt = load_consts(tile_after);                       // in flight while this tile is worked on
             const int64_t m0 = blk_m(tile) * BM, n0 = blk_n(tile) * BNT;
             float* const C_item = p.C + (SLICED ? (tile % S) * p.slice_stride : 0);
             int* w_exp = ctl->w_exp[t & 1];
-            if constexpr (EPI == kEpiStore) w_exp[tid_e] = cur.w_ex;
-            else w_exp[tid_e] = __float_as_int(p.alpha * 1.4426950408889634f * __uint_as_float((uint32_t)(cur.w_ex + 127) << 23));
+            w_exp[tid_e] = cur.w_ex;
             const int64_t m = m0 + q * 32 + lane;
             const int a_exp = cur.a_ex;
             ok = mbar_wait(&ctl->accum_full, t & 1, &ctl->abort, p.status);
@@ -565,119 +497,26 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueWarps * 32) : "memory");
             if (ok) {
                 const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)col_base;
-                if constexpr (EPI == kEpiStore) {
-                    uint32_t v[2][16];
-                    tmem_ld16(taddr, v[0]);
+                uint32_t v[2][16];
+                tmem_ld16(taddr, v[0]);
 #pragma unroll
-                    for (int c = 0; c < BNT / 2; c += 16) {
-                        const int buf = (c / 16) & 1;
-                        tmem_ld_wait();
-                        if (c + 16 < BNT / 2) tmem_ld16(taddr + c + 16, v[buf ^ 1]);   // next chunk loads while this one is stored
-                        const int col = col_base + c;
-                        float f[16];
+                for (int c = 0; c < BNT / 2; c += 16) {
+                    const int buf = (c / 16) & 1;
+                    tmem_ld_wait();
+                    if (c + 16 < BNT / 2) tmem_ld16(taddr + c + 16, v[buf ^ 1]);   // next chunk loads while this one is stored
+                    const int col = col_base + c;
+                    float f[16];
 #pragma unroll
-                        for (int j = 0; j < 16; j += 4) {
-                            const int4 we = *reinterpret_cast<const int4*>(&w_exp[col + j]);
-                            const int ex[4] = {we.x, we.y, we.z, we.w};
+                    for (int j = 0; j < 16; j += 4) {
+                        const int4 we = *reinterpret_cast<const int4*>(&w_exp[col + j]);
+                        const int ex[4] = {we.x, we.y, we.z, we.w};
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                const int sh = min(127, max(-126, a_exp + ex[i]));
-                                f[j + i] = __uint_as_float(v[buf][j + i]) * __uint_as_float((uint32_t)(sh + 127) << 23) * out_scale;
-                            }
-                        }
-                        if (m < p.M) store_row16(C_item + m * p.ld_c + n0 + col, f, p.vec_store != 0, p.N - (n0 + col));
-                    }
-                } else {
-                    // The thread's 128 columns come from tensor memory 16 at a time, the next chunk in flight while
-                    // the current one is worked on.  u = accumulator x (alpha log2(e) 2^w_exp[col]) is the logit in
-                    // base-2 units up to the row's power of two ra, by which multiplying is exact: t = u ra.
-                    const float* w_fac = reinterpret_cast<const float*>(w_exp);
-                    const float ra = __uint_as_float((uint32_t)(a_exp + 127) << 23);
-                    uint32_t v[2][16];
-                    tmem_ld16(taddr, v[0]);
-                    auto chunk16 = [&](int c, float (&u)[16]) {
-                        const int buf = (c / 16) & 1;
-                        tmem_ld_wait();
-                        if (c + 16 < BN / 2) tmem_ld16(taddr + c + 16, v[buf ^ 1]);
-#pragma unroll
-                        for (int j = 0; j < 16; j += 4) {
-                            const float4 k = *reinterpret_cast<const float4*>(&w_fac[col_base + c + j]);
-                            u[j] = __uint_as_float(v[buf][j]) * k.x;
-                            u[j + 1] = __uint_as_float(v[buf][j + 1]) * k.y;
-                            u[j + 2] = __uint_as_float(v[buf][j + 2]) * k.z;
-                            u[j + 3] = __uint_as_float(v[buf][j + 3]) * k.w;
-                        }
-                        if (CAUSAL && p.causal && n0 + col_base + c + 15 > m) {      // keys after this query: masked out
-#pragma unroll
-                            for (int j = 0; j < 16; ++j)
-                                if (n0 + col_base + c + j > m) u[j] = -INFINITY;
-                        }
-                    };
-                    auto exp2_approx = [](float y) {
-                        float r;
-                        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(y));
-                        return r;
-                    };
-                    if constexpr (EPI == kEpiStats) {
-                        // One sweep: running maximum (base-2 units), and the sum of 2^(t - max) rescaled whenever the
-                        // maximum grows.
-                        float mx = -INFINITY, sum = 0.f;
-#pragma unroll
-                        for (int c = 0; c < BN / 2; c += 16) {
-                            float u[16];
-                            chunk16(c, u);
-                            // four chains instead of one: the two epilogue warps of a scheduler are latency-bound
-                            float c4[4] = {u[0], u[1], u[2], u[3]};
-#pragma unroll
-                            for (int j = 4; j < 16; ++j) c4[j & 3] = fmaxf(c4[j & 3], u[j]);
-                            const float cm = fmaxf(fmaxf(c4[0], c4[1]), fmaxf(c4[2], c4[3]));
-                            const float nmx = fmaxf(mx, cm * ra);
-                            // 2^(-inf) = 0 on the first chunk; a maximum still at -inf (everything masked so far)
-                            // must not meet itself in a difference
-                            const float ref = nmx == -INFINITY ? 0.f : nmx;
-                            sum *= exp2_approx(mx - ref);
-                            mx = nmx;
-                            float s4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) s4[j & 3] += exp2_approx(fmaf(u[j], ra, -ref));
-                            sum += (s4[0] + s4[1]) + (s4[2] + s4[3]);
-                        }
-                        if (m < p.M) p.part[m * (2 * n_tiles) + blk_n(tile) * 2 + (e >> 2)] = make_float2(mx, sum);
-                    } else {
-                        // Four 32-column groups per thread: normalise with the row's statistics {-max, 1 / sum}, round
-                        // to bf16, cast.  P has no negative element: only its positive plane and scale factors exist.
-                        const float2 rs = cur.rs;
-                        const int kmax = cur.kmax;
-                        const int64_t G = p.N / 32, g0 = (n0 + col_base) / 32;
-                        const int64_t sf_row = sf_row_offset(m, p.p_nk64);
-#pragma unroll
-                        for (int gi = 0; gi < BN / 2 / 32; ++gi) {
-                            uint32_t w[16];
-#pragma unroll
-                            for (int h = 0; h < 2; ++h) {
-                                float u[16];
-                                chunk16(gi * 32 + h * 16, u);
-#pragma unroll
-                                for (int i = 0; i < 8; ++i) {
-                                    const __nv_bfloat162 pr = __floats2bfloat162_rn(exp2_approx(fmaf(u[2 * i], ra, rs.x)) * rs.y,
-                                                                                    exp2_approx(fmaf(u[2 * i + 1], ra, rs.x)) * rs.y);
-                                    w[h * 8 + i] = *reinterpret_cast<const uint32_t*>(&pr);
-                                }
-                            }
-                            if (m < p.M) {
-                                const int64_t g = g0 + gi;
-                                const uint32_t sc = cast::emit_nonneg_plane(w, m * G + g, p.p_pos, p.p_codes);
-                                const uint32_t up = to_ue4m3(sc, kmax);
-                                *reinterpret_cast<uint16_t*>(p.p_sf + sf_row + sf_group_offset((int)g)) = (uint16_t)(up | (up << 8));
-                                if (p.p_scales) p.p_scales[m * G + g] = (uint16_t)sc;
-                                if (p.p_bits) {
-#pragma unroll
-                                    for (int j = 0; j < 4; ++j)
-                                        p.p_bits[(m * G + g) * 4 + j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
-                                }
-                            }
+                        for (int i = 0; i < 4; ++i) {
+                            const int sh = min(127, max(-126, a_exp + ex[i]));
+                            f[j + i] = __uint_as_float(v[buf][j + i]) * __uint_as_float((uint32_t)(sh + 127) << 23) * out_scale;
                         }
                     }
+                    if (m < p.M) store_row16(C_item + m * p.ld_c + n0 + col, f, p.vec_store != 0, p.N - (n0 + col));
                 }
                 // this warp's part of the accumulator has been read: the next tile may overwrite it
                 tc_fence_before();
@@ -720,26 +559,26 @@ size_t gemm_fp4_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 
 namespace {
 
-template <int BK_, int EPI = kEpiStore, bool SLICED = false, bool CAUSAL = false, bool NHALF = false>
+template <int BK_, bool SLICED = false, bool NHALF = false>
 int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, const OperandLayout& ow, int64_t a_rows,
                int64_t w_rows, Params p, int dev, cudaStream_t st) {
     using C_ = Cfg<BK_>;
     constexpr int BNT = NHALF ? BN / 2 : BN;
     static bool configured[64] = {};
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(gemm_fp4_kernel<BK_, EPI, SLICED, CAUSAL, NHALF>, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(gemm_fp4_kernel<BK_, SLICED, NHALF>, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::kSmemBytes) != cudaSuccess)
             return AMX_ERR_CUDA;
         configured[dev] = true;
     }
     CUtensorMap tm_a, tm_w;
-    if (!make_map(&tm_a, pa, a_rows, p.K, oa.plane, BM, C_::kRowBytes, p.a_single ? 1 : 2) || !make_map(&tm_w, pw, w_rows, p.K, ow.plane, BNT, C_::kRowBytes))
+    if (!make_map(&tm_a, pa, a_rows, p.K, oa.plane, BM, C_::kRowBytes) || !make_map(&tm_w, pw, w_rows, p.K, ow.plane, BNT, C_::kRowBytes))
         return AMX_ERR_CUDA;
     static int sm_count[64] = {};
     if (!sm_count[dev] && cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return AMX_ERR_CUDA;
     const int64_t tiles = ((p.N + BNT - 1) / BNT) * ((p.M + BM - 1) / BM) * (SLICED ? p.slices : 1);
     const unsigned grid = (unsigned)(tiles < sm_count[dev] ? tiles : sm_count[dev]);   // one persistent CTA per SM
-    gemm_fp4_kernel<BK_, EPI, SLICED, CAUSAL, NHALF><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_a, tm_w, p);
+    gemm_fp4_kernel<BK_, SLICED, NHALF><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_a, tm_w, p);
     return launch_status();
 }
 
@@ -789,36 +628,6 @@ int fill_params(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, 
     return AMX_OK;
 }
 
-// One warp per query row: the row's softmax statistics from the per-tile partial ones, and the row word of
-// the cast attention map (its largest element is exp(0) / sum, whose group has the row's largest scale).
-__global__ void __launch_bounds__(256)
-attn_row_reduce_kernel(const float2* __restrict__ part, int n_parts_all, int64_t L, int causal,
-                       float2* __restrict__ rowstat, int* __restrict__ p_kmax, int* __restrict__ p_row_word) {
-    const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (row >= L) return;
-    const float2* pr = part + row * n_parts_all;      // {max, sum of 2^(t - max)} per half tile, base-2 units
-    // causal: the half tiles (128 keys each) that start after this query were skipped and hold nothing
-    const int n_parts = causal ? min(n_parts_all, (int)(row / 128) + 1) : n_parts_all;
-    float mx = -INFINITY;
-    for (int j = lane; j < n_parts; j += 32) mx = fmaxf(mx, pr[j].x);
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, d));
-    float sum = 0.f;
-    for (int j = lane; j < n_parts; j += 32) sum += pr[j].y * exp2f(pr[j].x - mx);
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, d);
-    if (lane) return;
-    const float inv = 1.0f / sum;
-    rowstat[row] = make_float2(-mx, inv);
-    // the row's largest element is 2^0 / sum
-    const __nv_bfloat16 pmax = __float2bfloat16_rn(inv);
-    float inv_p, inv_n;
-    const uint32_t sc = cast::group_scales((uint32_t)__bfloat16_as_ushort(pmax), inv_p, inv_n);   // {nmax = 0 : pmax}
-    const int kmax = scale_key(sc & 0xFFu);
-    p_kmax[row] = kmax;
-    p_row_word[row] = row_word(kmax, side_bits_of(sc));
-}
 }  // namespace
 
 // Few output tiles and a long K (a few token rows against a big weight): K ranges as separate work items, so
@@ -840,31 +649,21 @@ size_t gemm_fp4_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 // The GEMM proper on two prepared operands (each laid out by operand_layout()), or on row ranges of them.
 // workspace_bytes >= gemm_fp4_prepared_workspace_bytes() enables the K ranges; 256 bytes always suffice.
 int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
-                         int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes, int causal_pv, int batch,
-                         int64_t w_batch_rows, const int* gate, const float* scale_a, const float* scale_w) {
-    if (batch > 1 && (N > BN / 2 || M % batch || (M / batch) % BM || w_batch_rows % 128)) return AMX_ERR_SHAPE;
+                         int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes, const int* gate,
+                         const float* scale_a, const float* scale_w) {
     Params p;
     OperandLayout oa, ow;
     int dev;
     const int rc = fill_params(a, w, M, N, K, C, ld_c, workspace, st, p, oa, ow, dev);
     if (rc != AMX_OK) return rc;
-    p.causal = causal_pv ? 2 : 0;
-    p.a_single = a.single_plane ? 1 : 0;
     p.gate = gate;
     p.scale_a = scale_a;
     p.scale_w = scale_w;
     const uint8_t* pa = static_cast<const uint8_t*>(a.prepared);
     const uint8_t* pw = static_cast<const uint8_t*>(w.prepared);
-    const int slices = batch > 1 ? 1 : gemm_fp4_slices(M, N, K);
-    // at most 128 columns (P V at head dimension 128): tiles of 128 x 128, so that no half of a W tile is padding
-    const bool half = N <= BN / 2 && (batch > 1 || !getenv("AMX_FP4_NO_HALF_TILE"));
-    if (batch > 1) {
-        p.mt_batch = (int)(M / batch / BM);
-        p.w_batch_rows = w_batch_rows;
-    }
-    if (causal_pv)
-        return half ? launch_fp4<128, kEpiStore, false, true, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st)
-                    : launch_fp4<128, kEpiStore, false, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
+    const int slices = gemm_fp4_slices(M, N, K);
+    // at most 128 columns: tiles of 128 x 128, so that no half of a W tile is padding
+    const bool half = N <= BN / 2 && !getenv("AMX_FP4_NO_HALF_TILE");
     if (!gate && !scale_a && slices > 1 && fp4_block_k() == 128 && workspace_bytes >= gemm_fp4_prepared_workspace_bytes(M, N, K)) {
         float* part = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 256);
         p.C = part;
@@ -872,69 +671,18 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
         p.vec_store = N % 8 == 0;
         p.slices = slices;
         p.slice_stride = M * N;
-        const int r2 = launch_fp4<128, kEpiStore, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
+        const int r2 = launch_fp4<128, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
         return r2 != AMX_OK ? r2 : reduce_slices(part, slices, M, N, C, ld_c, st);
     }
-    if (fp4_block_k() == 256 && batch == 1) return launch_fp4<256>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
-    return half ? launch_fp4<128, kEpiStore, false, false, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st)
+    if (fp4_block_k() == 256) return launch_fp4<256>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
+    return half ? launch_fp4<128, false, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st)
                 : launch_fp4<128>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
-}
-
-// Attention scores without the logits in memory: P = softmax(alpha * Q K^T) cast to AMXFP4 as the prepared
-// left-hand operand of P V (and its canonical codes and scales).  The product runs twice: the first pass keeps
-// only per-row softmax statistics of each tile, a small kernel merges them, the second pass normalises, rounds
-// to bf16 and casts each tile in the epilogue.  L % 256 == 0.  scratch: fused_attention_scratch_bytes(L).
-size_t gemm_fp4_attn_scratch_bytes(int64_t L) {
-    return up256((size_t)L * (2 * (L / BN)) * sizeof(float2)) + up256((size_t)L * sizeof(float2)) + up256((size_t)L * 4);
-}
-int gemm_fp4_attn_scores(const Fp4Operand& q, const Fp4Operand& k, int64_t L, int64_t d, float alpha, void* scratch,
-                         uint8_t* p_codes, uint8_t* p_scales, void* p_prepared, void* workspace, cudaStream_t st,
-                         int causal, int64_t p_layout_rows, int64_t p_row0, void* p_bits) {
-    if (p_layout_rows == 0) p_layout_rows = L;
-    if (p_row0 % 128 || p_row0 + L > p_layout_rows) return AMX_ERR_SHAPE;
-    if (L % BN) return AMX_ERR_SHAPE;
-    Params p;
-    OperandLayout oq, ok_;
-    int dev;
-    int rc = fill_params(q, k, L, L, d, nullptr, L, workspace, st, p, oq, ok_, dev);
-    if (rc != AMX_OK) return rc;
-    const uint8_t* pq = static_cast<const uint8_t*>(q.prepared);
-    const uint8_t* pk = static_cast<const uint8_t*>(k.prepared);
-    const int n_parts = (int)(2 * (L / BN));
-    uint8_t* sc = static_cast<uint8_t*>(scratch);
-    float2* part = reinterpret_cast<float2*>(sc);
-    float2* rowstat = reinterpret_cast<float2*>(sc + up256((size_t)L * n_parts * sizeof(float2)));
-    int* p_kmax = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(rowstat) + up256((size_t)L * sizeof(float2)));
-    const OperandLayout op = operand_layout(p_layout_rows, L, BM);
-    uint8_t* pp = static_cast<uint8_t*>(p_prepared);
-    uint8_t* p_plane = pp + (size_t)p_row0 * (L / 2);
-    uint8_t* p_sf = pp + 2 * op.plane + (size_t)(p_row0 / 128) * op.nk64 * kSfChunk;
-    int* p_words = reinterpret_cast<int*>(pp + 2 * op.plane + 2 * op.sf) + p_row0;
-    p.alpha = alpha;
-    p.causal = causal ? 1 : 0;
-    p.part = part;
-    p.rowstat = rowstat;
-    p.p_kmax = p_kmax;
-    p.p_codes = reinterpret_cast<uint4*>(p_codes);      // optional: the prepared operand is all P V needs
-    p.p_scales = reinterpret_cast<uint16_t*>(p_scales);
-    p.p_bits = reinterpret_cast<uint4*>(p_bits);
-    p.p_pos = reinterpret_cast<uint4*>(p_plane);
-    p.p_sf = p_sf;
-    p.p_nk64 = op.nk64;
-    rc = causal ? launch_fp4<128, kEpiStats, false, true>(pq, pk, oq, ok_, q.rows_total, k.rows_total, p, dev, st)
-                : launch_fp4<128, kEpiStats>(pq, pk, oq, ok_, q.rows_total, k.rows_total, p, dev, st);
-    if (rc != AMX_OK) return rc;
-    attn_row_reduce_kernel<<<(unsigned)((L + 7) / 8), 256, 0, st>>>(part, n_parts, L, causal, rowstat, p_kmax, p_words);
-    rc = launch_status();
-    if (rc != AMX_OK) return rc;
-    return causal ? launch_fp4<128, kEpiCast, false, true>(pq, pk, oq, ok_, q.rows_total, k.rows_total, p, dev, st)
-                  : launch_fp4<128, kEpiCast>(pq, pk, oq, ok_, q.rows_total, k.rows_total, p, dev, st);
 }
 
 int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K, float* C,
                       int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes, const int* gate) {
     return gemm_fp4_prepared_at({a_prepared, M, M, 0}, {w_prepared, N, N, 0}, M, N, K, C, ld_c, workspace, st,
-                                workspace_bytes, 0, 1, 0, gate);
+                                workspace_bytes, gate);
 }
 
 // Size of a prepared operand: as the A operand (rows padded to 128) or the W operand (rows padded to 256).

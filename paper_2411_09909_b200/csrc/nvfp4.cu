@@ -237,5 +237,5 @@ extern "C" int amx_gemm_nvfp4(const void* a_prepared, const void* w_prepared, in
     const float* sa = reinterpret_cast<const float*>(static_cast<const uint8_t*>(a_prepared) + fp4::operand_layout(M, K, 128).total);
     const float* sw = reinterpret_cast<const float*>(static_cast<const uint8_t*>(w_prepared) + fp4::operand_layout(N, K, 256).total);
     return gemm_fp4_prepared_at({a_prepared, M, M, 0}, {w_prepared, N, N, 0}, M, N, K, C, ld_c, workspace,
-                                static_cast<cudaStream_t>(stream), 256, 0, 1, 0, nullptr, sa, sw);
+                                static_cast<cudaStream_t>(stream), 256, nullptr, sa, sw);
 }

@@ -639,7 +639,7 @@ def test_attention_all_heads_entry_point_matches_per_head_pipeline(heads, seq, f
 
 @pytest.mark.parametrize("heads,seq,flags", [(2, 192, amx.GEMM_AUTO),        # stored logits, small-product kernel
                                              (1, 320, amx.GEMM_FP4),         # stored logits, FP4 kernel
-                                             (2, 512, amx.GEMM_FP4),         # two-pass scores, tiles skipped
+                                             (2, 512, amx.GEMM_FP4),         # fused kernel, key blocks after the queries skipped
                                              (1, 1024, amx.GEMM_AUTO)])
 def test_attention_causal_against_oracle_pipeline(heads, seq, flags):
     """Causal attention (query i sees keys 0..i) against the all-CPU pipeline with the mask applied before the
