@@ -61,6 +61,14 @@ def lib() -> ctypes.CDLL:
         L.amx_oracle_quantize_nv.argtypes = [p, i64, i64, i64, ctypes.c_int, p, p, p]
         L.amx_oracle_dequantize_nv.argtypes = [p, p, ctypes.c_float, i64, i64, p]
         L.amx_oracle_gemm_nv.argtypes = [p, p, ctypes.c_float, p, p, ctypes.c_float, i64, i64, i64, p, i64, p]
+        L.amx_oracle_f16_value.restype = dbl
+        L.amx_oracle_f16_value.argtypes = [ctypes.c_uint16]
+        L.amx_oracle_f16_encode.restype = ctypes.c_uint16
+        L.amx_oracle_f16_encode.argtypes = [dbl]
+        L.amx_oracle_quantize_f16s.argtypes = [p, i64, i64, i64, ctypes.c_int, ctypes.c_int, p, p]
+        L.amx_oracle_dequantize_f16s.argtypes = [p, p, i64, i64, ctypes.c_int, p]
+        L.amx_oracle_gemm_f16s.argtypes = [p, p, p, p, i64, i64, i64, ctypes.c_int, p]
+        L.amx_oracle_quant_error_f16s.argtypes = [p, i64, i64, i64, p, p, ctypes.c_int, p]
         L.amx_oracle_num_threads.restype = ctypes.c_int
         _lib = L
     return _lib
@@ -264,3 +272,60 @@ def gemm_nv(codesA, scalesA, tA, codesW, scalesW, tW, rows=None) -> np.ndarray:
     if rc:
         raise ValueError(f"amx_oracle_gemm_nv failed (rc={rc})")
     return C
+
+
+# ---- FP16 shared scales (the scale-encoding ablation of the appendix) ----
+
+def f16_value(bits: int) -> float:
+    return float(lib().amx_oracle_f16_value(int(bits)))
+
+
+def f16_encode(q: float) -> int:
+    return int(lib().amx_oracle_f16_encode(float(q)))
+
+
+def quantize_f16s(x_bf16_bits: np.ndarray, group_size: int, asym: bool):
+    """bf16 bit patterns [rows, K] -> (codes u8 [rows, K/2], binary16 scales u16 [rows, K/gs, 2]).
+    asym True: one scale per sign (positive side, negative side); False: the group's one scale in both."""
+    x = _c(x_bf16_bits, np.uint16)
+    rows, K = x.shape
+    codes = np.zeros((rows, K // 2), np.uint8)
+    scales = np.zeros((rows, K // group_size, 2), np.uint16)
+    rc = lib().amx_oracle_quantize_f16s(_ptr(x), rows, K, K, int(group_size), int(asym), _ptr(codes), _ptr(scales))
+    if rc:
+        raise ValueError("amx_oracle_quantize_f16s: K must be a multiple of the group size")
+    return codes, scales
+
+
+def dequantize_f16s(codes: np.ndarray, scales: np.ndarray, group_size: int) -> np.ndarray:
+    codes, scales = _c(codes, np.uint8), _c(scales, np.uint16)
+    rows, K = codes.shape[0], codes.shape[1] * 2
+    out = np.zeros((rows, K), np.float64)
+    rc = lib().amx_oracle_dequantize_f16s(_ptr(codes), _ptr(scales), rows, K, int(group_size), _ptr(out))
+    if rc:
+        raise ValueError("amx_oracle_dequantize_f16s: bad shape")
+    return out
+
+
+def gemm_f16s(codesA, scalesA, codesW, scalesW, group_size: int) -> np.ndarray:
+    codesA, scalesA = _c(codesA, np.uint8), _c(scalesA, np.uint16)
+    codesW, scalesW = _c(codesW, np.uint8), _c(scalesW, np.uint16)
+    M, K = codesA.shape[0], codesA.shape[1] * 2
+    N = codesW.shape[0]
+    assert codesW.shape[1] * 2 == K
+    C = np.zeros((M, N), np.float32)
+    rc = lib().amx_oracle_gemm_f16s(_ptr(codesA), _ptr(scalesA), _ptr(codesW), _ptr(scalesW), M, N, K, int(group_size),
+                                    _ptr(C))
+    if rc:
+        raise ValueError(f"amx_oracle_gemm_f16s failed (rc={rc})")
+    return C
+
+
+def quant_error_f16s(x_bf16_bits: np.ndarray, codes: np.ndarray, scales: np.ndarray, group_size: int) -> np.ndarray:
+    x, codes, scales = _c(x_bf16_bits, np.uint16), _c(codes, np.uint8), _c(scales, np.uint16)
+    rows, K = x.shape
+    out = np.zeros(4, np.float64)
+    rc = lib().amx_oracle_quant_error_f16s(_ptr(x), rows, K, K, _ptr(codes), _ptr(scales), int(group_size), _ptr(out))
+    if rc:
+        raise ValueError("amx_oracle_quant_error_f16s: bad shape")
+    return out

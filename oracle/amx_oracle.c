@@ -714,6 +714,166 @@ int amx_oracle_gemm_nv(const uint8_t *codesA, const uint8_t *scalesA, float tA,
     return 0;
 }
 
+/* ------------------------------------ FP16 shared scales (scale-encoding ablation) -- */
+
+/*
+ * The appendix's ablation of the shared-scale encoding compares the FP8 scale with
+ * a 16-bit floating-point one, for the symmetric FP4 format and for the asymmetric
+ * one, at group sizes 16 to 128.  Here: the quantizer of Sections 4.2-4.3 with
+ * every "nearest E5M2" replaced by "nearest IEEE binary16" (ties to even, subnormals
+ * kept, saturating at 65504; a quotient that rounds to zero gives a zero scale and
+ * zero magnitudes, as in the FP8 quantizer).  Element rounding, clamping and the
+ * sign bit are unchanged.
+ * Layout: codes as everywhere, scales uint16 [rows][K/gs][2] = binary16 bit
+ * patterns {positive side, negative side}; the symmetric format stores the one
+ * scale of max|x| / 6 in both.
+ */
+
+/* Value of a binary16 bit pattern (never an infinity or NaN from the quantizer). */
+double amx_oracle_f16_value(uint16_t bits)
+{
+    int e = (bits >> 10) & 31, m = bits & 1023;
+    double v;
+    if (e == 0)
+        v = ldexp((double)m, -24);            /* subnormal: m/1024 * 2^-14 */
+    else if (e == 31)
+        v = m ? NAN : INFINITY;
+    else
+        v = ldexp(1.0 + m / 1024.0, e - 15);
+    return (bits & 0x8000) ? -v : v;
+}
+
+/* binary16 pattern nearest to q >= 0; ties to even; saturate at 65504 (0x7BFF). */
+uint16_t amx_oracle_f16_encode(double q)
+{
+    if (!(q > 0.0))
+        return 0;
+    int ex;
+    (void)frexp(q, &ex);
+    int e = ex - 1;                           /* floor(log2 q) */
+    if (e < -14)
+        e = -14;                              /* subnormal spacing below 2^-14 */
+    double quantum = ldexp(1.0, e - 10);
+    double t = q / quantum;                   /* exact: power-of-two divisor */
+    double lo = floor(t), frac = t - lo, n = lo;
+    if (frac > 0.5 || (frac == 0.5 && fmod(lo, 2.0) == 1.0))
+        n = lo + 1.0;
+    if (n == 2048.0) {                        /* rounded up into the next binade */
+        n = 1024.0;
+        e += 1;
+    }
+    if (e > 15)
+        return 0x7BFF;
+    if (n < 1024.0)                           /* only possible with e == -14 */
+        return (uint16_t)n;
+    return (uint16_t)(((e + 15) << 10) | ((int)n - 1024));
+}
+
+/* asym = 1: one scale per sign (AMXFP4 with FP16 scales); 0: one per group. */
+int amx_oracle_quantize_f16s(const uint16_t *x, int64_t rows, int64_t K, int64_t ld, int gs, int asym,
+                             uint8_t *codes, uint16_t *scales)
+{
+    if (gs <= 0 || K % gs != 0 || (K & 1))
+        return -1;
+    int64_t G = K / gs;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t g = 0; g < G; ++g) {
+            const uint16_t *xg = x + r * ld + g * gs;
+            double pmax = 0.0, nmax = 0.0;
+            for (int i = 0; i < gs; ++i) {
+                double a = fabs(bf16_to_double(xg[i]));
+                if (xg[i] >> 15) { if (a > nmax) nmax = a; }
+                else             { if (a > pmax) pmax = a; }
+            }
+            if (!asym)
+                pmax = nmax = (pmax > nmax ? pmax : nmax);
+            uint16_t sb[2] = {amx_oracle_f16_encode(pmax / 6.0), amx_oracle_f16_encode(nmax / 6.0)};
+            for (int i = 0; i < gs; ++i) {
+                int sign = xg[i] >> 15;
+                double sv = amx_oracle_f16_value(sb[sign]);
+                int mag = sv > 0.0 ? amx_oracle_e2m1_encode(fabs(bf16_to_double(xg[i])) / sv) : 0;
+                uint8_t c = (uint8_t)((sign << 3) | mag);
+                int64_t k = g * gs + i;
+                uint8_t *byte = codes + r * (K / 2) + k / 2;
+                if (k & 1) *byte = (uint8_t)((*byte & 0x0F) | (c << 4));
+                else       *byte = (uint8_t)((*byte & 0xF0) | c);
+            }
+            scales[(r * G + g) * 2 + 0] = sb[0];
+            scales[(r * G + g) * 2 + 1] = sb[1];
+        }
+    return 0;
+}
+
+/* Eq. 1 with binary16 scales. */
+int amx_oracle_dequantize_f16s(const uint8_t *codes, const uint16_t *scales,
+                               int64_t rows, int64_t K, int gs, double *out)
+{
+    if (gs <= 0 || K % gs != 0 || (K & 1))
+        return -1;
+    int64_t G = K / gs;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t k = 0; k < K; ++k) {
+            uint8_t byte = codes[r * (K / 2) + k / 2];
+            int c = (k & 1) ? (byte >> 4) : (byte & 15);
+            double s = amx_oracle_f16_value(scales[(r * G + k / gs) * 2 + ((c >> 3) & 1)]);
+            out[r * K + k] = amx_oracle_e2m1_value(c) * s;
+        }
+    return 0;
+}
+
+/* C[m][n] = sum_k Ahat[m][k] * What[n][k]: fp64 sums in index order, rounded once to fp32. */
+int amx_oracle_gemm_f16s(const uint8_t *codesA, const uint16_t *scalesA,
+                         const uint8_t *codesW, const uint16_t *scalesW,
+                         int64_t M, int64_t N, int64_t K, int gs, float *C)
+{
+    if (gs <= 0 || K % gs != 0 || (K & 1))
+        return -1;
+    double *a = (double *)malloc(sizeof(double) * (size_t)M * (size_t)K);
+    double *w = (double *)malloc(sizeof(double) * (size_t)N * (size_t)K);
+    if (!a || !w) {
+        free(a); free(w);
+        return -2;
+    }
+    amx_oracle_dequantize_f16s(codesA, scalesA, M, K, gs, a);
+    amx_oracle_dequantize_f16s(codesW, scalesW, N, K, gs, w);
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int64_t k = 0; k < K; ++k) acc += a[m * K + k] * w[n * K + k];
+            C[m * N + n] = (float)acc;
+        }
+    free(a); free(w);
+    return 0;
+}
+
+/* amx_oracle_quant_error with binary16 scales (same four sums). */
+int amx_oracle_quant_error_f16s(const uint16_t *x, int64_t rows, int64_t K, int64_t ld,
+                                const uint8_t *codes, const uint16_t *scales, int gs, double *out)
+{
+    if (gs <= 0 || K % gs != 0 || (K & 1))
+        return -1;
+    int64_t G = K / gs;
+    double x2 = 0.0, e2 = 0.0, c2 = 0.0, cnt = 0.0;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t k = 0; k < K; ++k) {
+            double v = bf16_to_double(x[r * ld + k]);
+            uint8_t byte = codes[r * (K / 2) + k / 2];
+            int c = (k & 1) ? (byte >> 4) : (byte & 15);
+            double s = amx_oracle_f16_value(scales[(r * G + k / gs) * 2 + ((c >> 3) & 1)]);
+            double e = v - amx_oracle_e2m1_value(c) * s;
+            x2 += v * v;
+            e2 += e * e;
+            if (fabs(v) > 6.0 * s) {
+                c2 += e * e;
+                cnt += 1.0;
+            }
+        }
+    out[0] = x2; out[1] = e2; out[2] = c2; out[3] = cnt;
+    return 0;
+}
+
 int amx_oracle_num_threads(void)
 {
     int n = 1;
