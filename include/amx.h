@@ -374,6 +374,34 @@ int amx_gemm_nvfp4(const void* a_prepared, const void* w_prepared, int64_t M, in
                    int64_t ld_c, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * FP4 with binary16 shared scales - the "FP16" row of the paper's ablation of the shared-scale encoding (appendix
+ * "Ablation Study on Shared-Scale Bit-Encoding"): the quantizer of Sections 4.2-4.3 with "nearest E5M2" replaced by
+ * "nearest binary16" (ties to even, subnormals kept, saturating at 65504; a quotient that rounds to zero gives a
+ * zero scale and zero magnitudes).  flags: AMX_F16S_ASYMMETRIC = one scale per sign (AMXFP4 with FP16 scales),
+ * 0 = one scale per group from max|x| / 6, stored in both slots.
+ *   x        device, bf16 [rows, ld_x], 16-byte aligned, ld_x % 8 == 0
+ *   codes    device out/in, [rows, K/2], 4-byte aligned (layout as amx_quantize)
+ *   scales   device out/in, uint16 [rows, K/group_size, 2]: binary16 bit patterns {positive side, negative side},
+ *            4-byte aligned
+ *   group_size 16, 32, 64 or 128; K % group_size == 0
+ * amx_dequantize_f16s writes fp32 [rows, ld_out] (a decoded value has up to 13 significant bits: exact in fp32, not
+ * in bf16; out 16-byte aligned, ld_out % 4 == 0).  amx_gemm_f16s: C[m, n] = sum_k Ahat[m, k] What[n, k] on the
+ * CUDA cores, fp32 products (exact) and fp32 accumulation - no tensor-core type holds 13-bit operands exactly;
+ * C fp32 [M, ld_c].  amx_quant_error_f16s: amx_quant_error (below) for this layout.
+ * One launch each (the error report two) on `stream`; nothing is synchronised; on error nothing was launched.
+ */
+#define AMX_F16S_ASYMMETRIC 0x1u
+int amx_quantize_f16s(const void* x, int64_t rows, int64_t K, int64_t ld_x, int group_size, uint32_t flags,
+                      uint8_t* codes, uint16_t* scales, void* stream);
+int amx_dequantize_f16s(const uint8_t* codes, const uint16_t* scales, int64_t rows, int64_t K, int group_size,
+                        float* out, int64_t ld_out, void* stream);
+int amx_gemm_f16s(const uint8_t* a_codes, const uint16_t* a_scales, const uint8_t* w_codes, const uint16_t* w_scales,
+                  int64_t M, int64_t N, int64_t K, int group_size, float* C, int64_t ld_c, void* stream);
+int amx_quant_error_f16s(const void* x, int64_t rows, int64_t K, int64_t ld_x, const uint8_t* codes,
+                         const uint16_t* scales, int group_size, double* out, void* workspace,
+                         size_t workspace_bytes, void* stream);
+
+/*
  * amx_quant_error - squared error of a quantized tensor against its bf16 source, split as the appendix
  * "Determining PoT Shared Scale: Floor vs. Round" splits the error of a shared scale: elements whose magnitude
  * exceeds the largest value their side represents (|x| > 6 * scale of the element's side) make up the

@@ -39,6 +39,7 @@ SYMBOLS = (
     "amx_attention_map", "amx_gemm_flushed_scales", "amx_prepared_flushed_scales", "amx_selftest_wait_timeout",
     "amx_quant_gemm_static_status",
     "amx_quantize_nvfp4", "amx_nvfp4_prepared_bytes", "amx_dequantize_nvfp4", "amx_gemm_nvfp4",
+    "amx_quantize_f16s", "amx_dequantize_f16s", "amx_gemm_f16s", "amx_quant_error_f16s",
 )
 
 
@@ -75,6 +76,10 @@ def lib() -> ctypes.CDLL:
         L.amx_nvfp4_prepared_bytes.restype = sz
         L.amx_dequantize_nvfp4.argtypes = [p, p, p, i64, i64, u32, p, i64, p]
         L.amx_gemm_nvfp4.argtypes = [p, p, i64, i64, i64, p, i64, p, sz, p]
+        L.amx_quantize_f16s.argtypes = [p, i64, i64, i64, i, u32, p, p, p]
+        L.amx_dequantize_f16s.argtypes = [p, p, i64, i64, i, p, i64, p]
+        L.amx_gemm_f16s.argtypes = [p, p, p, p, i64, i64, i64, i, p, i64, p]
+        L.amx_quant_error_f16s.argtypes = [p, i64, i64, i64, p, p, i, p, p, sz, p]
         L.amx_quant_gemm_static.argtypes = [p, i64, p, p, i64, i64, i64, i, u32, p, i64, p]
         L.amx_quant_gemm_static_capacity.argtypes = []
         L.amx_quant_gemm_static_capacity.restype = sz
@@ -361,6 +366,57 @@ def gemm_nvfp4(a_prepared: torch.Tensor, w_prepared: torch.Tensor, M: int, N: in
         workspace = _ws(256, a_prepared.device)
     _check(lib().amx_gemm_nvfp4(a_prepared.data_ptr(), w_prepared.data_ptr(), M, N, K, out.data_ptr(), N, workspace.data_ptr(),
                                 workspace.numel(), _stream()), "amx_gemm_nvfp4")
+    return out
+
+
+F16S_ASYMMETRIC = 0x1
+
+
+def quantize_f16s(x: torch.Tensor, group_size: int = 32, asym: bool = True):
+    """bf16 [rows, K] -> (codes u8 [rows, K/2], binary16 scale bit patterns int16 [rows, K/group_size, 2])."""
+    _dev(x, torch.bfloat16, "x")
+    assert x.dim() == 2 and x.stride(1) == 1
+    rows, K = x.shape
+    codes = torch.empty((rows, K // 2), dtype=torch.uint8, device=x.device)
+    scales = torch.empty((rows, K // group_size, 2), dtype=torch.int16, device=x.device)
+    _check(lib().amx_quantize_f16s(x.data_ptr(), rows, K, x.stride(0), group_size, F16S_ASYMMETRIC if asym else 0,
+                                   codes.data_ptr(), scales.data_ptr(), _stream()), "amx_quantize_f16s")
+    return codes, scales
+
+
+def dequantize_f16s(codes: torch.Tensor, scales: torch.Tensor, group_size: int = 32) -> torch.Tensor:
+    _dev(codes, torch.uint8, "codes"), _dev(scales, torch.int16, "scales")
+    assert codes.is_contiguous() and scales.is_contiguous()
+    rows, K = codes.shape[0], codes.shape[1] * 2
+    out = torch.empty((rows, K), dtype=torch.float32, device=codes.device)
+    _check(lib().amx_dequantize_f16s(codes.data_ptr(), scales.data_ptr(), rows, K, group_size, out.data_ptr(), K, _stream()),
+           "amx_dequantize_f16s")
+    return out
+
+
+def gemm_f16s(a_codes, a_scales, w_codes, w_scales, group_size: int = 32) -> torch.Tensor:
+    for t, d, n in ((a_codes, torch.uint8, "a_codes"), (a_scales, torch.int16, "a_scales"), (w_codes, torch.uint8, "w_codes"),
+                    (w_scales, torch.int16, "w_scales")):
+        _dev(t, d, n)
+        assert t.is_contiguous()
+    M, K = a_codes.shape[0], a_codes.shape[1] * 2
+    N = w_codes.shape[0]
+    assert w_codes.shape[1] * 2 == K
+    out = torch.empty((M, N), dtype=torch.float32, device=a_codes.device)
+    _check(lib().amx_gemm_f16s(a_codes.data_ptr(), a_scales.data_ptr(), w_codes.data_ptr(), w_scales.data_ptr(), M, N, K,
+                               group_size, out.data_ptr(), N, _stream()), "amx_gemm_f16s")
+    return out
+
+
+def quant_error_f16s(x: torch.Tensor, codes: torch.Tensor, scales: torch.Tensor, group_size: int = 32) -> torch.Tensor:
+    """quant_error for operands with binary16 scales."""
+    _dev(x, torch.bfloat16, "x"), _dev(codes, torch.uint8, "codes"), _dev(scales, torch.int16, "scales")
+    assert x.dim() == 2 and x.stride(1) == 1 and codes.is_contiguous() and scales.is_contiguous()
+    rows, K = x.shape
+    out = torch.empty(4, dtype=torch.float64, device=x.device)
+    ws = torch.empty(lib().amx_quant_error_workspace_bytes(), dtype=torch.uint8, device=x.device)
+    _check(lib().amx_quant_error_f16s(x.data_ptr(), rows, K, x.stride(0), codes.data_ptr(), scales.data_ptr(), group_size,
+                                      out.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "amx_quant_error_f16s")
     return out
 
 

@@ -9,6 +9,11 @@ int gemm_simt(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_
               const uint8_t* w_scales, int64_t M, int64_t N, int64_t K, int gs, float* C,
               int64_t ld_c, cudaStream_t st);
 
+// The same kernel on operands with binary16 shared scales ([rows, K/gs, 2] uint16).
+int gemm_simt_f16s(const uint8_t* a_codes, const uint16_t* a_scales, const uint8_t* w_codes,
+                   const uint16_t* w_scales, int64_t M, int64_t N, int64_t K, int gs, float* C,
+                   int64_t ld_c, cudaStream_t st);
+
 // Tensor-core (tcgen05) kernel: shapes it accepts, scratch it needs, launcher.
 bool gemm_tc_supported(int64_t M, int64_t N, int64_t K, int gs);
 size_t gemm_tc_workspace_bytes(int64_t M, int64_t N, int64_t K);

@@ -2,25 +2,34 @@
 // C[m,n] = sum_k Ahat[m,k] * What[n,k]: every factor is decoded with the shared scale its own
 // sign selects (arXiv 2411.09909, Section 4.3), products and sums in fp32.
 // This is the general-shape path and the on-device cross-check for the tensor-core kernel.
+// The same kernel takes binary16 shared scales (ScaleT = uint16_t, the scale-encoding ablation of the appendix):
+// an E2M1 magnitude times a binary16 scale has at most 13 significant bits, exact in fp32.
+#include <cuda_fp16.h>
+
 #include "amx_common.cuh"
+#include "gemm.cuh"
 
 namespace amx {
 namespace {
 
 constexpr int BM = 64, BN = 64, BK = 32, PAD = 4;
 
+__device__ __forceinline__ float scale_value(uint8_t b) { return e5m2_to_float(b); }
+__device__ __forceinline__ float scale_value(uint16_t h) { return __half2float(__ushort_as_half(h)); }
+
 // Decodes 8 codes of one row (one 32-bit word) into column `r` of a [BK][B + PAD] tile.
+template <typename ScaleT>
 __device__ __forceinline__ void decode_word(const uint8_t* __restrict__ codes,
-                                            const uint8_t* __restrict__ scales, int64_t row,
+                                            const ScaleT* __restrict__ scales, int64_t row,
                                             int64_t rows, int64_t K, int gs, int64_t k,
                                             float (*tile)[BM + PAD], int r, int kk) {
     uint32_t nib = 0;
     float sp = 0.f, sn = 0.f;
     if (row < rows && k < K) {
         nib = *reinterpret_cast<const uint32_t*>(codes + row * (K / 2) + k / 2);
-        const uint8_t* sc = scales + (row * (K / gs) + k / gs) * 2;
-        sp = e5m2_to_float(sc[0]);
-        sn = e5m2_to_float(sc[1]);
+        const ScaleT* sc = scales + (row * (K / gs) + k / gs) * 2;
+        sp = scale_value(sc[0]);
+        sn = scale_value(sc[1]);
     }
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -30,9 +39,10 @@ __device__ __forceinline__ void decode_word(const uint8_t* __restrict__ codes,
     }
 }
 
+template <typename ScaleT>
 __global__ void __launch_bounds__(256)
-gemm_simt_kernel(const uint8_t* __restrict__ a_codes, const uint8_t* __restrict__ a_scales,
-                 const uint8_t* __restrict__ w_codes, const uint8_t* __restrict__ w_scales,
+gemm_simt_kernel(const uint8_t* __restrict__ a_codes, const ScaleT* __restrict__ a_scales,
+                 const uint8_t* __restrict__ w_codes, const ScaleT* __restrict__ w_scales,
                  int64_t M, int64_t N, int64_t K, int gs, float* __restrict__ C, int64_t ld_c) {
     __shared__ __align__(16) float As[BK][BM + PAD];
     __shared__ __align__(16) float Ws[BK][BN + PAD];
@@ -75,7 +85,16 @@ int gemm_simt(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* w_
               int64_t ld_c, cudaStream_t st) {
     dim3 grid((unsigned)((N + BN - 1) / BN), (unsigned)((M + BM - 1) / BM));
     if (grid.y > 65535) return AMX_ERR_SHAPE;
-    gemm_simt_kernel<<<grid, 256, 0, st>>>(a_codes, a_scales, w_codes, w_scales, M, N, K, gs, C, ld_c);
+    gemm_simt_kernel<uint8_t><<<grid, 256, 0, st>>>(a_codes, a_scales, w_codes, w_scales, M, N, K, gs, C, ld_c);
+    return launch_status();
+}
+
+int gemm_simt_f16s(const uint8_t* a_codes, const uint16_t* a_scales, const uint8_t* w_codes,
+                   const uint16_t* w_scales, int64_t M, int64_t N, int64_t K, int gs, float* C,
+                   int64_t ld_c, cudaStream_t st) {
+    dim3 grid((unsigned)((N + BN - 1) / BN), (unsigned)((M + BM - 1) / BM));
+    if (grid.y > 65535) return AMX_ERR_SHAPE;
+    gemm_simt_kernel<uint16_t><<<grid, 256, 0, st>>>(a_codes, a_scales, w_codes, w_scales, M, N, K, gs, C, ld_c);
     return launch_status();
 }
 

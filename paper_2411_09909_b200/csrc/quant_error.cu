@@ -10,6 +10,10 @@
 // non-negative), everything above a chunk in fp64 - fp64 arithmetic per element would bound the kernel (the
 // conversions alone cost more than the memory traffic).  The clamped count is an integer.  The summation order is fixed (grid-stride per thread, shuffles in a warp, warps in
 // order, then one block over the per-block partial sums), so the result is the same bits on every run.
+// F16S instantiation: binary16 shared scales ([rows, K/gs, 2] uint16); xhat then has up to 13 significant bits and
+// x - xhat is still exact in fp32.
+#include <cuda_fp16.h>
+
 #include "amx_common.cuh"
 
 namespace amx {
@@ -65,6 +69,7 @@ __device__ __forceinline__ Sums block_sum(Sums s, double (*sh)[4]) {
     return t;
 }
 
+template <bool F16S>
 __global__ void __launch_bounds__(kThreads) quant_error_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K,
                                                                int64_t ld_x, const uint8_t* __restrict__ codes,
                                                                const uint8_t* __restrict__ scales, int gs_log2,
@@ -76,14 +81,20 @@ __global__ void __launch_bounds__(kThreads) quant_error_kernel(const uint16_t* _
     for (int64_t row = blockIdx.y; row < rows; row += gridDim.y) {
         const uint16_t* xr = x + row * ld_x;
         const uint8_t* cr = codes + row * (K / 2);
-        const uint8_t* sr = scales + row * groups * 2;
+        const uint8_t* sr = scales + row * groups * (F16S ? 4 : 2);
         for (int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x; c < per_row; c += (int64_t)gridDim.x * kThreads) {
             const int64_t k = c * 16;
             const uint4* xp = reinterpret_cast<const uint4*>(xr + k);
             const uint4 xw[2] = {__ldg(xp), __ldg(xp + 1)};
             const uint2 cw = __ldg(reinterpret_cast<const uint2*>(cr + k / 2));
-            const uint32_t sc = __ldg(reinterpret_cast<const unsigned short*>(sr + (k >> gs_log2) * 2));
-            add16(s, xw, cw, e5m2_to_float(sc & 0xFFu), e5m2_to_float(sc >> 8));
+            if (F16S) {
+                const uint32_t sc = __ldg(reinterpret_cast<const uint32_t*>(sr + (k >> gs_log2) * 4));
+                add16(s, xw, cw, __half2float(__ushort_as_half((unsigned short)(sc & 0xFFFFu))),
+                      __half2float(__ushort_as_half((unsigned short)(sc >> 16))));
+            } else {
+                const uint32_t sc = __ldg(reinterpret_cast<const unsigned short*>(sr + (k >> gs_log2) * 2));
+                add16(s, xw, cw, e5m2_to_float(sc & 0xFFu), e5m2_to_float(sc >> 8));
+            }
         }
     }
     const Sums t = block_sum(s, sh);
@@ -111,14 +122,14 @@ using namespace amx;
 
 extern "C" size_t amx_quant_error_workspace_bytes(void) { return (size_t)kMaxBlocks * 4 * sizeof(double); }
 
-extern "C" int amx_quant_error(const void* x, int64_t rows, int64_t K, int64_t ld_x, const uint8_t* codes,
-                               const uint8_t* scales, int group_size, double* out, void* workspace,
-                               size_t workspace_bytes, void* stream) {
+namespace {
+int quant_error(const void* x, int64_t rows, int64_t K, int64_t ld_x, const uint8_t* codes, const void* scales,
+                bool f16s, int group_size, double* out, void* workspace, size_t workspace_bytes, void* stream) {
     if (!fixed_group_size(group_size) || rows < 0 || K <= 0 || K % group_size || ld_x < K) return AMX_ERR_SHAPE;
     if (!out) return AMX_ERR_NULL;
     if (rows > 0 && (!x || !codes || !scales)) return AMX_ERR_NULL;
     if (!workspace || workspace_bytes < amx_quant_error_workspace_bytes()) return AMX_ERR_WORKSPACE;
-    if (!aligned(x, 16) || ld_x % 8 || !aligned(codes, 8) || !aligned(scales, 2) || !aligned(out, 8) ||
+    if (!aligned(x, 16) || ld_x % 8 || !aligned(codes, 8) || !aligned(scales, f16s ? 4 : 2) || !aligned(out, 8) ||
         !aligned(workspace, 8))
         return AMX_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -128,9 +139,28 @@ extern "C" int amx_quant_error(const void* x, int64_t rows, int64_t K, int64_t l
     int64_t by = rows < 1 ? 1 : rows > kMaxBlocks / bx ? kMaxBlocks / bx : rows;
     const int64_t blocks = bx * by;
     double* partial = static_cast<double*>(workspace);
-    quant_error_kernel<<<dim3((unsigned)bx, (unsigned)by), kThreads, 0, st>>>(static_cast<const uint16_t*>(x), rows, K, ld_x,
-                                                                             codes, scales, group_size == 16 ? 4 : group_size == 32 ? 5 : group_size == 64 ? 6 : 7, partial);
+    const int gs_log2 = group_size == 16 ? 4 : group_size == 32 ? 5 : group_size == 64 ? 6 : 7;
+    const dim3 grid((unsigned)bx, (unsigned)by);
+    if (f16s)
+        quant_error_kernel<true><<<grid, kThreads, 0, st>>>(static_cast<const uint16_t*>(x), rows, K, ld_x, codes,
+                                                            static_cast<const uint8_t*>(scales), gs_log2, partial);
+    else
+        quant_error_kernel<false><<<grid, kThreads, 0, st>>>(static_cast<const uint16_t*>(x), rows, K, ld_x, codes,
+                                                             static_cast<const uint8_t*>(scales), gs_log2, partial);
     if (launch_status() != AMX_OK) return AMX_ERR_CUDA;
     quant_error_final_kernel<<<1, kThreads, 0, st>>>(partial, (int)blocks, out);
     return launch_status();
+}
+}  // namespace
+
+extern "C" int amx_quant_error(const void* x, int64_t rows, int64_t K, int64_t ld_x, const uint8_t* codes,
+                               const uint8_t* scales, int group_size, double* out, void* workspace,
+                               size_t workspace_bytes, void* stream) {
+    return quant_error(x, rows, K, ld_x, codes, scales, false, group_size, out, workspace, workspace_bytes, stream);
+}
+
+extern "C" int amx_quant_error_f16s(const void* x, int64_t rows, int64_t K, int64_t ld_x, const uint8_t* codes,
+                                    const uint16_t* scales, int group_size, double* out, void* workspace,
+                                    size_t workspace_bytes, void* stream) {
+    return quant_error(x, rows, K, ld_x, codes, scales, true, group_size, out, workspace, workspace_bytes, stream);
 }

@@ -1,6 +1,7 @@
 """Synthetic quantization-error report: relative squared error of AMXFP4 and of the symmetric comparison formats
 across group sizes, split into the max-clamping and the rounding part (arXiv 2411.09909, appendix "Determining PoT
-Shared Scale: Floor vs. Round" and the shared-scale ablation).  Runs on the GPU through amx_quantize(_fmt) and
+Shared Scale: Floor vs. Round" and the shared-scale ablation, whose FP16-scale rows come from amx_quantize_f16s
+and amx_quant_error_f16s).  Runs on the GPU through amx_quantize(_fmt) and
 amx_quant_error on seeded synthetic tensors shaped like the paper's workloads; the paper's own numbers come from
 LLM checkpoints and are not reproduced here.
 
@@ -17,7 +18,8 @@ from . import amx, build, inputs
 
 FORMATS = (("AMXFP4 (two FP8 scales)", amx.FMT_AMXFP4), ("symmetric, FP8 scale", amx.FMT_SYM_FP8),
            ("MXFP4 (power-of-two floor)", amx.FMT_MXFP4), ("per-sign power-of-two floor", amx.FMT_AMXFP4_POT),
-           ("power-of-two round", amx.FMT_MXFP4_POT_ROUND), ("per-sign power-of-two round", amx.FMT_AMXFP4_POT_ROUND))
+           ("power-of-two round", amx.FMT_MXFP4_POT_ROUND), ("per-sign power-of-two round", amx.FMT_AMXFP4_POT_ROUND),
+           ("symmetric, FP16 scale", "f16s"), ("two FP16 scales", "f16s-asym"))
 TENSORS = (("activation, channel outliers (config 2, 4096 wide)", 2, 0, "a"),
            ("activation, SiLU-skewed (config 3, 14336 wide)", 3, 3, "a"),
            ("weight N(0, 0.02) (config 2, 4096 -> 4096)", 2, 1, "w"))
@@ -37,8 +39,12 @@ def report(rows: int = 2048):
         lines.append("|---|---|---|---|---|")
         for name, fmt in FORMATS:
             for gs in (128, 64, 32, 16):
-                codes, scales = amx.quantize(x, gs, fmt)
-                e = amx.quant_error(x, codes, scales, gs).cpu().numpy()
+                if isinstance(fmt, str):
+                    codes, scales = amx.quantize_f16s(x, gs, fmt == "f16s-asym")
+                    e = amx.quant_error_f16s(x, codes, scales, gs).cpu().numpy()
+                else:
+                    codes, scales = amx.quantize(x, gs, fmt)
+                    e = amx.quant_error(x, codes, scales, gs).cpu().numpy()
                 lines.append(f"| {name} | {gs} | {e[1] / e[0]:.3e} | {100 * e[2] / max(e[1], 1e-300):.1f} % | "
                              f"{100 * e[3] / x.numel():.2f} % |")
     return "\n".join(lines)
