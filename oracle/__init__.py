@@ -65,7 +65,7 @@ def lib() -> ctypes.CDLL:
         L.amx_oracle_f16_value.argtypes = [ctypes.c_uint16]
         L.amx_oracle_f16_encode.restype = ctypes.c_uint16
         L.amx_oracle_f16_encode.argtypes = [dbl]
-        L.amx_oracle_quantize_f16s.argtypes = [p, i64, i64, i64, ctypes.c_int, ctypes.c_int, p, p]
+        L.amx_oracle_quantize_f16s.argtypes = [p, i64, i64, i64, ctypes.c_int, ctypes.c_int, ctypes.c_int, p, p]
         L.amx_oracle_dequantize_f16s.argtypes = [p, p, i64, i64, ctypes.c_int, p]
         L.amx_oracle_gemm_f16s.argtypes = [p, p, p, p, i64, i64, i64, ctypes.c_int, p]
         L.amx_oracle_quant_error_f16s.argtypes = [p, i64, i64, i64, p, p, ctypes.c_int, p]
@@ -284,14 +284,15 @@ def f16_encode(q: float) -> int:
     return int(lib().amx_oracle_f16_encode(float(q)))
 
 
-def quantize_f16s(x_bf16_bits: np.ndarray, group_size: int, asym: bool):
+def quantize_f16s(x_bf16_bits: np.ndarray, group_size: int, asym: bool, e4m3: bool = False):
     """bf16 bit patterns [rows, K] -> (codes u8 [rows, K/2], binary16 scales u16 [rows, K/gs, 2]).
-    asym True: one scale per sign (positive side, negative side); False: the group's one scale in both."""
+    asym True: one scale per sign (positive side, negative side); False: the group's one scale in both.
+    e4m3 True: scales rounded to FP8 E4M3 ("1-4-3") and stored as the binary16 pattern of that value."""
     x = _c(x_bf16_bits, np.uint16)
     rows, K = x.shape
     codes = np.zeros((rows, K // 2), np.uint8)
     scales = np.zeros((rows, K // group_size, 2), np.uint16)
-    rc = lib().amx_oracle_quantize_f16s(_ptr(x), rows, K, K, int(group_size), int(asym), _ptr(codes), _ptr(scales))
+    rc = lib().amx_oracle_quantize_f16s(_ptr(x), rows, K, K, int(group_size), int(asym), int(e4m3), _ptr(codes), _ptr(scales))
     if rc:
         raise ValueError("amx_oracle_quantize_f16s: K must be a multiple of the group size")
     return codes, scales

@@ -769,8 +769,13 @@ uint16_t amx_oracle_f16_encode(double q)
     return (uint16_t)(((e + 15) << 10) | ((int)n - 1024));
 }
 
-/* asym = 1: one scale per sign (AMXFP4 with FP16 scales); 0: one per group. */
-int amx_oracle_quantize_f16s(const uint16_t *x, int64_t rows, int64_t K, int64_t ld, int gs, int asym,
+/*
+ * asym = 1: one scale per sign (AMXFP4 with FP16 scales); 0: one per group.
+ * e4m3 = 1: the ablation's other FP8 scale, "1-4-3": the scale is the nearest FP8 E4M3 value (ties to even,
+ * subnormals kept, saturating at 448) instead of the nearest binary16; every E4M3 value is a binary16 value, so
+ * it is stored as that value's binary16 pattern in the same layout and everything downstream is unchanged.
+ */
+int amx_oracle_quantize_f16s(const uint16_t *x, int64_t rows, int64_t K, int64_t ld, int gs, int asym, int e4m3,
                              uint8_t *codes, uint16_t *scales)
 {
     if (gs <= 0 || K % gs != 0 || (K & 1))
@@ -788,7 +793,14 @@ int amx_oracle_quantize_f16s(const uint16_t *x, int64_t rows, int64_t K, int64_t
             }
             if (!asym)
                 pmax = nmax = (pmax > nmax ? pmax : nmax);
-            uint16_t sb[2] = {amx_oracle_f16_encode(pmax / 6.0), amx_oracle_f16_encode(nmax / 6.0)};
+            uint16_t sb[2];
+            if (e4m3) {
+                sb[0] = amx_oracle_f16_encode(amx_oracle_e4m3_value(amx_oracle_e4m3_encode(pmax / 6.0)));
+                sb[1] = amx_oracle_f16_encode(amx_oracle_e4m3_value(amx_oracle_e4m3_encode(nmax / 6.0)));
+            } else {
+                sb[0] = amx_oracle_f16_encode(pmax / 6.0);
+                sb[1] = amx_oracle_f16_encode(nmax / 6.0);
+            }
             for (int i = 0; i < gs; ++i) {
                 int sign = xg[i] >> 15;
                 double sv = amx_oracle_f16_value(sb[sign]);

@@ -159,6 +159,52 @@ def test_invariants(asym):
                     assert abs(hat[i] - ext) <= abs(ext) * 2.0 ** -11
 
 
+def nearest_e4m3_as_f16(q: Fraction) -> int:
+    """binary16 pattern of the FP8 E4M3 value nearest to q >= 0 (exact comparison over all 127 finite values; ties to
+    the even E4M3 code; saturating at 448), with ml_dtypes as the table of E4M3 values."""
+    import ml_dtypes
+    vals = np.arange(0x7F, dtype=np.uint8).view(ml_dtypes.float8_e4m3fn).astype(np.float64)
+    best = None
+    for code, v in enumerate(vals):
+        d = abs(Fraction(float(v)) - q)
+        if best is None or d < best[0] or (d == best[0] and code % 2 == 0):
+            best = (d, code)
+    return int(np.float16(vals[best[1]]).view(np.uint16))
+
+
+@pytest.mark.parametrize("asym", [False, True])
+def test_e4m3_scale_option(asym):
+    rng = np.random.default_rng(15 + asym)
+    gs, rows, K = 32, 6, 128
+    x = rng.standard_normal((rows, K)) * 2.0 ** rng.integers(-8, 9, (rows, 1))
+    x[0, :gs] *= 2.0 ** -9                                           # E4M3-subnormal scales
+    x[1, 0] = 1.0e5                                                  # saturates at 448: everything above 2688 clamps
+    x[2, gs:2 * gs] = 0.0
+    b = bits(x)
+    v = values(b)
+    codes, scales = oracle.quantize_f16s(b, gs, asym, e4m3=True)
+    c4 = oracle.unpack_codes(codes)
+    for r in range(rows):
+        for g in range(K // gs):
+            seg, sb = v[r, g * gs:(g + 1) * gs], b[r, g * gs:(g + 1) * gs]
+            neg = (sb >> 15).astype(bool)
+            pmax = max([Fraction(float(a)) for a, n in zip(seg, neg) if not n], default=Fraction(0))
+            nmax = max([Fraction(float(-a)) for a, n in zip(seg, neg) if n], default=Fraction(0))
+            if not asym:
+                pmax = nmax = max(pmax, nmax)
+            want = (nearest_e4m3_as_f16(pmax / 6), nearest_e4m3_as_f16(nmax / 6))
+            assert tuple(int(s) for s in scales[r, g]) == want
+            sv = [Fraction(float(np.uint16(w).view(np.float16))) for w in want]
+            for i in range(gs):
+                assert c4[r, g * gs + i] == (int(neg[i]) << 3 | nearest_code(Fraction(float(seg[i])), sv[int(neg[i])]))
+    assert scales.view(np.float16).astype(np.float64).max() == 448.0
+    # where the binary16 scale happens to be an E4M3 value the two options agree
+    c16, s16 = oracle.quantize_f16s(b, gs, asym)
+    same = (s16 == scales).all(axis=2)
+    k = np.repeat(same, gs, axis=1)
+    assert np.array_equal(oracle.unpack_codes(c16)[k], c4[k])
+
+
 def test_gemm_and_error_sums():
     rng = np.random.default_rng(14)
     gs = 16
