@@ -378,7 +378,9 @@ int amx_gemm_nvfp4(const void* a_prepared, const void* w_prepared, int64_t M, in
  * "Ablation Study on Shared-Scale Bit-Encoding"): the quantizer of Sections 4.2-4.3 with "nearest E5M2" replaced by
  * "nearest binary16" (ties to even, subnormals kept, saturating at 65504; a quotient that rounds to zero gives a
  * zero scale and zero magnitudes).  flags: AMX_F16S_ASYMMETRIC = one scale per sign (AMXFP4 with FP16 scales),
- * 0 = one scale per group from max|x| / 6, stored in both slots.
+ * 0 = one scale per group from max|x| / 6, stored in both slots; AMX_F16S_SCALE_E4M3 = the same table's "FP8
+ * 1-4-3" row: the scale is the nearest FP8 E4M3 value (ties to even, subnormals kept, saturating at 448), stored as
+ * the binary16 pattern of that value, so that dequantize, product and error report take it unchanged.
  *   x        device, bf16 [rows, ld_x], 16-byte aligned, ld_x % 8 == 0
  *   codes    device out/in, [rows, K/2], 4-byte aligned (layout as amx_quantize)
  *   scales   device out/in, uint16 [rows, K/group_size, 2]: binary16 bit patterns {positive side, negative side},
@@ -391,6 +393,7 @@ int amx_gemm_nvfp4(const void* a_prepared, const void* w_prepared, int64_t M, in
  * One launch each (the error report two) on `stream`; nothing is synchronised; on error nothing was launched.
  */
 #define AMX_F16S_ASYMMETRIC 0x1u
+#define AMX_F16S_SCALE_E4M3 0x2u
 int amx_quantize_f16s(const void* x, int64_t rows, int64_t K, int64_t ld_x, int group_size, uint32_t flags,
                       uint8_t* codes, uint16_t* scales, void* stream);
 int amx_dequantize_f16s(const uint8_t* codes, const uint16_t* scales, int64_t rows, int64_t K, int group_size,

@@ -370,17 +370,20 @@ def gemm_nvfp4(a_prepared: torch.Tensor, w_prepared: torch.Tensor, M: int, N: in
 
 
 F16S_ASYMMETRIC = 0x1
+F16S_SCALE_E4M3 = 0x2
 
 
-def quantize_f16s(x: torch.Tensor, group_size: int = 32, asym: bool = True):
-    """bf16 [rows, K] -> (codes u8 [rows, K/2], binary16 scale bit patterns int16 [rows, K/group_size, 2])."""
+def quantize_f16s(x: torch.Tensor, group_size: int = 32, asym: bool = True, e4m3: bool = False):
+    """bf16 [rows, K] -> (codes u8 [rows, K/2], binary16 scale bit patterns int16 [rows, K/group_size, 2]);
+    e4m3: scales rounded to FP8 E4M3 (stored as the binary16 pattern of that value)."""
     _dev(x, torch.bfloat16, "x")
     assert x.dim() == 2 and x.stride(1) == 1
     rows, K = x.shape
     codes = torch.empty((rows, K // 2), dtype=torch.uint8, device=x.device)
     scales = torch.empty((rows, K // group_size, 2), dtype=torch.int16, device=x.device)
-    _check(lib().amx_quantize_f16s(x.data_ptr(), rows, K, x.stride(0), group_size, F16S_ASYMMETRIC if asym else 0,
-                                   codes.data_ptr(), scales.data_ptr(), _stream()), "amx_quantize_f16s")
+    flags = (F16S_ASYMMETRIC if asym else 0) | (F16S_SCALE_E4M3 if e4m3 else 0)
+    _check(lib().amx_quantize_f16s(x.data_ptr(), rows, K, x.stride(0), group_size, flags, codes.data_ptr(), scales.data_ptr(),
+                                   _stream()), "amx_quantize_f16s")
     return codes, scales
 
 

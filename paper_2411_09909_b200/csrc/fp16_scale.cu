@@ -1,7 +1,9 @@
 // FP4 elements with binary16 shared scales, one per group or one per sign: the "FP16" row of the paper's ablation
 // of the shared-scale encoding (arXiv 2411.09909, appendix "Ablation Study on Shared-Scale Bit-Encoding"), there to
 // show how close the 8-bit E5M2 scale comes to a 16-bit one.  The quantizer is that of Sections 4.2-4.3 with every
-// "nearest E5M2" replaced by "nearest binary16" (ties to even, subnormals kept, saturating at 65504).
+// "nearest E5M2" replaced by "nearest binary16" (ties to even, subnormals kept, saturating at 65504).  The same
+// table has a row for the other FP8 scale type, E4M3 ("1-4-3"): an option of the cast here, stored as the binary16
+// pattern of the E4M3 value (every E4M3 value is a binary16 value), so that nothing else changes.
 //
 // Layout: codes as everywhere ([rows, K/2], element 2j in the low nibble), scales uint16 [rows, K/gs, 2] = binary16
 // bit patterns {positive side, negative side} (equal in the symmetric format).
@@ -21,14 +23,25 @@
 namespace amx {
 namespace {
 
+// binary16 pattern of the scale of a side maximum.  E4M3: the nearest FP8 E4M3 value instead (the hardware's
+// convert: nearest even, subnormals, saturating at 448), widened exactly to binary16.  The double rounding through
+// fp32 is harmless for the same reason as above (an E4M3 boundary has even fewer bits).
+template <bool E4M3>
 __device__ __forceinline__ uint32_t scale_bits(float side_max) {
-    const float q = fminf(__fdiv_rn(side_max, 6.0f), 65504.0f);
-    return (uint32_t)__half_as_ushort(__float2half_rn(q));
+    const float q = __fdiv_rn(side_max, 6.0f);
+    if (E4M3) {
+        unsigned short b;
+        uint32_t h2;
+        asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(b) : "f"(0.0f), "f"(q));
+        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(b));
+        return h2 & 0xFFFFu;
+    }
+    return (uint32_t)__half_as_ushort(__float2half_rn(fminf(q, 65504.0f)));
 }
 __device__ __forceinline__ float half_bits_to_float(uint32_t h) { return __half2float(__ushort_as_half((unsigned short)h)); }
 
 // One thread per group: a sweep for the side maxima, a second one (the group is in the L1 by then) for the codes.
-template <bool ASYM>
+template <bool ASYM, bool E4M3>
 __global__ void __launch_bounds__(256) quantize_f16s_kernel(const uint16_t* __restrict__ x, int64_t n_groups, int64_t G,
                                                             int64_t ld_x, int gs, uint32_t* __restrict__ codes,
                                                             uint32_t* __restrict__ scales) {
@@ -49,7 +62,7 @@ __global__ void __launch_bounds__(256) quantize_f16s_kernel(const uint16_t* __re
         }
     }
     if (!ASYM) pmax = nmax = fmaxf(pmax, nmax);
-    const uint32_t hp = scale_bits(pmax), hn = scale_bits(nmax);
+    const uint32_t hp = scale_bits<E4M3>(pmax), hn = scale_bits<E4M3>(nmax);
     const float sp = half_bits_to_float(hp), sn = half_bits_to_float(hn);
     uint32_t* out = codes + (row * G * gs + g * gs) / 8;
     for (int c = 0; c < gs / 8; ++c) {
@@ -98,7 +111,7 @@ using namespace amx;
 extern "C" int amx_quantize_f16s(const void* x, int64_t rows, int64_t K, int64_t ld_x, int group_size, uint32_t flags,
                                  uint8_t* codes, uint16_t* scales, void* stream) {
     if (!fixed_group_size(group_size) || rows < 0 || K <= 0 || K % group_size || ld_x < K) return AMX_ERR_SHAPE;
-    if (flags & ~AMX_F16S_ASYMMETRIC) return AMX_ERR_FLAGS;
+    if (flags & ~(AMX_F16S_ASYMMETRIC | AMX_F16S_SCALE_E4M3)) return AMX_ERR_FLAGS;
     if (rows == 0) return AMX_OK;
     if (!x || !codes || !scales) return AMX_ERR_NULL;
     if (!aligned(x, 16) || ld_x % 8 || !aligned(codes, 4) || !aligned(scales, 4)) return AMX_ERR_ALIGN;
@@ -108,10 +121,10 @@ extern "C" int amx_quantize_f16s(const void* x, int64_t rows, int64_t K, int64_t
     auto* xv = static_cast<const uint16_t*>(x);
     auto* cv = reinterpret_cast<uint32_t*>(codes);
     auto* sv = reinterpret_cast<uint32_t*>(scales);
-    if (flags & AMX_F16S_ASYMMETRIC)
-        quantize_f16s_kernel<true><<<(unsigned)blocks, 256, 0, st>>>(xv, n_groups, G, ld_x, group_size, cv, sv);
-    else
-        quantize_f16s_kernel<false><<<(unsigned)blocks, 256, 0, st>>>(xv, n_groups, G, ld_x, group_size, cv, sv);
+    const bool asym = flags & AMX_F16S_ASYMMETRIC, e4m3 = flags & AMX_F16S_SCALE_E4M3;
+    auto* kernel = asym ? (e4m3 ? quantize_f16s_kernel<true, true> : quantize_f16s_kernel<true, false>)
+                        : (e4m3 ? quantize_f16s_kernel<false, true> : quantize_f16s_kernel<false, false>);
+    kernel<<<(unsigned)blocks, 256, 0, st>>>(xv, n_groups, G, ld_x, group_size, cv, sv);
     return launch_status();
 }
 

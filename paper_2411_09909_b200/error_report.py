@@ -19,7 +19,8 @@ from . import amx, build, inputs
 FORMATS = (("AMXFP4 (two FP8 scales)", amx.FMT_AMXFP4), ("symmetric, FP8 scale", amx.FMT_SYM_FP8),
            ("MXFP4 (power-of-two floor)", amx.FMT_MXFP4), ("per-sign power-of-two floor", amx.FMT_AMXFP4_POT),
            ("power-of-two round", amx.FMT_MXFP4_POT_ROUND), ("per-sign power-of-two round", amx.FMT_AMXFP4_POT_ROUND),
-           ("symmetric, FP16 scale", "f16s"), ("two FP16 scales", "f16s-asym"))
+           ("symmetric, FP16 scale", "f16s"), ("two FP16 scales", "f16s-asym"),
+           ("symmetric, FP8 E4M3 scale", "e4m3"), ("two FP8 E4M3 scales", "e4m3-asym"))
 TENSORS = (("activation, channel outliers (config 2, 4096 wide)", 2, 0, "a"),
            ("activation, SiLU-skewed (config 3, 14336 wide)", 3, 3, "a"),
            ("weight N(0, 0.02) (config 2, 4096 -> 4096)", 2, 1, "w"))
@@ -40,7 +41,7 @@ def report(rows: int = 2048):
         for name, fmt in FORMATS:
             for gs in (128, 64, 32, 16):
                 if isinstance(fmt, str):
-                    codes, scales = amx.quantize_f16s(x, gs, fmt == "f16s-asym")
+                    codes, scales = amx.quantize_f16s(x, gs, fmt.endswith("-asym"), e4m3=fmt.startswith("e4m3"))
                     e = amx.quant_error_f16s(x, codes, scales, gs).cpu().numpy()
                 else:
                     codes, scales = amx.quantize(x, gs, fmt)

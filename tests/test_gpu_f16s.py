@@ -36,6 +36,28 @@ def test_quantize_f16s_bit_exact(asym, gs, kind, rows, K):
     assert np.array_equal(d.astype(np.float64), oracle.dequantize_f16s(oc, os_, gs))     # exact in fp32
 
 
+@pytest.mark.parametrize("asym", [False, True])
+@pytest.mark.parametrize("gs", [16, 128])
+def test_quantize_e4m3_scale_bit_exact(asym, gs):
+    for kind, rows, K in (("normal", 130, 768), ("mixed", 64, 512), ("wide", 40, 256)):
+        bits = inputs.random_groups(3600 + rows + gs, rows, K, kind)
+        c, s = amx.quantize_f16s(dev_bf16(bits), gs, asym, e4m3=True)
+        oc, os_ = oracle.quantize_f16s(bits, gs, asym, e4m3=True)
+        assert np.array_equal(host_u16(s), os_) and np.array_equal(c.cpu().numpy(), oc)
+        d = amx.dequantize_f16s(c, s, gs).cpu().numpy()
+        assert np.array_equal(d.astype(np.float64), oracle.dequantize_f16s(oc, os_, gs))
+    # every bf16 magnitude as a side maximum: E4M3 rounding, subnormals, saturation at 448
+    mags = np.arange(0x0001, 0x7F80, dtype=np.uint16)
+    n = (mags.size // 64) * 64
+    b = np.zeros((n, 16), np.uint16)
+    b[:, 2] = mags[:n]
+    b[:, 11] = mags[:n][::-1] | 0x8000
+    b = b.reshape(-1, 64 * 16)
+    c, s = amx.quantize_f16s(dev_bf16(b), 16, asym, e4m3=True)
+    oc, os_ = oracle.quantize_f16s(b, 16, asym, e4m3=True)
+    assert np.array_equal(host_u16(s), os_) and np.array_equal(c.cpu().numpy(), oc)
+
+
 def test_every_bf16_value_as_group_maximum_and_as_element():
     """Every finite bf16 magnitude as a side maximum (scale rounding, binary16 subnormals, saturation), and every
     finite bf16 value as an element under a few hundred scales (element rounding and ties)."""
@@ -110,7 +132,7 @@ def test_f16s_argument_errors():
     s = torch.zeros((4, 2, 2), dtype=torch.int16, device="cuda")
     st = torch.cuda.current_stream().cuda_stream
     assert L.amx_quantize_f16s(x.data_ptr(), 4, 64, 64, 24, 0, c.data_ptr(), s.data_ptr(), st) == -2
-    assert L.amx_quantize_f16s(x.data_ptr(), 4, 64, 64, 32, 2, c.data_ptr(), s.data_ptr(), st) == -5
+    assert L.amx_quantize_f16s(x.data_ptr(), 4, 64, 64, 32, 4, c.data_ptr(), s.data_ptr(), st) == -5
     assert L.amx_quantize_f16s(None, 4, 64, 64, 32, 0, c.data_ptr(), s.data_ptr(), st) == -1
     assert L.amx_quantize_f16s(x.data_ptr() + 2, 4, 64, 64, 32, 0, c.data_ptr(), s.data_ptr(), st) == -3
     assert L.amx_quantize_f16s(x.data_ptr(), 0, 64, 64, 32, 0, None, None, st) == 0
