@@ -626,12 +626,12 @@ def test_attention_small_head_against_oracle_pipeline():
 def test_attention_all_heads_entry_point_matches_per_head_pipeline(heads, seq, flags):
     q, k, v = (dev_bf16(t) for t in inputs.attention_qkv(heads=heads, seq=seq))
     O = amx.attention_heads(q, k, v, flags=flags)
-    two_pass = seq % 128 == 0 and amx.lib().amx_gemm_kernel_for(seq, seq, 128, 32, flags) == amx.GEMM_FP4
+    fused = seq % 128 == 0 and amx.lib().amx_gemm_kernel_for(seq, seq, 128, 32, flags) == amx.GEMM_FP4
     for h in range(heads):
         Oh, _ = amx.attention(q[h], k[h], v[h], flags=flags)
-        if two_pass:
-            # softmax in the first product's epilogue: the row sums are taken in another order, so a few elements
-            # of P round to the neighbouring bf16 value
+        if fused:
+            # fused kernel: the row sums are taken tile by tile, in another order than the one-kernel softmax of the
+            # per-head pipeline, so a few elements of P round to the neighbouring bf16 value
             assert rel_fro(O[h].cpu().numpy(), Oh.cpu().numpy()) <= 1e-4, h
         else:
             assert torch.equal(O[h], Oh), h
@@ -657,9 +657,9 @@ def test_attention_causal_against_oracle_pipeline(heads, seq, flags):
         assert np.allclose(O[h][0], 0.9375 * oracle.dequantize(*vq, 32)[:, 0], rtol=1e-6, atol=0)
 
 
-def test_attention_two_pass_against_oracle_pipeline():
-    """Attention with the softmax and the cast of P in the epilogue of Q K^T (FP4 kernel, sequence a multiple of
-    256): output against the all-CPU pipeline, every query row."""
+def test_attention_fused_kernel_against_oracle_pipeline():
+    """Attention in the fused kernel (FP4 kernel forced, head dimension 128, sequence a multiple of 128): output
+    against the all-CPU pipeline, every query row."""
     qb, kb, vb = (t[0] for t in inputs.attention_qkv(heads=1, seq=512))
     O = amx.attention_heads(dev_bf16(qb)[None], dev_bf16(kb)[None], dev_bf16(vb)[None], flags=amx.GEMM_FP4)[0]
     S = oracle.gemm(*oracle.quantize(qb, 32), *oracle.quantize(kb, 32), 32)
