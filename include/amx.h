@@ -136,6 +136,18 @@ int amx_quantize_fmt(const void* x, int64_t rows, int64_t K, int64_t ld_x, int g
                      uint8_t* codes, uint8_t* scales, void* stream);
 
 /*
+ * amx_fake_quantize - quantize and dequantize in one pass: out[r, k] = the value amx_dequantize would return for
+ * the codes and scales amx_quantize_fmt produces (any AMX_FMT_* format), as bf16, without the codes reaching memory.
+ * This is the operation the paper's emulation applies to every tensor (Algorithm 1 is this routine for the MX
+ * power-of-two scale; Sections 4.2-4.3 give the FP8 and the asymmetric scales).  Bit-identical to the two calls.
+ *   x, out   device, bf16 [rows, ld], 16-byte aligned, ld % 8 == 0, ld >= K; out may be x (in place)
+ *   group_size 16, 32, 64 or 128; K % group_size == 0
+ * One launch on `stream`; nothing is synchronised; on error nothing was launched.
+ */
+int amx_fake_quantize(const void* x, int64_t rows, int64_t K, int64_t ld_x, int group_size, int format,
+                      void* out, int64_t ld_out, void* stream);
+
+/*
  * amx_quantize_t - the same cast with the groups running DOWN the rows of x (the strided axis):
  * x is bf16 [R, C] row-major (ld_x >= C), groups are gs consecutive rows of one column, and the
  * result is laid out as the canonical quantization of x transposed:

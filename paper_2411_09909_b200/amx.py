@@ -40,6 +40,7 @@ SYMBOLS = (
     "amx_quant_gemm_static_status",
     "amx_quantize_nvfp4", "amx_nvfp4_prepared_bytes", "amx_dequantize_nvfp4", "amx_gemm_nvfp4",
     "amx_quantize_f16s", "amx_dequantize_f16s", "amx_gemm_f16s", "amx_quant_error_f16s",
+    "amx_fake_quantize",
 )
 
 
@@ -77,6 +78,7 @@ def lib() -> ctypes.CDLL:
         L.amx_dequantize_nvfp4.argtypes = [p, p, p, i64, i64, u32, p, i64, p]
         L.amx_gemm_nvfp4.argtypes = [p, p, i64, i64, i64, p, i64, p, sz, p]
         L.amx_quantize_f16s.argtypes = [p, i64, i64, i64, i, u32, p, p, p]
+        L.amx_fake_quantize.argtypes = [p, i64, i64, i64, i, i, p, i64, p]
         L.amx_dequantize_f16s.argtypes = [p, p, i64, i64, i, p, i64, p]
         L.amx_gemm_f16s.argtypes = [p, p, p, p, i64, i64, i64, i, p, i64, p]
         L.amx_quant_error_f16s.argtypes = [p, i64, i64, i64, p, p, i, p, p, sz, p]
@@ -148,6 +150,20 @@ def quantize(x: torch.Tensor, group_size: int = 32, fmt: int = FMT_AMXFP4):
         _check(lib().amx_quantize_fmt(x.data_ptr(), rows, K, ld, group_size, fmt, codes.data_ptr(), scales.data_ptr(),
                                       _stream()), "amx_quantize_fmt")
     return codes, scales
+
+
+def fake_quantize(x: torch.Tensor, group_size: int = 32, fmt: int = FMT_AMXFP4, out: torch.Tensor | None = None):
+    """bf16 [rows, K] (row stride allowed) -> the dequantized cast of x as bf16 (same strides rules); out may be x."""
+    _dev(x, torch.bfloat16, "x")
+    assert x.dim() == 2 and x.stride(1) == 1
+    rows, K = x.shape
+    if out is None:
+        out = torch.empty((rows, K), dtype=torch.bfloat16, device=x.device)
+    assert out.shape == x.shape and out.stride(1) == 1
+    ld = lambda t: t.stride(0) if rows > 1 else max(K, t.stride(0))
+    _check(lib().amx_fake_quantize(x.data_ptr(), rows, K, ld(x), group_size, fmt, out.data_ptr(), ld(out), _stream()),
+           "amx_fake_quantize")
+    return out
 
 
 def quantize_t(x: torch.Tensor, group_size: int = 32):

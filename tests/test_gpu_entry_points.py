@@ -211,3 +211,30 @@ def test_quantize_prepared_without_canonical_codes(rows, K, is_w):
     plane = -(-(rows * K // 2) // 256) * 256
     planes = p1.cpu().numpy()
     assert np.array_equal(planes[: rows * K // 2] | planes[plane: plane + rows * K // 2], oc.reshape(-1))
+
+
+@pytest.mark.parametrize("fmt", [0, 1, 2, 3, 4, 5])
+@pytest.mark.parametrize("gs", [16, 32, 64, 128])
+def test_fake_quantize_equals_cast_then_decode(fmt, gs):
+    """amx_fake_quantize against the oracle's quantize -> dequantize (every format and group size; ragged row count,
+    row-strided input, in place), and against Algorithm 1's own fake-quant routine for MXFP4."""
+    rows, K = 77, 5 * 128
+    bits = inputs.random_groups(5100 + fmt * 10 + gs, rows, K, "mixed")
+    oc, os_ = oracle.quantize(bits, gs) if fmt == 0 else oracle.quantize_variant(bits, gs, fmt)
+    want = inputs.f32_to_bf16_bits(oracle.dequantize(oc, os_, gs).astype(np.float32))
+    x = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    got = amx.fake_quantize(x, gs, fmt).view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(got, want)
+    wide = torch.zeros((rows, K + 24), dtype=torch.bfloat16, device="cuda")
+    wide[:, 8:8 + K] = x
+    view = wide[:, 8:8 + K]
+    amx.fake_quantize(view, gs, fmt, out=view)                        # strided, in place
+    assert np.array_equal(view.contiguous().view(torch.int16).cpu().numpy().view(np.uint16), want)
+    assert not wide[:, :8].any() and not wide[:, 8 + K:].any()
+    if fmt == amx.FMT_MXFP4:
+        v = inputs.bf16_bits_to_f32(bits).astype(np.float64)
+        keep = np.isfinite(v).all(axis=1)
+        alg1 = oracle.fakequant_pot_floor(v[keep], gs, False)
+        scale_ok = np.abs(v[keep]).reshape(keep.sum(), -1, gs).max(axis=2)     # inside the E5M2 range of the stored power of two
+        inr = np.repeat((scale_ok == 0) | ((scale_ok >= 2.0 ** -14) & (scale_ok < 2.0 ** 17)), gs, axis=1)
+        assert np.array_equal(inputs.bf16_bits_to_f32(got[keep]).astype(np.float64)[inr], alg1[inr])
