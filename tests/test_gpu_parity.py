@@ -695,6 +695,25 @@ def test_config5_full_size_attention_sampled():
     assert np.array_equal(pc.cpu().numpy()[rows], opc) and np.array_equal(ps.cpu().numpy()[rows], ops)
 
 
+@pytest.mark.parametrize("causal", [False, True])
+def test_attention_long_sequence_sampled(causal):
+    """Twice config 5's sequence length (16384 tokens, the fused kernel, logits and map never stored): sampled query
+    rows against the all-CPU pipeline."""
+    L = 16384
+    qb, kb, vb = (t[0] for t in inputs.attention_qkv(heads=1, seq=L))
+    O = amx.attention_heads(dev_bf16(qb)[None], dev_bf16(kb)[None], dev_bf16(vb)[None],
+                            flags=amx.ATTN_CAUSAL if causal else 0)[0].cpu().numpy()
+    assert np.all(np.isfinite(O))
+    rows = np.sort(np.random.default_rng(56).choice(L, size=32, replace=False))
+    S = oracle.gemm(*oracle.quantize(qb[rows], 32), *oracle.quantize(kb, 32), 32)
+    if causal:
+        for i, r in enumerate(rows):
+            S[i, r + 1:] = -np.inf
+    P = oracle.softmax_bf16(S, 128 ** -0.5)
+    ref = oracle.gemm(*oracle.quantize(P, 32), *oracle.quantize(np.ascontiguousarray(vb.T), 32), 32)
+    assert rel_fro(O[rows], ref) <= GEMM_TOL
+
+
 # ------------------------------------------------ full-size configurations --
 
 @pytest.mark.parametrize("config,layer", [(c, l) for c in (2, 3, 4) for l in range(len(inputs.LINEAR_CONFIGS[c]["layers"]))])
