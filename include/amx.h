@@ -267,24 +267,28 @@ int amx_softmax_quantize(const float* S, int64_t rows, int64_t cols, int64_t ld_
  * leave in 16 bits).  Per head h:
  *   S = AMX(Q_h) AMX(K_h)^T          groups along head_dim
  *   P = softmax(S / sqrt(d)) per row, fp32, rounded to bf16; no mask.  P itself is never stored.  When both
- *       products run on the FP4 kernel, S is not stored either if d == 128 and L % 128 == 0 (one kernel per
- *       pass does both products and the softmax) or L % 256 == 0: Q K^T runs twice, the first pass keeps
- *       per-row softmax statistics, the second normalises and casts each tile in registers
- *       (row sums are then taken tile by tile, so single elements of P may round to the neighbouring bf16
- *       value compared with amx_softmax_quantize on a stored S; O agrees to ~1e-5 relative)
+ *       products run on the FP4 kernel, d == 128 and L % 128 == 0, S is not stored either: one fused kernel does both
+ *       products and the softmax in two launches - the first pass over Q K^T keeps per-row softmax statistics, the
+ *       second recomputes each tile, normalises and casts it in registers and multiplies it with V on the tensor
+ *       cores (row sums are taken tile by tile, so single elements of P may round to the neighbouring bf16 value
+ *       compared with amx_softmax_quantize on a stored S; O agrees to ~1e-5 relative).  Other shapes and kernels
+ *       store one head's S in the workspace.
  *   O_h = AMX(P) AMX(V_h)            groups along the key axis (V is quantized down its rows)
  *   flags    AMX_GEMM_* kernel choice for both products, optionally | AMX_ATTN_CAUSAL: query i sees keys 0..i only
- *            (the mask is applied to the logits before the softmax; masked entries of P are exactly 0).  On the
- *            two-pass path the blocks of Q K^T that lie entirely after their queries, and the matching part of
- *            P V, are not computed at all.
+ *            (the mask is applied to the logits before the softmax; masked entries of P are exactly 0).  In the
+ *            fused kernel the blocks of keys that lie entirely after their queries are not visited at all.
  *   q, k, v  bf16 [heads, L, d] contiguous;  o  out fp32 [heads, L, d]
  *   d % 32 == 0, L % 32 == 0 (group size 32 on both axes)
- *   workspace  at least amx_attention_workspace_bytes(L, d) bytes (reused head after head), 256-aligned
+ *   workspace  at least amx_attention_workspace_bytes_for(L, d, flags) bytes (reused head after head), 256-aligned.
+ *            amx_attention_workspace_bytes(L, d) is the size that suffices for every flag: it includes one head's
+ *            logits and attention map (L x L x 4.6 bytes), which the fused kernel does not need - at long
+ *            sequences ask with the flags of the call (32768 tokens: 5 GB against 40 MB).
  * The heads are processed one after another on `stream`.
  */
 int amx_attention(const void* q, const void* k, const void* v, int64_t heads, int64_t L, int64_t d,
                   uint32_t flags, float* o, void* workspace, size_t workspace_bytes, void* stream);
 size_t amx_attention_workspace_bytes(int64_t L, int64_t d);
+size_t amx_attention_workspace_bytes_for(int64_t L, int64_t d, uint32_t flags);
 
 /*
  * amx_attention_map - ONE head through the launch sequence amx_attention uses at head dimension 128 (both products

@@ -40,7 +40,7 @@ SYMBOLS = (
     "amx_quant_gemm_static_status",
     "amx_quantize_nvfp4", "amx_nvfp4_prepared_bytes", "amx_dequantize_nvfp4", "amx_gemm_nvfp4",
     "amx_quantize_f16s", "amx_dequantize_f16s", "amx_gemm_f16s", "amx_quant_error_f16s",
-    "amx_fake_quantize",
+    "amx_fake_quantize", "amx_attention_workspace_bytes_for",
 )
 
 
@@ -88,6 +88,8 @@ def lib() -> ctypes.CDLL:
         L.amx_attention.argtypes = [p, p, p, i64, i64, i64, u32, p, p, sz, p]
         L.amx_attention_workspace_bytes.argtypes = [i64, i64]
         L.amx_attention_workspace_bytes.restype = sz
+        L.amx_attention_workspace_bytes_for.argtypes = [i64, i64, u32]
+        L.amx_attention_workspace_bytes_for.restype = sz
         L.amx_prepared_bytes.argtypes = [i64, i64, i, i]
         L.amx_prepared_bytes.restype = sz
         L.amx_prepare.argtypes = [p, p, i64, i64, i, i, p, sz, p]
@@ -461,7 +463,7 @@ def attention_heads(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, flags: in
         _dev(t, torch.bfloat16, "q/k/v")
         assert t.is_contiguous() and t.shape == q.shape
     H, Lq, d = q.shape
-    need = lib().amx_attention_workspace_bytes(Lq, d)
+    need = lib().amx_attention_workspace_bytes_for(Lq, d, flags)
     if workspace is None:
         workspace = _ws(need, q.device)
     out = torch.empty((H, Lq, d), dtype=torch.float32, device=q.device)

@@ -330,23 +330,27 @@ int64_t attn_chunk(int64_t L, int64_t d) {
 struct AttnLayout {
     size_t qc, qs, kc, ks, vc, vs, pc, ps, S, pq, pk, pv, pp, stats, gemm, total;
 };
-AttnLayout attn_layout(int64_t L, int64_t d) {
+// fused_only: the fused kernel will run (both products on the FP4 kernel, attn_fused_supported): no room for one
+// head's logits, cast map and prepared map, nor for the other kernels' scratch.
+AttnLayout attn_layout(int64_t L, int64_t d, bool fused_only = false) {
     AttnLayout a;
     const int64_t hc = attn_chunk(L, d);
     const QuantSizes qd = quant_sizes(hc * L, d, 32), ql = quant_sizes(L, L, 32), qv = quant_sizes(hc * d, L, 32);
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off += round_up(bytes); return o; };
     a.qc = take(qd.codes); a.qs = take(qd.scales); a.kc = take(qd.codes); a.ks = take(qd.scales);
-    a.vc = take(qv.codes); a.vs = take(qv.scales); a.pc = take(ql.codes); a.ps = take(ql.scales);
-    a.S = take((size_t)L * L * 4);
+    a.vc = take(qv.codes); a.vs = take(qv.scales);
+    a.pc = take(fused_only ? 0 : ql.codes); a.ps = take(fused_only ? 0 : ql.scales);
+    a.S = take(fused_only ? 0 : (size_t)L * L * 4);
     // right-hand operands are laid out for 128 rows more: the last head's 256-row tiles may reach past the stack
     a.pq = take(gemm_fp4_prepared_bytes(hc * L, d, false));
     a.pk = take(gemm_fp4_prepared_bytes(hc * L + 128, d, true));
     a.pv = take(gemm_fp4_prepared_bytes(hc * d + 128, L, true));
-    a.pp = take(gemm_fp4_prepared_bytes(L, L, false));
+    a.pp = take(fused_only ? 0 : gemm_fp4_prepared_bytes(L, L, false));
     a.stats = take(attn_fused_supported(L, d) ? attn_fused_scratch_bytes(hc, L) : 0);
     a.gemm = off;
-    const size_t g1 = amx_workspace_bytes(L, L, d, 32, AMX_GEMM_TC), g2 = amx_workspace_bytes(L, d, L, 32, AMX_GEMM_TC);
+    const size_t g1 = fused_only ? 0 : amx_workspace_bytes(L, L, d, 32, AMX_GEMM_TC);
+    const size_t g2 = fused_only ? 0 : amx_workspace_bytes(L, d, L, 32, AMX_GEMM_TC);
     a.total = off + (g1 > g2 ? g1 : g2) + 256;
     return a;
 }
@@ -355,6 +359,21 @@ AttnLayout attn_layout(int64_t L, int64_t d) {
 extern "C" size_t amx_attention_workspace_bytes(int64_t L, int64_t d) {
     if (L <= 0 || d <= 0 || L % 32 || d % 32) return 0;
     return attn_layout(L, d).total;
+}
+
+namespace {
+// Whether a call with these flags runs the fused kernel.
+bool attn_runs_fused(int64_t L, int64_t d, uint32_t flags) {
+    flags &= ~AMX_ATTN_CAUSAL;
+    if (flags & ~kKernelMask) return false;
+    return attn_fused_supported(L, d) && pick_kernel(L, L, d, 32, flags) == AMX_GEMM_FP4 &&
+           pick_kernel(L, d, L, 32, flags) == AMX_GEMM_FP4;
+}
+}  // namespace
+
+extern "C" size_t amx_attention_workspace_bytes_for(int64_t L, int64_t d, uint32_t flags) {
+    if (L <= 0 || d <= 0 || L % 32 || d % 32) return 0;
+    return attn_layout(L, d, attn_runs_fused(L, d, flags)).total;
 }
 
 extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_t heads, int64_t L, int64_t d,
@@ -367,7 +386,7 @@ extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_
     if (!k_qk || !k_pv) return ((flags & kKernelMask) & ((flags & kKernelMask) - 1)) ? AMX_ERR_FLAGS : AMX_ERR_SHAPE;
     if (heads == 0) return AMX_OK;
     if (!q || !k || !v || !o) return AMX_ERR_NULL;
-    const AttnLayout a = attn_layout(L, d);
+    const AttnLayout a = attn_layout(L, d, attn_runs_fused(L, d, flags));
     if (!workspace || workspace_bytes < a.total) return AMX_ERR_WORKSPACE;
     if (!aligned(workspace, kAlign) || !aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 4))
         return AMX_ERR_ALIGN;
