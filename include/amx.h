@@ -289,6 +289,14 @@ int amx_attention(const void* q, const void* k, const void* v, int64_t heads, in
                   uint32_t flags, float* o, void* workspace, size_t workspace_bytes, void* stream);
 size_t amx_attention_workspace_bytes(int64_t L, int64_t d);
 size_t amx_attention_workspace_bytes_for(int64_t L, int64_t d, uint32_t flags);
+/*
+ * amx_attention_gqa - the same with grouped queries: k and v hold kv_heads heads [kv_heads, L, d] and query head h
+ * attends to head h / (heads / kv_heads) of them (heads % kv_heads == 0, else AMX_ERR_SHAPE); keys and values are
+ * cast once per head of theirs.  kv_heads == heads is amx_attention; the results are those of amx_attention on
+ * keys and values repeated heads / kv_heads times, bit for bit.  Same workspace.
+ */
+int amx_attention_gqa(const void* q, const void* k, const void* v, int64_t heads, int64_t kv_heads, int64_t L, int64_t d,
+                      uint32_t flags, float* o, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * amx_attention_map - ONE head through the launch sequence amx_attention uses at head dimension 128 (both products

@@ -40,7 +40,7 @@ SYMBOLS = (
     "amx_quant_gemm_static_status",
     "amx_quantize_nvfp4", "amx_nvfp4_prepared_bytes", "amx_dequantize_nvfp4", "amx_gemm_nvfp4",
     "amx_quantize_f16s", "amx_dequantize_f16s", "amx_gemm_f16s", "amx_quant_error_f16s",
-    "amx_fake_quantize", "amx_attention_workspace_bytes_for",
+    "amx_fake_quantize", "amx_attention_workspace_bytes_for", "amx_attention_gqa",
 )
 
 
@@ -86,6 +86,7 @@ def lib() -> ctypes.CDLL:
         L.amx_quant_gemm_static_capacity.argtypes = []
         L.amx_quant_gemm_static_capacity.restype = sz
         L.amx_attention.argtypes = [p, p, p, i64, i64, i64, u32, p, p, sz, p]
+        L.amx_attention_gqa.argtypes = [p, p, p, i64, i64, i64, i64, u32, p, p, sz, p]
         L.amx_attention_workspace_bytes.argtypes = [i64, i64]
         L.amx_attention_workspace_bytes.restype = sz
         L.amx_attention_workspace_bytes_for.argtypes = [i64, i64, u32]
@@ -457,18 +458,23 @@ def linear_host(a_host: torch.Tensor, w_host: torch.Tensor, c_host: torch.Tensor
 
 def attention_heads(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, flags: int = GEMM_AUTO,
                     workspace: torch.Tensor | None = None):
-    """Fully quantized attention for all heads through the single C entry point.  q, k, v: bf16 [H, L, d]
-    contiguous.  Returns O fp32 [H, L, d]."""
+    """Fully quantized attention for all heads through the single C entry point.  q: bf16 [H, L, d]; k, v: bf16
+    [H_kv, L, d] with H % H_kv == 0 (grouped queries when H_kv < H); all contiguous.  Returns O fp32 [H, L, d]."""
     for t in (q, k, v):
         _dev(t, torch.bfloat16, "q/k/v")
-        assert t.is_contiguous() and t.shape == q.shape
+        assert t.is_contiguous() and t.shape[1:] == q.shape[1:]
+    assert k.shape == v.shape
     H, Lq, d = q.shape
     need = lib().amx_attention_workspace_bytes_for(Lq, d, flags)
     if workspace is None:
         workspace = _ws(need, q.device)
     out = torch.empty((H, Lq, d), dtype=torch.float32, device=q.device)
-    _check(lib().amx_attention(q.data_ptr(), k.data_ptr(), v.data_ptr(), H, Lq, d, flags, out.data_ptr(),
-                               workspace.data_ptr(), workspace.numel(), _stream()), "amx_attention")
+    if k.shape[0] == H:
+        _check(lib().amx_attention(q.data_ptr(), k.data_ptr(), v.data_ptr(), H, Lq, d, flags, out.data_ptr(),
+                                   workspace.data_ptr(), workspace.numel(), _stream()), "amx_attention")
+    else:
+        _check(lib().amx_attention_gqa(q.data_ptr(), k.data_ptr(), v.data_ptr(), H, k.shape[0], Lq, d, flags, out.data_ptr(),
+                                       workspace.data_ptr(), workspace.numel(), _stream()), "amx_attention_gqa")
     return out
 
 

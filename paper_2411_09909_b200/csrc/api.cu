@@ -378,10 +378,18 @@ extern "C" size_t amx_attention_workspace_bytes_for(int64_t L, int64_t d, uint32
 
 extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_t heads, int64_t L, int64_t d,
                              uint32_t flags, float* o, void* workspace, size_t workspace_bytes, void* stream) {
+    return amx_attention_gqa(q, k, v, heads, heads, L, d, flags, o, workspace, workspace_bytes, stream);
+}
+
+extern "C" int amx_attention_gqa(const void* q, const void* k, const void* v, int64_t heads, int64_t kv_heads, int64_t L,
+                                 int64_t d, uint32_t flags, float* o, void* workspace, size_t workspace_bytes,
+                                 void* stream) {
     const int causal = (flags & AMX_ATTN_CAUSAL) ? 1 : 0;
     flags &= ~AMX_ATTN_CAUSAL;
     if (flags & ~kKernelMask) return AMX_ERR_FLAGS;
     if (heads < 0 || L <= 0 || d <= 0 || L % 32 || d % 32) return AMX_ERR_SHAPE;
+    if (heads > 0 && (kv_heads <= 0 || heads % kv_heads)) return AMX_ERR_SHAPE;
+    const int64_t group = heads > 0 ? heads / kv_heads : 1;        // query heads per head of keys and values
     const uint32_t k_qk = pick_kernel(L, L, d, 32, flags), k_pv = pick_kernel(L, d, L, 32, flags);
     if (!k_qk || !k_pv) return ((flags & kKernelMask) & ((flags & kKernelMask) - 1)) ? AMX_ERR_FLAGS : AMX_ERR_SHAPE;
     if (heads == 0) return AMX_OK;
@@ -395,64 +403,77 @@ extern "C" int amx_attention(const void* q, const void* k, const void* v, int64_
     const size_t gemm_bytes = a.total - a.gemm;
     const float alpha = 1.0f / sqrtf((float)d);
     float* S = reinterpret_cast<float*>(w + a.S);
-    const int64_t chunk = attn_chunk(L, d);
+    const int64_t chunk_max = attn_chunk(L, d);
+    // a chunk holds whole groups of query heads (or, when a group is larger than a chunk, part of one group)
+    const int64_t chunk = group >= chunk_max ? chunk_max : (chunk_max / group) * group;
     // both products on the FP4 kernel at head dimension 128: one fused kernel, logits and attention map stay on chip
     const bool fused = k_qk == AMX_GEMM_FP4 && k_pv == AMX_GEMM_FP4 && attn_fused_supported(L, d);
     const size_t head_in = (size_t)L * d * 2;                       // bytes of one head of q, k or v
     const size_t qk_codes = (size_t)L * d / 2, qk_scales = (size_t)L * (d / 32) * 2;   // one head of Q or K, canonical
     const size_t v_codes = (size_t)d * L / 2, v_scales = (size_t)d * (L / 32) * 2;     // one head of V^T
-    for (int64_t h0 = 0; h0 < heads; h0 += chunk) {
-        const int64_t hc = heads - h0 < chunk ? heads - h0 : chunk;
+    for (int64_t h0 = 0; h0 < heads;) {
+        // query heads h0 .. h0 + hc - 1 and the heads of keys and values they use, kv0 .. kv0 + kvc - 1
+        const int64_t left_in_group = group - h0 % group;
+        int64_t hc = heads - h0 < chunk ? heads - h0 : chunk;
+        if (group >= chunk_max && hc > left_in_group) hc = left_in_group;      // never across two large groups
+        const int64_t kv0 = h0 / group, kvc = (h0 + hc - 1) / group - kv0 + 1;
+        const int64_t h_off = h0 - kv0 * group;                     // first query head's place inside its group
         const uint8_t* qh = static_cast<const uint8_t*>(q) + h0 * head_in;
-        const uint8_t* kh = static_cast<const uint8_t*>(k) + h0 * head_in;
-        const uint8_t* vh = static_cast<const uint8_t*>(v) + h0 * head_in;
+        const uint8_t* kh = static_cast<const uint8_t*>(k) + kv0 * head_in;
+        const uint8_t* vh = static_cast<const uint8_t*>(v) + kv0 * head_in;
         // casts of the chunk's heads, stacked row-wise: Q and K along head_dim, V along the sequence (V^T)
         int rc;
         if (k_qk == AMX_GEMM_FP4) {
-            rc = gemm_fp4_quantize_prepared(qh, hc * L, d, false, nullptr, w + a.qs, w + a.pq, st, chunk * L);
+            rc = gemm_fp4_quantize_prepared(qh, hc * L, d, false, nullptr, w + a.qs, w + a.pq, st, chunk_max * L);
             if (rc == AMX_OK)
-                rc = gemm_fp4_quantize_prepared(kh, hc * L, d, true, nullptr, w + a.ks, w + a.pk, st, chunk * L + 128);
+                rc = gemm_fp4_quantize_prepared(kh, kvc * L, d, true, nullptr, w + a.ks, w + a.pk, st, chunk_max * L + 128);
         } else {
             rc = amx_quantize(qh, hc * L, d, d, 32, w + a.qc, w + a.qs, stream);
-            if (rc == AMX_OK) rc = amx_quantize(kh, hc * L, d, d, 32, w + a.kc, w + a.ks, stream);
+            if (rc == AMX_OK) rc = amx_quantize(kh, kvc * L, d, d, 32, w + a.kc, w + a.ks, stream);
         }
-        if (rc == AMX_OK) rc = quantize_cols_batched(vh, hc, L, d, w + a.vc, w + a.vs, st);
+        if (rc == AMX_OK) rc = quantize_cols_batched(vh, kvc, L, d, w + a.vc, w + a.vs, st);
         if (rc == AMX_OK && k_pv == AMX_GEMM_FP4)
-            rc = gemm_fp4_prepare(w + a.vc, w + a.vs, hc * d, L, true, w + a.pv, st, chunk * d + 128);
+            rc = gemm_fp4_prepare(w + a.vc, w + a.vs, kvc * d, L, true, w + a.pv, st, chunk_max * d + 128);
         if (rc != AMX_OK) return rc;
         if (fused) {
-            // head dimension 128: both products and the softmax of all the chunk's heads in two launches
-            rc = attn_fused({w + a.pq, hc * L, chunk * L, 0}, {w + a.pk, hc * L, chunk * L + 128, 0},
-                            {w + a.pv, hc * d, chunk * d + 128, 0}, (int)hc, L, alpha, causal, w + a.stats,
-                            o + (size_t)h0 * L * d, w + a.gemm, st);
+            // head dimension 128: both products and the softmax of all the chunk's heads in two launches.  The chunk
+            // starts at a group boundary unless the group is larger than a chunk, in which case it lies inside one
+            // group (every head maps to the chunk's one head of keys and values either way).
+            rc = attn_fused({w + a.pq, hc * L, chunk_max * L, 0}, {w + a.pk, kvc * L, chunk_max * L + 128, 0},
+                            {w + a.pv, kvc * d, chunk_max * d + 128, 0}, (int)hc, L, alpha, causal, w + a.stats,
+                            o + (size_t)h0 * L * d, w + a.gemm, st, nullptr, nullptr, nullptr, nullptr,
+                            (int)(group >= chunk_max ? chunk_max : group));
             if (rc != AMX_OK) return rc;
+            h0 += hc;
             continue;
         }
         for (int64_t i = 0; i < hc; ++i) {
+            const int64_t kv = (h_off + i) / group;                 // this head's keys and values inside the chunk
             float* oh = o + (size_t)(h0 + i) * L * d;
             // S = AMX(Q) AMX(K)^T
             if (k_qk == AMX_GEMM_FP4)
-                rc = gemm_fp4_prepared_at({w + a.pq, hc * L, chunk * L, i * L}, {w + a.pk, hc * L, chunk * L + 128, i * L}, L,
-                                          L, d, S, L, w + a.gemm, st);
+                rc = gemm_fp4_prepared_at({w + a.pq, hc * L, chunk_max * L, i * L},
+                                          {w + a.pk, kvc * L, chunk_max * L + 128, kv * L}, L, L, d, S, L, w + a.gemm, st);
             else
-                rc = amx_gemm(w + a.qc + i * qk_codes, w + a.qs + i * qk_scales, w + a.kc + i * qk_codes,
-                              w + a.ks + i * qk_scales, L, L, d, 32, k_qk, S, L, w + a.gemm, gemm_bytes, stream);
+                rc = amx_gemm(w + a.qc + i * qk_codes, w + a.qs + i * qk_scales, w + a.kc + kv * qk_codes,
+                              w + a.ks + kv * qk_scales, L, L, d, 32, k_qk, S, L, w + a.gemm, gemm_bytes, stream);
             if (rc != AMX_OK) return rc;
             // softmax, rounding to bf16 and the cast of P in one kernel; O = AMX(P) AMX(V)
             if (k_pv == AMX_GEMM_FP4) {
                 rc = gemm_fp4_softmax_prepared(S, L, L, L, alpha, false, w + a.pc, w + a.ps, w + a.pp, st, causal);
                 if (rc == AMX_OK)
-                    rc = gemm_fp4_prepared_at({w + a.pp, L, L, 0}, {w + a.pv, hc * d, chunk * d + 128, i * d}, L, d, L, oh, d,
-                                              w + a.gemm, st);
+                    rc = gemm_fp4_prepared_at({w + a.pp, L, L, 0}, {w + a.pv, kvc * d, chunk_max * d + 128, kv * d}, L, d, L, oh,
+                                              d, w + a.gemm, st);
             } else {
                 rc = softmax_cast_rows(S, L, L, L, alpha, w + a.pc, w + a.ps, nullptr, nullptr, nullptr, nullptr, nullptr, 0, L,
                                        st, causal);
                 if (rc == AMX_OK)
-                    rc = amx_gemm(w + a.pc, w + a.ps, w + a.vc + i * v_codes, w + a.vs + i * v_scales, L, d, L, 32, k_pv, oh,
+                    rc = amx_gemm(w + a.pc, w + a.ps, w + a.vc + kv * v_codes, w + a.vs + kv * v_scales, L, d, L, 32, k_pv, oh,
                                   d, w + a.gemm, gemm_bytes, stream);
             }
             if (rc != AMX_OK) return rc;
         }
+        h0 += hc;
     }
     return AMX_OK;
 }

@@ -82,12 +82,13 @@ constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17
 
 struct Params {
     // prepared operands (fp4_operand.cuh); row ranges of stacked heads: head h of the launch has its queries at
-    // rows q_row0 + h * L of Q, its keys at k_row0 + h * L of K, its 128 V^T rows at v_row0 + h * 128
+    // rows q_row0 + h * L of Q, its keys at k_row0 + (h / kv_group) * L of K, its 128 V^T rows at
+    // v_row0 + (h / kv_group) * 128 (kv_group query heads share one head of keys and values: grouped-query attention)
     const uint8_t *sfq[2], *sfk[2], *sfv[2];         // scale-factor chunks of the planes, from the operand's first chunk
     const int *q_words, *k_words, *v_words;          // row words, from the operand's first row
     int64_t q_row0, k_row0, v_row0;
     int nk64_q, nk64_k, nk64_v;
-    int heads, m_tiles, causal;
+    int heads, m_tiles, causal, kv_group;
     int64_t L;
     float alpha;
     float2* part;            // [heads * L][4]: per row and key-group column {max, sum of 2^(t - max)}, base-2 units
@@ -163,8 +164,8 @@ attention_fp4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     }
                     uint8_t* st = sm + S_::kOffKV + s * S_::kStageBytes;
                     mbar_expect_tx(&ctl->kv_full[s], S_::kStageBytes);
-                    tma_load_3d(st, &tm_k, 0, (int)(p.k_row0 + (int64_t)h * p.L + j * BNK), 0, &ctl->kv_full[s]);
-                    if (PASS == 2) tma_load_3d(st + kTileBytes, &tm_v, j * 64, (int)(p.v_row0 + (int64_t)h * HD), 0, &ctl->kv_full[s]);
+                    tma_load_3d(st, &tm_k, 0, (int)(p.k_row0 + (int64_t)(h / p.kv_group) * p.L + j * BNK), 0, &ctl->kv_full[s]);
+                    if (PASS == 2) tma_load_3d(st + kTileBytes, &tm_v, j * 64, (int)(p.v_row0 + (int64_t)(h / p.kv_group) * HD), 0, &ctl->kv_full[s]);
                 }
             }
             // after a timeout: let the copies already in flight land before shared memory is released
@@ -286,13 +287,13 @@ attention_fp4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             const int T = tiles_of(m_blk);
             for (int j = 0; j < T; ++j, ++it) {
                 const int s = it % kStages;
-                const int64_t k_row = p.k_row0 + (int64_t)h * p.L + j * BNK;
+                const int64_t k_row = p.k_row0 + (int64_t)(h / p.kv_group) * p.L + j * BNK;
                 uint4 vk[4], vv[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) vk[i] = chunk(p.sfk[i >> 1], k_row, p.nk64_k, i & 1);
                 if (PASS == 2) {
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) vv[i] = chunk(p.sfv[i >> 1], p.v_row0 + (int64_t)h * HD, p.nk64_v, j * 2 + (i & 1));
+                    for (int i = 0; i < 4; ++i) vv[i] = chunk(p.sfv[i >> 1], p.v_row0 + (int64_t)(h / p.kv_group) * HD, p.nk64_v, j * 2 + (i & 1));
                 }
                 const int kw = row_word_exp(__ldg(p.k_words + k_row + t));
                 if (ok && it >= kStages) ok = mbar_wait(&ctl->kv_empty[s], ((it / kStages) - 1) & 1, &ctl->abort, p.status);
@@ -485,7 +486,7 @@ attention_fp4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&ctl->o_empty);
-                const int4* vw = reinterpret_cast<const int4*>(p.v_words + p.v_row0 + (int64_t)h * HD + cg_o * 32);
+                const int4* vw = reinterpret_cast<const int4*>(p.v_words + p.v_row0 + (int64_t)(h / p.kv_group) * HD + cg_o * 32);
                 float* out = p.O + ((int64_t)h * p.L + m) * HD + cg_o * 32;
                 const int p_exp = kmax ? kmax - 25 : 0;
 #pragma unroll
@@ -540,7 +541,7 @@ size_t attn_fused_scratch_bytes(int64_t heads, int64_t L) { return up256((size_t
 // workspace: 256 bytes (status word).  dbg_*: optional verification outputs for head 0 (see Params).
 int attn_fused(const Fp4Operand& q, const Fp4Operand& k, const Fp4Operand& vt, int heads, int64_t L, float alpha, int causal,
                void* scratch, float* O, void* workspace, cudaStream_t st, void* dbg_bits, uint8_t* dbg_codes, uint8_t* dbg_scales,
-               void* dbg_prepared) {
+               void* dbg_prepared, int kv_group) {
     if (!attn_fused_supported(L, HD) || heads <= 0 || q.row0 % 128 || k.row0 % 128 || vt.row0 % 128) return AMX_ERR_SHAPE;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AMX_ERR_CUDA;
@@ -568,6 +569,7 @@ int attn_fused(const Fp4Operand& q, const Fp4Operand& k, const Fp4Operand& vt, i
     p.q_row0 = q.row0; p.k_row0 = k.row0; p.v_row0 = vt.row0;
     p.nk64_q = oq.nk64; p.nk64_k = ok_.nk64; p.nk64_v = ov.nk64;
     p.heads = heads; p.m_tiles = (int)(L / BM); p.causal = causal ? 1 : 0;
+    p.kv_group = kv_group > 0 ? kv_group : 1;
     p.L = L; p.alpha = alpha;
     p.part = static_cast<float2*>(scratch);
     p.O = O;

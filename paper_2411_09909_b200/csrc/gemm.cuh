@@ -86,7 +86,8 @@ bool attn_fused_supported(int64_t L, int64_t d);
 size_t attn_fused_scratch_bytes(int64_t heads, int64_t L);
 int attn_fused(const Fp4Operand& q, const Fp4Operand& k, const Fp4Operand& vt, int heads, int64_t L, float alpha, int causal,
                void* scratch, float* O, void* workspace /* 256 B: status word */, cudaStream_t st, void* dbg_bits = nullptr,
-               uint8_t* dbg_codes = nullptr, uint8_t* dbg_scales = nullptr, void* dbg_prepared = nullptr);
+               uint8_t* dbg_codes = nullptr, uint8_t* dbg_scales = nullptr, void* dbg_prepared = nullptr,
+               int kv_group = 1 /* query heads per head of keys and values; k and vt then stack heads / kv_group heads */);
 int quantize_cols_batched(const void* x, int64_t batch, int64_t R, int64_t C, uint8_t* codes, uint8_t* scales,
                           cudaStream_t st);
 int gemm_fp4_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,

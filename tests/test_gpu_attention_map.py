@@ -123,3 +123,30 @@ def test_attention_map_cast_bit_exact_full_size_sampled(causal):
     check_rows(rows, L, p_bits, c_np, s_np, prep.cpu().numpy(), causal)
     check_output(o.cpu().numpy(), rows[::4], c_np, s_np, vb)
     assert amx.prepared_flushed_scales(prep, L, L, False) == 0
+
+
+@pytest.mark.parametrize("heads,kv_heads,L,d,flags", [(8, 2, 256, 128, amx.GEMM_FP4),                    # fused kernel, groups of 4
+                                                       (20, 4, 128, 128, amx.GEMM_FP4 | amx.ATTN_CAUSAL),  # groups of 5: chunks of 15 heads
+                                                       (34, 1, 128, 128, amx.GEMM_FP4),                    # one group larger than a chunk
+                                                       (6, 2, 160, 64, amx.GEMM_AUTO),                     # stored logits, head by head
+                                                       (9, 3, 256, 128, amx.GEMM_TC | amx.ATTN_CAUSAL)])   # chunks of 8 heads, groups of 3
+def test_grouped_query_attention_equals_repeated_heads(heads, kv_heads, L, d, flags):
+    """amx_attention_gqa: query head h uses head h / (heads / kv_heads) of keys and values - the same bits as
+    amx_attention on keys and values repeated; one head also against the all-CPU pipeline."""
+    rng = np.random.default_rng(heads * 100 + kv_heads)
+    def bf(shape):
+        return torch.from_numpy(inputs.f32_to_bf16_bits(rng.standard_normal(shape).astype(np.float32)).view(np.int16)).cuda().view(torch.bfloat16)
+    q, k, v = bf((heads, L, d)), bf((kv_heads, L, d)), bf((kv_heads, L, d))
+    g = heads // kv_heads
+    got = amx.attention_heads(q, k, v, flags=flags)
+    want = amx.attention_heads(q, k.repeat_interleave(g, dim=0).contiguous(), v.repeat_interleave(g, dim=0).contiguous(), flags=flags)
+    assert torch.equal(got, want)
+    h = heads - 1
+    u16 = lambda t: t.view(torch.int16).cpu().numpy().view(np.uint16)
+    qb, kb, vb = u16(q[h]), u16(k[h // g]), u16(v[h // g])
+    S = oracle.gemm(*oracle.quantize(qb, 32), *oracle.quantize(kb, 32), 32)
+    P = oracle.softmax_bf16(S, d ** -0.5, causal_row0=0) if flags & amx.ATTN_CAUSAL else oracle.softmax_bf16(S, d ** -0.5)
+    ref = oracle.gemm(*oracle.quantize(P, 32), *oracle.quantize(np.ascontiguousarray(vb.T), 32), 32).astype(np.float64)
+    assert np.linalg.norm(got[h].cpu().numpy() - ref) <= 1e-3 * np.linalg.norm(ref)
+    L_ = amx.lib()
+    assert L_.amx_attention_gqa(q.data_ptr(), k.data_ptr(), v.data_ptr(), heads, heads + 1, L, d, 0, got.data_ptr(), None, 0, None) == -2
