@@ -227,7 +227,8 @@ __device__ __forceinline__ void store_row16(float* out, const float (&f)[16], bo
 // wide, the stage layout keeps its size.
 template <int BK_, bool SLICED = false, bool NHALF = false>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w, const Params p) {
+gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
+                const __grid_constant__ CUtensorMap tm_a1, const __grid_constant__ CUtensorMap tm_w1, const Params p) {
     using C_ = Cfg<BK_>;
     if (p.gate && *p.gate != 0) return;                          // uniform over the grid: nothing was set up yet
     constexpr int BNT = NHALF ? BN / 2 : BN;                     // tile width
@@ -295,14 +296,45 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem = ctl->tmem_base;
 
+    // Which sign planes a tile's rows use at all (bits of the row words, OR-ed over the tile's 128 + 256 rows; each
+    // lane its share, to be OR-ed over the warp): bit 0/1: A has +/-, bit 2/3: W has +/-.  The products with a plane
+    // that is zero for the whole tile are not issued, and that plane is not even loaded: an operand in a symmetric
+    // format, or the all-positive attention map, moves half the bytes.
+    auto tile_sides = [&](int64_t tile) {
+        int bits = 0;
+        if (tile < total_tiles) {
+            const int64_t m0 = blk_m(tile) * BM, n0 = blk_n(tile) * BNT;
+#pragma unroll
+            for (int i = 0; i < BM / 32; ++i)
+                if (m0 + i * 32 + lane < p.M) bits |= (__ldg(p.a_exp + m0 + i * 32 + lane) >> 16) & 3;
+#pragma unroll
+            for (int i = 0; i < BNT / 32; ++i)
+                if (n0 + i * 32 + lane < p.N) bits |= ((__ldg(p.w_exp + n0 + i * 32 + lane) >> 16) & 3) << 2;
+        }
+        return bits;
+    };
+    auto whole_sides = [&](int lane_bits) {                         // over the warp; an all-zero operand keeps one plane
+        int sides = __reduce_or_sync(0xFFFFFFFFu, lane_bits);
+        if (!(sides & 3)) sides |= 1;
+        if (!(sides & 12)) sides |= 4;
+        return sides;
+    };
+
     if (warp == 0) {
         // -------------------------------------------------------------- TMA producer
-        if (lane == 0) {
-            int it = 0;                                          // K blocks issued so far, over all tiles
-            bool ok = true;
-            for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int64_t m_blk = blk_m(tile), n_blk = blk_n(tile);
-                const int kb0 = kb_begin(tile), nkb = nkb_of(tile);
+        // The whole warp finds the tile's planes; one lane waits and issues.
+        constexpr int kTileWT = NHALF ? C_::kTileB / 2 : C_::kTileB;   // one plane of the W tile as loaded
+        int it = 0;                                                  // K blocks issued so far, over all tiles
+        bool ok = true;
+        int sides_next = tile_sides(blockIdx.x);
+        for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            const int sides = whole_sides(sides_next);
+            sides_next = tile_sides(tile + gridDim.x);
+            const int64_t m_blk = blk_m(tile), n_blk = blk_n(tile);
+            const int kb0 = kb_begin(tile), nkb = nkb_of(tile);
+            const int a_planes = sides & 3, w_planes = (sides >> 2) & 3;
+            const uint32_t bytes = (a_planes == 3 ? 2 : 1) * C_::kTileA + (w_planes == 3 ? 2 : 1) * kTileWT;
+            if (lane == 0) {
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % kStages;
                     if (it >= kStages && !mbar_wait(&ctl->empty[s], ((it / kStages) - 1) & 1, &ctl->abort, p.status)) {
@@ -310,17 +342,22 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                         break;
                     }
                     uint8_t* st = tiles + s * kStageBytes;
-                    mbar_expect_tx(&ctl->full[s], kStageBytes - (NHALF ? C_::kTileB : 0));
-                    // one 3-D tile per operand: {row bytes, rows, both sign planes}
-                    tma_load_3d(st + C_::kOffAp, &tm_a, (kb0 + kb) * kRowBytes, (int)(p.a_row0 + m_blk * BM), 0, &ctl->full[s]);
-                    tma_load_3d(st + C_::kOffWp, &tm_w, (kb0 + kb) * kRowBytes, (int)(p.w_row0 + n_blk * BNT), 0, &ctl->full[s]);
+                    mbar_expect_tx(&ctl->full[s], bytes);
+                    const int x = (kb0 + kb) * kRowBytes, ya = (int)(p.a_row0 + m_blk * BM), yw = (int)(p.w_row0 + n_blk * BNT);
+                    // one 3-D tile per operand: {row bytes, rows, both sign planes} - or the one plane that is not zero
+                    if (a_planes == 3) tma_load_3d(st + C_::kOffAp, &tm_a, x, ya, 0, &ctl->full[s]);
+                    else tma_load_3d(st + (a_planes == 2 ? C_::kOffAn : C_::kOffAp), &tm_a1, x, ya, a_planes == 2 ? 1 : 0, &ctl->full[s]);
+                    if (w_planes == 3) tma_load_3d(st + C_::kOffWp, &tm_w, x, yw, 0, &ctl->full[s]);
+                    else tma_load_3d(st + (w_planes == 2 ? kOffWnT : C_::kOffWp), &tm_w1, x, yw, w_planes == 2 ? 1 : 0, &ctl->full[s]);
                 }
             }
-            // after an abort: let the copies already in flight land before shared memory is released
-            if (ctl->abort)
-                for (int i = max(0, it - kStages); i < it; ++i)
-                    for (uint32_t n = 0; n < kSpinLimit && !mbar_try_wait(&ctl->full[i % kStages], (i / kStages) & 1); ++n) {}
+            it = __shfl_sync(0xFFFFFFFFu, it, 0);
+            ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
         }
+        // after an abort: let the copies already in flight land before shared memory is released
+        if (lane == 0 && ctl->abort)
+            for (int i = max(0, it - kStages); i < it; ++i)
+                for (uint32_t n = 0; n < kSpinLimit && !mbar_try_wait(&ctl->full[i % kStages], (i / kStages) & 1); ++n) {}
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer
         // The whole warp runs the loop (so that addresses and descriptors stay warp-uniform); one elected
@@ -329,30 +366,12 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         const uint64_t desc0 = operand_desc<BK_>(smem_u32(tiles));
         int it = 0, t = 0;
         bool ok = true, ready = false;                           // ready: the next K block's barrier was seen complete
-        // Which sign planes a tile's rows use at all (bits of the row words, OR-ed over the tile's 128 + 256
-        // rows): the products with a plane that is zero for the whole tile are not issued.  The words of the
-        // next tile are fetched while the current one runs.
-        auto tile_sides = [&](int64_t tile) {
-            int bits = 0;
-            if (tile < total_tiles) {
-                const int64_t m0 = blk_m(tile) * BM, n0 = blk_n(tile) * BNT;
-                const int* w_words = p.w_exp;
-#pragma unroll
-                for (int i = 0; i < BM / 32; ++i)
-                    if (m0 + i * 32 + lane < p.M) bits |= (__ldg(p.a_exp + m0 + i * 32 + lane) >> 16) & 3;
-#pragma unroll
-                for (int i = 0; i < BNT / 32; ++i)
-                    if (n0 + i * 32 + lane < p.N) bits |= ((__ldg(w_words + n0 + i * 32 + lane) >> 16) & 3) << 2;
-            }
-            return bits;
-        };
+        // (the planes of a tile: tile_sides above; the words of the next tile are fetched while the current one runs)
         int sides_next = tile_sides(blockIdx.x);
         for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-            int sides = __reduce_or_sync(0xFFFFFFFFu, sides_next);   // bit 0/1: A has +/-, bit 2/3: W has +/-
+            const int sides = whole_sides(sides_next);           // an all-zero operand: one product, which zeroes the tile
             sides_next = tile_sides(tile + gridDim.x);
             const int nkb = nkb_of(tile);
-            if (!(sides & 3)) sides |= 1;                        // an all-zero operand: one product, which zeroes the tile
-            if (!(sides & 12)) sides |= 4;
             const int n_mma = ((sides & 1) + ((sides >> 1) & 1)) * (((sides >> 2) & 1) + ((sides >> 3) & 1)) * kSteps;
             // the previous tile's accumulator must have been read out before it is overwritten
             if (t > 0) ok = mbar_wait(&ctl->accum_empty, (t - 1) & 1, &ctl->abort, p.status);
@@ -570,15 +589,17 @@ int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, co
             return AMX_ERR_CUDA;
         configured[dev] = true;
     }
-    CUtensorMap tm_a, tm_w;
-    if (!make_map(&tm_a, pa, a_rows, p.K, oa.plane, BM, C_::kRowBytes) || !make_map(&tm_w, pw, w_rows, p.K, ow.plane, BNT, C_::kRowBytes))
+    CUtensorMap tm_a, tm_w, tm_a1, tm_w1;                       // both planes of a tile in one box, and one plane alone
+    if (!make_map(&tm_a, pa, a_rows, p.K, oa.plane, BM, C_::kRowBytes) || !make_map(&tm_w, pw, w_rows, p.K, ow.plane, BNT, C_::kRowBytes) ||
+        !make_map(&tm_a1, pa, a_rows, p.K, oa.plane, BM, C_::kRowBytes, 1) ||
+        !make_map(&tm_w1, pw, w_rows, p.K, ow.plane, BNT, C_::kRowBytes, 1))
         return AMX_ERR_CUDA;
     static int sm_count[64] = {};
     if (!sm_count[dev] && cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return AMX_ERR_CUDA;
     const int64_t tiles = ((p.N + BNT - 1) / BNT) * ((p.M + BM - 1) / BM) * (SLICED ? p.slices : 1);
     const unsigned grid = (unsigned)(tiles < sm_count[dev] ? tiles : sm_count[dev]);   // one persistent CTA per SM
-    gemm_fp4_kernel<BK_, SLICED, NHALF><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_a, tm_w, p);
+    gemm_fp4_kernel<BK_, SLICED, NHALF><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_a, tm_w, tm_a1, tm_w1, p);
     return launch_status();
 }
 
