@@ -68,8 +68,10 @@ constexpr int kMaxStages = 4;
 
 struct __align__(16) Control {
     uint64_t full[kMaxStages], empty[kMaxStages], accum_full, accum_empty;
+    uint64_t sides_ready[2];        // the epilogue warps have written sides[i] for the CTA's tile number 2 k + i
     uint32_t tmem_base;
     volatile int abort;
+    volatile int sides[2][8];       // per epilogue warp: which sign planes its share of the tile's rows uses
     alignas(16) int w_exp[2][BN];   // read as int4 in the epilogue
 };
 static_assert(sizeof(Control) <= 2048 + 256, "Control must fit its reserved space");
@@ -287,6 +289,8 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         }
         mbar_init(&ctl->accum_full, 1);
         mbar_init(&ctl->accum_empty, kEpilogueWarps);
+        mbar_init(&ctl->sides_ready[0], kEpilogueWarps);
+        mbar_init(&ctl->sides_ready[1], kEpilogueWarps);
         ctl->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -322,19 +326,25 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 
     if (warp == 0) {
         // -------------------------------------------------------------- TMA producer
-        // The whole warp finds the tile's planes; one lane waits and issues.
-        constexpr int kTileWT = NHALF ? C_::kTileB / 2 : C_::kTileB;   // one plane of the W tile as loaded
-        int it = 0;                                                  // K blocks issued so far, over all tiles
-        bool ok = true;
-        int sides_next = tile_sides(blockIdx.x);
-        for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-            const int sides = whole_sides(sides_next);
-            sides_next = tile_sides(tile + gridDim.x);
-            const int64_t m_blk = blk_m(tile), n_blk = blk_n(tile);
-            const int kb0 = kb_begin(tile), nkb = nkb_of(tile);
-            const int a_planes = sides & 3, w_planes = (sides >> 2) & 3;
-            const uint32_t bytes = (a_planes == 3 ? 2 : 1) * C_::kTileA + (w_planes == 3 ? 2 : 1) * kTileWT;
-            if (lane == 0) {
+        // Which planes of a tile are not zero comes from the epilogue warps, which read the tile's row words a tile
+        // ahead anyway (sides[] in the control block): nothing on this lane's path but a barrier that has long
+        // completed and eight shared-memory words.
+        if (lane == 0) {
+            constexpr int kTileWT = NHALF ? C_::kTileB / 2 : C_::kTileB;   // one plane of the W tile as loaded
+            int it = 0, j = 0;                                   // K blocks issued so far over all tiles; tiles so far
+            bool ok = true;
+            for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++j) {
+                if (!mbar_wait(&ctl->sides_ready[j & 1], (j >> 1) & 1, &ctl->abort, p.status)) break;
+                int sides = 0;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) sides |= ctl->sides[j & 1][i];
+                if (!(sides & 3)) sides |= 1;                    // as the MMA warp: an all-zero operand keeps one plane
+                if (!(sides & 12)) sides |= 4;
+                const int a_planes = sides & 3, w_planes = (sides >> 2) & 3;
+                const uint32_t bytes = (a_planes == 3 ? 2 : 1) * C_::kTileA + (w_planes == 3 ? 2 : 1) * kTileWT;
+                const int64_t m_blk = blk_m(tile), n_blk = blk_n(tile);
+                const int kb0 = kb_begin(tile), nkb = nkb_of(tile);
+                const int ya = (int)(p.a_row0 + m_blk * BM), yw = (int)(p.w_row0 + n_blk * BNT);
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % kStages;
                     if (it >= kStages && !mbar_wait(&ctl->empty[s], ((it / kStages) - 1) & 1, &ctl->abort, p.status)) {
@@ -343,7 +353,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                     }
                     uint8_t* st = tiles + s * kStageBytes;
                     mbar_expect_tx(&ctl->full[s], bytes);
-                    const int x = (kb0 + kb) * kRowBytes, ya = (int)(p.a_row0 + m_blk * BM), yw = (int)(p.w_row0 + n_blk * BNT);
+                    const int x = (kb0 + kb) * kRowBytes;
                     // one 3-D tile per operand: {row bytes, rows, both sign planes} - or the one plane that is not zero
                     if (a_planes == 3) tma_load_3d(st + C_::kOffAp, &tm_a, x, ya, 0, &ctl->full[s]);
                     else tma_load_3d(st + (a_planes == 2 ? C_::kOffAn : C_::kOffAp), &tm_a1, x, ya, a_planes == 2 ? 1 : 0, &ctl->full[s]);
@@ -351,13 +361,11 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                     else tma_load_3d(st + (w_planes == 2 ? kOffWnT : C_::kOffWp), &tm_w1, x, yw, w_planes == 2 ? 1 : 0, &ctl->full[s]);
                 }
             }
-            it = __shfl_sync(0xFFFFFFFFu, it, 0);
-            ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+            // after an abort: let the copies already in flight land before shared memory is released
+            if (ctl->abort)
+                for (int i = max(0, it - kStages); i < it; ++i)
+                    for (uint32_t n = 0; n < kSpinLimit && !mbar_try_wait(&ctl->full[i % kStages], (i / kStages) & 1); ++n) {}
         }
-        // after an abort: let the copies already in flight land before shared memory is released
-        if (lane == 0 && ctl->abort)
-            for (int i = max(0, it - kStages); i < it; ++i)
-                for (uint32_t n = 0; n < kSpinLimit && !mbar_try_wait(&ctl->full[i % kStages], (i / kStages) & 1); ++n) {}
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer
         // The whole warp runs the loop (so that addresses and descriptors stay warp-uniform); one elected
@@ -486,24 +494,44 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         // The per-tile constants (this thread's column offset and row offset) are fetched one tile ahead, so that
         // their latency is off the path between two tiles.
         struct TileConsts {
-            int w_ex, a_ex;
+            int w_ex, a_ex, planes;     // planes: bit 0/1 this thread's row of A has +/-, bit 2/3 its row of W has
         };
         auto load_consts = [&](int64_t tl) {
-            TileConsts c = {0, 0};
+            TileConsts c = {0, 0, 0};
             if (tl < total_tiles) {
                 const int64_t n = blk_n(tl) * BNT + tid_e, mm = blk_m(tl) * BM + q * 32 + lane;
-                if (tid_e < BNT && n < p.N) c.w_ex = row_word_exp(__ldg(p.w_exp + n));
-                if (mm < p.M) c.a_ex = row_word_exp(__ldg(p.a_exp + mm));
+                if (tid_e < BNT && n < p.N) {
+                    const int w = __ldg(p.w_exp + n);
+                    c.w_ex = row_word_exp(w);
+                    c.planes |= ((w >> 16) & 3) << 2;
+                }
+                if (mm < p.M) {
+                    const int w = __ldg(p.a_exp + mm);
+                    c.a_ex = row_word_exp(w);
+                    c.planes |= (w >> 16) & 3;
+                }
             }
             return c;
+        };
+        // The eight warps' row words cover the tile's 128 + 256 rows: each tells the producer which planes its rows
+        // use (tile number j of this CTA); the producer reads them before the tile's first load.
+        auto publish = [&](const TileConsts& c, int64_t tl, int j) {
+            if (tl >= total_tiles) return;
+            const int bits = __reduce_or_sync(0xFFFFFFFFu, c.planes);
+            if (lane == 0) {
+                ctl->sides[j & 1][e] = bits;
+                mbar_arrive(&ctl->sides_ready[j & 1]);
+            }
         };
         const float out_scale = p.scale_a ? __ldg(p.scale_a) * __ldg(p.scale_w) : 1.0f;
         int64_t tile = blockIdx.x;
         TileConsts nxt = load_consts(tile);
+        publish(nxt, tile, 0);
         while (tile < total_tiles && ok) {
             const TileConsts cur = nxt;
             const int64_t tile_after = tile + gridDim.x;
             nxt = load_consts(tile_after);                       // in flight while this tile is worked on
+            publish(nxt, tile_after, t + 1);
             const int64_t m0 = blk_m(tile) * BM, n0 = blk_n(tile) * BNT;
             float* const C_item = p.C + (SLICED ? (tile % S) * p.slice_stride : 0);
             int* w_exp = ctl->w_exp[t & 1];
