@@ -630,7 +630,23 @@ def run_ours(args):
         quant_large = {"shape": [qr, qk], "us": q_us, "gb_per_s": gbs,
                        "pct_of_nominal_hbm_8TBs": 100.0 * gbs / NOMINAL_HBM_GBS,
                        "frac_of_measured_copy": gbs / peaks["hbm_gbs"]}
-        del xq, qc, qs
+        # the same tensor through the cast that writes the GEMM-ready operand (alone on the GPU, not beside a second cast)
+        qp = torch.empty(L.amx_prepared_bytes(qr, qk, GS, 0), dtype=torch.uint8, device="cuda")
+
+        def cast_prepared():
+            check(L.amx_quantize_prepared(xq.data_ptr(), qr, qk, GS, 0, None, qs.data_ptr(), qp.data_ptr(), qp.numel(), stream))
+        for _ in range(3):
+            cast_prepared()
+        torch.cuda.synchronize()
+        q0.record()
+        for _ in range(q_iters):
+            cast_prepared()
+        q1.record()
+        torch.cuda.synchronize()
+        qp_us = q0.elapsed_time(q1) * 1e3 / q_iters
+        qp_gbs = qr * qk * MOVED_BYTES_PER_ELEM / (qp_us * 1e-6) / 1e9
+        quant_large["prepared"] = {"us": qp_us, "gb_per_s_moved": qp_gbs, "frac_of_measured_copy": qp_gbs / peaks["hbm_gbs"]}
+        del xq, qc, qs, qp
 
     # ---- config 5: fully quantized attention for all heads (32 x 8192 x 128), one call of amx_attention
     attention = None
@@ -773,6 +789,12 @@ def run_ours(args):
                                                             "phase); bytes actually moved per element: 2 read, 1 of sign "
                                                             "planes, 0.0625 of scale bytes, 0.125 of scale factors (the "
                                                             "canonical codes are not written)"},
+                                  "prepared_cast_alone": (None if quant_large is None else
+                                                          {"bytes_per_element": moved,
+                                                           "achieved": quant_large["prepared"]["gb_per_s_moved"],
+                                                           "frac": quant_large["prepared"]["frac_of_measured_copy"],
+                                                           "what": "amx_quantize_prepared on 16384 x 8192 with nothing else "
+                                                                   "running (in the step two casts share the GPU)"}),
                                   "plain_cast": (None if quant_large is None else
                                                  {"bytes_per_element": BYTES_PER_ELEM, "achieved": quant_large["gb_per_s"],
                                                   "frac": quant_large["frac_of_measured_copy"],
