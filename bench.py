@@ -383,23 +383,26 @@ def run_ours(args):
         if rc != 0:
             raise RuntimeError(amx.status_string(rc))
 
+    # --format: the step in one of the symmetric comparison formats (profiling aid; the bench line is AMXFP4)
+    step_fmt = {"amxfp4": amx.FMT_AMXFP4, "sym_fp8": amx.FMT_SYM_FP8, "mxfp4": amx.FMT_MXFP4}[args.format]
+
     def cast_a(li, st):
         K, N = layers[li]
         b = bufs[li]
         if fused_prepare:   # the cast writes the FP4 kernel's operand (sign planes, scale factors) in the same pass
-            check(L.amx_quantize_prepared(A[li].data_ptr(), M, K, GS, 0, None, b["as"].data_ptr(),
-                                          b["pa"].data_ptr(), b["pa"].numel(), st))
+            check(L.amx_quantize_prepared_fmt(A[li].data_ptr(), M, K, GS, 0, step_fmt, None, b["as"].data_ptr(),
+                                              b["pa"].data_ptr(), b["pa"].numel(), st))
         else:
-            check(L.amx_quantize(A[li].data_ptr(), M, K, K, GS, b["ac"].data_ptr(), b["as"].data_ptr(), st))
+            check(L.amx_quantize_fmt(A[li].data_ptr(), M, K, K, GS, step_fmt, b["ac"].data_ptr(), b["as"].data_ptr(), st))
 
     def cast_w(li, st):
         K, N = layers[li]
         b = bufs[li]
         if fused_prepare:
-            check(L.amx_quantize_prepared(W[li].data_ptr(), N, K, GS, 1, None, b["ws"].data_ptr(),
-                                          b["pw"].data_ptr(), b["pw"].numel(), st))
+            check(L.amx_quantize_prepared_fmt(W[li].data_ptr(), N, K, GS, 1, step_fmt, None, b["ws"].data_ptr(),
+                                              b["pw"].data_ptr(), b["pw"].numel(), st))
         else:
-            check(L.amx_quantize(W[li].data_ptr(), N, K, K, GS, b["wc"].data_ptr(), b["ws"].data_ptr(), st))
+            check(L.amx_quantize_fmt(W[li].data_ptr(), N, K, K, GS, step_fmt, b["wc"].data_ptr(), b["ws"].data_ptr(), st))
 
     def gemm(li, st):
         K, N = layers[li]
@@ -754,7 +757,8 @@ def run_ours(args):
         "steps": args.steps, "warmup": warmup, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp4xfp4->f32",
         "data": "synthetic",
-        "config": {"workload": (WORKLOADS[CONFIG] + "; activations and weights both cast to AMXFP4 every step, then GEMM"),
+        "config": {"workload": (WORKLOADS[CONFIG] + "; activations and weights both cast to AMXFP4 every step, then GEMM"
+                                + ("" if args.format == "amxfp4" else f" [comparison format {args.format} instead of AMXFP4]")),
                    "group_size": GS, "gemm_kernel": gemm_kernel,
                    "entry_points": "amx_quantize_prepared + amx_gemm_prepared" if fused_prepare else "amx_quantize + amx_gemm",
                    "l2": f"per-step inputs (~{int(elems_step * 2 / 1e6)} MB of bf16) exceed the 126 MB L2",
@@ -838,6 +842,8 @@ def main():
                          "overlap: weight casts on a second stream, running ahead of the GEMMs")
     ap.add_argument("--graph", action="store_true", help="time replays of a CUDA graph of one step (the default for config 2)")
     ap.add_argument("--no-graph", action="store_true", help="config 2: time plain launches instead of the graph")
+    ap.add_argument("--format", default="amxfp4", choices=["amxfp4", "sym_fp8", "mxfp4"],
+                    help="cast format of the step (profiling aid: the symmetric comparison formats need one FP4 product per tile pair)")
     ap.add_argument("--layers", default="", help="comma-separated layer indices to run (profiling aid; default all)")
     ap.add_argument("--skip-extras", action="store_true", help="skip the e2e and cpu_baseline legs (profiling aid)")
     ap.add_argument("--attention-only", action="store_true", help="time only the config-5 attention call (profiling aid)")
