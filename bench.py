@@ -404,12 +404,13 @@ def run_ours(args):
         else:
             check(L.amx_quantize_fmt(W[li].data_ptr(), N, K, K, GS, step_fmt, b["wc"].data_ptr(), b["ws"].data_ptr(), st))
 
-    def gemm(li, st):
+    def gemm(li, st, sym=step_fmt != amx.FMT_AMXFP4):
         K, N = layers[li]
         b = bufs[li]
-        if fused_prepare:
-            check(L.amx_gemm_prepared(b["pa"].data_ptr(), b["pw"].data_ptr(), M, N, K, GS, b["c"].data_ptr(), N,
-                                      b["work"].data_ptr(), b["work"].numel(), st))
+        if fused_prepare:      # sym: both operands are single planes, the one-plane pipeline of the same kernel
+            fn = L.amx_gemm_prepared_sym if sym else L.amx_gemm_prepared
+            check(fn(b["pa"].data_ptr(), b["pw"].data_ptr(), M, N, K, GS, b["c"].data_ptr(), N,
+                     b["work"].data_ptr(), b["work"].numel(), st))
         else:
             check(L.amx_gemm(b["ac"].data_ptr(), b["as"].data_ptr(), b["wc"].data_ptr(), b["ws"].data_ptr(),
                              M, N, K, GS, gemm_flag, b["c"].data_ptr(), N, b["work"].data_ptr(), b["work"].numel(), st))
@@ -561,7 +562,7 @@ def run_ours(args):
     if fused_prepare and not args.layers and not args.skip_extras:
         format_variants = {}
         for name, fmt in (("sym_fp8", 1), ("mxfp4", 2)):
-            def fmt_step(st, with_casts=True, fmt=fmt):
+            def fmt_step(st, with_casts=True, fmt=fmt, sym=True):
                 for li, (K, N) in enumerate(layers):
                     b = bufs[li]
                     if with_casts:
@@ -569,14 +570,17 @@ def run_ours(args):
                                                           b["as"].data_ptr(), b["pa"].data_ptr(), b["pa"].numel(), st))
                         check(L.amx_quantize_prepared_fmt(W[li].data_ptr(), N, K, GS, 1, fmt, None,
                                                           b["ws"].data_ptr(), b["pw"].data_ptr(), b["pw"].numel(), st))
-                    gemm(li, st)
+                    gemm(li, st, sym)
             res = {}
-            for key, with_casts in (("step", True), ("gemm", False)):
+            for key, with_casts, sym in (("step", True, True), ("gemm", False, True), ("gemm_general_kernel", False, False)):
                 fmt_step(stream)
-                v_ms = timed_graph(lambda st: fmt_step(st, with_casts), extra_steps)
+                v_ms = timed_graph(lambda st: fmt_step(st, with_casts, sym=sym), extra_steps)
                 res[key + "_tflops"] = flops_step / (v_ms * 1e-3) / 1e12
                 res[key + "_ms"] = v_ms
             format_variants[name] = res
+            for li in range(len(layers)):                        # the one-plane promise held, no wait expired
+                if amx.gemm_status(bufs[li]["work"]) != 0:
+                    raise RuntimeError(f"{name}, layer {layer_ids[li]}: GEMM status {amx.status_string(amx.gemm_status(bufs[li]['work']))}")
         # NVFP4 / ANVFP4 (group 16, E4M3 group scales + fp32 tensor scale: Section 5's comparison format): the scale
         # bytes are the tensor cores' native type, NVFP4 is one product per tile pair, ANVFP4 four
         nv = []
@@ -594,8 +598,8 @@ def run_ours(args):
                                                    pa.numel(), st))
                         check(L.amx_quantize_nvfp4(W[li].data_ptr(), N, K, K, flag, None, None, tw.data_ptr(), 1, pw.data_ptr(),
                                                    pw.numel(), st))
-                    check(L.amx_gemm_nvfp4(pa.data_ptr(), pw.data_ptr(), M, N, K, b["c"].data_ptr(), N, b["work"].data_ptr(),
-                                           b["work"].numel(), st))
+                    check((L.amx_gemm_nvfp4 if flag else L.amx_gemm_nvfp4_sym)(
+                        pa.data_ptr(), pw.data_ptr(), M, N, K, b["c"].data_ptr(), N, b["work"].data_ptr(), b["work"].numel(), st))
             res = {}
             for key, with_casts in (("step", True), ("gemm", False)):
                 nv_step(stream)
@@ -603,11 +607,16 @@ def run_ours(args):
                 res[key + "_tflops"] = flops_step / (v_ms * 1e-3) / 1e12
                 res[key + "_ms"] = v_ms
             format_variants[name] = res
+            for li in range(len(layers)):                        # the one-plane promise held, no wait expired
+                if amx.gemm_status(bufs[li]["work"]) != 0:
+                    raise RuntimeError(f"{name}, layer {layer_ids[li]}: GEMM status {amx.status_string(amx.gemm_status(bufs[li]['work']))}")
         del nv
         format_variants["what"] = ("same workload and GEMM kernel with other formats: sym_fp8 / mxfp4 = the paper's symmetric "
                                    "comparison formats (amx_quantize_prepared_fmt), nvfp4 / anvfp4 = group 16 with E4M3 scales "
                                    "and a tensor scale (amx_quantize_nvfp4: two launches, the tensor maximum first); step = "
-                                   "casts of both operands + GEMMs, gemm = the GEMMs alone")
+                                   "casts of both operands + GEMMs, gemm = the GEMMs alone; the symmetric formats run the "
+                                   "one-plane pipeline (amx_gemm_prepared_sym, amx_gemm_nvfp4_sym), gemm_general_kernel = "
+                                   "the same operands through amx_gemm_prepared")
         run_step()                      # leave the buffers as the headline step writes them
         torch.cuda.synchronize()
 

@@ -216,6 +216,17 @@ size_t amx_gemm_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K, int gr
 int amx_gemm_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
                       int group_size, float* C, int64_t ld_c, void* workspace, size_t workspace_bytes,
                       void* stream);
+/* amx_gemm_prepared for two operands that the caller knows to be single planes: each prepared in a symmetric
+ * format (AMX_FMT_SYM_FP8 or AMX_FMT_MXFP4 through amx_quantize_prepared_fmt; any canonical operand whose two
+ * scales agree in every group through amx_prepare), or with all its values non-negative.  Same arguments and result.  With one product per K step the tensor cores wait for the operand loads, so this form
+ * keeps twice as many K blocks in flight, in the shared memory the second planes would have taken.  The promise
+ * is checked on the device, per output tile, against the operands' row words: if a tile has a second plane,
+ * amx_gemm_status(workspace) returns AMX_ERR_FLAGS and C is not the product (the kernel still runs to its end
+ * and touches nothing outside C).  Products narrower than 129 columns, or cut into K ranges, run the general
+ * kernel, where the promise changes nothing. */
+int amx_gemm_prepared_sym(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
+                          int group_size, float* C, int64_t ld_c, void* workspace, size_t workspace_bytes,
+                          void* stream);
 
 /*
  * amx_quant_gemm - the fully quantized linear layer of Section 5 ("quantize input operands for
@@ -396,6 +407,10 @@ int amx_dequantize_nvfp4(const uint8_t* codes, const uint8_t* scales, const floa
                          uint32_t flags, void* out, int64_t ld_out, void* stream);
 int amx_gemm_nvfp4(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K, float* C,
                    int64_t ld_c, void* workspace, size_t workspace_bytes, void* stream);
+/* The same for two operands cast without AMX_NV_ASYMMETRIC (see amx_gemm_prepared_sym: the deeper one-plane
+ * pipeline, AMX_ERR_FLAGS in the status word if an operand has a second plane after all). */
+int amx_gemm_nvfp4_sym(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K, float* C,
+                       int64_t ld_c, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * FP4 with binary16 shared scales - the "FP16" row of the paper's ablation of the shared-scale encoding (appendix
@@ -460,7 +475,7 @@ uint32_t amx_gemm_kernel_for(int64_t M, int64_t N, int64_t K, int group_size, ui
  * Status word of the most recent amx_gemm / amx_quant_gemm / amx_gemm_prepared that used `workspace` (its
  * first word, for every kernel that takes a workspace): AMX_OK, or AMX_ERR_TIMEOUT when a bounded wait inside
  * a tensor-core kernel expired (the kernel then stopped issuing work, released its resources and returned; C is
- * not valid).  The weight-streaming kernel has no such wait and always leaves AMX_OK.  Synchronises `stream`.
+ * not valid), or AMX_ERR_FLAGS after amx_gemm_prepared_sym / amx_gemm_nvfp4_sym on an operand with two planes.  The weight-streaming kernel has no such wait and always leaves AMX_OK.  Synchronises `stream`.
  */
 int amx_gemm_status(const void* workspace, void* stream);
 

@@ -41,6 +41,7 @@ SYMBOLS = (
     "amx_quantize_nvfp4", "amx_nvfp4_prepared_bytes", "amx_dequantize_nvfp4", "amx_gemm_nvfp4",
     "amx_quantize_f16s", "amx_dequantize_f16s", "amx_gemm_f16s", "amx_quant_error_f16s",
     "amx_fake_quantize", "amx_attention_workspace_bytes_for", "amx_attention_gqa",
+    "amx_gemm_prepared_sym", "amx_gemm_nvfp4_sym",
 )
 
 
@@ -77,6 +78,7 @@ def lib() -> ctypes.CDLL:
         L.amx_nvfp4_prepared_bytes.restype = sz
         L.amx_dequantize_nvfp4.argtypes = [p, p, p, i64, i64, u32, p, i64, p]
         L.amx_gemm_nvfp4.argtypes = [p, p, i64, i64, i64, p, i64, p, sz, p]
+        L.amx_gemm_nvfp4_sym.argtypes = [p, p, i64, i64, i64, p, i64, p, sz, p]
         L.amx_quantize_f16s.argtypes = [p, i64, i64, i64, i, u32, p, p, p]
         L.amx_fake_quantize.argtypes = [p, i64, i64, i64, i, i, p, i64, p]
         L.amx_dequantize_f16s.argtypes = [p, p, i64, i64, i, p, i64, p]
@@ -96,6 +98,7 @@ def lib() -> ctypes.CDLL:
         L.amx_prepare.argtypes = [p, p, i64, i64, i, i, p, sz, p]
         L.amx_quantize_prepared.argtypes = [p, i64, i64, i, i, p, p, p, sz, p]
         L.amx_gemm_prepared.argtypes = [p, p, i64, i64, i64, i, p, i64, p, sz, p]
+        L.amx_gemm_prepared_sym.argtypes = [p, p, i64, i64, i64, i, p, i64, p, sz, p]
         L.amx_gemm_prepared_workspace_bytes.argtypes = [i64, i64, i64, i]
         L.amx_gemm_prepared_workspace_bytes.restype = sz
         L.amx_softmax_bf16.argtypes = [p, i64, i64, i64, ctypes.c_float, p, i64, p]
@@ -255,13 +258,15 @@ def quantize_prepared(x: torch.Tensor, is_weight: bool, group_size: int = 32, pr
 
 
 def gemm_prepared(a_prepared: torch.Tensor, w_prepared: torch.Tensor, M: int, N: int, K: int, group_size: int = 32,
-                  out: torch.Tensor | None = None, workspace: torch.Tensor | None = None):
+                  out: torch.Tensor | None = None, workspace: torch.Tensor | None = None, sym: bool = False):
+    """sym: both operands are in a symmetric format (amx_gemm_prepared_sym; a violated promise shows in gemm_status)."""
     if out is None:
         out = torch.empty((M, N), dtype=torch.float32, device=a_prepared.device)
     if workspace is None:
         workspace = _ws(lib().amx_gemm_prepared_workspace_bytes(M, N, K, group_size), a_prepared.device)
-    _check(lib().amx_gemm_prepared(a_prepared.data_ptr(), w_prepared.data_ptr(), M, N, K, group_size, out.data_ptr(),
-                                   out.stride(0), workspace.data_ptr(), workspace.numel(), _stream()), "amx_gemm_prepared")
+    fn = lib().amx_gemm_prepared_sym if sym else lib().amx_gemm_prepared
+    _check(fn(a_prepared.data_ptr(), w_prepared.data_ptr(), M, N, K, group_size, out.data_ptr(),
+              out.stride(0), workspace.data_ptr(), workspace.numel(), _stream()), "amx_gemm_prepared")
     return out
 
 
@@ -379,12 +384,14 @@ def dequantize_nvfp4(codes: torch.Tensor, scales: torch.Tensor, ts: torch.Tensor
     return out
 
 
-def gemm_nvfp4(a_prepared: torch.Tensor, w_prepared: torch.Tensor, M: int, N: int, K: int, workspace: torch.Tensor | None = None):
+def gemm_nvfp4(a_prepared: torch.Tensor, w_prepared: torch.Tensor, M: int, N: int, K: int, workspace: torch.Tensor | None = None,
+               sym: bool = False):
     out = torch.empty((M, N), dtype=torch.float32, device=a_prepared.device)
     if workspace is None:
         workspace = _ws(256, a_prepared.device)
-    _check(lib().amx_gemm_nvfp4(a_prepared.data_ptr(), w_prepared.data_ptr(), M, N, K, out.data_ptr(), N, workspace.data_ptr(),
-                                workspace.numel(), _stream()), "amx_gemm_nvfp4")
+    fn = lib().amx_gemm_nvfp4_sym if sym else lib().amx_gemm_nvfp4
+    _check(fn(a_prepared.data_ptr(), w_prepared.data_ptr(), M, N, K, out.data_ptr(), N, workspace.data_ptr(),
+              workspace.numel(), _stream()), "amx_gemm_nvfp4")
     return out
 
 

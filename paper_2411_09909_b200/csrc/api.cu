@@ -183,6 +183,18 @@ extern "C" int amx_gemm_prepared(const void* a_prepared, const void* w_prepared,
                              workspace_bytes);
 }
 
+extern "C" int amx_gemm_prepared_sym(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
+                                     int group_size, float* C, int64_t ld_c, void* workspace, size_t workspace_bytes,
+                                     void* stream) {
+    if (M <= 0 || N <= 0 || !gemm_fp4_supported(M, N, K, group_size) || ld_c < N) return AMX_ERR_SHAPE;
+    if (!a_prepared || !w_prepared || !C) return AMX_ERR_NULL;
+    if (!workspace || workspace_bytes < 256) return AMX_ERR_WORKSPACE;
+    if (!aligned(a_prepared, kAlign) || !aligned(w_prepared, kAlign) || !aligned(workspace, kAlign) || !aligned(C, 4))
+        return AMX_ERR_ALIGN;
+    return gemm_fp4_prepared_at({a_prepared, M, M, 0}, {w_prepared, N, N, 0}, M, N, K, C, ld_c, workspace,
+                                static_cast<cudaStream_t>(stream), workspace_bytes, nullptr, nullptr, nullptr, true);
+}
+
 extern "C" int amx_quant_gemm(const void* A, int64_t ld_a, const uint8_t* w_codes, const uint8_t* w_scales,
                               const void* W_bf16, int64_t ld_w, int64_t M, int64_t N, int64_t K, int group_size,
                               uint32_t flags, float* C, int64_t ld_c, void* workspace, size_t workspace_bytes,

@@ -74,7 +74,10 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
                          int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes = 256,
                          const int* gate = nullptr /* device word: the kernel does nothing when it is nonzero */,
                          const float* scale_a = nullptr, const float* scale_w = nullptr /* device: one factor per
-                         operand; every result is multiplied by their product (NVFP4 tensor scales) */);
+                         operand; every result is multiplied by their product (NVFP4 tensor scales) */,
+                         bool one_plane = false /* the caller states that neither operand has a second sign plane:
+                         full-width tiles run the deeper one-plane pipeline, which reports AMX_ERR_FLAGS in the status
+                         word when a tile has a second plane after all */);
 // workspace that lets the kernel cut K into ranges for products with few output tiles (256 bytes otherwise)
 size_t gemm_fp4_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K);
 // C[m][n] = sum over `slices` partial products [slices][M][N], in slice order (defined with the bf16-decode kernel)

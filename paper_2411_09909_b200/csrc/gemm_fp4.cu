@@ -50,21 +50,26 @@ constexpr uint32_t kTmemSf = 256;      // scale-factor columns follow the 256 ac
 // Shared-memory stage geometry for a K block of BK elements (BK/2 bytes of codes per row and plane).
 // BK = 256: 128-byte rows, 128-byte swizzle, 2 stages of 96 KB.
 // BK = 128:  64-byte rows,  64-byte swizzle, 4 stages of 48 KB (finer-grained prefetch).
-template <int BK_>
+// ONE_PLANE (BK = 128): a stage holds one plane of each operand, 8 stages of 24 KB.  For two operands in a symmetric
+// format, whose one product per K step leaves the tensor pipe waiting for loads: twice as many K blocks in flight.
+template <int BK_, bool ONE_PLANE = false>
 struct Cfg {
     static constexpr int BK = BK_;
+    static constexpr int kPlanes = ONE_PLANE ? 1 : 2;
     static constexpr int kRowBytes = BK / 2;
     static constexpr int kSteps = BK / 64;                            // MMAs (K = 64) per K block and sign pair
-    static constexpr int kStages = BK == 256 ? 2 : 4;
+    static constexpr int kStages = (BK == 256 ? 2 : 4) * (ONE_PLANE ? 2 : 1);
     static constexpr int kTileA = BM * kRowBytes, kTileB = BN * kRowBytes;   // one plane
-    static constexpr int kOffAp = 0, kOffAn = kTileA, kOffWp = 2 * kTileA, kOffWn = 2 * kTileA + kTileB;
-    static constexpr int kStageBytes = 2 * kTileA + 2 * kTileB;       // {A+, A-} and {W+, W-}: one TMA each
+    static constexpr int kOffAp = 0, kOffAn = ONE_PLANE ? 0 : kTileA, kOffWp = kPlanes * kTileA,
+                         kOffWn = kOffWp + (ONE_PLANE ? 0 : kTileB);
+    static constexpr int kStageBytes = kPlanes * (kTileA + kTileB);   // {A+, A-} and {W+, W-}: one TMA each
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 2048 + 256;   // + alignment slack + Control
     // TMEM columns of one stage's scale factors: A planes (4 columns per K step), then W planes (8)
-    static constexpr int kSfColsA = 2 * kSteps * 4, kSfCols = kSfColsA + 2 * kSteps * 8;
+    static constexpr int kSfColsA = kPlanes * kSteps * 4, kSfCols = kSfColsA + kPlanes * kSteps * 8;
     static_assert(256 + kStages * kSfCols <= kTmemCols, "scale factors do not fit tensor memory");
+    static_assert(!ONE_PLANE || BK == 128, "the one-plane pipeline exists for 128-element K blocks");
 };
-constexpr int kMaxStages = 4;
+constexpr int kMaxStages = 8;
 
 struct __align__(16) Control {
     uint64_t full[kMaxStages], empty[kMaxStages], accum_full, accum_empty;
@@ -227,11 +232,15 @@ __device__ __forceinline__ void store_row16(float* out, const float (&f)[16], bo
 
 // NHALF: tiles of 128 x 128 for products with at most 128 columns: the W box, the MMA and the epilogue are half as
 // wide, the stage layout keeps its size.
-template <int BK_, bool SLICED = false, bool NHALF = false>
+// ONE_PLANE: the caller states that neither operand has a second sign plane (Cfg above): only the first planes and
+// their scale factors are read, one product per K step.  A tile whose row words show a second plane after all puts
+// AMX_ERR_FLAGS into the status word (the kernel runs to its end; C is then not the product).
+template <int BK_, bool SLICED = false, bool NHALF = false, bool ONE_PLANE = false>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
                 const __grid_constant__ CUtensorMap tm_a1, const __grid_constant__ CUtensorMap tm_w1, const Params p) {
-    using C_ = Cfg<BK_>;
+    using C_ = Cfg<BK_, ONE_PLANE>;
+    constexpr int kPlanes = C_::kPlanes;
     if (p.gate && *p.gate != 0) return;                          // uniform over the grid: nothing was set up yet
     constexpr int BNT = NHALF ? BN / 2 : BN;                     // tile width
     constexpr int kOffWnT = NHALF ? C_::kOffWp + C_::kTileB / 2 : C_::kOffWn;   // the box packs its two planes
@@ -334,12 +343,15 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             int it = 0, j = 0;                                   // K blocks issued so far over all tiles; tiles so far
             bool ok = true;
             for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++j) {
-                if (!mbar_wait(&ctl->sides_ready[j & 1], (j >> 1) & 1, &ctl->abort, p.status)) break;
-                int sides = 0;
+                int sides = 5;                                   // ONE_PLANE: the first plane of each operand, always
+                if (!ONE_PLANE) {
+                    if (!mbar_wait(&ctl->sides_ready[j & 1], (j >> 1) & 1, &ctl->abort, p.status)) break;
+                    sides = 0;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) sides |= ctl->sides[j & 1][i];
-                if (!(sides & 3)) sides |= 1;                    // as the MMA warp: an all-zero operand keeps one plane
-                if (!(sides & 12)) sides |= 4;
+                    for (int i = 0; i < 8; ++i) sides |= ctl->sides[j & 1][i];
+                    if (!(sides & 3)) sides |= 1;                // as the MMA warp: an all-zero operand keeps one plane
+                    if (!(sides & 12)) sides |= 4;
+                }
                 const int a_planes = sides & 3, w_planes = (sides >> 2) & 3;
                 const uint32_t bytes = (a_planes == 3 ? 2 : 1) * C_::kTileA + (w_planes == 3 ? 2 : 1) * kTileWT;
                 const int64_t m_blk = blk_m(tile), n_blk = blk_n(tile);
@@ -375,10 +387,10 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         int it = 0, t = 0;
         bool ok = true, ready = false;                           // ready: the next K block's barrier was seen complete
         // (the planes of a tile: tile_sides above; the words of the next tile are fetched while the current one runs)
-        int sides_next = tile_sides(blockIdx.x);
+        int sides_next = ONE_PLANE ? 0 : tile_sides(blockIdx.x);
         for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-            const int sides = whole_sides(sides_next);           // an all-zero operand: one product, which zeroes the tile
-            sides_next = tile_sides(tile + gridDim.x);
+            const int sides = ONE_PLANE ? 5 : whole_sides(sides_next);   // an all-zero operand: one product, which zeroes the tile
+            if (!ONE_PLANE) sides_next = tile_sides(tile + gridDim.x);
             const int nkb = nkb_of(tile);
             const int n_mma = ((sides & 1) + ((sides >> 1) & 1)) * (((sides >> 2) & 1) + ((sides >> 3) & 1)) * kSteps;
             // the previous tile's accumulator must have been read out before it is overwritten
@@ -400,9 +412,9 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 if (elect_one()) {
                     int idx = 0;                                 // MMAs issued so far in this K block
 #pragma unroll
-                    for (int pa = 0; pa < 2; ++pa)
+                    for (int pa = 0; pa < kPlanes; ++pa)
 #pragma unroll
-                        for (int pw = 0; pw < 2; ++pw)
+                        for (int pw = 0; pw < kPlanes; ++pw)
 #pragma unroll
                             for (int kk = 0; kk < kSteps; ++kk) {   // 64 elements = 32 bytes along the swizzled row
                                 if (((sides >> pa) & 1) && ((sides >> (2 + pw)) & 1)) {
@@ -435,12 +447,12 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         // scale factors are normally in place before the TMA tiles of the same stage land.
         // Two groups of four warps take alternate K blocks.
         const int q = warp & 3, group = (warp - 2) >> 2;
-        constexpr int kBlocks = 2 * kSteps * 3;                  // per K block: A (1) + W (2 row blocks), x planes x steps
+        constexpr int kBlocks = kPlanes * kSteps * 3;                  // per K block: A (1) + W (2 row blocks), x planes x steps
         uint4 sfv[kBlocks];
         auto fetch = [&](int64_t tile, int kb) {
             const int64_t m_blk = blk_m(tile), n_blk = blk_n(tile);
 #pragma unroll
-            for (int pl = 0; pl < 2; ++pl)
+            for (int pl = 0; pl < kPlanes; ++pl)
 #pragma unroll
                 for (int kk = 0; kk < kSteps; ++kk) {
                     const int64_t c = ((int64_t)kb_begin(tile) + kb) * kSteps + kk;
@@ -467,7 +479,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             tc_fence_after();
             const uint32_t sfa = tmem + ((uint32_t)(q * 32) << 16) + kTmemSf + s * C_::kSfCols, sfb = sfa + C_::kSfColsA;
 #pragma unroll
-            for (int i = 0; i < 2 * kSteps; ++i) {
+            for (int i = 0; i < kPlanes * kSteps; ++i) {
                 tmem_st4(sfa + i * 4, sfv[i * 3].x, sfv[i * 3].y, sfv[i * 3].z, sfv[i * 3].w);
                 tmem_st4(sfb + i * 8, sfv[i * 3 + 1].x, sfv[i * 3 + 1].y, sfv[i * 3 + 1].z, sfv[i * 3 + 1].w);
                 tmem_st4(sfb + i * 8 + 4, sfv[i * 3 + 2].x, sfv[i * 3 + 2].y, sfv[i * 3 + 2].z, sfv[i * 3 + 2].w);
@@ -518,6 +530,10 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         auto publish = [&](const TileConsts& c, int64_t tl, int j) {
             if (tl >= total_tiles) return;
             const int bits = __reduce_or_sync(0xFFFFFFFFu, c.planes);
+            if (ONE_PLANE) {                                     // nobody waits for the planes; a second one is an error
+                if (lane == 0 && (bits & 10)) atomicExch(p.status, (int)AMX_ERR_FLAGS);
+                return;
+            }
             if (lane == 0) {
                 ctl->sides[j & 1][e] = bits;
                 mbar_arrive(&ctl->sides_ready[j & 1]);
@@ -606,14 +622,14 @@ size_t gemm_fp4_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 
 namespace {
 
-template <int BK_, bool SLICED = false, bool NHALF = false>
+template <int BK_, bool SLICED = false, bool NHALF = false, bool ONE_PLANE = false>
 int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, const OperandLayout& ow, int64_t a_rows,
                int64_t w_rows, Params p, int dev, cudaStream_t st) {
-    using C_ = Cfg<BK_>;
+    using C_ = Cfg<BK_, ONE_PLANE>;
     constexpr int BNT = NHALF ? BN / 2 : BN;
     static bool configured[64] = {};
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(gemm_fp4_kernel<BK_, SLICED, NHALF>, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(gemm_fp4_kernel<BK_, SLICED, NHALF, ONE_PLANE>, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::kSmemBytes) != cudaSuccess)
             return AMX_ERR_CUDA;
         configured[dev] = true;
     }
@@ -627,7 +643,7 @@ int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, co
         return AMX_ERR_CUDA;
     const int64_t tiles = ((p.N + BNT - 1) / BNT) * ((p.M + BM - 1) / BM) * (SLICED ? p.slices : 1);
     const unsigned grid = (unsigned)(tiles < sm_count[dev] ? tiles : sm_count[dev]);   // one persistent CTA per SM
-    gemm_fp4_kernel<BK_, SLICED, NHALF><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_a, tm_w, tm_a1, tm_w1, p);
+    gemm_fp4_kernel<BK_, SLICED, NHALF, ONE_PLANE><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_a, tm_w, tm_a1, tm_w1, p);
     return launch_status();
 }
 
@@ -699,7 +715,7 @@ size_t gemm_fp4_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 // workspace_bytes >= gemm_fp4_prepared_workspace_bytes() enables the K ranges; 256 bytes always suffice.
 int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
                          int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes, const int* gate,
-                         const float* scale_a, const float* scale_w) {
+                         const float* scale_a, const float* scale_w, bool one_plane) {
     Params p;
     OperandLayout oa, ow;
     int dev;
@@ -724,6 +740,9 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
         return r2 != AMX_OK ? r2 : reduce_slices(part, slices, M, N, C, ld_c, st);
     }
     if (fp4_block_k() == 256) return launch_fp4<256>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
+    // both operands stated to be single planes: the deeper pipeline (full-width tiles; the other shapes are short
+    // products, where the depth does not matter, and run the general kernel, which skips absent planes by itself)
+    if (one_plane && !half) return launch_fp4<128, false, false, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
     return half ? launch_fp4<128, false, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st)
                 : launch_fp4<128>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
 }

@@ -228,8 +228,9 @@ extern "C" int amx_dequantize_nvfp4(const uint8_t* codes, const uint8_t* scales,
     return launch_status();
 }
 
-extern "C" int amx_gemm_nvfp4(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K, float* C,
-                              int64_t ld_c, void* workspace, size_t workspace_bytes, void* stream) {
+namespace {
+int gemm_nvfp4(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K, float* C, int64_t ld_c,
+               void* workspace, size_t workspace_bytes, void* stream, bool one_plane) {
     if (M <= 0 || N <= 0 || K <= 0 || K % 64 || ld_c < N || !gemm_fp4_supported(M, N, K, 32)) return AMX_ERR_SHAPE;
     if (!a_prepared || !w_prepared || !C) return AMX_ERR_NULL;
     if (!workspace || workspace_bytes < 256) return AMX_ERR_WORKSPACE;
@@ -237,5 +238,15 @@ extern "C" int amx_gemm_nvfp4(const void* a_prepared, const void* w_prepared, in
     const float* sa = reinterpret_cast<const float*>(static_cast<const uint8_t*>(a_prepared) + fp4::operand_layout(M, K, 128).total);
     const float* sw = reinterpret_cast<const float*>(static_cast<const uint8_t*>(w_prepared) + fp4::operand_layout(N, K, 256).total);
     return gemm_fp4_prepared_at({a_prepared, M, M, 0}, {w_prepared, N, N, 0}, M, N, K, C, ld_c, workspace,
-                                static_cast<cudaStream_t>(stream), 256, nullptr, sa, sw);
+                                static_cast<cudaStream_t>(stream), 256, nullptr, sa, sw, one_plane);
+}
+}  // namespace
+
+extern "C" int amx_gemm_nvfp4(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K, float* C,
+                              int64_t ld_c, void* workspace, size_t workspace_bytes, void* stream) {
+    return gemm_nvfp4(a_prepared, w_prepared, M, N, K, C, ld_c, workspace, workspace_bytes, stream, false);
+}
+extern "C" int amx_gemm_nvfp4_sym(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K, float* C,
+                                  int64_t ld_c, void* workspace, size_t workspace_bytes, void* stream) {
+    return gemm_nvfp4(a_prepared, w_prepared, M, N, K, C, ld_c, workspace, workspace_bytes, stream, true);
 }
