@@ -15,8 +15,8 @@
 // and are flushed to zero: their groups contribute less than 2^-14 of the row's largest group.
 //
 // Persistent CTAs (one per SM) walk over 128 x 256 tiles of C; K blocks of 128 elements cycle through
-// four 54 KB shared-memory stages (two 108 KB stages with 256-element blocks):
-//   warp 0   TMA producer: per stage one 3-D tile {A+, A-} and one {W+, W-} (64- or 128-byte swizzle),
+// four 48 KB shared-memory stages:
+//   warp 0   TMA producer: per stage one 3-D tile {A+, A-} and one {W+, W-} (64-byte swizzle),
 //            completion on the stage's `full` mbarrier
 //   warp 1   allocates TMEM; one lane issues the stage's MMAs (4 sign pairs x K steps of 64), then
 //            commits to the stage's `empty` mbarrier
@@ -25,7 +25,8 @@
 //            `full` barriers and so run ahead into the next tile
 //   warps 10-17 epilogue: TMEM -> registers (double-buffered loads), power-of-two rescale, 32-byte fp32
 //            stores.  While a tile's accumulator is read out the producer already prefetches the next
-//            tile's stages; the MMA issuer waits for `accum_empty`.
+//            tile's stages, and the MMA issuer starts the next tile as soon as the columns the two tiles
+//            share have been read (see "Tensor memory" below).
 // A preparation kernel per operand derives the planes, the UE4M3 scale-factor
 // blocks in the 128 x 4 interleaved layout the MMA reads, and the row offsets from the canonical
 // codes and scales.  Every device-side wait is bounded.
@@ -45,11 +46,19 @@ constexpr int BM = 128, BN = 256;
 constexpr int kSfGroups = 2, kSfWarps = 4 * kSfGroups, kEpilogueWarps = 8;
 constexpr int kThreads = (2 + kSfWarps + kEpilogueWarps) * 32;
 constexpr int kTmemCols = 512;
-constexpr uint32_t kTmemSf = 256;      // scale-factor columns follow the 256 accumulator columns
+// Tensor memory.  Two fp32 accumulators of 256 columns are all 512 columns, and the block-scaled MMA reads its
+// scale factors from tensor memory too.  So consecutive tiles of a CTA alternate between two accumulator windows
+// that overlap: columns [0, 256) for its even tiles, [160, 416) for the odd ones; the scale factors of the K blocks
+// in flight take the 96 columns from 416.  The epilogue reads the 96 shared columns of a finished tile first and
+// releases them (`ovl_free`); the next tile's MMAs start then, while the other 160 columns are still being read
+// and stored (`rest_free` guards their reuse by the tile after next).  Only the read of 96 of 256 columns stays
+// between two tiles, instead of the whole drain.  (Tiles of 128 columns use [0, 128) and [160, 288): no overlap.)
+constexpr int kAccWindow = 160;        // first column of the odd tiles' accumulator
+constexpr uint32_t kTmemSf = 416;      // scale-factor columns
+constexpr int kTmemSfCols = 96;
 
-// Shared-memory stage geometry for a K block of BK elements (BK/2 bytes of codes per row and plane).
-// BK = 256: 128-byte rows, 128-byte swizzle, 2 stages of 96 KB.
-// BK = 128:  64-byte rows,  64-byte swizzle, 4 stages of 48 KB (finer-grained prefetch).
+// Shared-memory stage geometry for a K block of BK = 128 elements (BK/2 = 64 bytes of codes per row and plane,
+// 64-byte swizzle): 4 stages of 48 KB.  (K blocks of 256 elements in two 96 KB stages measured slower.)
 // ONE_PLANE (BK = 128): a stage holds one plane of each operand, 8 stages of 24 KB.  For two operands in a symmetric
 // format, whose one product per K step leaves the tensor pipe waiting for loads: twice as many K blocks in flight.
 template <int BK_, bool ONE_PLANE = false>
@@ -58,7 +67,7 @@ struct Cfg {
     static constexpr int kPlanes = ONE_PLANE ? 1 : 2;
     static constexpr int kRowBytes = BK / 2;
     static constexpr int kSteps = BK / 64;                            // MMAs (K = 64) per K block and sign pair
-    static constexpr int kStages = (BK == 256 ? 2 : 4) * (ONE_PLANE ? 2 : 1);
+    static constexpr int kStages = ONE_PLANE ? 8 : 4;
     static constexpr int kTileA = BM * kRowBytes, kTileB = BN * kRowBytes;   // one plane
     static constexpr int kOffAp = 0, kOffAn = ONE_PLANE ? 0 : kTileA, kOffWp = kPlanes * kTileA,
                          kOffWn = kOffWp + (ONE_PLANE ? 0 : kTileB);
@@ -66,13 +75,19 @@ struct Cfg {
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 2048 + 256;   // + alignment slack + Control
     // TMEM columns of one stage's scale factors: A planes (4 columns per K step), then W planes (8)
     static constexpr int kSfColsA = kPlanes * kSteps * 4, kSfCols = kSfColsA + kPlanes * kSteps * 8;
-    static_assert(256 + kStages * kSfCols <= kTmemCols, "scale factors do not fit tensor memory");
-    static_assert(!ONE_PLANE || BK == 128, "the one-plane pipeline exists for 128-element K blocks");
+    // the scale factors of kSfSlots K blocks are in tensor memory at a time (fewer than shared-memory stages: the
+    // scale-factor warps store block i once the MMAs of block i - kSfSlots are done, while block i - 1 is multiplied)
+    static constexpr int kSfSlots = kTmemSfCols / kSfCols;
+    static_assert(kSfSlots >= 2 && kSfSlots % kSfGroups == 0 && kSfSlots <= kStages, "scale-factor ring");
+    static_assert(kAccWindow + BN <= (int)kTmemSf && kTmemSf + kSfSlots * kSfCols <= kTmemCols, "tensor memory map");
+    static_assert(BK == 128, "stages are laid out for 128-element K blocks (64-byte rows, 64-byte swizzle)");
 };
 constexpr int kMaxStages = 8;
 
 struct __align__(16) Control {
-    uint64_t full[kMaxStages], empty[kMaxStages], accum_full, accum_empty;
+    uint64_t full[kMaxStages], empty[kMaxStages], accum_full;
+    uint64_t ovl_free;              // the columns a finished tile shares with the next tile's accumulator have been read
+    uint64_t rest_free[2];          // its other columns have been read ([i]: tiles with number % 2 == i)
     uint64_t sides_ready[2];        // the epilogue warps have written sides[i] for the CTA's tile number 2 k + i
     uint32_t tmem_base;
     volatile int abort;
@@ -85,14 +100,10 @@ static_assert(sizeof(Control) <= 2048 + 256, "Control must fit its reserved spac
 __device__ __forceinline__ uint64_t smem_desc_sw64(uint32_t addr) {
     return (uint64_t)((addr >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)(512 >> 4) << 32) | (1ull << 46) | (4ull << 61);
 }
-template <int BK_>
-__device__ __forceinline__ uint64_t operand_desc(uint32_t addr) {
-    return BK_ == 256 ? smem_desc_sw128(addr) : smem_desc_sw64(addr);
-}
 
 // Instruction descriptor, kind::mxf4nvf4 block-scaled: A and B E2M1 (format code 1), K-major,
 // UE4M3 scale factors (bit 23 = 0), N >> 3 at bit 17, M >> 4 at bit 24, K = 64 (bit 31 = 0).
-constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+__host__ __device__ constexpr uint32_t instr_desc(int n) { return (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24); }
 
 // ------------------------------------------------------------------------- preparation --
 // One launch per operand; one block per 32 operand rows (rows beyond R, up to the padded row count,
@@ -244,7 +255,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     if (p.gate && *p.gate != 0) return;                          // uniform over the grid: nothing was set up yet
     constexpr int BNT = NHALF ? BN / 2 : BN;                     // tile width
     constexpr int kOffWnT = NHALF ? C_::kOffWp + C_::kTileB / 2 : C_::kOffWn;   // the box packs its two planes
-    constexpr uint32_t kIdescT = (1u << 7) | (1u << 10) | ((uint32_t)(BNT >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+    constexpr uint32_t kIdescT = instr_desc(BNT);
     constexpr int BK = C_::BK, kRowBytes = C_::kRowBytes, kSteps = C_::kSteps, kStages = C_::kStages;
     constexpr int kStageBytes = C_::kStageBytes;
     extern __shared__ uint8_t smem_raw[];
@@ -297,7 +308,9 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             mbar_init(&ctl->empty[s], 1);
         }
         mbar_init(&ctl->accum_full, 1);
-        mbar_init(&ctl->accum_empty, kEpilogueWarps);
+        mbar_init(&ctl->ovl_free, kEpilogueWarps);
+        mbar_init(&ctl->rest_free[0], kEpilogueWarps);
+        mbar_init(&ctl->rest_free[1], kEpilogueWarps);
         mbar_init(&ctl->sides_ready[0], kEpilogueWarps);
         mbar_init(&ctl->sides_ready[1], kEpilogueWarps);
         ctl->abort = 0;
@@ -383,7 +396,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         // The whole warp runs the loop (so that addresses and descriptors stay warp-uniform); one elected
         // lane issues.  All operand descriptors differ from the first stage's only in their 14-bit address
         // field (bytes >> 4); the per-plane and per-K-step offsets are compile-time constants.
-        const uint64_t desc0 = operand_desc<BK_>(smem_u32(tiles));
+        const uint64_t desc0 = smem_desc_sw64(smem_u32(tiles));
         int it = 0, t = 0;
         bool ok = true, ready = false;                           // ready: the next K block's barrier was seen complete
         // (the planes of a tile: tile_sides above; the words of the next tile are fetched while the current one runs)
@@ -393,8 +406,12 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             if (!ONE_PLANE) sides_next = tile_sides(tile + gridDim.x);
             const int nkb = nkb_of(tile);
             const int n_mma = ((sides & 1) + ((sides >> 1) & 1)) * (((sides >> 2) & 1) + ((sides >> 3) & 1)) * kSteps;
-            // the previous tile's accumulator must have been read out before it is overwritten
-            if (t > 0) ok = mbar_wait(&ctl->accum_empty, (t - 1) & 1, &ctl->abort, p.status);
+            // this tile's accumulator window: the columns it shares with the previous tile's must have been read, and
+            // so must the rest of the window's last use (tile t - 2).  Neither barrier can run a phase ahead of this
+            // wait: its next completion needs this tile's own MMAs.
+            const uint32_t acc = tmem + ((t & 1) ? kAccWindow : 0);
+            if (t > 0) ok = mbar_wait(&ctl->ovl_free, (t - 1) & 1, &ctl->abort, p.status);
+            if (t > 1 && ok) ok = mbar_wait(&ctl->rest_free[t & 1], ((t >> 1) - 1) & 1, &ctl->abort, p.status);
             tc_fence_after();
             uint32_t accumulate = 0;
             for (int kb = 0; kb < nkb && ok; ++kb, ++it) {
@@ -405,7 +422,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                 if (!ok) break;
                 tc_fence_after();
                 const uint64_t dstage = desc0 + (uint64_t)((s * kStageBytes) >> 4);
-                const uint32_t sfa = tmem + kTmemSf + s * C_::kSfCols, sfb = sfa + C_::kSfColsA;
+                const uint32_t sfa = tmem + kTmemSf + (it % C_::kSfSlots) * C_::kSfCols, sfb = sfa + C_::kSfColsA;
                 const int s_next = (it + 1) % kStages;
                 const uint32_t parity_next = ((it + 1) / kStages) & 1;
                 uint32_t seen = 0;
@@ -418,7 +435,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 #pragma unroll
                             for (int kk = 0; kk < kSteps; ++kk) {   // 64 elements = 32 bytes along the swizzled row
                                 if (((sides >> pa) & 1) && ((sides >> (2 + pw)) & 1)) {
-                                    mma_fp4_block16(tmem, dstage + (((pa ? C_::kOffAn : C_::kOffAp) + kk * 32) >> 4),
+                                    mma_fp4_block16(acc, dstage + (((pa ? C_::kOffAn : C_::kOffAp) + kk * 32) >> 4),
                                                     dstage + (((pw ? kOffWnT : C_::kOffWp) + kk * 32) >> 4), kIdescT,
                                                     sfa + (pa * kSteps + kk) * 4, sfb + (pw * kSteps + kk) * 8,
                                                     idx ? 1u : accumulate);
@@ -473,11 +490,15 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         if (tile < total_tiles) fetch(tile, kb);
         while (tile < total_tiles && ok) {
             const int s = it % kStages;
-            // the stage's TMEM scale-factor buffer is free once the MMAs of K block it - kStages are done
-            if (it >= kStages) ok = mbar_wait(&ctl->empty[s], ((it / kStages) - 1) & 1, &ctl->abort, p.status);
+            // the slot of the scale-factor ring is free once the MMAs of K block it - kSfSlots are done (the `empty`
+            // barrier of that block's stage; it cannot complete again before this block's factors are stored)
+            if (it >= C_::kSfSlots) {
+                const int j = it - C_::kSfSlots;
+                ok = mbar_wait(&ctl->empty[j % kStages], (j / kStages) & 1, &ctl->abort, p.status);
+            }
             if (!ok) break;
             tc_fence_after();
-            const uint32_t sfa = tmem + ((uint32_t)(q * 32) << 16) + kTmemSf + s * C_::kSfCols, sfb = sfa + C_::kSfColsA;
+            const uint32_t sfa = tmem + ((uint32_t)(q * 32) << 16) + kTmemSf + (it % C_::kSfSlots) * C_::kSfCols, sfb = sfa + C_::kSfColsA;
 #pragma unroll
             for (int i = 0; i < kPlanes * kSteps; ++i) {
                 tmem_st4(sfa + i * 4, sfv[i * 3].x, sfv[i * 3].y, sfv[i * 3].z, sfv[i * 3].w);
@@ -498,7 +519,10 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         // -------------------------------------------------------------- epilogue
         // Eight warps: quarter q = warp % 4 of the lanes (= rows), one half of the columns each.
         const int e = warp - (2 + kSfWarps);                     // 0..7
-        const int q = warp & 3, col_base = (e >> 2) * (BNT / 2);
+        const int q = warp & 3;
+        constexpr int kOvl = BNT > kAccWindow ? BNT - kAccWindow : 0;        // columns two consecutive tiles share
+        constexpr int kC1 = kOvl / 2 / 16, kC2 = (BNT - kOvl) / 2 / 16;       // this warp's chunks of either part
+        static_assert(kOvl % 32 == 0 && (BNT - kOvl) % 32 == 0, "both parts split into two halves of 16-column chunks");
         const int tid_e = threadIdx.x - (2 + kSfWarps) * 32;
         int t = 0;
         bool ok = true;
@@ -559,32 +583,50 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
             // every epilogue warp has written its part of w_exp (named barrier: the other roles do not join)
             asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueWarps * 32) : "memory");
             if (ok) {
-                const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)col_base;
+                // The tile's window starts at column 0 (even t) or kAccWindow (odd t).  The kOvl columns it shares with
+                // the next tile's window - its last ones when even, its first ones when odd - are read first; this warp
+                // takes its half h of both parts, kC1 + kC2 chunks of 16 columns.
+                const int h = e >> 2, odd = t & 1;
+                const int o1 = odd ? 0 : BNT - kOvl, o2 = odd ? kOvl : 0;
+                auto chunk_col = [&](int i) {                    // first column (inside the tile) of this warp's chunk i
+                    return i < kC1 ? o1 + h * (kOvl / 2) + 16 * i : o2 + h * ((BNT - kOvl) / 2) + 16 * (i - kC1);
+                };
+                const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(odd ? kAccWindow : 0);
                 uint32_t v[2][16];
-                tmem_ld16(taddr, v[0]);
+                if (kC1 == 0) {                                  // nothing shared: the next tile may start at once
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&ctl->ovl_free);
+                }
+                tmem_ld16(taddr + chunk_col(0), v[0]);
 #pragma unroll
-                for (int c = 0; c < BNT / 2; c += 16) {
-                    const int buf = (c / 16) & 1;
+                for (int i = 0; i < kC1 + kC2; ++i) {
+                    const int buf = i & 1;
                     tmem_ld_wait();
-                    if (c + 16 < BNT / 2) tmem_ld16(taddr + c + 16, v[buf ^ 1]);   // next chunk loads while this one is stored
-                    const int col = col_base + c;
+                    if (i + 1 == kC1) {                          // the shared columns are in registers
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&ctl->ovl_free);
+                    }
+                    if (i + 1 == kC1 + kC2) {                    // so is the rest: tile t + 2 may overwrite the window
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&ctl->rest_free[odd]);
+                    }
+                    if (i + 1 < kC1 + kC2) tmem_ld16(taddr + chunk_col(i + 1), v[buf ^ 1]);   // loads while this chunk is stored
+                    const int col = chunk_col(i);
                     float f[16];
 #pragma unroll
                     for (int j = 0; j < 16; j += 4) {
                         const int4 we = *reinterpret_cast<const int4*>(&w_exp[col + j]);
                         const int ex[4] = {we.x, we.y, we.z, we.w};
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int sh = min(127, max(-126, a_exp + ex[i]));
-                            f[j + i] = __uint_as_float(v[buf][j + i]) * __uint_as_float((uint32_t)(sh + 127) << 23) * out_scale;
+                        for (int k = 0; k < 4; ++k) {
+                            const int sh = min(127, max(-126, a_exp + ex[k]));
+                            f[j + k] = __uint_as_float(v[buf][j + k]) * __uint_as_float((uint32_t)(sh + 127) << 23) * out_scale;
                         }
                     }
                     if (m < p.M) store_row16(C_item + m * p.ld_c + n0 + col, f, p.vec_store != 0, p.N - (n0 + col));
                 }
-                // this warp's part of the accumulator has been read: the next tile may overwrite it
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&ctl->accum_empty);
             }
             ++t;
             tile = tile_after;
@@ -645,15 +687,6 @@ int launch_fp4(const uint8_t* pa, const uint8_t* pw, const OperandLayout& oa, co
     const unsigned grid = (unsigned)(tiles < sm_count[dev] ? tiles : sm_count[dev]);   // one persistent CTA per SM
     gemm_fp4_kernel<BK_, SLICED, NHALF, ONE_PLANE><<<grid, kThreads, C_::kSmemBytes, st>>>(tm_a, tm_w, tm_a1, tm_w1, p);
     return launch_status();
-}
-
-// K-block size of the main loop: 128 (four 54 KB stages) unless AMX_FP4_BK=256 asks for two 108 KB stages.
-int fp4_block_k() {
-    static const int bk = [] {
-        const char* e = getenv("AMX_FP4_BK");
-        return (e && atoi(e) == 256) ? 256 : 128;
-    }();
-    return bk;
 }
 
 }  // namespace
@@ -729,7 +762,7 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
     const int slices = gemm_fp4_slices(M, N, K);
     // at most 128 columns: tiles of 128 x 128, so that no half of a W tile is padding
     const bool half = N <= BN / 2 && !getenv("AMX_FP4_NO_HALF_TILE");
-    if (!gate && !scale_a && slices > 1 && fp4_block_k() == 128 && workspace_bytes >= gemm_fp4_prepared_workspace_bytes(M, N, K)) {
+    if (!gate && !scale_a && slices > 1 && workspace_bytes >= gemm_fp4_prepared_workspace_bytes(M, N, K)) {
         float* part = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 256);
         p.C = part;
         p.ld_c = N;
@@ -739,7 +772,6 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
         const int r2 = launch_fp4<128, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
         return r2 != AMX_OK ? r2 : reduce_slices(part, slices, M, N, C, ld_c, st);
     }
-    if (fp4_block_k() == 256) return launch_fp4<256>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
     // both operands stated to be single planes: the deeper pipeline (full-width tiles; the other shapes are short
     // products, where the depth does not matter, and run the general kernel, which skips absent planes by itself)
     if (one_plane && !half) return launch_fp4<128, false, false, true>(pa, pw, oa, ow, a.rows_total, w.rows_total, p, dev, st);
