@@ -41,7 +41,7 @@ BYTES_PER_ELEM = 2.0 + 0.5 + 2.0 / 32.0   # bf16 read + 4-bit code + two scale b
 MOVED_BYTES_PER_ELEM = 2.0 + 1.0 + 2.0 / 32.0 + 4.0 / 32.0
 # DRAM bytes (read + write) per GEMM launch of the FP4 kernel, mean over the layers of a config, from the ncu
 # captures summarised in profiles/ (None: no capture of the current kernel on that config).
-GEMM_DRAM_TRAFFIC_PER_LAUNCH = {2: 89.5e6, 3: 614.3e6, 4: 3.843e9}
+GEMM_DRAM_TRAFFIC_PER_LAUNCH = {2: 89.2e6, 3: 613.7e6, 4: 4.225e9}
 
 
 def measured_peaks():
