@@ -706,8 +706,9 @@ def run_ours(args):
         decode = time_decode(max(20, min(args.steps, 100)))
 
     # ---- end to end through the host-buffer entry point (pinned host tensors, copies inside the timing).
-    # Consecutive layers alternate between two streams and two workspaces and the call does not synchronise
-    # (AMX_HOST_NO_SYNC), so that one layer's result goes back to the host while the next layer's inputs come in.
+    # amx_linear_host_pipelined per layer on three streams (copies in, kernels, copies out), a workspace per layer,
+    # no synchronisation between the layers (AMX_HOST_NO_SYNC): the rows of A go through in chunks, so results go
+    # back to the host while later rows and the next layer's inputs come in.
     e2e = None
     if (rank == 0 or world > 1) and not args.skip_extras:
         pinned = []
@@ -716,18 +717,23 @@ def run_ours(args):
             pinned.append((torch.from_numpy(a_bits.view(np.int16)).view(torch.bfloat16).pin_memory(),
                            torch.from_numpy(w_bits.view(np.int16)).view(torch.bfloat16).pin_memory(),
                            torch.empty((M, N), dtype=torch.float32).pin_memory()))
-        lh_bytes = max(L.amx_linear_host_workspace_bytes(M, N, K, GS, gemm_flag) for K, N in layers)
-        lh_ws = [torch.empty(lh_bytes, dtype=torch.uint8, device="cuda") for _ in range(2)]
-        lh_streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+        lh_ws = [torch.empty(L.amx_linear_host_pipelined_workspace_bytes(M, N, K, GS, gemm_flag), dtype=torch.uint8, device="cuda")
+                 for K, N in layers]
+        lh_streams = [torch.cuda.Stream() for _ in range(3)]
 
         def e2e_step():
             for li, (K, N) in enumerate(layers):
                 a, w, c = pinned[li]
-                check(L.amx_linear_host(a.data_ptr(), w.data_ptr(), M, N, K, GS, gemm_flag | amx.HOST_NO_SYNC, c.data_ptr(),
-                                        lh_ws[li % 2].data_ptr(), lh_ws[li % 2].numel(), lh_streams[li % 2].cuda_stream))
+                check(L.amx_linear_host_pipelined(a.data_ptr(), w.data_ptr(), M, N, K, GS, gemm_flag | amx.HOST_NO_SYNC,
+                                                  c.data_ptr(), lh_ws[li].data_ptr(), lh_ws[li].numel(),
+                                                  *(s.cuda_stream for s in lh_streams)))
             torch.cuda.synchronize()
 
         e2e_step()
+        for li in range(len(layers)):
+            st_word = L.amx_linear_host_pipelined_status(lh_ws[li].data_ptr(), lh_streams[1].cuda_stream)
+            if st_word != 0:
+                raise RuntimeError(f"end-to-end leg, layer {layer_ids[li]}: status {amx.status_string(st_word)}")
         barrier()
         e2e_steps = max(2, min(args.steps, 5))
         t0 = time.perf_counter()
@@ -739,8 +745,9 @@ def run_ours(args):
                "h2d_bytes_per_step": int(elems_step * 2),
                "d2h_bytes_per_step": int(sum(M * N * 4 for _, N in layers)),
                "ms_per_step": e2e_s * 1e3,
-               "what": "amx_linear_host per layer from pinned host buffers; layers alternate between two streams, so "
-                       "host-to-device and device-to-host copies of neighbouring layers overlap; PCIe-bound"}
+               "what": "amx_linear_host_pipelined per layer from pinned host buffers on three streams (copies in, "
+                       "kernels, copies out): the rows of A go through in chunks of 2048, so host-to-device and "
+                       "device-to-host copies overlap within and across layers; PCIe-bound"}
         del pinned, lh_ws
 
     if rank != 0:

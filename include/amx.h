@@ -344,6 +344,31 @@ int amx_attention_map(const void* q, const void* k, const void* v, int64_t L, in
 int amx_linear_host(const void* A_host, const void* W_host, int64_t M, int64_t N, int64_t K,
                     int group_size, uint32_t flags, float* C_host,
                     void* workspace, size_t workspace_bytes, void* stream);
+/*
+ * amx_linear_host_pipelined - the same layer as a pipeline over THREE streams of the caller (no hidden streams):
+ * W_host goes in on stream_in and is cast once on stream_compute; the rows of A_host then go through in chunks
+ * of about 2048 rows (a multiple of 128) - chunk i is copied in on stream_in, cast and multiplied on
+ * stream_compute (amx_quant_gemm with the quantized weight), and its rows of C are copied out on stream_out while
+ * chunk i + 1 is copied in and chunk i + 2... follow; events recorded between the streams (created and destroyed
+ * inside the call) carry the dependencies.  Host-to-device and device-to-host copies so run at the same time
+ * within one layer, and consecutive calls on the same three streams (each with its own workspace) keep both copy
+ * directions busy across layers.  Same C as amx_linear_host, bit for bit when the chunks run the same kernel as
+ * the whole product would (a chunk is a smaller product: under AMX_GEMM_AUTO it may pick another kernel, whose fp32
+ * summation order differs).
+ *   flags      AMX_GEMM_* kernel choice (binds every chunk: AMX_ERR_SHAPE if a chunk does not fit it),
+ *              optionally | AMX_HOST_NO_SYNC (return once everything is enqueued; without it the call returns after
+ *              synchronising stream_out, when C_host is complete)
+ *   workspace  device scratch, amx_linear_host_pipelined_workspace_bytes() bytes, 256-aligned.  It may be used by
+ *              another call only after this call's work has completed on all three streams.
+ *   streams    three different streams (two equal ones: AMX_ERR_FLAGS)
+ * amx_linear_host_pipelined_status: the first nonzero status word of the call's chunks (see amx_gemm_status; each
+ * chunk's word is kept at the start of the workspace), or AMX_OK.  Synchronises `stream` (pass stream_compute).
+ */
+size_t amx_linear_host_pipelined_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size, uint32_t flags);
+int amx_linear_host_pipelined(const void* A_host, const void* W_host, int64_t M, int64_t N, int64_t K,
+                              int group_size, uint32_t flags, float* C_host, void* workspace,
+                              size_t workspace_bytes, void* stream_in, void* stream_compute, void* stream_out);
+int amx_linear_host_pipelined_status(const void* workspace, void* stream);
 
 /*
  * amx_quant_gemm_static - amx_quant_gemm (quantized-weight form) without a workspace argument, for callers

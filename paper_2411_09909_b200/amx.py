@@ -42,6 +42,7 @@ SYMBOLS = (
     "amx_quantize_f16s", "amx_dequantize_f16s", "amx_gemm_f16s", "amx_quant_error_f16s",
     "amx_fake_quantize", "amx_attention_workspace_bytes_for", "amx_attention_gqa",
     "amx_gemm_prepared_sym", "amx_gemm_nvfp4_sym",
+    "amx_linear_host_pipelined", "amx_linear_host_pipelined_workspace_bytes", "amx_linear_host_pipelined_status",
 )
 
 
@@ -104,6 +105,10 @@ def lib() -> ctypes.CDLL:
         L.amx_softmax_bf16.argtypes = [p, i64, i64, i64, ctypes.c_float, p, i64, p]
         L.amx_softmax_quantize.argtypes = [p, i64, i64, i64, ctypes.c_float, p, p, i, p, sz, p]
         L.amx_linear_host.argtypes = [p, p, i64, i64, i64, i, u32, p, p, sz, p]
+        L.amx_linear_host_pipelined.argtypes = [p, p, i64, i64, i64, i, u32, p, p, sz, p, p, p]
+        L.amx_linear_host_pipelined_workspace_bytes.argtypes = [i64, i64, i64, i, u32]
+        L.amx_linear_host_pipelined_workspace_bytes.restype = sz
+        L.amx_linear_host_pipelined_status.argtypes = [p, p]
         for name in ("amx_workspace_bytes", "amx_quant_gemm_workspace_bytes"):
             getattr(L, name).argtypes = [i64, i64, i64, i, u32]
             getattr(L, name).restype = sz
@@ -460,6 +465,21 @@ def linear_host(a_host: torch.Tensor, w_host: torch.Tensor, c_host: torch.Tensor
     _check(lib().amx_linear_host(a_host.data_ptr(), w_host.data_ptr(), M, N, K, group_size, flags,
                                  c_host.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream()),
            "amx_linear_host")
+    return c_host
+
+
+def linear_host_pipelined(a_host: torch.Tensor, w_host: torch.Tensor, c_host: torch.Tensor, workspace: torch.Tensor,
+                          streams, group_size: int = 32, flags: int = GEMM_AUTO):
+    """amx_linear_host as a pipeline over three torch streams (in, compute, out): the rows of a go through in chunks,
+    copies in both directions and the kernels overlap.  Synchronises the out stream unless flags carry HOST_NO_SYNC."""
+    assert not a_host.is_cuda and not w_host.is_cuda and not c_host.is_cuda and workspace.is_cuda
+    assert a_host.dtype == w_host.dtype == torch.bfloat16 and c_host.dtype == torch.float32
+    M, K = a_host.shape
+    N = w_host.shape[0]
+    s_in, s_cmp, s_out = (s.cuda_stream for s in streams)
+    _check(lib().amx_linear_host_pipelined(a_host.data_ptr(), w_host.data_ptr(), M, N, K, group_size, flags,
+                                           c_host.data_ptr(), workspace.data_ptr(), workspace.numel(), s_in, s_cmp, s_out),
+           "amx_linear_host_pipelined")
     return c_host
 
 

@@ -311,6 +311,125 @@ extern "C" int amx_linear_host(const void* A_host, const void* W_host, int64_t M
     return cudaStreamSynchronize(st) == cudaSuccess ? AMX_OK : AMX_ERR_CUDA;
 }
 
+// ---- the same layer as a pipeline over three caller-owned streams
+namespace {
+constexpr int kHostChunksMax = 16;                       // status slots at the start of the workspace
+// Rows of A per chunk: about 2048, a multiple of 128 (so that every chunk but the last fills whole tiles), at most
+// kHostChunksMax chunks.
+int64_t host_chunk_rows(int64_t M) {
+    int64_t n = (M + 2047) / 2048;
+    if (n > kHostChunksMax) n = kHostChunksMax;
+    if (n < 1) n = 1;
+    const int64_t rows = ((M + n - 1) / n + 127) / 128 * 128;
+    return rows < M ? rows : M;
+}
+struct HostLayout {
+    size_t w_dev, w_codes, w_scales, a_dev, c_dev, qg, total;
+    size_t qg_bytes;
+};
+HostLayout host_layout(int64_t M, int64_t N, int64_t K, int gs, uint32_t kernel_flags) {
+    HostLayout h{};
+    const QuantSizes w = quant_sizes(N, K, gs);
+    size_t off = 256;                                    // kHostChunksMax status slots of 8 bytes (+ padding)
+    h.w_dev = off;    off += round_up((size_t)N * K * 2);
+    h.w_codes = off;  off += round_up(w.codes);
+    h.w_scales = off; off += round_up(w.scales);
+    h.a_dev = off;    off += round_up((size_t)M * K * 2);
+    h.c_dev = off;    off += round_up((size_t)M * N * 4);
+    h.qg = off;
+    const int64_t mc = host_chunk_rows(M), last = M % mc ? M % mc : mc;     // the last chunk may pick another kernel
+    const size_t q_full = amx_quant_gemm_workspace_bytes(mc, N, K, gs, kernel_flags);
+    const size_t q_last = amx_quant_gemm_workspace_bytes(last, N, K, gs, kernel_flags);
+    h.qg_bytes = q_full > q_last ? q_full : q_last;
+    h.total = off + h.qg_bytes;
+    return h;
+}
+}  // namespace
+
+extern "C" size_t amx_linear_host_pipelined_workspace_bytes(int64_t M, int64_t N, int64_t K, int group_size,
+                                                            uint32_t flags) {
+    flags &= ~AMX_HOST_NO_SYNC;
+    if ((flags & ~kKernelMask) || !gemm_shape_ok(M, N, K, group_size) || M == 0 || N == 0) return 0;
+    return host_layout(M, N, K, group_size, flags).total;
+}
+
+extern "C" int amx_linear_host_pipelined(const void* A_host, const void* W_host, int64_t M, int64_t N, int64_t K,
+                                         int group_size, uint32_t flags, float* C_host, void* workspace,
+                                         size_t workspace_bytes, void* stream_in, void* stream_compute,
+                                         void* stream_out) {
+    const bool no_sync = flags & AMX_HOST_NO_SYNC;
+    flags &= ~AMX_HOST_NO_SYNC;
+    if (flags & ~kKernelMask) return AMX_ERR_FLAGS;
+    if (!gemm_shape_ok(M, N, K, group_size)) return AMX_ERR_SHAPE;
+    const int64_t mc = host_chunk_rows(M);
+    // every chunk must find a kernel under these flags (an explicit kernel choice binds every chunk)
+    if (!pick_kernel(M, N, K, group_size, flags)) return (flags & (flags - 1)) ? AMX_ERR_FLAGS : AMX_ERR_SHAPE;
+    if (M == 0 || N == 0) return AMX_OK;
+    for (int64_t m0 = 0; m0 < M; m0 += mc)
+        if (!pick_kernel(M - m0 < mc ? M - m0 : mc, N, K, group_size, flags)) return AMX_ERR_SHAPE;
+    if (!A_host || !W_host || !C_host) return AMX_ERR_NULL;
+    if (stream_in == stream_compute || stream_out == stream_compute || stream_in == stream_out) return AMX_ERR_FLAGS;
+    const HostLayout h = host_layout(M, N, K, group_size, flags);
+    if (!workspace || workspace_bytes < h.total) return AMX_ERR_WORKSPACE;
+    if (!aligned(workspace, kAlign)) return AMX_ERR_ALIGN;
+    cudaStream_t s_in = static_cast<cudaStream_t>(stream_in), s_cmp = static_cast<cudaStream_t>(stream_compute),
+                 s_out = static_cast<cudaStream_t>(stream_out);
+    uint8_t* base = static_cast<uint8_t*>(workspace);
+    uint8_t* w_dev = base + h.w_dev;
+    uint8_t* a_dev = base + h.a_dev;
+    float* c_dev = reinterpret_cast<float*>(base + h.c_dev);
+    // One event per hand-over between two streams; destroying an event that is still pending is allowed (its
+    // resources are released when it completes), so nothing outlives the call.
+    cudaEvent_t ev = nullptr;
+    auto hand_over = [&](cudaStream_t from, cudaStream_t to) -> bool {
+        if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return false;
+        const bool ok = cudaEventRecord(ev, from) == cudaSuccess && cudaStreamWaitEvent(to, ev, 0) == cudaSuccess;
+        cudaEventDestroy(ev);
+        return ok;
+    };
+    auto fail = [&]() { cudaGetLastError(); return AMX_ERR_CUDA; };
+    // weight: in, then cast once to canonical codes and scales
+    if (cudaMemsetAsync(base, 0, 256, s_cmp) != cudaSuccess) return fail();
+    if (cudaMemcpyAsync(w_dev, W_host, (size_t)N * K * 2, cudaMemcpyHostToDevice, s_in) != cudaSuccess) return fail();
+    if (!hand_over(s_in, s_cmp)) return fail();
+    int rc = amx_quantize(w_dev, N, K, K, group_size, base + h.w_codes, base + h.w_scales, stream_compute);
+    if (rc != AMX_OK) return rc;
+    // activation rows in chunks: copy in | cast + multiply | copy out, each on its stream
+    int slot = 0;
+    for (int64_t m0 = 0; m0 < M; m0 += mc, ++slot) {
+        const int64_t rows = M - m0 < mc ? M - m0 : mc;
+        uint8_t* a_rows = a_dev + (size_t)m0 * K * 2;
+        float* c_rows = c_dev + (size_t)m0 * N;
+        if (cudaMemcpyAsync(a_rows, static_cast<const uint8_t*>(A_host) + (size_t)m0 * K * 2, (size_t)rows * K * 2,
+                            cudaMemcpyHostToDevice, s_in) != cudaSuccess || !hand_over(s_in, s_cmp))
+            return fail();
+        rc = amx_quant_gemm(a_rows, K, base + h.w_codes, base + h.w_scales, nullptr, 0, rows, N, K, group_size, flags, c_rows,
+                            N, base + h.qg, h.qg_bytes, stream_compute);
+        if (rc != AMX_OK) return rc;
+        // the chunk's status word and flushed-scale count, kept past the next chunk's use of the same scratch
+        if (cudaMemcpyAsync(base + 8 * slot, base + h.qg, 8, cudaMemcpyDeviceToDevice, s_cmp) != cudaSuccess ||
+            !hand_over(s_cmp, s_out) ||
+            cudaMemcpyAsync(C_host + (size_t)m0 * N, c_rows, (size_t)rows * N * 4, cudaMemcpyDeviceToHost, s_out) != cudaSuccess)
+            return fail();
+    }
+    if (no_sync) return AMX_OK;
+    return cudaStreamSynchronize(s_out) == cudaSuccess ? AMX_OK : AMX_ERR_CUDA;
+}
+
+extern "C" int amx_linear_host_pipelined_status(const void* workspace, void* stream) {
+    if (!workspace) return AMX_ERR_NULL;
+    int words[2 * kHostChunksMax] = {};
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(words, workspace, sizeof(words), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return AMX_ERR_CUDA;
+    }
+    for (int i = 0; i < kHostChunksMax; ++i)
+        if (words[2 * i] != 0) return words[2 * i];
+    return AMX_OK;
+}
+
 extern "C" int amx_softmax_quantize(const float* S, int64_t rows, int64_t cols, int64_t ld_s, float alpha,
                                     uint8_t* codes, uint8_t* scales, int is_weight, void* prepared,
                                     size_t prepared_bytes, void* stream) {

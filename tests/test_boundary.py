@@ -74,6 +74,14 @@ def test_host_detected_argument_errors(L):
     assert qg(fake, 64, None, None, odd, 64, 4, 4, 64, 32, 0x10, fake, 4, fake, 1 << 20, None) == -3    # bf16 weight alignment
     assert L.amx_linear_host(fake, fake, 4, 4, 64, 32, 0x30, fake, fake, 1 << 30, None) == -5             # two kernels
     assert L.amx_linear_host(fake, fake, 4, 4, 64, 32, 0x40, fake, fake, 16, None) == -4                  # checked before any copy
+    s1, s2, s3 = ctypes.c_void_p(0x100), ctypes.c_void_p(0x200), ctypes.c_void_p(0x300)          # never dereferenced here
+    lp = L.amx_linear_host_pipelined
+    assert lp(fake, fake, 4, 4, 64, 32, 0x30, fake, fake, 1 << 30, s1, s2, s3) == -5                      # two kernels
+    assert lp(fake, fake, 4, 4, 64, 32, 0, fake, fake, 1 << 30, s1, s1, s3) == -5                         # two equal streams
+    assert lp(fake, fake, 4, 4, 64, 32, 0, fake, fake, 16, s1, s2, s3) == -4                              # before any copy
+    assert lp(fake, fake, 4, 4, 48, 32, 0, fake, fake, 1 << 30, s1, s2, s3) == -2
+    assert lp(None, fake, 4, 4, 64, 32, 0, fake, fake, 1 << 30, s1, s2, s3) == -1
+    assert L.amx_linear_host_pipelined_workspace_bytes(4096, 256, 512, 32, 0) > L.amx_linear_host_workspace_bytes(2048, 256, 512, 32, 0)
     am = L.amx_attention_map
     assert am(fake, fake, fake, 320, 128, 0, fake, fake, fake, fake, fake, 1 << 30, fake, 1 << 30, None) == -2   # L % 128
     assert am(fake, fake, fake, 512, 64, 0, fake, fake, fake, fake, fake, 1 << 30, fake, 1 << 30, None) == -2    # d != 128

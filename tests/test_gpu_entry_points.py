@@ -194,6 +194,63 @@ def test_linear_host_with_explicit_kernel(flags):
         assert np.array_equal(o.numpy(), c.numpy())
 
 
+@pytest.mark.parametrize("flags", [amx.GEMM_AUTO, amx.GEMM_FP4, amx.GEMM_TC, amx.GEMM_SIMT])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 1024), (4500, 520, 1056), (2049, 300, 512), (16, 512, 1024)])
+def test_linear_host_pipelined(flags, M, N, K):
+    """The three-stream pipeline over row chunks (4500 rows: three chunks of 1536, 1536 and 1428; 2049: 1152 + 897)
+    against the oracle and against the one-stream entry point; two layers in flight on the same streams."""
+    if not amx.lib().amx_gemm_kernel_for(M, N, K, 32, flags) or not amx.lib().amx_gemm_kernel_for(min(M, 897), N, K, 32, flags):
+        pytest.skip("kernel choice does not take this shape")
+    a_bits = inputs.random_groups(5100 + M, M, K, "normal")
+    w_bits = inputs.random_groups(5200 + N, N, K, "normal")
+    a = torch.from_numpy(a_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+    w = torch.from_numpy(w_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+    L = amx.lib()
+    nbytes = L.amx_linear_host_pipelined_workspace_bytes(M, N, K, 32, flags)
+    assert nbytes > 0
+    streams = [torch.cuda.Stream() for _ in range(3)]
+    works = [torch.full((nbytes,), 0xFF, dtype=torch.uint8, device="cuda") for _ in range(2)]
+    outs = [torch.full((M, N), float("nan"), dtype=torch.float32).pin_memory() for _ in range(2)]
+    torch.cuda.synchronize()
+    amx.linear_host_pipelined(a, w, outs[0], works[0], streams, flags=flags)                 # synchronous form
+    assert L.amx_linear_host_pipelined_status(works[0].data_ptr(), streams[1].cuda_stream) == 0
+    ref = oracle.gemm(*oracle.quantize(a_bits, 32), *oracle.quantize(w_bits, 32), 32)
+    assert rel_fro(outs[0].numpy(), ref) <= 1e-3
+    one = torch.empty((M, N), dtype=torch.float32).pin_memory()
+    amx.linear_host(a, w, one, torch.empty(L.amx_linear_host_workspace_bytes(M, N, K, 32, flags), dtype=torch.uint8,
+                                           device="cuda"), flags=flags)
+    assert rel_fro(outs[0].numpy(), one.numpy().astype(np.float64)) <= 1e-5
+    # two calls in flight on the same three streams, a workspace each
+    first = outs[0].numpy().copy()
+    for o in outs:
+        o.fill_(float("nan"))
+    for o, wk in zip(outs, works):
+        amx.linear_host_pipelined(a, w, o, wk, streams, flags=flags | amx.HOST_NO_SYNC)
+    torch.cuda.synchronize()
+    for o, wk in zip(outs, works):
+        assert np.array_equal(o.numpy(), first)
+        assert L.amx_linear_host_pipelined_status(wk.data_ptr(), None) == 0
+
+
+def test_linear_host_pipelined_argument_errors():
+    L = amx.lib()
+    a = torch.zeros((128, 64), dtype=torch.bfloat16).pin_memory()
+    c = torch.zeros((128, 128), dtype=torch.float32).pin_memory()
+    need = L.amx_linear_host_pipelined_workspace_bytes(128, 128, 64, 32, 0)
+    ws = torch.empty(need + 256, dtype=torch.uint8, device="cuda")
+    streams = [torch.cuda.Stream() for _ in range(3)]
+    s = [t.cuda_stream for t in streams]
+    args = (a.data_ptr(), a.data_ptr(), 128, 128, 64, 32)
+    assert L.amx_linear_host_pipelined(*args, 0, c.data_ptr(), ws.data_ptr(), ws.numel(), s[0], s[0], s[2]) == -5
+    assert L.amx_linear_host_pipelined(*args, 0x30, c.data_ptr(), ws.data_ptr(), ws.numel(), *s) == -5
+    assert L.amx_linear_host_pipelined(*args, 0, c.data_ptr(), ws.data_ptr(), 1024, *s) == -4
+    assert L.amx_linear_host_pipelined(*args, 0, None, ws.data_ptr(), ws.numel(), *s) == -1
+    assert L.amx_linear_host_pipelined(a.data_ptr(), a.data_ptr(), 128, 128, 48, 32, 0, c.data_ptr(), ws.data_ptr(), ws.numel(), *s) == -2
+    assert L.amx_linear_host_pipelined(*args, 0, c.data_ptr(), ws.data_ptr() + 16, need, *s) == -3
+    assert L.amx_linear_host_pipelined_workspace_bytes(128, 128, 48, 32, 0) == 0
+    torch.cuda.synchronize()
+
+
 @pytest.mark.parametrize("rows,K,is_w", [(300, 1056, False), (130, 96, True), (77, 11008, False), (9, 36864, True), (2100, 128, True)])
 def test_quantize_prepared_without_canonical_codes(rows, K, is_w):
     """The prepared cast with codes = NULL writes the same scales and the same prepared operand, byte for byte
