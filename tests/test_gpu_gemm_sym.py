@@ -69,6 +69,35 @@ def test_gemm_prepared_sym_full_size_layer():
     assert rel_fro(got[torch.from_numpy(rows).cuda()].cpu().numpy(), ref) <= GEMM_TOL
 
 
+@pytest.mark.parametrize("fmt,mode", [(amx.FMT_AMXFP4, 0), (amx.FMT_MXFP4, oracle.MXFP4)])
+@pytest.mark.parametrize("M,N,K", [(1100, 6200, 1056), (2304, 6400, 288), (130, 40000, 160)])
+def test_several_tiles_per_cta(fmt, mode, M, N, K):
+    """Products whose persistent CTAs get one and two, three and four, and two tiles each (225, 450 and 314 tiles on
+    148 CTAs): consecutive tiles of a CTA alternate between the two accumulator windows.  Two rows of every block of
+    128 rows against the oracle, so that every output tile is checked; the general and the one-plane kernel."""
+    a_bits = inputs.random_groups(4700 + M, M, K, "normal")
+    w_bits = inputs.random_groups(4800 + M, N, K, "normal")
+    quant = (lambda b: oracle.quantize(b, 32)) if mode == 0 else (lambda b: oracle.quantize_variant(b, 32, mode))
+    _, _, pa = amx.quantize_prepared(dev_bf16(a_bits), False, fmt=fmt)
+    wc, ws_, pw = amx.quantize_prepared(dev_bf16(w_bits), True, fmt=fmt)
+    rng = np.random.default_rng(47)
+    rows = np.sort(np.concatenate([b + rng.choice(min(128, M - b), size=2, replace=False) for b in range(0, M, 128)]))
+    qa = quant(a_bits[rows])
+    ref = oracle.gemm(*qa, wc.cpu().numpy(), ws_.cpu().numpy(), 32)
+    rows_dev = torch.from_numpy(rows).cuda()
+    for sym in ([False, True] if mode else [False]):
+        work = torch.full((256,), 0xFF, dtype=torch.uint8, device="cuda")
+        got = amx.gemm_prepared(pa, pw, M, N, K, workspace=work, sym=sym)
+        assert amx.gemm_status(work) == 0
+        assert rel_fro(got[rows_dev].cpu().numpy(), ref) <= GEMM_TOL
+        # no tile differs from the rest: per-tile error norms against the exact bf16-decode kernel's product
+        if not sym and mode == 0:
+            ac, as_ = amx.quantize(dev_bf16(a_bits), 32)
+            exact = amx.gemm(ac, as_, wc, ws_, 32, amx.GEMM_TC)
+            err = (got - exact).abs().amax(dim=0).cpu().numpy(), exact.abs().amax().item()
+            assert err[0].max() <= 1e-4 * err[1]
+
+
 def test_one_signed_amxfp4_operand_is_a_single_plane():
     """An AMXFP4 operand whose values are all non-negative (an activation after ReLU) has no negative plane."""
     M, N, K = 260, 515, 1024
