@@ -581,6 +581,18 @@ def run_ours(args):
             for li in range(len(layers)):                        # the one-plane promise held, no wait expired
                 if amx.gemm_status(bufs[li]["work"]) != 0:
                     raise RuntimeError(f"{name}, layer {layer_ids[li]}: GEMM status {amx.status_string(amx.gemm_status(bufs[li]['work']))}")
+        # the AMXFP4 GEMMs with a bf16 result (rounded in the epilogue: half the bytes stored); operands as the
+        # headline step's casts left them
+        run_step()
+        def amx_gemms(st, out_flags=0):
+            for li, (K, N) in enumerate(layers):
+                b = bufs[li]
+                check(L.amx_gemm_prepared_ex(b["pa"].data_ptr(), b["pw"].data_ptr(), M, N, K, GS, out_flags,
+                                             b["c"].data_ptr(), N, b["work"].data_ptr(), b["work"].numel(), st))
+        for name, out_flags in (("amxfp4_f32_result", 0), ("amxfp4_bf16_result", amx.PREP_OUT_BF16)):
+            amx_gemms(stream, out_flags)
+            v_ms = timed_graph(lambda st: amx_gemms(st, out_flags), extra_steps)
+            format_variants[name] = {"gemm_tflops": flops_step / (v_ms * 1e-3) / 1e12, "gemm_ms": v_ms}
         # NVFP4 / ANVFP4 (group 16, E4M3 group scales + fp32 tensor scale: Section 5's comparison format): the scale
         # bytes are the tensor cores' native type, NVFP4 is one product per tile pair, ANVFP4 four
         nv = []
@@ -616,7 +628,9 @@ def run_ours(args):
                                    "and a tensor scale (amx_quantize_nvfp4: two launches, the tensor maximum first); step = "
                                    "casts of both operands + GEMMs, gemm = the GEMMs alone; the symmetric formats run the "
                                    "one-plane pipeline (amx_gemm_prepared_sym, amx_gemm_nvfp4_sym), gemm_general_kernel = "
-                                   "the same operands through amx_gemm_prepared")
+                                   "the same operands through amx_gemm_prepared; amxfp4_bf16_result = the headline's "
+                                   "AMXFP4 GEMMs through amx_gemm_prepared_ex with AMX_PREP_OUT_BF16, amxfp4_f32_result = the same measurement "
+                                   "(GEMMs alone, graph replay) with the fp32 result")
         run_step()                      # leave the buffers as the headline step writes them
         torch.cuda.synchronize()
 

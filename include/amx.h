@@ -227,6 +227,17 @@ int amx_gemm_prepared(const void* a_prepared, const void* w_prepared, int64_t M,
 int amx_gemm_prepared_sym(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
                           int group_size, float* C, int64_t ld_c, void* workspace, size_t workspace_bytes,
                           void* stream);
+/* amx_gemm_prepared with options.  flags: AMX_PREP_ONE_PLANE = the promise of amx_gemm_prepared_sym;
+ * AMX_PREP_OUT_BF16 = C is bf16 [M, ld_c] (2-byte aligned; 32-byte stores when C is 32-byte aligned and
+ * ld_c % 16 == 0): every result is the fp32 accumulator value - what amx_gemm_prepared stores - rounded to bf16,
+ * ties to even, in the epilogue.  For layers whose output feeds the next cast: half the bytes written, and no
+ * separate conversion pass (Section 5 casts bf16 activations).  The K ranges of amx_gemm_prepared are not used
+ * with a bf16 result (their partial sums are fp32).  Other flag bits: AMX_ERR_FLAGS. */
+#define AMX_PREP_ONE_PLANE 0x1u
+#define AMX_PREP_OUT_BF16 0x2u
+int amx_gemm_prepared_ex(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
+                         int group_size, uint32_t flags, void* C, int64_t ld_c, void* workspace,
+                         size_t workspace_bytes, void* stream);
 
 /*
  * amx_quant_gemm - the fully quantized linear layer of Section 5 ("quantize input operands for

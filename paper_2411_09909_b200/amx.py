@@ -24,6 +24,7 @@ FMT_AMXFP4_POT, FMT_MXFP4_POT_ROUND, FMT_AMXFP4_POT_ROUND = 3, 4, 5   # amx_quan
 WEIGHT_BF16 = 0x200             # amx_quant_gemm_workspace_bytes: size for a bf16 weight
 ATTN_CAUSAL = 0x1000            # amx_attention / amx_attention_map
 HOST_NO_SYNC = 0x2000           # amx_linear_host: do not synchronise
+PREP_ONE_PLANE, PREP_OUT_BF16 = 0x1, 0x2   # amx_gemm_prepared_ex
 
 # every symbol include/amx.h declares
 SYMBOLS = (
@@ -41,7 +42,7 @@ SYMBOLS = (
     "amx_quantize_nvfp4", "amx_nvfp4_prepared_bytes", "amx_dequantize_nvfp4", "amx_gemm_nvfp4",
     "amx_quantize_f16s", "amx_dequantize_f16s", "amx_gemm_f16s", "amx_quant_error_f16s",
     "amx_fake_quantize", "amx_attention_workspace_bytes_for", "amx_attention_gqa",
-    "amx_gemm_prepared_sym", "amx_gemm_nvfp4_sym",
+    "amx_gemm_prepared_sym", "amx_gemm_nvfp4_sym", "amx_gemm_prepared_ex",
     "amx_linear_host_pipelined", "amx_linear_host_pipelined_workspace_bytes", "amx_linear_host_pipelined_status",
 )
 
@@ -100,6 +101,7 @@ def lib() -> ctypes.CDLL:
         L.amx_quantize_prepared.argtypes = [p, i64, i64, i, i, p, p, p, sz, p]
         L.amx_gemm_prepared.argtypes = [p, p, i64, i64, i64, i, p, i64, p, sz, p]
         L.amx_gemm_prepared_sym.argtypes = [p, p, i64, i64, i64, i, p, i64, p, sz, p]
+        L.amx_gemm_prepared_ex.argtypes = [p, p, i64, i64, i64, i, u32, p, i64, p, sz, p]
         L.amx_gemm_prepared_workspace_bytes.argtypes = [i64, i64, i64, i]
         L.amx_gemm_prepared_workspace_bytes.restype = sz
         L.amx_softmax_bf16.argtypes = [p, i64, i64, i64, ctypes.c_float, p, i64, p]
@@ -263,12 +265,20 @@ def quantize_prepared(x: torch.Tensor, is_weight: bool, group_size: int = 32, pr
 
 
 def gemm_prepared(a_prepared: torch.Tensor, w_prepared: torch.Tensor, M: int, N: int, K: int, group_size: int = 32,
-                  out: torch.Tensor | None = None, workspace: torch.Tensor | None = None, sym: bool = False):
-    """sym: both operands are in a symmetric format (amx_gemm_prepared_sym; a violated promise shows in gemm_status)."""
+                  out: torch.Tensor | None = None, workspace: torch.Tensor | None = None, sym: bool = False,
+                  out_dtype=torch.float32):
+    """sym: both operands are in a symmetric format (amx_gemm_prepared_sym; a violated promise shows in gemm_status);
+    out_dtype torch.bfloat16: the result rounded to bf16 in the epilogue (amx_gemm_prepared_ex)."""
     if out is None:
-        out = torch.empty((M, N), dtype=torch.float32, device=a_prepared.device)
+        out = torch.empty((M, N), dtype=out_dtype, device=a_prepared.device)
     if workspace is None:
         workspace = _ws(lib().amx_gemm_prepared_workspace_bytes(M, N, K, group_size), a_prepared.device)
+    if out.dtype == torch.bfloat16:
+        _check(lib().amx_gemm_prepared_ex(a_prepared.data_ptr(), w_prepared.data_ptr(), M, N, K, group_size,
+                                          PREP_OUT_BF16 | (PREP_ONE_PLANE if sym else 0), out.data_ptr(), out.stride(0),
+                                          workspace.data_ptr(), workspace.numel(), _stream()), "amx_gemm_prepared_ex")
+        return out
+    _dev(out, torch.float32, "out")
     fn = lib().amx_gemm_prepared_sym if sym else lib().amx_gemm_prepared
     _check(fn(a_prepared.data_ptr(), w_prepared.data_ptr(), M, N, K, group_size, out.data_ptr(),
               out.stride(0), workspace.data_ptr(), workspace.numel(), _stream()), "amx_gemm_prepared")

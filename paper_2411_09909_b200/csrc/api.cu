@@ -171,28 +171,42 @@ extern "C" size_t amx_gemm_prepared_workspace_bytes(int64_t M, int64_t N, int64_
     return round_up(gemm_fp4_prepared_workspace_bytes(M, N, K));
 }
 
-extern "C" int amx_gemm_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
-                                 int group_size, float* C, int64_t ld_c, void* workspace, size_t workspace_bytes,
-                                 void* stream) {
+namespace {
+int gemm_prepared_checked(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K, int group_size,
+                          void* C, int64_t ld_c, void* workspace, size_t workspace_bytes, void* stream, bool one_plane,
+                          bool out_bf16) {
     if (M <= 0 || N <= 0 || !gemm_fp4_supported(M, N, K, group_size) || ld_c < N) return AMX_ERR_SHAPE;
     if (!a_prepared || !w_prepared || !C) return AMX_ERR_NULL;
     if (!workspace || workspace_bytes < 256) return AMX_ERR_WORKSPACE;
-    if (!aligned(a_prepared, kAlign) || !aligned(w_prepared, kAlign) || !aligned(workspace, kAlign) || !aligned(C, 4))
+    if (!aligned(a_prepared, kAlign) || !aligned(w_prepared, kAlign) || !aligned(workspace, kAlign) ||
+        !aligned(C, out_bf16 ? 2 : 4))
         return AMX_ERR_ALIGN;
-    return gemm_fp4_prepared(a_prepared, w_prepared, M, N, K, C, ld_c, workspace, static_cast<cudaStream_t>(stream),
-                             workspace_bytes);
+    return gemm_fp4_prepared_at({a_prepared, M, M, 0}, {w_prepared, N, N, 0}, M, N, K, static_cast<float*>(C), ld_c, workspace,
+                                static_cast<cudaStream_t>(stream), workspace_bytes, nullptr, nullptr, nullptr, one_plane,
+                                out_bf16);
+}
+}  // namespace
+
+extern "C" int amx_gemm_prepared(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
+                                 int group_size, float* C, int64_t ld_c, void* workspace, size_t workspace_bytes,
+                                 void* stream) {
+    return gemm_prepared_checked(a_prepared, w_prepared, M, N, K, group_size, C, ld_c, workspace, workspace_bytes, stream,
+                                 false, false);
 }
 
 extern "C" int amx_gemm_prepared_sym(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
                                      int group_size, float* C, int64_t ld_c, void* workspace, size_t workspace_bytes,
                                      void* stream) {
-    if (M <= 0 || N <= 0 || !gemm_fp4_supported(M, N, K, group_size) || ld_c < N) return AMX_ERR_SHAPE;
-    if (!a_prepared || !w_prepared || !C) return AMX_ERR_NULL;
-    if (!workspace || workspace_bytes < 256) return AMX_ERR_WORKSPACE;
-    if (!aligned(a_prepared, kAlign) || !aligned(w_prepared, kAlign) || !aligned(workspace, kAlign) || !aligned(C, 4))
-        return AMX_ERR_ALIGN;
-    return gemm_fp4_prepared_at({a_prepared, M, M, 0}, {w_prepared, N, N, 0}, M, N, K, C, ld_c, workspace,
-                                static_cast<cudaStream_t>(stream), workspace_bytes, nullptr, nullptr, nullptr, true);
+    return gemm_prepared_checked(a_prepared, w_prepared, M, N, K, group_size, C, ld_c, workspace, workspace_bytes, stream,
+                                 true, false);
+}
+
+extern "C" int amx_gemm_prepared_ex(const void* a_prepared, const void* w_prepared, int64_t M, int64_t N, int64_t K,
+                                    int group_size, uint32_t flags, void* C, int64_t ld_c, void* workspace,
+                                    size_t workspace_bytes, void* stream) {
+    if (flags & ~(AMX_PREP_ONE_PLANE | AMX_PREP_OUT_BF16)) return AMX_ERR_FLAGS;
+    return gemm_prepared_checked(a_prepared, w_prepared, M, N, K, group_size, C, ld_c, workspace, workspace_bytes, stream,
+                                 flags & AMX_PREP_ONE_PLANE, flags & AMX_PREP_OUT_BF16);
 }
 
 extern "C" int amx_quant_gemm(const void* A, int64_t ld_a, const uint8_t* w_codes, const uint8_t* w_scales,

@@ -77,7 +77,8 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
                          operand; every result is multiplied by their product (NVFP4 tensor scales) */,
                          bool one_plane = false /* the caller states that neither operand has a second sign plane:
                          full-width tiles run the deeper one-plane pipeline, which reports AMX_ERR_FLAGS in the status
-                         word when a tile has a second plane after all */);
+                         word when a tile has a second plane after all */,
+                         bool out_bf16 = false /* C points to bf16 [M, ld_c]: results rounded to nearest even */);
 // workspace that lets the kernel cut K into ranges for products with few output tiles (256 bytes otherwise)
 size_t gemm_fp4_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K);
 // C[m][n] = sum over `slices` partial products [slices][M][N], in slice order (defined with the bf16-decode kernel)

@@ -30,6 +30,8 @@
 // A preparation kernel per operand derives the planes, the UE4M3 scale-factor
 // blocks in the 128 x 4 interleaved layout the MMA reads, and the row offsets from the canonical
 // codes and scales.  Every device-side wait is bounded.
+#include <cuda_bf16.h>
+
 #include <cstdlib>
 
 #include "fp4_operand.cuh"
@@ -218,6 +220,7 @@ struct Params {
 
     float* C;
     int nk64, vec_store;
+    int out_bf16;                // C holds bf16 (each fp32 result rounded to nearest even) instead of fp32
     int band;                    // tile order: row blocks of A per band, see blk_m / blk_n
     int slices;                  // SLICED instantiation: K is cut into this many ranges, each (tile, range) a work item
     int64_t slice_stride;        //   whose partial product goes to C + range * slice_stride
@@ -238,6 +241,24 @@ __device__ __forceinline__ void store_row16(float* out, const float (&f)[16], bo
 #pragma unroll
         for (int j = 0; j < 16; ++j)
             if (j < n_left) out[j] = f[j];
+    }
+}
+
+// The same 16 results rounded to bf16 (nearest even): one 32-byte store.
+__device__ __forceinline__ void store_row16_bf16(__nv_bfloat16* out, const float (&f)[16], bool vec, int64_t n_left) {
+    if (vec && n_left >= 16) {
+        uint32_t w[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * j], f[2 * j + 1]);
+            w[j] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(out), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+                     "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+    } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+            if (j < n_left) out[j] = __float2bfloat16_rn(f[j]);
     }
 }
 
@@ -625,7 +646,13 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                             f[j + k] = __uint_as_float(v[buf][j + k]) * __uint_as_float((uint32_t)(sh + 127) << 23) * out_scale;
                         }
                     }
-                    if (m < p.M) store_row16(C_item + m * p.ld_c + n0 + col, f, p.vec_store != 0, p.N - (n0 + col));
+                    if (m < p.M) {
+                        if (p.out_bf16)
+                            store_row16_bf16(reinterpret_cast<__nv_bfloat16*>(C_item) + m * p.ld_c + n0 + col, f, p.vec_store != 0,
+                                             p.N - (n0 + col));
+                        else
+                            store_row16(C_item + m * p.ld_c + n0 + col, f, p.vec_store != 0, p.N - (n0 + col));
+                    }
                 }
             }
             ++t;
@@ -748,7 +775,7 @@ size_t gemm_fp4_prepared_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 // workspace_bytes >= gemm_fp4_prepared_workspace_bytes() enables the K ranges; 256 bytes always suffice.
 int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, int64_t N, int64_t K, float* C,
                          int64_t ld_c, void* workspace, cudaStream_t st, size_t workspace_bytes, const int* gate,
-                         const float* scale_a, const float* scale_w, bool one_plane) {
+                         const float* scale_a, const float* scale_w, bool one_plane, bool out_bf16) {
     Params p;
     OperandLayout oa, ow;
     int dev;
@@ -757,12 +784,16 @@ int gemm_fp4_prepared_at(const Fp4Operand& a, const Fp4Operand& w, int64_t M, in
     p.gate = gate;
     p.scale_a = scale_a;
     p.scale_w = scale_w;
+    if (out_bf16) {                                         // 32-byte stores hold 16 results
+        p.out_bf16 = 1;
+        p.vec_store = aligned(C, 32) && ld_c % 16 == 0;
+    }
     const uint8_t* pa = static_cast<const uint8_t*>(a.prepared);
     const uint8_t* pw = static_cast<const uint8_t*>(w.prepared);
     const int slices = gemm_fp4_slices(M, N, K);
     // at most 128 columns: tiles of 128 x 128, so that no half of a W tile is padding
     const bool half = N <= BN / 2 && !getenv("AMX_FP4_NO_HALF_TILE");
-    if (!gate && !scale_a && slices > 1 && workspace_bytes >= gemm_fp4_prepared_workspace_bytes(M, N, K)) {
+    if (!gate && !scale_a && !out_bf16 && slices > 1 && workspace_bytes >= gemm_fp4_prepared_workspace_bytes(M, N, K)) {
         float* part = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 256);
         p.C = part;
         p.ld_c = N;

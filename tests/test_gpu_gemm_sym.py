@@ -157,6 +157,33 @@ def test_gemm_nvfp4_sym(M, N, K):
     assert amx.gemm_status(work) == (ERR_FLAGS if two_planes else 0)
 
 
+@pytest.mark.parametrize("sym", [False, True])
+@pytest.mark.parametrize("M,N,K,pad", [(300, 520, 1056, 8), (129, 257, 64, 3), (1100, 6200, 288, 0), (1, 16, 32, 0)])
+def test_bf16_result(sym, M, N, K, pad):
+    """amx_gemm_prepared_ex with AMX_PREP_OUT_BF16: the fp32 result of the same kernel rounded to bf16 (ties to even), bit
+    for bit; vector and scalar store paths (leading dimension a multiple of 16 or not), padding untouched."""
+    fmt = amx.FMT_MXFP4 if sym else amx.FMT_AMXFP4
+    a_bits = inputs.random_groups(4900 + M, M, K, "normal")
+    w_bits = inputs.random_groups(4950 + N, N, K, "normal")
+    _, _, pa = amx.quantize_prepared(dev_bf16(a_bits), False, fmt=fmt)
+    _, _, pw = amx.quantize_prepared(dev_bf16(w_bits), True, fmt=fmt)
+    work = torch.full((256,), 0xFF, dtype=torch.uint8, device="cuda")
+    f32 = amx.gemm_prepared(pa, pw, M, N, K, workspace=work, sym=sym)
+    wide = torch.full((M, N + pad), -3.0, dtype=torch.bfloat16, device="cuda")
+    got = amx.gemm_prepared(pa, pw, M, N, K, out=wide[:, :N], workspace=work, sym=sym)
+    assert amx.gemm_status(work) == 0
+    assert got.dtype == torch.bfloat16 and torch.equal(got, f32.to(torch.bfloat16))      # torch rounds to nearest even
+    assert torch.all(wide[:, N:] == -3.0)
+    L = amx.lib()
+    st = torch.cuda.current_stream().cuda_stream
+    assert L.amx_gemm_prepared_ex(pa.data_ptr(), pw.data_ptr(), M, N, K, 32, 0x4, wide.data_ptr(), N + pad, work.data_ptr(), 256, st) == -5
+    assert L.amx_gemm_prepared_ex(pa.data_ptr(), pw.data_ptr(), M, N, K, 32, 0x2, wide.data_ptr() + 1, N + pad, work.data_ptr(), 256, st) == -3
+    # without flags: amx_gemm_prepared
+    c = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    assert L.amx_gemm_prepared_ex(pa.data_ptr(), pw.data_ptr(), M, N, K, 32, 0, c.data_ptr(), N, work.data_ptr(), 256, st) == 0
+    assert torch.equal(c, amx.gemm_prepared(pa, pw, M, N, K, workspace=work))
+
+
 def test_sym_argument_errors():
     L = amx.lib()
     buf = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
