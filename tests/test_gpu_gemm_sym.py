@@ -1,4 +1,5 @@
-"""GPU parity of the one-plane form of the FP4 tensor-core GEMM (amx_gemm_prepared_sym, amx_gemm_nvfp4_sym): two
+"""GPU parity of the one-plane form of the FP4 tensor-core GEMM (amx_gemm_prepared_sym, amx_gemm_nvfp4_sym) and of the
+options of amx_gemm_prepared_ex (one plane, bf16 result); products with several tiles per persistent CTA.  Two
 operands in a symmetric comparison format (Section 5's MXFP4 and FP8-scaled baselines, NVFP4) need one product per K
 step.  The result must equal the general kernel's bit for bit (same MMAs in the same order on the same scale factors)
 and the CPU oracle's within the GEMM tolerance; an operand with two planes must show as AMX_ERR_FLAGS in the status."""
