@@ -159,7 +159,7 @@ def test_gemm_nvfp4_sym(M, N, K):
 
 
 @pytest.mark.parametrize("sym", [False, True])
-@pytest.mark.parametrize("M,N,K,pad", [(300, 520, 1056, 8), (129, 257, 64, 3), (1100, 6200, 288, 0), (1, 16, 32, 0)])
+@pytest.mark.parametrize("M,N,K,pad", [(300, 520, 1056, 8), (129, 257, 64, 3), (1100, 6200, 288, 0), (1, 16, 32, 0), (128, 256, 4096, 0)])
 def test_bf16_result(sym, M, N, K, pad):
     """amx_gemm_prepared_ex with AMX_PREP_OUT_BF16: the fp32 result of the same kernel rounded to bf16 (ties to even), bit
     for bit; vector and scalar store paths (leading dimension a multiple of 16 or not), padding untouched."""
@@ -179,6 +179,9 @@ def test_bf16_result(sym, M, N, K, pad):
     st = torch.cuda.current_stream().cuda_stream
     assert L.amx_gemm_prepared_ex(pa.data_ptr(), pw.data_ptr(), M, N, K, 32, 0x4, wide.data_ptr(), N + pad, work.data_ptr(), 256, st) == -5
     assert L.amx_gemm_prepared_ex(pa.data_ptr(), pw.data_ptr(), M, N, K, 32, 0x2, wide.data_ptr() + 1, N + pad, work.data_ptr(), 256, st) == -3
+    # a workspace that would allow K ranges changes nothing: a bf16 result is never assembled from partial sums
+    big = torch.empty(L.amx_gemm_prepared_workspace_bytes(M, N, K, 32), dtype=torch.uint8, device="cuda")
+    assert torch.equal(amx.gemm_prepared(pa, pw, M, N, K, workspace=big, sym=sym, out_dtype=torch.bfloat16), got)
     # without flags: amx_gemm_prepared
     c = torch.empty((M, N), dtype=torch.float32, device="cuda")
     assert L.amx_gemm_prepared_ex(pa.data_ptr(), pw.data_ptr(), M, N, K, 32, 0, c.data_ptr(), N, work.data_ptr(), 256, st) == 0
