@@ -240,8 +240,8 @@ int amx_gemm_prepared_ex(const void* a_prepared, const void* w_prepared, int64_t
                          size_t workspace_bytes, void* stream);
 
 /*
- * amx_quant_gemm - the fully quantized linear layer of Section 5 ("quantize input operands for
- * all decoder-layer matrix multiplications"): quantizes the bf16 activation A[M, ld_a] and
+ * amx_quant_gemm - the fully quantized linear layer of Section 5 (the evaluation setting there casts both
+ * inputs of every matrix multiplication of a decoder layer): quantizes the bf16 activation A[M, ld_a] and
  * multiplies it with the weight, which comes in exactly one of two forms:
  *   w_codes / w_scales   an already quantized weight, canonical [N, K] (then W_bf16 must be NULL), or
  *   W_bf16, ld_w         a bf16 weight [N, ld_w] that this call casts as well (then w_codes and w_scales must
